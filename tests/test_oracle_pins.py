@@ -1,0 +1,481 @@
+"""Pins of the CPU oracle against things it did not compute itself: closed forms, library
+routines, brute force over all subsets, and invariants the paper states.  A dropped term, a wrong
+sign or index, or a transposed operand in the oracle fails at least one of these."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import growpage_oracle as O
+
+RNG = np.random.default_rng(1234)
+
+
+# ----------------------------------------------------------------------------- defaults
+def _golden():
+    path = os.path.join(os.path.dirname(__file__), "golden", "paper_defaults.txt")
+    vals = {}
+    for line in open(path):
+        line = line.split("#")[0].strip()
+        if line:
+            key, val = line.split("=")
+            vals[key.strip()] = float(val)
+    return vals
+
+
+def test_defaults_match_the_paper():
+    g = _golden()
+    c = O.OracleConfig(1, 8, 2, 64, n_pages=8, max_pages_per_req=4)
+    assert c.beta_s == g["beta_S"] and c.beta_l == g["beta_L"]
+    assert c.top_p == g["p"] and c.tau == g["tau"]
+    assert c.max_requests == g["M"]
+    # quota is the paper's fraction of a block: 64 of 256 tokens
+    assert c.k_loc / c.page_size == g["k_loc"] / g["b"]
+
+
+# ----------------------------------------------------------------------------- attention
+def test_attention_single_token_returns_its_value():
+    q = RNG.standard_normal((8, 64))
+    K = RNG.standard_normal((2, 1, 64))
+    V = RNG.standard_normal((2, 1, 64))
+    out = O.attention_decode(q, K, V)
+    for g in range(8):
+        np.testing.assert_allclose(out[g], V[g // 4, 0], rtol=0, atol=1e-15)
+
+
+def test_attention_equal_keys_average_the_values():
+    q = RNG.standard_normal((4, 32))
+    K = np.repeat(RNG.standard_normal((2, 1, 32)), 7, axis=1)
+    V = RNG.standard_normal((2, 7, 32))
+    out = O.attention_decode(q, K, V)
+    for g in range(4):
+        np.testing.assert_allclose(out[g], V[g // 2].mean(axis=0), atol=1e-14)
+
+
+def test_attention_two_tokens_is_a_logistic_mix():
+    d = 16
+    q = RNG.standard_normal((1, d))
+    K = RNG.standard_normal((1, 2, d))
+    V = RNG.standard_normal((1, 2, d))
+    gap = (K[0, 0] - K[0, 1]) @ q[0] / math.sqrt(d)
+    w0 = 1.0 / (1.0 + math.exp(-gap))
+    np.testing.assert_allclose(O.attention_decode(q, K, V)[0], w0 * V[0, 0] + (1 - w0) * V[0, 1], atol=1e-14)
+
+
+def test_attention_is_permutation_invariant_and_matches_torch_sdpa():
+    torch = pytest.importorskip("torch")
+    h_q, h_kv, n, d = 8, 2, 37, 64
+    q = RNG.standard_normal((h_q, d))
+    K = RNG.standard_normal((h_kv, n, d))
+    V = RNG.standard_normal((h_kv, n, d))
+    out = O.attention_decode(q, K, V)
+    perm = RNG.permutation(n)
+    np.testing.assert_allclose(O.attention_decode(q, K[:, perm], V[:, perm]), out, atol=1e-13)
+    G = h_q // h_kv
+    tq = torch.from_numpy(q)[None, :, None, :]
+    tk = torch.from_numpy(K).repeat_interleave(G, dim=0)[None]
+    tv = torch.from_numpy(V).repeat_interleave(G, dim=0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv)[0, :, 0].numpy()
+    np.testing.assert_allclose(out, ref, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- Eq. 6
+def test_ema_closed_form_and_special_cases():
+    T, d = 40, 8
+    qs = RNG.standard_normal((T, 1, d))
+    bs, bl = 0.9, 0.999
+    S = L = np.zeros((1, d))
+    started = False
+    for t in range(T):
+        S, L = O.ema_update(S, L, qs[t], started, bs, bl)
+        started = True
+        if t == 0:                      # first decode step of a slot: both states are the query
+            assert np.array_equal(S, qs[0]) and np.array_equal(L, qs[0])
+    for beta, got in ((bs, S), (bl, L)):
+        want = beta ** (T - 1) * qs[0]
+        for j in range(1, T):
+            want = want + (1 - beta) * beta ** (T - 1 - j) * qs[j]
+        np.testing.assert_allclose(got, want, rtol=1e-12)
+    # a constant query is a fixed point
+    c = RNG.standard_normal((1, d))
+    S = L = np.zeros((1, d)); started = False
+    for _ in range(10):
+        S, L = O.ema_update(S, L, c, started, bs, bl); started = True
+    np.testing.assert_allclose(S, c, rtol=1e-14); np.testing.assert_allclose(L, c, rtol=1e-14)
+    # beta_S = 0: the short summary is the current query (the paper's beta ablation)
+    S, L = O.ema_update(RNG.standard_normal((1, d)), RNG.standard_normal((1, d)), c, True, 0.0, bl)
+    assert np.array_equal(S, c)
+
+
+def test_stale_slot_contents_do_not_leak_into_a_new_request():
+    stale = 1e6 * np.ones((2, 4))
+    q = RNG.standard_normal((2, 4))
+    S, L = O.ema_update(stale, stale, q, False, 0.9, 0.999)
+    assert np.array_equal(S, q) and np.array_equal(L, q)
+
+
+# ----------------------------------------------------------------------------- Eq. 12, RoPE
+def test_rms_calibration_identities():
+    q = RNG.standard_normal((6, 32))
+    qb = RNG.standard_normal((6, 32)) * RNG.uniform(0.01, 30, (6, 1))
+    qt = O.rms_calibrate(qb, q)
+    np.testing.assert_allclose(O.rms(qt), O.rms(q), rtol=1e-13)            # scales are matched
+    cos = np.sum(qt * qb, -1) / np.linalg.norm(qt, axis=-1) / np.linalg.norm(qb, axis=-1)
+    np.testing.assert_allclose(cos, 1.0, rtol=1e-13)                       # direction is kept
+    np.testing.assert_allclose(O.rms_calibrate(3.7 * q, q), q, rtol=1e-13)  # collinear: the query itself
+    z = np.zeros((1, 8))
+    assert np.array_equal(O.rms_calibrate(z, RNG.standard_normal((1, 8))), z)
+    x = np.array([[3.0, 4.0]])
+    assert O.rms(x)[0] == pytest.approx(math.sqrt(12.5))
+
+
+def test_rope_is_a_position_dependent_rotation():
+    d, theta = 16, 10000.0
+    x = RNG.standard_normal((3, d)); y = RNG.standard_normal((3, d))
+    assert np.array_equal(O.rope(x, 5, 0.0), x)                            # switched off
+    np.testing.assert_allclose(O.rope(x, 0, theta), x, atol=0)             # position 0
+    np.testing.assert_allclose(np.linalg.norm(O.rope(x, 123, theta), axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-13)
+    # scores depend on the position difference only
+    a = np.sum(O.rope(x, 40, theta) * O.rope(y, 33, theta), -1)
+    b_ = np.sum(O.rope(x, 107, theta) * O.rope(y, 100, theta), -1)
+    np.testing.assert_allclose(a, b_, rtol=1e-10)
+    # d = 2: a plain plane rotation by `pos` radians (frequency theta^0 = 1), counter-clockwise
+    v = np.array([[1.0, 0.0]])
+    np.testing.assert_allclose(O.rope(v, 1, theta), [[math.cos(1.0), math.sin(1.0)]], atol=1e-15)
+    # pairing is (i, i + d/2): rotating a vector that lives in one pair leaves the others zero
+    e = np.zeros((1, d)); e[0, 2] = 1.0
+    r = O.rope(e, 7, theta)
+    assert set(np.nonzero(np.abs(r[0]) > 1e-12)[0]) <= {2, 2 + d // 2}
+    ang = 7 * theta ** (-2.0 * 2 / d)
+    np.testing.assert_allclose([r[0, 2], r[0, 2 + d // 2]], [math.cos(ang), math.sin(ang)], atol=1e-14)
+
+
+def test_rope_matches_transformers_rotate_half():
+    torch = pytest.importorskip("torch")
+    mod = pytest.importorskip("transformers.models.llama.modeling_llama")
+    d, theta, pos = 32, 1e6, 77
+    x = RNG.standard_normal((4, d))
+    inv = 1.0 / (theta ** (torch.arange(0, d, 2, dtype=torch.float64) / d))
+    ang = pos * inv
+    emb = torch.cat([ang, ang])
+    cos, sin = emb.cos()[None, None], emb.sin()[None, None]
+    tx = torch.from_numpy(x)[None]
+    ref, _ = mod.apply_rotary_pos_emb(tx, tx, cos, sin, unsqueeze_dim=1)
+    np.testing.assert_allclose(O.rope(x, pos, theta), ref.reshape(4, d).numpy(), atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- Eq. 2, Eq. 5, Theorem 1
+def test_p_coverage_closed_forms():
+    n = 50
+    assert O.p_coverage_demand(np.full(n, 1.0 / n), 0.5) == 25
+    assert O.p_coverage_demand(np.full(n, 1.0 / n), 0.503) == 26
+    one = np.zeros(n); one[17] = 1.0
+    assert O.p_coverage_demand(one, 0.99) == 1
+    # geometric weights: the top-k mass is 1 - r^k up to the normaliser
+    r = 0.8
+    a = (1 - r) * r ** np.arange(200)
+    a = RNG.permutation(a / a.sum())
+    k = O.p_coverage_demand(a, 0.99)
+    assert k == math.ceil(math.log(1 - 0.99 * (1 - r ** 200)) / math.log(r))
+    # order of the input does not matter; never reached -> everything
+    assert O.p_coverage_demand(np.array([0.2, 0.5, 0.3]), 0.75) == 2
+    assert O.p_coverage_demand(np.array([0.25, 0.25]), 0.99) == 2
+
+
+def test_worst_case_error_is_attained_and_theorem_1_by_brute_force():
+    for trial in range(20):
+        n = int(RNG.integers(4, 12))
+        a = RNG.dirichlet(np.full(n, RNG.uniform(0.2, 2.0)))
+        v_max = float(RNG.uniform(0.5, 3.0))
+        # Eq. 5: the bound is met by opposite directions of norm Vmax on and off S
+        S = sorted(RNG.choice(n, size=int(RNG.integers(1, n)), replace=False).tolist())
+        u = RNG.standard_normal(5); u /= np.linalg.norm(u)
+        v = np.array([(-v_max if i in S else v_max) * u for i in range(n)])
+        o = a @ v
+        o_hat, m = O.subset_output(a, v, S)
+        assert np.linalg.norm(o - o_hat) == pytest.approx(2 * v_max * (1 - m), rel=1e-10)
+        assert O.worst_case_error(a, S, v_max) == pytest.approx(2 * v_max * (1 - m), rel=1e-12)
+        # random values never exceed it
+        w = RNG.standard_normal((n, 5)); w *= v_max / np.linalg.norm(w, axis=1, keepdims=True)
+        o_hat2, _ = O.subset_output(a, w, S)
+        assert np.linalg.norm(a @ w - o_hat2) <= 2 * v_max * (1 - m) + 1e-12
+        # Theorem 1: min |S| with worst-case error <= delta equals D_{1 - delta / (2 Vmax)}
+        delta = float(RNG.uniform(0.05, 1.9)) * v_max
+        best = None
+        for size in range(1, n + 1):
+            if any(O.worst_case_error(a, comb, v_max) <= delta for comb in itertools.combinations(range(n), size)):
+                best = size
+                break
+        assert best == O.p_coverage_demand(a, 1 - delta / (2 * v_max))
+
+
+def test_summary_attention_is_the_group_mean_of_softmaxes():
+    sp = pytest.importorskip("scipy.special")
+    G, n, d = 4, 33, 16
+    qt = RNG.standard_normal((G, d)); Kc = RNG.standard_normal((n, d))
+    a = O.summary_attention(qt, Kc)
+    assert a.sum() == pytest.approx(1.0, abs=1e-14)
+    ref = np.mean([sp.softmax(Kc @ qt[g] / math.sqrt(d)) for g in range(G)], axis=0)
+    np.testing.assert_allclose(a, ref, rtol=1e-12)
+    # a calibrated summary collinear with the query reproduces the query's own attention over C
+    q = RNG.standard_normal((1, d))
+    np.testing.assert_allclose(O.summary_attention(O.rms_calibrate(0.2 * q, q), Kc),
+                               sp.softmax(Kc @ q[0] / math.sqrt(d)), rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------- Eq. 9, Eq. 10
+def test_token_score_is_the_larger_view():
+    a = RNG.random(9); c = RNG.random(9)
+    s = O.token_scores(a, c)
+    assert np.all(s >= a) and np.all(s >= c) and np.all((s == a) | (s == c))
+
+
+def _best_subset(s, n_blocks, b, K_t, k_prime):
+    best, best_val = None, -1.0
+    for comb in itertools.combinations(range(n_blocks * b), K_t):
+        cnt = np.bincount(np.asarray(comb) // b, minlength=n_blocks)
+        if np.all(cnt >= k_prime):
+            val = s[list(comb)].sum()
+            if val > best_val:
+                best, best_val = comb, val
+    return np.asarray(best)
+
+
+@pytest.mark.parametrize("n_blocks,b,k_loc", [(3, 4, 1), (3, 4, 2), (4, 3, 1), (2, 6, 2), (3, 4, 0)])
+def test_selection_is_the_constrained_optimum(n_blocks, b, k_loc):
+    for _ in range(6):
+        s = RNG.random(n_blocks * b) ** 3
+        K_t = n_blocks * b - b
+        keep, _ = O.select_retained(s, n_blocks, b, K_t, k_loc)
+        assert keep.size == K_t and np.all(np.diff(keep) > 0)
+        k_prime = min(k_loc, K_t // n_blocks)
+        np.testing.assert_array_equal(keep, _best_subset(s, n_blocks, b, K_t, k_prime))
+
+
+def test_selection_special_cases_and_ties():
+    b, n_blocks = 16, 5
+    s = RNG.random(n_blocks * b)
+    K_t = (n_blocks - 1) * b
+    keep, _ = O.select_retained(s, n_blocks, b, K_t, 0)          # no quota: plain top-K_t
+    np.testing.assert_array_equal(keep, np.sort(np.argpartition(-s, K_t - 1)[:K_t]))
+    # quota large enough that the local picks fill the budget: floor(K_t / n_blocks) from each block
+    keep, _ = O.select_retained(s[:16], 4, 4, 12, 3)
+    assert np.all(np.bincount(keep // 4, minlength=4) == 3)
+    # exact duplicates: the older (lower) slot wins, in the local and in the global cut
+    s = np.array([0.5, 0.5, 0.5, 0.5, 0.1, 0.1, 0.1, 0.1])
+    keep, margin = O.select_retained(s, 2, 4, 4, 1)
+    np.testing.assert_array_equal(keep, [0, 1, 2, 4])
+    assert margin == 0.0
+    # block quota overrides global rank: the worst block still keeps its best k'
+    s = np.concatenate([np.full(4, 0.9), np.full(4, 0.8), np.array([0.01, 0.04, 0.02, 0.03])])
+    keep, _ = O.select_retained(s, 3, 4, 8, 1)
+    assert 9 in keep and np.bincount(keep // 4, minlength=3).tolist() == [4, 3, 1]
+
+
+# ----------------------------------------------------------------------------- state machine
+def _cfg(**kw):
+    base = dict(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=8, n_pages=12, max_pages_per_req=6, page_size=4,
+                recent_window=4, k_loc=1, max_requests=4)
+    base.update(kw)
+    return O.OracleConfig(**base)
+
+
+def _rand_step(c, B):
+    return (RNG.standard_normal((c.n_layers, B, c.n_q_heads, c.head_dim)),
+            RNG.standard_normal((c.n_layers, B, c.n_kv_heads, c.head_dim)),
+            RNG.standard_normal((c.n_layers, B, c.n_kv_heads, c.head_dim)))
+
+
+def _check_invariants(pool: O.OraclePool):
+    c = pool.cfg
+    b = c.page_size
+    refs = np.zeros(c.n_pages, dtype=np.int64)
+    for rid, r in pool.requests.items():
+        assert len(r.table) == r.P and r.n <= r.P * b
+        for page in r.table:
+            refs[page] += 1
+        for l in range(c.n_layers):
+            for h in range(c.n_kv_heads):
+                tok = r.tok[l, h, :r.n]
+                assert np.all(np.diff(tok) > 0)                       # slot order is token order
+                assert np.all(tok[-min(r.n, 1):] == r.pos - 1) or r.n == 0 or not r.started
+                assert np.all(r.tok[l, h, r.n:r.P * b] == -1) or not r.started
+    assert np.array_equal(refs, pool.refcount)                        # references are conserved
+    assert len(set(pool.free)) == len(pool.free)
+    assert len(pool.free) + int((pool.refcount > 0).sum()) == c.n_pages
+    assert all(pool.refcount[p] == 0 for p in pool.free)
+
+
+def test_capacity_moves_only_at_boundaries_and_only_up_by_one():
+    c = _cfg()
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((c.n_layers, 6, c.n_kv_heads, c.head_dim))
+    st, rid = pool.request_add(-1, 0, kt, kt.copy(), 6, 2)
+    assert st == O.OK and rid == 0
+    P, n, pos, table = pool.request_state(rid)
+    assert (P, n, pos) == (2, 6, 6)                                   # floor(6/4)+1 = 2 pages
+    seen = set()
+    for step in range(60):
+        q, k, v = _rand_step(c, 1)
+        P0, n0, _, _ = pool.request_state(rid)
+        rec = pool.decode_step([rid], q, k, v)
+        P1, n1, pos1, _ = pool.request_state(rid)
+        act = int(rec.actions[0]); seen.add(act)
+        assert pos1 == 7 + step
+        if n0 + 1 < P0 * c.page_size:
+            assert act == O.ACT_NONE and P1 == P0 and n1 == n0 + 1
+        elif act == O.ACT_GROW:
+            assert P1 == P0 + 1 and n1 == n0 + 1
+        else:
+            assert act in (O.ACT_COMPRESS, O.ACT_COMPRESS_FALLBACK)
+            assert P1 == P0 and n1 == (P0 - 1) * c.page_size          # exactly one page of slots freed
+            info = rec.boundary[rid]
+            for l in range(c.n_layers):
+                for h in range(c.n_kv_heads):
+                    tok = pool.retained(rid, l, h)
+                    assert np.array_equal(tok[-c.page_size:], np.arange(pos1 - c.page_size, pos1))  # newest survive
+                    assert info.keep[(l, h)].size == (P0 - 2) * c.page_size
+        assert P1 <= c.max_pages_per_req
+        _check_invariants(pool)
+    assert O.ACT_COMPRESS in seen or O.ACT_COMPRESS_FALLBACK in seen
+
+
+def test_first_boundary_with_equal_summaries_compresses():
+    # one free slot at admission: the first decode step is a boundary with S == L, so Delta = 0
+    c = _cfg()
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((c.n_layers, 7, c.n_kv_heads, c.head_dim))
+    _, rid = pool.request_add(-1, 0, kt, kt.copy(), 7, 0)
+    q, k, v = _rand_step(c, 1)
+    rec = pool.decode_step([rid], q, k, v)
+    info = rec.boundary[rid]
+    assert info.delta == 0.0 and np.array_equal(info.K_s, info.K_l)
+    assert int(rec.actions[0]) == O.ACT_COMPRESS
+    # and the attention output of that step saw all 8 tokens (append precedes attention)
+    r = pool.requests[rid]
+    assert r.n == 4
+
+
+def test_grow_fallback_and_stall_under_a_small_pool():
+    c = _cfg(n_pages=3, max_pages_per_req=3)
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((c.n_layers, 3, c.n_kv_heads, c.head_dim))
+    _, a = pool.request_add(-1, 0, kt, kt.copy(), 3, 0)              # P = 1
+    q, k, v = _rand_step(c, 1)
+    rec = pool.decode_step([a], q, k, v)                              # n = 4 = P b, C empty -> grow
+    assert int(rec.actions[0]) == O.ACT_GROW and pool.request_state(a)[0] == 2
+    st, b_id = pool.request_add(-1, 0, kt, kt.copy(), 3, 0)
+    assert st == O.OK and pool.n_free() == 0
+    rec = pool.decode_step([b_id], *_rand_step(c, 1))                 # P = 1, no page: nothing to evict
+    assert int(rec.actions[0]) == O.ACT_STALLED
+    rec = pool.decode_step([b_id], *_rand_step(c, 1))                 # stays stalled, untouched
+    assert int(rec.actions[0]) == O.ACT_STALLED and pool.request_state(b_id)[1] == 4
+    assert pool.request_add(-1, 0, kt, kt.copy(), 3, 0)[0] == O.ERR_NO_PAGES
+    # force "wants to grow" on a full pool: falls back to compression
+    for _ in range(3):
+        pool.decode_step([a], *_rand_step(c, 1))
+    rec = pool.step_compute([a], *_rand_step(c, 1))
+    pool.step_apply(rec, {a: {"want_grow": True}})
+    assert int(rec.actions[0]) == O.ACT_COMPRESS_FALLBACK
+    assert pool.release(b_id) == O.OK and pool.n_free() == 1
+    _check_invariants(pool)
+
+
+def test_prefix_sharing_copy_on_write_and_release():
+    c = _cfg(n_pages=16, max_pages_per_req=5)
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((c.n_layers, 8, c.n_kv_heads, c.head_dim))   # two full pages
+    _, a = pool.request_add(-1, 0, kt, kt.copy(), 8, 0)                   # P = 3
+    _, b_id = pool.request_add(a, 2, None, None, 0, 0)
+    _, c_id = pool.request_add(a, 2, None, None, 0, 0)
+    shared = pool.request_state(a)[3][:2]
+    assert pool.request_state(b_id)[3][:2] == shared and all(pool.refcount[p] == 3 for p in shared)
+    assert pool.request_add(a, 3, None, None, 0, 0)[0] == O.ERR_INVALID   # page 2 is not a full prompt page
+    snapshot = pool.requests[b_id].K[:, :, :8].copy()
+    free0 = pool.n_free()
+    # run a and b to their first boundary together, forcing compression for both
+    for step in range(4):
+        rec = pool.step_compute([a, b_id], *_rand_step(c, 2))
+        pool.step_apply(rec, {a: {"want_grow": False}, b_id: {"want_grow": False}})
+        _check_invariants(pool)
+    assert [int(x) for x in rec.actions] == [O.ACT_COMPRESS, O.ACT_COMPRESS]
+    assert rec.boundary[a].cow_pages == 2 and rec.boundary[b_id].cow_pages == 2
+    # both replaced both shared pages; the third sharer still holds them, untouched
+    assert all(pool.refcount[p] == 1 for p in shared)
+    assert pool.request_state(c_id)[3][:2] == shared
+    assert not set(pool.request_state(a)[3]) & set(pool.request_state(b_id)[3])
+    assert pool.n_free() == free0 - 4
+    np.testing.assert_array_equal(pool.requests[c_id].K[:, :, :8], snapshot)
+    assert pool.request_add(a, 1, None, None, 0, 0)[0] == O.ERR_INVALID   # a's prefix is no longer pristine
+    # last sharer compresses alone: it is the only owner now and keeps its pages
+    for step in range(4):
+        rec = pool.step_compute([c_id], *_rand_step(c, 1))
+        pool.step_apply(rec, {c_id: {"want_grow": False}})
+    assert rec.boundary[c_id].cow_pages == 0 and pool.request_state(c_id)[3][:2] == shared
+    for rid in (a, b_id, c_id):
+        assert pool.release(rid) == O.OK
+    assert pool.n_free() == c.n_pages and not pool.refcount.any()
+
+
+def test_simultaneous_last_sharers_both_copy_and_the_page_is_freed_afterwards():
+    c = _cfg(n_pages=10, max_pages_per_req=4)
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((c.n_layers, 4, c.n_kv_heads, c.head_dim))
+    _, a = pool.request_add(-1, 0, kt, kt.copy(), 4, 3)                   # P = 3 (budget above the prompt)
+    _, b_id = pool.request_add(a, 1, None, None, 0, 3)
+    page = pool.request_state(a)[3][0]
+    for step in range(8):
+        rec = pool.step_compute([a, b_id], *_rand_step(c, 2))
+        pool.step_apply(rec, {a: {"want_grow": False}, b_id: {"want_grow": False}})
+    assert pool.refcount[page] == 0 and page in pool.free
+    _check_invariants(pool)
+
+
+def test_stall_when_copy_on_write_targets_are_missing_leaves_the_request_unchanged():
+    c = _cfg(n_pages=5, max_pages_per_req=3)
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((c.n_layers, 8, c.n_kv_heads, c.head_dim))
+    _, a = pool.request_add(-1, 0, kt, kt.copy(), 8, 0)                   # 3 pages
+    _, b_id = pool.request_add(a, 2, None, None, 0, 0)                    # 1 private page; pool: 1 free
+    for step in range(4):
+        before = pool.request_state(b_id)
+        rec = pool.step_compute([b_id], *_rand_step(c, 1))
+        pool.step_apply(rec, {b_id: {"want_grow": False}})
+    assert int(rec.actions[0]) == O.ACT_STALLED                       # needs 2 targets, 1 free
+    P, n, pos, table = pool.request_state(b_id)
+    assert n == P * c.page_size and table == before[3]
+    _check_invariants(pool)
+
+
+def test_invalid_ids_and_duplicates_are_reported_per_request():
+    c = _cfg()
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((c.n_layers, 2, c.n_kv_heads, c.head_dim))
+    _, a = pool.request_add(-1, 0, kt, kt.copy(), 2, 0)
+    rec = pool.decode_step([a, 3, a], *_rand_step(c, 3))
+    assert [int(x) for x in rec.actions] == [O.ACT_NONE, O.ACT_INVALID, O.ACT_INVALID]
+    assert pool.request_state(a)[1] == 3
+    assert pool.release(2) == O.ERR_INVALID
+    for i in range(3):
+        assert pool.request_add(-1, 0, kt, kt.copy(), 2, 0)[0] == O.OK
+    assert pool.request_add(-1, 0, kt, kt.copy(), 2, 0)[0] == O.ERR_NO_SLOT
+
+
+def test_retained_output_error_respects_the_worst_case_bound():
+    # after a compression with retained set S, the view's own output error is bounded by Eq. 5
+    c = _cfg(n_layers=1, n_q_heads=2, n_kv_heads=2, n_pages=8, max_pages_per_req=4)
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((1, 11, 2, 8))
+    _, a = pool.request_add(-1, 0, kt, RNG.standard_normal((1, 11, 2, 8)), 11, 0)
+    r = pool.requests[a]
+    rec = pool.step_compute([a], *_rand_step(c, 1))
+    V_c = r.V[0, 0, :8].copy()
+    pool.step_apply(rec, {a: {"want_grow": False}})
+    info = rec.boundary[a]
+    S = info.keep[(0, 0)]
+    a_s = info.a_s[0, 0]
+    o_hat, m = O.subset_output(a_s, V_c, S)
+    v_max = np.linalg.norm(V_c, axis=1).max()
+    assert np.linalg.norm(a_s @ V_c - o_hat) <= 2 * v_max * (1 - m) + 1e-12
