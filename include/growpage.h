@@ -1,0 +1,172 @@
+/*
+ * growpage.h: C ABI of the GrowPage paged-decode library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-step decode path of GrowPage (on-demand KV budgeting): every
+ * request owns a page table over a shared pool of fixed-size KV pages; a decode step appends the
+ * new token, runs GQA paged attention fused with the update of the two exponentially smoothed
+ * query summaries (Sec. 3.2, Eq. 6), and, for requests whose allocation is now full, estimates
+ * the short- and long-horizon attention working sets (Eq. 7, Eq. 8) and either acquires one
+ * more page or evicts one page worth of tokens and compacts in place (Sec. 3.3, Eq. 9, Eq. 10).
+ *
+ * Conventions
+ *   - All functions return an int status (GP_OK or a negative GP_ERR_*), never throw or abort.
+ *   - "device pointer" = memory of the pool's CUDA device; "host pointer" = ordinary host memory.
+ *   - The caller owns every buffer it passes.  The pool owns only the partition of the single
+ *     device blob handed to gp_pool_create; the library never allocates device memory.
+ *   - `stream` arguments are CUDA stream handles (cudaStream_t) passed as void*; NULL is the
+ *     default stream.  Work is enqueued in stream order.
+ *   - bf16 tensors are raw 16-bit patterns, row-major with the last index fastest.
+ */
+#ifndef GROWPAGE_H_
+#define GROWPAGE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define GP_OK             0
+#define GP_ERR_INVALID   (-1)  /* bad argument, unknown or dead request id                        */
+#define GP_ERR_NO_SLOT   (-2)  /* all max_requests summary slots are bound                        */
+#define GP_ERR_NO_PAGES  (-3)  /* the free list or the per-request cap cannot supply the pages    */
+#define GP_ERR_CUDA      (-4)  /* a CUDA call failed or a kernel reported an internal error       */
+#define GP_ERR_STATE     (-5)  /* call not possible in the pool's current state                   */
+
+/* per-request action written by gp_decode_step (Sec. 3.3, Sec. 4.2) */
+#define GP_ACT_NONE               0   /* no capacity boundary this step                           */
+#define GP_ACT_GROW               1   /* Delta_t > tau: one page appended to the block table      */
+#define GP_ACT_COMPRESS           2   /* Compress & Hold: one page worth of slots freed in place  */
+#define GP_ACT_COMPRESS_FALLBACK  3   /* wanted to grow, cap or free list said no, compressed     */
+#define GP_ACT_STALLED          (-1)  /* full and neither a page nor copy-on-write targets could
+                                         be had: page state untouched, the caller should release
+                                         (preempt) the request; it is skipped while it stays full */
+#define GP_ACT_SCRATCH          (-2)  /* boundary skipped: scoring scratch exhausted
+                                         (max_batch_tokens too small); handled like a stall       */
+#define GP_ACT_INVALID          (-3)  /* id out of range, not live, or repeated in the batch      */
+
+typedef struct gp_pool gp_pool; /* opaque */
+
+typedef struct gp_config {
+  int32_t n_layers;          /* L                                                                  */
+  int32_t n_q_heads;         /* H_q, a multiple of n_kv_heads; group size G = H_q/H_kv <= 8        */
+  int32_t n_kv_heads;        /* H_kv                                                               */
+  int32_t head_dim;          /* d_h: 64 or 128                                                     */
+  int32_t page_size;         /* b: tokens per page, 16                                             */
+  int32_t max_requests;      /* M: summary slots = highest request id + 1 (App. D.1, default 512)  */
+  int32_t max_pages_per_req; /* per-request page cap and page-table stride, >= 1                   */
+  int32_t recent_window;     /* |R_t| protected tokens; must equal page_size                       */
+  int32_t k_loc;             /* block-local retention quota of Eq. 10 (default page_size / 4)      */
+  int32_t host_staging;      /* 1: reserve staging so that gp_decode_step_host can be used         */
+  int64_t n_pages;           /* physical pages; one page id covers all layers and KV heads         */
+  int64_t max_batch_tokens;  /* bound on the summed sequence lengths of one decode batch, used to
+                                size scratch; 0 = n_pages * page_size                              */
+  double  beta_s, beta_l;    /* Eq. 6, defaults 0.9 and 0.999                                      */
+  double  top_p;             /* Eq. 7, default 0.99                                                */
+  double  tau;               /* decision threshold, default 0                                      */
+  double  rope_theta;        /* RoPE base (rotate-half pairing); 0 = no rotation                   */
+} gp_config;
+
+/* Fills *cfg with the paper's defaults (Sec. 3.2, Sec. 5.1, App. B.2, App. D.1); the geometry
+ * fields (layers, heads, pages) are set to zero and must be filled by the caller. */
+int gp_config_default(gp_config* cfg);
+
+/* Bytes of device memory a pool of this configuration needs; 0 if the configuration is invalid. */
+size_t gp_pool_bytes(const gp_config* cfg);
+
+/* Creates a pool inside `dev_blob` (device pointer, 256-byte aligned, at least gp_pool_bytes(cfg)
+ * bytes, on CUDA device `device`).  The blob is cleared; every page starts on the free list
+ * (Sec. 4.2 "global free-page pool").  Synchronous.  The blob must outlive the pool. */
+int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int device, gp_pool** out);
+
+/* Frees the host-side handle.  Synchronises the device first.  The blob is left to its owner. */
+int gp_pool_destroy(gp_pool* pool);
+
+/* Admits a request (App. D.1 "query slots are bound to requests when they enter the running
+ * queue"; App. D.2 prefix sharing).  Its first `n_shared_pages` pages are shared by reference
+ * count with live request `share_from` (-1 for none), which must still hold them as untouched
+ * full prompt pages.  The rest of the prompt, `n_tail` tokens, is copied from k_tail / v_tail:
+ * device pointers, bf16 [L][n_tail][H_kv][d], keys already in cache form (post-RoPE).
+ * The request starts with max(initial_pages, floor(n_prompt / b) + 1) pages.
+ * On success *out_req receives the request id (the lowest free slot).  The summaries of the slot
+ * are not cleared: the first decode step overwrites them.  Synchronises `stream`.
+ * Errors: GP_ERR_INVALID, GP_ERR_NO_SLOT, GP_ERR_NO_PAGES (nothing is changed in these cases). */
+int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
+                   const void* k_tail, const void* v_tail, int32_t n_tail,
+                   int32_t initial_pages, void* stream, int32_t* out_req);
+
+/* One decode step for `n_req` requests (Sec. 3.2 - 3.3, App. D.1, App. D.2).
+ *   dev_req_ids  device int32 [n_req]: request ids, each at most once
+ *   q            device bf16 [L][n_req][H_q][d]: normalised queries before RoPE
+ *   k, v         device bf16 [L][n_req][H_kv][d]: the new token's key (cache form) and value
+ *   out          device fp32 [L][n_req][H_q][d]: attention output over all retained tokens,
+ *                the new one included; rows of requests whose action is GP_ACT_INVALID, or that
+ *                were already full on entry, are not written
+ *   dev_actions  device int32 [n_req]: GP_ACT_* per request
+ * Asynchronous on `stream`; nothing is read back to the host.  Steps of one pool must be
+ * issued on one stream (or otherwise serialised): they share scratch inside the blob. */
+int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
+                   const void* q, const void* k, const void* v,
+                   void* out, int32_t* dev_actions, void* stream);
+
+/* As gp_decode_step with HOST pointers (pinned memory recommended): copies the inputs to staging
+ * inside the blob, runs the step, copies `out` and `actions` back and synchronises `stream`.
+ * Needs host_staging = 1 at creation, else GP_ERR_STATE. */
+int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req,
+                        const void* q, const void* k, const void* v,
+                        void* out, int32_t* actions, void* stream);
+
+/* Ends a request: every page of its table loses one reference and returns to the free list at
+ * zero; the summary slot is recycled without clearing (App. D.1).  Asynchronous on `stream`. */
+int gp_release(gp_pool* pool, int32_t req, void* stream);
+
+/* Text for a status code. */
+const char* gp_strerror(int status);
+
+/* ---- introspection (host outputs; each call synchronises the device) ------------------------ */
+
+/* Pages P, occupied slots n, absolute position pos and the page table (host int32, room for
+ * max_pages_per_req entries; may be NULL) of a live request. */
+int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t* pos, int32_t* page_table);
+
+/* Original token index of every occupied slot of one (layer, KV head) stream, in slot order:
+ * host int32 [n].  This is the retained-index set of Sec. 3.3. */
+int gp_debug_retained(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_head, int32_t* token_ids);
+
+/* K and V rows of the occupied slots of one (layer, KV head) stream in slot order:
+ * host bf16 [n][d] each (either may be NULL). */
+int gp_debug_kv(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_head, void* k_rows, void* v_rows);
+
+/* The two summaries of a request: host double [L][2][H_q][d], short then long (Eq. 6, Eq. 11). */
+int gp_debug_summaries(gp_pool* pool, int32_t req, double* out);
+
+/* Working-set sizes of the request's most recent boundary: host int32 [L][H_kv] each, and
+ * Delta_t (Eq. 7, Eq. 8). */
+int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, double* delta);
+
+/* Free pages, per-page reference counts (host int32 [n_pages], may be NULL) and event counters:
+ * [0] grow [1] compress [2] fallback-compress [3] stalled [4] copy-on-write pages
+ * [5] decode steps [6] tokens decoded [7] internal error bits (0 when healthy). */
+int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[8]);
+
+/* ---- measurement ----------------------------------------------------------------------------- */
+
+#define GP_N_KERNELS 5   /* plan, attention, boundary scoring, decision, selection + compaction */
+
+/* With profiling on, every kernel of gp_decode_step is bracketed by CUDA events on the step's
+ * stream (this serialises nothing but adds event records).  Off by default. */
+int gp_set_profiling(gp_pool* pool, int32_t enable);
+
+/* Synchronises, then returns the accumulated device time in milliseconds and the launch count of
+ * each kernel since profiling was switched on (host arrays of GP_N_KERNELS), and resets them. */
+int gp_get_kernel_times(gp_pool* pool, float* ms, int64_t* launches);
+
+/* Kernels launched by this pool since creation (all calls). */
+int64_t gp_launch_count(gp_pool* pool);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GROWPAGE_H_ */

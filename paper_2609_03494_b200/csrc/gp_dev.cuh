@@ -1,0 +1,163 @@
+// Device-side view of a GrowPage pool and the small PTX wrappers the kernels share.
+//
+// HBM layout (all regions carved from the caller's blob, 256-byte aligned):
+//   kv        bf16  [L][n_pages][H_kv][2 (K|V)][b][d]   one (layer, page, KV head) tile is a
+//                   contiguous 2*b*d*2 bytes, so a single bulk copy stages K and V of a page.
+//                   Inside a row of d elements the 16-byte chunks are XOR-swizzled with the
+//                   slot index: logical chunk c of slot s lives at chunk c ^ (s & 7).  A tile
+//                   copied verbatim to shared memory is then bank-conflict free for ldmatrix.
+//   tok       int32 [L][n_pages][H_kv][b]               original token index of every slot
+//   summaries fp64  [L][M][2][H_q][d]                   Eq. 11 layout, short then long
+//   page_table / shadow int32 [M][cap]                  shadow holds copy-on-write targets
+//   scores    fp64  [2][L*H_kv][max_batch_tokens]       a^S, a^L of the requests at a boundary
+//   partials  fp32  split-KV partial outputs
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#define GP_PAGE 16             // tokens per page (b)
+#define GP_ATTN_WARPS 4
+#define GP_ATTN_STAGES 3
+#define GP_SPIN_LIMIT (1u << 24)
+
+// plan header slots (int32)
+enum {
+  HDR_N_RC = 0,      // (request, chunk) work items of this step
+  HDR_N_BND,         // requests at a capacity boundary
+  HDR_N_CMP,         // requests that compress
+  HDR_WORK_ATTN,     // dynamic work counter of the attention kernel
+  HDR_DONE_CMP,      // CTAs of the compaction kernel that have finished
+  HDR_STEP,          // step serial number
+  HDR_N_ACTIVE,      // requests actually stepped
+  HDR_COUNT = 16
+};
+
+// error bits
+enum {
+  GP_E_SPIN = 1,        // a bounded wait gave up
+  GP_E_FREELIST = 2,    // free-list accounting went negative or overflowed
+  GP_E_BOUNDS = 4,      // an index failed a bounds check and the access was skipped
+};
+
+struct GpDev {
+  // geometry
+  int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc, score_grid;
+  long long n_pages, max_batch_tokens;
+  double beta_s, beta_l, top_p, tau, rope_theta;
+  unsigned long long p_fix;              // top_p in 2^62 fixed point
+  // pool
+  __nv_bfloat16* kv;
+  int* tok;
+  int* refcount;
+  int* free_stack;
+  int* free_top;                         // number of free pages (stack height)
+  int* page_table;
+  int* shadow;
+  // per request
+  int* P; int* n; int* started; int* live; int* n_pristine; long long* pos;
+  double* summ;
+  int* Kx;                               // [M][L][H_kv][2]
+  double* delta;                         // [M]
+  // per step
+  int* hdr;
+  int4* rc;                              // {batch index, first page, pages, chunk | n_chunks << 16}
+  int* b_nold;                           // [M] occupied slots before the append, by batch index
+  int* b_flags;                          // [M] 1 = stepped this step
+  int* first_idx;                        // [M] lowest batch index naming a request
+  int* unit_cnt;                         // [M][L][H_kv] split-KV arrival counters
+  int* bnd_list;                         // [M] batch indices at a boundary
+  long long* bnd_off;                    // [M] token offset into the score scratch
+  int* cmp_list;                         // [M] batch indices that compress
+  double* rope_cs;                       // [M][d/2][2] cos, sin at the step's position
+  float* partials;
+  double* scores;
+  double* score_ws;                      // [score_grid][cap*b][2G] logits workspace
+  long long* counters;                   // [8]
+  int* err;
+};
+
+__device__ __forceinline__ size_t gp_tile_off(const GpDev& p, int l, long long page, int h) {
+  // element offset of the K tile of (layer, page, head); the V tile follows b*d elements later
+  return ((((size_t)l * (size_t)p.n_pages + (size_t)page) * p.Hkv + h) * 2) * (size_t)(GP_PAGE * p.d);
+}
+__device__ __forceinline__ size_t gp_tok_off(const GpDev& p, int l, long long page, int h) {
+  return (((size_t)l * (size_t)p.n_pages + (size_t)page) * p.Hkv + h) * GP_PAGE;
+}
+__device__ __forceinline__ size_t gp_summ_off(const GpDev& p, int l, int r, int x, int head) {
+  return ((((size_t)l * p.M + r) * 2 + x) * p.Hq + head) * (size_t)p.d;
+}
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false when the limit ran out (the caller records GP_E_SPIN and goes on).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < GP_SPIN_LIMIT; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+// 1-D bulk copy global -> shared of this CTA, completion counted on an mbarrier.  No multicast.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst_smem)),
+      "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo_f(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// ---- host-visible launchers (one per translation unit) -------------------------------------------
+void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
+                         float* out, int grid, cudaStream_t s);
+size_t gp_attention_smem(int d);
+int gp_attention_ctas_per_sm(int d);
+void gp_launch_score(const GpDev& p, const int* req_ids, int n_req, const void* q, cudaStream_t s);
+void gp_launch_compact(const GpDev& p, const int* req_ids, int n_req, int grid, cudaStream_t s);
+size_t gp_compact_smem(const GpDev& p);

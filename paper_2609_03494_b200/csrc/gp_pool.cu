@@ -1,0 +1,848 @@
+// Host side of the C ABI, the blob layout, and the small bookkeeping kernels:
+// step plan, decision + device allocator, admission, prompt ingest, release, debug gathers.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/growpage.h"
+#include "gp_dev.cuh"
+
+#define GP_MAX_REQ 1024
+#define GP_SCORE_GRID 296       // 2 CTAs per SM on 148 SMs
+#define GP_COMPACT_GRID 592     // 4 CTAs per SM
+#define GP_PLAN_THREADS 1024
+
+struct gp_pool {
+  gp_config cfg;
+  int device;
+  GpDev dev;
+  void* blob;
+  size_t bytes;
+  std::vector<uint8_t> live;      // host mirror of the slot free list
+  int num_sms, attn_grid;
+  // staging for the host-pointer entry point (inside the blob)
+  int* st_ids; void* st_q; void* st_k; void* st_v; float* st_out; int* st_act;
+  // small device words
+  int* d_status;
+  uint8_t* dbg;                   // gather target of the debug getters
+  int* aux;                       // [4][GP_MAX_REQ] decision scratch (spill of shared arrays, unused)
+  // measurement
+  int profiling;
+  cudaEvent_t ev[GP_N_KERNELS + 1];
+  float ms[GP_N_KERNELS];
+  int64_t launches[GP_N_KERNELS];
+  int64_t launch_count;
+};
+
+namespace {
+
+struct Layout {
+  size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
+      b_flags, first_idx, unit_cnt, bnd_list, bnd_off, cmp_list, rope_cs, partials, scores, score_ws, counters, dbg,
+      st_ids, st_q, st_k, st_v, st_out, st_act, total;
+  int max_rc;
+  long long max_batch_tokens;
+};
+
+inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+int chunk_pages_setting() {
+  const char* e = getenv("GP_CHUNK_PAGES");
+  int v = e ? atoi(e) : 16;
+  if (v < 1) v = 1;
+  if (v > 64) v = 64;
+  return v;
+}
+
+bool valid_config(const gp_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  const int G = c->n_q_heads / c->n_kv_heads;
+  if (G > 8 || (G & (G - 1))) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->page_size != GP_PAGE || c->recent_window != c->page_size) return false;
+  if (c->max_requests < 1 || c->max_requests > GP_MAX_REQ) return false;
+  if (c->max_pages_per_req < 1 || c->max_pages_per_req > (1 << 20)) return false;
+  if (c->n_pages < 1 || c->n_pages > 0x7fffffffLL / GP_PAGE) return false;
+  if (c->k_loc < 0 || c->k_loc > GP_PAGE) return false;
+  if (c->max_batch_tokens < 0) return false;
+  if (!(c->beta_s >= 0.0 && c->beta_s < 1.0 && c->beta_l >= 0.0 && c->beta_l < 1.0)) return false;
+  if (!(c->top_p > 0.0 && c->top_p < 1.0)) return false;
+  if (!(c->rope_theta >= 0.0)) return false;
+  return true;
+}
+
+Layout make_layout(const gp_config& c) {
+  Layout L;
+  const size_t M = c.max_requests, cap = c.max_pages_per_req, b = GP_PAGE, d = c.head_dim;
+  const size_t LH = (size_t)c.n_layers * c.n_kv_heads, G = c.n_q_heads / c.n_kv_heads;
+  const size_t np = (size_t)c.n_pages;
+  L.max_batch_tokens = c.max_batch_tokens > 0 ? c.max_batch_tokens : (long long)(np * b);
+  const int ch = chunk_pages_setting();
+  L.max_rc = (int)((size_t)L.max_batch_tokens / (b * ch) + 2 * M + 1);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  L.kv = take(LH * np * 2 * b * d * 2);
+  L.tok = take(LH * np * b * 4);
+  L.refcount = take(np * 4);
+  L.free_stack = take(np * 4);
+  L.words = take(256 * 4);                       // free_top, err, plan header, status
+  L.page_table = take(M * cap * 4);
+  L.shadow = take(M * cap * 4);
+  L.reqi = take(5 * M * 4);                      // P, n, started, live, n_pristine
+  L.pos = take(M * 8);
+  L.summ = take((size_t)c.n_layers * M * 2 * c.n_q_heads * d * 8);
+  L.Kx = take(M * LH * 2 * 4);
+  L.delta = take(M * 8);
+  L.rc = take((size_t)L.max_rc * 16);
+  L.b_nold = take(M * 4);
+  L.b_flags = take(M * 4);
+  L.first_idx = take(M * 4);
+  L.unit_cnt = take(M * LH * 4);
+  L.bnd_list = take(M * 4);
+  L.bnd_off = take(M * 8);
+  L.cmp_list = take(M * 4);
+  L.rope_cs = take(M * (d / 2) * 2 * 8);
+  L.partials = take((size_t)L.max_rc * LH * G * (d + 2) * 4);
+  L.scores = take(2 * LH * (size_t)L.max_batch_tokens * 8);
+  L.score_ws = take((size_t)GP_SCORE_GRID * cap * b * 2 * G * 8);
+  L.counters = take(8 * 8);
+  L.dbg = take(cap * b * (4 + 2 * d * 2));
+  if (c.host_staging) {
+    L.st_ids = take(M * 4);
+    L.st_q = take((size_t)c.n_layers * M * c.n_q_heads * d * 2);
+    L.st_k = take((size_t)c.n_layers * M * c.n_kv_heads * d * 2);
+    L.st_v = take((size_t)c.n_layers * M * c.n_kv_heads * d * 2);
+    L.st_out = take((size_t)c.n_layers * M * c.n_q_heads * d * 4);
+    L.st_act = take(M * 4);
+  } else {
+    L.st_ids = L.st_q = L.st_k = L.st_v = L.st_out = L.st_act = 0;
+  }
+  L.total = o;
+  return L;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// kernels
+// ---------------------------------------------------------------------------------------------------
+__global__ void gp_init_kernel(GpDev p) {
+  const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  // page 0 is handed out first
+  for (long long i = i0; i < p.n_pages; i += stride) p.free_stack[i] = (int)(p.n_pages - 1 - i);
+  for (long long i = i0; i < (long long)p.M * p.cap; i += stride) p.shadow[i] = -1;
+  for (long long i = i0; i < p.M; i += stride) p.first_idx[i] = 0x7fffffff;
+  if (i0 == 0) *p.free_top = (int)p.n_pages;
+}
+
+// exclusive scan over the CTA (1024 threads) of an int and a long long
+__device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long& ew, int& tv, long long& tw,
+                                          int* sv, long long* sw) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int iv = v; long long iw = w;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int a = __shfl_up_sync(0xffffffffu, iv, off);
+    const long long b2 = __shfl_up_sync(0xffffffffu, iw, off);
+    if (lane >= off) { iv += a; iw += b2; }
+  }
+  if (lane == 31) { sv[warp] = iv; sw[warp] = iw; }
+  __syncthreads();
+  int bv = 0; long long bw = 0;
+  tv = 0; tw = 0;
+  for (int i = 0; i < GP_PLAN_THREADS / 32; ++i) {
+    if (i < warp) { bv += sv[i]; bw += sw[i]; }
+    tv += sv[i]; tw += sw[i];
+  }
+  ev = bv + iv - v;
+  ew = bw + iw - w;
+  __syncthreads();
+}
+
+// Step plan: validates the batch, cuts every stepped request into (request, chunk) work items for the
+// attention kernel, lists the requests that reach their capacity boundary with this step's append
+// (trailing check: n + 1 == P b) and hands each a slice of the score scratch.
+__global__ void __launch_bounds__(GP_PLAN_THREADS)
+gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
+  __shared__ int sv[32];
+  __shared__ long long sw[32];
+  const int i = threadIdx.x;
+  const bool in = i < n_req;
+  int r = -1;
+  if (in) {
+    r = req_ids[i];
+    if (r >= 0 && r < p.M) atomicMin(&p.first_idx[r], i);
+  }
+  __syncthreads();
+  int chunks = 0, pages = 0, n_old = 0, act = GP_ACT_NONE;
+  long long nc = 0;
+  int isb = 0;
+  if (in) {
+    const bool valid = r >= 0 && r < p.M && p.live[r] && p.first_idx[r] == i;
+    if (!valid) {
+      act = GP_ACT_INVALID;
+    } else {
+      n_old = p.n[r];
+      const int Pr = p.P[r];
+      if (n_old >= Pr * GP_PAGE) {
+        act = GP_ACT_STALLED;
+      } else {
+        pages = n_old / GP_PAGE + 1;
+        chunks = (pages + p.chunk_pages - 1) / p.chunk_pages;
+        if (n_old + 1 == Pr * GP_PAGE) { isb = 1; nc = (long long)(Pr - 1) * GP_PAGE; }
+      }
+    }
+  }
+  int rc_off, n_rc; long long tok_off, tok_tot;
+  plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
+  if (isb && tok_off + nc > p.max_batch_tokens) { isb = 0; act = GP_ACT_SCRATCH; }
+  if (chunks > 0 && rc_off + chunks > p.max_rc) {      // cannot happen when max_batch_tokens is honoured
+    atomicOr(p.err, GP_E_BOUNDS);
+    chunks = 0; isb = 0; act = GP_ACT_SCRATCH;
+  }
+  int bnd_idx, n_bnd; long long dummy0, dummy1;
+  plan_scan(isb, 0, bnd_idx, dummy0, n_bnd, dummy1, sv, sw);
+  int act_idx, n_active;
+  plan_scan(chunks > 0, 0, act_idx, dummy0, n_active, dummy1, sv, sw);
+  if (in) {
+    p.b_nold[i] = n_old;
+    p.b_flags[i] = chunks > 0;
+    actions[i] = act;
+    for (int c = 0; c < chunks; ++c) {
+      const int pg0 = c * p.chunk_pages;
+      p.rc[rc_off + c] = make_int4(i, pg0, min(p.chunk_pages, pages - pg0), c | (chunks << 16));
+    }
+    if (isb) { p.bnd_list[bnd_idx] = i; p.bnd_off[i] = tok_off; }
+    if (r >= 0 && r < p.M) p.first_idx[r] = 0x7fffffff;          // ready for the next step
+  }
+  if (p.rope_theta != 0.0) {                                      // cos / sin of the step's position
+    const int half = p.d / 2;
+    for (int idx = threadIdx.x; idx < n_req * half; idx += GP_PLAN_THREADS) {
+      const int bi = idx / half, j = idx % half;
+      const int rr = req_ids[bi];
+      if (rr >= 0 && rr < p.M && p.live[rr]) {
+        const double inv = pow(p.rope_theta, -2.0 * (double)j / (double)p.d);
+        const double ang = (double)p.pos[rr] * inv;
+        double sn, cs;
+        sincos(ang, &sn, &cs);
+        p.rope_cs[(size_t)idx * 2] = cs;
+        p.rope_cs[(size_t)idx * 2 + 1] = sn;
+      }
+    }
+  }
+  if (threadIdx.x == 0) {
+    p.hdr[HDR_N_RC] = n_rc;
+    p.hdr[HDR_N_BND] = n_bnd;
+    p.hdr[HDR_N_CMP] = 0;
+    p.hdr[HDR_WORK_ATTN] = 0;
+    p.hdr[HDR_N_ACTIVE] = n_active;
+    p.hdr[HDR_STEP] += 1;
+  }
+}
+
+// After attention: advances n / pos of every stepped request, then for the requests at a boundary
+// aggregates Eq. 8, takes the grow-or-compress decision, and runs the device allocator:
+// grants first, then copy-on-write targets, each in ascending request id (Sec. 4.2, App. D.2).
+__global__ void __launch_bounds__(256)
+gp_decide_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
+  __shared__ int s_want[GP_MAX_REQ], s_ksh[GP_MAX_REQ], s_P[GP_MAX_REQ], s_order[GP_MAX_REQ], s_req[GP_MAX_REQ];
+  __shared__ int s_base[GP_MAX_REQ];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_bnd = p.hdr[HDR_N_BND];
+  for (int i = tid; i < n_req; i += 256) {
+    if (p.b_flags[i]) {
+      const int r = req_ids[i];
+      p.n[r] = p.b_nold[i] + 1;
+      p.pos[r] += 1;
+      p.started[r] = 1;
+    }
+  }
+  if (tid == 0) { p.counters[5] += 1; p.counters[6] += p.hdr[HDR_N_ACTIVE]; }
+  if (n_bnd == 0) return;
+  const int LH = p.L * p.Hkv;
+  for (int e = warp; e < n_bnd; e += 8) {
+    const int bi = p.bnd_list[e];
+    const int r = req_ids[bi];
+    const int Pr = p.P[r];
+    const int nC = (Pr - 1) * GP_PAGE;
+    long long sS = 0, sL = 0;
+    const int* kx = p.Kx + (size_t)r * LH * 2;
+    for (int j = lane; j < LH; j += 32) { sS += kx[2 * j]; sL += kx[2 * j + 1]; }
+    int ksh = 0;
+    const int* table = p.page_table + (size_t)r * p.cap;
+    for (int j = lane; j < Pr - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) {
+      sS += __shfl_xor_sync(0xffffffffu, sS, o2);
+      sL += __shfl_xor_sync(0xffffffffu, sL, o2);
+      ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
+    }
+    if (lane == 0) {
+      // Eq. 8 with a common |C|: Delta = (sum K^S - sum K^L) / (N |C|), one division of exact integers
+      double delta = 0.0;
+      int want = 1;
+      if (nC > 0) {
+        delta = (double)(sS - sL) / ((double)LH * (double)nC);
+        want = delta > p.tau;
+      }
+      p.delta[r] = delta;
+      s_want[e] = want; s_ksh[e] = ksh; s_P[e] = Pr; s_req[e] = r;
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < n_bnd; e += 256) {
+    int rank = 0;
+    for (int f = 0; f < n_bnd; ++f) rank += (s_req[f] < s_req[e]);
+    s_order[rank] = e;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int top = *p.free_top;
+    int n_cmp = 0;
+    long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0;
+    for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants
+      const int e = s_order[k];
+      const int r = s_req[e], Pr = s_P[e], bi = p.bnd_list[e];
+      if ((s_want[e] & 1) && Pr < p.cap && top > 0) {
+        const int page = p.free_stack[--top];
+        p.refcount[page] = 1;
+        p.page_table[(size_t)r * p.cap + Pr] = page;
+        p.P[r] = Pr + 1;
+        actions[bi] = GP_ACT_GROW;
+        s_want[e] |= 2;
+        ++grow;
+      } else if (Pr == 1) {
+        actions[bi] = GP_ACT_STALLED;
+        s_want[e] |= 4;
+        ++stall;
+      }
+    }
+    for (int k = 0; k < n_bnd; ++k) {                    // pass 2: copy-on-write targets
+      const int e = s_order[k];
+      if (s_want[e] & 6) continue;
+      const int r = s_req[e], bi = p.bnd_list[e];
+      if (s_ksh[e] > top) {
+        actions[bi] = GP_ACT_STALLED;
+        ++stall;
+        continue;
+      }
+      s_base[e] = top;
+      top -= s_ksh[e];
+      cow += s_ksh[e];
+      p.cmp_list[n_cmp++] = bi;
+      if (s_want[e] & 1) { actions[bi] = GP_ACT_COMPRESS_FALLBACK; ++fall; } else { actions[bi] = GP_ACT_COMPRESS; ++comp; }
+      p.n[r] = (s_P[e] - 1) * GP_PAGE;
+      p.n_pristine[r] = 0;
+      s_want[e] |= 8;
+    }
+    if (top < 0) atomicOr(p.err, GP_E_FREELIST);
+    *p.free_top = top;
+    p.hdr[HDR_N_CMP] = n_cmp;
+    p.counters[0] += grow; p.counters[1] += comp; p.counters[2] += fall; p.counters[3] += stall; p.counters[4] += cow;
+  }
+  __syncthreads();
+  for (int e = warp; e < n_bnd; e += 8) {                 // fill in the targets, in table order
+    if (!(s_want[e] & 8) || s_ksh[e] == 0) continue;
+    const int r = s_req[e], Pr = s_P[e], base = s_base[e];
+    const int* table = p.page_table + (size_t)r * p.cap;
+    int* shadow = p.shadow + (size_t)r * p.cap;
+    int running = 0;
+    for (int j0 = 0; j0 < Pr - 1; j0 += 32) {
+      const int j = j0 + lane;
+      const bool sh = j < Pr - 1 && p.refcount[table[j]] > 1;
+      const unsigned mask = __ballot_sync(0xffffffffu, sh);
+      if (sh) {
+        const int newp = p.free_stack[base - 1 - (running + __popc(mask & ((1u << lane) - 1u)))];
+        shadow[j] = newp;
+        p.refcount[newp] = 1;
+      }
+      running += __popc(mask);
+    }
+  }
+}
+
+__global__ void gp_admit_kernel(GpDev p, int r, int share_from, int n_shared, int n_tail, int P_target, int* status) {
+  const int lane = threadIdx.x;
+  const int need = P_target - n_shared;
+  const int top = *p.free_top;
+  int st = GP_OK;
+  if (n_shared > 0 && (!p.live[share_from] || p.n_pristine[share_from] < n_shared)) st = GP_ERR_INVALID;
+  else if (need > top || P_target > p.cap) st = GP_ERR_NO_PAGES;
+  __syncwarp();
+  if (st == GP_OK) {
+    int* table = p.page_table + (size_t)r * p.cap;
+    for (int j = lane; j < n_shared; j += 32) {
+      const int page = p.page_table[(size_t)share_from * p.cap + j];
+      table[j] = page;
+      atomicAdd(&p.refcount[page], 1);
+    }
+    for (int j = lane; j < need; j += 32) {
+      const int page = p.free_stack[top - 1 - j];
+      table[n_shared + j] = page;
+      p.refcount[page] = 1;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      const int n0 = n_shared * GP_PAGE + n_tail;
+      *p.free_top = top - need;
+      p.P[r] = P_target; p.n[r] = n0; p.pos[r] = n0; p.started[r] = 0; p.live[r] = 1;
+      p.n_pristine[r] = n0 / GP_PAGE;
+    }
+  }
+  if (lane == 0) *status = st;
+}
+
+// copies the private part of a prompt into its pages: one thread per 16-byte chunk
+__global__ void gp_ingest_kernel(GpDev p, int r, int n_shared, int n_tail, const __nv_bfloat16* k_tail,
+                                 const __nv_bfloat16* v_tail) {
+  const int CH = p.d / 8;
+  const long long total = (long long)p.L * n_tail * p.Hkv * 2 * CH;
+  const int row_bytes = p.d * 2;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % CH);
+    long long t2 = idx / CH;
+    const int isv = (int)(t2 % 2); t2 /= 2;
+    const int h = (int)(t2 % p.Hkv); t2 /= p.Hkv;
+    const int t = (int)(t2 % n_tail);
+    const int l = (int)(t2 / n_tail);
+    const __nv_bfloat16* src = (isv ? v_tail : k_tail) + (((size_t)l * n_tail + t) * p.Hkv + h) * p.d + c * 8;
+    const int slot = n_shared * GP_PAGE + t;
+    const int page = p.page_table[(size_t)r * p.cap + slot / GP_PAGE];
+    const int s = slot % GP_PAGE;
+    uint8_t* dst = reinterpret_cast<uint8_t*>(p.kv + gp_tile_off(p, l, page, h)) + isv * GP_PAGE * row_bytes +
+                   s * row_bytes + ((c ^ (s & 7)) << 4);
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    if (isv == 0 && c == 0) p.tok[gp_tok_off(p, l, page, h) + s] = slot;
+  }
+}
+
+__global__ void gp_release_kernel(GpDev p, int r) {
+  const int lane = threadIdx.x;
+  const int Pr = p.P[r];
+  const int* table = p.page_table + (size_t)r * p.cap;
+  for (int j0 = 0; j0 < Pr; j0 += 32) {
+    const int j = j0 + lane;
+    bool freed = false;
+    int page = -1;
+    if (j < Pr) {
+      page = table[j];
+      freed = (atomicSub(&p.refcount[page], 1) == 1);
+    }
+    const unsigned mask = __ballot_sync(0xffffffffu, freed);
+    int base = 0;
+    if (lane == 0) base = *reinterpret_cast<volatile int*>(p.free_top);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    if (freed) p.free_stack[base + __popc(mask & ((1u << lane) - 1u))] = page;
+    __syncwarp();
+    if (lane == 0 && mask) *reinterpret_cast<volatile int*>(p.free_top) = base + __popc(mask);
+    __syncwarp();
+  }
+  if (lane == 0) { p.live[r] = 0; p.P[r] = 0; p.n[r] = 0; p.started[r] = 0; p.n_pristine[r] = 0; }
+}
+
+// debug: token ids and un-swizzled K, V rows of one (layer, head) stream into the gather buffer
+__global__ void gp_gather_kernel(GpDev p, int r, int l, int h, int n, int* tok_out, uint4* k_out, uint4* v_out) {
+  const int CH = p.d / 8;
+  const int row_bytes = p.d * 2;
+  const long long total = (long long)n * 2 * CH;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % CH);
+    const int isv = (int)((idx / CH) % 2);
+    const int slot = (int)(idx / (2 * CH));
+    const int page = p.page_table[(size_t)r * p.cap + slot / GP_PAGE];
+    const int s = slot % GP_PAGE;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, l, page, h)) +
+                         isv * GP_PAGE * row_bytes + s * row_bytes + ((c ^ (s & 7)) << 4);
+    (isv ? v_out : k_out)[(size_t)slot * CH + c] = *reinterpret_cast<const uint4*>(src);
+    if (isv == 0 && c == 0) tok_out[slot] = p.tok[gp_tok_off(p, l, page, h) + s];
+  }
+}
+
+#define GP_CUDA(x)                      \
+  do {                                  \
+    if ((x) != cudaSuccess) return GP_ERR_CUDA; \
+  } while (0)
+
+int check_req(gp_pool* pool, int32_t req) {
+  if (!pool) return GP_ERR_INVALID;
+  if (req < 0 || req >= pool->cfg.max_requests || !pool->live[req]) return GP_ERR_INVALID;
+  return GP_OK;
+}
+
+}  // namespace
+
+// ===================================================================================================
+// C ABI
+// ===================================================================================================
+extern "C" {
+
+int gp_config_default(gp_config* cfg) {
+  if (!cfg) return GP_ERR_INVALID;
+  memset(cfg, 0, sizeof(*cfg));
+  cfg->page_size = GP_PAGE;
+  cfg->max_requests = 512;
+  cfg->recent_window = GP_PAGE;
+  cfg->k_loc = GP_PAGE / 4;
+  cfg->beta_s = 0.9;
+  cfg->beta_l = 0.999;
+  cfg->top_p = 0.99;
+  cfg->tau = 0.0;
+  cfg->rope_theta = 0.0;
+  return GP_OK;
+}
+
+size_t gp_pool_bytes(const gp_config* cfg) {
+  if (!valid_config(cfg)) return 0;
+  return make_layout(*cfg).total;
+}
+
+int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int device, gp_pool** out) {
+  if (!out) return GP_ERR_INVALID;
+  *out = nullptr;
+  if (!valid_config(cfg) || !dev_blob || ((uintptr_t)dev_blob & 255)) return GP_ERR_INVALID;
+  const Layout L = make_layout(*cfg);
+  if (bytes < L.total) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(device));
+  gp_pool* pool = new (std::nothrow) gp_pool();
+  if (!pool) return GP_ERR_STATE;
+  pool->cfg = *cfg;
+  pool->device = device;
+  pool->blob = dev_blob;
+  pool->bytes = bytes;
+  pool->live.assign(cfg->max_requests, 0);
+  pool->profiling = 0;
+  pool->launch_count = 0;
+  memset(pool->ms, 0, sizeof(pool->ms));
+  memset(pool->launches, 0, sizeof(pool->launches));
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+  pool->num_sms = prop.multiProcessorCount;
+  pool->attn_grid = pool->num_sms * gp_attention_ctas_per_sm(cfg->head_dim);
+
+  uint8_t* base = static_cast<uint8_t*>(dev_blob);
+  GpDev& d = pool->dev;
+  d.L = cfg->n_layers; d.Hq = cfg->n_q_heads; d.Hkv = cfg->n_kv_heads; d.G = cfg->n_q_heads / cfg->n_kv_heads;
+  d.d = cfg->head_dim; d.M = cfg->max_requests; d.cap = cfg->max_pages_per_req; d.k_loc = cfg->k_loc;
+  d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc; d.score_grid = GP_SCORE_GRID;
+  d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
+  d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
+  d.p_fix = (unsigned long long)llrint(cfg->top_p * 4611686018427387904.0);
+  d.kv = reinterpret_cast<__nv_bfloat16*>(base + L.kv);
+  d.tok = reinterpret_cast<int*>(base + L.tok);
+  d.refcount = reinterpret_cast<int*>(base + L.refcount);
+  d.free_stack = reinterpret_cast<int*>(base + L.free_stack);
+  int* words = reinterpret_cast<int*>(base + L.words);
+  d.free_top = words + 0;
+  d.err = words + 1;
+  pool->d_status = words + 2;
+  d.hdr = words + 64;
+  d.page_table = reinterpret_cast<int*>(base + L.page_table);
+  d.shadow = reinterpret_cast<int*>(base + L.shadow);
+  int* reqi = reinterpret_cast<int*>(base + L.reqi);
+  const int M = cfg->max_requests;
+  d.P = reqi; d.n = reqi + M; d.started = reqi + 2 * M; d.live = reqi + 3 * M; d.n_pristine = reqi + 4 * M;
+  d.pos = reinterpret_cast<long long*>(base + L.pos);
+  d.summ = reinterpret_cast<double*>(base + L.summ);
+  d.Kx = reinterpret_cast<int*>(base + L.Kx);
+  d.delta = reinterpret_cast<double*>(base + L.delta);
+  d.rc = reinterpret_cast<int4*>(base + L.rc);
+  d.b_nold = reinterpret_cast<int*>(base + L.b_nold);
+  d.b_flags = reinterpret_cast<int*>(base + L.b_flags);
+  d.first_idx = reinterpret_cast<int*>(base + L.first_idx);
+  d.unit_cnt = reinterpret_cast<int*>(base + L.unit_cnt);
+  d.bnd_list = reinterpret_cast<int*>(base + L.bnd_list);
+  d.bnd_off = reinterpret_cast<long long*>(base + L.bnd_off);
+  d.cmp_list = reinterpret_cast<int*>(base + L.cmp_list);
+  d.rope_cs = reinterpret_cast<double*>(base + L.rope_cs);
+  d.partials = reinterpret_cast<float*>(base + L.partials);
+  d.scores = reinterpret_cast<double*>(base + L.scores);
+  d.score_ws = reinterpret_cast<double*>(base + L.score_ws);
+  d.counters = reinterpret_cast<long long*>(base + L.counters);
+  pool->dbg = base + L.dbg;
+  if (cfg->host_staging) {
+    pool->st_ids = reinterpret_cast<int*>(base + L.st_ids);
+    pool->st_q = base + L.st_q; pool->st_k = base + L.st_k; pool->st_v = base + L.st_v;
+    pool->st_out = reinterpret_cast<float*>(base + L.st_out);
+    pool->st_act = reinterpret_cast<int*>(base + L.st_act);
+  } else {
+    pool->st_ids = nullptr; pool->st_q = pool->st_k = pool->st_v = nullptr; pool->st_out = nullptr; pool->st_act = nullptr;
+  }
+  // Stale pages are read (masked) by the attention kernel, so they must hold finite numbers.
+  if (cudaMemset(dev_blob, 0, L.total) != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+  gp_init_kernel<<<1024, 256>>>(d);
+  pool->launch_count++;
+  for (int i = 0; i <= GP_N_KERNELS; ++i) {
+    if (cudaEventCreate(&pool->ev[i]) != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+  }
+  if (cudaDeviceSynchronize() != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+  *out = pool;
+  return GP_OK;
+}
+
+int gp_pool_destroy(gp_pool* pool) {
+  if (!pool) return GP_ERR_INVALID;
+  cudaSetDevice(pool->device);
+  cudaDeviceSynchronize();
+  for (int i = 0; i <= GP_N_KERNELS; ++i) cudaEventDestroy(pool->ev[i]);
+  delete pool;
+  return GP_OK;
+}
+
+int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, const void* k_tail, const void* v_tail,
+                   int32_t n_tail, int32_t initial_pages, void* stream, int32_t* out_req) {
+  if (!pool || !out_req || n_tail < 0 || n_shared_pages < 0 || initial_pages < 0) return GP_ERR_INVALID;
+  if (n_tail > 0 && (!k_tail || !v_tail)) return GP_ERR_INVALID;
+  *out_req = -1;
+  if (n_shared_pages > 0 && check_req(pool, share_from) != GP_OK) return GP_ERR_INVALID;
+  const gp_config& c = pool->cfg;
+  int slot = -1;
+  for (int i = 0; i < c.max_requests; ++i)
+    if (!pool->live[i]) { slot = i; break; }
+  if (slot < 0) return GP_ERR_NO_SLOT;
+  const long long n_prompt = (long long)n_shared_pages * GP_PAGE + n_tail;
+  long long P = n_prompt / GP_PAGE + 1;
+  if (initial_pages > P) P = initial_pages;
+  if (P > c.max_pages_per_req) return GP_ERR_NO_PAGES;
+  GP_CUDA(cudaSetDevice(pool->device));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  gp_admit_kernel<<<1, 32, 0, s>>>(pool->dev, slot, share_from, n_shared_pages, n_tail, (int)P, pool->d_status);
+  pool->launch_count++;
+  int st = GP_ERR_CUDA;
+  GP_CUDA(cudaMemcpyAsync(&st, pool->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  GP_CUDA(cudaStreamSynchronize(s));
+  if (st != GP_OK) return st;
+  if (n_tail > 0) {
+    const long long total = (long long)c.n_layers * n_tail * c.n_kv_heads * 2 * (c.head_dim / 8);
+    int grid = (int)((total + 255) / 256);
+    if (grid > 148 * 16) grid = 148 * 16;
+    gp_ingest_kernel<<<grid, 256, 0, s>>>(pool->dev, slot, n_shared_pages, n_tail,
+                                         static_cast<const __nv_bfloat16*>(k_tail),
+                                         static_cast<const __nv_bfloat16*>(v_tail));
+    pool->launch_count++;
+    GP_CUDA(cudaStreamSynchronize(s));     // the caller may free the prompt buffers on return
+  }
+  pool->live[slot] = 1;
+  *out_req = slot;
+  return GP_OK;
+}
+
+int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
+                   const void* v, void* out, int32_t* dev_actions, void* stream) {
+  if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
+  if (n_req == 0) return GP_OK;
+  if (!dev_req_ids || !q || !k || !v || !out || !dev_actions) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const GpDev& d = pool->dev;
+  const bool prof = pool->profiling != 0;
+  if (prof) cudaEventRecord(pool->ev[0], s);
+  gp_plan_kernel<<<1, GP_PLAN_THREADS, 0, s>>>(d, dev_req_ids, n_req, dev_actions);
+  if (prof) cudaEventRecord(pool->ev[1], s);
+  gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s);
+  if (prof) cudaEventRecord(pool->ev[2], s);
+  gp_launch_score(d, dev_req_ids, n_req, q, s);
+  if (prof) cudaEventRecord(pool->ev[3], s);
+  gp_decide_kernel<<<1, 256, 0, s>>>(d, dev_req_ids, n_req, dev_actions);
+  if (prof) cudaEventRecord(pool->ev[4], s);
+  gp_launch_compact(d, dev_req_ids, n_req, GP_COMPACT_GRID, s);
+  if (prof) cudaEventRecord(pool->ev[5], s);
+  pool->launch_count += GP_N_KERNELS;
+  GP_CUDA(cudaGetLastError());
+  if (prof) {
+    GP_CUDA(cudaEventSynchronize(pool->ev[GP_N_KERNELS]));
+    for (int i = 0; i < GP_N_KERNELS; ++i) {
+      float t = 0.f;
+      GP_CUDA(cudaEventElapsedTime(&t, pool->ev[i], pool->ev[i + 1]));
+      pool->ms[i] += t;
+      pool->launches[i] += 1;
+    }
+  }
+  return GP_OK;
+}
+
+int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
+                        const void* v, void* out, int32_t* actions, void* stream) {
+  if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
+  if (!pool->st_ids) return GP_ERR_STATE;
+  if (n_req == 0) return GP_OK;
+  if (!host_req_ids || !q || !k || !v || !out || !actions) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const gp_config& c = pool->cfg;
+  const size_t qb = (size_t)c.n_layers * n_req * c.n_q_heads * c.head_dim * 2;
+  const size_t kb = (size_t)c.n_layers * n_req * c.n_kv_heads * c.head_dim * 2;
+  GP_CUDA(cudaMemcpyAsync(pool->st_ids, host_req_ids, (size_t)n_req * 4, cudaMemcpyHostToDevice, s));
+  GP_CUDA(cudaMemcpyAsync(pool->st_q, q, qb, cudaMemcpyHostToDevice, s));
+  GP_CUDA(cudaMemcpyAsync(pool->st_k, k, kb, cudaMemcpyHostToDevice, s));
+  GP_CUDA(cudaMemcpyAsync(pool->st_v, v, kb, cudaMemcpyHostToDevice, s));
+  const int st = gp_decode_step(pool, pool->st_ids, n_req, pool->st_q, pool->st_k, pool->st_v, pool->st_out,
+                                pool->st_act, stream);
+  if (st != GP_OK) return st;
+  GP_CUDA(cudaMemcpyAsync(out, pool->st_out, qb * 2, cudaMemcpyDeviceToHost, s));
+  GP_CUDA(cudaMemcpyAsync(actions, pool->st_act, (size_t)n_req * 4, cudaMemcpyDeviceToHost, s));
+  GP_CUDA(cudaStreamSynchronize(s));
+  return GP_OK;
+}
+
+int gp_release(gp_pool* pool, int32_t req, void* stream) {
+  const int st = check_req(pool, req);
+  if (st != GP_OK) return st;
+  GP_CUDA(cudaSetDevice(pool->device));
+  gp_release_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(pool->dev, req);
+  pool->launch_count++;
+  pool->live[req] = 0;
+  GP_CUDA(cudaGetLastError());
+  return GP_OK;
+}
+
+const char* gp_strerror(int status) {
+  switch (status) {
+    case GP_OK: return "ok";
+    case GP_ERR_INVALID: return "invalid argument or request id";
+    case GP_ERR_NO_SLOT: return "no free request slot";
+    case GP_ERR_NO_PAGES: return "not enough free pages or per-request cap exceeded";
+    case GP_ERR_CUDA: return "CUDA error or internal kernel error";
+    case GP_ERR_STATE: return "call not possible in this state";
+    default: return "unknown status";
+  }
+}
+
+// ---- introspection ---------------------------------------------------------------------------------
+int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t* pos, int32_t* page_table) {
+  const int st = check_req(pool, req);
+  if (st != GP_OK) return st;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  int Pv = 0, nv = 0; long long pv = 0;
+  GP_CUDA(cudaMemcpy(&Pv, pool->dev.P + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&nv, pool->dev.n + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&pv, pool->dev.pos + req, 8, cudaMemcpyDeviceToHost));
+  if (P) *P = Pv;
+  if (n) *n = nv;
+  if (pos) *pos = pv;
+  if (page_table && Pv > 0)
+    GP_CUDA(cudaMemcpy(page_table, pool->dev.page_table + (size_t)req * pool->cfg.max_pages_per_req, (size_t)Pv * 4,
+                       cudaMemcpyDeviceToHost));
+  return GP_OK;
+}
+
+static int gather_stream(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_head, int* n_out) {
+  const int st = check_req(pool, req);
+  if (st != GP_OK) return st;
+  if (layer < 0 || layer >= pool->cfg.n_layers || kv_head < 0 || kv_head >= pool->cfg.n_kv_heads) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  int nv = 0;
+  GP_CUDA(cudaMemcpy(&nv, pool->dev.n + req, 4, cudaMemcpyDeviceToHost));
+  *n_out = nv;
+  if (nv == 0) return GP_OK;
+  const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * GP_PAGE;
+  int* tok = reinterpret_cast<int*>(pool->dbg);
+  uint4* kk = reinterpret_cast<uint4*>(pool->dbg + cap_tok * 4);
+  uint4* vv = reinterpret_cast<uint4*>(pool->dbg + cap_tok * 4 + cap_tok * pool->cfg.head_dim * 2);
+  gp_gather_kernel<<<148, 256>>>(pool->dev, req, layer, kv_head, nv, tok, kk, vv);
+  pool->launch_count++;
+  GP_CUDA(cudaDeviceSynchronize());
+  return GP_OK;
+}
+
+int gp_debug_retained(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_head, int32_t* token_ids) {
+  if (!token_ids) return GP_ERR_INVALID;
+  int n = 0;
+  const int st = gather_stream(pool, req, layer, kv_head, &n);
+  if (st != GP_OK) return st;
+  if (n > 0) GP_CUDA(cudaMemcpy(token_ids, pool->dbg, (size_t)n * 4, cudaMemcpyDeviceToHost));
+  return GP_OK;
+}
+
+int gp_debug_kv(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_head, void* k_rows, void* v_rows) {
+  int n = 0;
+  const int st = gather_stream(pool, req, layer, kv_head, &n);
+  if (st != GP_OK) return st;
+  const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * GP_PAGE;
+  const size_t rowb = (size_t)pool->cfg.head_dim * 2;
+  if (n > 0 && k_rows) GP_CUDA(cudaMemcpy(k_rows, pool->dbg + cap_tok * 4, n * rowb, cudaMemcpyDeviceToHost));
+  if (n > 0 && v_rows)
+    GP_CUDA(cudaMemcpy(v_rows, pool->dbg + cap_tok * 4 + cap_tok * rowb, n * rowb, cudaMemcpyDeviceToHost));
+  return GP_OK;
+}
+
+int gp_debug_summaries(gp_pool* pool, int32_t req, double* out) {
+  const int st = check_req(pool, req);
+  if (st != GP_OK) return st;
+  if (!out) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  const gp_config& c = pool->cfg;
+  const size_t per = (size_t)2 * c.n_q_heads * c.head_dim;
+  for (int l = 0; l < c.n_layers; ++l)
+    GP_CUDA(cudaMemcpy(out + (size_t)l * per, pool->dev.summ + ((size_t)l * c.max_requests + req) * per, per * 8,
+                       cudaMemcpyDeviceToHost));
+  return GP_OK;
+}
+
+int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, double* delta) {
+  const int st = check_req(pool, req);
+  if (st != GP_OK) return st;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  const int LH = pool->cfg.n_layers * pool->cfg.n_kv_heads;
+  std::vector<int> kx((size_t)LH * 2);
+  GP_CUDA(cudaMemcpy(kx.data(), pool->dev.Kx + (size_t)req * LH * 2, (size_t)LH * 8, cudaMemcpyDeviceToHost));
+  for (int i = 0; i < LH; ++i) {
+    if (K_S) K_S[i] = kx[2 * i];
+    if (K_L) K_L[i] = kx[2 * i + 1];
+  }
+  if (delta) GP_CUDA(cudaMemcpy(delta, pool->dev.delta + req, 8, cudaMemcpyDeviceToHost));
+  return GP_OK;
+}
+
+int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[8]) {
+  if (!pool) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  int top = 0, err = 0;
+  GP_CUDA(cudaMemcpy(&top, pool->dev.free_top, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&err, pool->dev.err, 4, cudaMemcpyDeviceToHost));
+  if (n_free) *n_free = top;
+  if (refcounts) GP_CUDA(cudaMemcpy(refcounts, pool->dev.refcount, (size_t)pool->cfg.n_pages * 4, cudaMemcpyDeviceToHost));
+  if (counters) {
+    long long c[8];
+    GP_CUDA(cudaMemcpy(c, pool->dev.counters, 64, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 7; ++i) counters[i] = c[i];
+    counters[7] = err;
+  }
+  return GP_OK;
+}
+
+int gp_set_profiling(gp_pool* pool, int32_t enable) {
+  if (!pool) return GP_ERR_INVALID;
+  pool->profiling = enable ? 1 : 0;
+  memset(pool->ms, 0, sizeof(pool->ms));
+  memset(pool->launches, 0, sizeof(pool->launches));
+  return GP_OK;
+}
+
+int gp_get_kernel_times(gp_pool* pool, float* ms, int64_t* launches) {
+  if (!pool) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  for (int i = 0; i < GP_N_KERNELS; ++i) {
+    if (ms) ms[i] = pool->ms[i];
+    if (launches) launches[i] = pool->launches[i];
+  }
+  memset(pool->ms, 0, sizeof(pool->ms));
+  memset(pool->launches, 0, sizeof(pool->launches));
+  return GP_OK;
+}
+
+int64_t gp_launch_count(gp_pool* pool) { return pool ? pool->launch_count : 0; }
+
+}  // extern "C"

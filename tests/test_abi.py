@@ -1,0 +1,51 @@
+"""The C-ABI library builds, loads without a GPU, and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+from paper_2609_03494_b200 import binding as B
+from paper_2609_03494_b200 import build as builder
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "growpage.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gp_[a-z_]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_the_header():
+    path = builder.build()
+    assert os.path.exists(path)
+    lib = ctypes.CDLL(path)
+    names = _declared()
+    assert {"gp_pool_create", "gp_request_add", "gp_decode_step", "gp_release"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in growpage.h but not exported"
+
+
+def test_binding_mirrors_the_header_names():
+    for name in _declared():
+        assert hasattr(B, name), f"binding lacks {name}"
+
+
+def test_config_defaults_and_pool_bytes_need_no_gpu():
+    cfg = B.gp_config_default()
+    assert (cfg.beta_s, cfg.beta_l, cfg.top_p, cfg.tau) == (0.9, 0.999, 0.99, 0.0)
+    assert cfg.page_size == 16 and cfg.recent_window == 16 and cfg.k_loc == 4 and cfg.max_requests == 512
+    assert B.gp_pool_bytes(cfg) == 0                       # geometry not filled in: invalid
+    cfg = B.make_config(1, 32, 8, 128, n_pages=1024, max_pages_per_req=64, max_requests=64)
+    nbytes = B.gp_pool_bytes(cfg)
+    kv = 1024 * 16 * 4096                                   # K and V of every slot
+    assert kv < nbytes < 2 * kv + (256 << 20)
+    bad = B.make_config(1, 32, 8, 96, n_pages=1024, max_pages_per_req=64)
+    assert B.gp_pool_bytes(bad) == 0
+    bad = B.make_config(1, 30, 8, 128, n_pages=1024, max_pages_per_req=64)
+    assert B.gp_pool_bytes(bad) == 0
+    assert B.lib().gp_strerror(B.GP_ERR_NO_PAGES).decode().startswith("not enough")
+
+
+def test_struct_layout_matches_the_header():
+    # 10 int32, 2 int64, 5 double, no padding surprises
+    assert ctypes.sizeof(B.gp_config) == 10 * 4 + 2 * 8 + 5 * 8

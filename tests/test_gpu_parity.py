@@ -1,0 +1,119 @@
+"""GPU parity: the CUDA path against the float64 oracle on the same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import growpage_oracle as O
+from paper_2609_03494_b200 import binding as B
+from paper_2609_03494_b200 import workload as W
+from tests import lockstep as LS
+
+pytestmark = pytest.mark.gpu
+
+
+def _report(name, st):
+    print(f"\n[{name}] steps {st.steps} tokens {st.tokens} attn max {st.attn_max_abs:.2e} mean {st.attn_mean_abs:.2e} "
+          f"summary rel {st.summary_max_rel:.1e} decisions {st.decisions} near-ties {st.near_ties} actions {st.actions}")
+
+
+def test_config1_tiny_every_step():
+    st = LS.run_lockstep(W.parity_instance(1), summary_every=1, check_pool_every=1)
+    _report("tiny", st)
+    assert st.steps == 256 and st.tokens == 1024
+    assert st.actions.get(B.GP_ACT_COMPRESS, 0) > 0
+
+
+@pytest.mark.parametrize("config", [2, 3, 4, 5])
+def test_configs_2_to_5_reduced(config):
+    st = LS.run_lockstep(W.parity_instance(config))
+    _report(f"config{config}", st)
+    assert st.decisions["sel"] > 0
+    if config == 5:
+        assert st.counters[4] > 0            # copy-on-write happened
+
+
+def test_tiny_with_negative_threshold_mixes_grow_fallback_and_compress():
+    st = LS.run_lockstep(W.parity_instance(1), tau=-0.07)
+    _report("tiny tau=-0.07", st)
+    assert st.actions.get(B.GP_ACT_GROW, 0) > 0 and st.actions.get(B.GP_ACT_COMPRESS, 0) > 0
+    st = LS.run_lockstep(W.parity_instance(1), tau=-1.0)            # always wants to grow: cap 16 forces fallback
+    _report("tiny tau=-1", st)
+    assert st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) > 0 and st.actions.get(B.GP_ACT_COMPRESS, 0) == 0
+
+
+def test_tiny_with_rope():
+    st = LS.run_lockstep(W.parity_instance(1), rope_theta=1e6, tau=-0.05)
+    _report("tiny rope", st)
+
+
+def test_tiny_under_pool_pressure_falls_back_and_stalls():
+    wl = W.parity_instance(1)
+    st = LS.run_lockstep(wl, tau=-1.0, n_pages=4 * 5 + 3)           # three spare pages for four growers
+    _report("tiny small pool", st)
+    assert st.actions.get(B.GP_ACT_GROW, 0) == 3 and st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) > 0
+
+
+def test_other_quota_and_coverage_settings():
+    st = LS.run_lockstep(W.parity_instance(1), k_loc=0, top_p=0.9, beta_s=0.5, beta_l=0.95, max_steps=120)
+    _report("tiny k_loc=0", st)
+    st = LS.run_lockstep(W.parity_instance(1), k_loc=16, tau=-0.02, max_steps=120)
+    _report("tiny k_loc=16", st)
+
+
+def _single_request_case(shape, n_prompt, n_steps, seed=11):
+    wl = W.Workload("adhoc", seed, shape, [W.RequestSpec(0, n_prompt, n_steps, 0.05)], n_resident=1, initial_pages=0,
+                    max_pages_per_req=n_prompt // 16 + 4, n_pages=n_prompt // 16 + 8)
+    return LS.run_lockstep(wl, tau=-1.0)
+
+
+@pytest.mark.parametrize("hq,hkv,d,n_prompt", [(32, 8, 128, 1530), (64, 8, 128, 777), (4, 4, 64, 1100),
+                                               (2, 1, 64, 15), (8, 8, 128, 1), (16, 2, 128, 260)])
+def test_long_sequences_span_chunks_and_ragged_tails(hq, hkv, d, n_prompt):
+    st = _single_request_case(W.Shape(2, hq, hkv, d), n_prompt, 40)
+    _report(f"long {hq}/{hkv}/{d} n={n_prompt}", st)
+
+
+def test_batch_edge_cases_and_host_entry_point():
+    import torch
+    shape = W.Shape(1, 8, 2, 64)
+    cfg = B.make_config(1, 8, 2, 64, n_pages=32, max_pages_per_req=4, max_requests=8, host_staging=True)
+    pool = B.Pool(cfg)
+    try:
+        rng = np.random.default_rng(0)
+        kt = W.f32_to_bf16_bits(rng.standard_normal((1, 20, 2, 64)).astype(np.float32))
+        vt = W.f32_to_bf16_bits(rng.standard_normal((1, 20, 2, 64)).astype(np.float32))
+        st, a = pool.request_add(-1, 0, kt, vt, 20, 0)
+        assert (st, a) == (B.GP_OK, 0)
+        st, b_ = pool.request_add(-1, 0, kt, vt, 20, 0)
+        assert (st, b_) == (B.GP_OK, 1)
+        assert pool.request_add(5, 1, None, None, 0, 0)[0] == B.GP_ERR_INVALID      # donor not live
+        assert pool.request_add(a, 2, None, None, 0, 0)[0] == B.GP_ERR_INVALID      # only one full prompt page
+        assert pool.request_add(-1, 0, kt, vt, 20, 9)[0] == B.GP_ERR_NO_PAGES       # above the per-request cap
+        # empty batch is a no-op
+        B.gp_decode_step(pool.handle, 0, 0, 0, 0, 0, 0, 0, pool.stream())
+        # invalid, duplicate and dead ids are flagged per request; the valid ones still run
+        ids = torch.tensor([a, 7, a, b_, -1], dtype=torch.int32)
+        q = W.f32_to_bf16_bits(rng.standard_normal((1, 5, 8, 64)).astype(np.float32))
+        k = W.f32_to_bf16_bits(rng.standard_normal((1, 5, 2, 64)).astype(np.float32))
+        v = W.f32_to_bf16_bits(rng.standard_normal((1, 5, 2, 64)).astype(np.float32))
+        out = torch.zeros((1, 5, 8, 64), dtype=torch.float32).pin_memory()
+        act = torch.zeros(5, dtype=torch.int32).pin_memory()
+        tq, tk, tv = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (q, k, v))
+        pool.decode_step_host(ids.pin_memory(), tq, tk, tv, out, act)
+        assert act.tolist() == [B.GP_ACT_NONE, B.GP_ACT_INVALID, B.GP_ACT_INVALID, B.GP_ACT_NONE, B.GP_ACT_INVALID]
+        # the host entry point gives what the oracle gives
+        f = W.bf16_bits_to_f64
+        for col, rid in ((0, a), (3, b_)):
+            K = np.concatenate([f(kt)[0].transpose(1, 0, 2), f(k)[0, col][:, None, :]], axis=1)
+            V = np.concatenate([f(vt)[0].transpose(1, 0, 2), f(v)[0, col][:, None, :]], axis=1)
+            want = O.attention_decode(f(q)[0, col], K, V)
+            assert np.abs(out[0, col].numpy() - want).max() <= 1e-2
+            P, n, pos, _ = B.gp_debug_request(pool.handle, rid, 4)
+            assert (P, n, pos) == (2, 21, 21)
+        pool.release(a)
+        with pytest.raises(B.GpError):
+            pool.release(a)
+        n_free, ref, counters = B.gp_debug_pool(pool.handle, 32)
+        assert n_free == 30 and counters[7] == 0
+        assert B.gp_launch_count(pool.handle) > 0
+    finally:
+        pool.close()
