@@ -148,8 +148,10 @@ int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, do
 
 /* Free pages, per-page reference counts (host int32 [n_pages], may be NULL) and event counters:
  * [0] grow [1] compress [2] fallback-compress [3] stalled [4] copy-on-write pages
- * [5] decode steps [6] tokens decoded [7] internal error bits (0 when healthy). */
-int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[8]);
+ * [5] decode steps [6] tokens decoded [7] internal error bits (0 when healthy)
+ * [8] (layer, head, token) rows rewritten by compaction [9] candidate tokens scored at boundaries
+ * [10], [11] reserved. */
+int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[12]);
 
 /* ---- measurement ----------------------------------------------------------------------------- */
 

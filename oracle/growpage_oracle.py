@@ -279,7 +279,8 @@ class OraclePool:
         self.refcount = np.zeros(cfg.n_pages, dtype=np.int64)
         self.free: List[int] = list(range(cfg.n_pages - 1, -1, -1))   # pop() hands out page 0 first
         self.requests: Dict[int, _Request] = {}
-        self.counters = {"grow": 0, "compress": 0, "fallback": 0, "stalled": 0, "cow_pages": 0}
+        self.counters = {"grow": 0, "compress": 0, "fallback": 0, "stalled": 0, "cow_pages": 0,
+                         "moved_rows": 0, "scored_tokens": 0}
 
     # ---- pool primitives ------------------------------------------------------
     def _take_page(self) -> int:
@@ -450,6 +451,7 @@ class OraclePool:
             r = self.requests[rid]
             want = overrides.get(rid, {}).get("want_grow", info.want_grow)
             info.want_grow = bool(want)
+            self.counters["scored_tokens"] += info.n_c
             if want and r.P < c.max_pages_per_req and self.free:
                 r.table.append(self._take_page())
                 r.P += 1
@@ -514,6 +516,7 @@ class OraclePool:
                 r.tok[l, h, src.size:r.P * b] = -1
         r.n = n_c
         info.moved_tokens = moved
+        self.counters["moved_rows"] += moved
 
     # ---- introspection -----------------------------------------------------------
     def retained(self, rid: int, l: int, h: int) -> np.ndarray:

@@ -171,7 +171,7 @@ def gp_debug_boundary(pool: int, req: int, L: int, Hkv: int):
 
 def gp_debug_pool(pool: int, n_pages: int = 0):
     n_free = C.c_int64()
-    counters = np.zeros(8, dtype=np.int64)
+    counters = np.zeros(12, dtype=np.int64)
     ref = np.zeros(max(n_pages, 1), dtype=np.int32)
     _check(lib().gp_debug_pool(C.c_void_p(pool), C.byref(n_free), ref.ctypes.data_as(C.c_void_p) if n_pages else None,
                                counters.ctypes.data_as(C.c_void_p)), "gp_debug_pool")

@@ -367,7 +367,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 
     // ---- block-local quota: the k' best slots of every page of C (score desc, slot asc) ---------------
     for (int i = tid; i < (nC + 31) / 32; i += BT) loc[i] = 0;
-    if (tid == 0) { s_i[0] = 0; s_i[1] = 0x7fffffff; }
+    if (tid == 0) { s_i[0] = 0; s_i[1] = 0x7fffffff; s_i[3] = 0; }
     __syncthreads();
     for (int t0 = 0; t0 < nC; t0 += BT) {
       const int tokn = t0 + tid;
@@ -534,12 +534,14 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         }
       }
       if (tok_dst >= 0) {
+        atomicAdd(&s_i[3], 1);
         const int pg = tok_dst / GP_PAGE;
         const int page = shadow[pg] >= 0 ? shadow[pg] : table[pg];
         p.tok[gp_tok_off(p, l, page, h) + (tok_dst % GP_PAGE)] = tokv;
       }
       __syncthreads();
     }
+    if (tid == 0) atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 8), (unsigned long long)s_i[3]);
   }
 
   // ---- the last CTA swaps in the copy-on-write targets and drops the old references (App. D.2) ----------

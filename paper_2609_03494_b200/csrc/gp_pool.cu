@@ -29,7 +29,6 @@ struct gp_pool {
   // small device words
   int* d_status;
   uint8_t* dbg;                   // gather target of the debug getters
-  int* aux;                       // [4][GP_MAX_REQ] decision scratch (spill of shared arrays, unused)
   // measurement
   int profiling;
   cudaEvent_t ev[GP_N_KERNELS + 1];
@@ -111,7 +110,7 @@ Layout make_layout(const gp_config& c) {
   L.partials = take((size_t)L.max_rc * LH * G * (d + 2) * 4);
   L.scores = take(2 * LH * (size_t)L.max_batch_tokens * 8);
   L.score_ws = take((size_t)GP_SCORE_GRID * cap * b * 2 * G * 8);
-  L.counters = take(8 * 8);
+  L.counters = take(16 * 8);
   L.dbg = take(cap * b * (4 + 2 * d * 2));
   if (c.host_staging) {
     L.st_ids = take(M * 4);
@@ -304,10 +303,11 @@ gp_decide_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_id
   if (tid == 0) {
     int top = *p.free_top;
     int n_cmp = 0;
-    long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0;
+    long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0;
     for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants
       const int e = s_order[k];
       const int r = s_req[e], Pr = s_P[e], bi = p.bnd_list[e];
+      scored += (long long)(Pr - 1) * GP_PAGE;
       if ((s_want[e] & 1) && Pr < p.cap && top > 0) {
         const int page = p.free_stack[--top];
         p.refcount[page] = 1;
@@ -344,6 +344,7 @@ gp_decide_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_id
     *p.free_top = top;
     p.hdr[HDR_N_CMP] = n_cmp;
     p.counters[0] += grow; p.counters[1] += comp; p.counters[2] += fall; p.counters[3] += stall; p.counters[4] += cow;
+    p.counters[9] += scored;
   }
   __syncthreads();
   for (int e = warp; e < n_bnd; e += 8) {                 // fill in the targets, in table order
@@ -804,7 +805,7 @@ int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, do
   return GP_OK;
 }
 
-int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[8]) {
+int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[12]) {
   if (!pool) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
   GP_CUDA(cudaDeviceSynchronize());
@@ -814,9 +815,9 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
   if (n_free) *n_free = top;
   if (refcounts) GP_CUDA(cudaMemcpy(refcounts, pool->dev.refcount, (size_t)pool->cfg.n_pages * 4, cudaMemcpyDeviceToHost));
   if (counters) {
-    long long c[8];
-    GP_CUDA(cudaMemcpy(c, pool->dev.counters, 64, cudaMemcpyDeviceToHost));
-    for (int i = 0; i < 7; ++i) counters[i] = c[i];
+    long long c[12];
+    GP_CUDA(cudaMemcpy(c, pool->dev.counters, 96, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 12; ++i) counters[i] = c[i];
     counters[7] = err;
   }
   return GP_OK;

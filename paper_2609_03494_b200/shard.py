@@ -1,0 +1,75 @@
+"""Multi-GPU plumbing.  The decode path shards by request: every GPU owns a pool and a disjoint set
+of requests, and no step of the path exchanges data between them.  What is left for
+`torch.distributed` is the rendezvous, the barrier around the timed region and the max-over-ranks
+of the device time.  Works with NCCL (one process per GPU) and with gloo (CPU tests)."""
+from __future__ import annotations
+
+import os
+from typing import List, Tuple
+
+
+def env_world() -> Tuple[int, int, int]:
+    """(rank, local rank, world size) from the torchrun environment; (0, 0, 1) when absent."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def init(backend: str) -> Tuple[int, int, int]:
+    import torch.distributed as dist
+    rank, local_rank, world = env_world()
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, local_rank, world
+
+
+def shard_seed(base_seed: int, rank: int) -> int:
+    """Weak scaling: rank r decodes its own set of requests, drawn with this seed.  Rank 0 keeps the
+    configuration's own seed."""
+    return base_seed + 1000 * rank
+
+
+def shard_requests(n_requests: int, rank: int, world: int) -> List[int]:
+    """Strong-scaling split of a fixed request list: contiguous, sizes differ by at most one."""
+    base, extra = divmod(n_requests, world)
+    lo = rank * base + min(rank, extra)
+    return list(range(lo, lo + base + (1 if rank < extra else 0)))
+
+
+def barrier(device=None) -> None:
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        if device is not None and dist.get_backend() == "nccl":
+            dist.barrier(device_ids=[device])
+        else:
+            dist.barrier()
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    dev = f"cuda:{device}" if (device is not None and dist.get_backend() == "nccl") else "cpu"
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, device=None) -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    dev = f"cuda:{device}" if (device is not None and dist.get_backend() == "nccl") else "cpu"
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def job_throughput(units_this_rank: float, ms_this_rank: float, device=None) -> Tuple[float, float]:
+    """Whole-job throughput: units of all ranks over the slowest rank's time.  Returns (units/s, ms)."""
+    ms = max_over_ranks(ms_this_rank, device)
+    units = sum_over_ranks(units_this_rank, device)
+    return units / (ms * 1e-3), ms

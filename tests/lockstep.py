@@ -198,7 +198,8 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
                 assert frac < NEAR_TIE_FRACTION, f"{kind}: near-tie fraction {frac}"
         assert st.attn_mean_abs <= ATTN_MEAN_ABS, f"attention mean abs err {st.attn_mean_abs}"
         assert st.summary_max_rel <= SUMMARY_REL
-        for name, gi in (("grow", 0), ("compress", 1), ("fallback", 2), ("stalled", 3), ("cow_pages", 4)):
+        for name, gi in (("grow", 0), ("compress", 1), ("fallback", 2), ("stalled", 3), ("cow_pages", 4),
+                         ("moved_rows", 8), ("scored_tokens", 9)):
             assert int(st.counters[gi]) == ora.counters[name], f"counter {name}: gpu {st.counters[gi]} oracle {ora.counters[name]}"
     finally:
         gpu.close()
