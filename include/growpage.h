@@ -155,7 +155,8 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
 
 /* ---- measurement ----------------------------------------------------------------------------- */
 
-#define GP_N_KERNELS 5   /* plan, attention, boundary scoring, decision, selection + compaction */
+#define GP_N_KERNELS 6   /* plan, attention, softmax partials, probabilities, working sets + selection +
+                            decision, compaction */
 
 /* With profiling on, every kernel of gp_decode_step is bracketed by CUDA events on the step's
  * stream (this serialises nothing but adds event records).  Off by default. */

@@ -1,28 +1,40 @@
-// Capacity-boundary kernels (Sec. 3.2 - 3.3, App. D.1, App. D.2).
+// Capacity-boundary kernels (Sec. 3.2 - 3.3, App. D.1, App. D.2), launched every step after attention.
+// Work is spread over many CTAs per (request, layer, KV head) unit so that one long request does
+// not set the duration:
 //
-// gp_score_kernel   one CTA per (request at a boundary, layer, KV head):
-//                   Eq. 12 calibration (+ RoPE at the current position), summary-induced attention
-//                   a^S, a^L over the candidate set C (everything but the newest page), and the
-//                   working-set sizes K^S, K^L of Eq. 7.  All in fp64: these values decide integer
-//                   outcomes (set sizes, the retained set, grow or compress), which are compared
-//                   bit for bit with a float64 reference.
-// gp_compact_kernel one CTA per (compressing request, layer, KV head):
-//                   Eq. 9 scores, Eq. 10 block-local + global selection, then the stable in-place
-//                   compaction into (P-1) b slots, writing to copy-on-write targets where the source
-//                   page is shared.  The last CTA to finish swaps in the target pages and drops the
-//                   references to the replaced ones.
+//   gp_bstat_kernel   per (unit, tile of 128 candidate tokens): Eq. 12 calibration (+ RoPE at the current
+//                     position), logits of the two calibrated summaries against the tile's keys, and the
+//                     tile's softmax partials (max, sum of exponentials) per (view, query head).
+//   gp_bprob_kernel   per (unit, tile): merges the partials of the unit into the softmax normalisers,
+//                     recomputes the tile's logits (cheaper than storing them) and writes the
+//                     summary-induced attention a^S, a^L: the group mean of the per-head softmaxes.
+//   gp_bsel_kernel    per unit: working-set sizes K^S, K^L (Eq. 7) and, speculatively, the b slots a
+//                     compression would evict (Eq. 9, Eq. 10).  The last CTA to finish aggregates Eq. 8,
+//                     decides grow or compress per request and runs the device allocator:
+//                     grants first, then copy-on-write targets, each in ascending request id.
+//   gp_compact_kernel per (compressing unit, chunk of 64 source slots): stable in-place compaction into
+//                     (P-1) b slots, writing to copy-on-write targets where the source page is shared.
+//                     Chunks are claimed in order from a ticket counter; a chunk publishes "my sources
+//                     are read" before the next chunk may overwrite their tail.  The last CTA swaps in the
+//                     target pages and drops the references to the replaced ones.
 //
-// Top-p counting and top-k selection are radix descents over the IEEE bit patterns of the
-// (non-negative) scores: 11 bits per level, counts in shared-memory histograms.  The top-p mass is
-// accumulated in 2^62 fixed point with integer atomics, so the result does not depend on the order
-// in which threads add.
+// Everything that decides an integer outcome is fp64.  Top-p counting and top-k selection are radix
+// descents over the IEEE bit patterns of the (non-negative) scores, 11 bits per level, with histograms in
+// shared memory; the top-p mass is accumulated in 2^62 fixed point with integer atomics, so the result
+// does not depend on the order in which threads add.
+#include "../../include/growpage.h"
 #include "gp_dev.cuh"
 
 namespace {
 
-constexpr int BT = 256;              // threads per CTA
 constexpr int NBINS = 2048;
 constexpr double TWO62 = 4611686018427387904.0;
+constexpr int TILE_TOK = GP_SCORE_TILE;   // candidate tokens per scoring tile
+constexpr int ST = 256;              // threads of the scoring kernels
+constexpr int SEL_T = 1024;          // threads of the selection kernel
+constexpr int SEL_CAP = 6144;        // candidate tokens whose scores are staged in shared memory
+constexpr int CT = 256;              // threads of the compaction kernel
+constexpr int MOVE_TOK = GP_MOVE_TOK;     // source slots per compaction chunk
 
 __device__ __forceinline__ unsigned long long to_fix(double a) {
   return (unsigned long long)__double2ll_rn(a * TWO62);
@@ -30,7 +42,8 @@ __device__ __forceinline__ unsigned long long to_fix(double a) {
 
 struct PairCU { unsigned c; unsigned long long s; };
 
-// exclusive suffix sum over the block: result = sum of the values of threads with a higher id
+// exclusive suffix sum over the block: sum of the values of threads with a higher id
+template <int BT>
 __device__ __forceinline__ PairCU block_suffix_excl(unsigned c, unsigned long long s, unsigned* wc,
                                                     unsigned long long* wsum) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -49,6 +62,7 @@ __device__ __forceinline__ PairCU block_suffix_excl(unsigned c, unsigned long lo
   return r;
 }
 // exclusive prefix count over the block
+template <int BT>
 __device__ __forceinline__ unsigned block_prefix_excl(unsigned c, unsigned* wc) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned ic = c;
@@ -68,7 +82,8 @@ __device__ __forceinline__ unsigned block_prefix_excl(unsigned c, unsigned* wc) 
 __device__ __constant__ int kWidths[6] = {11, 11, 11, 11, 11, 8};   // 63 bits below the sign
 
 // Eq. 7: smallest k such that the k largest of a[0..n) sum to at least p.
-__device__ int top_p_count(const double* __restrict__ a, int n, unsigned long long p_fix, unsigned* hcnt,
+template <int BT>
+__device__ int top_p_count(const double* a, int n, unsigned long long p_fix, unsigned* hcnt,
                            unsigned long long* hsum, unsigned* wc, unsigned long long* wsum, long long* s_res) {
   const int tid = threadIdx.x;
   unsigned long long prefix = 0;
@@ -84,7 +99,7 @@ __device__ int top_p_count(const double* __restrict__ a, int n, unsigned long lo
     if (tid == 0) s_res[0] = -1;
     __syncthreads();
     for (int i = tid; i < n; i += BT) {
-      const double v = __ldcg(a + i);
+      const double v = a[i];
       const unsigned long long key = (unsigned long long)__double_as_longlong(v);
       if (lvl == 0 || (key >> (shift + w)) == prefix) {
         const int bin = (int)((key >> shift) & (unsigned long long)(nb - 1));
@@ -97,7 +112,7 @@ __device__ int top_p_count(const double* __restrict__ a, int n, unsigned long lo
     const int lo = tid * per, hi = lo + per;     // this thread's bins [lo, hi)
     unsigned c = 0; unsigned long long s = 0;
     if (lo < nb) for (int b = lo; b < hi; ++b) { c += hcnt[b]; s += hsum[b]; }
-    PairCU ex = block_suffix_excl(c, s, wc, wsum);
+    PairCU ex = block_suffix_excl<BT>(c, s, wc, wsum);
     if (lo < nb) {
       unsigned long long run_s = sum_above + ex.s;
       unsigned run_c = cnt_above + ex.c;
@@ -128,65 +143,113 @@ __device__ int top_p_count(const double* __restrict__ a, int n, unsigned long lo
   return (int)cnt_above + (int)j;
 }
 
+// ------------------------------------------------------------------------------------------------------
+// scoring tiles
+// ------------------------------------------------------------------------------------------------------
 template <int D>
 struct ScoreGeom {
   static constexpr int CH = D / 8;
-  static constexpr int TILE_TOK = 128;
   static constexpr size_t QT_BYTES = 2 * 8 * D * sizeof(double);
   static constexpr size_t KT_BYTES = TILE_TOK * D * 2;
-  static constexpr size_t H_BYTES = NBINS * 4 + NBINS * 8;
-  static constexpr size_t RED_BYTES = (BT + 64) * 8 + 64 * 8;
-  static constexpr size_t SMEM = QT_BYTES + KT_BYTES + H_BYTES + RED_BYTES + 256;
+  static constexpr size_t RED_BYTES = (64 + 16 + 16 + 16) * 8;
+  static constexpr size_t SMEM = QT_BYTES + KT_BYTES + RED_BYTES + 256;
 };
 
+struct TileCtx {
+  int bidx, tile, lh, l, h, bi, r, Pr, nC, nt, t0;
+};
+
+__device__ __forceinline__ TileCtx decode_tile(const GpDev& p, long long item, int NT, const int* req_ids) {
+  TileCtx c;
+  const int t = (int)(item % NT);
+  c.lh = (int)(item / NT);
+  c.l = c.lh / p.Hkv; c.h = c.lh % p.Hkv;
+  const int2 bt = p.bt_list[t];
+  c.bidx = bt.x; c.tile = bt.y;
+  c.bi = p.bnd_list[c.bidx];
+  c.r = req_ids[c.bi];
+  c.Pr = p.P[c.r];
+  c.nC = (c.Pr - 1) * GP_PAGE;
+  c.t0 = p.bnd_tile0[c.bidx];
+  c.nt = (c.nC + TILE_TOK - 1) / TILE_TOK;
+  return c;
+}
+
+// keys of one tile -> shared memory, rows kept in their swizzled order
 template <int D>
-__global__ void __launch_bounds__(BT)
-gp_score_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req,
+__device__ __forceinline__ void load_ktile(const GpDev& p, const TileCtx& c, uint4* ktile) {
+  constexpr int CH = D / 8;
+  const int* table = p.page_table + (size_t)c.r * p.cap;
+  const int tok0 = c.tile * TILE_TOK;
+  for (int i = threadIdx.x; i < TILE_TOK * CH; i += ST) {
+    const int rr = i / CH, pc = i % CH;
+    const int tokn = tok0 + rr;
+    if (tokn < c.nC) {
+      const int page = table[tokn / GP_PAGE];
+      const uint4* src =
+          reinterpret_cast<const uint4*>(p.kv + gp_tile_off(p, c.l, page, c.h)) + (tokn % GP_PAGE) * CH + pc;
+      ktile[i] = __ldg(src);
+    }
+  }
+}
+
+// logits of one token against the G calibrated summaries of one view: z_g = q~_g . k / sqrt(d)
+template <int D>
+__device__ __forceinline__ void token_logits(const double* qt, const uint4* ktile, int rowi, int x, int G,
+                                             double* z) {
+  constexpr int CH = D / 8;
+  double acc[8];
+#pragma unroll
+  for (int g = 0; g < 8; ++g) acc[g] = 0.0;
+  const int sw = rowi & 7;
+#pragma unroll 2
+  for (int c = 0; c < CH; ++c) {
+    const uint4 kk = ktile[rowi * CH + (c ^ sw)];
+    double kd[8];
+    kd[0] = (double)bf16_lo_f(kk.x); kd[1] = (double)bf16_hi_f(kk.x);
+    kd[2] = (double)bf16_lo_f(kk.y); kd[3] = (double)bf16_hi_f(kk.y);
+    kd[4] = (double)bf16_lo_f(kk.z); kd[5] = (double)bf16_hi_f(kk.z);
+    kd[6] = (double)bf16_lo_f(kk.w); kd[7] = (double)bf16_hi_f(kk.w);
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      if (g < G) {
+        const double* qq = qt + (x * 8 + g) * D + c * 8;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[g] = fma(kd[e], qq[e], acc[g]);
+      }
+    }
+  }
+  const double sqrt_d = sqrt((double)D);
+#pragma unroll
+  for (int g = 0; g < 8; ++g) z[g] = acc[g] / sqrt_d;
+}
+
+template <int D>
+__global__ void __launch_bounds__(ST)
+gp_bstat_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req,
                 const __nv_bfloat16* __restrict__ q) {
   using GEO = ScoreGeom<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
   double* qt = reinterpret_cast<double*>(smem);                               // [2][8][D]
   uint4* ktile = reinterpret_cast<uint4*>(smem + GEO::QT_BYTES);              // [128][CH]
-  unsigned* hcnt = reinterpret_cast<unsigned*>(smem + GEO::QT_BYTES + GEO::KT_BYTES);
-  unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + NBINS);
-  double* red = reinterpret_cast<double*>(hsum + NBINS);                      // [BT]
-  double* sM = red + BT;                                                      // [16] maxima
-  double* sZ = sM + 16;                                                       // [16] normalisers
-  unsigned long long* wsum = reinterpret_cast<unsigned long long*>(sZ + 16);  // [8]
-  unsigned* wc = reinterpret_cast<unsigned*>(wsum + 8);                       // [8]
-  long long* s_res = reinterpret_cast<long long*>(wc + 8);                    // [4]
+  double* red = reinterpret_cast<double*>(smem + GEO::QT_BYTES + GEO::KT_BYTES);   // [8 warps][8]
+  double* sM = red + 64;                                                       // [16]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.G, LH = p.L * p.Hkv, G2 = 2 * p.G;
-  const int n_bnd = p.hdr[HDR_N_BND];
-  const long long units = (long long)n_bnd * LH;
-  double* ws = p.score_ws + (size_t)blockIdx.x * ((size_t)p.cap * GP_PAGE) * G2;
-  const double sqrt_d = sqrt((double)D);
+  const int NT = p.hdr[HDR_N_BTILE];
+  const long long items = (long long)NT * LH;
 
-  for (long long u = blockIdx.x; u < units; u += gridDim.x) {
-    const int bidx = (int)(u / LH), lh = (int)(u % LH);
-    const int l = lh / p.Hkv, h = lh % p.Hkv;
-    const int bi = p.bnd_list[bidx];
-    const int r = req_ids[bi];
-    const int Pr = p.P[r];
-    const int nC = (Pr - 1) * GP_PAGE;
-    int* Kout = p.Kx + (((size_t)r * p.L + l) * p.Hkv + h) * 2;
-    if (nC == 0) {
-      if (tid == 0) { Kout[0] = 0; Kout[1] = 0; }
-      continue;
-    }
-    const long long off = p.bnd_off[bi];
-    double* aS = p.scores + ((size_t)lh) * p.max_batch_tokens + off;
-    double* aL = p.scores + ((size_t)LH + lh) * p.max_batch_tokens + off;
-    const int* table = p.page_table + (size_t)r * p.cap;
+  for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+    const TileCtx c = decode_tile(p, item, NT, req_ids);
     __syncthreads();
-
-    // ---- Eq. 12: per-head RMS calibration against this step's query, then RoPE at position t ----
-    for (int vec = warp; vec < G2; vec += BT / 32) {
-      const int x = vec / G, g = vec % G, head = h * G + g;
-      const __nv_bfloat16* qrow = q + (((size_t)l * n_req + bi) * p.Hq + head) * D;
-      const double* srow = p.summ + gp_summ_off(p, l, r, x, head);
+    // ---- Eq. 12: per-head RMS calibration against this step's query, then RoPE at position t -----------
+    double* qglob = p.qtilde + ((size_t)c.bidx * LH + c.lh) * (size_t)(G2 * D);
+    for (int vec = warp; vec < G2; vec += ST / 32) {
+      const int x = vec / G, g = vec % G, head = c.h * G + g;
+      const __nv_bfloat16* qrow = q + (((size_t)c.l * n_req + c.bi) * p.Hq + head) * D;
+      const double* srow = p.summ + gp_summ_off(p, c.l, c.r, x, head);
       double sq = 0.0, ss = 0.0;
       for (int dd = lane; dd < D; dd += 32) {
         const double qv = (double)__bfloat162float(qrow[dd]);
@@ -204,74 +267,33 @@ gp_score_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids
       for (int dd = lane; dd < D; dd += 32) dst[dd] = gamma * srow[dd];
       __syncwarp();
       if (p.rope_theta != 0.0) {
-        const double* cs = p.rope_cs + (size_t)bi * (D / 2) * 2;
+        const double* cs = p.rope_cs + (size_t)c.bi * (D / 2) * 2;
         for (int j = lane; j < D / 2; j += 32) {
-          const double c = cs[2 * j], s = cs[2 * j + 1];
+          const double co = cs[2 * j], si = cs[2 * j + 1];
           const double x1 = dst[j], x2 = dst[j + D / 2];
-          dst[j] = x1 * c - x2 * s;
-          dst[j + D / 2] = x2 * c + x1 * s;
+          dst[j] = x1 * co - x2 * si;
+          dst[j + D / 2] = x2 * co + x1 * si;
         }
+        __syncwarp();
       }
+      if (c.tile == 0)                                    // the probability kernel reads these back
+        for (int dd = lane; dd < D; dd += 32) qglob[(size_t)vec * D + dd] = dst[dd];
     }
+    load_ktile<D>(p, c, ktile);
     __syncthreads();
 
-    // ---- pass 1: logits of every (token of C, view, head of the group) -------------------------------
-    const int x = tid >> 7;                      // view handled by this thread: 0 short, 1 long
-    const int rowi = tid & 127;
-    double mx[8];
+    // ---- logits and the tile's softmax partials ---------------------------------------------------------
+    const int x = tid >> 7, rowi = tid & 127;
+    const int tokn = c.tile * TILE_TOK + rowi;
+    const bool valid = tokn < c.nC;
+    double z[8];
 #pragma unroll
-    for (int g = 0; g < 8; ++g) mx[g] = -INFINITY;
-    for (int t0 = 0; t0 < nC; t0 += GEO::TILE_TOK) {
-      for (int i = tid; i < GEO::TILE_TOK * GEO::CH; i += BT) {
-        const int rr = i / GEO::CH, pc = i % GEO::CH;
-        const int tokn = t0 + rr;
-        if (tokn < nC) {
-          const int page = table[tokn / GP_PAGE];
-          const uint4* src = reinterpret_cast<const uint4*>(p.kv + gp_tile_off(p, l, page, h)) +
-                             (tokn % GP_PAGE) * GEO::CH + pc;
-          ktile[i] = __ldg(src);
-        }
-      }
-      __syncthreads();
-      const int tokn = t0 + rowi;
-      if (tokn < nC) {
-        double acc[8];
-#pragma unroll
-        for (int g = 0; g < 8; ++g) acc[g] = 0.0;
-        const int sw = rowi & 7;
-#pragma unroll 2
-        for (int c = 0; c < GEO::CH; ++c) {
-          const uint4 kk = ktile[rowi * GEO::CH + (c ^ sw)];
-          double kd[8];
-          kd[0] = (double)bf16_lo_f(kk.x); kd[1] = (double)bf16_hi_f(kk.x);
-          kd[2] = (double)bf16_lo_f(kk.y); kd[3] = (double)bf16_hi_f(kk.y);
-          kd[4] = (double)bf16_lo_f(kk.z); kd[5] = (double)bf16_hi_f(kk.z);
-          kd[6] = (double)bf16_lo_f(kk.w); kd[7] = (double)bf16_hi_f(kk.w);
-#pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            if (g < G) {
-              const double* qq = qt + (x * 8 + g) * D + c * 8;
-#pragma unroll
-              for (int e = 0; e < 8; ++e) acc[g] = fma(kd[e], qq[e], acc[g]);
-            }
-          }
-        }
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          if (g < G) {
-            const double z = acc[g] / sqrt_d;
-            ws[(size_t)tokn * G2 + x * G + g] = z;
-            mx[g] = fmax(mx[g], z);
-          }
-        }
-      }
-      __syncthreads();
-    }
-    // maxima per (view, head)
+    for (int g = 0; g < 8; ++g) z[g] = 0.0;
+    if (valid) token_logits<D>(qt, ktile, rowi, x, G, z);
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
       if (g < G) {
-        double m = mx[g];
+        double m = valid ? z[g] : -INFINITY;
 #pragma unroll
         for (int o2 = 16; o2 > 0; o2 >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o2));
         if (lane == 0) red[warp * 8 + g] = m;
@@ -282,117 +304,301 @@ gp_score_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids
       const int xx = tid / G, g = tid % G;
       double m = -INFINITY;
       for (int w = 0; w < 4; ++w) m = fmax(m, red[(xx * 4 + w) * 8 + g]);
-      sM[tid] = m;
+      sM[xx * 8 + g] = m;
     }
     __syncthreads();
-
-    // ---- pass 2: w = exp(z - max), normalisers ---------------------------------------------------------
-    {
-      const int col = tid % G2;
-      const double m = sM[col];
-      double zs = 0.0;
-      const size_t entries = (size_t)nC * G2;
-      for (size_t e2 = tid; e2 < entries; e2 += BT) {
-        const double w = exp(ws[e2] - m);
-        ws[e2] = w;
-        zs += w;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      if (g < G) {
+        double e = valid ? exp(z[g] - sM[x * 8 + g]) : 0.0;
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o2);
+        if (lane == 0) red[warp * 8 + g] = e;
       }
-      red[tid] = zs;
-      __syncthreads();
-      if (tid < G2) {
-        double z = 0.0;
-        for (int k2 = tid; k2 < BT; k2 += G2) z += red[k2];
-        sZ[tid] = z;
-      }
-      __syncthreads();
-    }
-    // ---- pass 3: a^x = mean over the group of the per-head softmaxes ----------------------------------
-    for (int tokn = tid; tokn < nC; tokn += BT) {
-      const double* wr = ws + (size_t)tokn * G2;
-      double s0 = 0.0, s1 = 0.0;
-      for (int g = 0; g < G; ++g) {
-        s0 += wr[g] / sZ[g];
-        s1 += wr[G + g] / sZ[G + g];
-      }
-      aS[tokn] = s0 / (double)G;
-      aL[tokn] = s1 / (double)G;
     }
     __syncthreads();
-    // ---- Eq. 7 -----------------------------------------------------------------------------------------
-    const int KS = top_p_count(aS, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
-    const int KL = top_p_count(aL, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
-    if (tid == 0) { Kout[0] = KS; Kout[1] = KL; }
+    if (tid < G2) {
+      const int xx = tid / G, g = tid % G;
+      double s = 0.0;
+      for (int w = 0; w < 4; ++w) s += red[(xx * 4 + w) * 8 + g];
+      double* st = p.bstats + ((size_t)c.lh * NT + (c.t0 + c.tile)) * 32 + (size_t)tid * 2;
+      st[0] = sM[xx * 8 + g];
+      st[1] = s;
+    }
   }
 }
 
-// =====================================================================================================
 template <int D>
-__global__ void __launch_bounds__(BT)
-gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req) {
-  constexpr int CH = D / 8;
-  constexpr int ROW_BYTES = D * 2;
-  constexpr int MOVE_TOK = 64;                          // source slots per round
-  constexpr int PIECES = MOVE_TOK * 2 * CH / BT;        // 16-byte pieces per thread per round
+__global__ void __launch_bounds__(ST)
+gp_bprob_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req) {
+  using GEO = ScoreGeom<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
-  unsigned* hcnt = reinterpret_cast<unsigned*>(smem);                          // [NBINS]
-  double* stile = reinterpret_cast<double*>(hcnt + NBINS);                     // [BT]
-  unsigned* wc = reinterpret_cast<unsigned*>(stile + BT);                      // [8]
-  int* ev = reinterpret_cast<int*>(wc + 8);                                    // [16] evicted slots
-  int* s_i = ev + 16;                                                          // [8] misc
-  long long* s_res = reinterpret_cast<long long*>(s_i + 8);                    // [4]
-  unsigned* loc = reinterpret_cast<unsigned*>(s_res + 4);                      // [cap*b/32] local-quota bits
+  double* qt = reinterpret_cast<double*>(smem);
+  uint4* ktile = reinterpret_cast<uint4*>(smem + GEO::QT_BYTES);
+  double* red = reinterpret_cast<double*>(smem + GEO::QT_BYTES + GEO::KT_BYTES);
+  double* sM = red + 64;
+  double* sZ = sM + 16;
 
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x;
+  const int G = p.G, LH = p.L * p.Hkv, G2 = 2 * p.G;
+  const int NT = p.hdr[HDR_N_BTILE];
+  const long long items = (long long)NT * LH;
+
+  for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+    const TileCtx c = decode_tile(p, item, NT, req_ids);
+    __syncthreads();
+    if (tid < G2) {                                        // normalisers of the whole candidate set
+      const double* st = p.bstats + ((size_t)c.lh * NT + c.t0) * 32 + (size_t)tid * 2;
+      double M = -INFINITY;
+      for (int t = 0; t < c.nt; ++t) M = fmax(M, st[(size_t)t * 32]);
+      double Z = 0.0;
+      for (int t = 0; t < c.nt; ++t) Z += st[(size_t)t * 32 + 1] * exp(st[(size_t)t * 32] - M);
+      const int xx = tid / G, g = tid % G;
+      sM[xx * 8 + g] = M;
+      sZ[xx * 8 + g] = Z;
+    }
+    const double* qglob = p.qtilde + ((size_t)c.bidx * LH + c.lh) * (size_t)(G2 * D);
+    for (int i = tid; i < G2 * D; i += ST) {
+      const int vec = i / D, dd = i % D;
+      qt[((vec / G) * 8 + (vec % G)) * D + dd] = qglob[i];
+    }
+    load_ktile<D>(p, c, ktile);
+    __syncthreads();
+    const int x = tid >> 7, rowi = tid & 127;
+    const int tokn = c.tile * TILE_TOK + rowi;
+    if (tokn < c.nC) {
+      double z[8];
+      token_logits<D>(qt, ktile, rowi, x, G, z);
+      double s = 0.0;
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+        if (g < G) s += exp(z[g] - sM[x * 8 + g]) / sZ[x * 8 + g];
+      const long long off = p.bnd_off[c.bi];
+      double* dst = p.scores + ((size_t)x * LH + c.lh) * p.max_batch_tokens + off;
+      dst[tokn] = s / (double)G;                           // group mean of the per-head softmaxes
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// decision + allocator, run by the last CTA of the selection kernel
+// ------------------------------------------------------------------------------------------------------
+__device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int* actions, int* s_arr) {
+  int* s_want = s_arr;
+  int* s_ksh = s_arr + GP_MAX_REQ;
+  int* s_P = s_arr + 2 * GP_MAX_REQ;
+  int* s_order = s_arr + 3 * GP_MAX_REQ;
+  int* s_req = s_arr + 4 * GP_MAX_REQ;
+  int* s_base = s_arr + 5 * GP_MAX_REQ;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarp = blockDim.x >> 5;
+  const int n_bnd = p.hdr[HDR_N_BND];
+  for (int i = tid; i < n_req; i += blockDim.x) {
+    if (p.b_flags[i]) {
+      const int r = req_ids[i];
+      p.n[r] = p.b_nold[i] + 1;
+      p.pos[r] += 1;
+      p.started[r] = 1;
+    }
+  }
+  if (tid == 0) {
+    p.counters[5] += 1;
+    p.counters[6] += p.hdr[HDR_N_ACTIVE];
+    p.hdr[HDR_N_CMP] = 0;
+    p.hdr[HDR_N_CITEM] = 0;
+    p.hdr[HDR_WORK_CMP] = 0;
+  }
+  if (n_bnd == 0) return;
+  __syncthreads();
   const int LH = p.L * p.Hkv;
-  const int n_cmp = p.hdr[HDR_N_CMP];
-  const long long units = (long long)n_cmp * LH;
-
-  for (long long u = blockIdx.x; u < units; u += gridDim.x) {
-    const int ci = (int)(u / LH), lh = (int)(u % LH);
-    const int l = lh / p.Hkv, h = lh % p.Hkv;
-    const int bi = p.cmp_list[ci];
+  for (int e = warp; e < n_bnd; e += nwarp) {
+    const int bi = p.bnd_list[e];
     const int r = req_ids[bi];
     const int Pr = p.P[r];
     const int nC = (Pr - 1) * GP_PAGE;
+    long long sS = 0, sL = 0;
+    const int* kx = p.Kx + (size_t)r * LH * 2;
+    for (int j = lane; j < LH; j += 32) { sS += kx[2 * j]; sL += kx[2 * j + 1]; }
+    int ksh = 0;
+    const int* table = p.page_table + (size_t)r * p.cap;
+    for (int j = lane; j < Pr - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) {
+      sS += __shfl_xor_sync(0xffffffffu, sS, o2);
+      sL += __shfl_xor_sync(0xffffffffu, sL, o2);
+      ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
+    }
+    if (lane == 0) {
+      // Eq. 8 with a common |C|: Delta = (sum K^S - sum K^L) / (N |C|), one division of exact integers
+      double delta = 0.0;
+      int want = 1;
+      if (nC > 0) {
+        delta = (double)(sS - sL) / ((double)LH * (double)nC);
+        want = delta > p.tau;
+      }
+      p.delta[r] = delta;
+      s_want[e] = want; s_ksh[e] = ksh; s_P[e] = Pr; s_req[e] = r;
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < n_bnd; e += blockDim.x) {
+    int rank = 0;
+    for (int f = 0; f < n_bnd; ++f) rank += (s_req[f] < s_req[e]);
+    s_order[rank] = e;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int top = *p.free_top;
+    int n_cmp = 0, chunks = 0;
+    long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0;
+    for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants
+      const int e = s_order[k];
+      const int r = s_req[e], Pr = s_P[e], bi = p.bnd_list[e];
+      scored += (long long)(Pr - 1) * GP_PAGE;
+      if ((s_want[e] & 1) && Pr < p.cap && top > 0) {
+        const int page = p.free_stack[--top];
+        p.refcount[page] = 1;
+        p.page_table[(size_t)r * p.cap + Pr] = page;
+        p.P[r] = Pr + 1;
+        actions[bi] = GP_ACT_GROW;
+        s_want[e] |= 2;
+        ++grow;
+      } else if (Pr == 1) {
+        actions[bi] = GP_ACT_STALLED;
+        s_want[e] |= 4;
+        ++stall;
+      }
+    }
+    for (int k = 0; k < n_bnd; ++k) {                    // pass 2: copy-on-write targets
+      const int e = s_order[k];
+      if (s_want[e] & 6) continue;
+      const int r = s_req[e], bi = p.bnd_list[e];
+      if (s_ksh[e] > top) {
+        actions[bi] = GP_ACT_STALLED;
+        ++stall;
+        continue;
+      }
+      s_base[e] = top;
+      top -= s_ksh[e];
+      cow += s_ksh[e];
+      p.cmp_list[n_cmp] = bi;
+      p.cmp_bnd[n_cmp] = e;
+      p.cmp_chunk0[n_cmp] = chunks;
+      chunks += (s_P[e] * GP_PAGE + MOVE_TOK - 1) / MOVE_TOK;
+      ++n_cmp;
+      if (s_want[e] & 1) { actions[bi] = GP_ACT_COMPRESS_FALLBACK; ++fall; } else { actions[bi] = GP_ACT_COMPRESS; ++comp; }
+      p.n[r] = (s_P[e] - 1) * GP_PAGE;
+      p.n_pristine[r] = 0;
+      s_want[e] |= 8;
+    }
+    p.cmp_chunk0[n_cmp] = chunks;
+    if (top < 0) atomicOr(p.err, GP_E_FREELIST);
+    *p.free_top = top;
+    p.hdr[HDR_N_CMP] = n_cmp;
+    p.hdr[HDR_N_CITEM] = chunks * LH;
+    p.counters[0] += grow; p.counters[1] += comp; p.counters[2] += fall; p.counters[3] += stall; p.counters[4] += cow;
+    p.counters[9] += scored;
+  }
+  __syncthreads();
+  for (int e = warp; e < n_bnd; e += nwarp) {             // fill in the targets, in table order
+    if (!(s_want[e] & 8) || s_ksh[e] == 0) continue;
+    const int r = s_req[e], Pr = s_P[e], base = s_base[e];
+    const int* table = p.page_table + (size_t)r * p.cap;
+    int* shadow = p.shadow + (size_t)r * p.cap;
+    int running = 0;
+    for (int j0 = 0; j0 < Pr - 1; j0 += 32) {
+      const int j = j0 + lane;
+      const bool sh = j < Pr - 1 && p.refcount[table[j]] > 1;
+      const unsigned mask = __ballot_sync(0xffffffffu, sh);
+      if (sh) {
+        const int newp = p.free_stack[base - 1 - (running + __popc(mask & ((1u << lane) - 1u)))];
+        shadow[j] = newp;
+        p.refcount[newp] = 1;
+      }
+      running += __popc(mask);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// working sets + speculative eviction list per unit; the last CTA decides
+// ------------------------------------------------------------------------------------------------------
+struct SelGeom {
+  static constexpr size_t SA_BYTES = 2 * SEL_CAP * sizeof(double);
+  static constexpr size_t H_BYTES = NBINS * 4 + NBINS * 8;
+  static constexpr size_t MISC_BYTES = 32 * 8 + 32 * 4 + 8 * 8 + 16 * 4 + 16 * 4;
+};
+
+__global__ void __launch_bounds__(SEL_T)
+gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
+  double* sa = reinterpret_cast<double*>(smem);                                // [2][SEL_CAP]
+  unsigned* hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::SA_BYTES);
+  unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + NBINS);
+  unsigned long long* wsum = hsum + NBINS;                                     // [32]
+  unsigned* wc = reinterpret_cast<unsigned*>(wsum + 32);                       // [32]
+  long long* s_res = reinterpret_cast<long long*>(wc + 32);                    // [8]
+  int* ev = reinterpret_cast<int*>(s_res + 8);                                 // [16]
+  int* s_i = ev + 16;                                                          // [16]
+  unsigned* loc = reinterpret_cast<unsigned*>(s_i + 16);                       // [cap*b/32 + 1]
+  // the decision scratch aliases the score staging area: it is used after the last unit only
+
+  const int tid = threadIdx.x;
+  const int LH = p.L * p.Hkv;
+  const int n_bnd = p.hdr[HDR_N_BND];
+  const long long units = (long long)n_bnd * LH;
+
+  for (long long u = blockIdx.x; u < units; u += gridDim.x) {
+    const int bidx = (int)(u / LH), lh = (int)(u % LH);
+    const int l = lh / p.Hkv, h = lh % p.Hkv;
+    const int bi = p.bnd_list[bidx];
+    const int r = req_ids[bi];
+    const int Pr = p.P[r];
+    const int nC = (Pr - 1) * GP_PAGE;
+    int* Kout = p.Kx + (((size_t)r * p.L + l) * p.Hkv + h) * 2;
+    int* evout = p.evict + (size_t)u * GP_PAGE;
+    __syncthreads();
+    if (nC == 0) {
+      if (tid == 0) { Kout[0] = 0; Kout[1] = 0; }
+      continue;
+    }
+    const long long off = p.bnd_off[bi];
+    const double* gS = p.scores + ((size_t)lh) * p.max_batch_tokens + off;
+    const double* gL = p.scores + ((size_t)LH + lh) * p.max_batch_tokens + off;
+    const double* aS = gS;
+    const double* aL = gL;
+    if (nC <= SEL_CAP) {
+      for (int i = tid; i < nC; i += SEL_T) { sa[i] = __ldcg(gS + i); sa[SEL_CAP + i] = __ldcg(gL + i); }
+      aS = sa; aL = sa + SEL_CAP;
+    }
+    for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
+    if (tid == 0) s_i[0] = 0;
+    __syncthreads();
+    // ---- Eq. 7 ---------------------------------------------------------------------------------------------
+    const int KS = top_p_count<SEL_T>(aS, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
+    const int KL = top_p_count<SEL_T>(aL, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
+    if (tid == 0) { Kout[0] = KS; Kout[1] = KL; }
+
+    // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
     const int nblk = Pr - 1;
     const int K_t = nC - GP_PAGE;
-    const int kq = min(p.k_loc, K_t / nblk);             // k' of Eq. 10
-    const long long off = p.bnd_off[bi];
-    const double* aS = p.scores + ((size_t)lh) * p.max_batch_tokens + off;
-    const double* aL = p.scores + ((size_t)LH + lh) * p.max_batch_tokens + off;
-    const int* table = p.page_table + (size_t)r * p.cap;
-    const int* shadow = p.shadow + (size_t)r * p.cap;
-    __syncthreads();
-
-    // ---- block-local quota: the k' best slots of every page of C (score desc, slot asc) ---------------
-    for (int i = tid; i < (nC + 31) / 32; i += BT) loc[i] = 0;
-    if (tid == 0) { s_i[0] = 0; s_i[1] = 0x7fffffff; s_i[3] = 0; }
-    __syncthreads();
-    for (int t0 = 0; t0 < nC; t0 += BT) {
-      const int tokn = t0 + tid;
-      double s = 0.0;
-      if (tokn < nC) s = fmax(__ldcg(aS + tokn), __ldcg(aL + tokn));     // Eq. 9
-      stile[tid] = s;
-      __syncthreads();
-      if (tokn < nC && kq > 0) {
-        const int b0 = tid & ~15;
+    const int kq = min(p.k_loc, K_t / nblk);
+    if (kq > 0) {
+      for (int i = tid; i < nC; i += SEL_T) {
+        const double s = fmax(aS[i], aL[i]);                           // Eq. 9
+        const int b0 = i & ~15;
         int rank = 0;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const double sj = stile[b0 + j];
-          rank += (sj > s) || (sj == s && (b0 + j) < tid);
+          const double sj = fmax(aS[b0 + j], aL[b0 + j]);
+          rank += (sj > s) || (sj == s && (b0 + j) < i);
         }
-        if (rank < kq) atomicOr(&loc[tokn >> 5], 1u << (tokn & 31));
+        if (rank < kq) atomicOr(&loc[i >> 5], 1u << (i & 31));
       }
-      __syncthreads();
     }
-    // first page whose source is shared (copy-on-write): everything from there on is rewritten
-    for (int j = tid; j < Pr - 1; j += BT)
-      if (shadow[j] >= 0) atomicMin(&s_i[1], j * GP_PAGE);
     __syncthreads();
-
-    // ---- global cut: evict the b lowest of the rest (score asc, slot desc) --------------------------------
+    // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
     unsigned long long prefix = 0;
     unsigned cnt_below = 0;
     unsigned long long thr = 0;        // evict keys strictly below thr ...
@@ -405,23 +611,22 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         const int w = kWidths[lvl];
         shift -= w;
         const int nb = 1 << w;
-        for (int i = tid; i < nb; i += BT) hcnt[i] = 0;
+        for (int i = tid; i < nb; i += SEL_T) hcnt[i] = 0;
         if (tid == 0) s_res[0] = -1;
         __syncthreads();
-        for (int i = tid; i < nC; i += BT) {
+        for (int i = tid; i < nC; i += SEL_T) {
           if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-            const unsigned long long key =
-                (unsigned long long)__double_as_longlong(fmax(__ldcg(aS + i), __ldcg(aL + i)));
+            const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(aS[i], aL[i]));
             if (lvl == 0 || (key >> (shift + w)) == prefix)
               atomicAdd(&hcnt[(int)((key >> shift) & (unsigned long long)(nb - 1))], 1u);
           }
         }
         __syncthreads();
-        const int per = nb / BT > 0 ? nb / BT : 1;
+        const int per = nb / SEL_T > 0 ? nb / SEL_T : 1;
         const int lo = tid * per, hi = lo + per;
         unsigned c = 0;
         if (lo < nb) for (int b = lo; b < hi; ++b) c += hcnt[b];
-        const unsigned ex = block_prefix_excl(c, wc);
+        const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
         if (lo < nb) {
           unsigned run = cnt_below + ex;
           for (int b = lo; b < hi; ++b) {
@@ -451,10 +656,9 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         need_eq = GP_PAGE - (int)cnt_below;
       }
     }
-    // ---- list the evicted slots --------------------------------------------------------------------------
-    for (int i = tid; i < nC; i += BT) {
+    for (int i = tid; i < nC; i += SEL_T) {
       if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-        const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(__ldcg(aS + i), __ldcg(aL + i)));
+        const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(aS[i], aL[i]));
         if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < GP_PAGE) ev[at] = i; }
       }
     }
@@ -463,7 +667,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
       int cntv = s_i[0];
       for (int i = nC - 1; i >= 0 && need_eq > 0; --i) {     // rare: older (lower) slots win ties
         if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-          const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(__ldcg(aS + i), __ldcg(aL + i)));
+          const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(aS[i], aL[i]));
           if (key == tie_key) { if (cntv < GP_PAGE) ev[cntv] = i; ++cntv; --need_eq; }
         }
       }
@@ -474,75 +678,150 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         while (b2 >= 0 && ev[b2] > key) { ev[b2 + 1] = ev[b2]; --b2; }
         ev[b2 + 1] = key;
       }
+      for (int a = 0; a < GP_PAGE; ++a) evout[a] = ev[a];
+    }
+  }
+
+  // ---- the last CTA takes the decisions ----------------------------------------------------------------------
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int prev = atomicAdd(&p.hdr[HDR_DONE_SEL], 1);
+    s_i[2] = (prev == (int)gridDim.x - 1);
+    if (prev == (int)gridDim.x - 1) p.hdr[HDR_DONE_SEL] = 0;
+  }
+  __syncthreads();
+  if (s_i[2]) {
+    __threadfence();
+    decide_and_allocate(p, req_ids, n_req, actions, reinterpret_cast<int*>(sa));
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// compaction
+// ------------------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(CT)
+gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req) {
+  constexpr int CH = D / 8;
+  constexpr int ROW_BYTES = D * 2;
+  constexpr int PIECES = MOVE_TOK * 2 * CH / CT;        // 16-byte pieces per thread per chunk
+  __shared__ int s_pref[GP_MAX_REQ + 1];
+  __shared__ int ev[GP_PAGE];
+  __shared__ int s_i[8];
+
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int LH = p.L * p.Hkv;
+  const int n_cmp = p.hdr[HDR_N_CMP];
+  const int n_items = p.hdr[HDR_N_CITEM];
+  const int stamp = p.hdr[HDR_STEP];
+  for (int i = tid; i <= n_cmp; i += CT) s_pref[i] = p.cmp_chunk0[i];
+  if (tid == 0) s_i[3] = 0;
+  __syncthreads();
+
+  for (;;) {
+    __syncthreads();
+    if (tid == 0) s_i[0] = n_items > 0 ? atomicAdd(&p.hdr[HDR_WORK_CMP], 1) : 0x7fffffff;
+    __syncthreads();
+    const int item = s_i[0];
+    if (item >= n_items) break;
+    // item -> (compressing request, layer/head, chunk); chunks of a unit are consecutive and ascending
+    int lo = 0, hi = n_cmp;
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (LH * s_pref[mid] <= item) lo = mid; else hi = mid; }
+    const int ci = lo;
+    const int nchunk = s_pref[ci + 1] - s_pref[ci];
+    const int rem = item - LH * s_pref[ci];
+    const int lh = rem / nchunk, j = rem % nchunk;
+    const int l = lh / p.Hkv, h = lh % p.Hkv;
+    const int bi = p.cmp_list[ci];
+    const int r = req_ids[bi];
+    const int Pr = p.P[r];
+    const int n_src = Pr * GP_PAGE;
+    const int* table = p.page_table + (size_t)r * p.cap;
+    const int* shadow = p.shadow + (size_t)r * p.cap;
+    if (tid < GP_PAGE) ev[tid] = p.evict[((size_t)p.cmp_bnd[ci] * LH + lh) * GP_PAGE + tid];
+    __syncthreads();
+    const int c0 = j * MOVE_TOK;
+
+    uint4 val[PIECES];
+    int dst_code[PIECES];
+    int tokv = 0, tok_dst = -1;
+#pragma unroll
+    for (int k2 = 0; k2 < PIECES; ++k2) {
+      const int piece = tid + k2 * CT;
+      const int tl = piece / (2 * CH), pc = piece % (2 * CH);
+      const int i = c0 + tl;
+      dst_code[k2] = -1;
+      val[k2] = make_uint4(0, 0, 0, 0);
+      if (i < n_src) {
+        int sh = 0; bool evicted = false;
+#pragma unroll
+        for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < i); evicted |= (ev[e2] == i); }
+        const int pg = i / GP_PAGE;
+        const bool cow = (pg < Pr - 1) && (shadow[pg] >= 0);
+        if (!evicted && (sh > 0 || cow)) {
+          const int isv = pc / CH, cp = pc % CH;
+          const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, l, table[pg], h)) +
+                               isv * GP_PAGE * ROW_BYTES + (i % GP_PAGE) * ROW_BYTES + (cp << 4);
+          val[k2] = *reinterpret_cast<const uint4*>(src);
+          dst_code[k2] = ((i - sh) << 5) | ((cp ^ (i & 7)) << 1) | isv;   // slot, logical chunk, K or V
+        }
+      }
+    }
+    if (tid < MOVE_TOK) {
+      const int i = c0 + tid;
+      if (i < n_src) {
+        int sh = 0; bool evicted = false;
+#pragma unroll
+        for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < i); evicted |= (ev[e2] == i); }
+        const int pg = i / GP_PAGE;
+        const bool cow = (pg < Pr - 1) && (shadow[pg] >= 0);
+        if (!evicted && (sh > 0 || cow)) {
+          tokv = p.tok[gp_tok_off(p, l, table[pg], h) + (i % GP_PAGE)];
+          tok_dst = i - sh;
+        }
+      }
+    }
+    // Touch every loaded value so that the loads have completed before the flag below is published: the
+    // next chunk's CTA may overwrite the tail of this chunk's sources as soon as it sees the flag.
+    unsigned touched = (unsigned)tokv;
+#pragma unroll
+    for (int k2 = 0; k2 < PIECES; ++k2) touched ^= val[k2].x ^ val[k2].y ^ val[k2].z ^ val[k2].w;
+    if (touched == 0x9e3779b9u && c0 < 0) s_i[4] = 1;      // never true; keeps the dependency alive
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      *reinterpret_cast<volatile int*>(p.cflags + item) = stamp;      // "my sources are read"
+      if (j > 0) {                                          // the previous chunk's tail is my first destination
+        volatile int* prev = reinterpret_cast<volatile int*>(p.cflags + item - 1);
+        unsigned it = 0;
+        while (*prev != stamp && it < GP_SPIN_LIMIT) ++it;
+        if (it >= GP_SPIN_LIMIT) atomicOr(p.err, GP_E_SPIN);
+        __threadfence();
+      }
     }
     __syncthreads();
-
-    // ---- stable compaction: survivors of C in slot order, then the protected page ------------------------
-    const int n_src = Pr * GP_PAGE;
-    int start = min(ev[0], s_i[1]);
-    start = (start / MOVE_TOK) * MOVE_TOK;
-    for (int c0 = start; c0 < n_src; c0 += MOVE_TOK) {
-      uint4 val[PIECES];
-      int dst_slot[PIECES];
-      int tokv = 0, tok_dst = -1;
 #pragma unroll
-      for (int k2 = 0; k2 < PIECES; ++k2) {
-        const int piece = tid + k2 * BT;
-        const int tl = piece / (2 * CH), pc = piece % (2 * CH);
-        const int i = c0 + tl;
-        dst_slot[k2] = -1;
-        if (i < n_src) {
-          int sh = 0; bool evicted = false;
-#pragma unroll
-          for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < i); evicted |= (ev[e2] == i); }
-          const int pg = i / GP_PAGE;
-          const bool cow = (pg < Pr - 1) && (shadow[pg] >= 0);
-          if (!evicted && (sh > 0 || cow)) {
-            const int isv = pc / CH, cp = pc % CH;
-            const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, l, table[pg], h)) +
-                                 isv * GP_PAGE * ROW_BYTES + (i % GP_PAGE) * ROW_BYTES + (cp << 4);
-            val[k2] = *reinterpret_cast<const uint4*>(src);
-            // remember the logical chunk in the low bits of the destination code
-            dst_slot[k2] = ((i - sh) << 5) | ((cp ^ (i & 7)) << 1) | isv;
-          }
-        }
-      }
-      if (tid < MOVE_TOK) {
-        const int i = c0 + tid;
-        if (i < n_src) {
-          int sh = 0; bool evicted = false;
-#pragma unroll
-          for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < i); evicted |= (ev[e2] == i); }
-          const int pg = i / GP_PAGE;
-          const bool cow = (pg < Pr - 1) && (shadow[pg] >= 0);
-          if (!evicted && (sh > 0 || cow)) {
-            tokv = p.tok[gp_tok_off(p, l, table[pg], h) + (i % GP_PAGE)];
-            tok_dst = i - sh;
-          }
-        }
-      }
-      __syncthreads();
-#pragma unroll
-      for (int k2 = 0; k2 < PIECES; ++k2) {
-        if (dst_slot[k2] >= 0) {
-          const int ds = dst_slot[k2] >> 5, c = (dst_slot[k2] >> 1) & 15, isv = dst_slot[k2] & 1;
-          const int pg = ds / GP_PAGE;
-          const int page = shadow[pg] >= 0 ? shadow[pg] : table[pg];
-          uint8_t* dst = reinterpret_cast<uint8_t*>(p.kv + gp_tile_off(p, l, page, h)) + isv * GP_PAGE * ROW_BYTES +
-                         (ds % GP_PAGE) * ROW_BYTES + ((c ^ (ds & 7)) << 4);
-          *reinterpret_cast<uint4*>(dst) = val[k2];
-        }
-      }
-      if (tok_dst >= 0) {
-        atomicAdd(&s_i[3], 1);
-        const int pg = tok_dst / GP_PAGE;
+    for (int k2 = 0; k2 < PIECES; ++k2) {
+      if (dst_code[k2] >= 0) {
+        const int ds = dst_code[k2] >> 5, c = (dst_code[k2] >> 1) & 15, isv = dst_code[k2] & 1;
+        const int pg = ds / GP_PAGE;
         const int page = shadow[pg] >= 0 ? shadow[pg] : table[pg];
-        p.tok[gp_tok_off(p, l, page, h) + (tok_dst % GP_PAGE)] = tokv;
+        uint8_t* dst = reinterpret_cast<uint8_t*>(p.kv + gp_tile_off(p, l, page, h)) + isv * GP_PAGE * ROW_BYTES +
+                       (ds % GP_PAGE) * ROW_BYTES + ((c ^ (ds & 7)) << 4);
+        *reinterpret_cast<uint4*>(dst) = val[k2];
       }
-      __syncthreads();
     }
-    if (tid == 0) atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 8), (unsigned long long)s_i[3]);
+    if (tok_dst >= 0) {
+      atomicAdd(&s_i[3], 1);
+      const int pg = tok_dst / GP_PAGE;
+      const int page = shadow[pg] >= 0 ? shadow[pg] : table[pg];
+      p.tok[gp_tok_off(p, l, page, h) + (tok_dst % GP_PAGE)] = tokv;
+    }
   }
+  __syncthreads();
+  if (tid == 0 && s_i[3] > 0)
+    atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 8), (unsigned long long)s_i[3]);
 
   // ---- the last CTA swaps in the copy-on-write targets and drops the old references (App. D.2) ----------
   __threadfence();
@@ -585,32 +864,35 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 
 }  // namespace
 
-void gp_launch_score(const GpDev& p, const int* req_ids, int n_req, const void* q, cudaStream_t s) {
+size_t gp_bsel_smem(const GpDev& p) {
+  return SelGeom::SA_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
+}
+
+void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, const void* q, int* actions, int grid_score,
+                        int grid_sel, int grid_compact, cudaStream_t s, cudaEvent_t* ev) {
   const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
+  const size_t sel_sm = gp_bsel_smem(p);
   if (p.d == 128) {
-    auto kern = gp_score_kernel<128>;
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<128>::SMEM);
-    kern<<<p.score_grid, BT, ScoreGeom<128>::SMEM, s>>>(p, req_ids, n_req, qq);
+    auto k1 = gp_bstat_kernel<128>;
+    auto k2 = gp_bprob_kernel<128>;
+    cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<128>::SMEM);
+    cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<128>::SMEM);
+    k1<<<grid_score, ST, ScoreGeom<128>::SMEM, s>>>(p, req_ids, n_req, qq);
+    if (ev) cudaEventRecord(ev[0], s);
+    k2<<<grid_score, ST, ScoreGeom<128>::SMEM, s>>>(p, req_ids, n_req);
   } else {
-    auto kern = gp_score_kernel<64>;
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<64>::SMEM);
-    kern<<<p.score_grid, BT, ScoreGeom<64>::SMEM, s>>>(p, req_ids, n_req, qq);
+    auto k1 = gp_bstat_kernel<64>;
+    auto k2 = gp_bprob_kernel<64>;
+    cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<64>::SMEM);
+    cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<64>::SMEM);
+    k1<<<grid_score, ST, ScoreGeom<64>::SMEM, s>>>(p, req_ids, n_req, qq);
+    if (ev) cudaEventRecord(ev[0], s);
+    k2<<<grid_score, ST, ScoreGeom<64>::SMEM, s>>>(p, req_ids, n_req);
   }
-}
-
-size_t gp_compact_smem(const GpDev& p) {
-  return NBINS * 4 + BT * 8 + 8 * 4 + 16 * 4 + 8 * 4 + 4 * 8 + ((size_t)p.cap * GP_PAGE / 32 + 1) * 4 + 256 + 64;
-}
-
-void gp_launch_compact(const GpDev& p, const int* req_ids, int n_req, int grid, cudaStream_t s) {
-  const size_t sm = gp_compact_smem(p);
-  if (p.d == 128) {
-    auto kern = gp_compact_kernel<128>;
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    kern<<<grid, BT, sm, s>>>(p, req_ids, n_req);
-  } else {
-    auto kern = gp_compact_kernel<64>;
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    kern<<<grid, BT, sm, s>>>(p, req_ids, n_req);
-  }
+  if (ev) cudaEventRecord(ev[1], s);
+  cudaFuncSetAttribute(gp_bsel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
+  gp_bsel_kernel<<<grid_sel, SEL_T, sel_sm, s>>>(p, req_ids, n_req, actions);
+  if (ev) cudaEventRecord(ev[2], s);
+  if (p.d == 128) gp_compact_kernel<128><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);
+  else gp_compact_kernel<64><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);
 }

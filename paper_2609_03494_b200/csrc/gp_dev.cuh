@@ -20,6 +20,9 @@
 #define GP_ATTN_WARPS 4
 #define GP_ATTN_STAGES 3
 #define GP_SPIN_LIMIT (1u << 24)
+#define GP_MAX_REQ 1024        // upper limit of max_requests (shared-memory arrays are sized by it)
+#define GP_SCORE_TILE 128      // candidate tokens per boundary-scoring tile
+#define GP_MOVE_TOK 64         // source slots per compaction chunk
 
 // plan header slots (int32)
 enum {
@@ -30,6 +33,10 @@ enum {
   HDR_DONE_CMP,      // CTAs of the compaction kernel that have finished
   HDR_STEP,          // step serial number
   HDR_N_ACTIVE,      // requests actually stepped
+  HDR_N_BTILE,       // scoring tiles over all requests at a boundary
+  HDR_DONE_SEL,      // CTAs of the selection kernel that have finished
+  HDR_WORK_CMP,      // ticket counter of the compaction kernel
+  HDR_N_CITEM,       // compaction work items (chunks x layers x heads)
   HDR_COUNT = 16
 };
 
@@ -42,7 +49,7 @@ enum {
 
 struct GpDev {
   // geometry
-  int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc, score_grid;
+  int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc, max_btiles;
   long long n_pages, max_batch_tokens;
   double beta_s, beta_l, top_p, tau, rope_theta;
   unsigned long long p_fix;              // top_p in 2^62 fixed point
@@ -69,10 +76,17 @@ struct GpDev {
   int* bnd_list;                         // [M] batch indices at a boundary
   long long* bnd_off;                    // [M] token offset into the score scratch
   int* cmp_list;                         // [M] batch indices that compress
+  int* cmp_bnd;                          // [M] their index in bnd_list
+  int* cmp_chunk0;                       // [M+1] prefix of their compaction chunk counts
+  int2* bt_list;                         // [max_btiles] {index in bnd_list, tile} of every scoring tile
+  int* bnd_tile0;                        // [M] first scoring tile of a boundary request
+  double* bstats;                        // [L*H_kv][max_btiles][2G][2] softmax partials (max, sum)
+  double* qtilde;                        // [M][L*H_kv][2G][d] calibrated (and rotated) summaries
+  int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
+  int* cflags;                           // compaction chunk flags, stamped with the step number
   double* rope_cs;                       // [M][d/2][2] cos, sin at the step's position
   float* partials;
   double* scores;
-  double* score_ws;                      // [score_grid][cap*b][2G] logits workspace
   long long* counters;                   // [8]
   int* err;
 };
@@ -158,6 +172,7 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
                          float* out, int grid, cudaStream_t s);
 size_t gp_attention_smem(int d);
 int gp_attention_ctas_per_sm(int d);
-void gp_launch_score(const GpDev& p, const int* req_ids, int n_req, const void* q, cudaStream_t s);
-void gp_launch_compact(const GpDev& p, const int* req_ids, int n_req, int grid, cudaStream_t s);
-size_t gp_compact_smem(const GpDev& p);
+// boundary chain: partial softmax stats, probabilities, working sets + selection + decision, compaction.
+// `ev`, when not null, receives three events recorded between the four kernels.
+void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, const void* q, int* actions, int grid_score,
+                        int grid_sel, int grid_compact, cudaStream_t s, cudaEvent_t* ev);

@@ -11,8 +11,8 @@
 #include "../../include/growpage.h"
 #include "gp_dev.cuh"
 
-#define GP_MAX_REQ 1024
-#define GP_SCORE_GRID 296       // 2 CTAs per SM on 148 SMs
+#define GP_SCORE_GRID 592       // 4 CTAs per SM on 148 SMs
+#define GP_SEL_GRID 148         // one 1024-thread CTA per SM
 #define GP_COMPACT_GRID 592     // 4 CTAs per SM
 #define GP_PLAN_THREADS 1024
 
@@ -41,9 +41,10 @@ namespace {
 
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
-      b_flags, first_idx, unit_cnt, bnd_list, bnd_off, cmp_list, rope_cs, partials, scores, score_ws, counters, dbg,
+      b_flags, first_idx, unit_cnt, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, bt_list, bnd_tile0, bstats, qtilde,
+      evict, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
-  int max_rc;
+  int max_rc, max_btiles;
   long long max_batch_tokens;
 };
 
@@ -106,10 +107,18 @@ Layout make_layout(const gp_config& c) {
   L.bnd_list = take(M * 4);
   L.bnd_off = take(M * 8);
   L.cmp_list = take(M * 4);
+  L.cmp_bnd = take(M * 4);
+  L.cmp_chunk0 = take((M + 1) * 4);
+  L.max_btiles = (int)((size_t)L.max_batch_tokens / GP_SCORE_TILE + M + 1);
+  L.bt_list = take((size_t)L.max_btiles * 8);
+  L.bnd_tile0 = take(M * 4);
+  L.bstats = take(LH * (size_t)L.max_btiles * 32 * 8);
+  L.qtilde = take(M * LH * 2 * G * d * 8);
+  L.evict = take(M * LH * b * 4);
+  L.cflags = take(LH * ((size_t)L.max_batch_tokens / GP_MOVE_TOK + 2 * M + 1) * 4);
   L.rope_cs = take(M * (d / 2) * 2 * 8);
   L.partials = take((size_t)L.max_rc * LH * G * (d + 2) * 4);
   L.scores = take(2 * LH * (size_t)L.max_batch_tokens * 8);
-  L.score_ws = take((size_t)GP_SCORE_GRID * cap * b * 2 * G * 8);
   L.counters = take(16 * 8);
   L.dbg = take(cap * b * (4 + 2 * d * 2));
   if (c.host_staging) {
@@ -205,7 +214,10 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     chunks = 0; isb = 0; act = GP_ACT_SCRATCH;
   }
   int bnd_idx, n_bnd; long long dummy0, dummy1;
-  plan_scan(isb, 0, bnd_idx, dummy0, n_bnd, dummy1, sv, sw);
+  const int my_tiles = isb ? (int)((nc + GP_SCORE_TILE - 1) / GP_SCORE_TILE) : 0;
+  long long tile_off, n_btile;
+  plan_scan(isb, my_tiles, bnd_idx, tile_off, n_bnd, n_btile, sv, sw);
+  if (n_btile > p.max_btiles) { atomicOr(p.err, GP_E_BOUNDS); n_btile = 0; n_bnd = 0; isb = 0; }
   int act_idx, n_active;
   plan_scan(chunks > 0, 0, act_idx, dummy0, n_active, dummy1, sv, sw);
   if (in) {
@@ -216,7 +228,12 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       const int pg0 = c * p.chunk_pages;
       p.rc[rc_off + c] = make_int4(i, pg0, min(p.chunk_pages, pages - pg0), c | (chunks << 16));
     }
-    if (isb) { p.bnd_list[bnd_idx] = i; p.bnd_off[i] = tok_off; }
+    if (isb) {
+      p.bnd_list[bnd_idx] = i;
+      p.bnd_off[i] = tok_off;
+      p.bnd_tile0[bnd_idx] = (int)tile_off;
+      for (int t = 0; t < my_tiles; ++t) p.bt_list[tile_off + t] = make_int2(bnd_idx, t);
+    }
     if (r >= 0 && r < p.M) p.first_idx[r] = 0x7fffffff;          // ready for the next step
   }
   if (p.rope_theta != 0.0) {                                      // cos / sin of the step's position
@@ -237,133 +254,11 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   if (threadIdx.x == 0) {
     p.hdr[HDR_N_RC] = n_rc;
     p.hdr[HDR_N_BND] = n_bnd;
+    p.hdr[HDR_N_BTILE] = (int)n_btile;
     p.hdr[HDR_N_CMP] = 0;
     p.hdr[HDR_WORK_ATTN] = 0;
     p.hdr[HDR_N_ACTIVE] = n_active;
     p.hdr[HDR_STEP] += 1;
-  }
-}
-
-// After attention: advances n / pos of every stepped request, then for the requests at a boundary
-// aggregates Eq. 8, takes the grow-or-compress decision, and runs the device allocator:
-// grants first, then copy-on-write targets, each in ascending request id (Sec. 4.2, App. D.2).
-__global__ void __launch_bounds__(256)
-gp_decide_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
-  __shared__ int s_want[GP_MAX_REQ], s_ksh[GP_MAX_REQ], s_P[GP_MAX_REQ], s_order[GP_MAX_REQ], s_req[GP_MAX_REQ];
-  __shared__ int s_base[GP_MAX_REQ];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_bnd = p.hdr[HDR_N_BND];
-  for (int i = tid; i < n_req; i += 256) {
-    if (p.b_flags[i]) {
-      const int r = req_ids[i];
-      p.n[r] = p.b_nold[i] + 1;
-      p.pos[r] += 1;
-      p.started[r] = 1;
-    }
-  }
-  if (tid == 0) { p.counters[5] += 1; p.counters[6] += p.hdr[HDR_N_ACTIVE]; }
-  if (n_bnd == 0) return;
-  const int LH = p.L * p.Hkv;
-  for (int e = warp; e < n_bnd; e += 8) {
-    const int bi = p.bnd_list[e];
-    const int r = req_ids[bi];
-    const int Pr = p.P[r];
-    const int nC = (Pr - 1) * GP_PAGE;
-    long long sS = 0, sL = 0;
-    const int* kx = p.Kx + (size_t)r * LH * 2;
-    for (int j = lane; j < LH; j += 32) { sS += kx[2 * j]; sL += kx[2 * j + 1]; }
-    int ksh = 0;
-    const int* table = p.page_table + (size_t)r * p.cap;
-    for (int j = lane; j < Pr - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
-#pragma unroll
-    for (int o2 = 16; o2 > 0; o2 >>= 1) {
-      sS += __shfl_xor_sync(0xffffffffu, sS, o2);
-      sL += __shfl_xor_sync(0xffffffffu, sL, o2);
-      ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
-    }
-    if (lane == 0) {
-      // Eq. 8 with a common |C|: Delta = (sum K^S - sum K^L) / (N |C|), one division of exact integers
-      double delta = 0.0;
-      int want = 1;
-      if (nC > 0) {
-        delta = (double)(sS - sL) / ((double)LH * (double)nC);
-        want = delta > p.tau;
-      }
-      p.delta[r] = delta;
-      s_want[e] = want; s_ksh[e] = ksh; s_P[e] = Pr; s_req[e] = r;
-    }
-  }
-  __syncthreads();
-  for (int e = tid; e < n_bnd; e += 256) {
-    int rank = 0;
-    for (int f = 0; f < n_bnd; ++f) rank += (s_req[f] < s_req[e]);
-    s_order[rank] = e;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int top = *p.free_top;
-    int n_cmp = 0;
-    long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0;
-    for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants
-      const int e = s_order[k];
-      const int r = s_req[e], Pr = s_P[e], bi = p.bnd_list[e];
-      scored += (long long)(Pr - 1) * GP_PAGE;
-      if ((s_want[e] & 1) && Pr < p.cap && top > 0) {
-        const int page = p.free_stack[--top];
-        p.refcount[page] = 1;
-        p.page_table[(size_t)r * p.cap + Pr] = page;
-        p.P[r] = Pr + 1;
-        actions[bi] = GP_ACT_GROW;
-        s_want[e] |= 2;
-        ++grow;
-      } else if (Pr == 1) {
-        actions[bi] = GP_ACT_STALLED;
-        s_want[e] |= 4;
-        ++stall;
-      }
-    }
-    for (int k = 0; k < n_bnd; ++k) {                    // pass 2: copy-on-write targets
-      const int e = s_order[k];
-      if (s_want[e] & 6) continue;
-      const int r = s_req[e], bi = p.bnd_list[e];
-      if (s_ksh[e] > top) {
-        actions[bi] = GP_ACT_STALLED;
-        ++stall;
-        continue;
-      }
-      s_base[e] = top;
-      top -= s_ksh[e];
-      cow += s_ksh[e];
-      p.cmp_list[n_cmp++] = bi;
-      if (s_want[e] & 1) { actions[bi] = GP_ACT_COMPRESS_FALLBACK; ++fall; } else { actions[bi] = GP_ACT_COMPRESS; ++comp; }
-      p.n[r] = (s_P[e] - 1) * GP_PAGE;
-      p.n_pristine[r] = 0;
-      s_want[e] |= 8;
-    }
-    if (top < 0) atomicOr(p.err, GP_E_FREELIST);
-    *p.free_top = top;
-    p.hdr[HDR_N_CMP] = n_cmp;
-    p.counters[0] += grow; p.counters[1] += comp; p.counters[2] += fall; p.counters[3] += stall; p.counters[4] += cow;
-    p.counters[9] += scored;
-  }
-  __syncthreads();
-  for (int e = warp; e < n_bnd; e += 8) {                 // fill in the targets, in table order
-    if (!(s_want[e] & 8) || s_ksh[e] == 0) continue;
-    const int r = s_req[e], Pr = s_P[e], base = s_base[e];
-    const int* table = p.page_table + (size_t)r * p.cap;
-    int* shadow = p.shadow + (size_t)r * p.cap;
-    int running = 0;
-    for (int j0 = 0; j0 < Pr - 1; j0 += 32) {
-      const int j = j0 + lane;
-      const bool sh = j < Pr - 1 && p.refcount[table[j]] > 1;
-      const unsigned mask = __ballot_sync(0xffffffffu, sh);
-      if (sh) {
-        const int newp = p.free_stack[base - 1 - (running + __popc(mask & ((1u << lane) - 1u)))];
-        shadow[j] = newp;
-        p.refcount[newp] = 1;
-      }
-      running += __popc(mask);
-    }
   }
 }
 
@@ -531,7 +426,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   GpDev& d = pool->dev;
   d.L = cfg->n_layers; d.Hq = cfg->n_q_heads; d.Hkv = cfg->n_kv_heads; d.G = cfg->n_q_heads / cfg->n_kv_heads;
   d.d = cfg->head_dim; d.M = cfg->max_requests; d.cap = cfg->max_pages_per_req; d.k_loc = cfg->k_loc;
-  d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc; d.score_grid = GP_SCORE_GRID;
+  d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc; d.max_btiles = L.max_btiles;
   d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
   d.p_fix = (unsigned long long)llrint(cfg->top_p * 4611686018427387904.0);
@@ -561,10 +456,17 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.bnd_list = reinterpret_cast<int*>(base + L.bnd_list);
   d.bnd_off = reinterpret_cast<long long*>(base + L.bnd_off);
   d.cmp_list = reinterpret_cast<int*>(base + L.cmp_list);
+  d.cmp_bnd = reinterpret_cast<int*>(base + L.cmp_bnd);
+  d.cmp_chunk0 = reinterpret_cast<int*>(base + L.cmp_chunk0);
+  d.bt_list = reinterpret_cast<int2*>(base + L.bt_list);
+  d.bnd_tile0 = reinterpret_cast<int*>(base + L.bnd_tile0);
+  d.bstats = reinterpret_cast<double*>(base + L.bstats);
+  d.qtilde = reinterpret_cast<double*>(base + L.qtilde);
+  d.evict = reinterpret_cast<int*>(base + L.evict);
+  d.cflags = reinterpret_cast<int*>(base + L.cflags);
   d.rope_cs = reinterpret_cast<double*>(base + L.rope_cs);
   d.partials = reinterpret_cast<float*>(base + L.partials);
   d.scores = reinterpret_cast<double*>(base + L.scores);
-  d.score_ws = reinterpret_cast<double*>(base + L.score_ws);
   d.counters = reinterpret_cast<long long*>(base + L.counters);
   pool->dbg = base + L.dbg;
   if (cfg->host_staging) {
@@ -648,12 +550,9 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   if (prof) cudaEventRecord(pool->ev[1], s);
   gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s);
   if (prof) cudaEventRecord(pool->ev[2], s);
-  gp_launch_score(d, dev_req_ids, n_req, q, s);
-  if (prof) cudaEventRecord(pool->ev[3], s);
-  gp_decide_kernel<<<1, 256, 0, s>>>(d, dev_req_ids, n_req, dev_actions);
-  if (prof) cudaEventRecord(pool->ev[4], s);
-  gp_launch_compact(d, dev_req_ids, n_req, GP_COMPACT_GRID, s);
-  if (prof) cudaEventRecord(pool->ev[5], s);
+  gp_launch_boundary(d, dev_req_ids, n_req, q, dev_actions, GP_SCORE_GRID, GP_SEL_GRID, GP_COMPACT_GRID, s,
+                     prof ? &pool->ev[3] : nullptr);
+  if (prof) cudaEventRecord(pool->ev[6], s);
   pool->launch_count += GP_N_KERNELS;
   GP_CUDA(cudaGetLastError());
   if (prof) {
