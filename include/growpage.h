@@ -155,8 +155,7 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
 
 /* ---- measurement ----------------------------------------------------------------------------- */
 
-#define GP_N_KERNELS 6   /* plan, attention, softmax partials, probabilities, working sets + selection +
-                            decision, compaction */
+#define GP_N_KERNELS 4   /* plan, attention (+ boundary logits), selection + decision, compaction */
 
 /* With profiling on, every kernel of gp_decode_step is bracketed by CUDA events on the step's
  * stream (this serialises nothing but adds event records).  Off by default. */

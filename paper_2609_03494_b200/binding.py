@@ -16,8 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libgrowpage.so")
 GP_OK, GP_ERR_INVALID, GP_ERR_NO_SLOT, GP_ERR_NO_PAGES, GP_ERR_CUDA, GP_ERR_STATE = 0, -1, -2, -3, -4, -5
 GP_ACT_NONE, GP_ACT_GROW, GP_ACT_COMPRESS, GP_ACT_COMPRESS_FALLBACK = 0, 1, 2, 3
 GP_ACT_STALLED, GP_ACT_SCRATCH, GP_ACT_INVALID = -1, -2, -3
-GP_N_KERNELS = 6
-KERNEL_NAMES = ("plan", "attention", "bstat", "bprob", "bsel_decide", "compact")
+GP_N_KERNELS = 4
+KERNEL_NAMES = ("plan", "attention", "select_decide", "compact")
 
 
 class gp_config(C.Structure):

@@ -1,17 +1,12 @@
 // Capacity-boundary kernels (Sec. 3.2 - 3.3, App. D.1, App. D.2), launched every step after attention.
-// Work is spread over many CTAs per (request, layer, KV head) unit so that one long request does
-// not set the duration:
+// The attention kernel has already left, for every (request at a boundary, layer, KV head) unit, the
+// fp64 logits z of the two calibrated summaries against every candidate key.
 //
-//   gp_bstat_kernel   per (unit, tile of 128 candidate tokens): Eq. 12 calibration (+ RoPE at the current
-//                     position), logits of the two calibrated summaries against the tile's keys, and the
-//                     tile's softmax partials (max, sum of exponentials) per (view, query head).
-//   gp_bprob_kernel   per (unit, tile): merges the partials of the unit into the softmax normalisers,
-//                     recomputes the tile's logits (cheaper than storing them) and writes the
-//                     summary-induced attention a^S, a^L: the group mean of the per-head softmaxes.
-//   gp_bsel_kernel    per unit: working-set sizes K^S, K^L (Eq. 7) and, speculatively, the b slots a
-//                     compression would evict (Eq. 9, Eq. 10).  The last CTA to finish aggregates Eq. 8,
-//                     decides grow or compress per request and runs the device allocator:
-//                     grants first, then copy-on-write targets, each in ascending request id.
+//   gp_bsel_kernel    per unit: per-head softmax over the candidate set and group mean -> a^S, a^L;
+//                     working-set sizes K^S, K^L (Eq. 7); and, speculatively, the b slots a compression
+//                     would evict (Eq. 9, Eq. 10).  The last CTA to finish aggregates Eq. 8, decides grow
+//                     or compress per request and runs the device allocator: grants first, then
+//                     copy-on-write targets, each in ascending request id.
 //   gp_compact_kernel per (compressing unit, chunk of 64 source slots): stable in-place compaction into
 //                     (P-1) b slots, writing to copy-on-write targets where the source page is shared.
 //                     Chunks are claimed in order from a ticket counter; a chunk publishes "my sources
@@ -29,8 +24,6 @@ namespace {
 
 constexpr int NBINS = 2048;
 constexpr double TWO62 = 4611686018427387904.0;
-constexpr int TILE_TOK = GP_SCORE_TILE;   // candidate tokens per scoring tile
-constexpr int ST = 256;              // threads of the scoring kernels
 constexpr int SEL_T = 1024;          // threads of the selection kernel
 constexpr int SEL_CAP = 6144;        // candidate tokens whose scores are staged in shared memory
 constexpr int CT = 256;              // threads of the compaction kernel
@@ -144,244 +137,6 @@ __device__ int top_p_count(const double* a, int n, unsigned long long p_fix, uns
 }
 
 // ------------------------------------------------------------------------------------------------------
-// scoring tiles
-// ------------------------------------------------------------------------------------------------------
-template <int D>
-struct ScoreGeom {
-  static constexpr int CH = D / 8;
-  static constexpr size_t QT_BYTES = 2 * 8 * D * sizeof(double);
-  static constexpr size_t KT_BYTES = TILE_TOK * D * 2;
-  static constexpr size_t RED_BYTES = (64 + 16 + 16 + 16) * 8;
-  static constexpr size_t SMEM = QT_BYTES + KT_BYTES + RED_BYTES + 256;
-};
-
-struct TileCtx {
-  int bidx, tile, lh, l, h, bi, r, Pr, nC, nt, t0;
-};
-
-__device__ __forceinline__ TileCtx decode_tile(const GpDev& p, long long item, int NT, const int* req_ids) {
-  TileCtx c;
-  const int t = (int)(item % NT);
-  c.lh = (int)(item / NT);
-  c.l = c.lh / p.Hkv; c.h = c.lh % p.Hkv;
-  const int2 bt = p.bt_list[t];
-  c.bidx = bt.x; c.tile = bt.y;
-  c.bi = p.bnd_list[c.bidx];
-  c.r = req_ids[c.bi];
-  c.Pr = p.P[c.r];
-  c.nC = (c.Pr - 1) * GP_PAGE;
-  c.t0 = p.bnd_tile0[c.bidx];
-  c.nt = (c.nC + TILE_TOK - 1) / TILE_TOK;
-  return c;
-}
-
-// keys of one tile -> shared memory, rows kept in their swizzled order
-template <int D>
-__device__ __forceinline__ void load_ktile(const GpDev& p, const TileCtx& c, uint4* ktile) {
-  constexpr int CH = D / 8;
-  const int* table = p.page_table + (size_t)c.r * p.cap;
-  const int tok0 = c.tile * TILE_TOK;
-  for (int i = threadIdx.x; i < TILE_TOK * CH; i += ST) {
-    const int rr = i / CH, pc = i % CH;
-    const int tokn = tok0 + rr;
-    if (tokn < c.nC) {
-      const int page = table[tokn / GP_PAGE];
-      const uint4* src =
-          reinterpret_cast<const uint4*>(p.kv + gp_tile_off(p, c.l, page, c.h)) + (tokn % GP_PAGE) * CH + pc;
-      ktile[i] = __ldg(src);
-    }
-  }
-}
-
-// logits of one token against the G calibrated summaries of one view: z_g = q~_g . k / sqrt(d)
-template <int D>
-__device__ __forceinline__ void token_logits(const double* qt, const uint4* ktile, int rowi, int x, int G,
-                                             double* z) {
-  constexpr int CH = D / 8;
-  double acc[8];
-#pragma unroll
-  for (int g = 0; g < 8; ++g) acc[g] = 0.0;
-  const int sw = rowi & 7;
-#pragma unroll 2
-  for (int c = 0; c < CH; ++c) {
-    const uint4 kk = ktile[rowi * CH + (c ^ sw)];
-    double kd[8];
-    kd[0] = (double)bf16_lo_f(kk.x); kd[1] = (double)bf16_hi_f(kk.x);
-    kd[2] = (double)bf16_lo_f(kk.y); kd[3] = (double)bf16_hi_f(kk.y);
-    kd[4] = (double)bf16_lo_f(kk.z); kd[5] = (double)bf16_hi_f(kk.z);
-    kd[6] = (double)bf16_lo_f(kk.w); kd[7] = (double)bf16_hi_f(kk.w);
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      if (g < G) {
-        const double* qq = qt + (x * 8 + g) * D + c * 8;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[g] = fma(kd[e], qq[e], acc[g]);
-      }
-    }
-  }
-  const double sqrt_d = sqrt((double)D);
-#pragma unroll
-  for (int g = 0; g < 8; ++g) z[g] = acc[g] / sqrt_d;
-}
-
-template <int D>
-__global__ void __launch_bounds__(ST)
-gp_bstat_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req,
-                const __nv_bfloat16* __restrict__ q) {
-  using GEO = ScoreGeom<D>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
-  double* qt = reinterpret_cast<double*>(smem);                               // [2][8][D]
-  uint4* ktile = reinterpret_cast<uint4*>(smem + GEO::QT_BYTES);              // [128][CH]
-  double* red = reinterpret_cast<double*>(smem + GEO::QT_BYTES + GEO::KT_BYTES);   // [8 warps][8]
-  double* sM = red + 64;                                                       // [16]
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int G = p.G, LH = p.L * p.Hkv, G2 = 2 * p.G;
-  const int NT = p.hdr[HDR_N_BTILE];
-  const long long items = (long long)NT * LH;
-
-  for (long long item = blockIdx.x; item < items; item += gridDim.x) {
-    const TileCtx c = decode_tile(p, item, NT, req_ids);
-    __syncthreads();
-    // ---- Eq. 12: per-head RMS calibration against this step's query, then RoPE at position t -----------
-    double* qglob = p.qtilde + ((size_t)c.bidx * LH + c.lh) * (size_t)(G2 * D);
-    for (int vec = warp; vec < G2; vec += ST / 32) {
-      const int x = vec / G, g = vec % G, head = c.h * G + g;
-      const __nv_bfloat16* qrow = q + (((size_t)c.l * n_req + c.bi) * p.Hq + head) * D;
-      const double* srow = p.summ + gp_summ_off(p, c.l, c.r, x, head);
-      double sq = 0.0, ss = 0.0;
-      for (int dd = lane; dd < D; dd += 32) {
-        const double qv = (double)__bfloat162float(qrow[dd]);
-        const double sv = srow[dd];
-        sq += qv * qv;
-        ss += sv * sv;
-      }
-#pragma unroll
-      for (int o2 = 16; o2 > 0; o2 >>= 1) {
-        sq += __shfl_xor_sync(0xffffffffu, sq, o2);
-        ss += __shfl_xor_sync(0xffffffffu, ss, o2);
-      }
-      const double gamma = ss > 0.0 ? sqrt(sq / (double)D) / sqrt(ss / (double)D) : 1.0;
-      double* dst = qt + (x * 8 + g) * D;
-      for (int dd = lane; dd < D; dd += 32) dst[dd] = gamma * srow[dd];
-      __syncwarp();
-      if (p.rope_theta != 0.0) {
-        const double* cs = p.rope_cs + (size_t)c.bi * (D / 2) * 2;
-        for (int j = lane; j < D / 2; j += 32) {
-          const double co = cs[2 * j], si = cs[2 * j + 1];
-          const double x1 = dst[j], x2 = dst[j + D / 2];
-          dst[j] = x1 * co - x2 * si;
-          dst[j + D / 2] = x2 * co + x1 * si;
-        }
-        __syncwarp();
-      }
-      if (c.tile == 0)                                    // the probability kernel reads these back
-        for (int dd = lane; dd < D; dd += 32) qglob[(size_t)vec * D + dd] = dst[dd];
-    }
-    load_ktile<D>(p, c, ktile);
-    __syncthreads();
-
-    // ---- logits and the tile's softmax partials ---------------------------------------------------------
-    const int x = tid >> 7, rowi = tid & 127;
-    const int tokn = c.tile * TILE_TOK + rowi;
-    const bool valid = tokn < c.nC;
-    double z[8];
-#pragma unroll
-    for (int g = 0; g < 8; ++g) z[g] = 0.0;
-    if (valid) token_logits<D>(qt, ktile, rowi, x, G, z);
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      if (g < G) {
-        double m = valid ? z[g] : -INFINITY;
-#pragma unroll
-        for (int o2 = 16; o2 > 0; o2 >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o2));
-        if (lane == 0) red[warp * 8 + g] = m;
-      }
-    }
-    __syncthreads();
-    if (tid < G2) {
-      const int xx = tid / G, g = tid % G;
-      double m = -INFINITY;
-      for (int w = 0; w < 4; ++w) m = fmax(m, red[(xx * 4 + w) * 8 + g]);
-      sM[xx * 8 + g] = m;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      if (g < G) {
-        double e = valid ? exp(z[g] - sM[x * 8 + g]) : 0.0;
-#pragma unroll
-        for (int o2 = 16; o2 > 0; o2 >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o2);
-        if (lane == 0) red[warp * 8 + g] = e;
-      }
-    }
-    __syncthreads();
-    if (tid < G2) {
-      const int xx = tid / G, g = tid % G;
-      double s = 0.0;
-      for (int w = 0; w < 4; ++w) s += red[(xx * 4 + w) * 8 + g];
-      double* st = p.bstats + ((size_t)c.lh * NT + (c.t0 + c.tile)) * 32 + (size_t)tid * 2;
-      st[0] = sM[xx * 8 + g];
-      st[1] = s;
-    }
-  }
-}
-
-template <int D>
-__global__ void __launch_bounds__(ST)
-gp_bprob_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req) {
-  using GEO = ScoreGeom<D>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
-  double* qt = reinterpret_cast<double*>(smem);
-  uint4* ktile = reinterpret_cast<uint4*>(smem + GEO::QT_BYTES);
-  double* red = reinterpret_cast<double*>(smem + GEO::QT_BYTES + GEO::KT_BYTES);
-  double* sM = red + 64;
-  double* sZ = sM + 16;
-
-  const int tid = threadIdx.x;
-  const int G = p.G, LH = p.L * p.Hkv, G2 = 2 * p.G;
-  const int NT = p.hdr[HDR_N_BTILE];
-  const long long items = (long long)NT * LH;
-
-  for (long long item = blockIdx.x; item < items; item += gridDim.x) {
-    const TileCtx c = decode_tile(p, item, NT, req_ids);
-    __syncthreads();
-    if (tid < G2) {                                        // normalisers of the whole candidate set
-      const double* st = p.bstats + ((size_t)c.lh * NT + c.t0) * 32 + (size_t)tid * 2;
-      double M = -INFINITY;
-      for (int t = 0; t < c.nt; ++t) M = fmax(M, st[(size_t)t * 32]);
-      double Z = 0.0;
-      for (int t = 0; t < c.nt; ++t) Z += st[(size_t)t * 32 + 1] * exp(st[(size_t)t * 32] - M);
-      const int xx = tid / G, g = tid % G;
-      sM[xx * 8 + g] = M;
-      sZ[xx * 8 + g] = Z;
-    }
-    const double* qglob = p.qtilde + ((size_t)c.bidx * LH + c.lh) * (size_t)(G2 * D);
-    for (int i = tid; i < G2 * D; i += ST) {
-      const int vec = i / D, dd = i % D;
-      qt[((vec / G) * 8 + (vec % G)) * D + dd] = qglob[i];
-    }
-    load_ktile<D>(p, c, ktile);
-    __syncthreads();
-    const int x = tid >> 7, rowi = tid & 127;
-    const int tokn = c.tile * TILE_TOK + rowi;
-    if (tokn < c.nC) {
-      double z[8];
-      token_logits<D>(qt, ktile, rowi, x, G, z);
-      double s = 0.0;
-#pragma unroll
-      for (int g = 0; g < 8; ++g)
-        if (g < G) s += exp(z[g] - sM[x * 8 + g]) / sZ[x * 8 + g];
-      const long long off = p.bnd_off[c.bi];
-      double* dst = p.scores + ((size_t)x * LH + c.lh) * p.max_batch_tokens + off;
-      dst[tokn] = s / (double)G;                           // group mean of the per-head softmaxes
-    }
-  }
-}
-
-// ------------------------------------------------------------------------------------------------------
 // decision + allocator, run by the last CTA of the selection kernel
 // ------------------------------------------------------------------------------------------------------
 __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int* actions, int* s_arr) {
@@ -399,6 +154,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       p.n[r] = p.b_nold[i] + 1;
       p.pos[r] += 1;
       p.started[r] = 1;
+      p.sum_par[r] ^= 1;                                  // the attention kernel wrote the other buffer
     }
   }
   if (tid == 0) {
@@ -564,13 +320,53 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       continue;
     }
     const long long off = p.bnd_off[bi];
-    const double* gS = p.scores + ((size_t)lh) * p.max_batch_tokens + off;
-    const double* gL = p.scores + ((size_t)LH + lh) * p.max_batch_tokens + off;
-    const double* aS = gS;
-    const double* aL = gL;
-    if (nC <= SEL_CAP) {
-      for (int i = tid; i < nC; i += SEL_T) { sa[i] = __ldcg(gS + i); sa[SEL_CAP + i] = __ldcg(gL + i); }
-      aS = sa; aL = sa + SEL_CAP;
+    const int G = p.G, G2 = 2 * p.G;
+    const double* z = p.zbuf + ((size_t)lh * p.max_batch_tokens + off) * G2;      // [nC][2][G]
+    double* gS = p.scores + ((size_t)lh) * p.max_batch_tokens + off;
+    double* gL = p.scores + ((size_t)LH + lh) * p.max_batch_tokens + off;
+    double* aS = gS;
+    double* aL = gL;
+    if (nC <= SEL_CAP) { aS = sa; aL = sa + SEL_CAP; }
+    // ---- per-head softmax over C, then the group mean (Sec. 3.2) --------------------------------------------
+    {
+      double* red = reinterpret_cast<double*>(hsum);          // [SEL_T] scratch, free until the histograms
+      double* sM = reinterpret_cast<double*>(hcnt);           // [16]
+      double* sZ = sM + 16;                                   // [16]
+      const int col = tid % G2;                               // SEL_T is a multiple of 2G
+      const size_t entries = (size_t)nC * G2;
+      double m = -INFINITY;
+      for (size_t e = tid; e < entries; e += SEL_T) m = fmax(m, __ldcg(z + e));
+      red[tid] = m;
+      __syncthreads();
+      if (tid < G2) {
+        double mm = -INFINITY;
+        for (int k2 = tid; k2 < SEL_T; k2 += G2) mm = fmax(mm, red[k2]);
+        sM[tid] = mm;
+      }
+      __syncthreads();
+      const double mc = sM[col];
+      double zs = 0.0;
+      for (size_t e = tid; e < entries; e += SEL_T) zs += exp(__ldcg(z + e) - mc);
+      __syncthreads();
+      red[tid] = zs;
+      __syncthreads();
+      if (tid < G2) {
+        double t = 0.0;
+        for (int k2 = tid; k2 < SEL_T; k2 += G2) t += red[k2];
+        sZ[tid] = t;
+      }
+      __syncthreads();
+      for (int i = tid; i < nC; i += SEL_T) {
+        const double* zr = z + (size_t)i * G2;
+        double s0 = 0.0, s1 = 0.0;
+        for (int g = 0; g < G; ++g) {
+          s0 += exp(__ldcg(zr + g) - sM[g]) / sZ[g];
+          s1 += exp(__ldcg(zr + G + g) - sM[G + g]) / sZ[G + g];
+        }
+        aS[i] = s0 / (double)G;
+        aL[i] = s1 / (double)G;
+      }
+      __syncthreads();
     }
     for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
     if (tid == 0) s_i[0] = 0;
@@ -868,31 +664,12 @@ size_t gp_bsel_smem(const GpDev& p) {
   return SelGeom::SA_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
 }
 
-void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, const void* q, int* actions, int grid_score,
-                        int grid_sel, int grid_compact, cudaStream_t s, cudaEvent_t* ev) {
-  const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
+void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, int grid_sel, int grid_compact,
+                        cudaStream_t s, cudaEvent_t ev) {
   const size_t sel_sm = gp_bsel_smem(p);
-  if (p.d == 128) {
-    auto k1 = gp_bstat_kernel<128>;
-    auto k2 = gp_bprob_kernel<128>;
-    cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<128>::SMEM);
-    cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<128>::SMEM);
-    k1<<<grid_score, ST, ScoreGeom<128>::SMEM, s>>>(p, req_ids, n_req, qq);
-    if (ev) cudaEventRecord(ev[0], s);
-    k2<<<grid_score, ST, ScoreGeom<128>::SMEM, s>>>(p, req_ids, n_req);
-  } else {
-    auto k1 = gp_bstat_kernel<64>;
-    auto k2 = gp_bprob_kernel<64>;
-    cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<64>::SMEM);
-    cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScoreGeom<64>::SMEM);
-    k1<<<grid_score, ST, ScoreGeom<64>::SMEM, s>>>(p, req_ids, n_req, qq);
-    if (ev) cudaEventRecord(ev[0], s);
-    k2<<<grid_score, ST, ScoreGeom<64>::SMEM, s>>>(p, req_ids, n_req);
-  }
-  if (ev) cudaEventRecord(ev[1], s);
   cudaFuncSetAttribute(gp_bsel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
   gp_bsel_kernel<<<grid_sel, SEL_T, sel_sm, s>>>(p, req_ids, n_req, actions);
-  if (ev) cudaEventRecord(ev[2], s);
+  if (ev) cudaEventRecord(ev, s);
   if (p.d == 128) gp_compact_kernel<128><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);
   else gp_compact_kernel<64><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);
 }

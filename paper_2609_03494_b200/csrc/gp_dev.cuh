@@ -7,7 +7,7 @@
 //                   slot index: logical chunk c of slot s lives at chunk c ^ (s & 7).  A tile
 //                   copied verbatim to shared memory is then bank-conflict free for ldmatrix.
 //   tok       int32 [L][n_pages][H_kv][b]               original token index of every slot
-//   summaries fp64  [L][M][2][H_q][d]                   Eq. 11 layout, short then long
+//   summaries fp64  [L][M][2][2][H_q][d]                Eq. 11 layout (short then long), double-buffered
 //   page_table / shadow int32 [M][cap]                  shadow holds copy-on-write targets
 //   scores    fp64  [2][L*H_kv][max_batch_tokens]       a^S, a^L of the requests at a boundary
 //   partials  fp32  split-KV partial outputs
@@ -19,10 +19,11 @@
 #define GP_PAGE 16             // tokens per page (b)
 #define GP_ATTN_WARPS 4
 #define GP_ATTN_STAGES 3
-#define GP_SPIN_LIMIT (1u << 24)
+#define GP_SPIN_LIMIT (1u << 23)
 #define GP_MAX_REQ 1024        // upper limit of max_requests (shared-memory arrays are sized by it)
 #define GP_SCORE_TILE 128      // candidate tokens per boundary-scoring tile
 #define GP_MOVE_TOK 64         // source slots per compaction chunk
+#define GP_DESC_INTS 48        // ints per attention work descriptor: 16 header words + 32 page ids
 
 // plan header slots (int32)
 enum {
@@ -33,7 +34,6 @@ enum {
   HDR_DONE_CMP,      // CTAs of the compaction kernel that have finished
   HDR_STEP,          // step serial number
   HDR_N_ACTIVE,      // requests actually stepped
-  HDR_N_BTILE,       // scoring tiles over all requests at a boundary
   HDR_DONE_SEL,      // CTAs of the selection kernel that have finished
   HDR_WORK_CMP,      // ticket counter of the compaction kernel
   HDR_N_CITEM,       // compaction work items (chunks x layers x heads)
@@ -49,7 +49,7 @@ enum {
 
 struct GpDev {
   // geometry
-  int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc, max_btiles;
+  int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;
   long long n_pages, max_batch_tokens;
   double beta_s, beta_l, top_p, tau, rope_theta;
   unsigned long long p_fix;              // top_p in 2^62 fixed point
@@ -68,7 +68,11 @@ struct GpDev {
   double* delta;                         // [M]
   // per step
   int* hdr;
-  int4* rc;                              // {batch index, first page, pages, chunk | n_chunks << 16}
+  int* rcx;                              // [max_rc][GP_DESC_INTS] attention work descriptors:
+                                         //   0 batch index, 1 request, 2 first page, 3 pages, 4 chunk, 5 chunks,
+                                         //   6 n before the append, 7 position, 8 flags (1 boundary, 2 started),
+                                         //   9 P, 10-11 offset into the logit scratch, 12 summary buffer in use,
+                                         //   13 own index, 16.. page ids
   int* b_nold;                           // [M] occupied slots before the append, by batch index
   int* b_flags;                          // [M] 1 = stepped this step
   int* first_idx;                        // [M] lowest batch index naming a request
@@ -78,10 +82,8 @@ struct GpDev {
   int* cmp_list;                         // [M] batch indices that compress
   int* cmp_bnd;                          // [M] their index in bnd_list
   int* cmp_chunk0;                       // [M+1] prefix of their compaction chunk counts
-  int2* bt_list;                         // [max_btiles] {index in bnd_list, tile} of every scoring tile
-  int* bnd_tile0;                        // [M] first scoring tile of a boundary request
-  double* bstats;                        // [L*H_kv][max_btiles][2G][2] softmax partials (max, sum)
-  double* qtilde;                        // [M][L*H_kv][2G][d] calibrated (and rotated) summaries
+  double* zbuf;                          // [L*H_kv][max_batch_tokens][2][G] summary logits of boundary units
+  int* sum_par;                          // [M] which of the two summary buffers is current
   int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
   int* cflags;                           // compaction chunk flags, stamped with the step number
   double* rope_cs;                       // [M][d/2][2] cos, sin at the step's position
@@ -98,8 +100,9 @@ __device__ __forceinline__ size_t gp_tile_off(const GpDev& p, int l, long long p
 __device__ __forceinline__ size_t gp_tok_off(const GpDev& p, int l, long long page, int h) {
   return (((size_t)l * (size_t)p.n_pages + (size_t)page) * p.Hkv + h) * GP_PAGE;
 }
-__device__ __forceinline__ size_t gp_summ_off(const GpDev& p, int l, int r, int x, int head) {
-  return ((((size_t)l * p.M + r) * 2 + x) * p.Hq + head) * (size_t)p.d;
+// summaries: [L][M][2 buffers][2 views][H_q][d]
+__device__ __forceinline__ size_t gp_summ_off(const GpDev& p, int l, int r, int buf, int x, int head) {
+  return ((((((size_t)l * p.M + r) * 2 + buf) * 2 + x) * p.Hq) + head) * (size_t)p.d;
 }
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -113,11 +116,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
 }
+// non-blocking test of a phase: the bounded spins below must not rely on the hardware's own wait limit
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(smem_u32(bar)), "r"(parity)
@@ -172,7 +176,7 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
                          float* out, int grid, cudaStream_t s);
 size_t gp_attention_smem(int d);
 int gp_attention_ctas_per_sm(int d);
-// boundary chain: partial softmax stats, probabilities, working sets + selection + decision, compaction.
-// `ev`, when not null, receives three events recorded between the four kernels.
-void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, const void* q, int* actions, int grid_score,
-                        int grid_sel, int grid_compact, cudaStream_t s, cudaEvent_t* ev);
+// boundary chain: probabilities + working sets + selection + decision, then compaction.
+// `ev`, when not null, is recorded between the two kernels.
+void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, int grid_sel, int grid_compact,
+                        cudaStream_t s, cudaEvent_t ev);

@@ -11,7 +11,6 @@
 #include "../../include/growpage.h"
 #include "gp_dev.cuh"
 
-#define GP_SCORE_GRID 592       // 4 CTAs per SM on 148 SMs
 #define GP_SEL_GRID 148         // one 1024-thread CTA per SM
 #define GP_COMPACT_GRID 592     // 4 CTAs per SM
 #define GP_PLAN_THREADS 1024
@@ -41,10 +40,10 @@ namespace {
 
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
-      b_flags, first_idx, unit_cnt, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, bt_list, bnd_tile0, bstats, qtilde,
+      b_flags, unit_cnt, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, zbuf, sum_par,
       evict, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
-  int max_rc, max_btiles;
+  int max_rc;
   long long max_batch_tokens;
 };
 
@@ -54,7 +53,7 @@ int chunk_pages_setting() {
   const char* e = getenv("GP_CHUNK_PAGES");
   int v = e ? atoi(e) : 16;
   if (v < 1) v = 1;
-  if (v > 64) v = 64;
+  if (v > 32) v = 32;
   return v;
 }
 
@@ -95,25 +94,21 @@ Layout make_layout(const gp_config& c) {
   L.page_table = take(M * cap * 4);
   L.shadow = take(M * cap * 4);
   L.reqi = take(5 * M * 4);                      // P, n, started, live, n_pristine
+  L.sum_par = take(M * 4);
   L.pos = take(M * 8);
-  L.summ = take((size_t)c.n_layers * M * 2 * c.n_q_heads * d * 8);
+  L.summ = take((size_t)c.n_layers * M * 2 * 2 * c.n_q_heads * d * 8);
   L.Kx = take(M * LH * 2 * 4);
   L.delta = take(M * 8);
-  L.rc = take((size_t)L.max_rc * 16);
+  L.rc = take((size_t)L.max_rc * GP_DESC_INTS * 4);
   L.b_nold = take(M * 4);
   L.b_flags = take(M * 4);
-  L.first_idx = take(M * 4);
   L.unit_cnt = take(M * LH * 4);
   L.bnd_list = take(M * 4);
   L.bnd_off = take(M * 8);
   L.cmp_list = take(M * 4);
   L.cmp_bnd = take(M * 4);
   L.cmp_chunk0 = take((M + 1) * 4);
-  L.max_btiles = (int)((size_t)L.max_batch_tokens / GP_SCORE_TILE + M + 1);
-  L.bt_list = take((size_t)L.max_btiles * 8);
-  L.bnd_tile0 = take(M * 4);
-  L.bstats = take(LH * (size_t)L.max_btiles * 32 * 8);
-  L.qtilde = take(M * LH * 2 * G * d * 8);
+  L.zbuf = take(LH * (size_t)L.max_batch_tokens * 2 * G * 8);
   L.evict = take(M * LH * b * 4);
   L.cflags = take(LH * ((size_t)L.max_batch_tokens / GP_MOVE_TOK + 2 * M + 1) * 4);
   L.rope_cs = take(M * (d / 2) * 2 * 8);
@@ -144,7 +139,6 @@ __global__ void gp_init_kernel(GpDev p) {
   // page 0 is handed out first
   for (long long i = i0; i < p.n_pages; i += stride) p.free_stack[i] = (int)(p.n_pages - 1 - i);
   for (long long i = i0; i < (long long)p.M * p.cap; i += stride) p.shadow[i] = -1;
-  for (long long i = i0; i < p.M; i += stride) p.first_idx[i] = 0x7fffffff;
   if (i0 == 0) *p.free_top = (int)p.n_pages;
 }
 
@@ -172,38 +166,45 @@ __device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long
   __syncthreads();
 }
 
-// Step plan: validates the batch, cuts every stepped request into (request, chunk) work items for the
-// attention kernel, lists the requests that reach their capacity boundary with this step's append
-// (trailing check: n + 1 == P b) and hands each a slice of the score scratch.
+// Step plan: validates the batch, cuts every stepped request into chunks and writes one self-contained work
+// descriptor per chunk for the attention kernel, lists the requests that reach their capacity boundary
+// with this step's append (trailing check: n + 1 == P b) and hands each a slice of the logit scratch.
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
   __shared__ int sv[32];
   __shared__ long long sw[32];
+  __shared__ int s_rcoff[GP_MAX_REQ], s_chunks[GP_MAX_REQ], s_pages[GP_MAX_REQ], s_nold[GP_MAX_REQ];
+  int* s_first = s_rcoff;          // lowest batch index naming a request; dead before s_rcoff is written
+  __shared__ int s_flags[GP_MAX_REQ], s_P[GP_MAX_REQ], s_r[GP_MAX_REQ], s_pos[GP_MAX_REQ], s_par[GP_MAX_REQ];
+  __shared__ long long s_zoff[GP_MAX_REQ];
   const int i = threadIdx.x;
   const bool in = i < n_req;
+  s_first[i] = 0x7fffffff;
+  __syncthreads();
   int r = -1;
   if (in) {
     r = req_ids[i];
-    if (r >= 0 && r < p.M) atomicMin(&p.first_idx[r], i);
+    if (r >= 0 && r < p.M) atomicMin(&s_first[r], i);
   }
   __syncthreads();
-  int chunks = 0, pages = 0, n_old = 0, act = GP_ACT_NONE;
-  long long nc = 0;
+  int chunks = 0, pages = 0, n_old = 0, act = GP_ACT_NONE, Pr = 0, started = 0, par = 0;
+  long long nc = 0, pos = 0;
   int isb = 0;
   if (in) {
-    const bool valid = r >= 0 && r < p.M && p.live[r] && p.first_idx[r] == i;
+    const bool inrange = r >= 0 && r < p.M;
+    int live = 0;
+    if (inrange) {                    // independent loads, issued together
+      live = p.live[r]; n_old = p.n[r]; Pr = p.P[r]; pos = p.pos[r]; started = p.started[r]; par = p.sum_par[r];
+    }
+    const bool valid = inrange && live && s_first[r] == i;
     if (!valid) {
       act = GP_ACT_INVALID;
+    } else if (n_old >= Pr * GP_PAGE) {
+      act = GP_ACT_STALLED;
     } else {
-      n_old = p.n[r];
-      const int Pr = p.P[r];
-      if (n_old >= Pr * GP_PAGE) {
-        act = GP_ACT_STALLED;
-      } else {
-        pages = n_old / GP_PAGE + 1;
-        chunks = (pages + p.chunk_pages - 1) / p.chunk_pages;
-        if (n_old + 1 == Pr * GP_PAGE) { isb = 1; nc = (long long)(Pr - 1) * GP_PAGE; }
-      }
+      pages = n_old / GP_PAGE + 1;
+      chunks = (pages + p.chunk_pages - 1) / p.chunk_pages;
+      if (n_old + 1 == Pr * GP_PAGE) { isb = 1; nc = (long long)(Pr - 1) * GP_PAGE; }
     }
   }
   int rc_off, n_rc; long long tok_off, tok_tot;
@@ -213,37 +214,60 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     atomicOr(p.err, GP_E_BOUNDS);
     chunks = 0; isb = 0; act = GP_ACT_SCRATCH;
   }
-  int bnd_idx, n_bnd; long long dummy0, dummy1;
-  const int my_tiles = isb ? (int)((nc + GP_SCORE_TILE - 1) / GP_SCORE_TILE) : 0;
-  long long tile_off, n_btile;
-  plan_scan(isb, my_tiles, bnd_idx, tile_off, n_bnd, n_btile, sv, sw);
-  if (n_btile > p.max_btiles) { atomicOr(p.err, GP_E_BOUNDS); n_btile = 0; n_bnd = 0; isb = 0; }
-  int act_idx, n_active;
-  plan_scan(chunks > 0, 0, act_idx, dummy0, n_active, dummy1, sv, sw);
+  int bnd_idx, n_bnd, act_idx, n_active; long long d0, d1;
+  plan_scan(isb, chunks > 0, bnd_idx, d0, n_bnd, d1, sv, sw);
+  act_idx = (int)d0; n_active = (int)d1;
+  (void)act_idx;
+  s_rcoff[i] = rc_off; s_chunks[i] = chunks; s_pages[i] = pages; s_nold[i] = n_old;
+  s_flags[i] = isb | (started ? 2 : 0); s_P[i] = Pr; s_r[i] = r; s_pos[i] = (int)pos; s_par[i] = par;
+  s_zoff[i] = tok_off;
   if (in) {
     p.b_nold[i] = n_old;
     p.b_flags[i] = chunks > 0;
     actions[i] = act;
-    for (int c = 0; c < chunks; ++c) {
+    if (isb) { p.bnd_list[bnd_idx] = i; p.bnd_off[i] = tok_off; }
+  }
+  __syncthreads();
+  // descriptors: one warp per request, lanes across the words
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int bi = warp; bi < n_req; bi += GP_PLAN_THREADS / 32) {
+    const int nch = s_chunks[bi];
+    if (nch == 0) continue;
+    const int rr = s_r[bi];
+    const int* table = p.page_table + (size_t)rr * p.cap;
+    for (int c = 0; c < nch; ++c) {
       const int pg0 = c * p.chunk_pages;
-      p.rc[rc_off + c] = make_int4(i, pg0, min(p.chunk_pages, pages - pg0), c | (chunks << 16));
+      const int npg = min(p.chunk_pages, s_pages[bi] - pg0);
+      int* d = p.rcx + (size_t)(s_rcoff[bi] + c) * GP_DESC_INTS;
+      int hv = 0;
+      switch (lane) {
+        case 0: hv = bi; break;
+        case 1: hv = rr; break;
+        case 2: hv = pg0; break;
+        case 3: hv = npg; break;
+        case 4: hv = c; break;
+        case 5: hv = nch; break;
+        case 6: hv = s_nold[bi]; break;
+        case 7: hv = s_pos[bi]; break;
+        case 8: hv = s_flags[bi]; break;
+        case 9: hv = s_P[bi]; break;
+        case 10: hv = (int)(unsigned)(s_zoff[bi] & 0xffffffffLL); break;
+        case 11: hv = (int)(s_zoff[bi] >> 32); break;
+        case 12: hv = s_par[bi]; break;
+        case 13: hv = s_rcoff[bi] + c; break;
+        default: break;
+      }
+      if (lane < 16) d[lane] = hv;
+      d[16 + lane] = lane < npg ? table[pg0 + lane] : -1;
     }
-    if (isb) {
-      p.bnd_list[bnd_idx] = i;
-      p.bnd_off[i] = tok_off;
-      p.bnd_tile0[bnd_idx] = (int)tile_off;
-      for (int t = 0; t < my_tiles; ++t) p.bt_list[tile_off + t] = make_int2(bnd_idx, t);
-    }
-    if (r >= 0 && r < p.M) p.first_idx[r] = 0x7fffffff;          // ready for the next step
   }
   if (p.rope_theta != 0.0) {                                      // cos / sin of the step's position
     const int half = p.d / 2;
     for (int idx = threadIdx.x; idx < n_req * half; idx += GP_PLAN_THREADS) {
       const int bi = idx / half, j = idx % half;
-      const int rr = req_ids[bi];
-      if (rr >= 0 && rr < p.M && p.live[rr]) {
+      if (s_chunks[bi] > 0) {
         const double inv = pow(p.rope_theta, -2.0 * (double)j / (double)p.d);
-        const double ang = (double)p.pos[rr] * inv;
+        const double ang = (double)s_pos[bi] * inv;
         double sn, cs;
         sincos(ang, &sn, &cs);
         p.rope_cs[(size_t)idx * 2] = cs;
@@ -254,8 +278,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   if (threadIdx.x == 0) {
     p.hdr[HDR_N_RC] = n_rc;
     p.hdr[HDR_N_BND] = n_bnd;
-    p.hdr[HDR_N_BTILE] = (int)n_btile;
-    p.hdr[HDR_N_CMP] = 0;
     p.hdr[HDR_WORK_ATTN] = 0;
     p.hdr[HDR_N_ACTIVE] = n_active;
     p.hdr[HDR_STEP] += 1;
@@ -426,7 +448,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   GpDev& d = pool->dev;
   d.L = cfg->n_layers; d.Hq = cfg->n_q_heads; d.Hkv = cfg->n_kv_heads; d.G = cfg->n_q_heads / cfg->n_kv_heads;
   d.d = cfg->head_dim; d.M = cfg->max_requests; d.cap = cfg->max_pages_per_req; d.k_loc = cfg->k_loc;
-  d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc; d.max_btiles = L.max_btiles;
+  d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc;
   d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
   d.p_fix = (unsigned long long)llrint(cfg->top_p * 4611686018427387904.0);
@@ -448,20 +470,17 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.summ = reinterpret_cast<double*>(base + L.summ);
   d.Kx = reinterpret_cast<int*>(base + L.Kx);
   d.delta = reinterpret_cast<double*>(base + L.delta);
-  d.rc = reinterpret_cast<int4*>(base + L.rc);
+  d.rcx = reinterpret_cast<int*>(base + L.rc);
   d.b_nold = reinterpret_cast<int*>(base + L.b_nold);
   d.b_flags = reinterpret_cast<int*>(base + L.b_flags);
-  d.first_idx = reinterpret_cast<int*>(base + L.first_idx);
   d.unit_cnt = reinterpret_cast<int*>(base + L.unit_cnt);
   d.bnd_list = reinterpret_cast<int*>(base + L.bnd_list);
   d.bnd_off = reinterpret_cast<long long*>(base + L.bnd_off);
   d.cmp_list = reinterpret_cast<int*>(base + L.cmp_list);
   d.cmp_bnd = reinterpret_cast<int*>(base + L.cmp_bnd);
   d.cmp_chunk0 = reinterpret_cast<int*>(base + L.cmp_chunk0);
-  d.bt_list = reinterpret_cast<int2*>(base + L.bt_list);
-  d.bnd_tile0 = reinterpret_cast<int*>(base + L.bnd_tile0);
-  d.bstats = reinterpret_cast<double*>(base + L.bstats);
-  d.qtilde = reinterpret_cast<double*>(base + L.qtilde);
+  d.zbuf = reinterpret_cast<double*>(base + L.zbuf);
+  d.sum_par = reinterpret_cast<int*>(base + L.sum_par);
   d.evict = reinterpret_cast<int*>(base + L.evict);
   d.cflags = reinterpret_cast<int*>(base + L.cflags);
   d.rope_cs = reinterpret_cast<double*>(base + L.rope_cs);
@@ -550,9 +569,8 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   if (prof) cudaEventRecord(pool->ev[1], s);
   gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s);
   if (prof) cudaEventRecord(pool->ev[2], s);
-  gp_launch_boundary(d, dev_req_ids, n_req, q, dev_actions, GP_SCORE_GRID, GP_SEL_GRID, GP_COMPACT_GRID, s,
-                     prof ? &pool->ev[3] : nullptr);
-  if (prof) cudaEventRecord(pool->ev[6], s);
+  gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, GP_SEL_GRID, GP_COMPACT_GRID, s, prof ? pool->ev[3] : nullptr);
+  if (prof) cudaEventRecord(pool->ev[4], s);
   pool->launch_count += GP_N_KERNELS;
   GP_CUDA(cudaGetLastError());
   if (prof) {
@@ -681,10 +699,12 @@ int gp_debug_summaries(gp_pool* pool, int32_t req, double* out) {
   GP_CUDA(cudaSetDevice(pool->device));
   GP_CUDA(cudaDeviceSynchronize());
   const gp_config& c = pool->cfg;
+  int par = 0;
+  GP_CUDA(cudaMemcpy(&par, pool->dev.sum_par + req, 4, cudaMemcpyDeviceToHost));
   const size_t per = (size_t)2 * c.n_q_heads * c.head_dim;
   for (int l = 0; l < c.n_layers; ++l)
-    GP_CUDA(cudaMemcpy(out + (size_t)l * per, pool->dev.summ + ((size_t)l * c.max_requests + req) * per, per * 8,
-                       cudaMemcpyDeviceToHost));
+    GP_CUDA(cudaMemcpy(out + (size_t)l * per, pool->dev.summ + (((size_t)l * c.max_requests + req) * 2 + par) * per,
+                       per * 8, cudaMemcpyDeviceToHost));
   return GP_OK;
 }
 
