@@ -10,26 +10,33 @@
 //               the K|V tiles of their pages (one contiguous `cp.async.bulk` per (layer, page, head))
 //               into a ring of stages shared by the CTA.  It runs ahead across item boundaries, so the
 //               ring never drains between items.
-//   warps 1..4  consumers: take the tiles of an item round-robin.  The G query heads of the group are
+//   warps 4..7  consumers: take the tiles of an item round-robin.  The G query heads of the group are
 //               rows 0..G-1 of an m16n8k16 bf16 MMA; S = Q K^T and O += P V run on the tensor cores with
 //               fp32 accumulation.  Rows 8..15 of the A operand carry the bf16 rounding residual of
 //               rows 0..7 (of the rotated query when RoPE is on, of P always), which costs nothing and
-//               gives ~16 mantissa bits.  At the end of an item the four warps merge through shared
-//               memory; requests split over several items merge through scratch, last arrival wins.
-//   warp 5      summaries: Eq. 6 on the un-rotated query (read from one of two buffers, written to the
+//               gives ~16 mantissa bits.  For boundary units the summary logits of a candidate page are
+//               an fp64 tensor-core contraction (m8n8k4 DMMA: 8 tokens x (2 views x G heads) x d).
+//   warp 1      summaries: Eq. 6 on the un-rotated query (read from one of two buffers, written to the
 //               other, so that every item of a unit sees the old state), and for boundary units the
 //               calibrated, rotated summaries q~ in fp64 for the consumers.
+//   warp 2      merger: combines the four consumers' partial (max, sum, O) of an item, writes the output
+//               or, for requests split over several items, the partial and, as last arrival, the merge.
+//               Consumers hand over through a double buffer and go straight on to the next item.
 //
+// The two warp groups re-split the register file (setmaxnreg): the service warps keep 56 registers per
+// thread, the consumers, which hold the output accumulators, get 200.
 // All waits are bounded; a wait that gives up sets an error bit and an abort flag that drains the CTA.
 #include "gp_dev.cuh"
 
 namespace {
 
-constexpr int NS = 8;                      // tile stages per CTA
-constexpr int NI = 4;                      // item slots per CTA
+constexpr int NI_MAX = 8;                  // item slots per CTA (4 when the group is 8 heads wide)
+constexpr int NSW = 2;                     // tile stages per consumer warp
 constexpr int NCW = 4;                     // consumer warps
-constexpr int NTHREADS = 32 * (NCW + 2);
-constexpr int CONS_THREADS = 32 * NCW;
+constexpr int NTHREADS = 256;              // warp group 0: producer, summaries, merger, spare; warp group 1: consumers
+constexpr int REGS_SERVICE = 56;           // registers per thread after the split (setmaxnreg)
+constexpr int REGS_CONSUMER = 200;
+constexpr int QT_PAD = 8;                  // doubles of padding per q~ row: rows alternate bank halves
 
 template <int D>
 struct Geo {
@@ -39,16 +46,28 @@ struct Geo {
   static constexpr int DTILES = D / 8;
   static constexpr int SLOT_DESC = 128;                                // 32 ints
   static constexpr int SLOT_BYTES = (SLOT_DESC + 8 * ROW_BYTES + 2 * ROW_BYTES + 127) / 128 * 128;
-  static constexpr int QT_BYTES = 2 * 8 * D * 8;
-  static constexpr int COMB_WARP = (16 + 8 * D) * 4;
-  static constexpr int OFF_SLOTS = NS * TILE_BYTES;
-  static constexpr int OFF_QT = OFF_SLOTS + NI * SLOT_BYTES;
-  static constexpr int OFF_COMB = OFF_QT + QT_BYTES;
-  static constexpr int OFF_BARS = OFF_COMB + NCW * COMB_WARP;
-  static constexpr int N_BARS = 2 * NS + 2 * NI + 2;
-  static constexpr int OFF_MISC = OFF_BARS + N_BARS * 8;
-  static constexpr int SMEM_BYTES = OFF_MISC + 64 + 256;
 };
+
+struct Lay {            // shared-memory layout, depends on the group size
+  int ni, ncomb, off_slots, off_qt, off_comb, comb_warp, off_bars, off_misc, total;
+};
+template <int D>
+__host__ __device__ inline Lay make_lay(int G) {
+  using GEO = Geo<D>;
+  Lay L;
+  const bool wide = (D == 128 && G == 8);
+  L.ni = wide ? 4 : NI_MAX;
+  L.ncomb = wide ? 1 : 2;
+  L.off_slots = NCW * NSW * GEO::TILE_BYTES;
+  L.off_qt = L.off_slots + L.ni * GEO::SLOT_BYTES;
+  const int nrows = 2 * G < 8 ? 8 : 2 * G;
+  L.off_comb = L.off_qt + nrows * (D + QT_PAD) * 8;
+  L.comb_warp = (16 + G * D) * 4;
+  L.off_bars = L.off_comb + L.ncomb * NCW * L.comb_warp;
+  L.off_misc = L.off_bars + (2 * NCW * NSW + 2 * NI_MAX + 2 + 4) * 8;
+  L.total = L.off_misc + 64 + 256;
+  return L;
+}
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -57,24 +76,15 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < GP_SPIN_LIMIT; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && *abort_flag) return false;
+    if ((it & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
 }
-__device__ __forceinline__ void cons_sync() { asm volatile("bar.sync 1, %0;" ::"n"(CONS_THREADS) : "memory"); }
-// barrier over the consumer warps that also ORs a predicate
-__device__ __forceinline__ bool cons_any(bool pred) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.or.pred p, 1, %2, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r)
-      : "r"((uint32_t)pred), "n"(CONS_THREADS)
-      : "memory");
-  return r != 0;
+__device__ __forceinline__ void dmma(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(d0), "+d"(d1)
+               : "d"(a), "d"(b));
 }
 
 template <int D, bool ROPE>
@@ -84,23 +94,30 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   using GEO = Geo<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + GEO::OFF_BARS);
-  uint64_t* full = bars;
-  uint64_t* empty = bars + NS;
-  uint64_t* slot_full = bars + 2 * NS;
-  uint64_t* slot_empty = bars + 2 * NS + NI;
-  uint64_t* qt_full = bars + 2 * NS + 2 * NI;
+  const int G = p.G;
+  const Lay L = make_lay<D>(G);
+  const uint32_t NI = (uint32_t)L.ni, NCOMB = (uint32_t)L.ncomb;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.off_bars);
+  uint64_t* full = bars;                       // [NCW][NSW]: each consumer warp owns a private ring, so a warp
+  uint64_t* empty = bars + NCW * NSW;          //   never waits more than one phase ahead of its barrier
+  uint64_t* slot_full = bars + 2 * NCW * NSW;  // [NI]
+  uint64_t* slot_empty = slot_full + NI_MAX;   // [NI]
+  uint64_t* qt_full = slot_empty + NI_MAX;
   uint64_t* qt_empty = qt_full + 1;
-  volatile int* s_misc = reinterpret_cast<volatile int*>(smem + GEO::OFF_MISC);   // [0] abort, [1] last flag
-  double* qt = reinterpret_cast<double*>(smem + GEO::OFF_QT);
+  uint64_t* comb_full = qt_empty + 1;          // [2]
+  uint64_t* comb_empty = comb_full + 2;        // [2]
+  volatile int* s_misc = reinterpret_cast<volatile int*>(smem + L.off_misc);   // [0] abort
+  double* qt = reinterpret_cast<double*>(smem + L.off_qt);                     // [2G][D + QT_PAD]
+  float* comb = reinterpret_cast<float*>(smem + L.off_comb);                   // [2][NCW][16 + G*D]
+  const int comb_w = L.comb_warp / 4;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int G = p.G;
   if (tid == 0) {
-    for (int i = 0; i < NS; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < NI; ++i) { mbar_init(&slot_full[i], 1); mbar_init(&slot_empty[i], NCW + 1); }
+    for (int i = 0; i < NCW * NSW; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < NI_MAX; ++i) { mbar_init(&slot_full[i], 1); mbar_init(&slot_empty[i], NCW + 2); }
     mbar_init(qt_full, 1);
     mbar_init(qt_empty, NCW);
+    for (int i = 0; i < 2; ++i) { mbar_init(&comb_full[i], NCW); mbar_init(&comb_empty[i], 1); }
     s_misc[0] = 0;
     fence_mbar_init();
   }
@@ -111,96 +128,141 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   const long long total = (long long)n_rc * LH;
   const int q_bytes = G * GEO::ROW_BYTES;
 
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE));
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_CONSUMER));
+  }
   if (warp == 0) {
     // ================================= producer ===========================================
-    uint32_t fillc = 0;
-    for (uint32_t it = 0;; ++it) {
-      long long item = 0;
-      if (lane == 0) item = atomicAdd(&p.hdr[HDR_WORK_ATTN], 1);
-      item = __shfl_sync(0xffffffffu, item, 0);
-      const int sl = it % NI;
-      if (!wait_bar(&slot_empty[sl], ((it / NI) & 1u) ^ 1u, s_misc)) break;
-      uint8_t* slot = smem + GEO::OFF_SLOTS + sl * GEO::SLOT_BYTES;
-      int* sd = reinterpret_cast<int*>(slot);
-      if (item >= total) {
-        if (lane == 0) { sd[3] = -1; }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&slot_full[sl]);
-        break;
+    // Software pipeline over items, one stage per tick, so that no global round trip sits between two
+    // tiles: claim (t), descriptor header (t-1), page ids (t-2), publish the item slot (t-3), stream its
+    // tiles (t-4).  The loads of the young stages are in flight while the oldest item streams.
+    long long itA = total, itB = total, itC = total, itD = total, itE = total;   // claimed item per stage
+    int hB = 0, hC = 0, hD = 0, hE = 0;        // descriptor header, word `lane` (lanes 0..15)
+    int pC = -1, pD = -1, pE = -1;             // page id of tile `lane` of the item
+    uint32_t wf0 = 0, wf1 = 0, wf2 = 0, wf3 = 0;   // tiles issued so far to each consumer warp
+    uint32_t n_pub = 0;
+    bool sentinel_out = false;
+    for (uint32_t tick = 0;; ++tick) {
+      // ---- issue the loads of the young stages --------------------------------------------------
+      long long claimed = 0;
+      if (lane == 0) claimed = atomicAdd(&p.hdr[HDR_WORK_ATTN], 1);
+      int hNew = 0;
+      if (itA < total && lane < GP_DESC_INTS) hNew = p.rcx[(size_t)(itA % n_rc) * GP_DESC_INTS + lane];
+      int pNew = -1;
+      if (itB < total) {
+        const int r = __shfl_sync(0xffffffffu, hB, 1), pg0 = __shfl_sync(0xffffffffu, hB, 2);
+        const int npg = __shfl_sync(0xffffffffu, hB, 3);
+        if (lane < npg) pNew = p.page_table[(size_t)r * p.cap + pg0 + lane];
       }
-      const int rc_i = (int)(item % n_rc);
-      const int lh = (int)(item / n_rc);
-      const int l = lh / p.Hkv, h = lh % p.Hkv;
-      const int* desc = p.rcx + (size_t)rc_i * GP_DESC_INTS;
-      const int w0 = desc[lane];                                  // header words 0..15, pages 0..15
-      const int w1 = (lane < GP_DESC_INTS - 32) ? desc[32 + lane] : -1;   // pages 16..31
-      const int bi = __shfl_sync(0xffffffffu, w0, 0);
-      const int npg = __shfl_sync(0xffffffffu, w0, 3);
-      const int chunk = __shfl_sync(0xffffffffu, w0, 4);
-      const int nchunks = __shfl_sync(0xffffffffu, w0, 5);
-      const int last_pg = (npg - 1 < 16) ? __shfl_sync(0xffffffffu, w0, 16 + ((npg - 1) & 15))
-                                         : __shfl_sync(0xffffffffu, w1, (npg - 1 - 16) & 15);
-      if (lane < 14) sd[lane] = w0;
-      if (lane == 14) sd[14] = lh;
-      if (lane == 15) sd[15] = (int)fillc;
-      if (lane == 16) sd[16] = last_pg;
-      __syncwarp();
-      if (lane == 0) {
-        const bool has_new = (chunk == nchunks - 1);
-        fence_proxy_async();
-        mbar_expect_tx(&slot_full[sl], q_bytes + (has_new ? 2 * GEO::ROW_BYTES : 0));
-        bulk_g2s(slot + GEO::SLOT_DESC, q + (((size_t)l * n_req + bi) * p.Hq + h * G) * D, q_bytes, &slot_full[sl]);
-        if (has_new) {
-          const size_t kvo = (((size_t)l * n_req + bi) * p.Hkv + h) * D;
-          bulk_g2s(slot + GEO::SLOT_DESC + 8 * GEO::ROW_BYTES, k + kvo, GEO::ROW_BYTES, &slot_full[sl]);
-          bulk_g2s(slot + GEO::SLOT_DESC + 9 * GEO::ROW_BYTES, v + kvo, GEO::ROW_BYTES, &slot_full[sl]);
+      // ---- publish the slot of the item two stages from streaming ---------------------------------
+      if (tick >= 3 && !sentinel_out) {
+        const int sl = n_pub % NI;
+        const long long t_p0 = GP_T_NOW();
+        (void)t_p0;
+        if (!wait_bar(&slot_empty[sl], ((n_pub / NI) & 1u) ^ 1u, s_misc)) break;
+        if (lane == 0) GP_T_ADD(11, GP_T_NOW() - t_p0);
+        uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
+        int* sd = reinterpret_cast<int*>(slot);
+        if (itC >= total) {
+          if (lane == 0) sd[3] = -1;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&slot_full[sl]);
+          sentinel_out = true;
+        } else {
+          const int lh = (int)(itC / n_rc);
+          const int l = lh / p.Hkv, h = lh % p.Hkv;
+          const int bi = __shfl_sync(0xffffffffu, hC, 0);
+          const int npg = __shfl_sync(0xffffffffu, hC, 3);
+          const int chunk = __shfl_sync(0xffffffffu, hC, 4);
+          const int nchunks = __shfl_sync(0xffffffffu, hC, 5);
+          const int last_pg = __shfl_sync(0xffffffffu, pC, (npg - 1) & 31);
+          if (lane < 14) sd[lane] = hC;
+          if (lane == 14) sd[14] = lh;
+          if (lane == 16) sd[16] = last_pg;
+          __syncwarp();
+          if (lane == 0) {
+            const bool has_new = (chunk == nchunks - 1);
+            fence_proxy_async();
+            mbar_expect_tx(&slot_full[sl], q_bytes + (has_new ? 2 * GEO::ROW_BYTES : 0));
+            bulk_g2s(slot + GEO::SLOT_DESC, q + (((size_t)l * n_req + bi) * p.Hq + h * G) * D, q_bytes, &slot_full[sl]);
+            if (has_new) {
+              const size_t kvo = (((size_t)l * n_req + bi) * p.Hkv + h) * D;
+              bulk_g2s(slot + GEO::SLOT_DESC + 8 * GEO::ROW_BYTES, k + kvo, GEO::ROW_BYTES, &slot_full[sl]);
+              bulk_g2s(slot + GEO::SLOT_DESC + 9 * GEO::ROW_BYTES, v + kvo, GEO::ROW_BYTES, &slot_full[sl]);
+            }
+          }
         }
+        ++n_pub;
       }
-      bool ok = true;
-      for (int j = 0; j < npg; ++j) {
-        const int page = (j < 16) ? __shfl_sync(0xffffffffu, w0, 16 + j) : __shfl_sync(0xffffffffu, w1, j - 16);
-        const uint32_t st = fillc % NS;
-        if (!wait_bar(&empty[st], ((fillc / NS) & 1u) ^ 1u, s_misc)) { ok = false; break; }
-        if (lane == 0) {
-          fence_proxy_async();
-          mbar_expect_tx(&full[st], GEO::TILE_BYTES);
-          bulk_g2s(smem + st * GEO::TILE_BYTES, p.kv + gp_tile_off(p, l, page, h), GEO::TILE_BYTES, &full[st]);
+      // ---- stream the tiles of the oldest item ----------------------------------------------------------
+      if (tick >= 4) {
+        if (itD >= total) break;
+        const int lh = (int)(itD / n_rc);
+        const int l = lh / p.Hkv, h = lh % p.Hkv;
+        const int npg = __shfl_sync(0xffffffffu, hD, 3);
+        bool ok = true;
+        for (int j = 0; j < npg; ++j) {
+          const int page = __shfl_sync(0xffffffffu, pD, j);
+          const int cwj = j & (NCW - 1);                        // tile j of an item goes to consumer warp j mod 4
+          const uint32_t kf = cwj == 0 ? wf0 : cwj == 1 ? wf1 : cwj == 2 ? wf2 : wf3;
+          const uint32_t st = cwj * NSW + (kf % NSW);
+          const long long t_p1 = GP_T_NOW();
+          (void)t_p1;
+          if (!wait_bar(&empty[st], ((kf / NSW) & 1u) ^ 1u, s_misc)) { ok = false; break; }
+          if (lane == 0) GP_T_ADD(10, GP_T_NOW() - t_p1);
+          if (lane == 0) {
+            fence_proxy_async();
+            mbar_expect_tx(&full[st], GEO::TILE_BYTES);
+            bulk_g2s(smem + st * GEO::TILE_BYTES, p.kv + gp_tile_off(p, l, page, h), GEO::TILE_BYTES, &full[st]);
+          }
+          wf0 += (cwj == 0); wf1 += (cwj == 1); wf2 += (cwj == 2); wf3 += (cwj == 3);
         }
-        ++fillc;
+        if (!ok) break;
       }
-      if (!ok) break;
+      // ---- rotate -----------------------------------------------------------------------------------------
+      itE = itD; hE = hD; pE = pD;
+      itD = itC; hD = hC; pD = pC;
+      itC = itB; hC = hB; pC = pNew;
+      itB = itA; hB = hNew;
+      itA = __shfl_sync(0xffffffffu, claimed, 0);
+      (void)itE; (void)hE; (void)pE;
     }
     if (s_misc[0]) {
       // aborted: let the copies already issued land before the CTA goes away
       if (lane == 0) atomicOr(p.err, GP_E_SPIN);
-      for (uint32_t f = (fillc > NS ? fillc - NS : 0); f < fillc; ++f)
-        for (uint32_t it = 0; it < (1u << 20); ++it)
-          if (mbar_try_wait(&full[f % NS], (f / NS) & 1u)) break;
+      const uint32_t wf[NCW] = {wf0, wf1, wf2, wf3};
+      for (int c = 0; c < NCW; ++c)
+        for (uint32_t f = (wf[c] > NSW ? wf[c] - NSW : 0); f < wf[c]; ++f)
+          for (uint32_t it2 = 0; it2 < (1u << 16); ++it2)
+            if (mbar_try_wait(&full[c * NSW + (f % NSW)], (f / NSW) & 1u)) break;
     }
-  } else if (warp <= NCW) {
+  } else if (warp >= 4) {
     // ================================= consumers ==========================================
-    const int cw = warp - 1;
-    const int ctid = tid - 32;
+    const int cw = warp - 4;
     const float sc = 1.4426950408889634f * rsqrtf((float)D);
     const int row = lane >> 2;
     const int qc = (lane & 3) * 2;
-    uint32_t qt_uses = 0;
-    float* comb = reinterpret_cast<float*>(smem + GEO::OFF_COMB);
-    float* my_comb = comb + cw * (GEO::COMB_WARP / 4);
+    uint32_t qt_uses = 0, my_tiles = 0;
+    const bool tr = (cw == 0 && lane == 0);
+    const long long t_loop0 = GP_T_NOW();
+    (void)tr; (void)t_loop0;
     for (uint32_t it = 0;; ++it) {
       const int sl = it % NI;
+      const long long t_a = GP_T_NOW();
+      (void)t_a;
       if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc)) break;
-      const uint8_t* slot = smem + GEO::OFF_SLOTS + sl * GEO::SLOT_BYTES;
+      const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
       if (npg < 0) break;
-      const int bi = sd[0], r = sd[1], pg0 = sd[2], chunk = sd[4], nchunks = sd[5], n_old = sd[6];
+      if (tr) { GP_T_ADD(0, 1); GP_T_ADD(2, GP_T_NOW() - t_a); }
+      const int bi = sd[0], pg0 = sd[2], chunk = sd[4], nchunks = sd[5], n_old = sd[6];
       const int flags = sd[8], Pr = sd[9], lh = sd[14];
-      const uint32_t stage_base = (uint32_t)sd[15];
       const int l = lh / p.Hkv, h = lh % p.Hkv;
       const int n_new = n_old + 1;
       const bool need_qt = (flags & 1) && (pg0 < Pr - 1);
-      const int rc_i_slot = sd[13];
 
       // ---- query fragments (A operand), rotated when RoPE is on ----------------------------------
       uint32_t qa[GEO::KSTEPS][2];
@@ -252,9 +314,14 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       bool ok = true;
 
       for (int pgl = cw; pgl < npg; pgl += NCW) {
-        const uint32_t fidx = stage_base + (uint32_t)pgl;
-        const uint32_t st = fidx % NS;
-        if (!wait_bar(&full[st], (fidx / NS) & 1u, s_misc)) ok = false;   // keep the control flow uniform
+        const uint32_t st = cw * NSW + (my_tiles % NSW);
+        const long long t_b = GP_T_NOW();
+        (void)t_b;
+        if (!wait_bar(&full[st], (my_tiles / NSW) & 1u, s_misc)) { ok = false; break; }
+        ++my_tiles;
+        const long long t_c = GP_T_NOW();
+        (void)t_c;
+        if (tr) { GP_T_ADD(1, 1); GP_T_ADD(3, t_c - t_b); }
         uint8_t* tile = smem + st * GEO::TILE_BYTES;
         const int tok0 = (pg0 + pgl) * GP_PAGE;
         const bool has_new = last_chunk && (pgl == npg - 1);
@@ -343,123 +410,107 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
             mma_bf16(o[jd + 1], pa[0], pa[1], pa[2], pa[3], v2, v3);
           }
         }
-        // boundary unit: fp64 logits of the calibrated summaries against the 16 keys of a candidate page
+        const long long t_d = GP_T_NOW();
+        (void)t_d;
+        if (tr) GP_T_ADD(4, t_d - t_c);
+        // Boundary unit: fp64 logits of the calibrated summaries against the 16 keys of a candidate page,
+        // Z[token][n] = sum_d K[token][d] q~[n][d], n = view * G + head.  One m8n8k4 DMMA covers 8 tokens,
+        // 8 columns and 4 values of d; inside a 16-byte chunk of a key row lane t of a quad takes the
+        // bf16 pair at byte 4t, whose low and high element feed two successive k-steps (q~ is read with
+        // the same mapping, so the contraction is over the same d on both sides).
         if (need_qt && (pg0 + pgl) < Pr - 1) {
           constexpr int CH = D / 8;
-          const int t = lane & 15, x = lane >> 4;
-          double acc[8];
+          const int grp = lane >> 2, t4 = lane & 3;
+          const int n_tiles = (2 * G + 7) / 8;
+          const double sqrt_d = sqrt((double)D);
+          const long long zoff = ((long long)(unsigned)sd[10]) | ((long long)sd[11] << 32);
+          for (int nt = 0; nt < n_tiles; ++nt) {
+            const int n = nt * 8 + grp;                           // B column held by this lane's group
+            const bool ncol = n < 2 * G;
+            const double* qrow = qt + (size_t)(ncol ? n : 0) * (D + QT_PAD) + 2 * t4;
+            double z00 = 0.0, z01 = 0.0, z10 = 0.0, z11 = 0.0;    // [m-tile][column pair]
+            const uint8_t* krow0 = tile + grp * GEO::ROW_BYTES + 4 * t4;
+            const uint8_t* krow1 = tile + (8 + grp) * GEO::ROW_BYTES + 4 * t4;
+#pragma unroll 4
+            for (int c = 0; c < CH; ++c) {
+              const uint32_t ka = *reinterpret_cast<const uint32_t*>(krow0 + ((c ^ grp) << 4));   // grp == token & 7
+              const uint32_t kb = *reinterpret_cast<const uint32_t*>(krow1 + ((c ^ grp) << 4));
+              const double2 qq = *reinterpret_cast<const double2*>(qrow + c * 8);
+              const double b0 = ncol ? qq.x : 0.0, b1 = ncol ? qq.y : 0.0;
+              dmma(z00, z01, (double)bf16_lo_f(ka), b0);
+              dmma(z10, z11, (double)bf16_lo_f(kb), b0);
+              dmma(z00, z01, (double)bf16_hi_f(ka), b1);
+              dmma(z10, z11, (double)bf16_hi_f(kb), b1);
+            }
+            // D fragment: row = grp (token), columns 2*t4, 2*t4 + 1
+            const int col = nt * 8 + 2 * t4;
+            z00 /= sqrt_d; z01 /= sqrt_d; z10 /= sqrt_d; z11 /= sqrt_d;
+            // the page's softmax partials per column: max and sum of exponentials over its 16 tokens
+            double m0 = fmax(z00, z10), m1 = fmax(z01, z11);
 #pragma unroll
-          for (int g = 0; g < 8; ++g) acc[g] = 0.0;
-          const uint8_t* krow = tile + t * GEO::ROW_BYTES;
-#pragma unroll 2
-          for (int c = 0; c < CH; ++c) {
-            const uint4 kk = *reinterpret_cast<const uint4*>(krow + ((c ^ (t & 7)) << 4));
-            double kd[8];
-            kd[0] = (double)bf16_lo_f(kk.x); kd[1] = (double)bf16_hi_f(kk.x);
-            kd[2] = (double)bf16_lo_f(kk.y); kd[3] = (double)bf16_hi_f(kk.y);
-            kd[4] = (double)bf16_lo_f(kk.z); kd[5] = (double)bf16_hi_f(kk.z);
-            kd[6] = (double)bf16_lo_f(kk.w); kd[7] = (double)bf16_hi_f(kk.w);
+            for (int o2 = 4; o2 < 32; o2 <<= 1) {
+              m0 = fmax(m0, __shfl_xor_sync(0xffffffffu, m0, o2));
+              m1 = fmax(m1, __shfl_xor_sync(0xffffffffu, m1, o2));
+            }
+            double e0 = exp(z00 - m0) + exp(z10 - m0), e1 = exp(z01 - m1) + exp(z11 - m1);
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              if (g < G) {
-                const double* qq = qt + (x * 8 + g) * D + c * 8;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[g] = fma(kd[e], qq[e], acc[g]);
+            for (int o2 = 4; o2 < 32; o2 <<= 1) {
+              e0 += __shfl_xor_sync(0xffffffffu, e0, o2);
+              e1 += __shfl_xor_sync(0xffffffffu, e1, o2);
+            }
+            if (col < 2 * G) {
+              double* z0 = p.zbuf + ((size_t)lh * p.max_batch_tokens + zoff + tok0 + grp) * (2 * G) + col;
+              double* z1 = z0 + (size_t)8 * (2 * G);
+              z0[0] = z00; z1[0] = z10;
+              if (col + 1 < 2 * G) { z0[1] = z01; z1[1] = z11; }
+              if (grp == 0) {
+                double* st2 = p.zstat + (((size_t)lh * (p.max_batch_tokens / GP_PAGE) + (zoff + tok0) / GP_PAGE) * (2 * G) + col) * 2;
+                st2[0] = m0; st2[1] = e0;
+                if (col + 1 < 2 * G) { st2[2] = m1; st2[3] = e1; }
               }
             }
           }
-          const double sqrt_d = sqrt((double)D);
-          const long long zoff = ((long long)(unsigned)sd[10]) | ((long long)sd[11] << 32);
-          double* zrow = p.zbuf + (((size_t)lh * p.max_batch_tokens + zoff + tok0 + t) * 2 + x) * G;
-#pragma unroll
-          for (int g = 0; g < 8; ++g)
-            if (g < G) zrow[g] = acc[g] / sqrt_d;
+          if (tr) { GP_T_ADD(8, GP_T_NOW() - t_d); GP_T_ADD(9, 1); }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[st]);
       }
-      // ---- merge the consumer warps ------------------------------------------------------------
+      if (!ok) break;
+      const long long t_e = GP_T_NOW();
+      (void)t_e;
+
+      // ---- hand the partial result to the merger warp ---------------------------------------------
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-      cons_sync();                      // everyone is done reading the previous item's merge buffer
+      const int cb = it % NCOMB;
+      if (!wait_bar(&comb_empty[cb], ((it / NCOMB) & 1u) ^ 1u, s_misc)) break;
+      float* my_comb = comb + (cb * NCW + cw) * comb_w;
       if (row < G) {
         if ((lane & 3) == 0) { my_comb[row] = m_run; my_comb[8 + row] = l_run; }
 #pragma unroll
         for (int jd = 0; jd < GEO::DTILES; ++jd) {
-          my_comb[16 + row * D + jd * 8 + qc] = o[jd][0] + o[jd][2];
-          my_comb[16 + row * D + jd * 8 + qc + 1] = o[jd][1] + o[jd][3];
+          *reinterpret_cast<float2*>(&my_comb[16 + row * D + jd * 8 + qc]) =
+              make_float2(o[jd][0] + o[jd][2], o[jd][1] + o[jd][3]);
         }
-      }
-      cons_sync();
-      const size_t out_row0 = (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
-      const int PSTRIDE = G * (D + 2);
-      const int rc_i = rc_i_slot;
-      float* part = p.partials + ((size_t)lh * n_rc + rc_i) * PSTRIDE;
-      for (int idx = ctid; idx < G * D; idx += CONS_THREADS) {
-        const int g = idx / D, dc = idx % D;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < NCW; ++w) M = fmaxf(M, comb[w * (GEO::COMB_WARP / 4) + g]);
-        float acc = 0.f, ls = 0.f;
-#pragma unroll
-        for (int w = 0; w < NCW; ++w) {
-          const float* base = comb + w * (GEO::COMB_WARP / 4);
-          const float wgt = exp2f(base[g] - M);
-          acc += wgt * base[16 + g * D + dc];
-          ls += wgt * base[8 + g];
-        }
-        if (nchunks == 1) {
-          out[out_row0 + idx] = acc / ls;
-        } else {
-          part[g * (D + 2) + dc] = acc;
-          if (dc == 0) { part[g * (D + 2) + D] = M; part[g * (D + 2) + D + 1] = ls; }
-        }
-      }
-      if (nchunks > 1) {
-        __threadfence();
-        cons_sync();
-        if (ctid == 0) {
-          int* cnt = p.unit_cnt + (size_t)bi * LH + lh;
-          const int prev = atomicAdd(cnt, 1);
-          s_misc[1] = (prev == nchunks - 1);
-          if (prev == nchunks - 1) *cnt = 0;
-        }
-        cons_sync();
-        if (s_misc[1]) {
-          __threadfence();
-          const float* first = p.partials + ((size_t)lh * n_rc + (rc_i - chunk)) * PSTRIDE;
-          for (int idx = ctid; idx < G * D; idx += CONS_THREADS) {
-            const int g = idx / D, dc = idx % D;
-            float M = -INFINITY;
-            for (int c = 0; c < nchunks; ++c) M = fmaxf(M, __ldcg(first + (size_t)c * PSTRIDE + g * (D + 2) + D));
-            float acc = 0.f, ls = 0.f;
-            for (int c = 0; c < nchunks; ++c) {
-              const float* pc = first + (size_t)c * PSTRIDE + g * (D + 2);
-              const float wgt = exp2f(__ldcg(pc + D) - M);
-              acc += wgt * __ldcg(pc + dc);
-              ls += wgt * __ldcg(pc + D + 1);
-            }
-            out[out_row0 + idx] = acc / ls;
-          }
-        }
-      }
-      if (need_qt) {
-        ++qt_uses;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(qt_empty);
       }
       __syncwarp();
+      if (lane == 0) mbar_arrive(&comb_full[cb]);
+      if (need_qt) {
+        ++qt_uses;
+        if (lane == 0) mbar_arrive(qt_empty);
+      }
       if (lane == 0) mbar_arrive(&slot_empty[sl]);
-      if (cons_any(!ok || s_misc[0] != 0)) break;        // same verdict in all four warps
+      if (tr) GP_T_ADD(5, GP_T_NOW() - t_e);
     }
-  } else {
+    if (tr) GP_T_ADD(6, GP_T_NOW() - t_loop0);
+  } else if (warp == 1) {
     // ================================= summaries ==========================================
     uint32_t qt_uses = 0;
     constexpr int PER = D / 32;
     for (uint32_t it = 0;; ++it) {
       const int sl = it % NI;
       if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc)) break;
-      const uint8_t* slot = smem + GEO::OFF_SLOTS + sl * GEO::SLOT_BYTES;
+      const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
       if (npg < 0) break;
@@ -504,7 +555,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
               }
               // Eq. 12
               const double gamma = ss > 0.0 ? sqrt(sq2 / (double)D) / sqrt(ss / (double)D) : 1.0;
-              double* dst = qt + (x * 8 + g) * D;
+              double* dst = qt + (size_t)(x * G + g) * (D + QT_PAD);
               if (p.rope_theta != 0.0) {
                 const double* cs = p.rope_cs + (size_t)bi * (D / 2) * 2;
 #pragma unroll
@@ -531,13 +582,89 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       __syncwarp();
       if (lane == 0) mbar_arrive(&slot_empty[sl]);
     }
+  } else if (warp == 2) {
+    // ================================= merger =============================================
+    for (uint32_t it = 0;; ++it) {
+      const int sl = it % NI;
+      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc)) break;
+      const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
+      const int* sd = reinterpret_cast<const int*>(slot);
+      const int npg = sd[3];
+      if (npg < 0) break;
+      const int bi = sd[0], chunk = sd[4], nchunks = sd[5], rc_i = sd[13], lh = sd[14];
+      const int l = lh / p.Hkv, h = lh % p.Hkv;
+      const int cb = it % NCOMB;
+      if (!wait_bar(&comb_full[cb], (it / NCOMB) & 1u, s_misc)) break;
+      const float* cbuf = comb + (size_t)cb * NCW * comb_w;
+      const size_t out_row0 = (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
+      const int PSTRIDE = G * (D + 2);
+      float* part = p.partials + ((size_t)lh * n_rc + rc_i) * PSTRIDE;
+      for (int g = 0; g < G; ++g) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NCW; ++w) M = fmaxf(M, cbuf[w * comb_w + g]);
+        float wgt[NCW];
+        float ls = 0.f;
+#pragma unroll
+        for (int w = 0; w < NCW; ++w) {
+          wgt[w] = exp2f(cbuf[w * comb_w + g] - M);
+          ls += wgt[w] * cbuf[w * comb_w + 8 + g];
+        }
+        const float inv = 1.f / ls;
+        for (int dc = lane; dc < D; dc += 32) {
+          float acc = 0.f;
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) acc += wgt[w] * cbuf[w * comb_w + 16 + g * D + dc];
+          if (nchunks == 1) out[out_row0 + g * D + dc] = acc * inv;
+          else part[g * (D + 2) + dc] = acc;
+        }
+        if (nchunks > 1 && lane == 0) { part[g * (D + 2) + D] = M; part[g * (D + 2) + D + 1] = ls; }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&comb_empty[cb]);
+      if (nchunks > 1) {
+        __syncwarp();                    // the lanes' partial stores are ordered before lane 0's release
+        int last = 0;
+        if (lane == 0) {
+          int* cnt = p.unit_cnt + (size_t)bi * LH + lh;
+          int prev;
+          asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(cnt) : "memory");
+          last = (prev == nchunks - 1);
+          if (last) *cnt = 0;
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+          const float* first = p.partials + ((size_t)lh * n_rc + (rc_i - chunk)) * PSTRIDE;
+          for (int g = 0; g < G; ++g) {
+            float M = -INFINITY;
+            for (int c = 0; c < nchunks; ++c) M = fmaxf(M, __ldcg(first + (size_t)c * PSTRIDE + g * (D + 2) + D));
+            float ls = 0.f;
+            for (int c = 0; c < nchunks; ++c) {
+              const float* pc = first + (size_t)c * PSTRIDE + g * (D + 2);
+              ls += exp2f(__ldcg(pc + D) - M) * __ldcg(pc + D + 1);
+            }
+            const float inv = 1.f / ls;
+            for (int dc = lane; dc < D; dc += 32) {
+              float acc = 0.f;
+              for (int c = 0; c < nchunks; ++c) {
+                const float* pc = first + (size_t)c * PSTRIDE + g * (D + 2);
+                acc += exp2f(__ldcg(pc + D) - M) * __ldcg(pc + dc);
+              }
+              out[out_row0 + g * D + dc] = acc * inv;
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&slot_empty[sl]);
+    }
   }
   __syncthreads();
 }
 
 }  // namespace
 
-size_t gp_attention_smem(int d) { return d == 128 ? Geo<128>::SMEM_BYTES : Geo<64>::SMEM_BYTES; }
+size_t gp_attention_smem(int d, int G) { return d == 128 ? make_lay<128>(G).total : make_lay<64>(G).total; }
 int gp_attention_ctas_per_sm(int d) { (void)d; return 2; }
 
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
@@ -547,11 +674,12 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
   const __nv_bfloat16* kk = static_cast<const __nv_bfloat16*>(k);
   const __nv_bfloat16* vv = static_cast<const __nv_bfloat16*>(v);
   const bool rope = p.rope_theta != 0.0;
-#define GP_LAUNCH(DD, RR)                                                                              \
-  do {                                                                                                 \
-    auto kern = gp_attn_kernel<DD, RR>;                                                                \
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<DD>::SMEM_BYTES);      \
-    kern<<<grid, NTHREADS, Geo<DD>::SMEM_BYTES, s>>>(p, n_req, qq, kk, vv, out);                      \
+  const int sm = (int)gp_attention_smem(p.d, p.G);
+#define GP_LAUNCH(DD, RR)                                                                 \
+  do {                                                                                    \
+    auto kern = gp_attn_kernel<DD, RR>;                                                   \
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);          \
+    kern<<<grid, NTHREADS, sm, s>>>(p, n_req, qq, kk, vv, out);                          \
   } while (0)
   if (p.d == 128) {
     if (rope) GP_LAUNCH(128, true); else GP_LAUNCH(128, false);

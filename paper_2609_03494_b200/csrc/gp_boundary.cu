@@ -23,8 +23,10 @@
 namespace {
 
 constexpr int NBINS = 2048;
+constexpr int NBINS_PAD = NBINS + NBINS / 8;     // bins are stored at b + (b >> 3): a thread's 8 consecutive bins and
+#define HIDX(b) ((b) + ((b) >> 3))              // its neighbours' then fall into different banks
 constexpr double TWO62 = 4611686018427387904.0;
-constexpr int SEL_T = 1024;          // threads of the selection kernel
+constexpr int SEL_T = 256;           // threads of the selection kernel
 constexpr int SEL_CAP = 6144;        // candidate tokens whose scores are staged in shared memory
 constexpr int CT = 256;              // threads of the compaction kernel
 constexpr int MOVE_TOK = GP_MOVE_TOK;     // source slots per compaction chunk
@@ -74,10 +76,21 @@ __device__ __forceinline__ unsigned block_prefix_excl(unsigned c, unsigned* wc) 
 
 __device__ __constant__ int kWidths[6] = {11, 11, 11, 11, 11, 8};   // 63 bits below the sign
 
+// 64-bit add into a (low, high) pair of 32-bit shared-memory words with two native atomics; the pair is
+// exact once all adds have landed (the carry travels with the high word's add).
+__device__ __forceinline__ void add64_split(unsigned* lo, unsigned* hi, unsigned long long x) {
+  const unsigned xl = (unsigned)x, xh = (unsigned)(x >> 32);
+  const unsigned old = atomicAdd(lo, xl);
+  const unsigned carry = (old + xl) < old ? 1u : 0u;
+  if (xh + carry) atomicAdd(hi, xh + carry);
+}
+
 // Eq. 7: smallest k such that the k largest of a[0..n) sum to at least p.
 template <int BT>
-__device__ int top_p_count(const double* a, int n, unsigned long long p_fix, unsigned* hcnt,
-                           unsigned long long* hsum, unsigned* wc, unsigned long long* wsum, long long* s_res) {
+__device__ int top_p_count(const GpDev& p, const double* a, int n, unsigned long long p_fix, unsigned* hcnt,
+                           unsigned long long* hsum64, unsigned* wc, unsigned long long* wsum, long long* s_res) {
+  unsigned* hlo = reinterpret_cast<unsigned*>(hsum64);
+  unsigned* hhi = hlo + NBINS_PAD;
   const int tid = threadIdx.x;
   unsigned long long prefix = 0;
   unsigned cnt_above = 0;
@@ -88,47 +101,54 @@ __device__ int top_p_count(const double* a, int n, unsigned long long p_fix, uns
     const int w = kWidths[lvl];
     shift -= w;
     const int nb = 1 << w;
-    for (int i = tid; i < nb; i += BT) { hcnt[i] = 0; hsum[i] = 0; }
+    const long long t_l0 = GP_T_NOW();
+    (void)t_l0;
+    for (int i = tid; i < nb + (nb >> 3); i += BT) { hcnt[i] = 0; hlo[i] = 0; hhi[i] = 0; }
     if (tid == 0) s_res[0] = -1;
     __syncthreads();
+    const long long t_l1 = GP_T_NOW();
+    (void)t_l1;
     for (int i = tid; i < n; i += BT) {
       const double v = a[i];
       const unsigned long long key = (unsigned long long)__double_as_longlong(v);
       if (lvl == 0 || (key >> (shift + w)) == prefix) {
         const int bin = (int)((key >> shift) & (unsigned long long)(nb - 1));
-        atomicAdd(&hcnt[bin], 1u);
-        atomicAdd(&hsum[bin], to_fix(v));
+        atomicAdd(&hcnt[HIDX(bin)], 1u);
+        add64_split(&hlo[HIDX(bin)], &hhi[HIDX(bin)], to_fix(v));
       }
     }
     __syncthreads();
+    const long long t_l2 = GP_T_NOW();
+    (void)t_l2;
     const int per = nb / BT > 0 ? nb / BT : 1;
     const int lo = tid * per, hi = lo + per;     // this thread's bins [lo, hi)
     unsigned c = 0; unsigned long long s = 0;
-    if (lo < nb) for (int b = lo; b < hi; ++b) { c += hcnt[b]; s += hsum[b]; }
+    if (lo < nb) for (int b = lo; b < hi; ++b) { c += hcnt[HIDX(b)]; s += ((unsigned long long)hhi[HIDX(b)] << 32) + hlo[HIDX(b)]; }
     PairCU ex = block_suffix_excl<BT>(c, s, wc, wsum);
     if (lo < nb) {
       unsigned long long run_s = sum_above + ex.s;
       unsigned run_c = cnt_above + ex.c;
       for (int b = hi - 1; b >= lo; --b) {
         const unsigned long long before = run_s;
-        run_s += hsum[b];
+        run_s += ((unsigned long long)hhi[HIDX(b)] << 32) + hlo[HIDX(b)];
         if (before < p_fix && run_s >= p_fix) { s_res[0] = b; s_res[1] = run_c; s_res[2] = (long long)before; }
-        run_c += hcnt[b];
+        run_c += hcnt[HIDX(b)];
       }
     }
     __syncthreads();
+    if (tid == 0) { GP_T_ADD(30, 1); GP_T_ADD(12, t_l1 - t_l0); GP_T_ADD(13, t_l2 - t_l1); GP_T_ADD(14, GP_T_NOW() - t_l2); }
     if (s_res[0] < 0) return n;                  // rounding kept the total below p: everything
     bin_star = (int)s_res[0];
     cnt_above = (unsigned)s_res[1];
     sum_above = (unsigned long long)s_res[2];
-    const unsigned cstar = hcnt[bin_star];
+    const unsigned cstar = hcnt[HIDX(bin_star)];
     __syncthreads();
     if (cstar == 1) return (int)cnt_above + 1;
     prefix = (prefix << w) | (unsigned long long)bin_star;
   }
   // all bits fixed: the bin holds copies of one value
-  const unsigned c = hcnt[bin_star];
-  const unsigned long long f = hsum[bin_star] / c;
+  const unsigned c = hcnt[HIDX(bin_star)];
+  const unsigned long long f = (((unsigned long long)hhi[HIDX(bin_star)] << 32) + hlo[HIDX(bin_star)]) / c;
   unsigned long long j = (p_fix - sum_above + f - 1) / f;
   if (j < 1) j = 1;
   if (j > c) j = c;
@@ -277,35 +297,60 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
 }
 
 // ------------------------------------------------------------------------------------------------------
-// working sets + speculative eviction list per unit; the last CTA decides
+// working sets + speculative eviction list; three independent jobs per unit, one CTA each; the last CTA decides
 // ------------------------------------------------------------------------------------------------------
 struct SelGeom {
-  static constexpr size_t SA_BYTES = 2 * SEL_CAP * sizeof(double);
-  static constexpr size_t H_BYTES = NBINS * 4 + NBINS * 8;
-  static constexpr size_t MISC_BYTES = 32 * 8 + 32 * 4 + 8 * 8 + 16 * 4 + 16 * 4;
+  static constexpr size_t BUF_BYTES = SEL_CAP * sizeof(double);
+  static constexpr size_t H_BYTES = NBINS_PAD * 4 + NBINS_PAD * 8;
+  static constexpr size_t MISC_BYTES = 8 * 8 + 8 * 4 + 8 * 8 + 16 * 4 + 16 * 4 + (8 * 16 + 32) * 8;
 };
+
+// max or sum over the block of one value per thread, separately for each of `ncols` interleaved columns
+// (thread t belongs to column t % ncols); fixed shuffle tree, so the sum does not depend on timing
+template <bool IS_MAX>
+__device__ __forceinline__ void column_reduce(double v, int ncols, double* red, double* result) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int off = ncols; off < 32; off <<= 1) {
+    const double o = __shfl_xor_sync(0xffffffffu, v, off);
+    v = IS_MAX ? fmax(v, o) : v + o;
+  }
+  if (lane < ncols) red[warp * 16 + lane] = v;
+  __syncthreads();
+  if (threadIdx.x < ncols) {
+    double r = red[threadIdx.x];
+    for (int w = 1; w < SEL_T / 32; ++w) r = IS_MAX ? fmax(r, red[w * 16 + threadIdx.x]) : r + red[w * 16 + threadIdx.x];
+    result[threadIdx.x] = r;
+  }
+  __syncthreads();
+}
 
 __global__ void __launch_bounds__(SEL_T)
 gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
-  double* sa = reinterpret_cast<double*>(smem);                                // [2][SEL_CAP]
-  unsigned* hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::SA_BYTES);
-  unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + NBINS);
-  unsigned long long* wsum = hsum + NBINS;                                     // [32]
-  unsigned* wc = reinterpret_cast<unsigned*>(wsum + 32);                       // [32]
-  long long* s_res = reinterpret_cast<long long*>(wc + 32);                    // [8]
+  double* sbuf = reinterpret_cast<double*>(smem);                              // [SEL_CAP] a^S, a^L or s
+  unsigned* hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::BUF_BYTES);
+  unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + NBINS_PAD);
+  unsigned long long* wsum = hsum + NBINS_PAD;                                 // [8]
+  unsigned* wc = reinterpret_cast<unsigned*>(wsum + 8);                        // [8]
+  long long* s_res = reinterpret_cast<long long*>(wc + 8);                     // [8]
   int* ev = reinterpret_cast<int*>(s_res + 8);                                 // [16]
   int* s_i = ev + 16;                                                          // [16]
-  unsigned* loc = reinterpret_cast<unsigned*>(s_i + 16);                       // [cap*b/32 + 1]
-  // the decision scratch aliases the score staging area: it is used after the last unit only
+  double* red = reinterpret_cast<double*>(s_i + 16);                           // [8][16]
+  double* sM = red + 8 * 16;                                                   // [16]
+  double* sZ = sM + 16;                                                        // [16]
+  unsigned* loc = reinterpret_cast<unsigned*>(sZ + 16);                        // [cap*b/32 + 1]
+  // the decision scratch aliases the score staging area: it is used after the last item only
 
   const int tid = threadIdx.x;
   const int LH = p.L * p.Hkv;
   const int n_bnd = p.hdr[HDR_N_BND];
-  const long long units = (long long)n_bnd * LH;
+  const long long items = (long long)n_bnd * LH * 3;
+  const int G = p.G, G2 = 2 * p.G;
 
-  for (long long u = blockIdx.x; u < units; u += gridDim.x) {
+  for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+    const long long u = item / 3;
+    const int task = (int)(item % 3);               // 0: K^S, 1: K^L, 2: eviction list
     const int bidx = (int)(u / LH), lh = (int)(u % LH);
     const int l = lh / p.Hkv, h = lh % p.Hkv;
     const int bi = p.bnd_list[bidx];
@@ -316,84 +361,94 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     int* evout = p.evict + (size_t)u * GP_PAGE;
     __syncthreads();
     if (nC == 0) {
-      if (tid == 0) { Kout[0] = 0; Kout[1] = 0; }
+      if (tid == 0 && task < 2) Kout[task] = 0;
       continue;
     }
+    const long long t_s0 = GP_T_NOW();
+    (void)t_s0;
     const long long off = p.bnd_off[bi];
-    const int G = p.G, G2 = 2 * p.G;
     const double* z = p.zbuf + ((size_t)lh * p.max_batch_tokens + off) * G2;      // [nC][2][G]
-    double* gS = p.scores + ((size_t)lh) * p.max_batch_tokens + off;
-    double* gL = p.scores + ((size_t)LH + lh) * p.max_batch_tokens + off;
-    double* aS = gS;
-    double* aL = gL;
-    if (nC <= SEL_CAP) { aS = sa; aL = sa + SEL_CAP; }
+    double* a = nC <= SEL_CAP ? sbuf : p.scores + ((size_t)task * LH + lh) * p.max_batch_tokens + off;
     // ---- per-head softmax over C, then the group mean (Sec. 3.2) --------------------------------------------
+    // The attention kernel left, per 16-token page and column, the page's (max, sum of exponentials); they
+    // merge into the normalisers of the whole candidate set without another pass over the logits.
     {
-      double* red = reinterpret_cast<double*>(hsum);          // [SEL_T] scratch, free until the histograms
-      double* sM = reinterpret_cast<double*>(hcnt);           // [16]
-      double* sZ = sM + 16;                                   // [16]
-      const int col = tid % G2;                               // SEL_T is a multiple of 2G
-      const size_t entries = (size_t)nC * G2;
+      const int ncols = task == 2 ? G2 : G;
+      const int col0 = task == 1 ? G : 0;
+      const int mycol = col0 + tid % ncols;                  // SEL_T is a multiple of ncols
+      const int ntile = nC / GP_PAGE;
+      const double* zs = p.zstat + ((size_t)lh * (p.max_batch_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
       double m = -INFINITY;
-      for (size_t e = tid; e < entries; e += SEL_T) m = fmax(m, __ldcg(z + e));
-      red[tid] = m;
-      __syncthreads();
-      if (tid < G2) {
-        double mm = -INFINITY;
-        for (int k2 = tid; k2 < SEL_T; k2 += G2) mm = fmax(mm, red[k2]);
-        sM[tid] = mm;
+      for (int t = tid / ncols; t < ntile; t += SEL_T / ncols) m = fmax(m, __ldcg(zs + ((size_t)t * G2 + mycol) * 2));
+      column_reduce<true>(m, ncols, red, sM);
+      const double mc = sM[tid % ncols];
+      double acc = 0.0;
+      for (int t = tid / ncols; t < ntile; t += SEL_T / ncols) {
+        const double2 ms = __ldcg(reinterpret_cast<const double2*>(zs + ((size_t)t * G2 + mycol) * 2));
+        acc += ms.y * exp(ms.x - mc);
       }
-      __syncthreads();
-      const double mc = sM[col];
-      double zs = 0.0;
-      for (size_t e = tid; e < entries; e += SEL_T) zs += exp(__ldcg(z + e) - mc);
-      __syncthreads();
-      red[tid] = zs;
-      __syncthreads();
-      if (tid < G2) {
-        double t = 0.0;
-        for (int k2 = tid; k2 < SEL_T; k2 += G2) t += red[k2];
-        sZ[tid] = t;
-      }
-      __syncthreads();
-      for (int i = tid; i < nC; i += SEL_T) {
-        const double* zr = z + (size_t)i * G2;
-        double s0 = 0.0, s1 = 0.0;
-        for (int g = 0; g < G; ++g) {
-          s0 += exp(__ldcg(zr + g) - sM[g]) / sZ[g];
-          s1 += exp(__ldcg(zr + G + g) - sM[G + g]) / sZ[G + g];
+      column_reduce<false>(acc, ncols, red, sZ);
+      for (int i0 = tid; i0 < nC; i0 += 4 * SEL_T) {         // four tokens per thread in flight
+        double zv[4][16];
+#pragma unroll
+        for (int u4 = 0; u4 < 4; ++u4) {
+          const int i = i0 + u4 * SEL_T;
+          if (i < nC) {
+            const double* zr = z + (size_t)i * G2 + col0;
+            for (int g = 0; g < ncols; ++g) zv[u4][g] = __ldcg(zr + g);
+          }
         }
-        aS[i] = s0 / (double)G;
-        aL[i] = s1 / (double)G;
+#pragma unroll
+        for (int u4 = 0; u4 < 4; ++u4) {
+          const int i = i0 + u4 * SEL_T;
+          if (i < nC) {
+            double s0 = 0.0, s1 = 0.0;
+            for (int g = 0; g < G; ++g) s0 += exp(zv[u4][g] - sM[g]) / sZ[g];
+            if (task == 2) {
+              for (int g = 0; g < G; ++g) s1 += exp(zv[u4][G + g] - sM[G + g]) / sZ[G + g];
+              a[i] = fmax(s0 / (double)G, s1 / (double)G);   // Eq. 9
+            } else {
+              a[i] = s0 / (double)G;
+            }
+          }
+        }
       }
       __syncthreads();
     }
+    const long long t_s1 = GP_T_NOW();
+    (void)t_s1;
+    if (task < 2) {
+      // ---- Eq. 7 -------------------------------------------------------------------------------------------
+      const int K = top_p_count<SEL_T>(p, a, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
+      if (tid == 0) {
+        Kout[task] = K;
+        GP_T_ADD(16, 1); GP_T_ADD(17, t_s1 - t_s0); GP_T_ADD(18, GP_T_NOW() - t_s1); GP_T_ADD(25, nC);
+      }
+      continue;
+    }
+    // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
     for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
     if (tid == 0) s_i[0] = 0;
     __syncthreads();
-    // ---- Eq. 7 ---------------------------------------------------------------------------------------------
-    const int KS = top_p_count<SEL_T>(aS, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
-    const int KL = top_p_count<SEL_T>(aL, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
-    if (tid == 0) { Kout[0] = KS; Kout[1] = KL; }
-
-    // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
     const int nblk = Pr - 1;
     const int K_t = nC - GP_PAGE;
     const int kq = min(p.k_loc, K_t / nblk);
     if (kq > 0) {
       for (int i = tid; i < nC; i += SEL_T) {
-        const double s = fmax(aS[i], aL[i]);                           // Eq. 9
+        const double s = a[i];
         const int b0 = i & ~15;
         int rank = 0;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const double sj = fmax(aS[b0 + j], aL[b0 + j]);
+          const double sj = a[b0 + j];
           rank += (sj > s) || (sj == s && (b0 + j) < i);
         }
         if (rank < kq) atomicOr(&loc[i >> 5], 1u << (i & 31));
       }
     }
     __syncthreads();
+    const long long t_s3 = GP_T_NOW();
+    (void)t_s3;
     // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
     unsigned long long prefix = 0;
     unsigned cnt_below = 0;
@@ -407,27 +462,27 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
         const int w = kWidths[lvl];
         shift -= w;
         const int nb = 1 << w;
-        for (int i = tid; i < nb; i += SEL_T) hcnt[i] = 0;
+        for (int i = tid; i < nb + (nb >> 3); i += SEL_T) hcnt[i] = 0;
         if (tid == 0) s_res[0] = -1;
         __syncthreads();
         for (int i = tid; i < nC; i += SEL_T) {
           if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-            const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(aS[i], aL[i]));
+            const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
             if (lvl == 0 || (key >> (shift + w)) == prefix)
-              atomicAdd(&hcnt[(int)((key >> shift) & (unsigned long long)(nb - 1))], 1u);
+              atomicAdd(&hcnt[HIDX((int)((key >> shift) & (unsigned long long)(nb - 1)))], 1u);
           }
         }
         __syncthreads();
         const int per = nb / SEL_T > 0 ? nb / SEL_T : 1;
         const int lo = tid * per, hi = lo + per;
         unsigned c = 0;
-        if (lo < nb) for (int b = lo; b < hi; ++b) c += hcnt[b];
+        if (lo < nb) for (int b = lo; b < hi; ++b) c += hcnt[HIDX(b)];
         const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
         if (lo < nb) {
           unsigned run = cnt_below + ex;
           for (int b = lo; b < hi; ++b) {
             const unsigned before = run;
-            run += hcnt[b];
+            run += hcnt[HIDX(b)];
             if (before < (unsigned)GP_PAGE && run >= (unsigned)GP_PAGE) { s_res[0] = b; s_res[1] = before; }
           }
         }
@@ -438,7 +493,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
         }
         const int bin_star = (int)s_res[0];
         cnt_below = (unsigned)s_res[1];
-        const unsigned cstar = hcnt[bin_star];
+        const unsigned cstar = hcnt[HIDX(bin_star)];
         __syncthreads();
         prefix = (prefix << w) | (unsigned long long)bin_star;
         if (cnt_below + cstar == (unsigned)GP_PAGE) {        // the bin fits exactly: no tie to break
@@ -452,29 +507,33 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
         need_eq = GP_PAGE - (int)cnt_below;
       }
     }
+    const long long t_s4 = GP_T_NOW();
+    (void)t_s4;
     for (int i = tid; i < nC; i += SEL_T) {
       if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-        const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(aS[i], aL[i]));
+        const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
         if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < GP_PAGE) ev[at] = i; }
       }
     }
     __syncthreads();
     if (tid == 0) {
+      GP_T_ADD(31, 1); GP_T_ADD(19, t_s3 - t_s1); GP_T_ADD(20, t_s4 - t_s3); GP_T_ADD(22, t_s1 - t_s0);
       int cntv = s_i[0];
       for (int i = nC - 1; i >= 0 && need_eq > 0; --i) {     // rare: older (lower) slots win ties
         if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-          const unsigned long long key = (unsigned long long)__double_as_longlong(fmax(aS[i], aL[i]));
+          const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
           if (key == tie_key) { if (cntv < GP_PAGE) ev[cntv] = i; ++cntv; --need_eq; }
         }
       }
       if (cntv != GP_PAGE) atomicOr(p.err, GP_E_BOUNDS);
-      for (int a = 1; a < GP_PAGE; ++a) {                    // sort the 16 slots ascending
-        const int key = ev[a];
-        int b2 = a - 1;
+      for (int x = 1; x < GP_PAGE; ++x) {                    // sort the 16 slots ascending
+        const int key = ev[x];
+        int b2 = x - 1;
         while (b2 >= 0 && ev[b2] > key) { ev[b2 + 1] = ev[b2]; --b2; }
         ev[b2 + 1] = key;
       }
-      for (int a = 0; a < GP_PAGE; ++a) evout[a] = ev[a];
+      for (int x = 0; x < GP_PAGE; ++x) evout[x] = ev[x];
+      GP_T_ADD(21, GP_T_NOW() - t_s4);
     }
   }
 
@@ -489,7 +548,10 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (s_i[2]) {
     __threadfence();
-    decide_and_allocate(p, req_ids, n_req, actions, reinterpret_cast<int*>(sa));
+    const long long t_d0 = GP_T_NOW();
+    (void)t_d0;
+    decide_and_allocate(p, req_ids, n_req, actions, reinterpret_cast<int*>(sbuf));
+    if (tid == 0) { GP_T_ADD(23, GP_T_NOW() - t_d0); GP_T_ADD(24, 1); }
   }
 }
 
@@ -592,7 +654,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         volatile int* prev = reinterpret_cast<volatile int*>(p.cflags + item - 1);
         unsigned it = 0;
         while (*prev != stamp && it < GP_SPIN_LIMIT) ++it;
-        if (it >= GP_SPIN_LIMIT) atomicOr(p.err, GP_E_SPIN);
+        if (it >= GP_SPIN_LIMIT) atomicOr(p.err, GP_E_SPIN_CMP);
         __threadfence();
       }
     }
@@ -661,7 +723,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 }  // namespace
 
 size_t gp_bsel_smem(const GpDev& p) {
-  return SelGeom::SA_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
+  return SelGeom::BUF_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
 }
 
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, int grid_sel, int grid_compact,

@@ -19,11 +19,11 @@
 #define GP_PAGE 16             // tokens per page (b)
 #define GP_ATTN_WARPS 4
 #define GP_ATTN_STAGES 3
-#define GP_SPIN_LIMIT (1u << 23)
+#define GP_SPIN_LIMIT (1u << 21)
 #define GP_MAX_REQ 1024        // upper limit of max_requests (shared-memory arrays are sized by it)
 #define GP_SCORE_TILE 128      // candidate tokens per boundary-scoring tile
 #define GP_MOVE_TOK 64         // source slots per compaction chunk
-#define GP_DESC_INTS 48        // ints per attention work descriptor: 16 header words + 32 page ids
+#define GP_DESC_INTS 16        // ints per attention work descriptor
 
 // plan header slots (int32)
 enum {
@@ -45,6 +45,7 @@ enum {
   GP_E_SPIN = 1,        // a bounded wait gave up
   GP_E_FREELIST = 2,    // free-list accounting went negative or overflowed
   GP_E_BOUNDS = 4,      // an index failed a bounds check and the access was skipped
+  GP_E_SPIN_CMP = 8,    // the compaction kernel's bounded wait on the previous chunk gave up
 };
 
 struct GpDev {
@@ -72,7 +73,7 @@ struct GpDev {
                                          //   0 batch index, 1 request, 2 first page, 3 pages, 4 chunk, 5 chunks,
                                          //   6 n before the append, 7 position, 8 flags (1 boundary, 2 started),
                                          //   9 P, 10-11 offset into the logit scratch, 12 summary buffer in use,
-                                         //   13 own index, 16.. page ids
+                                         //   13 own index
   int* b_nold;                           // [M] occupied slots before the append, by batch index
   int* b_flags;                          // [M] 1 = stepped this step
   int* first_idx;                        // [M] lowest batch index naming a request
@@ -83,14 +84,16 @@ struct GpDev {
   int* cmp_bnd;                          // [M] their index in bnd_list
   int* cmp_chunk0;                       // [M+1] prefix of their compaction chunk counts
   double* zbuf;                          // [L*H_kv][max_batch_tokens][2][G] summary logits of boundary units
+  double* zstat;                         // [L*H_kv][max_batch_tokens / b][2][G][2] per-page softmax partials (max, sum)
   int* sum_par;                          // [M] which of the two summary buffers is current
   int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
   int* cflags;                           // compaction chunk flags, stamped with the step number
   double* rope_cs;                       // [M][d/2][2] cos, sin at the step's position
   float* partials;
   double* scores;
-  long long* counters;                   // [8]
+  long long* counters;                   // [16]
   int* err;
+  long long* trace;                      // development builds only (-DGP_TRACE), else null
 };
 
 __device__ __forceinline__ size_t gp_tile_off(const GpDev& p, int l, long long page, int h) {
@@ -105,6 +108,16 @@ __device__ __forceinline__ size_t gp_summ_off(const GpDev& p, int l, int r, int 
   return ((((((size_t)l * p.M + r) * 2 + buf) * 2 + x) * p.Hq) + head) * (size_t)p.d;
 }
 
+// ---- optional cycle trace (compiled in only with -DGP_TRACE, for development builds) ----------------
+#ifdef GP_TRACE
+#define GP_TRACE_WORDS 32
+#define GP_T_ADD(slot, val) atomicAdd(reinterpret_cast<unsigned long long*>(&p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + (slot)]), (unsigned long long)(val))
+#define GP_T_NOW() clock64()
+#else
+#define GP_T_ADD(slot, val) do { } while (0)
+#define GP_T_NOW() 0ll
+#endif
+
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -116,15 +129,16 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
 }
-// non-blocking test of a phase: the bounded spins below must not rely on the hardware's own wait limit
+// One bounded hardware wait (the thread may be suspended for up to about a microsecond); the spins built
+// on it are bounded by an iteration limit on top.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
       : "memory");
   return ok != 0;
 }
@@ -174,7 +188,7 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 // ---- host-visible launchers (one per translation unit) -------------------------------------------
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
                          float* out, int grid, cudaStream_t s);
-size_t gp_attention_smem(int d);
+size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
 // boundary chain: probabilities + working sets + selection + decision, then compaction.
 // `ev`, when not null, is recorded between the two kernels.

@@ -11,7 +11,7 @@
 #include "../../include/growpage.h"
 #include "gp_dev.cuh"
 
-#define GP_SEL_GRID 148         // one 1024-thread CTA per SM
+#define GP_SEL_GRID 444         // three 256-thread CTAs per SM
 #define GP_COMPACT_GRID 592     // 4 CTAs per SM
 #define GP_PLAN_THREADS 1024
 
@@ -36,11 +36,22 @@ struct gp_pool {
   int64_t launch_count;
 };
 
+#ifdef GP_TRACE
+static long long* g_trace_dev = nullptr;
+extern "C" int gp_trace_read(long long* out, int reset) {
+  if (!g_trace_dev || cudaDeviceSynchronize() != cudaSuccess) return -1;
+  const size_t nb = sizeof(long long) * 1024 * GP_TRACE_WORDS;
+  if (cudaMemcpy(out, g_trace_dev, nb, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  if (reset) cudaMemset(g_trace_dev, 0, nb);
+  return 0;
+}
+#endif
+
 namespace {
 
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
-      b_flags, unit_cnt, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, zbuf, sum_par,
+      b_flags, unit_cnt, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, zbuf, zstat, sum_par,
       evict, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
   int max_rc;
@@ -51,7 +62,7 @@ inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 int chunk_pages_setting() {
   const char* e = getenv("GP_CHUNK_PAGES");
-  int v = e ? atoi(e) : 16;
+  int v = e ? atoi(e) : 32;
   if (v < 1) v = 1;
   if (v > 32) v = 32;
   return v;
@@ -109,11 +120,12 @@ Layout make_layout(const gp_config& c) {
   L.cmp_bnd = take(M * 4);
   L.cmp_chunk0 = take((M + 1) * 4);
   L.zbuf = take(LH * (size_t)L.max_batch_tokens * 2 * G * 8);
+  L.zstat = take(LH * ((size_t)L.max_batch_tokens / b + 1) * 2 * G * 2 * 8);
   L.evict = take(M * LH * b * 4);
   L.cflags = take(LH * ((size_t)L.max_batch_tokens / GP_MOVE_TOK + 2 * M + 1) * 4);
   L.rope_cs = take(M * (d / 2) * 2 * 8);
   L.partials = take((size_t)L.max_rc * LH * G * (d + 2) * 4);
-  L.scores = take(2 * LH * (size_t)L.max_batch_tokens * 8);
+  L.scores = take(3 * LH * (size_t)L.max_batch_tokens * 8);
   L.counters = take(16 * 8);
   L.dbg = take(cap * b * (4 + 2 * d * 2));
   if (c.host_staging) {
@@ -142,7 +154,7 @@ __global__ void gp_init_kernel(GpDev p) {
   if (i0 == 0) *p.free_top = (int)p.n_pages;
 }
 
-// exclusive scan over the CTA (1024 threads) of an int and a long long
+// exclusive scan over the CTA (1024 threads) of an int and a long long; also returns the totals
 __device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long& ew, int& tv, long long& tw,
                                           int* sv, long long* sw) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -155,30 +167,39 @@ __device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long
   }
   if (lane == 31) { sv[warp] = iv; sw[warp] = iw; }
   __syncthreads();
-  int bv = 0; long long bw = 0;
-  tv = 0; tw = 0;
-  for (int i = 0; i < GP_PLAN_THREADS / 32; ++i) {
-    if (i < warp) { bv += sv[i]; bw += sw[i]; }
-    tv += sv[i]; tw += sw[i];
+  if (warp == 0) {                       // scan of the 32 warp totals: exclusive prefix in [0..31], total in [32]
+    int xv = sv[lane]; long long xw = sw[lane];
+    const int ov = xv; const long long ow = xw;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, xv, off);
+      const long long b2 = __shfl_up_sync(0xffffffffu, xw, off);
+      if (lane >= off) { xv += a; xw += b2; }
+    }
+    sv[lane] = xv - ov; sw[lane] = xw - ow;
+    if (lane == 31) { sv[32] = xv; sw[32] = xw; }
   }
-  ev = bv + iv - v;
-  ew = bw + iw - w;
+  __syncthreads();
+  ev = sv[warp] + iv - v;
+  ew = sw[warp] + iw - w;
+  tv = sv[32];
+  tw = sw[32];
   __syncthreads();
 }
 
-// Step plan: validates the batch, cuts every stepped request into chunks and writes one self-contained work
-// descriptor per chunk for the attention kernel, lists the requests that reach their capacity boundary
-// with this step's append (trailing check: n + 1 == P b) and hands each a slice of the logit scratch.
+// Step plan: validates the batch, cuts every stepped request into chunks and writes one work descriptor
+// per chunk for the attention kernel, lists the requests that reach their capacity boundary with this
+// step's append (trailing check: n + 1 == P b) and hands each a slice of the logit scratch.
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
-  __shared__ int sv[32];
-  __shared__ long long sw[32];
-  __shared__ int s_rcoff[GP_MAX_REQ], s_chunks[GP_MAX_REQ], s_pages[GP_MAX_REQ], s_nold[GP_MAX_REQ];
-  int* s_first = s_rcoff;          // lowest batch index naming a request; dead before s_rcoff is written
-  __shared__ int s_flags[GP_MAX_REQ], s_P[GP_MAX_REQ], s_r[GP_MAX_REQ], s_pos[GP_MAX_REQ], s_par[GP_MAX_REQ];
-  __shared__ long long s_zoff[GP_MAX_REQ];
+  __shared__ int sv[33];
+  __shared__ long long sw[33];
+  __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
+  __shared__ int s_chunks[GP_MAX_REQ], s_pos[GP_MAX_REQ];
   const int i = threadIdx.x;
   const bool in = i < n_req;
+  const long long t_plan0 = GP_T_NOW();
+  (void)t_plan0;
   s_first[i] = 0x7fffffff;
   __syncthreads();
   int r = -1;
@@ -207,6 +228,8 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       if (n_old + 1 == Pr * GP_PAGE) { isb = 1; nc = (long long)(Pr - 1) * GP_PAGE; }
     }
   }
+  const long long t_plan1 = GP_T_NOW();
+  (void)t_plan1;
   int rc_off, n_rc; long long tok_off, tok_tot;
   plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
   if (isb && tok_off + nc > p.max_batch_tokens) { isb = 0; act = GP_ACT_SCRATCH; }
@@ -214,54 +237,30 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     atomicOr(p.err, GP_E_BOUNDS);
     chunks = 0; isb = 0; act = GP_ACT_SCRATCH;
   }
-  int bnd_idx, n_bnd, act_idx, n_active; long long d0, d1;
+  int bnd_idx, n_bnd, n_active; long long d0, d1;
   plan_scan(isb, chunks > 0, bnd_idx, d0, n_bnd, d1, sv, sw);
-  act_idx = (int)d0; n_active = (int)d1;
-  (void)act_idx;
-  s_rcoff[i] = rc_off; s_chunks[i] = chunks; s_pages[i] = pages; s_nold[i] = n_old;
-  s_flags[i] = isb | (started ? 2 : 0); s_P[i] = Pr; s_r[i] = r; s_pos[i] = (int)pos; s_par[i] = par;
-  s_zoff[i] = tok_off;
+  n_active = (int)d1;
+  const long long t_plan2 = GP_T_NOW();
+  (void)t_plan2;
+  s_chunks[i] = chunks; s_pos[i] = (int)pos;
   if (in) {
     p.b_nold[i] = n_old;
     p.b_flags[i] = chunks > 0;
     actions[i] = act;
     if (isb) { p.bnd_list[bnd_idx] = i; p.bnd_off[i] = tok_off; }
-  }
-  __syncthreads();
-  // descriptors: one warp per request, lanes across the words
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int bi = warp; bi < n_req; bi += GP_PLAN_THREADS / 32) {
-    const int nch = s_chunks[bi];
-    if (nch == 0) continue;
-    const int rr = s_r[bi];
-    const int* table = p.page_table + (size_t)rr * p.cap;
-    for (int c = 0; c < nch; ++c) {
+    // descriptors of this request's chunks: four 16-byte stores each
+    const int flags = isb | (started ? 2 : 0);
+    for (int c = 0; c < chunks; ++c) {
       const int pg0 = c * p.chunk_pages;
-      const int npg = min(p.chunk_pages, s_pages[bi] - pg0);
-      int* d = p.rcx + (size_t)(s_rcoff[bi] + c) * GP_DESC_INTS;
-      int hv = 0;
-      switch (lane) {
-        case 0: hv = bi; break;
-        case 1: hv = rr; break;
-        case 2: hv = pg0; break;
-        case 3: hv = npg; break;
-        case 4: hv = c; break;
-        case 5: hv = nch; break;
-        case 6: hv = s_nold[bi]; break;
-        case 7: hv = s_pos[bi]; break;
-        case 8: hv = s_flags[bi]; break;
-        case 9: hv = s_P[bi]; break;
-        case 10: hv = (int)(unsigned)(s_zoff[bi] & 0xffffffffLL); break;
-        case 11: hv = (int)(s_zoff[bi] >> 32); break;
-        case 12: hv = s_par[bi]; break;
-        case 13: hv = s_rcoff[bi] + c; break;
-        default: break;
-      }
-      if (lane < 16) d[lane] = hv;
-      d[16 + lane] = lane < npg ? table[pg0 + lane] : -1;
+      int4* d = reinterpret_cast<int4*>(p.rcx + (size_t)(rc_off + c) * GP_DESC_INTS);
+      d[0] = make_int4(i, r, pg0, min(p.chunk_pages, pages - pg0));
+      d[1] = make_int4(c, chunks, n_old, (int)pos);
+      d[2] = make_int4(flags, Pr, (int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32));
+      d[3] = make_int4(par, rc_off + c, 0, 0);
     }
   }
   if (p.rope_theta != 0.0) {                                      // cos / sin of the step's position
+    __syncthreads();
     const int half = p.d / 2;
     for (int idx = threadIdx.x; idx < n_req * half; idx += GP_PLAN_THREADS) {
       const int bi = idx / half, j = idx % half;
@@ -276,6 +275,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     }
   }
   if (threadIdx.x == 0) {
+    GP_T_ADD(26, 1); GP_T_ADD(27, t_plan1 - t_plan0); GP_T_ADD(28, t_plan2 - t_plan1); GP_T_ADD(29, GP_T_NOW() - t_plan2);
     p.hdr[HDR_N_RC] = n_rc;
     p.hdr[HDR_N_BND] = n_bnd;
     p.hdr[HDR_WORK_ATTN] = 0;
@@ -480,6 +480,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.cmp_bnd = reinterpret_cast<int*>(base + L.cmp_bnd);
   d.cmp_chunk0 = reinterpret_cast<int*>(base + L.cmp_chunk0);
   d.zbuf = reinterpret_cast<double*>(base + L.zbuf);
+  d.zstat = reinterpret_cast<double*>(base + L.zstat);
   d.sum_par = reinterpret_cast<int*>(base + L.sum_par);
   d.evict = reinterpret_cast<int*>(base + L.evict);
   d.cflags = reinterpret_cast<int*>(base + L.cflags);
@@ -487,6 +488,14 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.partials = reinterpret_cast<float*>(base + L.partials);
   d.scores = reinterpret_cast<double*>(base + L.scores);
   d.counters = reinterpret_cast<long long*>(base + L.counters);
+  d.trace = nullptr;
+#ifdef GP_TRACE
+  if (!g_trace_dev) {
+    cudaMalloc(&g_trace_dev, sizeof(long long) * 1024 * GP_TRACE_WORDS);
+    cudaMemset(g_trace_dev, 0, sizeof(long long) * 1024 * GP_TRACE_WORDS);
+  }
+  d.trace = g_trace_dev;
+#endif
   pool->dbg = base + L.dbg;
   if (cfg->host_staging) {
     pool->st_ids = reinterpret_cast<int*>(base + L.st_ids);
