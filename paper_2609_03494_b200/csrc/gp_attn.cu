@@ -3,10 +3,11 @@
 // summaries against every candidate key (Eq. 12, App. D.1) while the key tile is in shared memory.
 //
 // Work decomposition.  The plan kernel cuts every stepped request into chunks of `chunk_pages` pages and
-// writes one descriptor per chunk; a work item is (chunk, layer, KV head).  A persistent grid (two CTAs
-// per SM) pulls items from a global counter.  Each CTA is warp-specialised:
+// writes one descriptor per chunk, sorted by descending cost; a work item is (chunk, layer, KV head).  A
+// persistent grid (two CTAs per SM) deals the items out round by round, alternating the CTA order so that
+// every CTA gets about the same total.  Each CTA is warp-specialised:
 //
-//   warp 0      producer: claims items, publishes their descriptor in a ring of item slots, and streams
+//   warp 0      producer: takes its items (a static deal of the cost-sorted list), publishes their descriptor in a ring of item slots, and streams
 //               the K|V tiles of their pages (one contiguous `cp.async.bulk` per (layer, page, head))
 //               into a ring of stages shared by the CTA.  It runs ahead across item boundaries, so the
 //               ring never drains between items.
@@ -19,8 +20,8 @@
 //   warp 1      summaries: Eq. 6 on the un-rotated query (read from one of two buffers, written to the
 //               other, so that every item of a unit sees the old state), and for boundary units the
 //               calibrated, rotated summaries q~ in fp64 for the consumers.
-//   warp 2      merger: combines the four consumers' partial (max, sum, O) of an item, writes the output
-//               or, for requests split over several items, the partial and, as last arrival, the merge.
+//   warp 2      merger: combines the four consumers' partial (max, sum, O) of an item and writes the output
+//               or, for requests split over several items, the partial (the next kernel merges those).
 //               Consumers hand over through a double buffer and go straight on to the next item.
 //
 // The two warp groups re-split the register file (setmaxnreg): the service warps keep 56 registers per
@@ -112,6 +113,9 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   const int comb_w = L.comb_warp / 4;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef GP_TRACE
+  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 7] = (long long)gt; }
+#endif
   if (tid == 0) {
     for (int i = 0; i < NCW * NSW; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < NI_MAX; ++i) { mbar_init(&slot_full[i], 1); mbar_init(&slot_empty[i], NCW + 2); }
@@ -138,49 +142,49 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     // Software pipeline over items, one stage per tick, so that no global round trip sits between two
     // tiles: claim (t), descriptor header (t-1), page ids (t-2), publish the item slot (t-3), stream its
     // tiles (t-4).  The loads of the young stages are in flight while the oldest item streams.
-    long long itA = total, itB = total, itC = total, itD = total, itE = total;   // claimed item per stage
-    int hB = 0, hC = 0, hD = 0, hE = 0;        // descriptor header, word `lane` (lanes 0..15)
-    int pC = -1, pD = -1, pE = -1;             // page id of tile `lane` of the item
+    // Stages: A = item known, header load issued; B = header here: slot published, page ids requested;
+    // C = page ids here: last page id written to the slot; D = tiles streamed.  The first item of a CTA
+    // is its block index, later ones come from the global counter.
+    const long long grid = gridDim.x;
+    long long itA = blockIdx.x, itB = total, itC = total, itD = total;
+    int hB = 0, hC = 0, hD = 0;                // descriptor header, word `lane` (lanes 0..15)
+    int pC = -1, pD = -1;                      // page id of tile `lane` of the item
+    int slC = 0;                               // slot of the item in stage C
     uint32_t wf0 = 0, wf1 = 0, wf2 = 0, wf3 = 0;   // tiles issued so far to each consumer warp
     uint32_t n_pub = 0;
     bool sentinel_out = false;
     for (uint32_t tick = 0;; ++tick) {
       // ---- issue the loads of the young stages --------------------------------------------------
-      long long claimed = 0;
-      if (lane == 0) claimed = atomicAdd(&p.hdr[HDR_WORK_ATTN], 1);
       int hNew = 0;
-      if (itA < total && lane < GP_DESC_INTS) hNew = p.rcx[(size_t)(itA % n_rc) * GP_DESC_INTS + lane];
+      if (itA < total && lane < GP_DESC_INTS) hNew = p.rcx[(size_t)(itA / LH) * GP_DESC_INTS + lane];
       int pNew = -1;
-      if (itB < total) {
-        const int r = __shfl_sync(0xffffffffu, hB, 1), pg0 = __shfl_sync(0xffffffffu, hB, 2);
-        const int npg = __shfl_sync(0xffffffffu, hB, 3);
-        if (lane < npg) pNew = p.page_table[(size_t)r * p.cap + pg0 + lane];
-      }
-      // ---- publish the slot of the item two stages from streaming ---------------------------------
-      if (tick >= 3 && !sentinel_out) {
+      int slNew = 0;
+      // ---- header of stage B has arrived: load its page ids and publish its slot --------------------
+      if (tick >= 1 && !sentinel_out) {
         const int sl = n_pub % NI;
+        slNew = sl;
         const long long t_p0 = GP_T_NOW();
         (void)t_p0;
         if (!wait_bar(&slot_empty[sl], ((n_pub / NI) & 1u) ^ 1u, s_misc)) break;
         if (lane == 0) GP_T_ADD(11, GP_T_NOW() - t_p0);
         uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
         int* sd = reinterpret_cast<int*>(slot);
-        if (itC >= total) {
+        if (itB >= total) {
           if (lane == 0) sd[3] = -1;
           __syncwarp();
           if (lane == 0) mbar_arrive(&slot_full[sl]);
           sentinel_out = true;
         } else {
-          const int lh = (int)(itC / n_rc);
+          const int lh = (int)(itB % LH);
           const int l = lh / p.Hkv, h = lh % p.Hkv;
-          const int bi = __shfl_sync(0xffffffffu, hC, 0);
-          const int npg = __shfl_sync(0xffffffffu, hC, 3);
-          const int chunk = __shfl_sync(0xffffffffu, hC, 4);
-          const int nchunks = __shfl_sync(0xffffffffu, hC, 5);
-          const int last_pg = __shfl_sync(0xffffffffu, pC, (npg - 1) & 31);
-          if (lane < 14) sd[lane] = hC;
+          const int bi = __shfl_sync(0xffffffffu, hB, 0);
+          const int r = __shfl_sync(0xffffffffu, hB, 1), pg0 = __shfl_sync(0xffffffffu, hB, 2);
+          const int npg = __shfl_sync(0xffffffffu, hB, 3);
+          const int chunk = __shfl_sync(0xffffffffu, hB, 4);
+          const int nchunks = __shfl_sync(0xffffffffu, hB, 5);
+          if (lane < npg) pNew = p.page_table[(size_t)r * p.cap + pg0 + lane];
+          if (lane < 14) sd[lane] = hB;
           if (lane == 14) sd[14] = lh;
-          if (lane == 16) sd[16] = last_pg;
           __syncwarp();
           if (lane == 0) {
             const bool has_new = (chunk == nchunks - 1);
@@ -196,10 +200,16 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         }
         ++n_pub;
       }
+      // ---- page ids of stage C have arrived: the consumer that appends needs the last one ------------
+      if (itC < total) {
+        const int npg = __shfl_sync(0xffffffffu, hC, 3);
+        const int last_pg = __shfl_sync(0xffffffffu, pC, (npg - 1) & 31);
+        if (lane == 0) reinterpret_cast<int*>(smem + L.off_slots + slC * GEO::SLOT_BYTES)[16] = last_pg;
+      }
       // ---- stream the tiles of the oldest item ----------------------------------------------------------
-      if (tick >= 4) {
+      if (tick >= 3) {
         if (itD >= total) break;
-        const int lh = (int)(itD / n_rc);
+        const int lh = (int)(itD % LH);
         const int l = lh / p.Hkv, h = lh % p.Hkv;
         const int npg = __shfl_sync(0xffffffffu, hD, 3);
         bool ok = true;
@@ -222,12 +232,14 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         if (!ok) break;
       }
       // ---- rotate -----------------------------------------------------------------------------------------
-      itE = itD; hE = hD; pE = pD;
       itD = itC; hD = hC; pD = pC;
-      itC = itB; hC = hB; pC = pNew;
+      itC = itB; hC = hB; pC = pNew; slC = slNew;
       itB = itA; hB = hNew;
-      itA = __shfl_sync(0xffffffffu, claimed, 0);
-      (void)itE; (void)hE; (void)pE;
+      {   // static schedule: items are sorted by descending cost; round k goes to the CTAs in alternating order
+        const long long kk = (long long)tick + 1;
+        itA = kk * grid + ((kk & 1) ? grid - 1 - (long long)blockIdx.x : (long long)blockIdx.x);
+        if (itA >= total) itA = total;
+      }
     }
     if (s_misc[0]) {
       // aborted: let the copies already issued land before the CTA goes away
@@ -428,20 +440,30 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
             const int n = nt * 8 + grp;                           // B column held by this lane's group
             const bool ncol = n < 2 * G;
             const double* qrow = qt + (size_t)(ncol ? n : 0) * (D + QT_PAD) + 2 * t4;
-            double z00 = 0.0, z01 = 0.0, z10 = 0.0, z11 = 0.0;    // [m-tile][column pair]
+            double z00 = 0.0, z01 = 0.0, z10 = 0.0, z11 = 0.0;    // [m-tile][column pair], even chunks
+            double y00 = 0.0, y01 = 0.0, y10 = 0.0, y11 = 0.0;    // odd chunks: four independent DMMA chains
             const uint8_t* krow0 = tile + grp * GEO::ROW_BYTES + 4 * t4;
             const uint8_t* krow1 = tile + (8 + grp) * GEO::ROW_BYTES + 4 * t4;
 #pragma unroll 4
-            for (int c = 0; c < CH; ++c) {
+            for (int c = 0; c < CH; c += 2) {
               const uint32_t ka = *reinterpret_cast<const uint32_t*>(krow0 + ((c ^ grp) << 4));   // grp == token & 7
               const uint32_t kb = *reinterpret_cast<const uint32_t*>(krow1 + ((c ^ grp) << 4));
+              const uint32_t kc = *reinterpret_cast<const uint32_t*>(krow0 + (((c + 1) ^ grp) << 4));
+              const uint32_t kd = *reinterpret_cast<const uint32_t*>(krow1 + (((c + 1) ^ grp) << 4));
               const double2 qq = *reinterpret_cast<const double2*>(qrow + c * 8);
+              const double2 qr = *reinterpret_cast<const double2*>(qrow + c * 8 + 8);
               const double b0 = ncol ? qq.x : 0.0, b1 = ncol ? qq.y : 0.0;
+              const double b2 = ncol ? qr.x : 0.0, b3 = ncol ? qr.y : 0.0;
               dmma(z00, z01, (double)bf16_lo_f(ka), b0);
               dmma(z10, z11, (double)bf16_lo_f(kb), b0);
+              dmma(y00, y01, (double)bf16_lo_f(kc), b2);
+              dmma(y10, y11, (double)bf16_lo_f(kd), b2);
               dmma(z00, z01, (double)bf16_hi_f(ka), b1);
               dmma(z10, z11, (double)bf16_hi_f(kb), b1);
+              dmma(y00, y01, (double)bf16_hi_f(kc), b3);
+              dmma(y10, y11, (double)bf16_hi_f(kd), b3);
             }
+            z00 += y00; z01 += y01; z10 += y10; z11 += y11;
             // D fragment: row = grp (token), columns 2*t4, 2*t4 + 1
             const int col = nt * 8 + 2 * t4;
             z00 /= sqrt_d; z01 /= sqrt_d; z10 /= sqrt_d; z11 /= sqrt_d;
@@ -503,6 +525,9 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       if (tr) GP_T_ADD(5, GP_T_NOW() - t_e);
     }
     if (tr) GP_T_ADD(6, GP_T_NOW() - t_loop0);
+#ifdef GP_TRACE
+    if (tr) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 28] = (long long)gt; }
+#endif
   } else if (warp == 1) {
     // ================================= summaries ==========================================
     uint32_t qt_uses = 0;
@@ -533,16 +558,22 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
             qv[e] = (double)__bfloat162float(qrow[lane + 32 * e]);
             sq += qv[e] * qv[e];
           }
+          double ov[2][PER];
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {                       // both views' loads in flight together
+            const double* oldp = p.summ + gp_summ_off(p, l, r, par, x, head);
+#pragma unroll
+            for (int e = 0; e < PER; ++e) ov[x][e] = started ? __ldcg(oldp + lane + 32 * e) : 0.0;
+          }
 #pragma unroll
           for (int x = 0; x < 2; ++x) {
             const double beta = x ? p.beta_l : p.beta_s;
-            const double* oldp = p.summ + gp_summ_off(p, l, r, par, x, head);
             double* newp = p.summ + gp_summ_off(p, l, r, par ^ 1, x, head);
             double nv[PER];
             double ss = 0.0;
 #pragma unroll
             for (int e = 0; e < PER; ++e) {
-              nv[e] = started ? beta * oldp[lane + 32 * e] + (1.0 - beta) * qv[e] : qv[e];     // Eq. 6
+              nv[e] = started ? beta * ov[x][e] + (1.0 - beta) * qv[e] : qv[e];     // Eq. 6
               if (chunk == 0) newp[lane + 32 * e] = nv[e];
               ss += nv[e] * nv[e];
             }
@@ -591,7 +622,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
       if (npg < 0) break;
-      const int bi = sd[0], chunk = sd[4], nchunks = sd[5], rc_i = sd[13], lh = sd[14];
+      const int bi = sd[0], nchunks = sd[5], rc_i = sd[13], lh = sd[14];
       const int l = lh / p.Hkv, h = lh % p.Hkv;
       const int cb = it % NCOMB;
       if (!wait_bar(&comb_full[cb], (it / NCOMB) & 1u, s_misc)) break;
@@ -622,44 +653,18 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&comb_empty[cb]);
-      if (nchunks > 1) {
-        __syncwarp();                    // the lanes' partial stores are ordered before lane 0's release
-        int last = 0;
-        if (lane == 0) {
-          int* cnt = p.unit_cnt + (size_t)bi * LH + lh;
-          int prev;
-          asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(cnt) : "memory");
-          last = (prev == nchunks - 1);
-          if (last) *cnt = 0;
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-          const float* first = p.partials + ((size_t)lh * n_rc + (rc_i - chunk)) * PSTRIDE;
-          for (int g = 0; g < G; ++g) {
-            float M = -INFINITY;
-            for (int c = 0; c < nchunks; ++c) M = fmaxf(M, __ldcg(first + (size_t)c * PSTRIDE + g * (D + 2) + D));
-            float ls = 0.f;
-            for (int c = 0; c < nchunks; ++c) {
-              const float* pc = first + (size_t)c * PSTRIDE + g * (D + 2);
-              ls += exp2f(__ldcg(pc + D) - M) * __ldcg(pc + D + 1);
-            }
-            const float inv = 1.f / ls;
-            for (int dc = lane; dc < D; dc += 32) {
-              float acc = 0.f;
-              for (int c = 0; c < nchunks; ++c) {
-                const float* pc = first + (size_t)c * PSTRIDE + g * (D + 2);
-                acc += exp2f(__ldcg(pc + D) - M) * __ldcg(pc + dc);
-              }
-              out[out_row0 + g * D + dc] = acc * inv;
-            }
-          }
-        }
-      }
       __syncwarp();
       if (lane == 0) mbar_arrive(&slot_empty[sl]);
     }
   }
+#ifdef GP_TRACE
+  if (lane == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 16 + warp] = (long long)gt; }
+#endif
   __syncthreads();
+#ifdef GP_TRACE
+  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 15] = (long long)gt; }
+  if (tid == 128) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 29] = (long long)gt; }
+#endif
 }
 
 }  // namespace

@@ -2,7 +2,8 @@
 // The attention kernel has already left, for every (request at a boundary, layer, KV head) unit, the
 // fp64 logits z of the two calibrated summaries against every candidate key.
 //
-//   gp_bsel_kernel    per unit: per-head softmax over the candidate set and group mean -> a^S, a^L;
+//   gp_bsel_kernel    first merges the partial attention outputs of requests split over several work items;
+//                     then, per unit: per-head softmax over the candidate set and group mean -> a^S, a^L;
 //                     working-set sizes K^S, K^L (Eq. 7); and, speculatively, the b slots a compression
 //                     would evict (Eq. 9, Eq. 10).  The last CTA to finish aggregates Eq. 8, decides grow
 //                     or compress per request and runs the device allocator: grants first, then
@@ -325,7 +326,8 @@ __device__ __forceinline__ void column_reduce(double v, int ncols, double* red, 
 }
 
 __global__ void __launch_bounds__(SEL_T)
-gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
+gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
+               float* __restrict__ out) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
   double* sbuf = reinterpret_cast<double*>(smem);                              // [SEL_CAP] a^S, a^L or s
@@ -347,6 +349,34 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const int n_bnd = p.hdr[HDR_N_BND];
   const long long items = (long long)n_bnd * LH * 3;
   const int G = p.G, G2 = 2 * p.G;
+
+  // ---- attention outputs of requests that were split over several work items: merge the partials -----------
+  {
+    const int n_mc = p.hdr[HDR_N_MC], n_rc = p.hdr[HDR_N_RC], D = p.d;
+    const int PSTRIDE = G * (D + 2);
+    for (long long mi = blockIdx.x; mi < (long long)n_mc * LH; mi += gridDim.x) {
+      const int4 mc = p.mc_list[mi / LH];
+      const int lh = (int)(mi % LH), l = lh / p.Hkv, h = lh % p.Hkv;
+      const int bi = mc.x, nch = mc.z;
+      const float* first = p.partials + ((size_t)lh * n_rc + mc.y) * PSTRIDE;
+      float* orow = out + (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
+      for (int idx = tid; idx < G * D; idx += SEL_T) {
+        const int g = idx / D, dc = idx % D;
+        const float* pg = first + g * (D + 2);
+        float M = -INFINITY;
+        for (int c = 0; c < nch; ++c) M = fmaxf(M, __ldcg(pg + (size_t)c * PSTRIDE + D));
+        float acc = 0.f, ls = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < nch; ++c) {
+          const float* pc = pg + (size_t)c * PSTRIDE;
+          const float w = exp2f(__ldcg(pc + D) - M);
+          acc += w * __ldcg(pc + dc);
+          ls += w * __ldcg(pc + D + 1);
+        }
+        orow[idx] = acc / ls;
+      }
+    }
+  }
 
   for (long long item = blockIdx.x; item < items; item += gridDim.x) {
     const long long u = item / 3;
@@ -726,11 +756,11 @@ size_t gp_bsel_smem(const GpDev& p) {
   return SelGeom::BUF_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
 }
 
-void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, int grid_sel, int grid_compact,
-                        cudaStream_t s, cudaEvent_t ev) {
+void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
+                        int grid_compact, cudaStream_t s, cudaEvent_t ev) {
   const size_t sel_sm = gp_bsel_smem(p);
   cudaFuncSetAttribute(gp_bsel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
-  gp_bsel_kernel<<<grid_sel, SEL_T, sel_sm, s>>>(p, req_ids, n_req, actions);
+  gp_bsel_kernel<<<grid_sel, SEL_T, sel_sm, s>>>(p, req_ids, n_req, actions, out);
   if (ev) cudaEventRecord(ev, s);
   if (p.d == 128) gp_compact_kernel<128><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);
   else gp_compact_kernel<64><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);

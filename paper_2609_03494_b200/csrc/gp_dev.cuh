@@ -23,7 +23,11 @@
 #define GP_MAX_REQ 1024        // upper limit of max_requests (shared-memory arrays are sized by it)
 #define GP_SCORE_TILE 128      // candidate tokens per boundary-scoring tile
 #define GP_MOVE_TOK 64         // source slots per compaction chunk
+#define GP_COST_BINS 160       // cost classes of attention work items (pages, x4 at a boundary)
 #define GP_DESC_INTS 16        // ints per attention work descriptor
+
+// pages per work item of a request that is at its capacity boundary
+__host__ __device__ inline int gp_boundary_chunk(int chunk_pages) { return chunk_pages / 4 > 4 ? chunk_pages / 4 : 4; }
 
 // plan header slots (int32)
 enum {
@@ -37,6 +41,7 @@ enum {
   HDR_DONE_SEL,      // CTAs of the selection kernel that have finished
   HDR_WORK_CMP,      // ticket counter of the compaction kernel
   HDR_N_CITEM,       // compaction work items (chunks x layers x heads)
+  HDR_N_MC,          // requests whose attention was split over several work items
   HDR_COUNT = 16
 };
 
@@ -73,11 +78,11 @@ struct GpDev {
                                          //   0 batch index, 1 request, 2 first page, 3 pages, 4 chunk, 5 chunks,
                                          //   6 n before the append, 7 position, 8 flags (1 boundary, 2 started),
                                          //   9 P, 10-11 offset into the logit scratch, 12 summary buffer in use,
-                                         //   13 own index
+                                         //   13 index of its partial-output slot
   int* b_nold;                           // [M] occupied slots before the append, by batch index
   int* b_flags;                          // [M] 1 = stepped this step
   int* first_idx;                        // [M] lowest batch index naming a request
-  int* unit_cnt;                         // [M][L][H_kv] split-KV arrival counters
+  int4* mc_list;                         // [M] split requests: {batch index, first partial, chunks, 0}
   int* bnd_list;                         // [M] batch indices at a boundary
   long long* bnd_off;                    // [M] token offset into the score scratch
   int* cmp_list;                         // [M] batch indices that compress
@@ -192,5 +197,5 @@ size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
 // boundary chain: probabilities + working sets + selection + decision, then compaction.
 // `ev`, when not null, is recorded between the two kernels.
-void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, int grid_sel, int grid_compact,
-                        cudaStream_t s, cudaEvent_t ev);
+void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
+                        int grid_compact, cudaStream_t s, cudaEvent_t ev);

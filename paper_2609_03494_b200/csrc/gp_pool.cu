@@ -51,7 +51,7 @@ namespace {
 
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
-      b_flags, unit_cnt, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, zbuf, zstat, sum_par,
+      b_flags, mc_list, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, zbuf, zstat, sum_par,
       evict, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
   int max_rc;
@@ -94,7 +94,7 @@ Layout make_layout(const gp_config& c) {
   const size_t np = (size_t)c.n_pages;
   L.max_batch_tokens = c.max_batch_tokens > 0 ? c.max_batch_tokens : (long long)(np * b);
   const int ch = chunk_pages_setting();
-  L.max_rc = (int)((size_t)L.max_batch_tokens / (b * ch) + 2 * M + 1);
+  L.max_rc = (int)((size_t)L.max_batch_tokens / (b * gp_boundary_chunk(ch)) + 2 * M + 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
   L.kv = take(LH * np * 2 * b * d * 2);
@@ -113,7 +113,7 @@ Layout make_layout(const gp_config& c) {
   L.rc = take((size_t)L.max_rc * GP_DESC_INTS * 4);
   L.b_nold = take(M * 4);
   L.b_flags = take(M * 4);
-  L.unit_cnt = take(M * LH * 4);
+  L.mc_list = take(M * 16);
   L.bnd_list = take(M * 4);
   L.bnd_off = take(M * 8);
   L.cmp_list = take(M * 4);
@@ -196,11 +196,14 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __shared__ long long sw[33];
   __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
   __shared__ int s_chunks[GP_MAX_REQ], s_pos[GP_MAX_REQ];
+  __shared__ int s_bin[GP_COST_BINS], s_binbase[GP_COST_BINS], s_nmc;
   const int i = threadIdx.x;
   const bool in = i < n_req;
   const long long t_plan0 = GP_T_NOW();
   (void)t_plan0;
   s_first[i] = 0x7fffffff;
+  if (i < GP_COST_BINS) s_bin[i] = 0;
+  if (i == 0) s_nmc = 0;
   __syncthreads();
   int r = -1;
   if (in) {
@@ -211,6 +214,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   int chunks = 0, pages = 0, n_old = 0, act = GP_ACT_NONE, Pr = 0, started = 0, par = 0;
   long long nc = 0, pos = 0;
   int isb = 0;
+  int cp = p.chunk_pages;                 // pages per work item of this request
   if (in) {
     const bool inrange = r >= 0 && r < p.M;
     int live = 0;
@@ -224,8 +228,14 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       act = GP_ACT_STALLED;
     } else {
       pages = n_old / GP_PAGE + 1;
-      chunks = (pages + p.chunk_pages - 1) / p.chunk_pages;
-      if (n_old + 1 == Pr * GP_PAGE) { isb = 1; nc = (long long)(Pr - 1) * GP_PAGE; }
+      if (n_old + 1 == Pr * GP_PAGE) {
+        // a page of a boundary request also pays for the fp64 summary logits: four times smaller items
+        // keep the cost of an item about the same
+        isb = 1; nc = (long long)(Pr - 1) * GP_PAGE;
+        cp = gp_boundary_chunk(p.chunk_pages);
+      }
+      chunks = (pages + cp - 1) / cp;
+      cp = (pages + chunks - 1) / chunks;            // equal sizes: chunks of cp pages, the last one shorter
     }
   }
   const long long t_plan1 = GP_T_NOW();
@@ -240,6 +250,29 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   int bnd_idx, n_bnd, n_active; long long d0, d1;
   plan_scan(isb, chunks > 0, bnd_idx, d0, n_bnd, d1, sv, sw);
   n_active = (int)d1;
+  // Work items are listed by descending cost (pages, times four for boundary requests, which also pay for the
+  // fp64 logits): the attention kernel deals them out in that order, largest first.  Counting sort.
+  const int key = chunks > 0 ? min(GP_COST_BINS - 1, cp * (isb ? 4 : 1)) : 0;
+  int within = 0;
+  if (chunks > 0) within = atomicAdd(&s_bin[key], chunks);
+  __syncthreads();
+  if (threadIdx.x < 32) {                             // descending exclusive scan over the cost bins
+    int carry = 0;
+    for (int b0 = GP_COST_BINS - 32; b0 >= 0; b0 -= 32) {
+      const int b = b0 + 31 - (int)threadIdx.x;       // lane 0 takes the costliest bin of the block of 32
+      const int v = s_bin[b];
+      int inc = v;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, inc, off);
+        if ((int)threadIdx.x >= off) inc += a;
+      }
+      s_binbase[b] = carry + inc - v;
+      carry += __shfl_sync(0xffffffffu, inc, 31);
+    }
+  }
+  __syncthreads();
+  const int sorted0 = s_binbase[key] + within;
   const long long t_plan2 = GP_T_NOW();
   (void)t_plan2;
   s_chunks[i] = chunks; s_pos[i] = (int)pos;
@@ -251,13 +284,14 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     // descriptors of this request's chunks: four 16-byte stores each
     const int flags = isb | (started ? 2 : 0);
     for (int c = 0; c < chunks; ++c) {
-      const int pg0 = c * p.chunk_pages;
-      int4* d = reinterpret_cast<int4*>(p.rcx + (size_t)(rc_off + c) * GP_DESC_INTS);
-      d[0] = make_int4(i, r, pg0, min(p.chunk_pages, pages - pg0));
+      const int pg0 = c * cp;
+      int4* d = reinterpret_cast<int4*>(p.rcx + (size_t)(sorted0 + c) * GP_DESC_INTS);
+      d[0] = make_int4(i, r, pg0, min(cp, pages - pg0));
       d[1] = make_int4(c, chunks, n_old, (int)pos);
       d[2] = make_int4(flags, Pr, (int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32));
       d[3] = make_int4(par, rc_off + c, 0, 0);
     }
+    if (chunks > 1) p.mc_list[atomicAdd(&s_nmc, 1)] = make_int4(i, rc_off, chunks, 0);
   }
   if (p.rope_theta != 0.0) {                                      // cos / sin of the step's position
     __syncthreads();
@@ -274,7 +308,9 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       }
     }
   }
+  __syncthreads();
   if (threadIdx.x == 0) {
+    p.hdr[HDR_N_MC] = s_nmc;
     GP_T_ADD(26, 1); GP_T_ADD(27, t_plan1 - t_plan0); GP_T_ADD(28, t_plan2 - t_plan1); GP_T_ADD(29, GP_T_NOW() - t_plan2);
     p.hdr[HDR_N_RC] = n_rc;
     p.hdr[HDR_N_BND] = n_bnd;
@@ -473,7 +509,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.rcx = reinterpret_cast<int*>(base + L.rc);
   d.b_nold = reinterpret_cast<int*>(base + L.b_nold);
   d.b_flags = reinterpret_cast<int*>(base + L.b_flags);
-  d.unit_cnt = reinterpret_cast<int*>(base + L.unit_cnt);
+  d.mc_list = reinterpret_cast<int4*>(base + L.mc_list);
   d.bnd_list = reinterpret_cast<int*>(base + L.bnd_list);
   d.bnd_off = reinterpret_cast<long long*>(base + L.bnd_off);
   d.cmp_list = reinterpret_cast<int*>(base + L.cmp_list);
@@ -578,7 +614,8 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   if (prof) cudaEventRecord(pool->ev[1], s);
   gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s);
   if (prof) cudaEventRecord(pool->ev[2], s);
-  gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, GP_SEL_GRID, GP_COMPACT_GRID, s, prof ? pool->ev[3] : nullptr);
+  gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), GP_SEL_GRID, GP_COMPACT_GRID, s,
+                     prof ? pool->ev[3] : nullptr);
   if (prof) cudaEventRecord(pool->ev[4], s);
   pool->launch_count += GP_N_KERNELS;
   GP_CUDA(cudaGetLastError());
