@@ -34,6 +34,7 @@ extern "C" {
 #define GP_ERR_NO_PAGES  (-3)  /* the free list or the per-request cap cannot supply the pages    */
 #define GP_ERR_CUDA      (-4)  /* a CUDA call failed or a kernel reported an internal error       */
 #define GP_ERR_STATE     (-5)  /* call not possible in the pool's current state                   */
+#define GP_ERR_TOO_LARGE (-6)  /* problem exceeds the fixed scratch of gp_attention_noalloc        */
 
 /* per-request action written by gp_decode_step (Sec. 3.3, Sec. 4.2) */
 #define GP_ACT_NONE               0   /* no capacity boundary this step                           */
@@ -167,6 +168,35 @@ int gp_get_kernel_times(gp_pool* pool, float* ms, int64_t* launches);
 
 /* Kernels launched by this pool since creation (all calls). */
 int64_t gp_launch_count(gp_pool* pool);
+
+/* ---- attention without any allocation ------------------------------------------------------------ */
+
+#define GP_NOALLOC_SPLITS   8      /* parts a request's tokens are split into                           */
+#define GP_NOALLOC_MAX_ROWS 2048   /* limit on n_req * n_q_heads                                        */
+
+/* (The paper has no counterpart of this call; it exists for deployments, not for the method.)
+ *
+ * GQA decode attention over plain, un-paged K/V, for callers that cannot give the library any memory to
+ * work in and must not have it allocate: for instance a server that handed every byte of the GPU to its KV
+ * pool at start-up, or a host that loads this library as a plug-in and forbids allocator calls from it.
+ * The split-KV partial results go to an 8.5 MB array that is part of the library image; each GPU that loads
+ * the library holds that array until the process exits.
+ *
+ *   q     device bf16 [n_req][n_q_heads][d]
+ *   k, v  device bf16 [n_req][n_kv_heads][max_len][d], rows in plain order (no page layout, no swizzle)
+ *   lens  device int32 [n_req]: tokens of each request, 1..max_len (values above max_len are clipped)
+ *   out   device fp32 [n_req][n_q_heads][d]: softmax(q.K/sqrt(d)).V per query head, KV head g / G
+ *
+ * Limits: d is 64 or 128, G = n_q_heads / n_kv_heads <= 8, n_req * n_q_heads <= GP_NOALLOC_MAX_ROWS;
+ * beyond that the call returns GP_ERR_TOO_LARGE and does nothing.  It calls no cudaMalloc, cudaFree or
+ * other allocating routine.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress) with that device current; make that first call outside any stream capture.
+ * All calls share the one array and nothing in it has to be cleared (every slot a call reads it has
+ * written first), but two calls that overlap on the GPU, e.g. on different streams, race on it:
+ * serialise them.  Asynchronous on `stream`. */
+int gp_attention_noalloc(const void* q, const void* k, const void* v, const int32_t* lens, int32_t n_req,
+                         int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t max_len,
+                         void* out, void* stream);
 
 #ifdef __cplusplus
 }

@@ -14,6 +14,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgrowpage.so")
 
 GP_OK, GP_ERR_INVALID, GP_ERR_NO_SLOT, GP_ERR_NO_PAGES, GP_ERR_CUDA, GP_ERR_STATE = 0, -1, -2, -3, -4, -5
+GP_ERR_TOO_LARGE = -6
+GP_NOALLOC_MAX_ROWS = 2048
 GP_ACT_NONE, GP_ACT_GROW, GP_ACT_COMPRESS, GP_ACT_COMPRESS_FALLBACK = 0, 1, 2, 3
 GP_ACT_STALLED, GP_ACT_SCRATCH, GP_ACT_INVALID = -1, -2, -3
 GP_N_KERNELS = 4
@@ -62,6 +64,7 @@ def lib() -> C.CDLL:
     L.gp_set_profiling.argtypes = [vp, i32]
     L.gp_get_kernel_times.argtypes = [vp, vp, vp]
     L.gp_launch_count.argtypes = [vp]; L.gp_launch_count.restype = i64
+    L.gp_attention_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
     _lib = L
     return L
 
@@ -192,6 +195,16 @@ def gp_get_kernel_times(pool: int):
 
 def gp_launch_count(pool: int) -> int:
     return int(lib().gp_launch_count(C.c_void_p(pool)))
+
+
+def gp_attention_noalloc(q_ptr: int, k_ptr: int, v_ptr: int, lens_ptr: int, n_req: int, n_q_heads: int,
+                         n_kv_heads: int, head_dim: int, max_len: int, out_ptr: int, stream: int) -> None:
+    """Decode attention over plain K/V for callers that may not allocate: the library brings its own fixed
+    scratch.  All pointers are device addresses the caller owns; raises GpError (GP_ERR_TOO_LARGE when
+    n_req * n_q_heads exceeds GP_NOALLOC_MAX_ROWS).  Do not overlap two calls on the GPU."""
+    _check(lib().gp_attention_noalloc(C.c_void_p(q_ptr), C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(lens_ptr),
+                                      n_req, n_q_heads, n_kv_heads, head_dim, max_len, C.c_void_p(out_ptr),
+                                      C.c_void_p(stream)), "gp_attention_noalloc")
 
 
 # ------------------------------------------------------------------------------- convenience holder

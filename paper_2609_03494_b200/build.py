@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgrowpage.so")
-SOURCES = ["gp_pool.cu", "gp_attn.cu", "gp_boundary.cu"]
+SOURCES = ["gp_pool.cu", "gp_attn.cu", "gp_boundary.cu", "gp_noalloc.cu"]
 HEADERS = ["gp_dev.cuh", os.path.join("..", "..", "include", "growpage.h")]
 
 

@@ -674,6 +674,7 @@ const char* gp_strerror(int status) {
     case GP_ERR_NO_PAGES: return "not enough free pages or per-request cap exceeded";
     case GP_ERR_CUDA: return "CUDA error or internal kernel error";
     case GP_ERR_STATE: return "call not possible in this state";
+    case GP_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }
