@@ -114,7 +114,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef GP_TRACE
-  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 7] = (long long)gt; }
+  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 32] = (long long)gt; }
 #endif
   if (tid == 0) {
     for (int i = 0; i < NCW * NSW; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -526,7 +526,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     }
     if (tr) GP_T_ADD(6, GP_T_NOW() - t_loop0);
 #ifdef GP_TRACE
-    if (tr) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 28] = (long long)gt; }
+    if (tr) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 35] = (long long)gt; }
 #endif
   } else if (warp == 1) {
     // ================================= summaries ==========================================
@@ -658,12 +658,12 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     }
   }
 #ifdef GP_TRACE
-  if (lane == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 16 + warp] = (long long)gt; }
+  if (lane == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 40 + warp] = (long long)gt; }
 #endif
   __syncthreads();
 #ifdef GP_TRACE
-  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 15] = (long long)gt; }
-  if (tid == 128) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 29] = (long long)gt; }
+  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 33] = (long long)gt; }
+  if (tid == 128) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 34] = (long long)gt; }
 #endif
 }
 
@@ -671,6 +671,17 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
 
 size_t gp_attention_smem(int d, int G) { return d == 128 ? make_lay<128>(G).total : make_lay<64>(G).total; }
 int gp_attention_ctas_per_sm(int d) { (void)d; return 2; }
+
+void gp_attention_setup(const GpDev& p) {           // once per pool: opt into the kernel's shared memory
+  const int sm = (int)gp_attention_smem(p.d, p.G);
+  if (p.d == 128) {
+    cudaFuncSetAttribute(gp_attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+    cudaFuncSetAttribute(gp_attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  } else {
+    cudaFuncSetAttribute(gp_attn_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+    cudaFuncSetAttribute(gp_attn_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  }
+}
 
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
                          float* out, int grid, cudaStream_t s) {
@@ -683,7 +694,6 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
 #define GP_LAUNCH(DD, RR)                                                                 \
   do {                                                                                    \
     auto kern = gp_attn_kernel<DD, RR>;                                                   \
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);          \
     kern<<<grid, NTHREADS, sm, s>>>(p, n_req, qq, kk, vv, out);                          \
   } while (0)
   if (p.d == 128) {

@@ -88,7 +88,7 @@ __device__ __forceinline__ void add64_split(unsigned* lo, unsigned* hi, unsigned
 
 // Eq. 7: smallest k such that the k largest of a[0..n) sum to at least p.
 template <int BT>
-__device__ int top_p_count(const GpDev& p, const double* a, int n, unsigned long long p_fix, unsigned* hcnt,
+__device__ __noinline__ int top_p_count(const GpDev& p, const double* a, int n, unsigned long long p_fix, unsigned* hcnt,
                            unsigned long long* hsum64, unsigned* wc, unsigned long long* wsum, long long* s_res) {
   unsigned* hlo = reinterpret_cast<unsigned*>(hsum64);
   unsigned* hhi = hlo + NBINS_PAD;
@@ -158,65 +158,247 @@ __device__ int top_p_count(const GpDev& p, const double* a, int n, unsigned long
 }
 
 // ------------------------------------------------------------------------------------------------------
+// fast path: one pass fills a 4096-bin histogram and its 256-bin summary; a one-warp sort finishes
+// ------------------------------------------------------------------------------------------------------
+// Scores of a candidate set are probabilities of similar magnitude: bits 62..58 of their IEEE patterns are
+// nearly always the same (the softmax pass reports whether they are).  Then bits 57..46 (low exponent bits and
+// the top of the mantissa) order the scores finely enough that the crossing point falls into a bin with a
+// handful of members.  The 256-bin summary (bits 57..50) is scanned by the block, one bin per thread; the 16
+// fine bins under the crossing summary bin by half a warp; the members of the crossing fine bin are sorted by
+// one warp.  When the top bits differ or the bin is crowded, the callers fall back on the general radix
+// descent above.
+constexpr int FBINS = 4096;
+constexpr int FB_PAD = FBINS + FBINS / 16;       // plane stride (the general routine pads its bins)
+constexpr int CBINS = 256;                       // summary bins: 16 fine bins each, one per thread
+constexpr int FSHIFT = 46;
+static_assert(CBINS == SEL_T, "one summary bin per thread");
+
+struct FastHist {
+  unsigned* cnt; unsigned* lo; unsigned* hi;       // [FBINS] members, and their fixed-point mass in two halves
+  unsigned* ccnt; unsigned* clo; unsigned* chi;    // [CBINS] the same per summary bin
+};
+
+__device__ __forceinline__ void fast_hist_zero(const FastHist& H, bool with_mass) {
+  const uint4 z = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < FBINS / 4; i += SEL_T) {
+    reinterpret_cast<uint4*>(H.cnt)[i] = z;
+    if (with_mass) { reinterpret_cast<uint4*>(H.lo)[i] = z; reinterpret_cast<uint4*>(H.hi)[i] = z; }
+  }
+  H.ccnt[threadIdx.x] = 0;
+  if (with_mass) { H.clo[threadIdx.x] = 0; H.chi[threadIdx.x] = 0; }
+}
+
+// sorts (v, tag) across the 32 lanes: descending v when DESC, else ascending v with larger tag first among
+// equal v
+template <bool DESC>
+__device__ __forceinline__ void warp_sort(double& v, int& tag) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      const double ov = __shfl_xor_sync(0xffffffffu, v, j);
+      const int ot = __shfl_xor_sync(0xffffffffu, tag, j);
+      // "first" = the element that belongs earlier in the final order
+      const bool mine_first = DESC ? (v > ov || (v == ov && tag < ot)) : (v < ov || (v == ov && tag > ot));
+      const bool want_first = (((lane & k) == 0) == ((lane & j) == 0));
+      if (mine_first != want_first) { v = ov; tag = ot; }
+    }
+  }
+}
+
+// Eq. 7 on the fast path (histograms already zeroed, s_res[0] = -1, *s_cnt = 0); returns -1 when the general
+// routine has to take over
+__device__ int top_p_fast(const GpDev& p, const double* a, int n, unsigned long long p_fix, const FastHist& H,
+                          unsigned* wc, unsigned long long* wsum, long long* s_res, double* list, int* s_cnt) {
+  const int tid = threadIdx.x;
+  const long long f2 = GP_T_NOW(); (void)f2;
+  for (int i = tid; i < n; i += SEL_T) {
+    const double v = a[i];
+    const int bin = (int)(((unsigned long long)__double_as_longlong(v) >> FSHIFT) & (FBINS - 1));
+    const unsigned long long f = to_fix(v);
+    atomicAdd(&H.cnt[bin], 1u);
+    add64_split(&H.lo[bin], &H.hi[bin], f);
+    atomicAdd(&H.ccnt[bin >> 4], 1u);
+    add64_split(&H.clo[bin >> 4], &H.chi[bin >> 4], f);
+  }
+  __syncthreads();
+  const long long f3 = GP_T_NOW(); (void)f3;
+  {                                               // summary level: thread t owns bin t; higher bins = larger scores
+    const unsigned c = H.ccnt[tid];
+    const unsigned long long m = ((unsigned long long)H.chi[tid] << 32) + H.clo[tid];
+    const PairCU ex = block_suffix_excl<SEL_T>(c, m, wc, wsum);
+    if (ex.s < p_fix && ex.s + m >= p_fix) { s_res[0] = tid; s_res[1] = ex.c; s_res[2] = (long long)ex.s; }
+  }
+  __syncthreads();
+  if (s_res[0] < 0) return n;                    // rounding kept the total below p: everything
+  if (tid < 32) {                                // fine level: lane j owns the (j+1)-th highest bin of the 16
+    const int cb = (int)s_res[0];
+    const int fb = cb * 16 + 15 - (tid & 15);
+    const unsigned c = tid < 16 ? H.cnt[fb] : 0u;
+    const unsigned long long m = tid < 16 ? ((unsigned long long)H.hi[fb] << 32) + H.lo[fb] : 0ull;
+    unsigned ic = c; unsigned long long im = m;
+#pragma unroll
+    for (int off = 1; off < 16; off <<= 1) {
+      const unsigned tc = __shfl_up_sync(0xffffffffu, ic, off);
+      const unsigned long long tm = __shfl_up_sync(0xffffffffu, im, off);
+      if (tid >= off) { ic += tc; im += tm; }
+    }
+    const unsigned long long before = (unsigned long long)s_res[2] + im - m;
+    if (tid < 16 && before < p_fix && before + m >= p_fix) {
+      s_res[4] = fb; s_res[5] = s_res[1] + (long long)(ic - c); s_res[6] = (long long)before; s_res[7] = c;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) { GP_T_ADD(54, 1); GP_T_ADD(57, f3 - f2); GP_T_ADD(58, GP_T_NOW() - f3); }
+  const int bstar = (int)s_res[4];
+  const unsigned cnt_above = (unsigned)s_res[5];
+  const unsigned long long sum_above = (unsigned long long)s_res[6];
+  const unsigned cstar = (unsigned)s_res[7];
+  if (cstar == 1) return (int)cnt_above + 1;
+  if (cstar > 32) return -1;
+  for (int i = tid; i < n; i += SEL_T) {
+    const double v = a[i];
+    if ((int)(((unsigned long long)__double_as_longlong(v) >> FSHIFT) & (FBINS - 1)) == bstar) list[atomicAdd(s_cnt, 1)] = v;
+  }
+  __syncthreads();
+  if (tid < 32) {
+    double v = tid < (int)cstar ? list[tid] : -1.0;
+    int tag = tid;
+    warp_sort<true>(v, tag);
+    unsigned long long inc = tid < (int)cstar ? to_fix(v) : 0ull;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const unsigned long long o = __shfl_up_sync(0xffffffffu, inc, off);
+      if (tid >= off) inc += o;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, tid < (int)cstar && sum_above + inc >= p_fix);
+    if (tid == 0) s_res[3] = (long long)cnt_above + (hit ? __ffs(hit) : (int)cstar);
+  }
+  __syncthreads();
+  return (int)s_res[3];
+}
+
+// Eq. 10 global cut on the fast path (counts already zeroed, s_res[0] = -1, s_cnt[0..1] = 0): lists the b
+// evicted slots in ev[] (unsorted) and returns true, or returns false when the general routine has to take
+// over.  `a` holds Eq. 9 scores, `loc` the block-local quota bits (those slots are never evicted).
+__device__ bool evict_fast(const double* a, int nC, const unsigned* loc, const FastHist& H, unsigned* wc, long long* s_res,
+                           double* list, int* list_slot, int* s_cnt, int* ev) {
+  const int tid = threadIdx.x;
+  for (int i = tid; i < nC; i += SEL_T) {
+    if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
+      const int bin = (int)(((unsigned long long)__double_as_longlong(a[i]) >> FSHIFT) & (FBINS - 1));
+      atomicAdd(&H.cnt[bin], 1u);
+      atomicAdd(&H.ccnt[bin >> 4], 1u);
+    }
+  }
+  __syncthreads();
+  {                                               // summary level, ascending: the b lowest scores go
+    const unsigned c = H.ccnt[tid];
+    const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
+    if (ex < (unsigned)GP_PAGE && ex + c >= (unsigned)GP_PAGE) { s_res[0] = tid; s_res[1] = ex; }
+  }
+  __syncthreads();
+  if (s_res[0] < 0) return false;
+  if (tid < 32) {
+    const int fb = (int)s_res[0] * 16 + (tid & 15);
+    const unsigned c = tid < 16 ? H.cnt[fb] : 0u;
+    unsigned ic = c;
+#pragma unroll
+    for (int off = 1; off < 16; off <<= 1) {
+      const unsigned tc = __shfl_up_sync(0xffffffffu, ic, off);
+      if (tid >= off) ic += tc;
+    }
+    const unsigned before = (unsigned)s_res[1] + ic - c;
+    if (tid < 16 && before < (unsigned)GP_PAGE && before + c >= (unsigned)GP_PAGE) { s_res[4] = fb; s_res[5] = before; s_res[6] = c; }
+  }
+  __syncthreads();
+  const int bstar = (int)s_res[4];
+  const int cnt_below = (int)s_res[5], cstar = (int)s_res[6];
+  const bool exact = (cnt_below + cstar == GP_PAGE);
+  if (!exact && cstar > 32) return false;
+  for (int i = tid; i < nC; i += SEL_T) {
+    if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
+      const int bin = (int)(((unsigned long long)__double_as_longlong(a[i]) >> FSHIFT) & (FBINS - 1));
+      if (bin < bstar || (exact && bin == bstar)) ev[atomicAdd(&s_cnt[0], 1)] = i;
+      else if (bin == bstar) { const int at = atomicAdd(&s_cnt[1], 1); list[at] = a[i]; list_slot[at] = i; }
+    }
+  }
+  __syncthreads();
+  if (!exact && tid < 32) {                      // the lowest scores of the bin, later slots first among equals
+    double v = tid < cstar ? list[tid] : INFINITY;
+    int slot = tid < cstar ? list_slot[tid] : -1;
+    warp_sort<false>(v, slot);
+    if (tid < GP_PAGE - cnt_below) ev[cnt_below + tid] = slot;
+  }
+  __syncthreads();
+  return true;
+}
+
+// ------------------------------------------------------------------------------------------------------
 // decision + allocator, run by the last CTA of the selection kernel
 // ------------------------------------------------------------------------------------------------------
-__device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int* actions, int* s_arr) {
+__device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr) {
   int* s_want = s_arr;
   int* s_ksh = s_arr + GP_MAX_REQ;
   int* s_P = s_arr + 2 * GP_MAX_REQ;
   int* s_order = s_arr + 3 * GP_MAX_REQ;
   int* s_req = s_arr + 4 * GP_MAX_REQ;
   int* s_base = s_arr + 5 * GP_MAX_REQ;
+  int* s_bi = s_arr + 6 * GP_MAX_REQ;
+  int* s_free = s_arr + 7 * GP_MAX_REQ;      // the free pages the grants of this step can take, top first
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarp = blockDim.x >> 5;
-  const int n_bnd = p.hdr[HDR_N_BND];
-  for (int i = tid; i < n_req; i += blockDim.x) {
-    if (p.b_flags[i]) {
-      const int r = req_ids[i];
-      p.n[r] = p.b_nold[i] + 1;
-      p.pos[r] += 1;
-      p.started[r] = 1;
-      p.sum_par[r] ^= 1;                                  // the attention kernel wrote the other buffer
-    }
-  }
-  if (tid == 0) {
-    p.counters[5] += 1;
-    p.counters[6] += p.hdr[HDR_N_ACTIVE];
-    p.hdr[HDR_N_CMP] = 0;
-    p.hdr[HDR_N_CITEM] = 0;
-    p.hdr[HDR_WORK_CMP] = 0;
-  }
-  if (n_bnd == 0) return;
-  __syncthreads();
+  // everything the decisions need arrives in one round trip: the jobs summed K^S and K^L per request, a job
+  // counted its shared pages, and the plan kernel copied the top of the free list
   const int LH = p.L * p.Hkv;
-  for (int e = warp; e < n_bnd; e += nwarp) {
-    const int bi = p.bnd_list[e];
-    const int r = req_ids[bi];
-    const int Pr = p.P[r];
-    const int nC = (Pr - 1) * GP_PAGE;
-    long long sS = 0, sL = 0;
-    const int* kx = p.Kx + (size_t)r * LH * 2;
-    for (int j = lane; j < LH; j += 32) { sS += kx[2 * j]; sL += kx[2 * j + 1]; }
-    int ksh = 0;
-    const int* table = p.page_table + (size_t)r * p.cap;
-    for (int j = lane; j < Pr - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
+  constexpr int RPT = GP_MAX_REQ / SEL_T;                 // stepped requests per thread
+  int fl[RPT], rq[RPT], no[RPT];
 #pragma unroll
-    for (int o2 = 16; o2 > 0; o2 >>= 1) {
-      sS += __shfl_xor_sync(0xffffffffu, sS, o2);
-      sL += __shfl_xor_sync(0xffffffffu, sL, o2);
-      ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
-    }
-    if (lane == 0) {
+  for (int k = 0; k < RPT; ++k) {
+    const int i = tid + k * SEL_T;
+    fl[k] = i < n_req ? p.b_flags[i] : 0;
+    rq[k] = i < n_req ? req_ids[i] : 0;
+    no[k] = i < n_req ? p.b_nold[i] : 0;
+  }
+  const int n_active = p.hdr[HDR_N_ACTIVE];
+  int top0 = 0;
+  if (n_bnd > 0) {
+    top0 = __ldcg(p.free_peek);
+    for (int e = tid; e < n_bnd; e += blockDim.x) {
+      const int4 inf = p.bnd_info[2 * e];
+      const int4 acc = __ldcg(reinterpret_cast<const int4*>(p.bnd_acc) + e);
+      s_free[e] = __ldcg(p.free_peek + 1 + e);
+      const int r = inf.y, Pr = inf.z;
+      const int nC = (Pr - 1) * GP_PAGE;
       // Eq. 8 with a common |C|: Delta = (sum K^S - sum K^L) / (N |C|), one division of exact integers
       double delta = 0.0;
       int want = 1;
       if (nC > 0) {
-        delta = (double)(sS - sL) / ((double)LH * (double)nC);
+        delta = (double)((long long)acc.x - (long long)acc.y) / ((double)LH * (double)nC);
         want = delta > p.tau;
       }
       p.delta[r] = delta;
-      s_want[e] = want; s_ksh[e] = ksh; s_P[e] = Pr; s_req[e] = r;
+      s_want[e] = want; s_ksh[e] = acc.z; s_P[e] = Pr; s_req[e] = r; s_bi[e] = inf.x;
     }
   }
+  // every stepped request: one more token; fire-and-forget updates, nothing here waits for memory
+#pragma unroll
+  for (int k = 0; k < RPT; ++k) {
+    if (fl[k]) {
+      const int r = rq[k];
+      p.n[r] = no[k] + 1;
+      atomicAdd(reinterpret_cast<unsigned long long*>(p.pos + r), 1ull);
+      p.started[r] = 1;
+      atomicXor(p.sum_par + r, 1);                       // the attention kernel wrote the other buffer
+    }
+  }
+  if (tid == 0) {
+    atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 5), 1ull);
+    atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 6), (unsigned long long)n_active);
+    p.hdr[HDR_WORK_CMP] = 0;
+    if (n_bnd == 0) { p.hdr[HDR_N_CMP] = 0; p.hdr[HDR_N_CITEM] = 0; p.hdr[HDR_N_COW] = 0; }
+  }
+  if (n_bnd == 0) return;
   __syncthreads();
   for (int e = tid; e < n_bnd; e += blockDim.x) {
     int rank = 0;
@@ -224,16 +406,17 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     s_order[rank] = e;
   }
   __syncthreads();
-  if (tid == 0) {
-    int top = *p.free_top;
+  if (tid == 0) {                                        // sequential allocator: shared memory only
+    int top = top0;
     int n_cmp = 0, chunks = 0;
-    long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0;
-    for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants
+    unsigned long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0;
+    for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants, ascending request id
       const int e = s_order[k];
-      const int r = s_req[e], Pr = s_P[e], bi = p.bnd_list[e];
-      scored += (long long)(Pr - 1) * GP_PAGE;
+      const int r = s_req[e], Pr = s_P[e], bi = s_bi[e];
+      scored += (unsigned long long)(Pr - 1) * GP_PAGE;
       if ((s_want[e] & 1) && Pr < p.cap && top > 0) {
-        const int page = p.free_stack[--top];
+        const int page = s_free[top0 - top];
+        --top;
         p.refcount[page] = 1;
         p.page_table[(size_t)r * p.cap + Pr] = page;
         p.P[r] = Pr + 1;
@@ -249,7 +432,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     for (int k = 0; k < n_bnd; ++k) {                    // pass 2: copy-on-write targets
       const int e = s_order[k];
       if (s_want[e] & 6) continue;
-      const int r = s_req[e], bi = p.bnd_list[e];
+      const int r = s_req[e], bi = s_bi[e];
       if (s_ksh[e] > top) {
         actions[bi] = GP_ACT_STALLED;
         ++stall;
@@ -258,9 +441,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       s_base[e] = top;
       top -= s_ksh[e];
       cow += s_ksh[e];
-      p.cmp_list[n_cmp] = bi;
-      p.cmp_bnd[n_cmp] = e;
-      p.cmp_chunk0[n_cmp] = chunks;
+      p.cmp_info[n_cmp] = make_int4(r, s_P[e], e, chunks);
       chunks += (s_P[e] * GP_PAGE + MOVE_TOK - 1) / MOVE_TOK;
       ++n_cmp;
       if (s_want[e] & 1) { actions[bi] = GP_ACT_COMPRESS_FALLBACK; ++fall; } else { actions[bi] = GP_ACT_COMPRESS; ++comp; }
@@ -268,13 +449,19 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       p.n_pristine[r] = 0;
       s_want[e] |= 8;
     }
-    p.cmp_chunk0[n_cmp] = chunks;
+    p.cmp_info[n_cmp] = make_int4(0, 0, 0, chunks);
     if (top < 0) atomicOr(p.err, GP_E_FREELIST);
     *p.free_top = top;
     p.hdr[HDR_N_CMP] = n_cmp;
     p.hdr[HDR_N_CITEM] = chunks * LH;
-    p.counters[0] += grow; p.counters[1] += comp; p.counters[2] += fall; p.counters[3] += stall; p.counters[4] += cow;
-    p.counters[9] += scored;
+    p.hdr[HDR_N_COW] = (int)cow;
+    unsigned long long* cn = reinterpret_cast<unsigned long long*>(p.counters);
+    if (grow) atomicAdd(cn + 0, grow);
+    if (comp) atomicAdd(cn + 1, comp);
+    if (fall) atomicAdd(cn + 2, fall);
+    if (stall) atomicAdd(cn + 3, stall);
+    if (cow) atomicAdd(cn + 4, cow);
+    atomicAdd(cn + 9, scored);
   }
   __syncthreads();
   for (int e = warp; e < n_bnd; e += nwarp) {             // fill in the targets, in table order
@@ -297,15 +484,17 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
   }
 }
 
-// ------------------------------------------------------------------------------------------------------
-// working sets + speculative eviction list; three independent jobs per unit, one CTA each; the last CTA decides
-// ------------------------------------------------------------------------------------------------------
-struct SelGeom {
-  static constexpr size_t BUF_BYTES = SEL_CAP * sizeof(double);
-  static constexpr size_t H_BYTES = NBINS_PAD * 4 + NBINS_PAD * 8;
-  static constexpr size_t MISC_BYTES = 8 * 8 + 8 * 4 + 8 * 8 + 16 * 4 + 16 * 4 + (8 * 16 + 32) * 8;
-};
+// a^x of one token from its logits: sum over the group of exp(z - max) * 1 / (G Z); G is a template
+// parameter so that the exponentials of a thread's tokens overlap
+__device__ __forceinline__ double exp_once(double x) { return exp(x); }
 
+template <int GG>
+__device__ __forceinline__ double group_prob(const double* zv, const double* sM, const double* rZ) {
+  double s = 0.0;
+#pragma unroll
+  for (int g = 0; g < GG; ++g) s += exp_once(zv[g] - sM[g]) * rZ[g];
+  return s;
+}
 // max or sum over the block of one value per thread, separately for each of `ncols` interleaved columns
 // (thread t belongs to column t % ncols); fixed shuffle tree, so the sum does not depend on timing
 template <bool IS_MAX>
@@ -325,15 +514,146 @@ __device__ __forceinline__ void column_reduce(double v, int ncols, double* red, 
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(SEL_T)
+// Per-head softmax over C and the group mean (Sec. 3.2), then a^S, a^L or s = max(a^S, a^L) (Eq. 9) of every
+// candidate into a[].  The attention kernel left, per 16-token page and column, the page's (max, sum of
+// exponentials); they merge into the normalisers of the whole candidate set without another pass over the
+// logits.  All loads of the prologue (page partials and the first batch of logits) are issued together.
+template <int GG>
+__device__ __noinline__ bool job_softmax(const double* __restrict__ z, const double* __restrict__ zs,
+                                         double* __restrict__ a, int nC, int task, double* red, double* sM,
+                                         double* sZ) {
+  constexpr int G2 = 2 * GG;
+  constexpr int U = GG == 8 ? 1 : GG == 4 ? 2 : 4;       // tokens per thread in flight
+  constexpr int KEEP = 2;                                // page partials per thread held in registers
+  const int tid = threadIdx.x;
+  const int ncols = task == 2 ? G2 : GG;
+  const int col0 = task == 1 ? GG : 0;
+  const int mycol = col0 + tid % ncols;                  // SEL_T is a multiple of ncols
+  const int ntile = nC / GP_PAGE;
+  const int t0 = tid / ncols, tstep = SEL_T / ncols;
+  double2 keep[KEEP];
+#pragma unroll
+  for (int k = 0; k < KEEP; ++k) {
+    const int t = t0 + k * tstep;
+    keep[k] = t < ntile ? __ldcg(reinterpret_cast<const double2*>(zs + ((size_t)t * G2 + mycol) * 2))
+                        : make_double2(-INFINITY, 0.0);
+  }
+  double zv[U][G2];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const int i = tid + u * SEL_T;
+    if (i < nC) {
+      const double* zr = z + (size_t)i * G2 + col0;
+#pragma unroll
+      for (int g = 0; g < G2; ++g)
+        if (g < GG || task == 2) zv[u][g] = __ldcg(zr + g);
+    }
+  }
+  double m = fmax(keep[0].x, keep[1].x);
+  for (int t = t0 + KEEP * tstep; t < ntile; t += tstep) m = fmax(m, __ldcg(zs + ((size_t)t * G2 + mycol) * 2));
+  column_reduce<true>(m, ncols, red, sM);
+  const double mc = sM[tid % ncols];
+  double acc = 0.0;
+#pragma unroll
+  for (int k = 0; k < KEEP; ++k)
+    if (t0 + k * tstep < ntile) acc += keep[k].y * exp_once(keep[k].x - mc);
+  for (int t = t0 + KEEP * tstep; t < ntile; t += tstep) {
+    const double2 ms = __ldcg(reinterpret_cast<const double2*>(zs + ((size_t)t * G2 + mycol) * 2));
+    acc += ms.y * exp_once(ms.x - mc);
+  }
+  column_reduce<false>(acc, ncols, red, sZ);
+  if (tid < ncols) sZ[tid] = 1.0 / ((double)GG * sZ[tid]);     // group mean and normaliser in one factor
+  __syncthreads();
+  unsigned top_bits = 0;
+  for (int i0 = tid; i0 < nC; i0 += U * SEL_T) {
+    if (i0 != tid) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * SEL_T;
+        if (i < nC) {
+          const double* zr = z + (size_t)i * G2 + col0;
+#pragma unroll
+          for (int g = 0; g < G2; ++g)
+            if (g < GG || task == 2) zv[u][g] = __ldcg(zr + g);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * SEL_T;
+      if (i < nC) {
+        double s0 = group_prob<GG>(zv[u], sM, sZ);                // column c of this job sits at index c - col0
+        if (task == 2) s0 = fmax(s0, group_prob<GG>(zv[u] + GG, sM + GG, sZ + GG));       // Eq. 9
+        a[i] = s0;
+        top_bits |= 1u << (unsigned)(((unsigned long long)__double_as_longlong(s0) >> 58) & 31ull);
+      }
+    }
+  }
+  // bits 62..58 of every score, as a set: the fast selection path needs them all equal
+  return __popc(__syncthreads_or((int)top_bits)) == 1;
+}
+
+// Attention outputs of requests that were split over several work items: merges the items' partial results
+// (running maximum in the log2 domain, sum of exponentials, unnormalised output) into the output row.  The
+// calling CTA takes merges first, first + stride, ...
+__device__ __noinline__ void merge_partials(const GpDev& p, int n_req, float* __restrict__ out, int n_mc, int n_rc,
+                                            int first_item, int stride) {
+  const int LH = p.L * p.Hkv, G = p.G, D = p.d;
+  const int PSTRIDE = G * (D + 2);
+  for (long long mi = first_item; mi < (long long)n_mc * LH; mi += stride) {
+    const int4 mc = p.mc_list[mi / LH];
+    const int lh = (int)(mi % LH), l = lh / p.Hkv, h = lh % p.Hkv;
+    const int bi = mc.x, nch = mc.z;
+    const float* first = p.partials + ((size_t)lh * n_rc + mc.y) * PSTRIDE;
+    float* orow = out + (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
+    for (int idx = threadIdx.x; idx < G * D; idx += SEL_T) {
+      const int g = idx / D, dc = idx % D;
+      const float* pg = first + g * (D + 2);
+      float M = -INFINITY, acc = 0.f, ls = 0.f;
+      for (int c0 = 0; c0 < nch; c0 += 4) {               // four items' values in flight together
+        float m[4], lv[4], vv[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float* pc = pg + (size_t)(c0 + k) * PSTRIDE;
+          const bool on = c0 + k < nch;
+          m[k] = on ? __ldcg(pc + D) : -INFINITY;
+          lv[k] = on ? __ldcg(pc + D + 1) : 0.f;
+          vv[k] = on ? __ldcg(pc + dc) : 0.f;
+        }
+        const float Mn = fmaxf(fmaxf(M, fmaxf(m[0], m[1])), fmaxf(m[2], m[3]));
+        const float sc = exp2f(M - Mn);
+        acc *= sc; ls *= sc;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float w = exp2f(m[k] - Mn);
+          acc += w * vv[k];
+          ls += w * lv[k];
+        }
+        M = Mn;
+      }
+      orow[idx] = acc / ls;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// working sets + speculative eviction list; three independent jobs per unit, one CTA each; the last CTA decides
+// ------------------------------------------------------------------------------------------------------
+struct SelGeom {
+  static constexpr size_t BUF_BYTES = SEL_CAP * sizeof(double);
+  static constexpr size_t H_BYTES = (size_t)FB_PAD * 12;
+  static constexpr size_t MISC_BYTES = 8 * 8 + 8 * 4 + 8 * 8 + 16 * 4 + 16 * 4 + (8 * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
+};
+
+__global__ void __launch_bounds__(SEL_T, 2)
 gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
                float* __restrict__ out) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
   double* sbuf = reinterpret_cast<double*>(smem);                              // [SEL_CAP] a^S, a^L or s
   unsigned* hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::BUF_BYTES);
-  unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + NBINS_PAD);
-  unsigned long long* wsum = hsum + NBINS_PAD;                                 // [8]
+  unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + FB_PAD);   // two u32 planes (low, high)
+  unsigned long long* wsum = hsum + FB_PAD;                                    // [8]
   unsigned* wc = reinterpret_cast<unsigned*>(wsum + 8);                        // [8]
   long long* s_res = reinterpret_cast<long long*>(wc + 8);                     // [8]
   int* ev = reinterpret_cast<int*>(s_res + 8);                                 // [16]
@@ -341,51 +661,63 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   double* red = reinterpret_cast<double*>(s_i + 16);                           // [8][16]
   double* sM = red + 8 * 16;                                                   // [16]
   double* sZ = sM + 16;                                                        // [16]
-  unsigned* loc = reinterpret_cast<unsigned*>(sZ + 16);                        // [cap*b/32 + 1]
+  double* flist = sZ + 16;                                                     // [32] members of the crossing bin
+  int* flist_slot = reinterpret_cast<int*>(flist + 32);                        // [32]
+  unsigned* coarse = reinterpret_cast<unsigned*>(flist_slot + 32);             // [3][CBINS] summary bins
+  unsigned* loc = coarse + 3 * CBINS;                                          // [cap*b/32 + 1]
+  FastHist H;
+  H.cnt = hcnt; H.lo = reinterpret_cast<unsigned*>(hsum); H.hi = H.lo + FB_PAD;
+  H.ccnt = coarse; H.clo = coarse + CBINS; H.chi = coarse + 2 * CBINS;
   // the decision scratch aliases the score staging area: it is used after the last item only
 
   const int tid = threadIdx.x;
   const int LH = p.L * p.Hkv;
-  const int n_bnd = p.hdr[HDR_N_BND];
-  const long long items = (long long)n_bnd * LH * 3;
   const int G = p.G, G2 = 2 * p.G;
-
-  // ---- attention outputs of requests that were split over several work items: merge the partials -----------
+  // the first item's descriptor is fetched before the number of items is known (same round trip); slots of
+  // bnd_info past the count hold stale but readable data that is then not used
+  int4 inf_first = make_int4(0, 0, 0, 0), inf2_first = inf_first;
   {
-    const int n_mc = p.hdr[HDR_N_MC], n_rc = p.hdr[HDR_N_RC], D = p.d;
-    const int PSTRIDE = G * (D + 2);
-    for (long long mi = blockIdx.x; mi < (long long)n_mc * LH; mi += gridDim.x) {
-      const int4 mc = p.mc_list[mi / LH];
-      const int lh = (int)(mi % LH), l = lh / p.Hkv, h = lh % p.Hkv;
-      const int bi = mc.x, nch = mc.z;
-      const float* first = p.partials + ((size_t)lh * n_rc + mc.y) * PSTRIDE;
-      float* orow = out + (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
-      for (int idx = tid; idx < G * D; idx += SEL_T) {
-        const int g = idx / D, dc = idx % D;
-        const float* pg = first + g * (D + 2);
-        float M = -INFINITY;
-        for (int c = 0; c < nch; ++c) M = fmaxf(M, __ldcg(pg + (size_t)c * PSTRIDE + D));
-        float acc = 0.f, ls = 0.f;
-#pragma unroll 4
-        for (int c = 0; c < nch; ++c) {
-          const float* pc = pg + (size_t)c * PSTRIDE;
-          const float w = exp2f(__ldcg(pc + D) - M);
-          acc += w * __ldcg(pc + dc);
-          ls += w * __ldcg(pc + D + 1);
-        }
-        orow[idx] = acc / ls;
-      }
-    }
+    const int b0 = (int)(blockIdx.x / (3 * LH));
+    if (b0 < p.M) { inf_first = p.bnd_info[2 * b0]; inf2_first = p.bnd_info[2 * b0 + 1]; }
   }
+  const int n_bnd = p.hdr[HDR_N_BND];
+  const int n_mc = p.hdr[HDR_N_MC], n_rc = p.hdr[HDR_N_RC];
+  const long long items = (long long)n_bnd * LH * 3;
+  if (tid == 0) GP_T_STAMP(59);
 
-  for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+  // CTAs without a job merge the split requests' attention partials while the others work; when fewer than a
+  // quarter of the CTAs are idle, everybody merges after the jobs instead
+  const long long n_busy = items + n_bnd < (long long)gridDim.x ? items + n_bnd : (long long)gridDim.x;
+  const int n_idle = (int)gridDim.x - (int)n_busy;
+  const bool idle_merge = n_idle * 4 >= (int)gridDim.x;
+  if (idle_merge && (long long)blockIdx.x >= n_busy)
+    merge_partials(p, n_req, out, n_mc, n_rc, (int)blockIdx.x - (int)n_busy, n_idle);
+
+  if (tid == 0) GP_T_STAMP(60);
+  for (long long item = blockIdx.x; item < items + n_bnd; item += gridDim.x) {
+    if (item >= items) {
+      // pages of C that other requests share: each needs a copy-on-write target if this request compresses
+      const int e = (int)(item - items);
+      if (tid < 32) {
+        const int4 inf = p.bnd_info[2 * e];
+        const int* table = p.page_table + (size_t)inf.y * p.cap;
+        int ksh = 0;
+        for (int j = tid; j < inf.z - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
+        if (tid == 0) p.bnd_acc[4 * e + 2] = ksh;
+      }
+      continue;
+    }
     const long long u = item / 3;
     const int task = (int)(item % 3);               // 0: K^S, 1: K^L, 2: eviction list
     const int bidx = (int)(u / LH), lh = (int)(u % LH);
     const int l = lh / p.Hkv, h = lh % p.Hkv;
-    const int bi = p.bnd_list[bidx];
-    const int r = req_ids[bi];
-    const int Pr = p.P[r];
+    const bool is_first = item == (long long)blockIdx.x;
+    const int4 inf = is_first ? inf_first : p.bnd_info[2 * bidx];          // {slot in the batch, request, P}
+    const int4 inf2 = is_first ? inf2_first : p.bnd_info[2 * bidx + 1];    // {offset into the logit scratch}
+    const int r = inf.y, Pr = inf.z;
+    const long long off = (long long)(unsigned)inf2.x | ((long long)inf2.y << 32);
     const int nC = (Pr - 1) * GP_PAGE;
     int* Kout = p.Kx + (((size_t)r * p.L + l) * p.Hkv + h) * 2;
     int* evout = p.evict + (size_t)u * GP_PAGE;
@@ -396,70 +728,36 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     }
     const long long t_s0 = GP_T_NOW();
     (void)t_s0;
-    const long long off = p.bnd_off[bi];
     const double* z = p.zbuf + ((size_t)lh * p.max_batch_tokens + off) * G2;      // [nC][2][G]
     double* a = nC <= SEL_CAP ? sbuf : p.scores + ((size_t)task * LH + lh) * p.max_batch_tokens + off;
-    // ---- per-head softmax over C, then the group mean (Sec. 3.2) --------------------------------------------
-    // The attention kernel left, per 16-token page and column, the page's (max, sum of exponentials); they
-    // merge into the normalisers of the whole candidate set without another pass over the logits.
+    // the fast path's bins are cleared while the first loads of the softmax pass are in flight
+    fast_hist_zero(H, task < 2);
+    if (task == 2) for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
+    if (tid == 0) { s_res[0] = -1; s_i[0] = 0; s_i[5] = 0; s_i[6] = 0; s_i[7] = 0; }
+    bool uniform;
     {
-      const int ncols = task == 2 ? G2 : G;
-      const int col0 = task == 1 ? G : 0;
-      const int mycol = col0 + tid % ncols;                  // SEL_T is a multiple of ncols
-      const int ntile = nC / GP_PAGE;
       const double* zs = p.zstat + ((size_t)lh * (p.max_batch_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
-      double m = -INFINITY;
-      for (int t = tid / ncols; t < ntile; t += SEL_T / ncols) m = fmax(m, __ldcg(zs + ((size_t)t * G2 + mycol) * 2));
-      column_reduce<true>(m, ncols, red, sM);
-      const double mc = sM[tid % ncols];
-      double acc = 0.0;
-      for (int t = tid / ncols; t < ntile; t += SEL_T / ncols) {
-        const double2 ms = __ldcg(reinterpret_cast<const double2*>(zs + ((size_t)t * G2 + mycol) * 2));
-        acc += ms.y * exp(ms.x - mc);
+      switch (G) {
+        case 1: uniform = job_softmax<1>(z, zs, a, nC, task, red, sM, sZ); break;
+        case 2: uniform = job_softmax<2>(z, zs, a, nC, task, red, sM, sZ); break;
+        case 4: uniform = job_softmax<4>(z, zs, a, nC, task, red, sM, sZ); break;
+        default: uniform = job_softmax<8>(z, zs, a, nC, task, red, sM, sZ); break;
       }
-      column_reduce<false>(acc, ncols, red, sZ);
-      for (int i0 = tid; i0 < nC; i0 += 4 * SEL_T) {         // four tokens per thread in flight
-        double zv[4][16];
-#pragma unroll
-        for (int u4 = 0; u4 < 4; ++u4) {
-          const int i = i0 + u4 * SEL_T;
-          if (i < nC) {
-            const double* zr = z + (size_t)i * G2 + col0;
-            for (int g = 0; g < ncols; ++g) zv[u4][g] = __ldcg(zr + g);
-          }
-        }
-#pragma unroll
-        for (int u4 = 0; u4 < 4; ++u4) {
-          const int i = i0 + u4 * SEL_T;
-          if (i < nC) {
-            double s0 = 0.0, s1 = 0.0;
-            for (int g = 0; g < G; ++g) s0 += exp(zv[u4][g] - sM[g]) / sZ[g];
-            if (task == 2) {
-              for (int g = 0; g < G; ++g) s1 += exp(zv[u4][G + g] - sM[G + g]) / sZ[G + g];
-              a[i] = fmax(s0 / (double)G, s1 / (double)G);   // Eq. 9
-            } else {
-              a[i] = s0 / (double)G;
-            }
-          }
-        }
-      }
-      __syncthreads();
     }
     const long long t_s1 = GP_T_NOW();
     (void)t_s1;
     if (task < 2) {
       // ---- Eq. 7 -------------------------------------------------------------------------------------------
-      const int K = top_p_count<SEL_T>(p, a, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res);
+      int K = uniform ? top_p_fast(p, a, nC, p.p_fix, H, wc, wsum, s_res, flist, &s_i[5]) : -1;
+      if (K < 0) { __syncthreads(); K = top_p_count<SEL_T>(p, a, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res); }
       if (tid == 0) {
         Kout[task] = K;
+        atomicAdd(&p.bnd_acc[4 * bidx + task], K);            // Eq. 8 needs only the sums over layers and heads
         GP_T_ADD(16, 1); GP_T_ADD(17, t_s1 - t_s0); GP_T_ADD(18, GP_T_NOW() - t_s1); GP_T_ADD(25, nC);
       }
       continue;
     }
     // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
-    for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
-    if (tid == 0) s_i[0] = 0;
-    __syncthreads();
     const int nblk = Pr - 1;
     const int K_t = nC - GP_PAGE;
     const int kq = min(p.k_loc, K_t / nblk);
@@ -480,97 +778,102 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     const long long t_s3 = GP_T_NOW();
     (void)t_s3;
     // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
-    unsigned long long prefix = 0;
-    unsigned cnt_below = 0;
-    unsigned long long thr = 0;        // evict keys strictly below thr ...
-    unsigned long long tie_key = 0;    // ... and need_eq of the highest slots whose key equals tie_key
-    int need_eq = 0;
-    {
-      int shift = 63;
-      bool done = false;
-      for (int lvl = 0; lvl < 6 && !done; ++lvl) {
-        const int w = kWidths[lvl];
-        shift -= w;
-        const int nb = 1 << w;
-        for (int i = tid; i < nb + (nb >> 3); i += SEL_T) hcnt[i] = 0;
-        if (tid == 0) s_res[0] = -1;
-        __syncthreads();
-        for (int i = tid; i < nC; i += SEL_T) {
+    if (!uniform || !evict_fast(a, nC, loc, H, wc, s_res, flist, flist_slot, &s_i[6], ev)) {
+      __syncthreads();
+        unsigned long long prefix = 0;
+      unsigned cnt_below = 0;
+      unsigned long long thr = 0;        // evict keys strictly below thr ...
+      unsigned long long tie_key = 0;    // ... and need_eq of the highest slots whose key equals tie_key
+      int need_eq = 0;
+      {
+        int shift = 63;
+        bool done = false;
+        for (int lvl = 0; lvl < 6 && !done; ++lvl) {
+          const int w = kWidths[lvl];
+          shift -= w;
+          const int nb = 1 << w;
+          for (int i = tid; i < nb + (nb >> 3); i += SEL_T) hcnt[i] = 0;
+          if (tid == 0) s_res[0] = -1;
+          __syncthreads();
+          for (int i = tid; i < nC; i += SEL_T) {
+            if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
+              const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
+              if (lvl == 0 || (key >> (shift + w)) == prefix)
+                atomicAdd(&hcnt[HIDX((int)((key >> shift) & (unsigned long long)(nb - 1)))], 1u);
+            }
+          }
+          __syncthreads();
+          const int per = nb / SEL_T > 0 ? nb / SEL_T : 1;
+          const int lo = tid * per, hi = lo + per;
+          unsigned c = 0;
+          if (lo < nb) for (int b = lo; b < hi; ++b) c += hcnt[HIDX(b)];
+          const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
+          if (lo < nb) {
+            unsigned run = cnt_below + ex;
+            for (int b = lo; b < hi; ++b) {
+              const unsigned before = run;
+              run += hcnt[HIDX(b)];
+              if (before < (unsigned)GP_PAGE && run >= (unsigned)GP_PAGE) { s_res[0] = b; s_res[1] = before; }
+            }
+          }
+          __syncthreads();
+          if (s_res[0] < 0) {                                  // fewer than b candidates: cannot happen
+            if (tid == 0) atomicOr(p.err, GP_E_BOUNDS);
+            break;
+          }
+          const int bin_star = (int)s_res[0];
+          cnt_below = (unsigned)s_res[1];
+          const unsigned cstar = hcnt[HIDX(bin_star)];
+          __syncthreads();
+          prefix = (prefix << w) | (unsigned long long)bin_star;
+          if (cnt_below + cstar == (unsigned)GP_PAGE) {        // the bin fits exactly: no tie to break
+            thr = (prefix + 1ull) << shift;
+            done = true;
+          }
+        }
+        if (!done) {                                           // equal scores straddle the cut
+          thr = prefix;
+          tie_key = prefix;
+          need_eq = GP_PAGE - (int)cnt_below;
+        }
+      }
+      const long long t_s4 = GP_T_NOW();
+      (void)t_s4;
+      for (int i = tid; i < nC; i += SEL_T) {
+        if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
+          const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
+          if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < GP_PAGE) ev[at] = i; }
+        }
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int cntv = s_i[0];
+        for (int i = nC - 1; i >= 0 && need_eq > 0; --i) {     // rare: older (lower) slots win ties
           if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
             const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-            if (lvl == 0 || (key >> (shift + w)) == prefix)
-              atomicAdd(&hcnt[HIDX((int)((key >> shift) & (unsigned long long)(nb - 1)))], 1u);
+            if (key == tie_key) { if (cntv < GP_PAGE) ev[cntv] = i; ++cntv; --need_eq; }
           }
         }
-        __syncthreads();
-        const int per = nb / SEL_T > 0 ? nb / SEL_T : 1;
-        const int lo = tid * per, hi = lo + per;
-        unsigned c = 0;
-        if (lo < nb) for (int b = lo; b < hi; ++b) c += hcnt[HIDX(b)];
-        const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
-        if (lo < nb) {
-          unsigned run = cnt_below + ex;
-          for (int b = lo; b < hi; ++b) {
-            const unsigned before = run;
-            run += hcnt[HIDX(b)];
-            if (before < (unsigned)GP_PAGE && run >= (unsigned)GP_PAGE) { s_res[0] = b; s_res[1] = before; }
-          }
-        }
-        __syncthreads();
-        if (s_res[0] < 0) {                                  // fewer than b candidates: cannot happen
-          if (tid == 0) atomicOr(p.err, GP_E_BOUNDS);
-          break;
-        }
-        const int bin_star = (int)s_res[0];
-        cnt_below = (unsigned)s_res[1];
-        const unsigned cstar = hcnt[HIDX(bin_star)];
-        __syncthreads();
-        prefix = (prefix << w) | (unsigned long long)bin_star;
-        if (cnt_below + cstar == (unsigned)GP_PAGE) {        // the bin fits exactly: no tie to break
-          thr = (prefix + 1ull) << shift;
-          done = true;
-        }
-      }
-      if (!done) {                                           // equal scores straddle the cut
-        thr = prefix;
-        tie_key = prefix;
-        need_eq = GP_PAGE - (int)cnt_below;
-      }
-    }
-    const long long t_s4 = GP_T_NOW();
-    (void)t_s4;
-    for (int i = tid; i < nC; i += SEL_T) {
-      if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-        const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-        if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < GP_PAGE) ev[at] = i; }
+        if (cntv != GP_PAGE) atomicOr(p.err, GP_E_BOUNDS);
+        GP_T_ADD(21, GP_T_NOW() - t_s4);
       }
     }
     __syncthreads();
-    if (tid == 0) {
-      GP_T_ADD(31, 1); GP_T_ADD(19, t_s3 - t_s1); GP_T_ADD(20, t_s4 - t_s3); GP_T_ADD(22, t_s1 - t_s0);
-      int cntv = s_i[0];
-      for (int i = nC - 1; i >= 0 && need_eq > 0; --i) {     // rare: older (lower) slots win ties
-        if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-          const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-          if (key == tie_key) { if (cntv < GP_PAGE) ev[cntv] = i; ++cntv; --need_eq; }
-        }
-      }
-      if (cntv != GP_PAGE) atomicOr(p.err, GP_E_BOUNDS);
-      for (int x = 1; x < GP_PAGE; ++x) {                    // sort the 16 slots ascending
-        const int key = ev[x];
-        int b2 = x - 1;
-        while (b2 >= 0 && ev[b2] > key) { ev[b2 + 1] = ev[b2]; --b2; }
-        ev[b2 + 1] = key;
-      }
-      for (int x = 0; x < GP_PAGE; ++x) evout[x] = ev[x];
-      GP_T_ADD(21, GP_T_NOW() - t_s4);
+    if (tid < GP_PAGE) {                                     // the 16 slots in ascending order, by rank
+      const int mine = ev[tid];
+      int rank = 0;
+#pragma unroll
+      for (int j = 0; j < GP_PAGE; ++j) rank += (ev[j] < mine);
+      evout[rank] = mine;
     }
+    if (tid == 0) { GP_T_ADD(31, 1); GP_T_ADD(19, t_s3 - t_s1); GP_T_ADD(20, GP_T_NOW() - t_s3); GP_T_ADD(22, t_s1 - t_s0); }
   }
 
   // ---- the last CTA takes the decisions ----------------------------------------------------------------------
-  __threadfence();
+  if (tid == 0) GP_T_STAMP(61);
   __syncthreads();
   if (tid == 0) {
+    __threadfence();
     const int prev = atomicAdd(&p.hdr[HDR_DONE_SEL], 1);
     s_i[2] = (prev == (int)gridDim.x - 1);
     if (prev == (int)gridDim.x - 1) p.hdr[HDR_DONE_SEL] = 0;
@@ -580,9 +883,13 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     __threadfence();
     const long long t_d0 = GP_T_NOW();
     (void)t_d0;
-    decide_and_allocate(p, req_ids, n_req, actions, reinterpret_cast<int*>(sbuf));
+    if (tid == 0) GP_T_STAMP(62);
+    decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(sbuf));
+    if (tid == 0) GP_T_STAMP(63);
     if (tid == 0) { GP_T_ADD(23, GP_T_NOW() - t_d0); GP_T_ADD(24, 1); }
   }
+
+  if (!idle_merge) merge_partials(p, n_req, out, n_mc, n_rc, (int)gridDim.x - 1 - (int)blockIdx.x, (int)gridDim.x);
 }
 
 // ------------------------------------------------------------------------------------------------------
@@ -594,41 +901,50 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   constexpr int CH = D / 8;
   constexpr int ROW_BYTES = D * 2;
   constexpr int PIECES = MOVE_TOK * 2 * CH / CT;        // 16-byte pieces per thread per chunk
-  __shared__ int s_pref[GP_MAX_REQ + 1];
+  __shared__ int4 s_info[GP_MAX_REQ + 1];     // compressing requests: {request, P, boundary index, first chunk}
   __shared__ int ev[GP_PAGE];
   __shared__ int s_i[8];
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int LH = p.L * p.Hkv;
+  // the first round trip fetches everything at once: the header, the list of compressing requests (its first
+  // CT entries before their count is known; entries past the count are never looked at) and the first ticket
+  if (tid == 0) { GP_T_STAMP(36); s_i[0] = atomicAdd(&p.hdr[HDR_WORK_CMP], 1); s_i[3] = 0; }
+  if (tid <= p.M) s_info[tid] = p.cmp_info[tid];
   const int n_cmp = p.hdr[HDR_N_CMP];
   const int n_items = p.hdr[HDR_N_CITEM];
+  const int n_cow = p.hdr[HDR_N_COW];
   const int stamp = p.hdr[HDR_STEP];
-  for (int i = tid; i <= n_cmp; i += CT) s_pref[i] = p.cmp_chunk0[i];
-  if (tid == 0) s_i[3] = 0;
-  __syncthreads();
+  for (int i = tid + CT; i <= n_cmp; i += CT) s_info[i] = p.cmp_info[i];
 
-  for (;;) {
+  const long long t_c0 = GP_T_NOW();
+  (void)t_c0;
+  for (bool first = true;; first = false) {
     __syncthreads();
-    if (tid == 0) s_i[0] = n_items > 0 ? atomicAdd(&p.hdr[HDR_WORK_CMP], 1) : 0x7fffffff;
-    __syncthreads();
+    const long long t_c1 = GP_T_NOW();
+    (void)t_c1;
+    if (!first) {
+      if (tid == 0) s_i[0] = atomicAdd(&p.hdr[HDR_WORK_CMP], 1);
+      __syncthreads();
+    }
     const int item = s_i[0];
     if (item >= n_items) break;
+    if (tid == 0) { GP_T_ADD(48, 1); GP_T_ADD(49, GP_T_NOW() - t_c1); }
     // item -> (compressing request, layer/head, chunk); chunks of a unit are consecutive and ascending
     int lo = 0, hi = n_cmp;
-    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (LH * s_pref[mid] <= item) lo = mid; else hi = mid; }
-    const int ci = lo;
-    const int nchunk = s_pref[ci + 1] - s_pref[ci];
-    const int rem = item - LH * s_pref[ci];
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (LH * s_info[mid].w <= item) lo = mid; else hi = mid; }
+    const int4 inf = s_info[lo];
+    const int nchunk = s_info[lo + 1].w - inf.w;
+    const int rem = item - LH * inf.w;
     const int lh = rem / nchunk, j = rem % nchunk;
     const int l = lh / p.Hkv, h = lh % p.Hkv;
-    const int bi = p.cmp_list[ci];
-    const int r = req_ids[bi];
-    const int Pr = p.P[r];
-    const int n_src = Pr * GP_PAGE;
+    const int r = inf.x;
+    const int Pr = inf.y;
     const int* table = p.page_table + (size_t)r * p.cap;
     const int* shadow = p.shadow + (size_t)r * p.cap;
-    if (tid < GP_PAGE) ev[tid] = p.evict[((size_t)p.cmp_bnd[ci] * LH + lh) * GP_PAGE + tid];
+    if (tid < GP_PAGE) ev[tid] = p.evict[((size_t)inf.z * LH + lh) * GP_PAGE + tid];
     __syncthreads();
+    const int n_src = Pr * GP_PAGE;
     const int c0 = j * MOVE_TOK;
 
     uint4 val[PIECES];
@@ -670,6 +986,8 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         }
       }
     }
+    const long long t_c2 = GP_T_NOW();
+    (void)t_c2;
     // Touch every loaded value so that the loads have completed before the flag below is published: the
     // next chunk's CTA may overwrite the tail of this chunk's sources as soon as it sees the flag.
     unsigned touched = (unsigned)tokv;
@@ -689,6 +1007,9 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
       }
     }
     __syncthreads();
+    const long long t_c3 = GP_T_NOW();
+    (void)t_c3;
+    if (tid == 0) { GP_T_ADD(50, t_c2 - t_c1); GP_T_ADD(51, t_c3 - t_c2); }
 #pragma unroll
     for (int k2 = 0; k2 < PIECES; ++k2) {
       if (dst_code[k2] >= 0) {
@@ -708,10 +1029,12 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
     }
   }
   __syncthreads();
+  if (tid == 0) { GP_T_ADD(52, GP_T_NOW() - t_c0); GP_T_ADD(53, 1); GP_T_STAMP(37); GP_T_STAMP(38); }
   if (tid == 0 && s_i[3] > 0)
     atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 8), (unsigned long long)s_i[3]);
 
   // ---- the last CTA swaps in the copy-on-write targets and drops the old references (App. D.2) ----------
+  if (n_cow == 0) return;                                 // nothing was shared: no targets to swap in
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -723,8 +1046,8 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   if (s_i[2] && tid < 32) {
     __threadfence();
     for (int ci = 0; ci < n_cmp; ++ci) {
-      const int r = req_ids[p.cmp_list[ci]];
-      const int Pr = p.P[r];
+      const int r = s_info[ci].x;
+      const int Pr = s_info[ci].y;
       int* table = p.page_table + (size_t)r * p.cap;
       int* shadow = p.shadow + (size_t)r * p.cap;
       for (int j0 = 0; j0 < Pr - 1; j0 += 32) {
@@ -748,6 +1071,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
       }
     }
   }
+  if (tid == 0) GP_T_STAMP(38);
 }
 
 }  // namespace
@@ -756,10 +1080,23 @@ size_t gp_bsel_smem(const GpDev& p) {
   return SelGeom::BUF_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
 }
 
+// one-time setup for a pool: opts the selection kernel into its shared memory and sizes both grids to
+// exactly one resident wave, so that no CTA waits for another to leave before it can start
+void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact) {
+  const size_t sel_sm = gp_bsel_smem(p);
+  cudaFuncSetAttribute(gp_bsel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
+  int occ = 0;
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_bsel_kernel, SEL_T, sel_sm);
+  *grid_sel = num_sms * (occ > 0 ? occ : 1);
+  occ = 0;
+  if (p.d == 128) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_compact_kernel<128>, CT, 0);
+  else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_compact_kernel<64>, CT, 0);
+  *grid_compact = num_sms * (occ > 0 ? occ : 1);
+}
+
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
                         int grid_compact, cudaStream_t s, cudaEvent_t ev) {
   const size_t sel_sm = gp_bsel_smem(p);
-  cudaFuncSetAttribute(gp_bsel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
   gp_bsel_kernel<<<grid_sel, SEL_T, sel_sm, s>>>(p, req_ids, n_req, actions, out);
   if (ev) cudaEventRecord(ev, s);
   if (p.d == 128) gp_compact_kernel<128><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);

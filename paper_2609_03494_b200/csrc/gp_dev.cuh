@@ -42,6 +42,7 @@ enum {
   HDR_WORK_CMP,      // ticket counter of the compaction kernel
   HDR_N_CITEM,       // compaction work items (chunks x layers x heads)
   HDR_N_MC,          // requests whose attention was split over several work items
+  HDR_N_COW,         // copy-on-write targets allotted this step
   HDR_COUNT = 16
 };
 
@@ -83,11 +84,10 @@ struct GpDev {
   int* b_flags;                          // [M] 1 = stepped this step
   int* first_idx;                        // [M] lowest batch index naming a request
   int4* mc_list;                         // [M] split requests: {batch index, first partial, chunks, 0}
-  int* bnd_list;                         // [M] batch indices at a boundary
-  long long* bnd_off;                    // [M] token offset into the score scratch
-  int* cmp_list;                         // [M] batch indices that compress
-  int* cmp_bnd;                          // [M] their index in bnd_list
-  int* cmp_chunk0;                       // [M+1] prefix of their compaction chunk counts
+  int4* bnd_info;                        // [M][2] requests at a boundary: {slot in the batch, request, P, 0}, {score offset lo, hi, 0, 0}
+  int* bnd_acc;                          // [M][4] per boundary request: sum of K^S, sum of K^L, shared pages of C, 0
+  int* free_peek;                        // [M+1] free_top at plan time, then the top entries of the free list, top first
+  int4* cmp_info;                        // [M+1] compressing requests: {request, P, index in bnd_info, first compaction chunk}
   double* zbuf;                          // [L*H_kv][max_batch_tokens][2][G] summary logits of boundary units
   double* zstat;                         // [L*H_kv][max_batch_tokens / b][2][G][2] per-page softmax partials (max, sum)
   int* sum_par;                          // [M] which of the two summary buffers is current
@@ -115,12 +115,14 @@ __device__ __forceinline__ size_t gp_summ_off(const GpDev& p, int l, int r, int 
 
 // ---- optional cycle trace (compiled in only with -DGP_TRACE, for development builds) ----------------
 #ifdef GP_TRACE
-#define GP_TRACE_WORDS 32
+#define GP_TRACE_WORDS 64
 #define GP_T_ADD(slot, val) atomicAdd(reinterpret_cast<unsigned long long*>(&p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + (slot)]), (unsigned long long)(val))
 #define GP_T_NOW() clock64()
+#define GP_T_STAMP(slot) do { unsigned long long gt_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + (slot)] = (long long)gt_; } while (0)
 #else
 #define GP_T_ADD(slot, val) do { } while (0)
 #define GP_T_NOW() 0ll
+#define GP_T_STAMP(slot) do { } while (0)
 #endif
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -197,5 +199,7 @@ size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
 // boundary chain: probabilities + working sets + selection + decision, then compaction.
 // `ev`, when not null, is recorded between the two kernels.
+void gp_attention_setup(const GpDev& p);
+void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact);
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
                         int grid_compact, cudaStream_t s, cudaEvent_t ev);

@@ -11,8 +11,6 @@
 #include "../../include/growpage.h"
 #include "gp_dev.cuh"
 
-#define GP_SEL_GRID 444         // three 256-thread CTAs per SM
-#define GP_COMPACT_GRID 592     // 4 CTAs per SM
 #define GP_PLAN_THREADS 1024
 
 struct gp_pool {
@@ -22,7 +20,7 @@ struct gp_pool {
   void* blob;
   size_t bytes;
   std::vector<uint8_t> live;      // host mirror of the slot free list
-  int num_sms, attn_grid;
+  int num_sms, attn_grid, sel_grid, compact_grid;
   // staging for the host-pointer entry point (inside the blob)
   int* st_ids; void* st_q; void* st_k; void* st_v; float* st_out; int* st_act;
   // small device words
@@ -51,7 +49,7 @@ namespace {
 
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
-      b_flags, mc_list, bnd_list, bnd_off, cmp_list, cmp_bnd, cmp_chunk0, zbuf, zstat, sum_par,
+      b_flags, mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, zstat, sum_par,
       evict, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
   int max_rc;
@@ -114,11 +112,10 @@ Layout make_layout(const gp_config& c) {
   L.b_nold = take(M * 4);
   L.b_flags = take(M * 4);
   L.mc_list = take(M * 16);
-  L.bnd_list = take(M * 4);
-  L.bnd_off = take(M * 8);
-  L.cmp_list = take(M * 4);
-  L.cmp_bnd = take(M * 4);
-  L.cmp_chunk0 = take((M + 1) * 4);
+  L.bnd_info = take(M * 32);
+  L.bnd_acc = take(M * 16);
+  L.free_peek = take((M + 1) * 4);
+  L.cmp_info = take((M + 1) * 16);
   L.zbuf = take(LH * (size_t)L.max_batch_tokens * 2 * G * 8);
   L.zstat = take(LH * ((size_t)L.max_batch_tokens / b + 1) * 2 * G * 2 * 8);
   L.evict = take(M * LH * b * 4);
@@ -197,8 +194,10 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
   __shared__ int s_chunks[GP_MAX_REQ], s_pos[GP_MAX_REQ];
   __shared__ int s_bin[GP_COST_BINS], s_binbase[GP_COST_BINS], s_nmc;
+  __shared__ int s_peek[GP_MAX_REQ];       // the free list from its top down, for the decisions of this step
   const int i = threadIdx.x;
   const bool in = i < n_req;
+  const int free_top0 = *p.free_top;
   const long long t_plan0 = GP_T_NOW();
   (void)t_plan0;
   s_first[i] = 0x7fffffff;
@@ -218,6 +217,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   if (in) {
     const bool inrange = r >= 0 && r < p.M;
     int live = 0;
+    if (i < free_top0) s_peek[i] = p.free_stack[free_top0 - 1 - i];
     if (inrange) {                    // independent loads, issued together
       live = p.live[r]; n_old = p.n[r]; Pr = p.P[r]; pos = p.pos[r]; started = p.started[r]; par = p.sum_par[r];
     }
@@ -280,7 +280,12 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     p.b_nold[i] = n_old;
     p.b_flags[i] = chunks > 0;
     actions[i] = act;
-    if (isb) { p.bnd_list[bnd_idx] = i; p.bnd_off[i] = tok_off; }
+    if (isb) {
+      p.bnd_info[2 * bnd_idx] = make_int4(i, r, Pr, 0);
+      p.bnd_info[2 * bnd_idx + 1] = make_int4((int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32), 0, 0);
+      reinterpret_cast<int4*>(p.bnd_acc)[bnd_idx] = make_int4(0, 0, 0, 0);
+      if (bnd_idx < free_top0) p.free_peek[1 + bnd_idx] = s_peek[bnd_idx];
+    }
     // descriptors of this request's chunks: four 16-byte stores each
     const int flags = isb | (started ? 2 : 0);
     for (int c = 0; c < chunks; ++c) {
@@ -311,6 +316,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (threadIdx.x == 0) {
     p.hdr[HDR_N_MC] = s_nmc;
+    p.free_peek[0] = free_top0;
     GP_T_ADD(26, 1); GP_T_ADD(27, t_plan1 - t_plan0); GP_T_ADD(28, t_plan2 - t_plan1); GP_T_ADD(29, GP_T_NOW() - t_plan2);
     p.hdr[HDR_N_RC] = n_rc;
     p.hdr[HDR_N_BND] = n_bnd;
@@ -510,11 +516,10 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.b_nold = reinterpret_cast<int*>(base + L.b_nold);
   d.b_flags = reinterpret_cast<int*>(base + L.b_flags);
   d.mc_list = reinterpret_cast<int4*>(base + L.mc_list);
-  d.bnd_list = reinterpret_cast<int*>(base + L.bnd_list);
-  d.bnd_off = reinterpret_cast<long long*>(base + L.bnd_off);
-  d.cmp_list = reinterpret_cast<int*>(base + L.cmp_list);
-  d.cmp_bnd = reinterpret_cast<int*>(base + L.cmp_bnd);
-  d.cmp_chunk0 = reinterpret_cast<int*>(base + L.cmp_chunk0);
+  d.bnd_info = reinterpret_cast<int4*>(base + L.bnd_info);
+  d.bnd_acc = reinterpret_cast<int*>(base + L.bnd_acc);
+  d.free_peek = reinterpret_cast<int*>(base + L.free_peek);
+  d.cmp_info = reinterpret_cast<int4*>(base + L.cmp_info);
   d.zbuf = reinterpret_cast<double*>(base + L.zbuf);
   d.zstat = reinterpret_cast<double*>(base + L.zstat);
   d.sum_par = reinterpret_cast<int*>(base + L.sum_par);
@@ -532,6 +537,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   }
   d.trace = g_trace_dev;
 #endif
+  gp_attention_setup(d);
+  gp_boundary_setup(d, pool->num_sms, &pool->sel_grid, &pool->compact_grid);
   pool->dbg = base + L.dbg;
   if (cfg->host_staging) {
     pool->st_ids = reinterpret_cast<int*>(base + L.st_ids);
@@ -614,7 +621,7 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   if (prof) cudaEventRecord(pool->ev[1], s);
   gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s);
   if (prof) cudaEventRecord(pool->ev[2], s);
-  gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), GP_SEL_GRID, GP_COMPACT_GRID, s,
+  gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s,
                      prof ? pool->ev[3] : nullptr);
   if (prof) cudaEventRecord(pool->ev[4], s);
   pool->launch_count += GP_N_KERNELS;
