@@ -125,6 +125,8 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     s_misc[0] = 0;
     fence_mbar_init();
   }
+  gp_pdl_wait();                  // everything above touched only this CTA's shared memory
+  gp_pdl_launch_dependents();
   __syncthreads();
 
   const int n_rc = p.hdr[HDR_N_RC];
@@ -467,28 +469,37 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
             // D fragment: row = grp (token), columns 2*t4, 2*t4 + 1
             const int col = nt * 8 + 2 * t4;
             z00 /= sqrt_d; z01 /= sqrt_d; z10 /= sqrt_d; z11 /= sqrt_d;
-            // the page's softmax partials per column: max and sum of exponentials over its 16 tokens
+            // the page's softmax partials per column: max and sum of exponentials over its 16 tokens; the
+            // exponentials themselves are what is stored per token
             double m0 = fmax(z00, z10), m1 = fmax(z01, z11);
 #pragma unroll
             for (int o2 = 4; o2 < 32; o2 <<= 1) {
               m0 = fmax(m0, __shfl_xor_sync(0xffffffffu, m0, o2));
               m1 = fmax(m1, __shfl_xor_sync(0xffffffffu, m1, o2));
             }
-            double e0 = exp(z00 - m0) + exp(z10 - m0), e1 = exp(z01 - m1) + exp(z11 - m1);
+            z00 = exp(z00 - m0); z10 = exp(z10 - m0); z01 = exp(z01 - m1); z11 = exp(z11 - m1);
+            double e0 = z00 + z10, e1 = z01 + z11;
 #pragma unroll
             for (int o2 = 4; o2 < 32; o2 <<= 1) {
               e0 += __shfl_xor_sync(0xffffffffu, e0, o2);
               e1 += __shfl_xor_sync(0xffffffffu, e1, o2);
             }
             if (col < 2 * G) {
-              double* z0 = p.zbuf + ((size_t)lh * p.max_batch_tokens + zoff + tok0 + grp) * (2 * G) + col;
-              double* z1 = z0 + (size_t)8 * (2 * G);
-              z0[0] = z00; z1[0] = z10;
-              if (col + 1 < 2 * G) { z0[1] = z01; z1[1] = z11; }
+              // view = col / G (short or long summary); a view's values of one unit are contiguous [token][G]
+              const size_t tokrow = (size_t)(zoff + tok0 + grp);
+              if (G >= 2) {
+                double* z0 = p.zbuf + (((size_t)lh * 2 + col / G) * p.z_stride + tokrow) * G + col % G;
+                *reinterpret_cast<double2*>(z0) = make_double2(z00, z01);
+                *reinterpret_cast<double2*>(z0 + (size_t)8 * G) = make_double2(z10, z11);
+              } else {
+                double* zS = p.zbuf + ((size_t)lh * 2 * p.z_stride + tokrow);
+                double* zL = zS + p.z_stride;
+                zS[0] = z00; zS[8] = z10; zL[0] = z01; zL[8] = z11;
+              }
               if (grp == 0) {
                 double* st2 = p.zstat + (((size_t)lh * (p.max_batch_tokens / GP_PAGE) + (zoff + tok0) / GP_PAGE) * (2 * G) + col) * 2;
-                st2[0] = m0; st2[1] = e0;
-                if (col + 1 < 2 * G) { st2[2] = m1; st2[3] = e1; }
+                *reinterpret_cast<double2*>(st2) = make_double2(m0, e0);
+                *reinterpret_cast<double2*>(st2 + 2) = make_double2(m1, e1);
               }
             }
           }
@@ -684,7 +695,7 @@ void gp_attention_setup(const GpDev& p) {           // once per pool: opt into t
 }
 
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s) {
+                         float* out, int grid, cudaStream_t s, bool pdl) {
   (void)req_ids;
   const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kk = static_cast<const __nv_bfloat16*>(k);
@@ -694,7 +705,7 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
 #define GP_LAUNCH(DD, RR)                                                                 \
   do {                                                                                    \
     auto kern = gp_attn_kernel<DD, RR>;                                                   \
-    kern<<<grid, NTHREADS, sm, s>>>(p, n_req, qq, kk, vv, out);                          \
+    gp_launch(kern, grid, NTHREADS, (size_t)sm, s, pdl, p, n_req, qq, kk, vv, out);       \
   } while (0)
   if (p.d == 128) {
     if (rope) GP_LAUNCH(128, true); else GP_LAUNCH(128, false);

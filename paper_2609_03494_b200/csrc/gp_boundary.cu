@@ -27,7 +27,8 @@ constexpr int NBINS = 2048;
 constexpr int NBINS_PAD = NBINS + NBINS / 8;     // bins are stored at b + (b >> 3): a thread's 8 consecutive bins and
 #define HIDX(b) ((b) + ((b) >> 3))              // its neighbours' then fall into different banks
 constexpr double TWO62 = 4611686018427387904.0;
-constexpr int SEL_T = 256;           // threads of the selection kernel
+constexpr int SEL_T = 512;           // threads of the selection kernel
+constexpr int SEL_NW = SEL_T / 32;
 constexpr int SEL_CAP = 6144;        // candidate tokens whose scores are staged in shared memory
 constexpr int CT = 256;              // threads of the compaction kernel
 constexpr int MOVE_TOK = GP_MOVE_TOK;     // source slots per compaction chunk
@@ -40,7 +41,7 @@ struct PairCU { unsigned c; unsigned long long s; };
 
 // exclusive suffix sum over the block: sum of the values of threads with a higher id
 template <int BT>
-__device__ __forceinline__ PairCU block_suffix_excl(unsigned c, unsigned long long s, unsigned* wc,
+__device__ __noinline__ PairCU block_suffix_excl(unsigned c, unsigned long long s, unsigned* wc,
                                                     unsigned long long* wsum) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned ic = c; unsigned long long is = s;
@@ -59,7 +60,7 @@ __device__ __forceinline__ PairCU block_suffix_excl(unsigned c, unsigned long lo
 }
 // exclusive prefix count over the block
 template <int BT>
-__device__ __forceinline__ unsigned block_prefix_excl(unsigned c, unsigned* wc) {
+__device__ __noinline__ unsigned block_prefix_excl(unsigned c, unsigned* wc) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned ic = c;
 #pragma unroll
@@ -137,7 +138,6 @@ __device__ __noinline__ int top_p_count(const GpDev& p, const double* a, int n, 
       }
     }
     __syncthreads();
-    if (tid == 0) { GP_T_ADD(30, 1); GP_T_ADD(12, t_l1 - t_l0); GP_T_ADD(13, t_l2 - t_l1); GP_T_ADD(14, GP_T_NOW() - t_l2); }
     if (s_res[0] < 0) return n;                  // rounding kept the total below p: everything
     bin_star = (int)s_res[0];
     cnt_above = (unsigned)s_res[1];
@@ -171,7 +171,7 @@ constexpr int FBINS = 4096;
 constexpr int FB_PAD = FBINS + FBINS / 16;       // plane stride (the general routine pads its bins)
 constexpr int CBINS = 256;                       // summary bins: 16 fine bins each, one per thread
 constexpr int FSHIFT = 46;
-static_assert(CBINS == SEL_T, "one summary bin per thread");
+static_assert(CBINS <= SEL_T, "one summary bin per thread");
 
 struct FastHist {
   unsigned* cnt; unsigned* lo; unsigned* hi;       // [FBINS] members, and their fixed-point mass in two halves
@@ -184,8 +184,10 @@ __device__ __forceinline__ void fast_hist_zero(const FastHist& H, bool with_mass
     reinterpret_cast<uint4*>(H.cnt)[i] = z;
     if (with_mass) { reinterpret_cast<uint4*>(H.lo)[i] = z; reinterpret_cast<uint4*>(H.hi)[i] = z; }
   }
-  H.ccnt[threadIdx.x] = 0;
-  if (with_mass) { H.clo[threadIdx.x] = 0; H.chi[threadIdx.x] = 0; }
+  if (threadIdx.x < CBINS) {
+    H.ccnt[threadIdx.x] = 0;
+    if (with_mass) { H.clo[threadIdx.x] = 0; H.chi[threadIdx.x] = 0; }
+  }
 }
 
 // sorts (v, tag) across the 32 lanes: descending v when DESC, else ascending v with larger tag first among
@@ -225,10 +227,10 @@ __device__ int top_p_fast(const GpDev& p, const double* a, int n, unsigned long 
   __syncthreads();
   const long long f3 = GP_T_NOW(); (void)f3;
   {                                               // summary level: thread t owns bin t; higher bins = larger scores
-    const unsigned c = H.ccnt[tid];
-    const unsigned long long m = ((unsigned long long)H.chi[tid] << 32) + H.clo[tid];
+    const unsigned c = tid < CBINS ? H.ccnt[tid] : 0u;
+    const unsigned long long m = tid < CBINS ? ((unsigned long long)H.chi[tid] << 32) + H.clo[tid] : 0ull;
     const PairCU ex = block_suffix_excl<SEL_T>(c, m, wc, wsum);
-    if (ex.s < p_fix && ex.s + m >= p_fix) { s_res[0] = tid; s_res[1] = ex.c; s_res[2] = (long long)ex.s; }
+    if (tid < CBINS && ex.s < p_fix && ex.s + m >= p_fix) { s_res[0] = tid; s_res[1] = ex.c; s_res[2] = (long long)ex.s; }
   }
   __syncthreads();
   if (s_res[0] < 0) return n;                    // rounding kept the total below p: everything
@@ -294,9 +296,9 @@ __device__ bool evict_fast(const double* a, int nC, const unsigned* loc, const F
   }
   __syncthreads();
   {                                               // summary level, ascending: the b lowest scores go
-    const unsigned c = H.ccnt[tid];
+    const unsigned c = tid < CBINS ? H.ccnt[tid] : 0u;
     const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
-    if (ex < (unsigned)GP_PAGE && ex + c >= (unsigned)GP_PAGE) { s_res[0] = tid; s_res[1] = ex; }
+    if (tid < CBINS && ex < (unsigned)GP_PAGE && ex + c >= (unsigned)GP_PAGE) { s_res[0] = tid; s_res[1] = ex; }
   }
   __syncthreads();
   if (s_res[0] < 0) return false;
@@ -335,10 +337,94 @@ __device__ bool evict_fast(const double* a, int nC, const unsigned* loc, const F
   return true;
 }
 
+// Eq. 10 global cut, general routine (radix descent over the score bits): lists the b evicted slots in ev[]
+__device__ __noinline__ void evict_general(const GpDev& p, const double* a, int nC, const unsigned* loc, unsigned* hcnt,
+                                           unsigned* wc, long long* s_res, int* s_i, int* ev) {
+  const int tid = threadIdx.x;
+      __syncthreads();
+    unsigned long long prefix = 0;
+  unsigned cnt_below = 0;
+  unsigned long long thr = 0;        // evict keys strictly below thr ...
+  unsigned long long tie_key = 0;    // ... and need_eq of the highest slots whose key equals tie_key
+  int need_eq = 0;
+  {
+    int shift = 63;
+    bool done = false;
+    for (int lvl = 0; lvl < 6 && !done; ++lvl) {
+      const int w = kWidths[lvl];
+      shift -= w;
+      const int nb = 1 << w;
+      for (int i = tid; i < nb + (nb >> 3); i += SEL_T) hcnt[i] = 0;
+      if (tid == 0) s_res[0] = -1;
+      __syncthreads();
+      for (int i = tid; i < nC; i += SEL_T) {
+        if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
+          const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
+          if (lvl == 0 || (key >> (shift + w)) == prefix)
+            atomicAdd(&hcnt[HIDX((int)((key >> shift) & (unsigned long long)(nb - 1)))], 1u);
+        }
+      }
+      __syncthreads();
+      const int per = nb / SEL_T > 0 ? nb / SEL_T : 1;
+      const int lo = tid * per, hi = lo + per;
+      unsigned c = 0;
+      if (lo < nb) for (int b = lo; b < hi; ++b) c += hcnt[HIDX(b)];
+      const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
+      if (lo < nb) {
+        unsigned run = cnt_below + ex;
+        for (int b = lo; b < hi; ++b) {
+          const unsigned before = run;
+          run += hcnt[HIDX(b)];
+          if (before < (unsigned)GP_PAGE && run >= (unsigned)GP_PAGE) { s_res[0] = b; s_res[1] = before; }
+        }
+      }
+      __syncthreads();
+      if (s_res[0] < 0) {                                  // fewer than b candidates: cannot happen
+        if (tid == 0) atomicOr(p.err, GP_E_BOUNDS);
+        break;
+      }
+      const int bin_star = (int)s_res[0];
+      cnt_below = (unsigned)s_res[1];
+      const unsigned cstar = hcnt[HIDX(bin_star)];
+      __syncthreads();
+      prefix = (prefix << w) | (unsigned long long)bin_star;
+      if (cnt_below + cstar == (unsigned)GP_PAGE) {        // the bin fits exactly: no tie to break
+        thr = (prefix + 1ull) << shift;
+        done = true;
+      }
+    }
+    if (!done) {                                           // equal scores straddle the cut
+      thr = prefix;
+      tie_key = prefix;
+      need_eq = GP_PAGE - (int)cnt_below;
+    }
+  }
+  const long long t_s4 = GP_T_NOW();
+  (void)t_s4;
+  for (int i = tid; i < nC; i += SEL_T) {
+    if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
+      const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
+      if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < GP_PAGE) ev[at] = i; }
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int cntv = s_i[0];
+    for (int i = nC - 1; i >= 0 && need_eq > 0; --i) {     // rare: older (lower) slots win ties
+      if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
+        const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
+        if (key == tie_key) { if (cntv < GP_PAGE) ev[cntv] = i; ++cntv; --need_eq; }
+      }
+    }
+    if (cntv != GP_PAGE) atomicOr(p.err, GP_E_BOUNDS);
+    GP_T_ADD(21, GP_T_NOW() - t_s4);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------------
 // decision + allocator, run by the last CTA of the selection kernel
 // ------------------------------------------------------------------------------------------------------
-__device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr) {
+__device__ __noinline__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr) {
   int* s_want = s_arr;
   int* s_ksh = s_arr + GP_MAX_REQ;
   int* s_P = s_arr + 2 * GP_MAX_REQ;
@@ -484,21 +570,24 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
   }
 }
 
-// a^x of one token from its logits: sum over the group of exp(z - max) * 1 / (G Z); G is a template
-// parameter so that the exponentials of a thread's tokens overlap
-__device__ __forceinline__ double exp_once(double x) { return exp(x); }
+// one copy of the fp64 exponential in the image: the selection jobs run once per launch, so what they cost
+// is mostly the fetching of their instructions
+__device__ __noinline__ double exp_once(double x) { return exp(x); }
+// factor of a page and column when the factors' table does not fit (very large candidate sets)
+__device__ __noinline__ double factor_slow(const double* zs_entry, double M) { return exp(__ldcg(zs_entry) - M); }
 
-template <int GG>
-__device__ __forceinline__ double group_prob(const double* zv, const double* sM, const double* rZ) {
-  double s = 0.0;
-#pragma unroll
-  for (int g = 0; g < GG; ++g) s += exp_once(zv[g] - sM[g]) * rZ[g];
-  return s;
+// L2 loads the compiler may not sink towards their first use: the selection jobs issue all loads of a phase
+// together and only then wait (a plain load is free to drift past the block barriers in between)
+__device__ __forceinline__ double2 ld_early2(const double* ptr) {
+  double2 v;
+  asm volatile("ld.global.cg.v2.f64 {%0, %1}, [%2];" : "=d"(v.x), "=d"(v.y) : "l"(ptr));
+  return v;
 }
+
 // max or sum over the block of one value per thread, separately for each of `ncols` interleaved columns
 // (thread t belongs to column t % ncols); fixed shuffle tree, so the sum does not depend on timing
 template <bool IS_MAX>
-__device__ __forceinline__ void column_reduce(double v, int ncols, double* red, double* result) {
+__device__ __noinline__ void column_reduce(double v, int ncols, double* red, double* result) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int off = ncols; off < 32; off <<= 1) {
     const double o = __shfl_xor_sync(0xffffffffu, v, off);
@@ -515,80 +604,132 @@ __device__ __forceinline__ void column_reduce(double v, int ncols, double* red, 
 }
 
 // Per-head softmax over C and the group mean (Sec. 3.2), then a^S, a^L or s = max(a^S, a^L) (Eq. 9) of every
-// candidate into a[].  The attention kernel left, per 16-token page and column, the page's (max, sum of
-// exponentials); they merge into the normalisers of the whole candidate set without another pass over the
-// logits.  All loads of the prologue (page partials and the first batch of logits) are issued together.
+// candidate into a[].  The attention kernel left, per 16-token page t and column c, the page's maximum logit
+// m_tc and s_tc = sum of exp(z - m_tc), and per token x = exp(z - m_tc).  With M_c the maximum over pages and
+// f_tc = exp(m_tc - M_c):  softmax = x f_tc / Z_c,  Z_c = sum_t s_tc f_tc.  So this pass takes one exponential
+// per page and column instead of one per token and column; the factors f_tc sit in shared memory (F, f_cap
+// entries; when the candidate set has more page-columns than that, they are recomputed per token).
+// All loads of the prologue (page partials and the first batch of x) are issued together.
 template <int GG>
-__device__ __noinline__ bool job_softmax(const double* __restrict__ z, const double* __restrict__ zs,
-                                         double* __restrict__ a, int nC, int task, double* red, double* sM,
-                                         double* sZ) {
+__device__ __noinline__ bool job_softmax(const GpDev& p, const double* __restrict__ x, size_t view_stride,
+                                         const double* __restrict__ zs, double* __restrict__ a, int nC, int task,
+                                         double* red, double* sM, double* sZ, double* F, int f_cap) {
   constexpr int G2 = 2 * GG;
-  constexpr int U = GG == 8 ? 1 : GG == 4 ? 2 : 4;       // tokens per thread in flight
+  constexpr int U = 4;                                   // 16-byte loads per thread and view in flight
   constexpr int KEEP = 2;                                // page partials per thread held in registers
+  constexpr int LPT = GG >= 2 ? GG / 2 : 1;              // lanes that share a token (two columns each)
   const int tid = threadIdx.x;
-  const int ncols = task == 2 ? G2 : GG;
+  const int nview = task == 2 ? 2 : 1;
+  const int ncols = nview * GG;
   const int col0 = task == 1 ? GG : 0;
-  const int mycol = col0 + tid % ncols;                  // SEL_T is a multiple of ncols
+  const int myc = tid % ncols;                           // SEL_T is a multiple of ncols
+  const int mycol = col0 + myc;
   const int ntile = nC / GP_PAGE;
   const int t0 = tid / ncols, tstep = SEL_T / ncols;
+  const bool table = ntile * ncols <= f_cap;
+  const int nv = nC * GG / 2;                            // 16-byte pieces of one view: consecutive lanes, consecutive pieces
+  const double* xb = x + (task == 1 ? view_stride : 0);
   double2 keep[KEEP];
 #pragma unroll
   for (int k = 0; k < KEEP; ++k) {
     const int t = t0 + k * tstep;
-    keep[k] = t < ntile ? __ldcg(reinterpret_cast<const double2*>(zs + ((size_t)t * G2 + mycol) * 2))
-                        : make_double2(-INFINITY, 0.0);
+    keep[k] = make_double2(-INFINITY, 0.0);
+    if (t < ntile) keep[k] = ld_early2(zs + ((size_t)t * G2 + mycol) * 2);
   }
-  double zv[U][G2];
+  double2 xv[2][U];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
-    const int i = tid + u * SEL_T;
-    if (i < nC) {
-      const double* zr = z + (size_t)i * G2 + col0;
-#pragma unroll
-      for (int g = 0; g < G2; ++g)
-        if (g < GG || task == 2) zv[u][g] = __ldcg(zr + g);
+    const int k = tid + u * SEL_T;
+    xv[0][u] = xv[1][u] = make_double2(0.0, 0.0);
+    if (k < nv) {
+      xv[0][u] = ld_early2(xb + 2 * (size_t)k);
+      if (task == 2) xv[1][u] = ld_early2(xb + view_stride + 2 * (size_t)k);
     }
   }
+  const long long j0 = GP_T_NOW(); (void)j0;
   double m = fmax(keep[0].x, keep[1].x);
   for (int t = t0 + KEEP * tstep; t < ntile; t += tstep) m = fmax(m, __ldcg(zs + ((size_t)t * G2 + mycol) * 2));
   column_reduce<true>(m, ncols, red, sM);
-  const double mc = sM[tid % ncols];
+  const long long j1 = GP_T_NOW(); (void)j1;
+  const double mc = sM[myc];
   double acc = 0.0;
 #pragma unroll
-  for (int k = 0; k < KEEP; ++k)
-    if (t0 + k * tstep < ntile) acc += keep[k].y * exp_once(keep[k].x - mc);
+  for (int k = 0; k < KEEP; ++k) {
+    const int t = t0 + k * tstep;
+    if (t < ntile) {
+      const double f = exp_once(keep[k].x - mc);
+      acc += keep[k].y * f;
+      if (table) F[t * ncols + myc] = f;
+    }
+  }
   for (int t = t0 + KEEP * tstep; t < ntile; t += tstep) {
     const double2 ms = __ldcg(reinterpret_cast<const double2*>(zs + ((size_t)t * G2 + mycol) * 2));
-    acc += ms.y * exp_once(ms.x - mc);
+    const double f = exp_once(ms.x - mc);
+    acc += ms.y * f;
+    if (table) F[t * ncols + myc] = f;
   }
   column_reduce<false>(acc, ncols, red, sZ);
   if (tid < ncols) sZ[tid] = 1.0 / ((double)GG * sZ[tid]);     // group mean and normaliser in one factor
   __syncthreads();
+  const long long j2 = GP_T_NOW(); (void)j2;
   unsigned top_bits = 0;
-  for (int i0 = tid; i0 < nC; i0 += U * SEL_T) {
-    if (i0 != tid) {
+  for (int k0 = tid; k0 - tid < nv; k0 += U * SEL_T) {   // uniform trip count: the shuffles below need whole warps
+    if (k0 != tid) {
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        const int i = i0 + u * SEL_T;
-        if (i < nC) {
-          const double* zr = z + (size_t)i * G2 + col0;
-#pragma unroll
-          for (int g = 0; g < G2; ++g)
-            if (g < GG || task == 2) zv[u][g] = __ldcg(zr + g);
+        const int k = k0 + u * SEL_T;
+        xv[0][u] = xv[1][u] = make_double2(0.0, 0.0);
+        if (k < nv) {
+          xv[0][u] = __ldcg(reinterpret_cast<const double2*>(xb + 2 * (size_t)k));
+          if (task == 2) xv[1][u] = __ldcg(reinterpret_cast<const double2*>(xb + view_stride + 2 * (size_t)k));
         }
       }
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * SEL_T;
-      if (i < nC) {
-        double s0 = group_prob<GG>(zv[u], sM, sZ);                // column c of this job sits at index c - col0
-        if (task == 2) s0 = fmax(s0, group_prob<GG>(zv[u] + GG, sM + GG, sZ + GG));       // Eq. 9
-        a[i] = s0;
-        top_bits |= 1u << (unsigned)(((unsigned long long)__double_as_longlong(s0) >> 58) & 31ull);
+      const int k = k0 + u * SEL_T;
+      const bool on = k < nv;
+      const int flat = 2 * (on ? k : 0);
+      const int tok = flat / GG, g = flat % GG;           // GG = 1: tokens tok and tok + 1 (same page), column 0
+      const int t = tok / GP_PAGE;
+      double part[2][2];                                  // [view][element of the piece]
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        part[q][0] = part[q][1] = 0.0;
+        if (q < nview && on) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int c = q * GG + (GG == 1 ? 0 : g + e); // column of this job: index into F, sM, sZ
+            const double f = table ? F[t * ncols + c] : factor_slow(zs + ((size_t)t * G2 + col0 + c) * 2, sM[c]);
+            part[q][e] = (e == 0 ? xv[q][u].x : xv[q][u].y) * f * sZ[c];
+          }
+        }
+      }
+      if (GG == 1) {
+        if (on) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const double s0 = task == 2 ? fmax(part[0][e], part[1][e]) : part[0][e];       // Eq. 9
+            a[tok + e] = s0;
+            top_bits |= 1u << (unsigned)(((unsigned long long)__double_as_longlong(s0) >> 58) & 31ull);
+          }
+        }
+      } else {
+        double sv0 = part[0][0] + part[0][1], sv1 = part[1][0] + part[1][1];
+#pragma unroll
+        for (int o = 1; o < LPT; o <<= 1) {
+          sv0 += __shfl_xor_sync(0xffffffffu, sv0, o);
+          sv1 += __shfl_xor_sync(0xffffffffu, sv1, o);
+        }
+        if (on && g == 0) {
+          const double s0 = task == 2 ? fmax(sv0, sv1) : sv0;                              // Eq. 9
+          a[tok] = s0;
+          top_bits |= 1u << (unsigned)(((unsigned long long)__double_as_longlong(s0) >> 58) & 31ull);
+        }
       }
     }
   }
+  if (tid == 0) { GP_T_ADD(12, j1 - j0); GP_T_ADD(13, j2 - j1); GP_T_ADD(14, GP_T_NOW() - j2); GP_T_ADD(30, 1); }
   // bits 62..58 of every score, as a set: the fast selection path needs them all equal
   return __popc(__syncthreads_or((int)top_bits)) == 1;
 }
@@ -642,10 +783,10 @@ __device__ __noinline__ void merge_partials(const GpDev& p, int n_req, float* __
 struct SelGeom {
   static constexpr size_t BUF_BYTES = SEL_CAP * sizeof(double);
   static constexpr size_t H_BYTES = (size_t)FB_PAD * 12;
-  static constexpr size_t MISC_BYTES = 8 * 8 + 8 * 4 + 8 * 8 + 16 * 4 + 16 * 4 + (8 * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
+  static constexpr size_t MISC_BYTES = SEL_NW * 8 + SEL_NW * 4 + 8 * 8 + 16 * 4 + 16 * 4 + (SEL_NW * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
 };
 
-__global__ void __launch_bounds__(SEL_T, 2)
+__global__ void __launch_bounds__(SEL_T, 1)
 gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
                float* __restrict__ out) {
   extern __shared__ uint8_t smem_raw[];
@@ -653,18 +794,20 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   double* sbuf = reinterpret_cast<double*>(smem);                              // [SEL_CAP] a^S, a^L or s
   unsigned* hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::BUF_BYTES);
   unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + FB_PAD);   // two u32 planes (low, high)
-  unsigned long long* wsum = hsum + FB_PAD;                                    // [8]
-  unsigned* wc = reinterpret_cast<unsigned*>(wsum + 8);                        // [8]
-  long long* s_res = reinterpret_cast<long long*>(wc + 8);                     // [8]
+  unsigned long long* wsum = hsum + FB_PAD;                                    // [SEL_NW]
+  unsigned* wc = reinterpret_cast<unsigned*>(wsum + SEL_NW);                   // [SEL_NW]
+  long long* s_res = reinterpret_cast<long long*>(wc + SEL_NW);                // [8]
   int* ev = reinterpret_cast<int*>(s_res + 8);                                 // [16]
   int* s_i = ev + 16;                                                          // [16]
-  double* red = reinterpret_cast<double*>(s_i + 16);                           // [8][16]
-  double* sM = red + 8 * 16;                                                   // [16]
+  double* red = reinterpret_cast<double*>(s_i + 16);                           // [SEL_NW][16]
+  double* sM = red + SEL_NW * 16;                                                   // [16]
   double* sZ = sM + 16;                                                        // [16]
   double* flist = sZ + 16;                                                     // [32] members of the crossing bin
   int* flist_slot = reinterpret_cast<int*>(flist + 32);                        // [32]
   unsigned* coarse = reinterpret_cast<unsigned*>(flist_slot + 32);             // [3][CBINS] summary bins
   unsigned* loc = coarse + 3 * CBINS;                                          // [cap*b/32 + 1]
+  double* F = reinterpret_cast<double*>(hcnt);                                 // softmax factors, before the bins are used
+  constexpr int F_CAP = (int)(SelGeom::H_BYTES / sizeof(double));
   FastHist H;
   H.cnt = hcnt; H.lo = reinterpret_cast<unsigned*>(hsum); H.hi = H.lo + FB_PAD;
   H.ccnt = coarse; H.clo = coarse + CBINS; H.chi = coarse + 2 * CBINS;
@@ -673,6 +816,8 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const int tid = threadIdx.x;
   const int LH = p.L * p.Hkv;
   const int G = p.G, G2 = 2 * p.G;
+  gp_pdl_wait();
+  gp_pdl_launch_dependents();
   // the first item's descriptor is fetched before the number of items is known (same round trip); slots of
   // bnd_info past the count hold stale but readable data that is then not used
   int4 inf_first = make_int4(0, 0, 0, 0), inf2_first = inf_first;
@@ -728,25 +873,26 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     }
     const long long t_s0 = GP_T_NOW();
     (void)t_s0;
-    const double* z = p.zbuf + ((size_t)lh * p.max_batch_tokens + off) * G2;      // [nC][2][G]
+    const size_t view_stride = (size_t)p.z_stride * G;
+    const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;   // [2 views][nC][G] exp(logit - page max)
     double* a = nC <= SEL_CAP ? sbuf : p.scores + ((size_t)task * LH + lh) * p.max_batch_tokens + off;
-    // the fast path's bins are cleared while the first loads of the softmax pass are in flight
-    fast_hist_zero(H, task < 2);
     if (task == 2) for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
     if (tid == 0) { s_res[0] = -1; s_i[0] = 0; s_i[5] = 0; s_i[6] = 0; s_i[7] = 0; }
     bool uniform;
     {
       const double* zs = p.zstat + ((size_t)lh * (p.max_batch_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
       switch (G) {
-        case 1: uniform = job_softmax<1>(z, zs, a, nC, task, red, sM, sZ); break;
-        case 2: uniform = job_softmax<2>(z, zs, a, nC, task, red, sM, sZ); break;
-        case 4: uniform = job_softmax<4>(z, zs, a, nC, task, red, sM, sZ); break;
-        default: uniform = job_softmax<8>(z, zs, a, nC, task, red, sM, sZ); break;
+        case 1: uniform = job_softmax<1>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
+        case 2: uniform = job_softmax<2>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
+        case 4: uniform = job_softmax<4>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
+        default: uniform = job_softmax<8>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
       }
     }
+    fast_hist_zero(H, task < 2);                   // the factors' table shared this memory
     const long long t_s1 = GP_T_NOW();
     (void)t_s1;
     if (task < 2) {
+      __syncthreads();
       // ---- Eq. 7 -------------------------------------------------------------------------------------------
       int K = uniform ? top_p_fast(p, a, nC, p.p_fix, H, wc, wsum, s_res, flist, &s_i[5]) : -1;
       if (K < 0) { __syncthreads(); K = top_p_count<SEL_T>(p, a, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res); }
@@ -778,86 +924,8 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     const long long t_s3 = GP_T_NOW();
     (void)t_s3;
     // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
-    if (!uniform || !evict_fast(a, nC, loc, H, wc, s_res, flist, flist_slot, &s_i[6], ev)) {
-      __syncthreads();
-        unsigned long long prefix = 0;
-      unsigned cnt_below = 0;
-      unsigned long long thr = 0;        // evict keys strictly below thr ...
-      unsigned long long tie_key = 0;    // ... and need_eq of the highest slots whose key equals tie_key
-      int need_eq = 0;
-      {
-        int shift = 63;
-        bool done = false;
-        for (int lvl = 0; lvl < 6 && !done; ++lvl) {
-          const int w = kWidths[lvl];
-          shift -= w;
-          const int nb = 1 << w;
-          for (int i = tid; i < nb + (nb >> 3); i += SEL_T) hcnt[i] = 0;
-          if (tid == 0) s_res[0] = -1;
-          __syncthreads();
-          for (int i = tid; i < nC; i += SEL_T) {
-            if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-              const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-              if (lvl == 0 || (key >> (shift + w)) == prefix)
-                atomicAdd(&hcnt[HIDX((int)((key >> shift) & (unsigned long long)(nb - 1)))], 1u);
-            }
-          }
-          __syncthreads();
-          const int per = nb / SEL_T > 0 ? nb / SEL_T : 1;
-          const int lo = tid * per, hi = lo + per;
-          unsigned c = 0;
-          if (lo < nb) for (int b = lo; b < hi; ++b) c += hcnt[HIDX(b)];
-          const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
-          if (lo < nb) {
-            unsigned run = cnt_below + ex;
-            for (int b = lo; b < hi; ++b) {
-              const unsigned before = run;
-              run += hcnt[HIDX(b)];
-              if (before < (unsigned)GP_PAGE && run >= (unsigned)GP_PAGE) { s_res[0] = b; s_res[1] = before; }
-            }
-          }
-          __syncthreads();
-          if (s_res[0] < 0) {                                  // fewer than b candidates: cannot happen
-            if (tid == 0) atomicOr(p.err, GP_E_BOUNDS);
-            break;
-          }
-          const int bin_star = (int)s_res[0];
-          cnt_below = (unsigned)s_res[1];
-          const unsigned cstar = hcnt[HIDX(bin_star)];
-          __syncthreads();
-          prefix = (prefix << w) | (unsigned long long)bin_star;
-          if (cnt_below + cstar == (unsigned)GP_PAGE) {        // the bin fits exactly: no tie to break
-            thr = (prefix + 1ull) << shift;
-            done = true;
-          }
-        }
-        if (!done) {                                           // equal scores straddle the cut
-          thr = prefix;
-          tie_key = prefix;
-          need_eq = GP_PAGE - (int)cnt_below;
-        }
-      }
-      const long long t_s4 = GP_T_NOW();
-      (void)t_s4;
-      for (int i = tid; i < nC; i += SEL_T) {
-        if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-          const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-          if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < GP_PAGE) ev[at] = i; }
-        }
-      }
-      __syncthreads();
-      if (tid == 0) {
-        int cntv = s_i[0];
-        for (int i = nC - 1; i >= 0 && need_eq > 0; --i) {     // rare: older (lower) slots win ties
-          if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
-            const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-            if (key == tie_key) { if (cntv < GP_PAGE) ev[cntv] = i; ++cntv; --need_eq; }
-          }
-        }
-        if (cntv != GP_PAGE) atomicOr(p.err, GP_E_BOUNDS);
-        GP_T_ADD(21, GP_T_NOW() - t_s4);
-      }
-    }
+    if (!uniform || !evict_fast(a, nC, loc, H, wc, s_res, flist, flist_slot, &s_i[6], ev))
+      evict_general(p, a, nC, loc, hcnt, wc, s_res, s_i, ev);
     __syncthreads();
     if (tid < GP_PAGE) {                                     // the 16 slots in ascending order, by rank
       const int mine = ev[tid];
@@ -907,6 +975,8 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int LH = p.L * p.Hkv;
+  gp_pdl_wait();
+  gp_pdl_launch_dependents();
   // the first round trip fetches everything at once: the header, the list of compressing requests (its first
   // CT entries before their count is known; entries past the count are never looked at) and the first ticket
   if (tid == 0) { GP_T_STAMP(36); s_i[0] = atomicAdd(&p.hdr[HDR_WORK_CMP], 1); s_i[3] = 0; }
@@ -1095,10 +1165,10 @@ void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_com
 }
 
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
-                        int grid_compact, cudaStream_t s, cudaEvent_t ev) {
+                        int grid_compact, cudaStream_t s, cudaEvent_t ev, bool pdl) {
   const size_t sel_sm = gp_bsel_smem(p);
-  gp_bsel_kernel<<<grid_sel, SEL_T, sel_sm, s>>>(p, req_ids, n_req, actions, out);
+  gp_launch(gp_bsel_kernel, grid_sel, SEL_T, sel_sm, s, pdl, p, req_ids, n_req, actions, out);
   if (ev) cudaEventRecord(ev, s);
-  if (p.d == 128) gp_compact_kernel<128><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);
-  else gp_compact_kernel<64><<<grid_compact, CT, 0, s>>>(p, req_ids, n_req);
+  if (p.d == 128) gp_launch(gp_compact_kernel<128>, grid_compact, CT, 0, s, pdl, p, req_ids, n_req);
+  else gp_launch(gp_compact_kernel<64>, grid_compact, CT, 0, s, pdl, p, req_ids, n_req);
 }

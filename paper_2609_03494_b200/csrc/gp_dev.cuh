@@ -88,7 +88,8 @@ struct GpDev {
   int* bnd_acc;                          // [M][4] per boundary request: sum of K^S, sum of K^L, shared pages of C, 0
   int* free_peek;                        // [M+1] free_top at plan time, then the top entries of the free list, top first
   int4* cmp_info;                        // [M+1] compressing requests: {request, P, index in bnd_info, first compaction chunk}
-  double* zbuf;                          // [L*H_kv][max_batch_tokens][2][G] summary logits of boundary units
+  double* zbuf;                          // [L*H_kv][2][z_stride][G] boundary units, per view (short, long): exp(summary logit - its page's max)
+  long long z_stride;                    // max_batch_tokens rounded up to a multiple of the page size
   double* zstat;                         // [L*H_kv][max_batch_tokens / b][2][G][2] per-page softmax partials (max, sum)
   int* sum_par;                          // [M] which of the two summary buffers is current
   int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
@@ -194,12 +195,36 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 
 // ---- host-visible launchers (one per translation unit) -------------------------------------------
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s);
+                         float* out, int grid, cudaStream_t s, bool pdl);
 size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
-// boundary chain: probabilities + working sets + selection + decision, then compaction.
-// `ev`, when not null, is recorded between the two kernels.
+// ---- programmatic dependent launch -------------------------------------------------------------------
+// Every kernel of the decode step waits at its top for the kernel before it in the stream (completion and
+// memory flush), then lets the kernel after it be scheduled: the next grid's CTAs become resident while this
+// one drains, which hides the launch latency between the step's kernels.  All of the step's grids are a
+// single resident wave, so early-scheduled dependents only ever take resources nobody else is waiting for.
+// Without the launch attribute both instructions do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void gp_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void gp_pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t gp_launch(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, bool pdl,
+                             Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)block);
+  cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 void gp_attention_setup(const GpDev& p);
 void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact);
+// boundary chain: probabilities + working sets + selection + decision, then compaction.
+// `ev`, when not null, is recorded between the two kernels.  `pdl`: launch with programmatic stream serialization.
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
-                        int grid_compact, cudaStream_t s, cudaEvent_t ev);
+                        int grid_compact, cudaStream_t s, cudaEvent_t ev, bool pdl);

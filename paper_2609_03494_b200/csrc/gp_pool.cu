@@ -116,7 +116,7 @@ Layout make_layout(const gp_config& c) {
   L.bnd_acc = take(M * 16);
   L.free_peek = take((M + 1) * 4);
   L.cmp_info = take((M + 1) * 16);
-  L.zbuf = take(LH * (size_t)L.max_batch_tokens * 2 * G * 8);
+  L.zbuf = take(LH * (size_t)(L.max_batch_tokens + b) * 2 * G * 8);
   L.zstat = take(LH * ((size_t)L.max_batch_tokens / b + 1) * 2 * G * 2 * 8);
   L.evict = take(M * LH * b * 4);
   L.cflags = take(LH * ((size_t)L.max_batch_tokens / GP_MOVE_TOK + 2 * M + 1) * 4);
@@ -197,6 +197,8 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __shared__ int s_peek[GP_MAX_REQ];       // the free list from its top down, for the decisions of this step
   const int i = threadIdx.x;
   const bool in = i < n_req;
+  gp_pdl_wait();
+  gp_pdl_launch_dependents();
   const int free_top0 = *p.free_top;
   const long long t_plan0 = GP_T_NOW();
   (void)t_plan0;
@@ -492,6 +494,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.d = cfg->head_dim; d.M = cfg->max_requests; d.cap = cfg->max_pages_per_req; d.k_loc = cfg->k_loc;
   d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc;
   d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
+  d.z_stride = (L.max_batch_tokens + GP_PAGE - 1) / GP_PAGE * GP_PAGE;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
   d.p_fix = (unsigned long long)llrint(cfg->top_p * 4611686018427387904.0);
   d.kv = reinterpret_cast<__nv_bfloat16*>(base + L.kv);
@@ -617,12 +620,13 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   const GpDev& d = pool->dev;
   const bool prof = pool->profiling != 0;
   if (prof) cudaEventRecord(pool->ev[0], s);
-  gp_plan_kernel<<<1, GP_PLAN_THREADS, 0, s>>>(d, dev_req_ids, n_req, dev_actions);
+  const bool pdl = !prof;                      // events between the kernels need them serialised the plain way
+  gp_launch(gp_plan_kernel, 1, GP_PLAN_THREADS, 0, s, pdl, d, dev_req_ids, n_req, dev_actions);
   if (prof) cudaEventRecord(pool->ev[1], s);
-  gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s);
+  gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl);
   if (prof) cudaEventRecord(pool->ev[2], s);
   gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s,
-                     prof ? pool->ev[3] : nullptr);
+                     prof ? pool->ev[3] : nullptr, pdl);
   if (prof) cudaEventRecord(pool->ev[4], s);
   pool->launch_count += GP_N_KERNELS;
   GP_CUDA(cudaGetLastError());
