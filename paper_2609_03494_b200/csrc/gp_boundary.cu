@@ -41,7 +41,7 @@ struct PairCU { unsigned c; unsigned long long s; };
 
 // exclusive suffix sum over the block: sum of the values of threads with a higher id
 template <int BT>
-__device__ __noinline__ PairCU block_suffix_excl(unsigned c, unsigned long long s, unsigned* wc,
+__device__ __forceinline__ PairCU block_suffix_excl(unsigned c, unsigned long long s, unsigned* wc,
                                                     unsigned long long* wsum) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned ic = c; unsigned long long is = s;
@@ -60,7 +60,7 @@ __device__ __noinline__ PairCU block_suffix_excl(unsigned c, unsigned long long 
 }
 // exclusive prefix count over the block
 template <int BT>
-__device__ __noinline__ unsigned block_prefix_excl(unsigned c, unsigned* wc) {
+__device__ __forceinline__ unsigned block_prefix_excl(unsigned c, unsigned* wc) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned ic = c;
 #pragma unroll
@@ -424,7 +424,7 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
 // ------------------------------------------------------------------------------------------------------
 // decision + allocator, run by the last CTA of the selection kernel
 // ------------------------------------------------------------------------------------------------------
-__device__ __noinline__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr) {
+__device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr) {
   int* s_want = s_arr;
   int* s_ksh = s_arr + GP_MAX_REQ;
   int* s_P = s_arr + 2 * GP_MAX_REQ;
@@ -587,7 +587,7 @@ __device__ __forceinline__ double2 ld_early2(const double* ptr) {
 // max or sum over the block of one value per thread, separately for each of `ncols` interleaved columns
 // (thread t belongs to column t % ncols); fixed shuffle tree, so the sum does not depend on timing
 template <bool IS_MAX>
-__device__ __noinline__ void column_reduce(double v, int ncols, double* red, double* result) {
+__device__ __forceinline__ void column_reduce(double v, int ncols, double* red, double* result) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int off = ncols; off < 32; off <<= 1) {
     const double o = __shfl_xor_sync(0xffffffffu, v, off);
