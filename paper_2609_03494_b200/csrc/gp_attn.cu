@@ -1,38 +1,40 @@
-// Fused append + GQA paged decode attention + dual EMA summary update (Sec. 3.2 Eq. 6, Sec. 4.1), plus,
-// for requests that reach their capacity boundary with this step, the logits of the two calibrated
-// summaries against every candidate key (Eq. 12, App. D.1) while the key tile is in shared memory.
+// Fused append + GQA paged decode attention (Sec. 4.1), plus, for requests that reach their capacity boundary
+// with this step, the logits of the two calibrated summaries against every candidate key (Eq. 12, App. D.1)
+// while the key tile is in shared memory.  (The summaries themselves, Eq. 6, and the calibrated q~ are updated
+// by the plan kernel's summary CTAs before this kernel starts.)
 //
 // Work decomposition.  The plan kernel cuts every stepped request into chunks of `chunk_pages` pages and
 // writes one descriptor per chunk, sorted by descending cost; a work item is (chunk, layer, KV head).  A
 // persistent grid (two CTAs per SM) deals the items out round by round, alternating the CTA order so that
 // every CTA gets about the same total.  Each CTA is warp-specialised:
 //
-//   warp 0      producer: takes its items (a static deal of the cost-sorted list), publishes their descriptor in a ring of item slots, and streams
-//               the K|V tiles of their pages (one contiguous `cp.async.bulk` per (layer, page, head))
-//               into a ring of stages shared by the CTA.  It runs ahead across item boundaries, so the
-//               ring never drains between items.
-//   warps 4..7  consumers: take the tiles of an item round-robin.  The G query heads of the group are
-//               rows 0..G-1 of an m16n8k16 bf16 MMA; S = Q K^T and O += P V run on the tensor cores with
-//               fp32 accumulation.  Rows 8..15 of the A operand carry the bf16 rounding residual of
-//               rows 0..7 (of the rotated query when RoPE is on, of P always), which costs nothing and
-//               gives ~16 mantissa bits.  For boundary units the summary logits of a candidate page are
-//               an fp64 tensor-core contraction (m8n8k4 DMMA: 8 tokens x (2 views x G heads) x d).
-//   warp 1      summaries: Eq. 6 on the un-rotated query (read from one of two buffers, written to the
-//               other, so that every item of a unit sees the old state), and for boundary units the
-//               calibrated, rotated summaries q~ in fp64 for the consumers.
+//   warp 0      producer: takes its items (a static deal of the cost-sorted list) and publishes each in a ring
+//               of item slots: descriptor, query rows (and the new key/value row) by bulk copy, page ids.  For
+//               boundary items it also brings q~ into the CTA's single q~ buffer.
+//   warps 4..7  consumers: take the tiles of an item round-robin (tile j belongs to warp j mod 4).  Each warp
+//               fetches its own K|V tiles (one contiguous 8 KB per (layer, page, head)) with 16-byte
+//               asynchronous copies into a private ring of stages, running ahead across item boundaries, so
+//               the ring never drains between items.  The G query heads of the group are rows 0..G-1 of an
+//               m16n8k16 bf16 MMA; S = Q K^T and O += P V run on the tensor cores with fp32 accumulation.
+//               Rows 8..15 of the A operand carry the bf16 rounding residual of rows 0..7 (of the rotated
+//               query when RoPE is on, of P always), which costs nothing and gives ~16 mantissa bits.  For
+//               boundary units the summary logits of a candidate page are an fp64 tensor-core contraction
+//               (m8n8k4 DMMA: 8 tokens x (2 views x G heads) x d).
 //   warp 2      merger: combines the four consumers' partial (max, sum, O) of an item and writes the output
 //               or, for requests split over several items, the partial (the next kernel merges those).
 //               Consumers hand over through a double buffer and go straight on to the next item.
+//   warps 1, 3  idle.
 //
 // The two warp groups re-split the register file (setmaxnreg): the service warps keep 56 registers per
 // thread, the consumers, which hold the output accumulators, get 200.
-// All waits are bounded; a wait that gives up sets an error bit and an abort flag that drains the CTA.
+// All waits are bounded; a wait that gives up sets an error bit (with a code for which wait it was) and an
+// abort flag that drains the CTA.  No wait of an item depends on a later item being published.
 #include "gp_dev.cuh"
 
 namespace {
 
 constexpr int NI_MAX = 8;                  // item slots per CTA (4 when the group is 8 heads wide)
-constexpr int NSW = 2;                     // tile stages per consumer warp
+constexpr int NSW = 2;                     // tile stages per consumer warp (at most 3: see the wait in the tile loop)
 constexpr int NCW = 4;                     // consumer warps
 constexpr int NTHREADS = 256;              // warp group 0: producer, summaries, merger, spare; warp group 1: consumers
 constexpr int REGS_SERVICE = 56;           // registers per thread after the split (setmaxnreg)
@@ -45,7 +47,8 @@ struct Geo {
   static constexpr int TILE_BYTES = 2 * GP_PAGE * ROW_BYTES;
   static constexpr int KSTEPS = D / 16;
   static constexpr int DTILES = D / 8;
-  static constexpr int SLOT_DESC = 128;                                // 32 ints
+  static constexpr int SLOT_DESC = 256;                                // 64 ints: descriptor, then the page ids
+  static constexpr int SLOT_PAGES = 32;                                // first page id (int index)
   static constexpr int SLOT_BYTES = (SLOT_DESC + 8 * ROW_BYTES + 2 * ROW_BYTES + 127) / 128 * 128;
 };
 
@@ -66,7 +69,7 @@ __host__ __device__ inline Lay make_lay(int G) {
   L.comb_warp = (16 + G * D) * 4;
   L.off_bars = L.off_comb + L.ncomb * NCW * L.comb_warp;
   L.off_misc = L.off_bars + (2 * NCW * NSW + 2 * NI_MAX + 2 + 4) * 8;
-  L.total = L.off_misc + 64 + 256;
+  L.total = L.off_misc + 128 + 256;          // abort flag and code, then the queue of q~ copies
   return L;
 }
 
@@ -74,11 +77,12 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // bounded, abort-aware wait
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int where = 0) {
   for (uint32_t it = 0; it < GP_SPIN_LIMIT; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 63u && *abort_flag) return false;
   }
+  if (*abort_flag == 0) abort_flag[1] = where;      // which wait gave up first (reported with the error bit)
   *abort_flag = 1;
   return false;
 }
@@ -99,8 +103,6 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   const Lay L = make_lay<D>(G);
   const uint32_t NI = (uint32_t)L.ni, NCOMB = (uint32_t)L.ncomb;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.off_bars);
-  uint64_t* full = bars;                       // [NCW][NSW]: each consumer warp owns a private ring, so a warp
-  uint64_t* empty = bars + NCW * NSW;          //   never waits more than one phase ahead of its barrier
   uint64_t* slot_full = bars + 2 * NCW * NSW;  // [NI]
   uint64_t* slot_empty = slot_full + NI_MAX;   // [NI]
   uint64_t* qt_full = slot_empty + NI_MAX;
@@ -117,12 +119,12 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 32] = (long long)gt; }
 #endif
   if (tid == 0) {
-    for (int i = 0; i < NCW * NSW; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < NI_MAX; ++i) { mbar_init(&slot_full[i], 1); mbar_init(&slot_empty[i], NCW + 2); }
+    for (int i = 0; i < NI_MAX; ++i) { mbar_init(&slot_full[i], 2); mbar_init(&slot_empty[i], NCW + 1); }
     mbar_init(qt_full, 1);
     mbar_init(qt_empty, NCW);
     for (int i = 0; i < 2; ++i) { mbar_init(&comb_full[i], NCW); mbar_init(&comb_empty[i], 1); }
     s_misc[0] = 0;
+    s_misc[1] = 0;
     fence_mbar_init();
   }
   gp_pdl_wait();                  // everything above touched only this CTA's shared memory
@@ -141,40 +143,84 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   }
   if (warp == 0) {
     // ================================= producer ===========================================
-    // Software pipeline over items, one stage per tick, so that no global round trip sits between two
-    // tiles: claim (t), descriptor header (t-1), page ids (t-2), publish the item slot (t-3), stream its
-    // tiles (t-4).  The loads of the young stages are in flight while the oldest item streams.
-    // Stages: A = item known, header load issued; B = header here: slot published, page ids requested;
-    // C = page ids here: last page id written to the slot; D = tiles streamed.  The first item of a CTA
-    // is its block index, later ones come from the global counter.
+    // Software pipeline over items, one stage per tick, so that no global round trip of one item delays
+    // another: A = item known, descriptor header load issued; B = header here: the slot is claimed, the
+    // descriptor written, the query rows (and the new key/value row) copied in, the page ids requested;
+    // C = page ids here: written to the slot, which completes its `full` barrier (two arrivals: B and C, plus
+    // the bytes of B's copies).  The ring of slots paces the producer: it runs NI items ahead at most.
     const long long grid = gridDim.x;
-    long long itA = blockIdx.x, itB = total, itC = total, itD = total;
-    int hB = 0, hC = 0, hD = 0;                // descriptor header, word `lane` (lanes 0..15)
-    int pC = -1, pD = -1;                      // page id of tile `lane` of the item
+    // static schedule: items are sorted by descending cost; round k goes to the CTAs in alternating order.
+    // A CTA takes its second item first: the costliest items are those of boundary requests, whose
+    // calibrated summaries the summary warps then prepare while the consumers are busy with another item.
+    auto item_of_round = [&](long long kk) -> long long {
+      const long long item = kk * grid + ((kk & 1) ? grid - 1 - (long long)blockIdx.x : (long long)blockIdx.x);
+      return item < total ? item : total;
+    };
+    const bool swap01 = item_of_round(1) < total;
+    auto item_of_tick = [&](long long t) -> long long { return item_of_round(swap01 && t < 2 ? 1 - t : t); };
+    long long itA = item_of_tick(0), itB = total, itC = total;
+    int hB = 0, hC = 0;                        // descriptor header, word `lane` (lanes 0..15)
+    int pC = -1;                               // page id of tile `lane` of the item
     int slC = 0;                               // slot of the item in stage C
-    uint32_t wf0 = 0, wf1 = 0, wf2 = 0, wf3 = 0;   // tiles issued so far to each consumer warp
     uint32_t n_pub = 0;
     bool sentinel_out = false;
+    // The q~ buffer is single: the copy for a boundary item is issued once the consumers are done with the
+    // previous boundary item.  The producer never blocks on that (it would hold back the slots of other
+    // items, possibly of the very item the consumers have to finish first): copies wait in a queue (never
+    // more entries than item slots) and are issued from the polls below, oldest first.
+    volatile int* qt_queue = s_misc + 16;          // [NI_MAX][2]: batch slot, layer/head
+    uint32_t qt_head = 0, qt_tail = 0;              // qt_head = copies issued so far
+    auto poll_qt = [&]() {
+      if (qt_head != qt_tail && mbar_test_wait(qt_empty, (qt_head & 1u) ^ 1u)) {
+        if (lane == 0) {
+          const int qbi = qt_queue[(qt_head % NI_MAX) * 2], qlh = qt_queue[(qt_head % NI_MAX) * 2 + 1];
+          fence_proxy_async();
+          mbar_expect_tx(qt_full, 2 * G * D * 8);
+          const double* src = p.qtil + ((size_t)qbi * LH + qlh) * 2 * G * D;
+          for (int row2 = 0; row2 < 2 * G; ++row2)
+            bulk_g2s(qt + (size_t)row2 * (D + QT_PAD), src + (size_t)row2 * D, D * 8, qt_full);
+        }
+        ++qt_head;
+      }
+    };
+    auto wait_polling = [&](uint64_t* bar, uint32_t parity) -> bool {     // bounded, abort-aware, keeps q~ moving
+      for (uint32_t w = 0; w < GP_SPIN_LIMIT; ++w) {
+        if (mbar_try_wait(bar, parity)) return true;
+        poll_qt();
+        if ((w & 63u) == 63u && s_misc[0]) return false;
+      }
+      if (s_misc[0] == 0) s_misc[1] = 1;
+      s_misc[0] = 1;
+      return false;
+    };
     for (uint32_t tick = 0;; ++tick) {
       // ---- issue the loads of the young stages --------------------------------------------------
       int hNew = 0;
       if (itA < total && lane < GP_DESC_INTS) hNew = p.rcx[(size_t)(itA / LH) * GP_DESC_INTS + lane];
       int pNew = -1;
       int slNew = 0;
-      // ---- header of stage B has arrived: load its page ids and publish its slot --------------------
+      // ---- page ids of stage C have arrived: into the slot, which is then complete ----------------------
+      if (itC < total) {
+        int* sd = reinterpret_cast<int*>(smem + L.off_slots + slC * GEO::SLOT_BYTES);
+        sd[GEO::SLOT_PAGES + lane] = pC;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&slot_full[slC]);
+      }
+      poll_qt();
+      // ---- header of stage B has arrived: load its page ids and fill its slot -----------------------
       if (tick >= 1 && !sentinel_out) {
         const int sl = n_pub % NI;
         slNew = sl;
         const long long t_p0 = GP_T_NOW();
         (void)t_p0;
-        if (!wait_bar(&slot_empty[sl], ((n_pub / NI) & 1u) ^ 1u, s_misc)) break;
+        if (!wait_polling(&slot_empty[sl], ((n_pub / NI) & 1u) ^ 1u)) break;
         if (lane == 0) GP_T_ADD(11, GP_T_NOW() - t_p0);
         uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
         int* sd = reinterpret_cast<int*>(slot);
         if (itB >= total) {
           if (lane == 0) sd[3] = -1;
           __syncwarp();
-          if (lane == 0) mbar_arrive(&slot_full[sl]);
+          if (lane == 0) { mbar_arrive(&slot_full[sl]); mbar_arrive(&slot_full[sl]); }
           sentinel_out = true;
         } else {
           const int lh = (int)(itB % LH);
@@ -199,59 +245,30 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
               bulk_g2s(slot + GEO::SLOT_DESC + 9 * GEO::ROW_BYTES, v + kvo, GEO::ROW_BYTES, &slot_full[sl]);
             }
           }
+          // boundary unit with candidate pages in this chunk: its calibrated summaries q~ (written by the
+          // plan kernel's summary CTAs) go into the single q~ buffer once the previous such item is done
+          const int flags = __shfl_sync(0xffffffffu, hB, 8), Pr = __shfl_sync(0xffffffffu, hB, 9);
+          if ((flags & 1) && pg0 < Pr - 1) {
+            if (lane == 0) { qt_queue[(qt_tail % NI_MAX) * 2] = bi; qt_queue[(qt_tail % NI_MAX) * 2 + 1] = lh; }
+            __syncwarp();
+            ++qt_tail;
+            poll_qt();
+          }
         }
         ++n_pub;
       }
-      // ---- page ids of stage C have arrived: the consumer that appends needs the last one ------------
-      if (itC < total) {
-        const int npg = __shfl_sync(0xffffffffu, hC, 3);
-        const int last_pg = __shfl_sync(0xffffffffu, pC, (npg - 1) & 31);
-        if (lane == 0) reinterpret_cast<int*>(smem + L.off_slots + slC * GEO::SLOT_BYTES)[16] = last_pg;
-      }
-      // ---- stream the tiles of the oldest item ----------------------------------------------------------
-      if (tick >= 3) {
-        if (itD >= total) break;
-        const int lh = (int)(itD % LH);
-        const int l = lh / p.Hkv, h = lh % p.Hkv;
-        const int npg = __shfl_sync(0xffffffffu, hD, 3);
-        bool ok = true;
-        for (int j = 0; j < npg; ++j) {
-          const int page = __shfl_sync(0xffffffffu, pD, j);
-          const int cwj = j & (NCW - 1);                        // tile j of an item goes to consumer warp j mod 4
-          const uint32_t kf = cwj == 0 ? wf0 : cwj == 1 ? wf1 : cwj == 2 ? wf2 : wf3;
-          const uint32_t st = cwj * NSW + (kf % NSW);
-          const long long t_p1 = GP_T_NOW();
-          (void)t_p1;
-          if (!wait_bar(&empty[st], ((kf / NSW) & 1u) ^ 1u, s_misc)) { ok = false; break; }
-          if (lane == 0) GP_T_ADD(10, GP_T_NOW() - t_p1);
-          if (lane == 0) {
-            fence_proxy_async();
-            mbar_expect_tx(&full[st], GEO::TILE_BYTES);
-            bulk_g2s(smem + st * GEO::TILE_BYTES, p.kv + gp_tile_off(p, l, page, h), GEO::TILE_BYTES, &full[st]);
-          }
-          wf0 += (cwj == 0); wf1 += (cwj == 1); wf2 += (cwj == 2); wf3 += (cwj == 3);
-        }
-        if (!ok) break;
-      }
+      if (sentinel_out && itC >= total) break;
       // ---- rotate -----------------------------------------------------------------------------------------
-      itD = itC; hD = hC; pD = pC;
       itC = itB; hC = hB; pC = pNew; slC = slNew;
       itB = itA; hB = hNew;
-      {   // static schedule: items are sorted by descending cost; round k goes to the CTAs in alternating order
-        const long long kk = (long long)tick + 1;
-        itA = kk * grid + ((kk & 1) ? grid - 1 - (long long)blockIdx.x : (long long)blockIdx.x);
-        if (itA >= total) itA = total;
-      }
+      itA = item_of_tick((long long)tick + 1);
     }
-    if (s_misc[0]) {
-      // aborted: let the copies already issued land before the CTA goes away
-      if (lane == 0) atomicOr(p.err, GP_E_SPIN);
-      const uint32_t wf[NCW] = {wf0, wf1, wf2, wf3};
-      for (int c = 0; c < NCW; ++c)
-        for (uint32_t f = (wf[c] > NSW ? wf[c] - NSW : 0); f < wf[c]; ++f)
-          for (uint32_t it2 = 0; it2 < (1u << 16); ++it2)
-            if (mbar_try_wait(&full[c * NSW + (f % NSW)], (f / NSW) & 1u)) break;
+    (void)hC;
+    while (qt_head != qt_tail && !s_misc[0]) {           // copies still queued when the last slot is out
+      if (!wait_polling(qt_empty, (qt_head & 1u) ^ 1u)) break;
+      poll_qt();
     }
+    if (s_misc[0] && lane == 0) atomicOr(p.err, GP_E_SPIN | (1 << (7 + s_misc[1])));
   } else if (warp >= 4) {
     // ================================= consumers ==========================================
     const int cw = warp - 4;
@@ -262,16 +279,62 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     const bool tr = (cw == 0 && lane == 0);
     const long long t_loop0 = GP_T_NOW();
     (void)tr; (void)t_loop0;
+    if (tr) GP_T_STAMP(64);
+    // Each consumer warp fetches its own tiles (tile j of an item belongs to warp j mod 4) into its private
+    // ring of NSW stages: as soon as it is done with a stage it issues the copy of its next tile but NSW - 1,
+    // which may belong to a later item (the fetch position runs ahead of the compute position, across item
+    // boundaries, but never further than the ring of item slots allows).  No other warp touches the ring, so
+    // program order plus a proxy fence orders the reads of a stage before the copy that overwrites it.
+    uint32_t my_fetch = 0, f_it = 0;
+    int f_pgl = 0, f_npg = 0, f_lh = 0;
+    bool f_have = false, f_done = false;
+    auto top_up = [&](uint32_t it_now) -> bool {           // false: a wait gave up
+      while (!f_done && my_fetch - my_tiles < (uint32_t)NSW) {
+        const int* fsd = reinterpret_cast<const int*>(smem + L.off_slots + (f_it % NI) * GEO::SLOT_BYTES);
+        if (!f_have) {
+          if (f_it + 1 >= it_now + NI) break;              // that slot may still hold an item this warp has not finished
+          // an item ahead of the one being computed is fetched from only if its slot is already there:
+          // nothing the current item needs may wait for a later item to be published
+          if (f_it > it_now) {
+            if (!mbar_test_wait(&slot_full[f_it % NI], (f_it / NI) & 1u)) break;
+          } else if (!wait_bar(&slot_full[f_it % NI], (f_it / NI) & 1u, s_misc, 3)) {
+            return false;
+          }
+          f_npg = fsd[3];
+          if (f_npg < 0) { f_done = true; break; }
+          f_lh = fsd[14];
+          f_pgl = cw;
+          f_have = true;
+        }
+        if (f_pgl >= f_npg) { ++f_it; f_have = false; continue; }
+        const int page = fsd[GEO::SLOT_PAGES + f_pgl];
+        const uint32_t fst = cw * NSW + (my_fetch % NSW);
+        {
+          // 16-byte asynchronous copies through the load/store path, 512 contiguous bytes per warp instruction:
+          // the bulk-copy engine takes several hundred cycles to accept an 8 KB copy, which paced the kernel
+          const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, f_lh / p.Hkv, page, f_lh % p.Hkv)) + lane * 16;
+          const uint32_t dst = smem_u32(smem + fst * GEO::TILE_BYTES) + lane * 16;
+#pragma unroll
+          for (int c = 0; c < GEO::TILE_BYTES / 512; ++c) cp_async16(dst + c * 512, src + c * 512);
+          cp_async_commit();
+        }
+        ++my_fetch;
+        f_pgl += NCW;
+      }
+      return true;
+    };
     for (uint32_t it = 0;; ++it) {
       const int sl = it % NI;
       const long long t_a = GP_T_NOW();
       (void)t_a;
-      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc)) break;
+      if (!top_up(it)) break;
+      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc, 4)) break;
       const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
       if (npg < 0) break;
-      if (tr) { GP_T_ADD(0, 1); GP_T_ADD(2, GP_T_NOW() - t_a); }
+      if (tr) { GP_T_ADD(0, 1); GP_T_ADD(2, GP_T_NOW() - t_a); if (it == 0) GP_T_STAMP(65); if (it == 1) GP_T_STAMP(69); if (it == 2) GP_T_STAMP(70); }
+      const long long t_a2 = GP_T_NOW(); (void)t_a2;
       const int bi = sd[0], pg0 = sd[2], chunk = sd[4], nchunks = sd[5], n_old = sd[6];
       const int flags = sd[8], Pr = sd[9], lh = sd[14];
       const int l = lh / p.Hkv, h = lh % p.Hkv;
@@ -317,7 +380,10 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         }
       }
       if (need_qt) {
-        if (!wait_bar(qt_full, qt_uses & 1u, s_misc)) break;
+        const long long t_q = GP_T_NOW();
+        (void)t_q;
+        if (!wait_bar(qt_full, qt_uses & 1u, s_misc, 5)) break;
+        if (tr) { GP_T_ADD(15, GP_T_NOW() - t_q); GP_T_ADD(7, 1); }
       }
 
       const bool last_chunk = (chunk == nchunks - 1);
@@ -327,22 +393,29 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       float m_run = -INFINITY, l_run = 0.f;
       bool ok = true;
 
+      if (tr) GP_T_ADD(77, GP_T_NOW() - t_a2);
+      long long t_prev = GP_T_NOW(); (void)t_prev;
       for (int pgl = cw; pgl < npg; pgl += NCW) {
         const uint32_t st = cw * NSW + (my_tiles % NSW);
         const long long t_b = GP_T_NOW();
         (void)t_b;
-        if (!wait_bar(&full[st], (my_tiles / NSW) & 1u, s_misc)) { ok = false; break; }
+        {
+          // one copy group per tile, in fetch order: all but the groups younger than this tile's must be done
+          const uint32_t younger = my_fetch - my_tiles - 1;
+          if (younger == 0) cp_async_wait<0>(); else if (younger == 1) cp_async_wait<1>(); else cp_async_wait<2>();
+          __syncwarp();
+        }
         ++my_tiles;
         const long long t_c = GP_T_NOW();
         (void)t_c;
-        if (tr) { GP_T_ADD(1, 1); GP_T_ADD(3, t_c - t_b); }
+        if (tr) { GP_T_ADD(1, 1); GP_T_ADD(3, t_c - t_b); if (my_tiles == 1) GP_T_STAMP(66); if (pgl == cw) { GP_T_ADD(71, t_c - t_b); GP_T_ADD(72, 1); } }
         uint8_t* tile = smem + st * GEO::TILE_BYTES;
         const int tok0 = (pg0 + pgl) * GP_PAGE;
         const bool has_new = last_chunk && (pgl == npg - 1);
         if (has_new) {
           // append: slot n_old of this page receives k_t, v_t; patch the staged copy too
           const int s = n_old - tok0;
-          const int page = sd[16];
+          const int page = sd[GEO::SLOT_PAGES + npg - 1];
           constexpr int CH = D / 8;
           if (lane < 2 * CH) {
             const int isv = lane / CH, c = lane % CH;
@@ -506,8 +579,9 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           if (tr) { GP_T_ADD(8, GP_T_NOW() - t_d); GP_T_ADD(9, 1); }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[st]);
+        if (!top_up(it)) { ok = false; break; }            // the stage is free: fetch the next tile into it
       }
+      if (tr) GP_T_ADD(78, GP_T_NOW() - t_prev);
       if (!ok) break;
       const long long t_e = GP_T_NOW();
       (void)t_e;
@@ -516,7 +590,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
       const int cb = it % NCOMB;
-      if (!wait_bar(&comb_empty[cb], ((it / NCOMB) & 1u) ^ 1u, s_misc)) break;
+      if (!wait_bar(&comb_empty[cb], ((it / NCOMB) & 1u) ^ 1u, s_misc, 6)) break;
       float* my_comb = comb + (cb * NCW + cw) * comb_w;
       if (row < G) {
         if ((lane & 3) == 0) { my_comb[row] = m_run; my_comb[8 + row] = l_run; }
@@ -533,102 +607,18 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         if (lane == 0) mbar_arrive(qt_empty);
       }
       if (lane == 0) mbar_arrive(&slot_empty[sl]);
-      if (tr) GP_T_ADD(5, GP_T_NOW() - t_e);
+      if (tr) { GP_T_ADD(5, GP_T_NOW() - t_e); if (it == 0) GP_T_STAMP(67); }
     }
+    cp_async_wait<0>();                  // after an abort copies may still be in flight: let them land
     if (tr) GP_T_ADD(6, GP_T_NOW() - t_loop0);
 #ifdef GP_TRACE
     if (tr) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 35] = (long long)gt; }
 #endif
-  } else if (warp == 1) {
-    // ================================= summaries ==========================================
-    uint32_t qt_uses = 0;
-    constexpr int PER = D / 32;
-    for (uint32_t it = 0;; ++it) {
-      const int sl = it % NI;
-      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc)) break;
-      const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
-      const int* sd = reinterpret_cast<const int*>(slot);
-      const int npg = sd[3];
-      if (npg < 0) break;
-      const int bi = sd[0], r = sd[1], pg0 = sd[2], chunk = sd[4];
-      const int flags = sd[8], Pr = sd[9], par = sd[12], started = (flags >> 1) & 1;
-      const int lh = sd[14];
-      const int l = lh / p.Hkv, h = lh % p.Hkv;
-      const bool need_qt = (flags & 1) && (pg0 < Pr - 1);
-      if (chunk == 0 || need_qt) {
-        if (need_qt) {
-          if (!wait_bar(qt_empty, (qt_uses & 1u) ^ 1u, s_misc)) break;
-        }
-        for (int g = 0; g < G; ++g) {
-          const int head = h * G + g;
-          const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(slot + GEO::SLOT_DESC + g * GEO::ROW_BYTES);
-          double qv[PER];
-          double sq = 0.0;
-#pragma unroll
-          for (int e = 0; e < PER; ++e) {
-            qv[e] = (double)__bfloat162float(qrow[lane + 32 * e]);
-            sq += qv[e] * qv[e];
-          }
-          double ov[2][PER];
-#pragma unroll
-          for (int x = 0; x < 2; ++x) {                       // both views' loads in flight together
-            const double* oldp = p.summ + gp_summ_off(p, l, r, par, x, head);
-#pragma unroll
-            for (int e = 0; e < PER; ++e) ov[x][e] = started ? __ldcg(oldp + lane + 32 * e) : 0.0;
-          }
-#pragma unroll
-          for (int x = 0; x < 2; ++x) {
-            const double beta = x ? p.beta_l : p.beta_s;
-            double* newp = p.summ + gp_summ_off(p, l, r, par ^ 1, x, head);
-            double nv[PER];
-            double ss = 0.0;
-#pragma unroll
-            for (int e = 0; e < PER; ++e) {
-              nv[e] = started ? beta * ov[x][e] + (1.0 - beta) * qv[e] : qv[e];     // Eq. 6
-              if (chunk == 0) newp[lane + 32 * e] = nv[e];
-              ss += nv[e] * nv[e];
-            }
-            if (need_qt) {
-              double sq2 = sq;
-#pragma unroll
-              for (int o2 = 16; o2 > 0; o2 >>= 1) {
-                sq2 += __shfl_xor_sync(0xffffffffu, sq2, o2);
-                ss += __shfl_xor_sync(0xffffffffu, ss, o2);
-              }
-              // Eq. 12
-              const double gamma = ss > 0.0 ? sqrt(sq2 / (double)D) / sqrt(ss / (double)D) : 1.0;
-              double* dst = qt + (size_t)(x * G + g) * (D + QT_PAD);
-              if (p.rope_theta != 0.0) {
-                const double* cs = p.rope_cs + (size_t)bi * (D / 2) * 2;
-#pragma unroll
-                for (int e = 0; e < PER / 2; ++e) {
-                  const int j = lane + 32 * e;
-                  const double co = cs[2 * j], si = cs[2 * j + 1];
-                  const double x1 = gamma * nv[e], x2 = gamma * nv[e + PER / 2];
-                  dst[j] = x1 * co - x2 * si;
-                  dst[j + D / 2] = x2 * co + x1 * si;
-                }
-              } else {
-#pragma unroll
-                for (int e = 0; e < PER; ++e) dst[lane + 32 * e] = gamma * nv[e];
-              }
-            }
-          }
-        }
-        if (need_qt) {
-          ++qt_uses;
-          __syncwarp();
-          if (lane == 0) mbar_arrive(qt_full);
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&slot_empty[sl]);
-    }
   } else if (warp == 2) {
     // ================================= merger =============================================
     for (uint32_t it = 0;; ++it) {
       const int sl = it % NI;
-      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc)) break;
+      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc, 7)) break;
       const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
@@ -636,7 +626,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       const int bi = sd[0], nchunks = sd[5], rc_i = sd[13], lh = sd[14];
       const int l = lh / p.Hkv, h = lh % p.Hkv;
       const int cb = it % NCOMB;
-      if (!wait_bar(&comb_full[cb], (it / NCOMB) & 1u, s_misc)) break;
+      if (!wait_bar(&comb_full[cb], (it / NCOMB) & 1u, s_misc, 8)) break;
       const float* cbuf = comb + (size_t)cb * NCW * comb_w;
       const size_t out_row0 = (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
       const int PSTRIDE = G * (D + 2);

@@ -90,6 +90,7 @@ struct GpDev {
   int4* cmp_info;                        // [M+1] compressing requests: {request, P, index in bnd_info, first compaction chunk}
   double* zbuf;                          // [L*H_kv][2][z_stride][G] boundary units, per view (short, long): exp(summary logit - its page's max)
   long long z_stride;                    // max_batch_tokens rounded up to a multiple of the page size
+  double* qtil;                          // [M][L*H_kv][2][G][d] calibrated, rotated summaries q~ of boundary requests, by batch slot
   double* zstat;                         // [L*H_kv][max_batch_tokens / b][2][G][2] per-page softmax partials (max, sum)
   int* sum_par;                          // [M] which of the two summary buffers is current
   int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
@@ -116,7 +117,7 @@ __device__ __forceinline__ size_t gp_summ_off(const GpDev& p, int l, int r, int 
 
 // ---- optional cycle trace (compiled in only with -DGP_TRACE, for development builds) ----------------
 #ifdef GP_TRACE
-#define GP_TRACE_WORDS 64
+#define GP_TRACE_WORDS 96
 #define GP_T_ADD(slot, val) atomicAdd(reinterpret_cast<unsigned long long*>(&p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + (slot)]), (unsigned long long)(val))
 #define GP_T_NOW() clock64()
 #define GP_T_STAMP(slot) do { unsigned long long gt_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + (slot)] = (long long)gt_; } while (0)
@@ -150,6 +151,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// non-blocking probe of a phase
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait: returns false when the limit ran out (the caller records GP_E_SPIN and goes on).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   for (uint32_t it = 0; it < GP_SPIN_LIMIT; ++it) {
@@ -165,6 +178,13 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, u
       "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
       : "memory");
 }
+// 16-byte asynchronous copy global -> shared (L2 only), tracked per thread in commit groups
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src_gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src_gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 

@@ -49,7 +49,7 @@ namespace {
 
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
-      b_flags, mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, zstat, sum_par,
+      b_flags, mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
       evict, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
   int max_rc;
@@ -117,6 +117,7 @@ Layout make_layout(const gp_config& c) {
   L.free_peek = take((M + 1) * 4);
   L.cmp_info = take((M + 1) * 16);
   L.zbuf = take(LH * (size_t)(L.max_batch_tokens + b) * 2 * G * 8);
+  L.qtil = take(M * LH * 2 * (size_t)G * d * 8);
   L.zstat = take(LH * ((size_t)L.max_batch_tokens / b + 1) * 2 * G * 2 * 8);
   L.evict = take(M * LH * b * 4);
   L.cflags = take(LH * ((size_t)L.max_batch_tokens / GP_MOVE_TOK + 2 * M + 1) * 4);
@@ -184,11 +185,93 @@ __device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long
   __syncthreads();
 }
 
+// Summary update of one (batch slot, layer, KV head) unit, run by the CTAs of the plan kernel other than the
+// first, concurrently with the planning: Eq. 6 on the un-rotated query of every head of the group (read from
+// one of the request's two buffers, written to the other; the decision step flips the buffers of the requests
+// that were really stepped, so a unit that turns out not to step leaves no trace), and, for a request that
+// reaches its capacity boundary, the calibrated (Eq. 12) and rotated summaries q~ in fp64 for the attention
+// kernel's logits.  One warp per (view, head) row; a CTA takes as many units at a time as its warps cover.
+template <int D>
+__device__ void prepare_row(const GpDev& p, const int* __restrict__ req_ids, int n_req, const __nv_bfloat16* __restrict__ q,
+                            int bi, int lh, int row) {
+  constexpr int PER = D / 32;
+  const int lane = threadIdx.x & 31;
+  const int G = p.G;
+  const int l = lh / p.Hkv, h = lh % p.Hkv;
+  const int x = row / G, g = row % G;
+  const int head = h * G + g;
+  // two round trips in all: the request id (with the ids before it, for the duplicate check and the query
+  // row, which do not depend on it), then the request's state and the old summary from both of its buffers
+  const int r = req_ids[bi];
+  bool dup = false;                                          // only the first batch slot naming a request counts
+  for (int j0 = 0; j0 < bi; j0 += 32) {
+    const int j = j0 + lane;
+    dup |= j < bi && req_ids[j] == r;
+  }
+  const __nv_bfloat16* qrow = q + (((size_t)l * n_req + bi) * p.Hq + head) * D;
+  float qf[PER];
+#pragma unroll
+  for (int e = 0; e < PER; ++e) qf[e] = __bfloat162float(qrow[lane + 32 * e]);
+  if (r < 0 || r >= p.M || __any_sync(0xffffffffu, dup)) return;
+  const int live = p.live[r], n_old = p.n[r], Pr = p.P[r], started = p.started[r], par = p.sum_par[r];
+  const long long pos = p.pos[r];
+  double ov0[PER], ov1[PER];
+  {
+    const double* o0 = p.summ + gp_summ_off(p, l, r, 0, x, head);
+    const double* o1 = p.summ + gp_summ_off(p, l, r, 1, x, head);
+#pragma unroll
+    for (int e = 0; e < PER; ++e) { ov0[e] = __ldcg(o0 + lane + 32 * e); ov1[e] = __ldcg(o1 + lane + 32 * e); }
+  }
+  if (!live) return;
+  const bool need_qt = (n_old + 1 == Pr * GP_PAGE) && Pr > 1;
+  {
+    const double beta = x ? p.beta_l : p.beta_s;
+    double* newp = p.summ + gp_summ_off(p, l, r, par ^ 1, x, head);
+    double nv[PER];
+    double sq = 0.0, ss = 0.0;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+      const double qv = (double)qf[e];
+      const double ov = par ? ov1[e] : ov0[e];
+      sq += qv * qv;
+      nv[e] = started ? beta * ov + (1.0 - beta) * qv : qv;              // Eq. 6
+      newp[lane + 32 * e] = nv[e];
+      ss += nv[e] * nv[e];
+    }
+    if (need_qt) {
+#pragma unroll
+      for (int o2 = 16; o2 > 0; o2 >>= 1) {
+        sq += __shfl_xor_sync(0xffffffffu, sq, o2);
+        ss += __shfl_xor_sync(0xffffffffu, ss, o2);
+      }
+      // Eq. 12
+      const double gamma = ss > 0.0 ? sqrt(sq / (double)D) / sqrt(ss / (double)D) : 1.0;
+      double* dst = p.qtil + (((size_t)bi * p.L * p.Hkv + lh) * 2 * G + row) * D;
+      if (p.rope_theta != 0.0) {
+#pragma unroll
+        for (int e = 0; e < PER / 2; ++e) {
+          const int j = lane + 32 * e;
+          const double inv = pow(p.rope_theta, -2.0 * (double)j / (double)D);
+          double si, co;
+          sincos((double)pos * inv, &si, &co);
+          const double x1 = gamma * nv[e], x2 = gamma * nv[e + PER / 2];
+          dst[j] = x1 * co - x2 * si;
+          dst[j + D / 2] = x2 * co + x1 * si;
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < PER; ++e) dst[lane + 32 * e] = gamma * nv[e];
+      }
+    }
+  }
+}
+
 // Step plan: validates the batch, cuts every stepped request into chunks and writes one work descriptor
 // per chunk for the attention kernel, lists the requests that reach their capacity boundary with this
 // step's append (trailing check: n + 1 == P b) and hands each a slice of the logit scratch.
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
-gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions) {
+gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
+               const __nv_bfloat16* __restrict__ q) {
   __shared__ int sv[33];
   __shared__ long long sw[33];
   __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
@@ -199,6 +282,19 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const bool in = i < n_req;
   gp_pdl_wait();
   gp_pdl_launch_dependents();
+  if (blockIdx.x > 0) {                       // summary CTAs: one warp per (unit, view, head)
+    const int LH = p.L * p.Hkv;
+    const int rows = 2 * p.G, upc = 32 / rows;             // units per CTA and pass
+    const int warp = threadIdx.x >> 5;
+    const long long units = (long long)n_req * LH;
+    if (warp < upc * rows) {
+      for (long long u = ((long long)blockIdx.x - 1) * upc + warp / rows; u < units; u += ((long long)gridDim.x - 1) * upc) {
+        if (p.d == 128) prepare_row<128>(p, req_ids, n_req, q, (int)(u / LH), (int)(u % LH), warp % rows);
+        else prepare_row<64>(p, req_ids, n_req, q, (int)(u / LH), (int)(u % LH), warp % rows);
+      }
+    }
+    return;
+  }
   const int free_top0 = *p.free_top;
   const long long t_plan0 = GP_T_NOW();
   (void)t_plan0;
@@ -524,6 +620,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.free_peek = reinterpret_cast<int*>(base + L.free_peek);
   d.cmp_info = reinterpret_cast<int4*>(base + L.cmp_info);
   d.zbuf = reinterpret_cast<double*>(base + L.zbuf);
+  d.qtil = reinterpret_cast<double*>(base + L.qtil);
   d.zstat = reinterpret_cast<double*>(base + L.zstat);
   d.sum_par = reinterpret_cast<int*>(base + L.sum_par);
   d.evict = reinterpret_cast<int*>(base + L.evict);
@@ -621,7 +718,15 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   const bool prof = pool->profiling != 0;
   if (prof) cudaEventRecord(pool->ev[0], s);
   const bool pdl = !prof;                      // events between the kernels need them serialised the plain way
-  gp_launch(gp_plan_kernel, 1, GP_PLAN_THREADS, 0, s, pdl, d, dev_req_ids, n_req, dev_actions);
+  {
+    // CTA 0 plans; the others update the query summaries of the batch, one (request, layer, KV head) at a time
+    const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
+    const long long want = ((long long)n_req * d.L * d.Hkv + upc - 1) / upc;
+    const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
+    const int prep = (int)(want < room ? want : room);
+    gp_launch(gp_plan_kernel, 1 + prep, GP_PLAN_THREADS, 0, s, pdl, d, dev_req_ids, n_req, dev_actions,
+              static_cast<const __nv_bfloat16*>(q));
+  }
   if (prof) cudaEventRecord(pool->ev[1], s);
   gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl);
   if (prof) cudaEventRecord(pool->ev[2], s);
