@@ -6,8 +6,8 @@
 Workload: the one-layer Qwen3-8B-shaped configuration (32 query / 8 KV heads, head_dim 128, bf16,
 page 16; 64 concurrent requests, prompts uniform in [128, 1024], 4096 decode steps each, per-request
 heavy-hitter fraction log-uniform in [0.5 %, 20 %], seed 1), synthetic inputs.  One "step" is one
-`gp_decode_step` over all 64 requests: plan, fused append + paged GQA attention + summary update,
-boundary scoring and working sets, decision + allocator, selection + compaction.
+`gp_decode_step` over all 64 requests: plan + summary update, fused append + paged GQA attention +
+boundary logits, working sets + selection + decision + allocator, compaction.
 
 The K timed steps are steps [S0, S0 + K) of the 4096-step job with S0 = (4096 - K) // 2, reached by
 running the S0 preceding steps untimed; K = 4096 (the default) times the whole job.  Warm-up steps
@@ -195,7 +195,7 @@ class Job:
         B = self.B
         s = self.wl.shape
         Wb = s.token_bytes
-        fixed = 2 * s.n_q_heads * s.head_dim + 4 * s.n_q_heads * s.head_dim + 2 * (2 * s.n_q_heads * s.head_dim * 4)
+        fixed = 2 * s.n_q_heads * s.head_dim + 4 * s.n_q_heads * s.head_dim        # query rows in, output rows out
         n_new = self.n + 1
         attn = float(s.n_layers * (n_new.sum() * Wb + self.nreq * (Wb + fixed)) + 4 * self.P.sum())
         at_b = n_new == self.P * 16
@@ -282,13 +282,14 @@ def run_ours(args):
     B.gp_set_profiling(job.pool.handle, False)
     moved = job.moved_rows() - moved0
     compact_bytes = 2.0 * moved * (2 * s.head_dim * 2 + 4)
-    step_bytes = attn_bytes + score_bytes + compact_bytes
+    summ_bytes = float(K) * job.nreq * s.n_layers * 2 * s.n_q_heads * s.head_dim * 8 * 2      # both views, read + write, fp64
+    step_bytes = attn_bytes + score_bytes + compact_bytes + summ_bytes
     peak, peak_kind = measured_peak()
     attn_ms = float(kms[1])
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
     ratio = traffic_ratio()
     roofline = {
-        "bound": "hbm", "kernel": "gp_attn_kernel<128> (append + paged GQA attention + EMA summaries)",
+        "bound": "hbm", "kernel": "gp_attn_kernel<128> (append + paged GQA attention + boundary logits)",
         "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
         "peak_kind": f"of {peak_kind}",
         "traffic": None if ratio is None else round(ratio * attn_bytes / K),
@@ -301,6 +302,7 @@ def run_ours(args):
     step_roofline = {
         "algorithmic_bytes_per_step": round(step_bytes / K),
         "attention": round(attn_bytes / K), "scoring": round(score_bytes / K), "compaction": round(compact_bytes / K),
+        "summaries": round(summ_bytes / K),
         "achieved_gbs": round(step_gbs, 1), "frac_of_8tbs": round(step_gbs / NOMINAL_HBM_GBS, 4),
         "frac_of_measured": round(step_gbs / peak, 4), "mean_tokens_per_request": round(n_sum / K / job.nreq, 1),
     }
