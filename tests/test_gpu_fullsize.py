@@ -1,0 +1,162 @@
+"""Parity at the full size of the benchmark's workload, in the launch configuration the benchmark times.
+
+All 64 requests of the one-layer Qwen3-8B-shaped configuration run through the C-ABI on the GPU, back to back
+on one stream as in the benchmark (same pool parameters, host staging on).  The float64 oracle cannot follow
+64 requests at that size in seconds, so it follows a sample of them, each simulated alone: in this
+configuration the per-request page cap never binds and the pool holds every request at its cap, so a request's
+trajectory does not depend on the others.  Compared per step for the sampled requests: action and attention
+output; at every capacity boundary: K^S, K^L, Delta and (on compression) the retained token set; at the end:
+page count, token count and query summaries.  Tolerances as in lockstep.py; near-ties are resolved the GPU's
+way so that both sides stay comparable, counted, and must stay below 0.1 % of decisions.
+For all requests, properties that hold at any size: one valid action per request and step, page accounting
+(free pages + pages held = pool size, every held page referenced once), step and token counters, no error bit.
+"""
+import numpy as np
+import pytest
+
+from oracle import growpage_oracle as O
+from paper_2609_03494_b200 import binding as B
+from paper_2609_03494_b200 import harness as H
+from paper_2609_03494_b200 import workload as W
+
+from tests.lockstep import ATTN_MAX_ABS, ATTN_MEAN_ABS, NEAR_TIE, NEAR_TIE_FRACTION, SUMMARY_REL
+
+pytestmark = pytest.mark.gpu
+
+SAMPLE = (5, 23, 41, 62)          # request indices the oracle follows
+STEPS = 448                        # 28 capacity boundaries per request
+
+
+def test_bench_configuration_sampled_requests():
+    import torch
+
+    wl = W.layer8b(seed=1)
+    s = wl.shape
+    b = s.page_size
+    nreq = len(wl.requests)
+    dev = "cuda:0"
+    cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
+                        max_pages_per_req=wl.max_pages_per_req, max_requests=nreq, k_loc=wl.k_loc, host_staging=True)
+    gpu = B.Pool(cfg, 0)
+    ocfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=len(SAMPLE) * wl.max_pages_per_req,
+                          max_pages_per_req=wl.max_pages_per_req, max_requests=len(SAMPLE), k_loc=wl.k_loc)
+    ora = O.OraclePool(ocfg)
+    try:
+        # ---- inputs: every request's prompt and its first STEPS decode inputs -------------------------------
+        q_all = np.empty((STEPS, s.n_layers, nreq, s.n_q_heads, s.head_dim), dtype=np.uint16)
+        k_all = np.empty((STEPS, s.n_layers, nreq, s.n_kv_heads, s.head_dim), dtype=np.uint16)
+        v_all = np.empty_like(k_all)
+        o_rid = {}
+        for i, spec in enumerate(wl.requests):
+            stream = wl.stream(spec)
+            kp, vp = stream.prompt_kv()
+            st, rid = gpu.request_add(-1, 0, torch.from_numpy(kp.view(np.int16)).to(dev),
+                                      torch.from_numpy(vp.view(np.int16)).to(dev), spec.prompt_len, wl.initial_pages)
+            assert st == B.GP_OK and rid == i
+            if i in SAMPLE:
+                ost, orid = ora.request_add(-1, 0, H.decode_bits(kp), H.decode_bits(vp), spec.prompt_len, wl.initial_pages)
+                assert ost == O.OK
+                o_rid[i] = orid
+            q_all[:, :, i], k_all[:, :, i], v_all[:, :, i] = stream.steps(0, STEPS)
+        to_dev = lambda a: torch.from_numpy(a.view(np.int16)).to(dev)
+        q_dev, k_dev, v_dev = to_dev(q_all), to_dev(k_all), to_dev(v_all)
+        ids = torch.arange(nreq, dtype=torch.int32, device=dev)
+        out_t = torch.zeros((s.n_layers, nreq, s.n_q_heads, s.head_dim), dtype=torch.float32, device=dev)
+        act_t = torch.zeros(nreq, dtype=torch.int32, device=dev)
+        sample = list(SAMPLE)
+        o_ids = [o_rid[i] for i in sample]
+
+        decisions = {"ws": 0, "sel": 0, "act": 0}
+        near = {"ws": 0, "sel": 0, "act": 0}
+        err_sum, err_cnt, err_max = 0.0, 0, 0.0
+        n_boundaries = n_compress = n_grow = 0
+        for t in range(STEPS):
+            gpu.decode_step(ids, q_dev[t], k_dev[t], v_dev[t], out_t, act_t)
+            rec = ora.step_compute(o_ids, H.decode_bits(q_all[t][:, sample]), H.decode_bits(k_all[t][:, sample]),
+                                   H.decode_bits(v_all[t][:, sample]))
+            g_act = act_t.cpu().numpy()
+            g_out = out_t[:, sample].cpu().numpy().astype(np.float64)
+            assert np.isin(g_act, (B.GP_ACT_NONE, B.GP_ACT_GROW, B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK)).all(), \
+                f"step {t}: actions {np.unique(g_act)}"
+            err = np.abs(g_out - rec.out)
+            err_max = max(err_max, float(err.max()))
+            err_sum += float(err.sum())
+            err_cnt += err.size
+            assert err.max() <= ATTN_MAX_ABS, f"step {t}: attention max abs err {err.max()}"
+
+            overrides = {}
+            for orid, info in rec.boundary.items():
+                i = sample[o_ids.index(orid)]
+                n_boundaries += 1
+                assert info.n_c > 0
+                ks, kl, delta = B.gp_debug_boundary(gpu.handle, i, s.n_layers, s.n_kv_heads)
+                for gk, ok, col in ((ks, info.K_s, 0), (kl, info.K_l, 1)):
+                    decisions["ws"] += ok.size
+                    for (l, h) in np.argwhere(gk != ok):
+                        assert info.ws_margin[l, h, col] < NEAR_TIE and abs(int(gk[l, h]) - int(ok[l, h])) == 1, \
+                            f"step {t} req {i}: working set [{l},{h},{col}] gpu {gk[l, h]} oracle {ok[l, h]}"
+                        near["ws"] += 1
+                if np.array_equal(ks, info.K_s) and np.array_equal(kl, info.K_l):
+                    assert delta == info.delta, f"step {t} req {i}: Delta gpu {delta} oracle {info.delta}"
+                decisions["act"] += 1
+                a = int(g_act[i])
+                g_want = a in (B.GP_ACT_GROW, B.GP_ACT_COMPRESS_FALLBACK)
+                if g_want != info.want_grow:
+                    assert info.action_near_tie, f"step {t} req {i}: grow decision differs outside a near-tie"
+                    near["act"] += 1
+                    overrides.setdefault(orid, {})["want_grow"] = g_want
+                n_grow += a == B.GP_ACT_GROW
+                if a in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK):
+                    n_compress += 1
+                    r = ora.requests[orid]
+                    K_t = info.n_c - b
+                    for l in range(s.n_layers):
+                        for h in range(s.n_kv_heads):
+                            decisions["sel"] += 1
+                            keep, margin = O.select_retained(O.token_scores(info.a_s[l, h], info.a_l[l, h]), r.P - 1, b,
+                                                             K_t, ocfg.k_loc)
+                            want_tok = r.tok[l, h, keep]
+                            got = B.gp_debug_retained(gpu.handle, i, l, h, info.n_c)
+                            assert np.array_equal(got[K_t:], r.tok[l, h, info.n_c:info.n_c + b]), "protected page lost"
+                            if not np.array_equal(got[:K_t], want_tok):
+                                assert margin < NEAR_TIE, f"step {t} req {i} ({l},{h}): retained set differs, margin {margin}"
+                                near["sel"] += 1
+                                slots = np.searchsorted(r.tok[l, h, :info.n_c], got[:K_t])
+                                overrides.setdefault(orid, {}).setdefault("keep", {})[(l, h)] = slots
+            ora.step_apply(rec, overrides)
+            for j, i in enumerate(sample):
+                assert int(g_act[i]) == int(rec.actions[j]), f"step {t} req {i}: action gpu {g_act[i]} oracle {rec.actions[j]}"
+
+        # ---- sampled requests: final state -----------------------------------------------------------------
+        assert n_boundaries == len(sample) * (STEPS // b)          # one boundary every b steps, whatever the prompt length
+        assert n_compress + n_grow == n_boundaries and n_compress > 0
+        for i in sample:
+            P, n, pos, table = B.gp_debug_request(gpu.handle, i, cfg.max_pages_per_req)
+            oP, on, opos, _ = ora.request_state(o_rid[i])
+            assert (P, n, pos) == (oP, on, opos)
+            g = B.gp_debug_summaries(gpu.handle, i, s.n_layers, s.n_q_heads, s.head_dim)
+            o = ora.summaries(o_rid[i])
+            rel = np.linalg.norm(g - o, axis=-1) / np.linalg.norm(o, axis=-1)
+            assert rel.max() <= SUMMARY_REL, f"req {i}: summary relative error {rel.max()}"
+        assert err_sum / err_cnt <= ATTN_MEAN_ABS
+        for kind in decisions:
+            assert near[kind] <= NEAR_TIE_FRACTION * max(decisions[kind], 1), (kind, near[kind], decisions[kind])
+
+        # ---- all requests: invariants ---------------------------------------------------------------------------
+        n_free, ref, counters = B.gp_debug_pool(gpu.handle, cfg.n_pages)
+        assert counters[7] == 0, f"kernel error bits {counters[7]}"
+        assert counters[5] == STEPS and counters[6] == STEPS * nreq
+        held = 0
+        seen = set()
+        for i in range(nreq):
+            P, n, pos, table = B.gp_debug_request(gpu.handle, i, cfg.max_pages_per_req)
+            assert pos == wl.requests[i].prompt_len + STEPS and 0 < n <= P * b and P <= cfg.max_pages_per_req
+            pages = [int(x) for x in table[:P]]
+            assert not (seen & set(pages)) and len(set(pages)) == P
+            seen |= set(pages)
+            held += P
+        assert held + n_free == cfg.n_pages
+        assert int((ref == 1).sum()) == held and int((ref > 1).sum()) == 0
+        assert counters[0] + counters[1] + counters[2] == nreq * (STEPS // b) and counters[3] == 0   # every boundary decided
+    finally:
+        gpu.close()
