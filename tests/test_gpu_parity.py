@@ -4,6 +4,7 @@ import pytest
 
 from oracle import growpage_oracle as O
 from paper_2609_03494_b200 import binding as B
+from paper_2609_03494_b200 import harness as H
 from paper_2609_03494_b200 import workload as W
 from tests import lockstep as LS
 
@@ -117,3 +118,70 @@ def test_batch_edge_cases_and_host_entry_point():
         assert B.gp_launch_count(pool.handle) > 0
     finally:
         pool.close()
+
+
+def test_synchronised_boundaries_put_several_boundary_items_on_every_cta():
+    # equal prompt lengths: every request reaches its capacity boundary in the same step, so the attention
+    # kernel's CTAs each get several boundary work items in a row (their calibrated summaries share one buffer
+    # per CTA) and the selection kernel has more jobs than CTAs
+    shape = W.Shape(2, 16, 8, 64)
+    reqs = [W.RequestSpec(i, 180, 40, 0.02 + 0.004 * i) for i in range(40)]
+    wl = W.Workload("sync-boundaries", 21, shape, reqs, n_resident=40, initial_pages=0, max_pages_per_req=16,
+                    n_pages=40 * 16)
+    st = LS.run_lockstep(wl, tau=-0.07)
+    _report("synchronised boundaries", st)
+    assert st.actions.get(B.GP_ACT_COMPRESS, 0) + st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) > 0
+
+
+def test_equal_scores_take_the_general_selection_paths():
+    # zero queries: summaries and calibrated summaries are zero, every candidate gets the same probability, so
+    # the single-histogram fast paths find one crowded bin and hand over to the general radix descent; ties are
+    # broken by slot order on both sides (Eq. 7 by count, Eq. 10 keeps the older slots)
+    import torch
+    L, Hq, Hkv, d, n_prompt, steps = 1, 4, 2, 64, 100, 70
+    kw = dict(n_pages=16, max_pages_per_req=9, max_requests=4, k_loc=2)
+    gpu = B.Pool(B.make_config(L, Hq, Hkv, d, tau=1.0, **kw))
+    ora = O.OraclePool(O.OracleConfig(L, Hq, Hkv, d, tau=1.0, **kw))
+    try:
+        rng = np.random.default_rng(5)
+        bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+        kp, vp = bits(L, n_prompt, Hkv, d), bits(L, n_prompt, Hkv, d)
+        assert gpu.request_add(-1, 0, kp, vp, n_prompt, 0) == (B.GP_OK, 0)
+        assert ora.request_add(-1, 0, H.decode_bits(kp), H.decode_bits(vp), n_prompt, 0) == (O.OK, 0)
+        ids = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+        out = torch.zeros((L, 1, Hq, d), dtype=torch.float32, device="cuda:0")
+        act = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+        n_compress = 0
+        for t in range(steps):
+            q = np.zeros((L, 1, Hq, d), dtype=np.uint16)
+            k, v = bits(L, 1, Hkv, d), bits(L, 1, Hkv, d)
+            dev = lambda a: torch.from_numpy(a.view(np.int16)).to("cuda:0")
+            gpu.decode_step(ids, dev(q), dev(k), dev(v), out, act)
+            rec = ora.step_compute([0], H.decode_bits(q), H.decode_bits(k), H.decode_bits(v))
+            assert np.abs(out.cpu().numpy() - rec.out).max() <= LS.ATTN_MAX_ABS
+            for rid, info in rec.boundary.items():
+                ks, kl, delta = B.gp_debug_boundary(gpu.handle, 0, L, Hkv)
+                assert np.array_equal(ks, info.K_s) and np.array_equal(kl, info.K_l) and delta == info.delta
+                if int(act.cpu()[0]) in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK):
+                    n_compress += 1
+                    r = ora.requests[0]
+                    K_t = info.n_c - 16
+                    for l in range(L):
+                        for h in range(Hkv):
+                            keep, _ = O.select_retained(O.token_scores(info.a_s[l, h], info.a_l[l, h]), r.P - 1, 16, K_t, 2)
+                            got = B.gp_debug_retained(gpu.handle, 0, l, h, info.n_c)
+                            assert np.array_equal(got[:K_t], r.tok[l, h, keep]), f"step {t} ({l},{h}): retained set differs"
+            ora.step_apply(rec, {})
+            assert int(act.cpu()[0]) == int(rec.actions[0]), f"step {t}"
+        assert n_compress >= 3
+        assert B.gp_debug_pool(gpu.handle)[2][7] == 0
+    finally:
+        gpu.close()
+
+
+def test_candidate_set_larger_than_the_staging_buffers():
+    # more than 6144 candidate tokens: the scores of a unit no longer fit the selection kernel's shared memory
+    # (they go through global scratch) and its softmax factors are recomputed per token instead of tabulated
+    st = _single_request_case(W.Shape(1, 4, 2, 64), 6300, 80)
+    _report("6300-token prompt", st)
+    assert st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) >= 1
