@@ -285,6 +285,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     // which may belong to a later item (the fetch position runs ahead of the compute position, across item
     // boundaries, but never further than the ring of item slots allows).  No other warp touches the ring, so
     // program order plus a proxy fence orders the reads of a stage before the copy that overwrites it.
+    const uint64_t kv_policy = l2_policy_evict_first();    // the K/V stream is read once per step: first out of the L2
     uint32_t my_fetch = 0, f_it = 0;
     int f_pgl = 0, f_npg = 0, f_lh = 0;
     bool f_have = false, f_done = false;
@@ -315,7 +316,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, f_lh / p.Hkv, page, f_lh % p.Hkv)) + lane * 16;
           const uint32_t dst = smem_u32(smem + fst * GEO::TILE_BYTES) + lane * 16;
 #pragma unroll
-          for (int c = 0; c < GEO::TILE_BYTES / 512; ++c) cp_async16(dst + c * 512, src + c * 512);
+          for (int c = 0; c < GEO::TILE_BYTES / 512; ++c) cp_async16_hint(dst + c * 512, src + c * 512, kv_policy);
           cp_async_commit();
         }
         ++my_fetch;
