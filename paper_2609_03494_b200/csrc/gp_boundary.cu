@@ -972,6 +972,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   __shared__ int4 s_info[GP_MAX_REQ + 1];     // compressing requests: {request, P, boundary index, first chunk}
   __shared__ int ev[GP_PAGE];
   __shared__ int s_i[8];
+  __shared__ int s_dst[MOVE_TOK], s_spage[MOVE_TOK], s_dpage[MOVE_TOK];   // per source slot of the chunk: destination slot (-1: stays or goes), source and destination page
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int LH = p.L * p.Hkv;
@@ -1012,48 +1013,55 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
     const int Pr = inf.y;
     const int* table = p.page_table + (size_t)r * p.cap;
     const int* shadow = p.shadow + (size_t)r * p.cap;
-    if (tid < GP_PAGE) ev[tid] = p.evict[((size_t)inf.z * LH + lh) * GP_PAGE + tid];
-    __syncthreads();
     const int n_src = Pr * GP_PAGE;
     const int c0 = j * MOVE_TOK;
+    // second round trip: the eviction list, and for every source slot of the chunk its page and the page one
+    // before it (a slot moves down by at most one page) with their copy-on-write targets
+    int t0 = 0, s0 = -1, tm = 0, sm = -1;
+    const int my_i = c0 + tid;                             // the slot this thread plans (first MOVE_TOK threads)
+    if (tid < MOVE_TOK && my_i < n_src) {
+      const int pg = my_i / GP_PAGE;
+      t0 = table[pg]; s0 = shadow[pg];
+      if (pg > 0) { tm = table[pg - 1]; sm = shadow[pg - 1]; }
+    }
+    if (tid < GP_PAGE) ev[tid] = p.evict[((size_t)inf.z * LH + lh) * GP_PAGE + tid];
+    __syncthreads();
+    int tokv = 0, tok_dst = -1, tok_page = 0;
+    if (tid < MOVE_TOK) {
+      int ds = -1, dpage = 0;
+      if (my_i < n_src) {
+        int sh = 0; bool evicted = false;
+#pragma unroll
+        for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < my_i); evicted |= (ev[e2] == my_i); }
+        const int pg = my_i / GP_PAGE;
+        const bool cow = (pg < Pr - 1) && (s0 >= 0);
+        if (!evicted && (sh > 0 || cow)) {
+          ds = my_i - sh;
+          dpage = (ds / GP_PAGE == pg) ? (s0 >= 0 ? s0 : t0) : (sm >= 0 ? sm : tm);
+          tokv = p.tok[gp_tok_off(p, l, t0, h) + (my_i % GP_PAGE)];
+          tok_dst = ds; tok_page = dpage;
+        }
+      }
+      s_dst[tid] = ds; s_spage[tid] = t0; s_dpage[tid] = dpage;
+    }
+    __syncthreads();
 
     uint4 val[PIECES];
     int dst_code[PIECES];
-    int tokv = 0, tok_dst = -1;
 #pragma unroll
     for (int k2 = 0; k2 < PIECES; ++k2) {
       const int piece = tid + k2 * CT;
       const int tl = piece / (2 * CH), pc = piece % (2 * CH);
       const int i = c0 + tl;
+      const int ds = s_dst[tl];
       dst_code[k2] = -1;
       val[k2] = make_uint4(0, 0, 0, 0);
-      if (i < n_src) {
-        int sh = 0; bool evicted = false;
-#pragma unroll
-        for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < i); evicted |= (ev[e2] == i); }
-        const int pg = i / GP_PAGE;
-        const bool cow = (pg < Pr - 1) && (shadow[pg] >= 0);
-        if (!evicted && (sh > 0 || cow)) {
-          const int isv = pc / CH, cp = pc % CH;
-          const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, l, table[pg], h)) +
-                               isv * GP_PAGE * ROW_BYTES + (i % GP_PAGE) * ROW_BYTES + (cp << 4);
-          val[k2] = *reinterpret_cast<const uint4*>(src);
-          dst_code[k2] = ((i - sh) << 5) | ((cp ^ (i & 7)) << 1) | isv;   // slot, logical chunk, K or V
-        }
-      }
-    }
-    if (tid < MOVE_TOK) {
-      const int i = c0 + tid;
-      if (i < n_src) {
-        int sh = 0; bool evicted = false;
-#pragma unroll
-        for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < i); evicted |= (ev[e2] == i); }
-        const int pg = i / GP_PAGE;
-        const bool cow = (pg < Pr - 1) && (shadow[pg] >= 0);
-        if (!evicted && (sh > 0 || cow)) {
-          tokv = p.tok[gp_tok_off(p, l, table[pg], h) + (i % GP_PAGE)];
-          tok_dst = i - sh;
-        }
+      if (ds >= 0) {
+        const int isv = pc / CH, cp = pc % CH;
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, l, s_spage[tl], h)) +
+                             isv * GP_PAGE * ROW_BYTES + (i % GP_PAGE) * ROW_BYTES + (cp << 4);
+        val[k2] = *reinterpret_cast<const uint4*>(src);
+        dst_code[k2] = (tl << 5) | ((cp ^ (i & 7)) << 1) | isv;   // slot of the chunk, logical 16-byte piece, K or V
       }
     }
     const long long t_c2 = GP_T_NOW();
@@ -1083,19 +1091,16 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 #pragma unroll
     for (int k2 = 0; k2 < PIECES; ++k2) {
       if (dst_code[k2] >= 0) {
-        const int ds = dst_code[k2] >> 5, c = (dst_code[k2] >> 1) & 15, isv = dst_code[k2] & 1;
-        const int pg = ds / GP_PAGE;
-        const int page = shadow[pg] >= 0 ? shadow[pg] : table[pg];
-        uint8_t* dst = reinterpret_cast<uint8_t*>(p.kv + gp_tile_off(p, l, page, h)) + isv * GP_PAGE * ROW_BYTES +
+        const int tl = dst_code[k2] >> 5, c = (dst_code[k2] >> 1) & 15, isv = dst_code[k2] & 1;
+        const int ds = s_dst[tl];
+        uint8_t* dst = reinterpret_cast<uint8_t*>(p.kv + gp_tile_off(p, l, s_dpage[tl], h)) + isv * GP_PAGE * ROW_BYTES +
                        (ds % GP_PAGE) * ROW_BYTES + ((c ^ (ds & 7)) << 4);
         *reinterpret_cast<uint4*>(dst) = val[k2];
       }
     }
     if (tok_dst >= 0) {
       atomicAdd(&s_i[3], 1);
-      const int pg = tok_dst / GP_PAGE;
-      const int page = shadow[pg] >= 0 ? shadow[pg] : table[pg];
-      p.tok[gp_tok_off(p, l, page, h) + (tok_dst % GP_PAGE)] = tokv;
+      p.tok[gp_tok_off(p, l, tok_page, h) + (tok_dst % GP_PAGE)] = tokv;
     }
   }
   __syncthreads();
