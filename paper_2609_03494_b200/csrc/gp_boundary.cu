@@ -1074,14 +1074,14 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
     if (touched == 0x9e3779b9u && c0 < 0) s_i[4] = 1;      // never true; keeps the dependency alive
     __syncthreads();
     if (tid == 0) {
-      __threadfence();
+      // No fence on either side: the flag only says that loads have returned (they have: their values were
+      // consumed above), and the stores below are issued after the flag has been seen.
       *reinterpret_cast<volatile int*>(p.cflags + item) = stamp;      // "my sources are read"
       if (j > 0) {                                          // the previous chunk's tail is my first destination
         volatile int* prev = reinterpret_cast<volatile int*>(p.cflags + item - 1);
         unsigned it = 0;
         while (*prev != stamp && it < GP_SPIN_LIMIT) ++it;
         if (it >= GP_SPIN_LIMIT) atomicOr(p.err, GP_E_SPIN_CMP);
-        __threadfence();
       }
     }
     __syncthreads();
