@@ -112,8 +112,10 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
                    const void* q, const void* k, const void* v,
                    void* out, int32_t* dev_actions, void* stream);
 
-/* As gp_decode_step with HOST pointers (pinned memory recommended): copies the inputs to staging
- * inside the blob, runs the step, copies `out` and `actions` back and synchronises `stream`.
+/* As gp_decode_step with HOST pointers: copies the inputs to staging inside the blob, runs the
+ * step, delivers `out` and `actions` and synchronises `stream`.  When `out` and `actions` are
+ * page-locked, mapped host memory (cudaHostAlloc / cudaHostRegister: "pinned"), the kernels write
+ * them directly while they run; otherwise the results are staged on the device and copied back.
  * Needs host_staging = 1 at creation, else GP_ERR_STATE. */
 int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req,
                         const void* q, const void* k, const void* v,

@@ -762,11 +762,22 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
   GP_CUDA(cudaMemcpyAsync(pool->st_q, q, qb, cudaMemcpyHostToDevice, s));
   GP_CUDA(cudaMemcpyAsync(pool->st_k, k, kb, cudaMemcpyHostToDevice, s));
   GP_CUDA(cudaMemcpyAsync(pool->st_v, v, kb, cudaMemcpyHostToDevice, s));
-  const int st = gp_decode_step(pool, pool->st_ids, n_req, pool->st_q, pool->st_k, pool->st_v, pool->st_out,
-                                pool->st_act, stream);
+  // Outputs: when the caller's buffers are page-locked and mapped (the usual pinned allocation), the kernels
+  // write them over the bus while they run and nothing is left to copy when the step ends.  (The same was tried
+  // for the inputs and was slower: rows read over the bus by the kernels stall the pipelines that wait for them.)
+  void* d_out = nullptr;
+  void* d_act = nullptr;
+  const bool direct = cudaHostGetDevicePointer(&d_out, out, 0) == cudaSuccess &&
+                      cudaHostGetDevicePointer(&d_act, actions, 0) == cudaSuccess;
+  if (!direct) (void)cudaGetLastError();           // pageable memory: not an error, the staged path takes over
+  const int st = gp_decode_step(pool, pool->st_ids, n_req, pool->st_q, pool->st_k, pool->st_v,
+                                direct ? d_out : static_cast<void*>(pool->st_out),
+                                direct ? static_cast<int32_t*>(d_act) : pool->st_act, stream);
   if (st != GP_OK) return st;
-  GP_CUDA(cudaMemcpyAsync(out, pool->st_out, qb * 2, cudaMemcpyDeviceToHost, s));
-  GP_CUDA(cudaMemcpyAsync(actions, pool->st_act, (size_t)n_req * 4, cudaMemcpyDeviceToHost, s));
+  if (!direct) {
+    GP_CUDA(cudaMemcpyAsync(out, pool->st_out, qb * 2, cudaMemcpyDeviceToHost, s));
+    GP_CUDA(cudaMemcpyAsync(actions, pool->st_act, (size_t)n_req * 4, cudaMemcpyDeviceToHost, s));
+  }
   GP_CUDA(cudaStreamSynchronize(s));
   return GP_OK;
 }
