@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the GrowPage decode path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload layer|stack]
 
 Workload: the one-layer Qwen3-8B-shaped configuration (32 query / 8 KV heads, head_dim 128, bf16,
 page 16; 64 concurrent requests, prompts uniform in [128, 1024], 4096 decode steps each, per-request
@@ -223,9 +223,11 @@ def run_ours(args):
     device = local_rank
     torch.cuda.set_device(device)
     K, Wm = args.steps, args.warmup
-    K = max(1, min(K, JOB_STEPS))
-    S0 = (JOB_STEPS - K) // 2
-    wl = W.layer8b(seed=shard.shard_seed(1, rank))
+    stack = args.workload == "stack"
+    job_steps = 128 if stack else JOB_STEPS
+    K = max(1, min(K, job_steps))
+    S0 = (job_steps - K) // 2
+    wl = W.stack8b_resident(seed=shard.shard_seed(2, rank)) if stack else W.layer8b(seed=shard.shard_seed(1, rank))
     s = wl.shape
     t_gen = time.time()
     q_all, k_all, v_all, prompts = generate_inputs(wl, S0 + K, torch, pin=True)
@@ -326,16 +328,19 @@ def run_ours(args):
     # ---- CPU baseline: the oracle as it stands, on a bounded sample -------------------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = time_oracle(wl, n_requests=8, n_steps=256, warmup=0)
+        cpu = time_oracle(wl, n_requests=8, n_steps=256, warmup=0) if not stack else time_oracle(wl, n_requests=2, n_steps=32, warmup=0)
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": max(Wm, 3),
             "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "qwen3-8b-layer: L=1, 32q/8kv heads, d=128, page 16, 64 requests x 4096 decode steps, "
-                                   "prompts U[128,1024], heavy-hitter fraction logU[0.5%,20%], seed 1",
-                       "requests_per_gpu": job.nreq, "timed_steps": [S0, S0 + K], "job_steps": JOB_STEPS,
+            "config": {"workload": ("qwen3-8b-stack-resident: L=36, 32q/8kv heads, d=128, page 16, 32 requests x 128 decode "
+                                    "steps, prompts U[400,1000], heavy-hitter fraction logU[0.5%,20%], seed 2 (not the headline "
+                                    "workload)") if stack else
+                                   ("qwen3-8b-layer: L=1, 32q/8kv heads, d=128, page 16, 64 requests x 4096 decode steps, "
+                                    "prompts U[128,1024], heavy-hitter fraction logU[0.5%,20%], seed 1"),
+                       "requests_per_gpu": job.nreq, "timed_steps": [S0, S0 + K], "job_steps": job_steps,
                        "l2": "per-step working set (all resident K/V) is larger than L2; no flush needed",
                        "input_generation_s": round(t_gen, 1)},
             "roofline": roofline, "step_roofline": step_roofline,
@@ -427,6 +432,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="layer", choices=["layer", "stack"],
+                    help="layer: the headline one-layer Qwen3-8B-shaped workload; stack: the 36-layer shape, 32 resident requests")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -229,6 +229,20 @@ def layer8b(seed: int = 1, n_requests: int = 64, n_steps: int = 4096,
                     note="cap never binds: prompt pages + 1 + one page per boundary")
 
 
+def stack8b_resident(seed: int = 2, n_layers: int = 36, n_requests: int = 32, n_steps: int = 128,
+                     prompt_range: Tuple[int, int] = (400, 1000)) -> Workload:
+    """The config-3 shape (36 Qwen3-8B-shaped layers) with every request resident from the first step and a
+    pool that never runs dry: the multi-layer shape without the continuous batching, for measurements."""
+    shape = Shape(n_layers, 32, 8, 128)
+    g = _rng(seed, _KIND_REQUEST)
+    plen = g.integers(prompt_range[0], prompt_range[1] + 1, n_requests)
+    frac = _log_uniform(g, 0.005, 0.2, n_requests)
+    reqs = [RequestSpec(i, int(plen[i]), n_steps, float(frac[i])) for i in range(n_requests)]
+    cap = _pages(prompt_range[1], 16) + 1 + _pages(n_steps, 16)
+    return Workload("qwen3-8b-stack-resident", seed, shape, reqs, n_resident=n_requests, initial_pages=0,
+                    max_pages_per_req=cap, n_pages=n_requests * cap, note="cap never binds")
+
+
 def stack8b(seed: int = 2, n_layers: int = 36, n_resident: int = 256, n_total: int = 1024,
             out_range: Tuple[int, int] = (1024, 16384), pool_bytes: float = 120e9,
             prompt_range: Tuple[int, int] = (128, 1024)) -> Workload:
