@@ -224,7 +224,7 @@ def run_ours(args):
     torch.cuda.set_device(device)
     K, Wm = args.steps, args.warmup
     stack = args.workload == "stack"
-    job_steps = 128 if stack else JOB_STEPS
+    job_steps = 96 if stack else JOB_STEPS
     K = max(1, min(K, job_steps))
     S0 = (job_steps - K) // 2
     wl = W.stack8b_resident(seed=shard.shard_seed(2, rank)) if stack else W.layer8b(seed=shard.shard_seed(1, rank))
@@ -335,7 +335,7 @@ def run_ours(args):
             "metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": max(Wm, 3),
             "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": ("qwen3-8b-stack-resident: L=36, 32q/8kv heads, d=128, page 16, 32 requests x 128 decode "
+            "config": {"workload": ("qwen3-8b-stack-resident: L=36, 32q/8kv heads, d=128, page 16, 16 requests x 96 decode "
                                     "steps, prompts U[400,1000], heavy-hitter fraction logU[0.5%,20%], seed 2 (not the headline "
                                     "workload)") if stack else
                                    ("qwen3-8b-layer: L=1, 32q/8kv heads, d=128, page 16, 64 requests x 4096 decode steps, "
@@ -433,7 +433,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="layer", choices=["layer", "stack"],
-                    help="layer: the headline one-layer Qwen3-8B-shaped workload; stack: the 36-layer shape, 32 resident requests")
+                    help="layer: the headline one-layer Qwen3-8B-shaped workload; stack: the 36-layer shape, 16 resident requests")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -229,7 +229,7 @@ def layer8b(seed: int = 1, n_requests: int = 64, n_steps: int = 4096,
                     note="cap never binds: prompt pages + 1 + one page per boundary")
 
 
-def stack8b_resident(seed: int = 2, n_layers: int = 36, n_requests: int = 32, n_steps: int = 128,
+def stack8b_resident(seed: int = 2, n_layers: int = 36, n_requests: int = 16, n_steps: int = 96,
                      prompt_range: Tuple[int, int] = (400, 1000)) -> Workload:
     """The config-3 shape (36 Qwen3-8B-shaped layers) with every request resident from the first step and a
     pool that never runs dry: the multi-layer shape without the continuous batching, for measurements."""
