@@ -185,3 +185,55 @@ def test_candidate_set_larger_than_the_staging_buffers():
     st = _single_request_case(W.Shape(1, 4, 2, 64), 6300, 80)
     _report("6300-token prompt", st)
     assert st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) >= 1
+
+
+def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches():
+    # gp_decode_step only enqueues kernels (chained with programmatic dependent launch): a sequence of steps can
+    # be captured into a CUDA graph once and replayed; the replay must leave exactly the state and outputs of
+    # the same steps launched directly
+    import torch
+    wl = W.parity_instance(2)
+    s = wl.shape
+    n, T = 6, 24
+    cfg = dict(n_pages=wl.n_pages, max_pages_per_req=wl.max_pages_per_req, max_requests=8, k_loc=wl.k_loc)
+    q = np.empty((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=np.uint16)
+    k = np.empty((T, s.n_layers, n, s.n_kv_heads, s.head_dim), dtype=np.uint16)
+    v = np.empty_like(k)
+    prompts = []
+    for i in range(n):
+        st = wl.stream(wl.requests[i])
+        prompts.append(st.prompt_kv())
+        q[:, :, i], k[:, :, i], v[:, :, i] = st.steps(0, T)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).to("cuda:0")
+    qd, kd, vd = dev(q), dev(k), dev(v)
+    ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+    results = []
+    for use_graph in (False, True):
+        pool = B.Pool(B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, tau=-0.05, **cfg))
+        try:
+            for i in range(n):
+                assert pool.request_add(-1, 0, prompts[i][0], prompts[i][1], wl.requests[i].prompt_len, 0)[0] == B.GP_OK
+            outs = torch.zeros((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda:0")
+            acts = torch.zeros((T, n), dtype=torch.int32, device="cuda:0")
+            torch.cuda.synchronize()
+            if use_graph:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for t in range(T):
+                        pool.decode_step(ids, qd[t], kd[t], vd[t], outs[t], acts[t])
+                g.replay()
+            else:
+                for t in range(T):
+                    pool.decode_step(ids, qd[t], kd[t], vd[t], outs[t], acts[t])
+            torch.cuda.synchronize()
+            state = [B.gp_debug_request(pool.handle, i, cfg["max_pages_per_req"])[:3] for i in range(n)]
+            kept = [B.gp_debug_retained(pool.handle, i, 0, 0, state[i][1]) for i in range(n)]
+            assert B.gp_debug_pool(pool.handle)[2][7] == 0
+            results.append((outs.cpu().numpy(), acts.cpu().numpy(), state, kept))
+        finally:
+            pool.close()
+    direct, replay = results
+    assert np.array_equal(direct[1], replay[1]) and direct[2] == replay[2]
+    assert all(np.array_equal(a, b_) for a, b_ in zip(direct[3], replay[3]))
+    assert np.array_equal(direct[0], replay[0])
+    assert (direct[1] != B.GP_ACT_NONE).any()
