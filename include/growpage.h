@@ -50,6 +50,21 @@ extern "C" {
 
 typedef struct gp_pool gp_pool; /* opaque */
 
+/* Capacity-control policies: the default and the controls of the paper's ablation ("Alternative
+ * Capacity-Control Policies", with Eq. 13).  The fixed-budget control needs no policy of its own: a
+ * threshold tau that Delta_t never exceeds (Delta_t <= 1) with initial_pages = the budget.
+ *   DEMAND   grow iff Delta_t > tau (Sec. 3.2, Eq. 8)
+ *   INVERSE  the reversed reading of the signal: grow iff Delta_t <= tau
+ *   RANDOM   ignores Delta_t: Compress & Hold with probability p_compress, else grow.  The draw of request
+ *            r whose step processes the token at absolute position pos is
+ *            u = (mix(policy_seed + 0x9E3779B97F4A7C15 * (r + 1) + 0xBF58476D1CE4E5B9 * pos) >> 11) * 2^-53,
+ *            arithmetic modulo 2^64, mix = the SplitMix64 finaliser; compress iff u < p_compress.
+ *            Working sets and Delta_t are still computed and reported.
+ * (The ablation's Shrink policy, which also gives pages back, is not implemented.) */
+#define GP_POLICY_DEMAND   0
+#define GP_POLICY_INVERSE  1
+#define GP_POLICY_RANDOM   2
+
 typedef struct gp_config {
   int32_t n_layers;          /* L                                                                  */
   int32_t n_q_heads;         /* H_q, a multiple of n_kv_heads; group size G = H_q/H_kv <= 8        */
@@ -61,6 +76,8 @@ typedef struct gp_config {
   int32_t recent_window;     /* |R_t| protected tokens; must equal page_size                       */
   int32_t k_loc;             /* block-local retention quota of Eq. 10 (default page_size / 4)      */
   int32_t host_staging;      /* 1: reserve staging so that gp_decode_step_host can be used         */
+  int32_t policy;            /* GP_POLICY_*: how Delta_t becomes an action (default: demand)       */
+  int32_t policy_seed;       /* GP_POLICY_RANDOM: seed of its counter-based draws                  */
   int64_t n_pages;           /* physical pages; one page id covers all layers and KV heads         */
   int64_t max_batch_tokens;  /* bound on the summed sequence lengths of one decode batch, used to
                                 size scratch; 0 = n_pages * page_size                              */
@@ -68,6 +85,7 @@ typedef struct gp_config {
   double  top_p;             /* Eq. 7, default 0.99                                                */
   double  tau;               /* decision threshold, default 0                                      */
   double  rope_theta;        /* RoPE base (rotate-half pairing); 0 = no rotation                   */
+  double  p_compress;        /* GP_POLICY_RANDOM: probability of Compress & Hold, default 0.7      */
 } gp_config;
 
 /* Fills *cfg with the paper's defaults (Sec. 3.2, Sec. 5.1, App. B.2, App. D.1); the geometry

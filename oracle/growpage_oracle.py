@@ -218,6 +218,19 @@ def select_retained(s: np.ndarray, n_blocks: int, b: int, K_t: int, k_loc: int) 
 # =============================================================================
 # the pool and the per-step state machine
 # =============================================================================
+def random_draw(seed: int, req: int, pos: int) -> float:
+    """Uniform draw in [0, 1) of the random capacity-control policy for request `req` at absolute position
+    `pos`: the SplitMix64 finaliser of seed + 0x9E3779B97F4A7C15 (req + 1) + 0xBF58476D1CE4E5B9 pos (mod 2^64),
+    top 53 bits.  The paper only fixes the probability (0.7); the generator is this build's, stated in the
+    C header so that both sides draw the same numbers."""
+    m = (1 << 64) - 1
+    z = (seed + 0x9E3779B97F4A7C15 * (req + 1) + 0xBF58476D1CE4E5B9 * pos) & m
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & m
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & m
+    z ^= z >> 31
+    return (z >> 11) / 9007199254740992.0
+
+
 @dataclasses.dataclass
 class OracleConfig:
     n_layers: int
@@ -235,6 +248,9 @@ class OracleConfig:
     recent_window: int = 16          # equals the page size in this build
     k_loc: int = 4                   # a quarter of a page, the paper's 64 of 256
     rope_theta: float = 0.0
+    policy: int = 0                  # 0 demand (Eq. 8), 1 inverse, 2 random: the ablation's controls (with Eq. 13)
+    policy_seed: int = 0
+    p_compress: float = 0.7
 
 
 class _Request:
@@ -427,6 +443,11 @@ class OraclePool:
         num = int(info.K_s.sum()) - int(info.K_l.sum())
         info.delta = num / float(L * H * n_c)
         info.want_grow = info.delta > c.tau
+        if c.policy == 1:            # inverse: grows when Delta <= tau, compresses when Delta > tau
+            info.want_grow = not info.want_grow
+        elif c.policy == 2:          # random: Compress & Hold with probability p_compress, whatever Delta says
+            info.want_grow = not (random_draw(c.policy_seed, rid, r.pos - 1) < c.p_compress)
+            return info              # no working-set near-tie can change a coin
         # could a +-1 change of near-tied working-set sizes change the decision?
         near = int((info.ws_margin < 1e-6).sum())
         if near:

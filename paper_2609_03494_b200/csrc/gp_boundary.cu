@@ -462,6 +462,16 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       if (nC > 0) {
         delta = (double)((long long)acc.x - (long long)acc.y) / ((double)LH * (double)nC);
         want = delta > p.tau;
+        if (p.policy == 1) {                                  // the reversed reading of the demand signal
+          want = !want;
+        } else if (p.policy == 2) {                           // frequency-matched random control
+          unsigned long long zz = p.policy_seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(r + 1) +
+                                  0xBF58476D1CE4E5B9ull * (unsigned long long)inf.w;
+          zz = (zz ^ (zz >> 30)) * 0xBF58476D1CE4E5B9ull;
+          zz = (zz ^ (zz >> 27)) * 0x94D049BB133111EBull;
+          zz ^= zz >> 31;
+          want = !((double)(zz >> 11) * (1.0 / 9007199254740992.0) < p.p_compress);
+        }
       }
       p.delta[r] = delta;
       s_want[e] = want; s_ksh[e] = acc.z; s_P[e] = Pr; s_req[e] = r; s_bi[e] = inf.x;

@@ -59,6 +59,9 @@ struct GpDev {
   int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;
   long long n_pages, max_batch_tokens;
   double beta_s, beta_l, top_p, tau, rope_theta;
+  int policy;                            // GP_POLICY_* (0 demand, 1 inverse, 2 random)
+  unsigned long long policy_seed;
+  double p_compress;
   unsigned long long p_fix;              // top_p in 2^62 fixed point
   // pool
   __nv_bfloat16* kv;
@@ -84,7 +87,7 @@ struct GpDev {
   int* b_flags;                          // [M] 1 = stepped this step
   int* first_idx;                        // [M] lowest batch index naming a request
   int4* mc_list;                         // [M] split requests: {batch index, first partial, chunks, 0}
-  int4* bnd_info;                        // [M][2] requests at a boundary: {slot in the batch, request, P, 0}, {score offset lo, hi, 0, 0}
+  int4* bnd_info;                        // [M][2] requests at a boundary: {slot in the batch, request, P, position of the step's token}, {score offset lo, hi, 0, 0}
   int* bnd_acc;                          // [M][4] per boundary request: sum of K^S, sum of K^L, shared pages of C, 0
   int* free_peek;                        // [M+1] free_top at plan time, then the top entries of the free list, top first
   int4* cmp_info;                        // [M+1] compressing requests: {request, P, index in bnd_info, first compaction chunk}

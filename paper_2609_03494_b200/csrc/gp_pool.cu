@@ -82,6 +82,8 @@ bool valid_config(const gp_config* c) {
   if (!(c->beta_s >= 0.0 && c->beta_s < 1.0 && c->beta_l >= 0.0 && c->beta_l < 1.0)) return false;
   if (!(c->top_p > 0.0 && c->top_p < 1.0)) return false;
   if (!(c->rope_theta >= 0.0)) return false;
+  if (c->policy < GP_POLICY_DEMAND || c->policy > GP_POLICY_RANDOM) return false;
+  if (!(c->p_compress >= 0.0 && c->p_compress <= 1.0)) return false;
   return true;
 }
 
@@ -379,7 +381,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     p.b_flags[i] = chunks > 0;
     actions[i] = act;
     if (isb) {
-      p.bnd_info[2 * bnd_idx] = make_int4(i, r, Pr, 0);
+      p.bnd_info[2 * bnd_idx] = make_int4(i, r, Pr, (int)pos);     // pos: position of this step's token
       p.bnd_info[2 * bnd_idx + 1] = make_int4((int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32), 0, 0);
       reinterpret_cast<int4*>(p.bnd_acc)[bnd_idx] = make_int4(0, 0, 0, 0);
       if (bnd_idx < free_top0) p.free_peek[1 + bnd_idx] = s_peek[bnd_idx];
@@ -553,6 +555,9 @@ int gp_config_default(gp_config* cfg) {
   cfg->top_p = 0.99;
   cfg->tau = 0.0;
   cfg->rope_theta = 0.0;
+  cfg->policy = GP_POLICY_DEMAND;
+  cfg->policy_seed = 0;
+  cfg->p_compress = 0.7;
   return GP_OK;
 }
 
@@ -592,6 +597,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
   d.z_stride = (L.max_batch_tokens + GP_PAGE - 1) / GP_PAGE * GP_PAGE;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
+  d.policy = cfg->policy; d.policy_seed = (unsigned long long)(unsigned)cfg->policy_seed; d.p_compress = cfg->p_compress;
   d.p_fix = (unsigned long long)llrint(cfg->top_p * 4611686018427387904.0);
   d.kv = reinterpret_cast<__nv_bfloat16*>(base + L.kv);
   d.tok = reinterpret_cast<int*>(base + L.tok);

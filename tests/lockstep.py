@@ -50,7 +50,8 @@ def make_pools(wl: W.Workload, device: int = 0, **over):
     s = wl.shape
     kw = dict(n_pages=wl.n_pages, max_pages_per_req=wl.max_pages_per_req,
               max_requests=max(4, wl.n_resident), k_loc=wl.k_loc)
-    tun = {k: over[k] for k in ("beta_s", "beta_l", "top_p", "tau", "rope_theta") if k in over}
+    tun = {k: over[k] for k in ("beta_s", "beta_l", "top_p", "tau", "rope_theta", "policy", "policy_seed", "p_compress")
+           if k in over}
     for k in ("n_pages", "max_pages_per_req", "k_loc", "max_requests"):
         if k in over:
             kw[k] = over[k]

@@ -47,5 +47,10 @@ def test_config_defaults_and_pool_bytes_need_no_gpu():
 
 
 def test_struct_layout_matches_the_header():
-    # 10 int32, 2 int64, 5 double, no padding surprises
-    assert ctypes.sizeof(B.gp_config) == 10 * 4 + 2 * 8 + 5 * 8
+    # 12 int32, 2 int64, 6 double, no padding surprises; and the same field order as the header's struct
+    assert ctypes.sizeof(B.gp_config) == 12 * 4 + 2 * 8 + 6 * 8
+    header = open(os.path.join(ROOT, "include", "growpage.h")).read()
+    body = header[header.index("typedef struct gp_config {"):header.index("} gp_config;")]
+    names = re.findall(r"^\s*(?:int32_t|int64_t|double)\s+([a-z_, ]+);", body, flags=re.M)
+    flat = [n.strip() for group in names for n in group.split(",")]
+    assert flat == [f[0] for f in B.gp_config._fields_]

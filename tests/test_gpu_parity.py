@@ -237,3 +237,18 @@ def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches():
     assert all(np.array_equal(a, b_) for a, b_ in zip(direct[3], replay[3]))
     assert np.array_equal(direct[0], replay[0])
     assert (direct[1] != B.GP_ACT_NONE).any()
+
+
+@pytest.mark.parametrize("over", [dict(policy=B.GP_POLICY_INVERSE), dict(policy=B.GP_POLICY_INVERSE, tau=-0.05),
+                                  dict(policy=B.GP_POLICY_RANDOM, policy_seed=7),
+                                  dict(policy=B.GP_POLICY_RANDOM, policy_seed=11, p_compress=0.3)])
+def test_inverse_and_random_capacity_control_policies(over):
+    # the controls of the paper's policy ablation: the reversed reading of Delta and a coin with P(compress) = p
+    st = LS.run_lockstep(W.parity_instance(1), **over)
+    _report(f"tiny {over}", st)
+    grows = st.actions.get(B.GP_ACT_GROW, 0) + st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0)
+    comps = st.actions.get(B.GP_ACT_COMPRESS, 0)
+    assert grows > 0 and comps + st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) > 0
+    if over["policy"] == B.GP_POLICY_RANDOM:
+        frac = comps / max(grows + comps, 1)
+        assert abs(frac - over.get("p_compress", 0.7)) < 0.25

@@ -479,3 +479,48 @@ def test_retained_output_error_respects_the_worst_case_bound():
     o_hat, m = O.subset_output(a_s, V_c, S)
     v_max = np.linalg.norm(V_c, axis=1).max()
     assert np.linalg.norm(a_s @ V_c - o_hat) <= 2 * v_max * (1 - m) + 1e-12
+
+
+def test_random_policy_draws_are_splitmix64_and_uniform():
+    # golden: the first two outputs of SplitMix64 seeded with 0 (published with the generator) are what the
+    # draw's mixing function gives for (seed 0, request 0, position 0) and (seed 0, request 1, position 0)
+    assert O.random_draw(0, 0, 0) == (0xE220A8397B1DCDAF >> 11) / 2.0 ** 53
+    assert O.random_draw(0, 1, 0) == (0x6E789E6AA1B965F4 >> 11) / 2.0 ** 53
+    u = np.array([O.random_draw(9, r, p) for r in range(40) for p in range(250)])
+    assert 0.0 <= u.min() and u.max() < 1.0
+    assert abs(u.mean() - 0.5) < 4 * (1 / 12) ** 0.5 / len(u) ** 0.5
+    assert abs((u < 0.7).mean() - 0.7) < 4 * (0.21 / len(u)) ** 0.5
+    # position and request both matter
+    assert len({O.random_draw(9, 3, p) for p in range(100)}) == 100
+    assert len({O.random_draw(9, r, 5) for r in range(100)}) == 100
+
+
+def test_inverse_and_random_policies_only_change_the_decision():
+    # same request, same inputs: the three policies see the same Delta at the first boundary that has history
+    # (the one after 16 more steps; the very first has S == L) and turn it into their own action
+    outs = {}
+    for policy, kw in ((0, {}), (1, {}), (2, dict(p_compress=1.0)), (3, dict(p_compress=0.0))):
+        c = _cfg(n_pages=16, max_pages_per_req=8)
+        c.policy = min(policy, 2)
+        for k_, v_ in kw.items():
+            setattr(c, k_, v_)
+        pool = O.OraclePool(c)
+        g = np.random.default_rng(3)
+        kt = g.standard_normal((c.n_layers, 20, c.n_kv_heads, c.head_dim))
+        _, rid = pool.request_add(-1, 0, kt, kt.copy(), 20, 0)
+        acts, deltas = [], []
+        for t in range(12):
+            shp_q = (c.n_layers, 1, c.n_q_heads, c.head_dim)
+            shp_k = (c.n_layers, 1, c.n_kv_heads, c.head_dim)
+            rec = pool.decode_step([rid], g.standard_normal(shp_q), g.standard_normal(shp_k), g.standard_normal(shp_k))
+            if rid in rec.boundary:
+                acts.append(int(rec.actions[0]))
+                deltas.append(rec.boundary[rid].delta)
+                break
+        outs[policy] = (acts, deltas)
+    assert outs[0][1] == outs[1][1] == outs[2][1] == outs[3][1]          # same Delta, whatever the policy
+    d = outs[0][1][0]
+    assert outs[0][0][0] == (O.ACT_GROW if d > 0 else O.ACT_COMPRESS)
+    assert outs[1][0][0] == (O.ACT_COMPRESS if d > 0 else O.ACT_GROW)
+    assert outs[2][0][0] == O.ACT_COMPRESS                               # p_compress = 1: always Compress & Hold
+    assert outs[3][0][0] == O.ACT_GROW                                   # p_compress = 0: always grows
