@@ -124,8 +124,10 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
  *                the new one included; rows of requests whose action is GP_ACT_INVALID, or that
  *                were already full on entry, are not written
  *   dev_actions  device int32 [n_req]: GP_ACT_* per request
- * Asynchronous on `stream`; nothing is read back to the host.  Steps of one pool must be
- * issued on one stream (or otherwise serialised): they share scratch inside the blob. */
+ * Asynchronous on `stream`; nothing is read back to the host, so (with profiling off) a sequence of
+ * steps can be captured into a CUDA graph and replayed.  The step's kernels are chained with
+ * programmatic dependent launch.  Steps of one pool must be issued on one stream (or otherwise
+ * serialised): they share scratch inside the blob. */
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
                    const void* q, const void* k, const void* v,
                    void* out, int32_t* dev_actions, void* stream);
