@@ -36,7 +36,7 @@ namespace {
 constexpr int NI_MAX = 8;                  // item slots per CTA (4 when the group is 8 heads wide)
 constexpr int NSW = 2;                     // tile stages per consumer warp (at most 3: see the wait in the tile loop)
 constexpr int NCW = 4;                     // consumer warps
-constexpr int NTHREADS = 256;              // warp group 0: producer, summaries, merger, spare; warp group 1: consumers
+constexpr int NTHREADS = 256;              // warp group 0: producer, idle, merger, idle; warp group 1: consumers
 constexpr int REGS_SERVICE = 56;           // registers per thread after the split (setmaxnreg)
 constexpr int REGS_CONSUMER = 200;
 constexpr int QT_PAD = 8;                  // doubles of padding per q~ row: rows alternate bank halves
@@ -149,15 +149,11 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     // C = page ids here: written to the slot, which completes its `full` barrier (two arrivals: B and C, plus
     // the bytes of B's copies).  The ring of slots paces the producer: it runs NI items ahead at most.
     const long long grid = gridDim.x;
-    // static schedule: items are sorted by descending cost; round k goes to the CTAs in alternating order.
-    // A CTA takes its second item first: the costliest items are those of boundary requests, whose
-    // calibrated summaries the summary warps then prepare while the consumers are busy with another item.
-    auto item_of_round = [&](long long kk) -> long long {
+    // static schedule: items are sorted by descending cost; round k goes to the CTAs in alternating order
+    auto item_of_tick = [&](long long kk) -> long long {
       const long long item = kk * grid + ((kk & 1) ? grid - 1 - (long long)blockIdx.x : (long long)blockIdx.x);
       return item < total ? item : total;
     };
-    const bool swap01 = item_of_round(1) < total;
-    auto item_of_tick = [&](long long t) -> long long { return item_of_round(swap01 && t < 2 ? 1 - t : t); };
     long long itA = item_of_tick(0), itB = total, itC = total;
     int hB = 0, hC = 0;                        // descriptor header, word `lane` (lanes 0..15)
     int pC = -1;                               // page id of tile `lane` of the item
