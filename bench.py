@@ -160,6 +160,7 @@ class Job:
         self.out_host = torch.zeros((s.n_layers, self.nreq, s.n_q_heads, s.head_dim), dtype=torch.float32).pin_memory()
         self.act_host = torch.zeros(self.nreq, dtype=torch.int32).pin_memory()
         self.live = False
+        self.by_layer = False           # True: steps go through gp_step_begin / gp_attn_layer / gp_step_end
         self.reset()
 
     def reset(self):
@@ -177,8 +178,8 @@ class Job:
         self.t = 0
 
     def step(self):
-        self.pool.decode_step(self.ids_dev, self.q_dev[self.t], self.k_dev[self.t], self.v_dev[self.t], self.out_dev,
-                              self.act_dev)
+        f = self.pool.decode_step_layers if self.by_layer else self.pool.decode_step
+        f(self.ids_dev, self.q_dev[self.t], self.k_dev[self.t], self.v_dev[self.t], self.out_dev, self.act_dev)
         self.t += 1
 
     def step_host(self):
@@ -233,6 +234,7 @@ def run_ours(args):
     q_all, k_all, v_all, prompts = generate_inputs(wl, S0 + K, torch, pin=True)
     t_gen = time.time() - t_gen
     job = Job(wl, torch, device, q_all, k_all, v_all, prompts)
+    job.by_layer = args.entry == "layers"
     B = job.B
     stream = torch.cuda.current_stream(device)
 
@@ -270,6 +272,7 @@ def run_ours(args):
     job.roll(S0)
     torch.cuda.synchronize(device)
     moved0 = job.moved_rows()
+    by_layer, job.by_layer = job.by_layer, False        # per-kernel times come from the whole-step entry (same kernels)
     B.gp_set_profiling(job.pool.handle, True)
     attn_bytes = score_bytes = 0.0
     n_sum = 0
@@ -282,6 +285,7 @@ def run_ours(args):
         n_sum += int(job.n.sum())
     kms, kn = B.gp_get_kernel_times(job.pool.handle)
     B.gp_set_profiling(job.pool.handle, False)
+    job.by_layer = by_layer
     moved = job.moved_rows() - moved0
     compact_bytes = 2.0 * moved * (2 * s.head_dim * 2 + 4)
     summ_bytes = float(K) * job.nreq * s.n_layers * 2 * s.n_q_heads * s.head_dim * 8 * 2      # both views, read + write, fp64
@@ -340,6 +344,7 @@ def run_ours(args):
                                     "workload)") if stack else
                                    ("qwen3-8b-layer: L=1, 32q/8kv heads, d=128, page 16, 64 requests x 4096 decode steps, "
                                     "prompts U[128,1024], heavy-hitter fraction logU[0.5%,20%], seed 1"),
+                       "entry": "gp_decode_step" if not job.by_layer else "gp_step_begin + gp_attn_layer per layer + gp_step_end",
                        "requests_per_gpu": job.nreq, "timed_steps": [S0, S0 + K], "job_steps": job_steps,
                        "l2": "per-step working set (all resident K/V) is larger than L2; no flush needed",
                        "input_generation_s": round(t_gen, 1)},
@@ -432,6 +437,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--entry", default="step", choices=["step", "layers"],
+                    help="step: gp_decode_step; layers: the same step through gp_step_begin / gp_attn_layer / gp_step_end")
     ap.add_argument("--workload", default="layer", choices=["layer", "stack"],
                     help="layer: the headline one-layer Qwen3-8B-shaped workload; stack: the 36-layer shape, 16 resident requests")
     args = ap.parse_args()

@@ -132,6 +132,24 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
                    const void* q, const void* k, const void* v,
                    void* out, int32_t* dev_actions, void* stream);
 
+/* The same step, layer by layer, for a model's forward pass, where layer l + 1's query exists only after
+ * layer l's attention output (the paper's setting: attention and the summary update run inside every
+ * layer, the capacity decision once per step, Sec. 3.2, Sec. 4.1):
+ *   gp_step_begin   validates the batch and plans the step (what gp_decode_step does first);
+ *   gp_attn_layer   for one layer: append, attention, summary update and, for requests at their
+ *                   boundary, the summary logits; q [n_req][H_q][d], k, v [n_req][H_kv][d] bf16 and
+ *                   out [n_req][H_q][d] fp32 are this layer's tensors (device pointers); when the call's
+ *                   work has run, `out` is complete.  Every layer exactly once, in any order;
+ *   gp_step_end     working sets, decisions, allocation, compaction; writes `dev_actions`.
+ * Same ids, n_req and stream discipline as gp_decode_step; between gp_step_begin and gp_step_end no other
+ * step of the pool may be issued (GP_ERR_STATE).  The results equal gp_decode_step's bit for bit. */
+int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions,
+                  void* stream);
+int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req,
+                  const void* q, const void* k, const void* v, void* out, void* stream);
+int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions,
+                void* stream);
+
 /* As gp_decode_step with HOST pointers: copies the inputs to staging inside the blob, runs the
  * step, delivers `out` and `actions` and synchronises `stream`.  When `out` and `actions` are
  * page-locked, mapped host memory (cudaHostAlloc / cudaHostRegister: "pinned"), the kernels write

@@ -63,6 +63,9 @@ def lib() -> C.CDLL:
     L.gp_debug_summaries.argtypes = [vp, i32, vp]
     L.gp_debug_boundary.argtypes = [vp, i32, vp, vp, C.POINTER(C.c_double)]
     L.gp_debug_pool.argtypes = [vp, C.POINTER(i64), vp, vp]
+    L.gp_step_begin.argtypes = [vp, vp, i32, vp, vp]
+    L.gp_attn_layer.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
+    L.gp_step_end.argtypes = [vp, vp, i32, vp, vp]
     L.gp_set_profiling.argtypes = [vp, i32]
     L.gp_get_kernel_times.argtypes = [vp, vp, vp]
     L.gp_launch_count.argtypes = [vp]; L.gp_launch_count.restype = i64
@@ -126,6 +129,23 @@ def gp_decode_step_host(pool: int, host_req_ids_ptr: int, n_req: int, q_ptr: int
     _check(lib().gp_decode_step_host(C.c_void_p(pool), C.c_void_p(host_req_ids_ptr), n_req, C.c_void_p(q_ptr),
                                      C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr),
                                      C.c_void_p(actions_ptr), C.c_void_p(stream)), "gp_decode_step_host")
+
+
+def gp_step_begin(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: int, stream: int) -> None:
+    _check(lib().gp_step_begin(C.c_void_p(pool), C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(dev_actions_ptr),
+                               C.c_void_p(stream)), "gp_step_begin")
+
+
+def gp_attn_layer(pool: int, layer: int, dev_req_ids_ptr: int, n_req: int, q_ptr: int, k_ptr: int, v_ptr: int,
+                  out_ptr: int, stream: int) -> None:
+    _check(lib().gp_attn_layer(C.c_void_p(pool), layer, C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(q_ptr),
+                               C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr), C.c_void_p(stream)),
+           "gp_attn_layer")
+
+
+def gp_step_end(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: int, stream: int) -> None:
+    _check(lib().gp_step_end(C.c_void_p(pool), C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(dev_actions_ptr),
+                             C.c_void_p(stream)), "gp_step_end")
 
 
 def gp_release(pool: int, req: int, stream: int) -> None:
@@ -249,6 +269,16 @@ class Pool:
         actions int32 [B]."""
         gp_decode_step(self.handle, req_ids.data_ptr(), int(req_ids.numel()), q.data_ptr(), k.data_ptr(),
                        v.data_ptr(), out.data_ptr(), actions.data_ptr(), self.stream())
+
+    def decode_step_layers(self, req_ids, q, k, v, out, actions) -> None:
+        """The same step through the per-layer entry points: q, k, v, out as for decode_step ([L][...]); every
+        layer's slice is passed to gp_attn_layer on its own."""
+        n = int(req_ids.numel())
+        gp_step_begin(self.handle, req_ids.data_ptr(), n, actions.data_ptr(), self.stream())
+        for layer in range(q.shape[0]):
+            gp_attn_layer(self.handle, layer, req_ids.data_ptr(), n, q[layer].data_ptr(), k[layer].data_ptr(),
+                          v[layer].data_ptr(), out[layer].data_ptr(), self.stream())
+        gp_step_end(self.handle, req_ids.data_ptr(), n, actions.data_ptr(), self.stream())
 
     def decode_step_host(self, req_ids, q, k, v, out, actions) -> None:
         """All arguments are host tensors (pinned recommended)."""

@@ -95,7 +95,9 @@ __device__ __forceinline__ void dmma(double& d0, double& d1, double a, double b)
 template <int D, bool ROPE>
 __global__ void __launch_bounds__(NTHREADS, 2)
 gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* __restrict__ q,
-               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, float* __restrict__ out) {
+               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, float* __restrict__ out, int lh0,
+               int lh_n) {
+  // lh0, lh_n: the (layer, KV head) units this launch covers, [lh0, lh0 + lh_n): all of them, or one layer's
   using GEO = Geo<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
@@ -133,7 +135,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
 
   const int n_rc = p.hdr[HDR_N_RC];
   const int LH = p.L * p.Hkv;
-  const long long total = (long long)n_rc * LH;
+  const long long total = (long long)n_rc * lh_n;
   const int q_bytes = G * GEO::ROW_BYTES;
 
   if (warp < 4) {
@@ -192,7 +194,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     for (uint32_t tick = 0;; ++tick) {
       // ---- issue the loads of the young stages --------------------------------------------------
       int hNew = 0;
-      if (itA < total && lane < GP_DESC_INTS) hNew = p.rcx[(size_t)(itA / LH) * GP_DESC_INTS + lane];
+      if (itA < total && lane < GP_DESC_INTS) hNew = p.rcx[(size_t)(itA / lh_n) * GP_DESC_INTS + lane];
       int pNew = -1;
       int slNew = 0;
       // ---- page ids of stage C have arrived: into the slot, which is then complete ----------------------
@@ -219,7 +221,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           if (lane == 0) { mbar_arrive(&slot_full[sl]); mbar_arrive(&slot_full[sl]); }
           sentinel_out = true;
         } else {
-          const int lh = (int)(itB % LH);
+          const int lh = lh0 + (int)(itB % lh_n);
           const int l = lh / p.Hkv, h = lh % p.Hkv;
           const int bi = __shfl_sync(0xffffffffu, hB, 0);
           const int r = __shfl_sync(0xffffffffu, hB, 1), pg0 = __shfl_sync(0xffffffffu, hB, 2);
@@ -682,7 +684,7 @@ void gp_attention_setup(const GpDev& p) {           // once per pool: opt into t
 }
 
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s, bool pdl) {
+                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n) {
   (void)req_ids;
   const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kk = static_cast<const __nv_bfloat16*>(k);
@@ -692,7 +694,7 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
 #define GP_LAUNCH(DD, RR)                                                                 \
   do {                                                                                    \
     auto kern = gp_attn_kernel<DD, RR>;                                                   \
-    gp_launch(kern, grid, NTHREADS, (size_t)sm, s, pdl, p, n_req, qq, kk, vv, out);       \
+    gp_launch(kern, grid, NTHREADS, (size_t)sm, s, pdl, p, n_req, qq, kk, vv, out, lh0, lh_n); \
   } while (0)
   if (p.d == 128) {
     if (rope) GP_LAUNCH(128, true); else GP_LAUNCH(128, false);

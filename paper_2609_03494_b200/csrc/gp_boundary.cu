@@ -748,16 +748,16 @@ __device__ __noinline__ bool job_softmax(const GpDev& p, const double* __restric
 // (running maximum in the log2 domain, sum of exponentials, unnormalised output) into the output row.  The
 // calling CTA takes merges first, first + stride, ...
 __device__ __noinline__ void merge_partials(const GpDev& p, int n_req, float* __restrict__ out, int n_mc, int n_rc,
-                                            int first_item, int stride) {
-  const int LH = p.L * p.Hkv, G = p.G, D = p.d;
+                                            int first_item, int stride, int lh0, int lh_n) {
+  const int G = p.G, D = p.d;
   const int PSTRIDE = G * (D + 2);
-  for (long long mi = first_item; mi < (long long)n_mc * LH; mi += stride) {
-    const int4 mc = p.mc_list[mi / LH];
-    const int lh = (int)(mi % LH), l = lh / p.Hkv, h = lh % p.Hkv;
+  for (long long mi = first_item; mi < (long long)n_mc * lh_n; mi += stride) {       // units [lh0, lh0 + lh_n)
+    const int4 mc = p.mc_list[mi / lh_n];
+    const int lh = lh0 + (int)(mi % lh_n), l = lh / p.Hkv, h = lh % p.Hkv;
     const int bi = mc.x, nch = mc.z;
     const float* first = p.partials + ((size_t)lh * n_rc + mc.y) * PSTRIDE;
     float* orow = out + (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
-    for (int idx = threadIdx.x; idx < G * D; idx += SEL_T) {
+    for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) {
       const int g = idx / D, dc = idx % D;
       const float* pg = first + g * (D + 2);
       float M = -INFINITY, acc = 0.f, ls = 0.f;
@@ -836,7 +836,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     if (b0 < p.M) { inf_first = p.bnd_info[2 * b0]; inf2_first = p.bnd_info[2 * b0 + 1]; }
   }
   const int n_bnd = p.hdr[HDR_N_BND];
-  const int n_mc = p.hdr[HDR_N_MC], n_rc = p.hdr[HDR_N_RC];
+  const int n_mc = out ? p.hdr[HDR_N_MC] : 0, n_rc = p.hdr[HDR_N_RC];   // out == null: already merged layer by layer
   const long long items = (long long)n_bnd * LH * 3;
   if (tid == 0) GP_T_STAMP(59);
 
@@ -846,7 +846,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const int n_idle = (int)gridDim.x - (int)n_busy;
   const bool idle_merge = n_idle * 4 >= (int)gridDim.x;
   if (idle_merge && (long long)blockIdx.x >= n_busy)
-    merge_partials(p, n_req, out, n_mc, n_rc, (int)blockIdx.x - (int)n_busy, n_idle);
+    merge_partials(p, n_req, out, n_mc, n_rc, (int)blockIdx.x - (int)n_busy, n_idle, 0, LH);
 
   if (tid == 0) GP_T_STAMP(60);
   for (long long item = blockIdx.x; item < items + n_bnd; item += gridDim.x) {
@@ -967,7 +967,16 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     if (tid == 0) { GP_T_ADD(23, GP_T_NOW() - t_d0); GP_T_ADD(24, 1); }
   }
 
-  if (!idle_merge) merge_partials(p, n_req, out, n_mc, n_rc, (int)gridDim.x - 1 - (int)blockIdx.x, (int)gridDim.x);
+  if (!idle_merge) merge_partials(p, n_req, out, n_mc, n_rc, (int)gridDim.x - 1 - (int)blockIdx.x, (int)gridDim.x, 0, LH);
+}
+
+// merges the partial outputs of the split requests for the units [lh0, lh0 + lh_n): the per-layer entry point
+// needs a layer's output complete before the next layer's query exists
+__global__ void __launch_bounds__(256)
+gp_merge_kernel(const __grid_constant__ GpDev p, int n_req, float* __restrict__ out, int lh0, int lh_n) {
+  gp_pdl_wait();
+  gp_pdl_launch_dependents();
+  merge_partials(p, n_req, out, p.hdr[HDR_N_MC], p.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, lh0, lh_n);
 }
 
 // ------------------------------------------------------------------------------------------------------
@@ -1177,6 +1186,10 @@ void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_com
   if (p.d == 128) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_compact_kernel<128>, CT, 0);
   else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_compact_kernel<64>, CT, 0);
   *grid_compact = num_sms * (occ > 0 ? occ : 1);
+}
+
+void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl) {
+  gp_launch(gp_merge_kernel, grid, 256, 0, s, pdl, p, n_req, out, lh0, lh_n);
 }
 
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,

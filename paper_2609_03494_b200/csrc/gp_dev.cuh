@@ -229,7 +229,7 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 
 // ---- host-visible launchers (one per translation unit) -------------------------------------------
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s, bool pdl);
+                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n);
 size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
 // ---- programmatic dependent launch -------------------------------------------------------------------
@@ -257,6 +257,8 @@ inline cudaError_t gp_launch(void (*kern)(KArgs...), int grid, int block, size_t
 #endif
 
 void gp_attention_setup(const GpDev& p);
+// merge of the split requests' partial outputs for the units [lh0, lh0 + lh_n) (per-layer entry point)
+void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl);
 void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact);
 // boundary chain: probabilities + working sets + selection + decision, then compaction.
 // `ev`, when not null, is recorded between the two kernels.  `pdl`: launch with programmatic stream serialization.

@@ -21,6 +21,7 @@ struct gp_pool {
   size_t bytes;
   std::vector<uint8_t> live;      // host mirror of the slot free list
   int num_sms, attn_grid, sel_grid, compact_grid;
+  int step_open, step_n_req, step_layers_done;      // per-layer entry points: a step begun and not yet ended
   // staging for the host-pointer entry point (inside the blob)
   int* st_ids; void* st_q; void* st_k; void* st_v; float* st_out; int* st_act;
   // small device words
@@ -273,7 +274,9 @@ __device__ void prepare_row(const GpDev& p, const int* __restrict__ req_ids, int
 // step's append (trailing check: n + 1 == P b) and hands each a slice of the logit scratch.
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
-               const __nv_bfloat16* __restrict__ q) {
+               const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n) {
+  // plan_on: CTA 0 plans (off for the per-layer calls after the step's first); the summary CTAs cover the
+  // (layer, KV head) units [lh0, lh0 + lh_n) (none when lh_n is 0: the query rows come layer by layer)
   __shared__ int sv[33];
   __shared__ long long sw[33];
   __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
@@ -285,18 +288,19 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   gp_pdl_wait();
   gp_pdl_launch_dependents();
   if (blockIdx.x > 0) {                       // summary CTAs: one warp per (unit, view, head)
-    const int LH = p.L * p.Hkv;
     const int rows = 2 * p.G, upc = 32 / rows;             // units per CTA and pass
     const int warp = threadIdx.x >> 5;
-    const long long units = (long long)n_req * LH;
+    const long long units = (long long)n_req * lh_n;
     if (warp < upc * rows) {
       for (long long u = ((long long)blockIdx.x - 1) * upc + warp / rows; u < units; u += ((long long)gridDim.x - 1) * upc) {
-        if (p.d == 128) prepare_row<128>(p, req_ids, n_req, q, (int)(u / LH), (int)(u % LH), warp % rows);
-        else prepare_row<64>(p, req_ids, n_req, q, (int)(u / LH), (int)(u % LH), warp % rows);
+        const int bi = (int)(u / lh_n), lh = lh0 + (int)(u % lh_n);
+        if (p.d == 128) prepare_row<128>(p, req_ids, n_req, q, bi, lh, warp % rows);
+        else prepare_row<64>(p, req_ids, n_req, q, bi, lh, warp % rows);
       }
     }
     return;
   }
+  if (!plan_on) return;
   const int free_top0 = *p.free_top;
   const long long t_plan0 = GP_T_NOW();
   (void)t_plan0;
@@ -581,6 +585,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   pool->bytes = bytes;
   pool->live.assign(cfg->max_requests, 0);
   pool->profiling = 0;
+  pool->step_open = 0; pool->step_n_req = 0; pool->step_layers_done = 0;
   pool->launch_count = 0;
   memset(pool->ms, 0, sizeof(pool->ms));
   memset(pool->launches, 0, sizeof(pool->launches));
@@ -713,28 +718,34 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   return GP_OK;
 }
 
+// CTA 0 plans (when plan_on); the others update the query summaries of the units [lh0, lh0 + lh_n)
+static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_t* actions, const void* q, int plan_on,
+                        int lh0, int lh_n, cudaStream_t s, bool pdl) {
+  const GpDev& d = pool->dev;
+  const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
+  const long long want = ((long long)n_req * lh_n + upc - 1) / upc;
+  const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
+  const int prep = (int)(want < room ? want : room);
+  gp_launch(gp_plan_kernel, 1 + prep, GP_PLAN_THREADS, 0, s, pdl, d, ids, n_req, actions,
+            static_cast<const __nv_bfloat16*>(q), plan_on, lh0, lh_n);
+}
+
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
                    const void* v, void* out, int32_t* dev_actions, void* stream) {
   if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
+  if (pool->step_open) return GP_ERR_STATE;
   if (n_req == 0) return GP_OK;
   if (!dev_req_ids || !q || !k || !v || !out || !dev_actions) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const GpDev& d = pool->dev;
+  const int LH = d.L * d.Hkv;
   const bool prof = pool->profiling != 0;
   if (prof) cudaEventRecord(pool->ev[0], s);
   const bool pdl = !prof;                      // events between the kernels need them serialised the plain way
-  {
-    // CTA 0 plans; the others update the query summaries of the batch, one (request, layer, KV head) at a time
-    const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
-    const long long want = ((long long)n_req * d.L * d.Hkv + upc - 1) / upc;
-    const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
-    const int prep = (int)(want < room ? want : room);
-    gp_launch(gp_plan_kernel, 1 + prep, GP_PLAN_THREADS, 0, s, pdl, d, dev_req_ids, n_req, dev_actions,
-              static_cast<const __nv_bfloat16*>(q));
-  }
+  launch_plan(pool, dev_req_ids, n_req, dev_actions, q, 1, 0, LH, s, pdl);
   if (prof) cudaEventRecord(pool->ev[1], s);
-  gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl);
+  gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH);
   if (prof) cudaEventRecord(pool->ev[2], s);
   gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s,
                      prof ? pool->ev[3] : nullptr, pdl);
@@ -750,6 +761,60 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
       pool->launches[i] += 1;
     }
   }
+  return GP_OK;
+}
+
+// ---- the same step, layer by layer: a model's forward pass has layer l + 1's query only after layer l's
+// attention output ---------------------------------------------------------------------------------------
+int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions, void* stream) {
+  if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
+  if (pool->step_open) return GP_ERR_STATE;
+  if (n_req == 0) return GP_OK;
+  if (!dev_req_ids || !dev_actions) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  launch_plan(pool, dev_req_ids, n_req, dev_actions, nullptr, 1, 0, 0, static_cast<cudaStream_t>(stream), true);
+  pool->launch_count += 1;
+  pool->step_open = 1;
+  pool->step_n_req = n_req;
+  pool->step_layers_done = 0;
+  GP_CUDA(cudaGetLastError());
+  return GP_OK;
+}
+
+int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
+                  const void* v, void* out, void* stream) {
+  if (!pool || !pool->step_open || n_req != pool->step_n_req) return pool && !pool->step_open ? GP_ERR_STATE : GP_ERR_INVALID;
+  if (layer < 0 || layer >= pool->cfg.n_layers || !dev_req_ids || !q || !k || !v || !out) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const GpDev& d = pool->dev;
+  // The kernels index their per-step tensors as [layer][request][head][d]: a layer's own tensors are handed over
+  // as the base such an array would have (the kernels only touch this layer's part of it).
+  const size_t qs = (size_t)layer * n_req * d.Hq * d.d, ks = (size_t)layer * n_req * d.Hkv * d.d;
+  const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(reinterpret_cast<uintptr_t>(q) - qs * 2);
+  const __nv_bfloat16* kb = reinterpret_cast<const __nv_bfloat16*>(reinterpret_cast<uintptr_t>(k) - ks * 2);
+  const __nv_bfloat16* vb = reinterpret_cast<const __nv_bfloat16*>(reinterpret_cast<uintptr_t>(v) - ks * 2);
+  float* ob = reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(out) - qs * 4);
+  const int lh0 = layer * d.Hkv, lh_n = d.Hkv;
+  launch_plan(pool, dev_req_ids, n_req, nullptr, qb, 0, lh0, lh_n, s, true);
+  gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n);
+  gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
+  pool->launch_count += 3;
+  pool->step_layers_done += 1;
+  GP_CUDA(cudaGetLastError());
+  return GP_OK;
+}
+
+int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions, void* stream) {
+  if (!pool || !pool->step_open) return pool ? GP_ERR_STATE : GP_ERR_INVALID;
+  if (n_req != pool->step_n_req || !dev_req_ids || !dev_actions) return GP_ERR_INVALID;
+  if (pool->step_layers_done != pool->cfg.n_layers) return GP_ERR_STATE;       // every layer exactly once
+  GP_CUDA(cudaSetDevice(pool->device));
+  gp_launch_boundary(pool->dev, dev_req_ids, n_req, dev_actions, nullptr, pool->sel_grid, pool->compact_grid,
+                     static_cast<cudaStream_t>(stream), nullptr, true);
+  pool->launch_count += 2;
+  pool->step_open = 0;
+  GP_CUDA(cudaGetLastError());
   return GP_OK;
 }
 

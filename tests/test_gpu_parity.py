@@ -252,3 +252,67 @@ def test_inverse_and_random_capacity_control_policies(over):
     if over["policy"] == B.GP_POLICY_RANDOM:
         frac = comps / max(grows + comps, 1)
         assert abs(frac - over.get("p_compress", 0.7)) < 0.25
+
+
+def test_layer_by_layer_entry_points_equal_the_whole_step():
+    # gp_step_begin / gp_attn_layer (layers in a shuffled order) / gp_step_end against gp_decode_step on the same
+    # inputs: outputs, actions, page state, retained sets and summaries bit for bit; and the state checks
+    import torch
+    shape = W.Shape(5, 8, 2, 64)
+    reqs = [W.RequestSpec(i, 150 + 37 * i, 60, 0.05) for i in range(6)]
+    wl = W.Workload("layers", 31, shape, reqs, n_resident=6, initial_pages=0, max_pages_per_req=48, n_pages=6 * 48)
+    s, n, T = shape, 6, 60
+    q = np.empty((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=np.uint16)
+    k = np.empty((T, s.n_layers, n, s.n_kv_heads, s.head_dim), dtype=np.uint16)
+    v = np.empty_like(k)
+    prompts = []
+    for i in range(n):
+        st = wl.stream(reqs[i])
+        prompts.append(st.prompt_kv())
+        q[:, :, i], k[:, :, i], v[:, :, i] = st.steps(0, T)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).to("cuda:0")
+    qd, kd, vd = dev(q), dev(k), dev(v)
+    ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+    rng = np.random.default_rng(0)
+    results = []
+    for by_layer in (False, True):
+        pool = B.Pool(B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
+                                    max_pages_per_req=48, max_requests=8, tau=-0.05))
+        try:
+            for i in range(n):
+                assert pool.request_add(-1, 0, prompts[i][0], prompts[i][1], reqs[i].prompt_len, 0)[0] == B.GP_OK
+            outs = torch.zeros((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda:0")
+            acts = torch.zeros((T, n), dtype=torch.int32, device="cuda:0")
+            if by_layer:
+                h, strm = pool.handle, pool.stream()
+                with pytest.raises(B.GpError):                       # no step begun
+                    B.gp_step_end(h, ids.data_ptr(), n, acts[0].data_ptr(), strm)
+                for t in range(T):
+                    B.gp_step_begin(h, ids.data_ptr(), n, acts[t].data_ptr(), strm)
+                    if t == 0:
+                        with pytest.raises(B.GpError):               # a step is open
+                            pool.decode_step(ids, qd[t], kd[t], vd[t], outs[t], acts[t])
+                        with pytest.raises(B.GpError):               # not every layer done yet
+                            B.gp_step_end(h, ids.data_ptr(), n, acts[t].data_ptr(), strm)
+                    for layer in rng.permutation(s.n_layers):
+                        layer = int(layer)
+                        B.gp_attn_layer(h, layer, ids.data_ptr(), n, qd[t, layer].data_ptr(), kd[t, layer].data_ptr(),
+                                        vd[t, layer].data_ptr(), outs[t, layer].data_ptr(), strm)
+                    B.gp_step_end(h, ids.data_ptr(), n, acts[t].data_ptr(), strm)
+            else:
+                for t in range(T):
+                    pool.decode_step(ids, qd[t], kd[t], vd[t], outs[t], acts[t])
+            torch.cuda.synchronize()
+            state = [B.gp_debug_request(pool.handle, i, 48)[:3] for i in range(n)]
+            kept = [B.gp_debug_retained(pool.handle, i, s.n_layers - 1, 1, state[i][1]) for i in range(n)]
+            summ = [B.gp_debug_summaries(pool.handle, i, s.n_layers, s.n_q_heads, s.head_dim) for i in range(n)]
+            assert B.gp_debug_pool(pool.handle)[2][7] == 0
+            results.append((outs.cpu().numpy(), acts.cpu().numpy(), state, kept, summ))
+        finally:
+            pool.close()
+    whole, layered = results
+    assert np.array_equal(whole[1], layered[1]) and whole[2] == layered[2]
+    assert all(np.array_equal(a, b_) for a, b_ in zip(whole[3], layered[3]))
+    assert all(np.array_equal(a, b_) for a, b_ in zip(whole[4], layered[4]))
+    assert np.array_equal(whole[0], layered[0])
+    assert (whole[1] == B.GP_ACT_GROW).any() and (whole[1] == B.GP_ACT_COMPRESS).any()
