@@ -11,7 +11,8 @@
 //   warp 0      producer: takes its items (a static deal of the cost-sorted list) and publishes each in a ring
 //               of item slots: descriptor, query rows (and the new key/value row) by bulk copy, page ids.  For
 //               boundary items it also brings q~ into the CTA's single q~ buffer.
-//   warps 4..7  consumers: take the tiles of an item round-robin (tile j belongs to warp j mod 4).  Each warp
+//   warps 4..7  consumers: take the tiles of an item round-robin (tile j belongs to warp (j - item number) mod 4,
+//               so the odd tiles of successive items fall on different warps).  Each warp
 //               fetches its own K|V tiles (one contiguous 8 KB per (layer, page, head)) with 16-byte
 //               asynchronous copies into a private ring of stages, running ahead across item boundaries, so
 //               the ring never drains between items.  The G query heads of the group are rows 0..G-1 of an
@@ -302,7 +303,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           f_npg = fsd[3];
           if (f_npg < 0) { f_done = true; break; }
           f_lh = fsd[14];
-          f_pgl = cw;
+          f_pgl = (cw + f_it) % NCW;                      // the first tile goes to another warp from item to item
           f_have = true;
         }
         if (f_pgl >= f_npg) { ++f_it; f_have = false; continue; }
@@ -394,7 +395,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
 
       if (tr) GP_T_ADD(77, GP_T_NOW() - t_a2);
       long long t_prev = GP_T_NOW(); (void)t_prev;
-      for (int pgl = cw; pgl < npg; pgl += NCW) {
+      for (int pgl = (cw + it) % NCW; pgl < npg; pgl += NCW) {
         const uint32_t st = cw * NSW + (my_tiles % NSW);
         const long long t_b = GP_T_NOW();
         (void)t_b;
@@ -407,7 +408,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         ++my_tiles;
         const long long t_c = GP_T_NOW();
         (void)t_c;
-        if (tr) { GP_T_ADD(1, 1); GP_T_ADD(3, t_c - t_b); if (my_tiles == 1) GP_T_STAMP(66); if (pgl == cw) { GP_T_ADD(71, t_c - t_b); GP_T_ADD(72, 1); } }
+        if (tr) { GP_T_ADD(1, 1); GP_T_ADD(3, t_c - t_b); if (my_tiles == 1) GP_T_STAMP(66); if (pgl < NCW) { GP_T_ADD(71, t_c - t_b); GP_T_ADD(72, 1); } }
         uint8_t* tile = smem + st * GEO::TILE_BYTES;
         const int tok0 = (pg0 + pgl) * GP_PAGE;
         const bool has_new = last_chunk && (pgl == npg - 1);
