@@ -44,8 +44,10 @@ extern "C" {
 #define GP_ACT_STALLED          (-1)  /* full and neither a page nor copy-on-write targets could
                                          be had: page state untouched, the caller should release
                                          (preempt) the request; it is skipped while it stays full */
-#define GP_ACT_SCRATCH          (-2)  /* boundary skipped: scoring scratch exhausted
-                                         (max_batch_tokens too small); handled like a stall       */
+#define GP_ACT_SCRATCH          (-2)  /* the batch exceeds max_batch_tokens: either the request was
+                                         stepped without its boundary (its last page is now full and
+                                         the next step reports it stalled), or it was not stepped at
+                                         all (its state is unchanged)                              */
 #define GP_ACT_INVALID          (-3)  /* id out of range, not live, or repeated in the batch      */
 
 typedef struct gp_pool gp_pool; /* opaque */
@@ -80,7 +82,10 @@ typedef struct gp_config {
   int32_t policy_seed;       /* GP_POLICY_RANDOM: seed of its counter-based draws                  */
   int64_t n_pages;           /* physical pages; one page id covers all layers and KV heads         */
   int64_t max_batch_tokens;  /* bound on the summed sequence lengths of one decode batch, used to
-                                size scratch; 0 = n_pages * page_size                              */
+                                size scratch; 0 = n_pages * page_size, which bounds it only while
+                                no prompt pages are shared (a shared page counts once in the pool
+                                and once per request in a batch).  A batch above the bound is not
+                                an error: requests that do not fit report GP_ACT_SCRATCH          */
   double  beta_s, beta_l;    /* Eq. 6, defaults 0.9 and 0.999                                      */
   double  top_p;             /* Eq. 7, default 0.99                                                */
   double  tau;               /* decision threshold, default 0                                      */

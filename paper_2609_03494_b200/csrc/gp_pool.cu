@@ -346,11 +346,14 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   (void)t_plan1;
   int rc_off, n_rc; long long tok_off, tok_tot;
   plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
-  if (isb && tok_off + nc > p.max_batch_tokens) { isb = 0; act = GP_ACT_SCRATCH; }
-  if (chunks > 0 && rc_off + chunks > p.max_rc) {      // cannot happen when max_batch_tokens is honoured
-    atomicOr(p.err, GP_E_BOUNDS);
-    chunks = 0; isb = 0; act = GP_ACT_SCRATCH;
-  }
+  // A batch whose summed lengths exceed max_batch_tokens (the caller's bound; with shared prompt pages the sum
+  // can exceed what the pool holds) does not fit the scratch: a boundary request whose logits do not fit is
+  // stepped without its boundary, and a request whose work items do not fit is not stepped at all.  The
+  // offsets are then taken again over what is left, so that the item list has no holes.
+  if (isb && tok_off + nc > p.max_batch_tokens) { isb = 0; nc = 0; act = GP_ACT_SCRATCH; }
+  const bool dropped = chunks > 0 && rc_off + chunks > p.max_rc;
+  if (dropped) { chunks = 0; isb = 0; nc = 0; act = GP_ACT_SCRATCH; }
+  if (__syncthreads_or(dropped)) plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
   int bnd_idx, n_bnd, n_active; long long d0, d1;
   plan_scan(isb, chunks > 0, bnd_idx, d0, n_bnd, d1, sv, sw);
   n_active = (int)d1;

@@ -120,6 +120,70 @@ def test_batch_edge_cases_and_host_entry_point():
         pool.close()
 
 
+def test_batch_larger_than_the_scratch_bound_is_reported_per_request():
+    """Twelve requests reach their capacity boundary in the same step, with max_batch_tokens far below their
+    summed lengths: the scoring scratch takes the candidates of two of them and the work-item list takes eleven
+    requests.  Two take their boundary, nine are stepped without it (GP_ACT_SCRATCH, last page full), one is not
+    stepped at all (GP_ACT_SCRATCH, state unchanged); every stepped request's output is its softmax-weighted mean
+    of values, and no error bit is raised."""
+    import torch
+    L, Hq, Hkv, d, b = 1, 8, 2, 64, 16
+    n_req, P0 = 12, 24
+    n0 = P0 * b - 1
+    cfg = B.make_config(L, Hq, Hkv, d, n_pages=n_req * (P0 + 2), max_pages_per_req=P0 + 2, max_requests=n_req,
+                        max_batch_tokens=1024)
+    pool = B.Pool(cfg)
+    try:
+        rng = np.random.default_rng(3)
+        bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+        kp, vp = bits(n_req, L, n0, Hkv, d), bits(n_req, L, n0, Hkv, d)
+        for i in range(n_req):
+            assert pool.request_add(-1, 0, kp[i], vp[i], n0, P0) == (B.GP_OK, i)
+        q, k, v = bits(L, n_req, Hq, d), bits(L, n_req, Hkv, d), bits(L, n_req, Hkv, d)
+        dev = lambda x: torch.from_numpy(x.view(np.int16)).to("cuda:0")
+        ids = torch.arange(n_req, dtype=torch.int32, device="cuda:0")
+        out = torch.zeros((L, n_req, Hq, d), dtype=torch.float32, device="cuda:0")
+        act = torch.zeros(n_req, dtype=torch.int32, device="cuda:0")
+        pool.decode_step(ids, dev(q), dev(k), dev(v), out, act)
+        a = act.cpu().numpy()
+        o = out.cpu().numpy().astype(np.float64)
+        f = W.bf16_bits_to_f64
+        kinds = {"boundary": 0, "stepped": 0, "skipped": 0}
+        for i in range(n_req):
+            P, n, pos, _ = B.gp_debug_request(pool.handle, i, cfg.max_pages_per_req)
+            if a[i] == B.GP_ACT_SCRATCH and n == n0:
+                assert (P, pos) == (P0, n0)
+                kinds["skipped"] += 1
+                continue
+            assert pos == n0 + 1
+            if a[i] == B.GP_ACT_SCRATCH:
+                assert (P, n) == (P0, P0 * b)
+                kinds["stepped"] += 1
+            else:
+                assert a[i] in (B.GP_ACT_GROW, B.GP_ACT_COMPRESS) and (P, n) in ((P0 + 1, n0 + 1), (P0, (P0 - 1) * b))
+                kinds["boundary"] += 1
+            K = np.concatenate([f(kp[i])[0].transpose(1, 0, 2), f(k)[0, i][:, None, :]], axis=1)   # [Hkv][n][d]
+            V = np.concatenate([f(vp[i])[0].transpose(1, 0, 2), f(v)[0, i][:, None, :]], axis=1)
+            want = O.attention_decode(f(q)[0, i], K, V)
+            assert np.abs(o[0, i] - want).max() <= 1e-2, f"request {i}"
+        assert kinds == {"boundary": 2, "stepped": 9, "skipped": 1}, kinds
+        # next step: the full requests are stalled, the skipped one now takes its boundary
+        pool.decode_step(ids, dev(q), dev(k), dev(v), out, act)
+        a2 = act.cpu().numpy()
+        for i in range(n_req):
+            if a[i] == B.GP_ACT_SCRATCH:
+                P, n, pos, _ = B.gp_debug_request(pool.handle, i, cfg.max_pages_per_req)
+                if n == P0 * b and pos == n0 + 1:
+                    assert a2[i] == B.GP_ACT_STALLED
+                else:
+                    assert a2[i] in (B.GP_ACT_GROW, B.GP_ACT_COMPRESS)
+            else:
+                assert a2[i] == B.GP_ACT_NONE
+        assert B.gp_debug_pool(pool.handle, 0)[2][7] == 0
+    finally:
+        pool.close()
+
+
 def test_synchronised_boundaries_put_several_boundary_items_on_every_cta():
     # equal prompt lengths: every request reaches its capacity boundary in the same step, so the attention
     # kernel's CTAs each get several boundary work items in a row (their calibrated summaries share one buffer
