@@ -31,6 +31,9 @@ design notes; the ones with no independent check are marked "parity unpinned":
   * simultaneous boundaries: grants, then copy-on-write targets, each in ascending
     request id; references to replaced pages are dropped after all compactions
   * every shared page below the last one is replaced at a compression
+  * Shrink (Eq. 13, App. "capacity-control policies"): evicts 2b tokens of C by the same Eq. 10 rule with the
+    target |C| - 2b, hands the request's last page back once compaction is over, and is replaced by
+    Compress & Hold when the capacity left, (P - 1) b tokens, would be under the minimum capacity
 """
 from __future__ import annotations
 
@@ -51,6 +54,7 @@ ACT_NONE = 0
 ACT_GROW = 1
 ACT_COMPRESS = 2
 ACT_COMPRESS_FALLBACK = 3
+ACT_SHRINK = 4
 ACT_STALLED = -1
 ACT_INVALID = -3
 
@@ -218,6 +222,16 @@ def select_retained(s: np.ndarray, n_blocks: int, b: int, K_t: int, k_loc: int) 
 # =============================================================================
 # the pool and the per-step state machine
 # =============================================================================
+def shrink_policy(delta: float, tau: float = 0.0, shrink_below: float = -0.005) -> int:
+    """Eq. 13: Shrink when Delta_t < -0.005, Compress & Hold when -0.005 <= Delta_t <= 0, Grow by One Page when
+    Delta_t > 0 (`tau` and `shrink_below` carry the two thresholds; growing wins if they are set to overlap)."""
+    if delta > tau:
+        return ACT_GROW
+    if delta < shrink_below:
+        return ACT_SHRINK
+    return ACT_COMPRESS
+
+
 def random_draw(seed: int, req: int, pos: int) -> float:
     """Uniform draw in [0, 1) of the random capacity-control policy for request `req` at absolute position
     `pos`: the SplitMix64 finaliser of seed + 0x9E3779B97F4A7C15 (req + 1) + 0xBF58476D1CE4E5B9 pos (mod 2^64),
@@ -248,9 +262,11 @@ class OracleConfig:
     recent_window: int = 16          # equals the page size in this build
     k_loc: int = 4                   # a quarter of a page, the paper's 64 of 256
     rope_theta: float = 0.0
-    policy: int = 0                  # 0 demand (Eq. 8), 1 inverse, 2 random: the ablation's controls (with Eq. 13)
+    policy: int = 0                  # 0 demand (Eq. 8), 1 inverse, 2 random, 3 shrink (Eq. 13): the ablation's controls
     policy_seed: int = 0
     p_compress: float = 0.7
+    shrink_below: float = -0.005     # Eq. 13: Shrink when Delta_t is under this
+    min_capacity: int = 1024         # tokens; a Shrink that would leave less is a Compress & Hold
 
 
 class _Request:
@@ -269,6 +285,7 @@ class BoundaryInfo:
     ws_margin: Optional[np.ndarray] = None  # [L][H_kv][2]
     delta: float = 0.0
     want_grow: bool = False
+    want_shrink: bool = False               # policy 3 only, and only where a Shrink is admissible
     action_near_tie: bool = False
     action: int = ACT_NONE
     keep: Dict[Tuple[int, int], np.ndarray] = dataclasses.field(default_factory=dict)      # slots kept
@@ -295,7 +312,7 @@ class OraclePool:
         self.refcount = np.zeros(cfg.n_pages, dtype=np.int64)
         self.free: List[int] = list(range(cfg.n_pages - 1, -1, -1))   # pop() hands out page 0 first
         self.requests: Dict[int, _Request] = {}
-        self.counters = {"grow": 0, "compress": 0, "fallback": 0, "stalled": 0, "cow_pages": 0,
+        self.counters = {"grow": 0, "compress": 0, "fallback": 0, "shrink": 0, "stalled": 0, "cow_pages": 0,
                          "moved_rows": 0, "scored_tokens": 0}
 
     # ---- pool primitives ------------------------------------------------------
@@ -448,12 +465,17 @@ class OraclePool:
         elif c.policy == 2:          # random: Compress & Hold with probability p_compress, whatever Delta says
             info.want_grow = not (random_draw(c.policy_seed, rid, r.pos - 1) < c.p_compress)
             return info              # no working-set near-tie can change a coin
+        # Eq. 13: a Shrink needs two blocks of candidates and must leave the minimum capacity
+        can_shrink = c.policy == 3 and r.P >= 3 and (r.P - 1) * b >= c.min_capacity
+        if c.policy == 3:
+            info.want_shrink = can_shrink and shrink_policy(info.delta, c.tau, c.shrink_below) == ACT_SHRINK
         # could a +-1 change of near-tied working-set sizes change the decision?
         near = int((info.ws_margin < 1e-6).sum())
         if near:
-            lo = (num - near) / float(L * H * n_c) > c.tau
-            hi = (num + near) / float(L * H * n_c) > c.tau
-            info.action_near_tie = (lo != hi)
+            d_lo, d_hi = (num - near) / float(L * H * n_c), (num + near) / float(L * H * n_c)
+            info.action_near_tie = (d_lo > c.tau) != (d_hi > c.tau)
+            if can_shrink:
+                info.action_near_tie |= (d_lo < c.shrink_below) != (d_hi < c.shrink_below)
         return info
 
     def step_apply(self, rec: StepRecord, overrides: Optional[dict] = None) -> None:
@@ -472,6 +494,7 @@ class OraclePool:
             r = self.requests[rid]
             want = overrides.get(rid, {}).get("want_grow", info.want_grow)
             info.want_grow = bool(want)
+            info.want_shrink = bool(overrides.get(rid, {}).get("want_shrink", info.want_shrink)) and not want
             self.counters["scored_tokens"] += info.n_c
             if want and r.P < c.max_pages_per_req and self.free:
                 r.table.append(self._take_page())
@@ -482,7 +505,7 @@ class OraclePool:
                 info.action = ACT_STALLED        # one page, nothing to evict, no page to be had
                 self.counters["stalled"] += 1
             else:
-                info.action = ACT_COMPRESS_FALLBACK if want else ACT_COMPRESS
+                info.action = ACT_COMPRESS_FALLBACK if want else (ACT_SHRINK if info.want_shrink else ACT_COMPRESS)
                 compress.append(rid)
         # pass 2: copy-on-write targets, ascending request id, then selection and compaction
         released: List[int] = []
@@ -499,21 +522,28 @@ class OraclePool:
                 r.table[j] = self._take_page()
             info.cow_pages = len(shared)
             self.counters["cow_pages"] += len(shared)
-            self.counters["fallback" if info.action == ACT_COMPRESS_FALLBACK else "compress"] += 1
-            self._compress(r, info, overrides.get(rid, {}).get("keep", {}), set(shared))
+            kind = {ACT_COMPRESS_FALLBACK: "fallback", ACT_SHRINK: "shrink"}.get(info.action, "compress")
+            self.counters[kind] += 1
+            n_evict = 2 * b if info.action == ACT_SHRINK else b
+            self._compress(r, info, overrides.get(rid, {}).get("keep", {}), set(shared), n_evict)
             r.n_pristine = 0
+            if info.action == ACT_SHRINK:        # Eq. 13: one physical page goes back to the pool
+                released.append(r.table.pop())
+                r.P -= 1
         # pass 3: the replaced pages lose this request's reference once compaction is over
         for page in released:
             self._drop_ref(page)
         for rid in order:
             rec.actions[index_of[rid]] = rec.boundary[rid].action
 
-    def _compress(self, r: _Request, info: BoundaryInfo, keep_override: dict, cow: set) -> None:
-        """Eq. 9, Eq. 10 and the compaction, independently for every (layer, KV head)."""
+    def _compress(self, r: _Request, info: BoundaryInfo, keep_override: dict, cow: set, n_evict: int) -> None:
+        """Eq. 9, Eq. 10 and the compaction, independently for every (layer, KV head).  `n_evict` tokens of C
+        go: one page worth at a compression (the target is (P-1) b tokens, the protected page included), two
+        at a Shrink."""
         c = self.cfg
         b = c.page_size
         n_c = info.n_c
-        K_t = n_c - c.recent_window              # target (P-1) b minus the protected tokens
+        K_t = n_c - n_evict
         moved = 0
         for l in range(c.n_layers):
             for h in range(c.n_kv_heads):
@@ -535,7 +565,7 @@ class OraclePool:
                 r.V[l, h, :src.size] = r.V[l, h, src]
                 r.tok[l, h, :src.size] = r.tok[l, h, src]
                 r.tok[l, h, src.size:r.P * b] = -1
-        r.n = n_c
+        r.n = K_t + b
         info.moved_tokens = moved
         self.counters["moved_rows"] += moved
 

@@ -252,6 +252,10 @@ def test_selection_is_the_constrained_optimum(n_blocks, b, k_loc):
         assert keep.size == K_t and np.all(np.diff(keep) > 0)
         k_prime = min(k_loc, K_t // n_blocks)
         np.testing.assert_array_equal(keep, _best_subset(s, n_blocks, b, K_t, k_prime))
+        if n_blocks >= 3:                                        # the Shrink target of Eq. 13: two pages go
+            K_t = n_blocks * b - 2 * b
+            keep, _ = O.select_retained(s, n_blocks, b, K_t, k_loc)
+            np.testing.assert_array_equal(keep, _best_subset(s, n_blocks, b, K_t, min(k_loc, K_t // n_blocks)))
 
 
 def test_selection_special_cases_and_ties():
@@ -524,3 +528,73 @@ def test_inverse_and_random_policies_only_change_the_decision():
     assert outs[1][0][0] == (O.ACT_COMPRESS if d > 0 else O.ACT_GROW)
     assert outs[2][0][0] == O.ACT_COMPRESS                               # p_compress = 1: always Compress & Hold
     assert outs[3][0][0] == O.ACT_GROW                                   # p_compress = 0: always grows
+
+
+def test_eq13_regions_of_the_shrink_policy():
+    # Eq. 13 with the paper's thresholds: Shrink under -0.005, Compress & Hold on [-0.005, 0], Grow above 0
+    assert O.shrink_policy(-0.0051) == O.ACT_SHRINK and O.shrink_policy(-1.0) == O.ACT_SHRINK
+    assert O.shrink_policy(-0.005) == O.ACT_COMPRESS          # both ends of the middle interval are closed
+    assert O.shrink_policy(-0.001) == O.ACT_COMPRESS and O.shrink_policy(0.0) == O.ACT_COMPRESS
+    assert O.shrink_policy(1e-12) == O.ACT_GROW and O.shrink_policy(1.0) == O.ACT_GROW
+    assert O.OracleConfig(1, 1, 1, 8, 1, 1).shrink_below == -0.005 and O.OracleConfig(1, 1, 1, 8, 1, 1).min_capacity == 1024
+
+
+def test_shrink_returns_one_page_evicts_two_and_respects_the_floor():
+    c = _cfg(n_pages=16, max_pages_per_req=6)                        # at most 20 candidates: brute force stays small
+    c.policy, c.min_capacity, c.shrink_below, c.tau = 3, 12, -0.005, 0.01
+    pool = O.OraclePool(c)
+    b = c.page_size
+    g = np.random.default_rng(11)
+    kt = g.standard_normal((c.n_layers, 14, c.n_kv_heads, c.head_dim))
+    _, rid = pool.request_add(-1, 0, kt, kt.copy(), 14, 0)
+    seen = {}
+    for step in range(160):
+        shp_q, shp_k = (c.n_layers, 1, c.n_q_heads, c.head_dim), (c.n_layers, 1, c.n_kv_heads, c.head_dim)
+        P0, n0, _, _ = pool.request_state(rid)
+        free0 = pool.n_free()
+        rec = pool.decode_step([rid], g.standard_normal(shp_q), g.standard_normal(shp_k), g.standard_normal(shp_k))
+        P1, n1, pos1, _ = pool.request_state(rid)
+        act = int(rec.actions[0])
+        seen[act] = seen.get(act, 0) + 1
+        if rid in rec.boundary:
+            info = rec.boundary[rid]
+            want = O.shrink_policy(info.delta, c.tau, c.shrink_below)
+            if want == O.ACT_SHRINK and (P0 - 1) * b < c.min_capacity:
+                want = O.ACT_COMPRESS                                  # the floor: capacity left would be under 12
+            if want == O.ACT_GROW and act != O.ACT_GROW:
+                assert act == O.ACT_COMPRESS_FALLBACK and (P0 == c.max_pages_per_req or free0 == 0)
+            else:
+                assert act == want
+        if act == O.ACT_SHRINK:
+            assert (P1, n1) == (P0 - 1, (P0 - 2) * b) and pool.n_free() == free0 + 1
+            assert P1 * b >= c.min_capacity
+            for l in range(c.n_layers):
+                for h in range(c.n_kv_heads):
+                    assert info.keep[(l, h)].size == (P0 - 3) * b
+                    s_tok = O.token_scores(info.a_s[l, h], info.a_l[l, h])
+                    np.testing.assert_array_equal(
+                        info.keep[(l, h)], _best_subset(s_tok, P0 - 1, b, (P0 - 3) * b, min(c.k_loc, ((P0 - 3) * b) // (P0 - 1))))
+                    tok = pool.retained(rid, l, h)
+                    assert np.array_equal(tok[-b:], np.arange(pos1 - b, pos1))       # the newest page survives
+        _check_invariants(pool)
+    assert seen.get(O.ACT_SHRINK, 0) > 0 and seen.get(O.ACT_GROW, 0) > 0 and seen.get(O.ACT_COMPRESS, 0) > 0, seen
+
+
+def test_shrink_with_shared_prompt_pages_copies_before_it_writes():
+    c = _cfg(n_pages=40, max_pages_per_req=12)
+    c.policy, c.min_capacity, c.shrink_below, c.tau = 3, 8, 0.5, 2.0     # every admissible boundary shrinks
+    pool = O.OraclePool(c)
+    g = np.random.default_rng(12)
+    kt = g.standard_normal((c.n_layers, 24, c.n_kv_heads, c.head_dim))
+    _, a = pool.request_add(-1, 0, kt, kt.copy(), 24, 0)
+    _, b_ = pool.request_add(a, 6, None, None, 0, 0)
+    K_before = pool.requests[b_].K[:, :, :24].copy()
+    for step in range(40):
+        shp_q, shp_k = (c.n_layers, 1, c.n_q_heads, c.head_dim), (c.n_layers, 1, c.n_kv_heads, c.head_dim)
+        rec = pool.decode_step([a], g.standard_normal(shp_q), g.standard_normal(shp_k), g.standard_normal(shp_k))
+        _check_invariants(pool)
+    assert pool.counters["shrink"] > 0 and pool.counters["cow_pages"] == 6
+    # the sharer's prompt is untouched by the other request's shrinking
+    np.testing.assert_array_equal(pool.requests[b_].K[:, :, :24], K_before)
+    pool.release(a); pool.release(b_)
+    assert pool.n_free() == c.n_pages
