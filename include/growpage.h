@@ -41,6 +41,8 @@ extern "C" {
 #define GP_ACT_GROW               1   /* Delta_t > tau: one page appended to the block table      */
 #define GP_ACT_COMPRESS           2   /* Compress & Hold: one page worth of slots freed in place  */
 #define GP_ACT_COMPRESS_FALLBACK  3   /* wanted to grow, cap or free list said no, compressed     */
+#define GP_ACT_SHRINK             4   /* GP_POLICY_SHRINK: two pages worth of slots freed in place,
+                                         the last page returned to the pool (Eq. 13)              */
 #define GP_ACT_STALLED          (-1)  /* full and neither a page nor copy-on-write targets could
                                          be had: page state untouched, the caller should release
                                          (preempt) the request; it is skipped while it stays full */
@@ -62,10 +64,16 @@ typedef struct gp_pool gp_pool; /* opaque */
  *            u = (mix(policy_seed + 0x9E3779B97F4A7C15 * (r + 1) + 0xBF58476D1CE4E5B9 * pos) >> 11) * 2^-53,
  *            arithmetic modulo 2^64, mix = the SplitMix64 finaliser; compress iff u < p_compress.
  *            Working sets and Delta_t are still computed and reported.
- * (The ablation's Shrink policy, which also gives pages back, is not implemented.) */
+ *   SHRINK   Eq. 13, three actions: grow iff Delta_t > tau; Shrink iff Delta_t < shrink_below (and not
+ *            growing); Compress & Hold in between.  A Shrink evicts two pages worth of the candidate set C
+ *            per (layer, KV head) by the rule of Eq. 10 with the target |C| - 2b, compacts in place, and
+ *            returns the request's last page to the pool: P pages become P - 1 with one page of free slots.
+ *            It needs P >= 3 and (P - 1) * page_size >= min_capacity (the capacity left); otherwise the
+ *            boundary is a Compress & Hold.  Shared pages are copied first as for a compression. */
 #define GP_POLICY_DEMAND   0
 #define GP_POLICY_INVERSE  1
 #define GP_POLICY_RANDOM   2
+#define GP_POLICY_SHRINK   3
 
 typedef struct gp_config {
   int32_t n_layers;          /* L                                                                  */
@@ -81,6 +89,7 @@ typedef struct gp_config {
   int32_t policy;            /* GP_POLICY_*: how Delta_t becomes an action (default: demand)       */
   int32_t policy_seed;       /* GP_POLICY_RANDOM: seed of its counter-based draws                  */
   int64_t n_pages;           /* physical pages; one page id covers all layers and KV heads         */
+  int64_t min_capacity;      /* GP_POLICY_SHRINK: tokens of capacity a Shrink must leave, default 1024 */
   int64_t max_batch_tokens;  /* bound on the summed sequence lengths of one decode batch, used to
                                 size scratch; 0 = n_pages * page_size, which bounds it only while
                                 no prompt pages are shared (a shared page counts once in the pool
@@ -91,6 +100,7 @@ typedef struct gp_config {
   double  tau;               /* decision threshold, default 0                                      */
   double  rope_theta;        /* RoPE base (rotate-half pairing); 0 = no rotation                   */
   double  p_compress;        /* GP_POLICY_RANDOM: probability of Compress & Hold, default 0.7      */
+  double  shrink_below;      /* GP_POLICY_SHRINK: Shrink iff Delta_t is under it, default -0.005    */
 } gp_config;
 
 /* Fills *cfg with the paper's defaults (Sec. 3.2, Sec. 5.1, App. B.2, App. D.1); the geometry
@@ -196,7 +206,7 @@ int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, do
  * [0] grow [1] compress [2] fallback-compress [3] stalled [4] copy-on-write pages
  * [5] decode steps [6] tokens decoded [7] internal error bits (0 when healthy)
  * [8] (layer, head, token) rows rewritten by compaction [9] candidate tokens scored at boundaries
- * [10], [11] reserved. */
+ * [10] Shrink events (not counted under [1]) [11] reserved. */
 int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[12]);
 
 /* ---- measurement ----------------------------------------------------------------------------- */

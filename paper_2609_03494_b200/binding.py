@@ -16,9 +16,9 @@ LIB_PATH = os.path.join(_HERE, "libgrowpage.so")
 GP_OK, GP_ERR_INVALID, GP_ERR_NO_SLOT, GP_ERR_NO_PAGES, GP_ERR_CUDA, GP_ERR_STATE = 0, -1, -2, -3, -4, -5
 GP_ERR_TOO_LARGE = -6
 GP_NOALLOC_MAX_ROWS = 2048
-GP_ACT_NONE, GP_ACT_GROW, GP_ACT_COMPRESS, GP_ACT_COMPRESS_FALLBACK = 0, 1, 2, 3
+GP_ACT_NONE, GP_ACT_GROW, GP_ACT_COMPRESS, GP_ACT_COMPRESS_FALLBACK, GP_ACT_SHRINK = 0, 1, 2, 3, 4
 GP_ACT_STALLED, GP_ACT_SCRATCH, GP_ACT_INVALID = -1, -2, -3
-GP_POLICY_DEMAND, GP_POLICY_INVERSE, GP_POLICY_RANDOM = 0, 1, 2
+GP_POLICY_DEMAND, GP_POLICY_INVERSE, GP_POLICY_RANDOM, GP_POLICY_SHRINK = 0, 1, 2, 3
 GP_N_KERNELS = 4
 KERNEL_NAMES = ("plan", "attention", "select_decide", "compact")
 
@@ -29,9 +29,9 @@ class gp_config(C.Structure):
         ("page_size", C.c_int32), ("max_requests", C.c_int32), ("max_pages_per_req", C.c_int32),
         ("recent_window", C.c_int32), ("k_loc", C.c_int32), ("host_staging", C.c_int32),
         ("policy", C.c_int32), ("policy_seed", C.c_int32),
-        ("n_pages", C.c_int64), ("max_batch_tokens", C.c_int64),
+        ("n_pages", C.c_int64), ("min_capacity", C.c_int64), ("max_batch_tokens", C.c_int64),
         ("beta_s", C.c_double), ("beta_l", C.c_double), ("top_p", C.c_double), ("tau", C.c_double),
-        ("rope_theta", C.c_double), ("p_compress", C.c_double),
+        ("rope_theta", C.c_double), ("p_compress", C.c_double), ("shrink_below", C.c_double),
     ]
 
 
@@ -304,11 +304,13 @@ class Pool:
 def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n_pages: int, max_pages_per_req: int,
                 max_requests: int = 512, k_loc: int = 4, host_staging: bool = False, max_batch_tokens: int = 0,
                 beta_s: float = 0.9, beta_l: float = 0.999, top_p: float = 0.99, tau: float = 0.0,
-                rope_theta: float = 0.0, policy: int = 0, policy_seed: int = 0, p_compress: float = 0.7) -> gp_config:
+                rope_theta: float = 0.0, policy: int = 0, policy_seed: int = 0, p_compress: float = 0.7,
+                shrink_below: float = -0.005, min_capacity: int = 1024) -> gp_config:
     cfg = gp_config_default()
     cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
     cfg.n_pages, cfg.max_pages_per_req, cfg.max_requests = n_pages, max_pages_per_req, max_requests
     cfg.k_loc, cfg.host_staging, cfg.max_batch_tokens = k_loc, 1 if host_staging else 0, max_batch_tokens
     cfg.beta_s, cfg.beta_l, cfg.top_p, cfg.tau, cfg.rope_theta = beta_s, beta_l, top_p, tau, rope_theta
     cfg.policy, cfg.policy_seed, cfg.p_compress = policy, policy_seed, p_compress
+    cfg.shrink_below, cfg.min_capacity = shrink_below, min_capacity
     return cfg

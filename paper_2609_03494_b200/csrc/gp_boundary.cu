@@ -32,6 +32,7 @@ constexpr int SEL_NW = SEL_T / 32;
 constexpr int SEL_CAP = 6144;        // candidate tokens whose scores are staged in shared memory
 constexpr int CT = 256;              // threads of the compaction kernel
 constexpr int MOVE_TOK = GP_MOVE_TOK;     // source slots per compaction chunk
+constexpr int CMP_SHRINK = 1 << 30;       // flag on a compressing request's boundary index: the action is a Shrink
 
 __device__ __forceinline__ unsigned long long to_fix(double a) {
   return (unsigned long long)__double2ll_rn(a * TWO62);
@@ -281,11 +282,11 @@ __device__ int top_p_fast(const GpDev& p, const double* a, int n, unsigned long 
   return (int)s_res[3];
 }
 
-// Eq. 10 global cut on the fast path (counts already zeroed, s_res[0] = -1, s_cnt[0..1] = 0): lists the b
-// evicted slots in ev[] (unsorted) and returns true, or returns false when the general routine has to take
+// Eq. 10 global cut on the fast path (counts already zeroed, s_res[0] = -1, s_cnt[0..1] = 0): lists the ne
+// (b, or 2b for a Shrink) evicted slots in ev[] (unsorted) and returns true, or returns false when the general routine has to take
 // over.  `a` holds Eq. 9 scores, `loc` the block-local quota bits (those slots are never evicted).
 __device__ bool evict_fast(const double* a, int nC, const unsigned* loc, const FastHist& H, unsigned* wc, long long* s_res,
-                           double* list, int* list_slot, int* s_cnt, int* ev) {
+                           double* list, int* list_slot, int* s_cnt, int* ev, const unsigned ne) {
   const int tid = threadIdx.x;
   for (int i = tid; i < nC; i += SEL_T) {
     if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
@@ -298,7 +299,7 @@ __device__ bool evict_fast(const double* a, int nC, const unsigned* loc, const F
   {                                               // summary level, ascending: the b lowest scores go
     const unsigned c = tid < CBINS ? H.ccnt[tid] : 0u;
     const unsigned ex = block_prefix_excl<SEL_T>(c, wc);
-    if (tid < CBINS && ex < (unsigned)GP_PAGE && ex + c >= (unsigned)GP_PAGE) { s_res[0] = tid; s_res[1] = ex; }
+    if (tid < CBINS && ex < ne && ex + c >= ne) { s_res[0] = tid; s_res[1] = ex; }
   }
   __syncthreads();
   if (s_res[0] < 0) return false;
@@ -312,12 +313,12 @@ __device__ bool evict_fast(const double* a, int nC, const unsigned* loc, const F
       if (tid >= off) ic += tc;
     }
     const unsigned before = (unsigned)s_res[1] + ic - c;
-    if (tid < 16 && before < (unsigned)GP_PAGE && before + c >= (unsigned)GP_PAGE) { s_res[4] = fb; s_res[5] = before; s_res[6] = c; }
+    if (tid < 16 && before < ne && before + c >= ne) { s_res[4] = fb; s_res[5] = before; s_res[6] = c; }
   }
   __syncthreads();
   const int bstar = (int)s_res[4];
   const int cnt_below = (int)s_res[5], cstar = (int)s_res[6];
-  const bool exact = (cnt_below + cstar == GP_PAGE);
+  const bool exact = (cnt_below + cstar == (int)ne);
   if (!exact && cstar > 32) return false;
   for (int i = tid; i < nC; i += SEL_T) {
     if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
@@ -331,15 +332,15 @@ __device__ bool evict_fast(const double* a, int nC, const unsigned* loc, const F
     double v = tid < cstar ? list[tid] : INFINITY;
     int slot = tid < cstar ? list_slot[tid] : -1;
     warp_sort<false>(v, slot);
-    if (tid < GP_PAGE - cnt_below) ev[cnt_below + tid] = slot;
+    if (tid < (int)ne - cnt_below) ev[cnt_below + tid] = slot;
   }
   __syncthreads();
   return true;
 }
 
-// Eq. 10 global cut, general routine (radix descent over the score bits): lists the b evicted slots in ev[]
+// Eq. 10 global cut, general routine (radix descent over the score bits): lists the ne evicted slots in ev[]
 __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int nC, const unsigned* loc, unsigned* hcnt,
-                                           unsigned* wc, long long* s_res, int* s_i, int* ev) {
+                                           unsigned* wc, long long* s_res, int* s_i, int* ev, const unsigned ne) {
   const int tid = threadIdx.x;
       __syncthreads();
     unsigned long long prefix = 0;
@@ -375,7 +376,7 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
         for (int b = lo; b < hi; ++b) {
           const unsigned before = run;
           run += hcnt[HIDX(b)];
-          if (before < (unsigned)GP_PAGE && run >= (unsigned)GP_PAGE) { s_res[0] = b; s_res[1] = before; }
+          if (before < ne && run >= ne) { s_res[0] = b; s_res[1] = before; }
         }
       }
       __syncthreads();
@@ -388,7 +389,7 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
       const unsigned cstar = hcnt[HIDX(bin_star)];
       __syncthreads();
       prefix = (prefix << w) | (unsigned long long)bin_star;
-      if (cnt_below + cstar == (unsigned)GP_PAGE) {        // the bin fits exactly: no tie to break
+      if (cnt_below + cstar == ne) {        // the bin fits exactly: no tie to break
         thr = (prefix + 1ull) << shift;
         done = true;
       }
@@ -396,7 +397,7 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
     if (!done) {                                           // equal scores straddle the cut
       thr = prefix;
       tie_key = prefix;
-      need_eq = GP_PAGE - (int)cnt_below;
+      need_eq = (int)ne - (int)cnt_below;
     }
   }
   const long long t_s4 = GP_T_NOW();
@@ -404,7 +405,7 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
   for (int i = tid; i < nC; i += SEL_T) {
     if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
       const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-      if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < GP_PAGE) ev[at] = i; }
+      if (key < thr) { const int at = atomicAdd(&s_i[0], 1); if (at < (int)ne) ev[at] = i; }
     }
   }
   __syncthreads();
@@ -413,10 +414,10 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
     for (int i = nC - 1; i >= 0 && need_eq > 0; --i) {     // rare: older (lower) slots win ties
       if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
         const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
-        if (key == tie_key) { if (cntv < GP_PAGE) ev[cntv] = i; ++cntv; --need_eq; }
+        if (key == tie_key) { if (cntv < (int)ne) ev[cntv] = i; ++cntv; --need_eq; }
       }
     }
-    if (cntv != GP_PAGE) atomicOr(p.err, GP_E_BOUNDS);
+    if (cntv != (int)ne) atomicOr(p.err, GP_E_BOUNDS);
     GP_T_ADD(21, GP_T_NOW() - t_s4);
   }
 }
@@ -471,6 +472,8 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
           zz = (zz ^ (zz >> 27)) * 0x94D049BB133111EBull;
           zz ^= zz >> 31;
           want = !((double)(zz >> 11) * (1.0 / 9007199254740992.0) < p.p_compress);
+        } else if (p.policy == GP_POLICY_SHRINK) {            // Eq. 13: the third action, where it is admissible
+          if (!want && delta < p.shrink_below && Pr - 1 >= p.min_pages_after_shrink) want = 16;
         }
       }
       p.delta[r] = delta;
@@ -505,7 +508,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
   if (tid == 0) {                                        // sequential allocator: shared memory only
     int top = top0;
     int n_cmp = 0, chunks = 0;
-    unsigned long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0;
+    unsigned long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0, shr = 0;
     for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants, ascending request id
       const int e = s_order[k];
       const int r = s_req[e], Pr = s_P[e], bi = s_bi[e];
@@ -537,11 +540,17 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       s_base[e] = top;
       top -= s_ksh[e];
       cow += s_ksh[e];
-      p.cmp_info[n_cmp] = make_int4(r, s_P[e], e, chunks);
+      const bool shrink = (s_want[e] & 16) != 0;
+      p.cmp_info[n_cmp] = make_int4(r, s_P[e], e | (shrink ? CMP_SHRINK : 0), chunks);
       chunks += (s_P[e] * GP_PAGE + MOVE_TOK - 1) / MOVE_TOK;
       ++n_cmp;
-      if (s_want[e] & 1) { actions[bi] = GP_ACT_COMPRESS_FALLBACK; ++fall; } else { actions[bi] = GP_ACT_COMPRESS; ++comp; }
-      p.n[r] = (s_P[e] - 1) * GP_PAGE;
+      if (s_want[e] & 1) { actions[bi] = GP_ACT_COMPRESS_FALLBACK; ++fall; }
+      else if (shrink) { actions[bi] = GP_ACT_SHRINK; ++shr; }
+      else { actions[bi] = GP_ACT_COMPRESS; ++comp; }
+      // a compression frees one page worth of slots; a Shrink frees two and gives the last page back (the
+      // compaction kernel returns it once nothing reads it any more)
+      p.n[r] = (s_P[e] - (shrink ? 2 : 1)) * GP_PAGE;
+      if (shrink) p.P[r] = s_P[e] - 1;
       p.n_pristine[r] = 0;
       s_want[e] |= 8;
     }
@@ -550,13 +559,14 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     *p.free_top = top;
     p.hdr[HDR_N_CMP] = n_cmp;
     p.hdr[HDR_N_CITEM] = chunks * LH;
-    p.hdr[HDR_N_COW] = (int)cow;
+    p.hdr[HDR_N_COW] = (int)(cow + shr);           // page-table work left for the compaction kernel's last CTA
     unsigned long long* cn = reinterpret_cast<unsigned long long*>(p.counters);
     if (grow) atomicAdd(cn + 0, grow);
     if (comp) atomicAdd(cn + 1, comp);
     if (fall) atomicAdd(cn + 2, fall);
     if (stall) atomicAdd(cn + 3, stall);
     if (cow) atomicAdd(cn + 4, cow);
+    if (shr) atomicAdd(cn + 10, shr);
     atomicAdd(cn + 9, scored);
   }
   __syncthreads();
@@ -788,14 +798,16 @@ __device__ __noinline__ void merge_partials(const GpDev& p, int n_req, float* __
 }
 
 // ------------------------------------------------------------------------------------------------------
-// working sets + speculative eviction list; three independent jobs per unit, one CTA each; the last CTA decides
+// working sets + speculative eviction list; three independent jobs per unit (four under the Shrink policy: its
+// list of 2b evictions), one CTA each; the last CTA decides
 // ------------------------------------------------------------------------------------------------------
 struct SelGeom {
   static constexpr size_t BUF_BYTES = SEL_CAP * sizeof(double);
   static constexpr size_t H_BYTES = (size_t)FB_PAD * 12;
-  static constexpr size_t MISC_BYTES = SEL_NW * 8 + SEL_NW * 4 + 8 * 8 + 16 * 4 + 16 * 4 + (SEL_NW * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
+  static constexpr size_t MISC_BYTES = SEL_NW * 8 + SEL_NW * 4 + 8 * 8 + 32 * 4 + 16 * 4 + (SEL_NW * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
 };
 
+template <bool SHR>      // SHR: the pool runs the Shrink policy (a fourth job per unit)
 __global__ void __launch_bounds__(SEL_T, 1)
 gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
                float* __restrict__ out) {
@@ -807,8 +819,8 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   unsigned long long* wsum = hsum + FB_PAD;                                    // [SEL_NW]
   unsigned* wc = reinterpret_cast<unsigned*>(wsum + SEL_NW);                   // [SEL_NW]
   long long* s_res = reinterpret_cast<long long*>(wc + SEL_NW);                // [8]
-  int* ev = reinterpret_cast<int*>(s_res + 8);                                 // [16]
-  int* s_i = ev + 16;                                                          // [16]
+  int* ev = reinterpret_cast<int*>(s_res + 8);                                 // [32]
+  int* s_i = ev + 32;                                                          // [16]
   double* red = reinterpret_cast<double*>(s_i + 16);                           // [SEL_NW][16]
   double* sM = red + SEL_NW * 16;                                                   // [16]
   double* sZ = sM + 16;                                                        // [16]
@@ -826,18 +838,19 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const int tid = threadIdx.x;
   const int LH = p.L * p.Hkv;
   const int G = p.G, G2 = 2 * p.G;
+  constexpr int NT = SHR ? 4 : 3;                           // jobs per unit: K^S, K^L, eviction list(s)
   gp_pdl_wait();
   gp_pdl_launch_dependents();
   // the first item's descriptor is fetched before the number of items is known (same round trip); slots of
   // bnd_info past the count hold stale but readable data that is then not used
   int4 inf_first = make_int4(0, 0, 0, 0), inf2_first = inf_first;
   {
-    const int b0 = (int)(blockIdx.x / (3 * LH));
+    const int b0 = (int)(blockIdx.x / (NT * LH));
     if (b0 < p.M) { inf_first = p.bnd_info[2 * b0]; inf2_first = p.bnd_info[2 * b0 + 1]; }
   }
   const int n_bnd = p.hdr[HDR_N_BND];
   const int n_mc = out ? p.hdr[HDR_N_MC] : 0, n_rc = p.hdr[HDR_N_RC];   // out == null: already merged layer by layer
-  const long long items = (long long)n_bnd * LH * 3;
+  const long long items = (long long)n_bnd * LH * NT;
   if (tid == 0) GP_T_STAMP(59);
 
   // CTAs without a job merge the split requests' attention partials while the others work; when fewer than a
@@ -864,8 +877,10 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       }
       continue;
     }
-    const long long u = item / 3;
-    const int task = (int)(item % 3);               // 0: K^S, 1: K^L, 2: eviction list
+    const long long u = item / NT;
+    const int job = (int)(item % NT);               // 0: K^S, 1: K^L, 2: eviction list, 3: a Shrink's eviction list
+    const int task = job < 2 ? job : 2;
+    const int ne = (SHR && job == 3) ? 2 * GP_PAGE : GP_PAGE;
     const int bidx = (int)(u / LH), lh = (int)(u % LH);
     const int l = lh / p.Hkv, h = lh % p.Hkv;
     const bool is_first = item == (long long)blockIdx.x;
@@ -875,17 +890,18 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     const long long off = (long long)(unsigned)inf2.x | ((long long)inf2.y << 32);
     const int nC = (Pr - 1) * GP_PAGE;
     int* Kout = p.Kx + (((size_t)r * p.L + l) * p.Hkv + h) * 2;
-    int* evout = p.evict + (size_t)u * GP_PAGE;
+    int* evout = (SHR && job == 3) ? p.evict2 + (size_t)u * 2 * GP_PAGE : p.evict + (size_t)u * GP_PAGE;
     __syncthreads();
     if (nC == 0) {
       if (tid == 0 && task < 2) Kout[task] = 0;
       continue;
     }
+    if (SHR && job == 3 && Pr - 1 < p.min_pages_after_shrink) continue;      // this boundary cannot be a Shrink
     const long long t_s0 = GP_T_NOW();
     (void)t_s0;
     const size_t view_stride = (size_t)p.z_stride * G;
     const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;   // [2 views][nC][G] exp(logit - page max)
-    double* a = nC <= SEL_CAP ? sbuf : p.scores + ((size_t)task * LH + lh) * p.max_batch_tokens + off;
+    double* a = nC <= SEL_CAP ? sbuf : p.scores + ((size_t)job * LH + lh) * p.max_batch_tokens + off;
     if (task == 2) for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
     if (tid == 0) { s_res[0] = -1; s_i[0] = 0; s_i[5] = 0; s_i[6] = 0; s_i[7] = 0; }
     bool uniform;
@@ -915,7 +931,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     }
     // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
     const int nblk = Pr - 1;
-    const int K_t = nC - GP_PAGE;
+    const int K_t = nC - ne;
     const int kq = min(p.k_loc, K_t / nblk);
     if (kq > 0) {
       for (int i = tid; i < nC; i += SEL_T) {
@@ -934,14 +950,13 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     const long long t_s3 = GP_T_NOW();
     (void)t_s3;
     // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
-    if (!uniform || !evict_fast(a, nC, loc, H, wc, s_res, flist, flist_slot, &s_i[6], ev))
-      evict_general(p, a, nC, loc, hcnt, wc, s_res, s_i, ev);
+    if (!uniform || !evict_fast(a, nC, loc, H, wc, s_res, flist, flist_slot, &s_i[6], ev, (unsigned)ne))
+      evict_general(p, a, nC, loc, hcnt, wc, s_res, s_i, ev, (unsigned)ne);
     __syncthreads();
-    if (tid < GP_PAGE) {                                     // the 16 slots in ascending order, by rank
+    if (tid < ne) {                                          // the evicted slots in ascending order, by rank
       const int mine = ev[tid];
       int rank = 0;
-#pragma unroll
-      for (int j = 0; j < GP_PAGE; ++j) rank += (ev[j] < mine);
+      for (int j = 0; j < ne; ++j) rank += (ev[j] < mine);
       evout[rank] = mine;
     }
     if (tid == 0) { GP_T_ADD(31, 1); GP_T_ADD(19, t_s3 - t_s1); GP_T_ADD(20, GP_T_NOW() - t_s3); GP_T_ADD(22, t_s1 - t_s0); }
@@ -982,14 +997,14 @@ gp_merge_kernel(const __grid_constant__ GpDev p, int n_req, float* __restrict__ 
 // ------------------------------------------------------------------------------------------------------
 // compaction
 // ------------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool SHR>
 __global__ void __launch_bounds__(CT)
 gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req) {
   constexpr int CH = D / 8;
   constexpr int ROW_BYTES = D * 2;
   constexpr int PIECES = MOVE_TOK * 2 * CH / CT;        // 16-byte pieces per thread per chunk
   __shared__ int4 s_info[GP_MAX_REQ + 1];     // compressing requests: {request, P, boundary index, first chunk}
-  __shared__ int ev[GP_PAGE];
+  __shared__ int ev[2 * GP_PAGE];
   __shared__ int s_i[8];
   __shared__ int s_dst[MOVE_TOK], s_spage[MOVE_TOK], s_dpage[MOVE_TOK];   // per source slot of the chunk: destination slot (-1: stays or goes), source and destination page
 
@@ -1034,16 +1049,22 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
     const int* shadow = p.shadow + (size_t)r * p.cap;
     const int n_src = Pr * GP_PAGE;
     const int c0 = j * MOVE_TOK;
-    // second round trip: the eviction list, and for every source slot of the chunk its page and the page one
-    // before it (a slot moves down by at most one page) with their copy-on-write targets
-    int t0 = 0, s0 = -1, tm = 0, sm = -1;
+    // second round trip: the eviction list, and for every source slot of the chunk its page and the pages
+    // before it that it can move to (a slot moves down by at most one page, two at a Shrink) with their
+    // copy-on-write targets
+    const bool shrink = SHR && (inf.z & CMP_SHRINK) != 0;
+    const int e_bnd = inf.z & (CMP_SHRINK - 1);
+    const int ne = shrink ? 2 * GP_PAGE : GP_PAGE;
+    int t0 = 0, s0 = -1, tm = 0, sm = -1, tm2 = 0, sm2 = -1;
     const int my_i = c0 + tid;                             // the slot this thread plans (first MOVE_TOK threads)
     if (tid < MOVE_TOK && my_i < n_src) {
       const int pg = my_i / GP_PAGE;
       t0 = table[pg]; s0 = shadow[pg];
       if (pg > 0) { tm = table[pg - 1]; sm = shadow[pg - 1]; }
+      if (shrink && pg > 1) { tm2 = table[pg - 2]; sm2 = shadow[pg - 2]; }
     }
-    if (tid < GP_PAGE) ev[tid] = p.evict[((size_t)inf.z * LH + lh) * GP_PAGE + tid];
+    if (tid < ne) ev[tid] = shrink ? p.evict2[((size_t)e_bnd * LH + lh) * 2 * GP_PAGE + tid]
+                                   : p.evict[((size_t)e_bnd * LH + lh) * GP_PAGE + tid];
     __syncthreads();
     int tokv = 0, tok_dst = -1, tok_page = 0;
     if (tid < MOVE_TOK) {
@@ -1052,11 +1073,16 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         int sh = 0; bool evicted = false;
 #pragma unroll
         for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < my_i); evicted |= (ev[e2] == my_i); }
+        if (shrink) {
+#pragma unroll
+          for (int e2 = GP_PAGE; e2 < 2 * GP_PAGE; ++e2) { sh += (ev[e2] < my_i); evicted |= (ev[e2] == my_i); }
+        }
         const int pg = my_i / GP_PAGE;
         const bool cow = (pg < Pr - 1) && (s0 >= 0);
         if (!evicted && (sh > 0 || cow)) {
           ds = my_i - sh;
-          dpage = (ds / GP_PAGE == pg) ? (s0 >= 0 ? s0 : t0) : (sm >= 0 ? sm : tm);
+          const int back = pg - ds / GP_PAGE;              // 0, 1, or (Shrink only) 2 pages down
+          dpage = back == 0 ? (s0 >= 0 ? s0 : t0) : back == 1 ? (sm >= 0 ? sm : tm) : (sm2 >= 0 ? sm2 : tm2);
           tokv = p.tok[gp_tok_off(p, l, t0, h) + (my_i % GP_PAGE)];
           tok_dst = ds; tok_page = dpage;
         }
@@ -1127,8 +1153,9 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   if (tid == 0 && s_i[3] > 0)
     atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 8), (unsigned long long)s_i[3]);
 
-  // ---- the last CTA swaps in the copy-on-write targets and drops the old references (App. D.2) ----------
-  if (n_cow == 0) return;                                 // nothing was shared: no targets to swap in
+  // ---- the last CTA swaps in the copy-on-write targets and drops the old references (App. D.2), and hands
+  // back the last page of every request that shrank (Eq. 13) ---------------------------------------------
+  if (n_cow == 0) return;                                 // nothing was shared and nobody shrank
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -1163,12 +1190,28 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         if (lane == 0 && mask) *reinterpret_cast<volatile int*>(p.free_top) = base + __popc(mask);
         __syncwarp();
       }
+      if (SHR && (s_info[ci].z & CMP_SHRINK) && lane == 0) {      // the page the request no longer owns
+        const int last = table[Pr - 1];
+        if (atomicSub(&p.refcount[last], 1) == 1) {
+          const int top = *reinterpret_cast<volatile int*>(p.free_top);
+          p.free_stack[top] = last;
+          *reinterpret_cast<volatile int*>(p.free_top) = top + 1;
+        }
+      }
+      __syncwarp();
     }
   }
   if (tid == 0) GP_T_STAMP(38);
 }
 
 }  // namespace
+
+// the compaction kernel of a pool: head dimension, and whether the Shrink policy is on
+static auto compact_kernel_of(const GpDev& p) -> void (*)(const GpDev, const int*, int) {
+  const bool shr = p.policy == GP_POLICY_SHRINK;
+  if (p.d == 128) return shr ? gp_compact_kernel<128, true> : gp_compact_kernel<128, false>;
+  return shr ? gp_compact_kernel<64, true> : gp_compact_kernel<64, false>;
+}
 
 size_t gp_bsel_smem(const GpDev& p) {
   return SelGeom::BUF_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
@@ -1178,13 +1221,14 @@ size_t gp_bsel_smem(const GpDev& p) {
 // exactly one resident wave, so that no CTA waits for another to leave before it can start
 void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact) {
   const size_t sel_sm = gp_bsel_smem(p);
-  cudaFuncSetAttribute(gp_bsel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
+  const bool shr = p.policy == GP_POLICY_SHRINK;
+  auto sel = shr ? gp_bsel_kernel<true> : gp_bsel_kernel<false>;
+  cudaFuncSetAttribute(sel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
   int occ = 0;
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_bsel_kernel, SEL_T, sel_sm);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, sel, SEL_T, sel_sm);
   *grid_sel = num_sms * (occ > 0 ? occ : 1);
   occ = 0;
-  if (p.d == 128) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_compact_kernel<128>, CT, 0);
-  else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gp_compact_kernel<64>, CT, 0);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, compact_kernel_of(p), CT, 0);
   *grid_compact = num_sms * (occ > 0 ? occ : 1);
 }
 
@@ -1195,8 +1239,9 @@ void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, i
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
                         int grid_compact, cudaStream_t s, cudaEvent_t ev, bool pdl) {
   const size_t sel_sm = gp_bsel_smem(p);
-  gp_launch(gp_bsel_kernel, grid_sel, SEL_T, sel_sm, s, pdl, p, req_ids, n_req, actions, out);
+  const bool shr = p.policy == GP_POLICY_SHRINK;
+  gp_launch(shr ? gp_bsel_kernel<true> : gp_bsel_kernel<false>, grid_sel, SEL_T, sel_sm, s, pdl, p, req_ids, n_req,
+            actions, out);
   if (ev) cudaEventRecord(ev, s);
-  if (p.d == 128) gp_launch(gp_compact_kernel<128>, grid_compact, CT, 0, s, pdl, p, req_ids, n_req);
-  else gp_launch(gp_compact_kernel<64>, grid_compact, CT, 0, s, pdl, p, req_ids, n_req);
+  gp_launch(compact_kernel_of(p), grid_compact, CT, 0, s, pdl, p, req_ids, n_req);
 }

@@ -59,9 +59,11 @@ struct GpDev {
   int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;
   long long n_pages, max_batch_tokens;
   double beta_s, beta_l, top_p, tau, rope_theta;
-  int policy;                            // GP_POLICY_* (0 demand, 1 inverse, 2 random)
+  int policy;                            // GP_POLICY_* (0 demand, 1 inverse, 2 random, 3 shrink)
   unsigned long long policy_seed;
   double p_compress;
+  double shrink_below;                   // Eq. 13: Shrink under this
+  int min_pages_after_shrink;            // a Shrink must leave at least this many pages (the minimum capacity)
   unsigned long long p_fix;              // top_p in 2^62 fixed point
   // pool
   __nv_bfloat16* kv;
@@ -97,6 +99,7 @@ struct GpDev {
   double* zstat;                         // [L*H_kv][max_batch_tokens / b][2][G][2] per-page softmax partials (max, sum)
   int* sum_par;                          // [M] which of the two summary buffers is current
   int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
+  int* evict2;                           // [M][L*H_kv][2b] slots a Shrink evicts, ascending (Shrink policy only)
   int* cflags;                           // compaction chunk flags, stamped with the step number
   double* rope_cs;                       // [M][d/2][2] cos, sin at the step's position
   float* partials;

@@ -51,7 +51,7 @@ namespace {
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
       b_flags, mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
-      evict, cflags, rope_cs, partials, scores, counters, dbg,
+      evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
   int max_rc;
   long long max_batch_tokens;
@@ -83,8 +83,9 @@ bool valid_config(const gp_config* c) {
   if (!(c->beta_s >= 0.0 && c->beta_s < 1.0 && c->beta_l >= 0.0 && c->beta_l < 1.0)) return false;
   if (!(c->top_p > 0.0 && c->top_p < 1.0)) return false;
   if (!(c->rope_theta >= 0.0)) return false;
-  if (c->policy < GP_POLICY_DEMAND || c->policy > GP_POLICY_RANDOM) return false;
+  if (c->policy < GP_POLICY_DEMAND || c->policy > GP_POLICY_SHRINK) return false;
   if (!(c->p_compress >= 0.0 && c->p_compress <= 1.0)) return false;
+  if (c->min_capacity < 0 || !(c->shrink_below == c->shrink_below)) return false;
   return true;
 }
 
@@ -123,10 +124,11 @@ Layout make_layout(const gp_config& c) {
   L.qtil = take(M * LH * 2 * (size_t)G * d * 8);
   L.zstat = take(LH * ((size_t)L.max_batch_tokens / b + 1) * 2 * G * 2 * 8);
   L.evict = take(M * LH * b * 4);
+  L.evict2 = take(c.policy == GP_POLICY_SHRINK ? M * LH * 2 * b * 4 : 16);
   L.cflags = take(LH * ((size_t)L.max_batch_tokens / GP_MOVE_TOK + 2 * M + 1) * 4);
   L.rope_cs = take(M * (d / 2) * 2 * 8);
   L.partials = take((size_t)L.max_rc * LH * G * (d + 2) * 4);
-  L.scores = take(3 * LH * (size_t)L.max_batch_tokens * 8);
+  L.scores = take((c.policy == GP_POLICY_SHRINK ? 4 : 3) * LH * (size_t)L.max_batch_tokens * 8);
   L.counters = take(16 * 8);
   L.dbg = take(cap * b * (4 + 2 * d * 2));
   if (c.host_staging) {
@@ -565,6 +567,8 @@ int gp_config_default(gp_config* cfg) {
   cfg->policy = GP_POLICY_DEMAND;
   cfg->policy_seed = 0;
   cfg->p_compress = 0.7;
+  cfg->shrink_below = -0.005;
+  cfg->min_capacity = 1024;
   return GP_OK;
 }
 
@@ -606,6 +610,11 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.z_stride = (L.max_batch_tokens + GP_PAGE - 1) / GP_PAGE * GP_PAGE;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
   d.policy = cfg->policy; d.policy_seed = (unsigned long long)(unsigned)cfg->policy_seed; d.p_compress = cfg->p_compress;
+  d.shrink_below = cfg->shrink_below;
+  {
+    const long long mp = (cfg->min_capacity + GP_PAGE - 1) / GP_PAGE;      // (P - 1) b >= min_capacity
+    d.min_pages_after_shrink = (int)(mp > (1 << 21) ? (1 << 21) : (mp < 2 ? 2 : mp));
+  }
   d.p_fix = (unsigned long long)llrint(cfg->top_p * 4611686018427387904.0);
   d.kv = reinterpret_cast<__nv_bfloat16*>(base + L.kv);
   d.tok = reinterpret_cast<int*>(base + L.tok);
@@ -638,6 +647,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.zstat = reinterpret_cast<double*>(base + L.zstat);
   d.sum_par = reinterpret_cast<int*>(base + L.sum_par);
   d.evict = reinterpret_cast<int*>(base + L.evict);
+  d.evict2 = reinterpret_cast<int*>(base + L.evict2);
   d.cflags = reinterpret_cast<int*>(base + L.cflags);
   d.rope_cs = reinterpret_cast<double*>(base + L.rope_cs);
   d.partials = reinterpret_cast<float*>(base + L.partials);

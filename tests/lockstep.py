@@ -50,7 +50,8 @@ def make_pools(wl: W.Workload, device: int = 0, **over):
     s = wl.shape
     kw = dict(n_pages=wl.n_pages, max_pages_per_req=wl.max_pages_per_req,
               max_requests=max(4, wl.n_resident), k_loc=wl.k_loc)
-    tun = {k: over[k] for k in ("beta_s", "beta_l", "top_p", "tau", "rope_theta", "policy", "policy_seed", "p_compress")
+    tun = {k: over[k] for k in ("beta_s", "beta_l", "top_p", "tau", "rope_theta", "policy", "policy_seed", "p_compress",
+                                    "shrink_below", "min_capacity")
            if k in over}
     for k in ("n_pages", "max_pages_per_req", "k_loc", "max_requests"):
         if k in over:
@@ -140,20 +141,25 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
                     assert info.action_near_tie, f"step {st.steps} req {rid}: grow decision differs outside a near-tie"
                     st.near_ties["act"] += 1
                     overrides.setdefault(rid, {})["want_grow"] = g_want
+                g_shrink = int(g_act[i]) == B.GP_ACT_SHRINK
+                if int(g_act[i]) in (B.GP_ACT_COMPRESS, B.GP_ACT_SHRINK) and g_shrink != info.want_shrink:
+                    assert info.action_near_tie, f"step {st.steps} req {rid}: shrink decision differs outside a near-tie"
+                    st.near_ties["act"] += 1
+                    overrides.setdefault(rid, {})["want_shrink"] = g_shrink
             # ---- retained sets of the requests the GPU compressed -----------------------------------------------
             for rid, info in rec.boundary.items():
                 i = rids.index(rid)
-                if int(g_act[i]) not in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK):
+                if int(g_act[i]) not in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK, B.GP_ACT_SHRINK):
                     continue
                 r = ora.requests[rid]
-                K_t = info.n_c - b
+                K_t = info.n_c - (2 * b if int(g_act[i]) == B.GP_ACT_SHRINK else b)    # Eq. 13: a Shrink evicts two pages
                 for l in range(s.n_layers):
                     for h in range(s.n_kv_heads):
                         st.decisions["sel"] += 1
                         keep, margin = O.select_retained(O.token_scores(info.a_s[l, h], info.a_l[l, h]),
                                                          r.P - 1, b, K_t, ora.cfg.k_loc)
                         want_tok = r.tok[l, h, keep]
-                        got = B.gp_debug_retained(gpu.handle, rid, l, h, info.n_c)
+                        got = B.gp_debug_retained(gpu.handle, rid, l, h, K_t + b)
                         got_hist, got_prot = got[:K_t], got[K_t:]
                         assert np.array_equal(got_prot, r.tok[l, h, info.n_c:info.n_c + b]), "protected page lost"
                         if not np.array_equal(got_hist, want_tok):
@@ -200,7 +206,7 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
         assert st.attn_mean_abs <= ATTN_MEAN_ABS, f"attention mean abs err {st.attn_mean_abs}"
         assert st.summary_max_rel <= SUMMARY_REL
         for name, gi in (("grow", 0), ("compress", 1), ("fallback", 2), ("stalled", 3), ("cow_pages", 4),
-                         ("moved_rows", 8), ("scored_tokens", 9)):
+                         ("moved_rows", 8), ("scored_tokens", 9), ("shrink", 10)):
             assert int(st.counters[gi]) == ora.counters[name], f"counter {name}: gpu {st.counters[gi]} oracle {ora.counters[name]}"
     finally:
         gpu.close()

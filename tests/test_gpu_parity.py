@@ -60,10 +60,10 @@ def test_other_quota_and_coverage_settings():
     _report("tiny k_loc=16", st)
 
 
-def _single_request_case(shape, n_prompt, n_steps, seed=11):
+def _single_request_case(shape, n_prompt, n_steps, seed=11, **over):
     wl = W.Workload("adhoc", seed, shape, [W.RequestSpec(0, n_prompt, n_steps, 0.05)], n_resident=1, initial_pages=0,
                     max_pages_per_req=n_prompt // 16 + 4, n_pages=n_prompt // 16 + 8)
-    return LS.run_lockstep(wl, tau=-1.0)
+    return LS.run_lockstep(wl, **(over or dict(tau=-1.0)))
 
 
 @pytest.mark.parametrize("hq,hkv,d,n_prompt", [(32, 8, 128, 1530), (64, 8, 128, 777), (4, 4, 64, 1100),
@@ -197,15 +197,19 @@ def test_synchronised_boundaries_put_several_boundary_items_on_every_cta():
     assert st.actions.get(B.GP_ACT_COMPRESS, 0) + st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) > 0
 
 
-def test_equal_scores_take_the_general_selection_paths():
+@pytest.mark.parametrize("shrink", [False, True])
+def test_equal_scores_take_the_general_selection_paths(shrink):
     # zero queries: summaries and calibrated summaries are zero, every candidate gets the same probability, so
     # the single-histogram fast paths find one crowded bin and hand over to the general radix descent; ties are
-    # broken by slot order on both sides (Eq. 7 by count, Eq. 10 keeps the older slots)
+    # broken by slot order on both sides (Eq. 7 by count, Eq. 10 keeps the older slots).  Once with Compress &
+    # Hold, once with the Shrink policy set so that Delta_t = 0 shrinks (two pages worth go).
     import torch
     L, Hq, Hkv, d, n_prompt, steps = 1, 4, 2, 64, 100, 70
     kw = dict(n_pages=16, max_pages_per_req=9, max_requests=4, k_loc=2)
-    gpu = B.Pool(B.make_config(L, Hq, Hkv, d, tau=1.0, **kw))
-    ora = O.OraclePool(O.OracleConfig(L, Hq, Hkv, d, tau=1.0, **kw))
+    pol = dict(policy=B.GP_POLICY_SHRINK, shrink_below=0.5, min_capacity=48) if shrink else {}
+    n_ev = 32 if shrink else 16
+    gpu = B.Pool(B.make_config(L, Hq, Hkv, d, tau=1.0, **kw, **pol))
+    ora = O.OraclePool(O.OracleConfig(L, Hq, Hkv, d, tau=1.0, **kw, **pol))
     try:
         rng = np.random.default_rng(5)
         bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
@@ -226,14 +230,15 @@ def test_equal_scores_take_the_general_selection_paths():
             for rid, info in rec.boundary.items():
                 ks, kl, delta = B.gp_debug_boundary(gpu.handle, 0, L, Hkv)
                 assert np.array_equal(ks, info.K_s) and np.array_equal(kl, info.K_l) and delta == info.delta
-                if int(act.cpu()[0]) in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK):
+                if int(act.cpu()[0]) in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK, B.GP_ACT_SHRINK):
+                    assert (int(act.cpu()[0]) == B.GP_ACT_SHRINK) == (shrink and info.n_c >= 48)
                     n_compress += 1
                     r = ora.requests[0]
-                    K_t = info.n_c - 16
+                    K_t = info.n_c - (n_ev if int(act.cpu()[0]) == B.GP_ACT_SHRINK else 16)
                     for l in range(L):
                         for h in range(Hkv):
                             keep, _ = O.select_retained(O.token_scores(info.a_s[l, h], info.a_l[l, h]), r.P - 1, 16, K_t, 2)
-                            got = B.gp_debug_retained(gpu.handle, 0, l, h, info.n_c)
+                            got = B.gp_debug_retained(gpu.handle, 0, l, h, K_t + 16)
                             assert np.array_equal(got[:K_t], r.tok[l, h, keep]), f"step {t} ({l},{h}): retained set differs"
             ora.step_apply(rec, {})
             assert int(act.cpu()[0]) == int(rec.actions[0]), f"step {t}"
@@ -249,6 +254,22 @@ def test_candidate_set_larger_than_the_staging_buffers():
     st = _single_request_case(W.Shape(1, 4, 2, 64), 6300, 80)
     _report("6300-token prompt", st)
     assert st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) >= 1
+
+
+def test_shrink_at_the_default_floor_and_beyond_the_staging_buffers():
+    # every admissible boundary shrinks (shrink_below above any Delta_t).  With the default minimum capacity of
+    # 1024 tokens a 1530-token request shrinks; a 6300-token one takes the Shrink's eviction list through the
+    # global score scratch
+    always = dict(policy=B.GP_POLICY_SHRINK, shrink_below=0.5, tau=1.0)
+    st = _single_request_case(W.Shape(2, 32, 8, 128), 1530, 40, **always)
+    _report("1530-token prompt, shrink", st)
+    assert st.actions.get(B.GP_ACT_SHRINK, 0) >= 2 and st.actions.get(B.GP_ACT_COMPRESS, 0) == 0
+    st = _single_request_case(W.Shape(1, 4, 2, 64), 1030, 40, **always)       # 65 pages: one Shrink, then the floor
+    _report("1030-token prompt, shrink", st)
+    assert st.actions.get(B.GP_ACT_SHRINK, 0) == 1 and st.actions.get(B.GP_ACT_COMPRESS, 0) >= 1
+    st = _single_request_case(W.Shape(1, 4, 2, 64), 6300, 50, **always)
+    _report("6300-token prompt, shrink", st)
+    assert st.actions.get(B.GP_ACT_SHRINK, 0) >= 2
 
 
 def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches():
@@ -316,6 +337,25 @@ def test_inverse_and_random_capacity_control_policies(over):
     if over["policy"] == B.GP_POLICY_RANDOM:
         frac = comps / max(grows + comps, 1)
         assert abs(frac - over.get("p_compress", 0.7)) < 0.25
+
+
+@pytest.mark.parametrize("config,over,mixed", [
+    (1, dict(min_capacity=64), False),                 # the paper's thresholds: the floor stops most Shrinks
+    (1, dict(min_capacity=48, tau=-0.06, shrink_below=-0.085), True),
+    (5, dict(min_capacity=64), False),                 # shared prompt pages: copy-on-write before a Shrink writes
+    (5, dict(min_capacity=64, tau=-0.03, shrink_below=-0.036), True)])
+def test_shrink_policy_of_eq13(config, over, mixed):
+    """Three-way capacity control: grants, Compress & Hold, and Shrinks that evict two pages worth per (layer,
+    head) and hand a page back, against the oracle step by step (actions, retained sets, page tables, free list,
+    reference counts).  The thresholds of the mixed cases sit inside the range Delta_t takes on these inputs, so
+    that all three actions occur."""
+    st = LS.run_lockstep(W.parity_instance(config), policy=B.GP_POLICY_SHRINK, **over)
+    _report(f"config {config} shrink {over}", st)
+    assert st.actions.get(B.GP_ACT_SHRINK, 0) > 0 and st.counters[10] == st.actions[B.GP_ACT_SHRINK]
+    if mixed:
+        assert st.actions.get(B.GP_ACT_GROW, 0) > 0 and st.actions.get(B.GP_ACT_COMPRESS, 0) > 0
+    if config == 5:
+        assert st.counters[4] > 0
 
 
 def test_layer_by_layer_entry_points_equal_the_whole_step():
