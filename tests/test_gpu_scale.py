@@ -67,8 +67,11 @@ def _pool_accounting(gpu, cfg, live):
 
 # tau below zero makes part of the boundaries ask for a page (with the synthetic streams Delta_t is seldom
 # positive), so that grants, fallbacks under an empty free list and stalls all occur
-@pytest.mark.parametrize("name,tau", [("stack8b", -0.05), ("stack32b", -0.03), ("prefix", 0.0), ("prefix", -0.05)])
-def test_invariants_under_continuous_batching(name, tau):
+@pytest.mark.parametrize("name,tau,shrink_below", [("stack8b", -0.05, None), ("stack32b", -0.03, None),
+                                                  ("prefix", 0.0, None), ("prefix", -0.05, None),
+                                                  ("stack8b", -0.04, -0.06), ("prefix", 0.0, -0.005)])
+def test_invariants_under_continuous_batching(name, tau, shrink_below):
+    """shrink_below set: the three-way Shrink policy (Eq. 13) with a 256-token minimum capacity."""
     import torch
 
     wl = _instance(name, tau)
@@ -78,6 +81,8 @@ def test_invariants_under_continuous_batching(name, tau):
     dev = "cuda:0"
     cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
                         max_pages_per_req=wl.max_pages_per_req, max_requests=max(4, wl.n_resident), k_loc=wl.k_loc, tau=tau,
+                        **(dict(policy=B.GP_POLICY_SHRINK, shrink_below=shrink_below, min_capacity=256)
+                           if shrink_below is not None else {}),
                         # shared prompt pages count once in the pool but once per request in a batch
                         max_batch_tokens=wl.n_resident * wl.max_pages_per_req * b)
     gpu = B.Pool(cfg, 0)
@@ -85,7 +90,7 @@ def test_invariants_under_continuous_batching(name, tau):
     rng = np.random.default_rng(7)
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev)
     steps = tokens = 0
-    seen = {k: 0 for k in ("none", "grow", "compress", "fallback", "stalled", "attn", "retained")}
+    seen = {k: 0 for k in ("none", "grow", "compress", "fallback", "shrink", "stalled", "attn", "retained")}
     compacted = set()
     try:
         while not sch.done():
@@ -130,6 +135,11 @@ def test_invariants_under_continuous_batching(name, tau):
                     assert (P1, n1, pos1) == (P0, (P0 - 1) * b, pos0 + 1), (steps, rid, a, P0, n0, P1, n1)
                     seen["compress" if a == B.GP_ACT_COMPRESS else "fallback"] += 1
                     compacted.add(rid)
+                elif a == B.GP_ACT_SHRINK:
+                    assert shrink_below is not None and (P0 - 1) * b >= 256
+                    assert (P1, n1, pos1) == (P0 - 1, (P0 - 2) * b, pos0 + 1), (steps, rid, P0, n0, P1, n1)
+                    seen["shrink"] += 1
+                    compacted.add(rid)
                 else:
                     assert a == B.GP_ACT_STALLED, f"step {steps} request {rid}: action {a} at a boundary"
                     seen["stalled"] += 1
@@ -170,13 +180,15 @@ def test_invariants_under_continuous_batching(name, tau):
         n_free, ref, counters = B.gp_debug_pool(gpu.handle, cfg.n_pages)
         assert counters[7] == 0 and counters[5] == steps and counters[6] == tokens
         assert n_free == cfg.n_pages and not ref.any(), "pages leaked after every request was released"
-        print(f"\n{name} tau={tau}: {steps} steps, {tokens} tokens, {seen}, cow pages {counters[4]}")
+        print(f"\n{name} tau={tau} shrink_below={shrink_below}: {steps} steps, {tokens} tokens, {seen}, cow pages {counters[4]}")
         assert seen["attn"] > 100
         if tau < 0:
             assert seen["grow"] > 0
         else:
-            assert seen["compress"] > 0
-        if name == "stack8b" or (name == "prefix" and tau < 0):
+            assert seen["compress"] + seen["shrink"] > 0
+        if shrink_below is not None:
+            assert seen["shrink"] > 0 and counters[10] == seen["shrink"]
+        if (name == "stack8b" and shrink_below is None) or (name == "prefix" and tau < 0):
             assert seen["fallback"] + seen["stalled"] > 0, "the pool never ran dry: no pressure in this instance"
         if name == "prefix":
             assert counters[4] > 0, "no copy-on-write happened"
