@@ -48,6 +48,13 @@ def _instance(name: str, tau: float) -> W.Workload:
             wl.max_pages_per_req = 65 + 5
             wl.n_pages = 6 * 64 + 48 * 6 + 640
         return wl
+    if name == "many":
+        # the most requests a pool takes (512), short sequences, dozens of boundaries in every step, a pool that
+        # runs dry: the planning, decision and compaction bookkeeping at their widest
+        g = np.random.default_rng(5)
+        reqs = [W.RequestSpec(i, int(g.integers(1, 61)), int(g.integers(24, 57)), 0.05) for i in range(640)]
+        return W.Workload("many", 5, W.Shape(2, 8, 2, 64), reqs, n_resident=512, initial_pages=0,
+                          max_pages_per_req=6, n_pages=512 * 3 + 100)
     raise ValueError(name)
 
 
@@ -69,7 +76,8 @@ def _pool_accounting(gpu, cfg, live):
 # positive), so that grants, fallbacks under an empty free list and stalls all occur
 @pytest.mark.parametrize("name,tau,shrink_below", [("stack8b", -0.05, None), ("stack32b", -0.03, None),
                                                   ("prefix", 0.0, None), ("prefix", -0.05, None),
-                                                  ("stack8b", -0.04, -0.06), ("prefix", 0.0, -0.005)])
+                                                  ("stack8b", -0.04, -0.06), ("prefix", 0.0, -0.005),
+                                                  ("many", -0.05, None), ("many", -0.03, -0.06)])
 def test_invariants_under_continuous_batching(name, tau, shrink_below):
     """shrink_below set: the three-way Shrink policy (Eq. 13) with a 256-token minimum capacity."""
     import torch
@@ -81,7 +89,7 @@ def test_invariants_under_continuous_batching(name, tau, shrink_below):
     dev = "cuda:0"
     cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
                         max_pages_per_req=wl.max_pages_per_req, max_requests=max(4, wl.n_resident), k_loc=wl.k_loc, tau=tau,
-                        **(dict(policy=B.GP_POLICY_SHRINK, shrink_below=shrink_below, min_capacity=256)
+                        **(dict(policy=B.GP_POLICY_SHRINK, shrink_below=shrink_below, min_capacity=48 if name == "many" else 256)
                            if shrink_below is not None else {}),
                         # shared prompt pages count once in the pool but once per request in a batch
                         max_batch_tokens=wl.n_resident * wl.max_pages_per_req * b)
@@ -136,7 +144,7 @@ def test_invariants_under_continuous_batching(name, tau, shrink_below):
                     seen["compress" if a == B.GP_ACT_COMPRESS else "fallback"] += 1
                     compacted.add(rid)
                 elif a == B.GP_ACT_SHRINK:
-                    assert shrink_below is not None and (P0 - 1) * b >= 256
+                    assert shrink_below is not None and (P0 - 1) * b >= cfg.min_capacity
                     assert (P1, n1, pos1) == (P0 - 1, (P0 - 2) * b, pos0 + 1), (steps, rid, P0, n0, P1, n1)
                     seen["shrink"] += 1
                     compacted.add(rid)
