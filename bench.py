@@ -139,14 +139,14 @@ class ClockSampler:
 # our arm
 # --------------------------------------------------------------------------------------------------
 class Job:
-    def __init__(self, wl, torch, device, q_all, k_all, v_all, prompts, host_staging=True):
+    def __init__(self, wl, torch, device, q_all, k_all, v_all, prompts, host_staging=True, policy=0):
         from paper_2609_03494_b200 import binding as B
         self.B, self.torch, self.wl, self.device = B, torch, wl, device
         s = wl.shape
         self.nreq = len(wl.requests)
         cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
                             max_pages_per_req=wl.max_pages_per_req, max_requests=max(4, self.nreq), k_loc=wl.k_loc,
-                            host_staging=host_staging)
+                            host_staging=host_staging, policy=policy)
         self.pool = B.Pool(cfg, device)
         dev = f"cuda:{device}"
         self.q_host, self.k_host, self.v_host = q_all, k_all, v_all
@@ -204,8 +204,11 @@ class Job:
         self.n = n_new
         grow = actions == B.GP_ACT_GROW
         comp = (actions == B.GP_ACT_COMPRESS) | (actions == B.GP_ACT_COMPRESS_FALLBACK)
+        shrink = actions == B.GP_ACT_SHRINK
         self.P = self.P + grow
         self.n = np.where(comp, (self.P - 1) * 16, self.n)
+        self.n = np.where(shrink, (self.P - 2) * 16, self.n)
+        self.P = self.P - shrink
         return attn, score
 
     def moved_rows(self):
@@ -233,7 +236,8 @@ def run_ours(args):
     t_gen = time.time()
     q_all, k_all, v_all, prompts = generate_inputs(wl, S0 + K, torch, pin=True)
     t_gen = time.time() - t_gen
-    job = Job(wl, torch, device, q_all, k_all, v_all, prompts)
+    policy = {"demand": 0, "inverse": 1, "random": 2, "shrink": 3}[args.policy]
+    job = Job(wl, torch, device, q_all, k_all, v_all, prompts, policy=policy)
     job.by_layer = args.entry == "layers"
     B = job.B
     stream = torch.cuda.current_stream(device)
@@ -345,7 +349,7 @@ def run_ours(args):
                                    ("qwen3-8b-layer: L=1, 32q/8kv heads, d=128, page 16, 64 requests x 4096 decode steps, "
                                     "prompts U[128,1024], heavy-hitter fraction logU[0.5%,20%], seed 1"),
                        "entry": "gp_decode_step" if not job.by_layer else "gp_step_begin + gp_attn_layer per layer + gp_step_end",
-                       "requests_per_gpu": job.nreq, "timed_steps": [S0, S0 + K], "job_steps": job_steps,
+                       "policy": args.policy, "requests_per_gpu": job.nreq, "timed_steps": [S0, S0 + K], "job_steps": job_steps,
                        "l2": "per-step working set (all resident K/V) is larger than L2; no flush needed",
                        "input_generation_s": round(t_gen, 1)},
             "roofline": roofline, "step_roofline": step_roofline,
@@ -355,7 +359,7 @@ def run_ours(args):
             "gpu_launches": int(gpu_launches),
             "clocks": clocks,
             "events": {"grow": int(counters[0]), "compress": int(counters[1]), "fallback": int(counters[2]),
-                       "stalled": int(counters[3])},
+                       "stalled": int(counters[3]), "shrink": int(counters[10])},
         }
         print(json.dumps(line))
     job.pool.close()
@@ -441,6 +445,8 @@ def main():
                     help="step: gp_decode_step; layers: the same step through gp_step_begin / gp_attn_layer / gp_step_end")
     ap.add_argument("--workload", default="layer", choices=["layer", "stack"],
                     help="layer: the headline one-layer Qwen3-8B-shaped workload; stack: the 36-layer shape, 16 resident requests")
+    ap.add_argument("--policy", default="demand", choices=["demand", "inverse", "random", "shrink"],
+                    help="capacity-control policy (the paper's default, or one of its ablation's controls)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
