@@ -420,3 +420,56 @@ def test_layer_by_layer_entry_points_equal_the_whole_step():
     assert all(np.array_equal(a, b_) for a, b_ in zip(whole[4], layered[4]))
     assert np.array_equal(whole[0], layered[0])
     assert (whole[1] == B.GP_ACT_GROW).any() and (whole[1] == B.GP_ACT_COMPRESS).any()
+
+
+def test_results_do_not_depend_on_batch_order_or_on_the_run():
+    # The same steps three times: ids ascending, ids ascending again (run-to-run determinism: the histograms use
+    # integer atomics only and every floating-point sum has a fixed order), and the batch in a different random
+    # order every step (a request's result does not depend on its position in the batch or on its neighbours):
+    # outputs, actions, page tables, retained sets and summaries must be equal bit for bit.
+    import torch
+    shape = W.Shape(2, 8, 2, 64)
+    reqs = [W.RequestSpec(i, 90 + 53 * i, 70, 0.05) for i in range(7)]
+    wl = W.Workload("order", 37, shape, reqs, n_resident=7, initial_pages=0, max_pages_per_req=40, n_pages=7 * 40)
+    s, n, T = shape, 7, 70
+    q = np.empty((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=np.uint16)
+    k = np.empty((T, s.n_layers, n, s.n_kv_heads, s.head_dim), dtype=np.uint16)
+    v = np.empty_like(k)
+    prompts = []
+    for i in range(n):
+        st = wl.stream(reqs[i])
+        prompts.append(st.prompt_kv())
+        q[:, :, i], k[:, :, i], v[:, :, i] = st.steps(0, T)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to("cuda:0")
+    rng = np.random.default_rng(1)
+    results = []
+    for mode in ("sorted", "sorted", "shuffled"):
+        pool = B.Pool(B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
+                                    max_pages_per_req=40, max_requests=8, tau=-0.05))
+        try:
+            for i in range(n):
+                assert pool.request_add(-1, 0, prompts[i][0], prompts[i][1], reqs[i].prompt_len, 0)[0] == B.GP_OK
+            outs = np.zeros((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=np.float32)
+            acts = np.zeros((T, n), dtype=np.int32)
+            for t in range(T):
+                perm = rng.permutation(n) if mode == "shuffled" else np.arange(n)
+                ids = torch.tensor(perm, dtype=torch.int32, device="cuda:0")
+                out = torch.zeros((s.n_layers, n, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda:0")
+                act = torch.zeros(n, dtype=torch.int32, device="cuda:0")
+                pool.decode_step(ids, dev(q[t][:, perm]), dev(k[t][:, perm]), dev(v[t][:, perm]), out, act)
+                outs[t][:, perm] = out.cpu().numpy()
+                acts[t][perm] = act.cpu().numpy()
+            state = [B.gp_debug_request(pool.handle, i, 40) for i in range(n)]
+            kept = [B.gp_debug_retained(pool.handle, i, 1, 1, state[i][1]) for i in range(n)]
+            summ = [B.gp_debug_summaries(pool.handle, i, s.n_layers, s.n_q_heads, s.head_dim) for i in range(n)]
+            assert B.gp_debug_pool(pool.handle)[2][7] == 0
+            results.append((outs, acts, state, kept, summ))
+        finally:
+            pool.close()
+    first = results[0]
+    assert (first[1] == B.GP_ACT_GROW).any() and (first[1] == B.GP_ACT_COMPRESS).any()
+    for other in results[1:]:
+        assert np.array_equal(first[1], other[1]) and first[2] == other[2]
+        assert all(np.array_equal(a, b_) for a, b_ in zip(first[3], other[3]))
+        assert all(np.array_equal(a, b_) for a, b_ in zip(first[4], other[4]))
+        assert np.array_equal(first[0], other[0])
