@@ -1,23 +1,28 @@
 // Capacity-boundary kernels (Sec. 3.2 - 3.3, App. D.1, App. D.2), launched every step after attention.
-// The attention kernel has already left, for every (request at a boundary, layer, KV head) unit, the
-// fp64 logits z of the two calibrated summaries against every candidate key.
+// The attention kernel has already left, for every (request at a boundary, layer, KV head) unit and both
+// calibrated summaries, exp(logit - the page's maximum logit) of every candidate key, and per 16-token page
+// the maximum and the sum of those exponentials.
 //
-//   gp_bsel_kernel    first merges the partial attention outputs of requests split over several work items;
-//                     then, per unit: per-head softmax over the candidate set and group mean -> a^S, a^L;
-//                     working-set sizes K^S, K^L (Eq. 7); and, speculatively, the b slots a compression
-//                     would evict (Eq. 9, Eq. 10).  The last CTA to finish aggregates Eq. 8, decides grow
-//                     or compress per request and runs the device allocator: grants first, then
+//   gp_bsel_kernel    per unit, three independent jobs, one CTA each: per-head softmax over the candidate
+//                     set and group mean -> a^S or a^L and its working-set size K^S or K^L (Eq. 7); and,
+//                     speculatively, the b slots a compression would evict (Eq. 9, Eq. 10).  Under the
+//                     Shrink policy a fourth job lists the 2b slots a Shrink would evict (Eq. 13).  CTAs
+//                     without a job merge the partial attention outputs of requests that were split over
+//                     several work items.  The last CTA to finish aggregates Eq. 8, decides per request
+//                     (grow, compress, shrink) and runs the device allocator: grants first, then
 //                     copy-on-write targets, each in ascending request id.
 //   gp_compact_kernel per (compressing unit, chunk of 64 source slots): stable in-place compaction into
-//                     (P-1) b slots, writing to copy-on-write targets where the source page is shared.
-//                     Chunks are claimed in order from a ticket counter; a chunk publishes "my sources
-//                     are read" before the next chunk may overwrite their tail.  The last CTA swaps in the
-//                     target pages and drops the references to the replaced ones.
+//                     (P-1) b slots ((P-2) b at a Shrink), writing to copy-on-write targets where the
+//                     source page is shared.  Chunks are claimed in order from a ticket counter; a chunk
+//                     publishes "my sources are read" before the next chunk may overwrite their tail.  The
+//                     last CTA swaps in the target pages, drops the references to the replaced ones and
+//                     returns the last page of every request that shrank.
 //
-// Everything that decides an integer outcome is fp64.  Top-p counting and top-k selection are radix
-// descents over the IEEE bit patterns of the (non-negative) scores, 11 bits per level, with histograms in
-// shared memory; the top-p mass is accumulated in 2^62 fixed point with integer atomics, so the result
-// does not depend on the order in which threads add.
+// Everything that decides an integer outcome is fp64.  Top-p counting and the eviction cut work on the
+// IEEE bit patterns of the (non-negative) scores: one pass into a two-level histogram (4096 fine bins under
+// 256 coarse ones) when the scores' top bits are uniform, else a radix descent, 11 bits per level; the
+// histograms live in shared memory, and the top-p mass is accumulated in 2^62 fixed point with integer
+// atomics, so the result does not depend on the order in which threads add.
 #include "../../include/growpage.h"
 #include "gp_dev.cuh"
 
