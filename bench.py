@@ -363,6 +363,7 @@ def run_ours(args):
         }
         print(json.dumps(line))
     job.pool.close()
+    shard.finish()
 
 
 # --------------------------------------------------------------------------------------------------

@@ -24,6 +24,14 @@ def init(backend: str) -> Tuple[int, int, int]:
     return rank, local_rank, world
 
 
+def finish() -> None:
+    """Leaves the process group (a no-op for a single process)."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def shard_seed(base_seed: int, rank: int) -> int:
     """Weak scaling: rank r decodes its own set of requests, drawn with this seed.  Rank 0 keeps the
     configuration's own seed."""

@@ -35,6 +35,8 @@ def test_two_gloo_ranks_agree_on_job_throughput():
         assert ms == 150.0 and abs(value - 70 / 0.150) < 1e-9, (value, ms)
         assert shard.max_over_ranks(rank) == 1.0 and shard.sum_over_ranks(1.0) == 2.0
         shard.barrier()
+        shard.finish()
+        shard.finish()                     # idempotent
         print("rank", rank, "ok")
     """ % ROOT)
     procs = []
