@@ -410,7 +410,7 @@ def time_oracle(wl, n_requests: int, n_steps: int, warmup: int, budget_s: float 
     return {"value": round(done * n_requests / wall, 2), "unit": "tokens/s", "cores": cores, "kind": "oracle",
             "sample": f"first {n_requests} requests of the workload, decode steps {warmup}..{warmup + done} of the job "
                       f"(float64 numpy, {os.cpu_count()} host cores present, timed region excludes input decoding)",
-            "steps": done, "wall_s": round(wall, 2)}
+            "steps": done, "wall_s": round(wall, 4)}
 
 
 def run_reference(args):
