@@ -755,8 +755,18 @@ __device__ __noinline__ bool job_softmax(const GpDev& p, const double* __restric
     }
   }
   if (tid == 0) { GP_T_ADD(12, j1 - j0); GP_T_ADD(13, j2 - j1); GP_T_ADD(14, GP_T_NOW() - j2); GP_T_ADD(30, 1); }
-  // bits 62..58 of every score, as a set: the fast selection path needs them all equal
-  return __popc(__syncthreads_or((int)top_bits)) == 1;
+  // bits 62..58 of every score, as a set: the fast selection path needs them all equal.  (The block-wide
+  // barrier reductions combine predicates, not words, so the sets are OR-ed by hand: per warp, then over the
+  // warps through shared memory; `red` is free here.)
+  top_bits = __reduce_or_sync(0xffffffffu, top_bits);
+  unsigned* sets = reinterpret_cast<unsigned*>(red);
+  if ((tid & 31) == 0) sets[tid >> 5] = top_bits;
+  __syncthreads();
+  unsigned all_bits = 0;
+#pragma unroll
+  for (int w = 0; w < SEL_NW; ++w) all_bits |= sets[w];
+  __syncthreads();
+  return __popc(all_bits) == 1;
 }
 
 // Attention outputs of requests that were split over several work items: merges the items' partial results

@@ -473,3 +473,38 @@ def test_results_do_not_depend_on_batch_order_or_on_the_run():
         assert all(np.array_equal(a, b_) for a, b_ in zip(first[3], other[3]))
         assert all(np.array_equal(a, b_) for a, b_ in zip(first[4], other[4]))
         assert np.array_equal(first[0], other[0])
+
+
+class _ScaledStream:
+    """A request's inputs with queries and keys multiplied by a power of two (exact in bf16)."""
+
+    def __init__(self, inner, q_scale, k_scale):
+        self.inner, self.q_scale, self.k_scale = inner, q_scale, k_scale
+
+    @staticmethod
+    def _mul(bits, f):
+        return W.f32_to_bf16_bits((W.bf16_bits_to_f64(bits) * f).astype(np.float32))
+
+    def prompt_kv(self):
+        k, v = self.inner.prompt_kv()
+        return self._mul(k, self.k_scale), v
+
+    def steps(self, t0, t1):
+        q, k, v = self.inner.steps(t0, t1)
+        return self._mul(q, self.q_scale), self._mul(k, self.k_scale), v
+
+
+@pytest.mark.parametrize("config,q_scale,k_scale,steps", [(1, 16.0, 8.0, 256), (1, 16.0, 1.0, 120), (1, 64.0, 32.0, 120),
+                                                          (1, 1.0 / 64, 1.0 / 64, 120), (2, 8.0, 4.0, 40)])
+def test_saturated_and_flat_softmax(config, q_scale, k_scale, steps):
+    # Logits in the tens, hundreds or thousands: the summary probabilities of a candidate set span far more than
+    # the 2^64 range the one-pass selection handles (many underflow to denormals or exactly zero, a mass of equal
+    # scores under a few large ones), so working sets and eviction lists come from the general radix descent;
+    # softmaxes are one-hot up to rounding and working sets hold a few tokens.  And logits near zero: uniform
+    # attention, working sets of about p |C|.  All against the oracle, ties by slot order.
+    wl = W.parity_instance(config)
+    plain = wl.stream
+    object.__setattr__(wl, "stream", lambda spec: _ScaledStream(plain(spec), q_scale, k_scale))
+    st = LS.run_lockstep(wl, max_steps=steps)
+    _report(f"config {config}, q x{q_scale}, k x{k_scale}", st)
+    assert st.decisions["sel"] > 0
