@@ -508,3 +508,22 @@ def test_saturated_and_flat_softmax(config, q_scale, k_scale, steps):
     st = LS.run_lockstep(wl, max_steps=steps)
     _report(f"config {config}, q x{q_scale}, k x{k_scale}", st)
     assert st.decisions["sel"] > 0
+
+
+@pytest.mark.parametrize("name,shape,n_prompt,over", [
+    ("rope at the 8B shape, several chunks", (2, 32, 8, 128), 1530, dict(rope_theta=1e4, tau=-0.02)),
+    ("rope, G = 8, d = 64", (2, 64, 8, 64), 700, dict(rope_theta=5e5, tau=-0.02)),
+    ("beta_S = 0: the short summary is the current query", (1, 8, 2, 64), 300, dict(beta_s=0.0, tau=-0.02)),
+    ("beta_S = beta_L: equal summaries, Delta = 0 at every boundary", (1, 8, 2, 64), 300, dict(beta_s=0.9, beta_l=0.9)),
+    ("top_p close to one", (1, 8, 2, 64), 300, dict(top_p=0.999999, tau=-0.02)),
+    ("top_p small", (1, 8, 2, 64), 300, dict(top_p=0.05, tau=-0.002)),
+    ("tau above any Delta: fixed budget", (1, 8, 2, 64), 300, dict(tau=1.5)),
+])
+def test_setting_variants_on_one_request(name, shape, n_prompt, over):
+    # the paper's ablation settings (Sec. 5, "Dual-Timescale Signal Ablation": beta_S = 0; fixed budget) and the
+    # ends of the parameter ranges, each against the oracle over several capacity boundaries
+    st = _single_request_case(W.Shape(*shape), n_prompt, 70, **over)
+    _report(name, st)
+    assert st.decisions["act"] >= 3
+    if ("beta_l" in over and over["beta_l"] == over["beta_s"]) or over.get("tau", 0) > 1:
+        assert st.actions.get(B.GP_ACT_GROW, 0) == 0
