@@ -527,3 +527,45 @@ def test_setting_variants_on_one_request(name, shape, n_prompt, over):
     assert st.decisions["act"] >= 3
     if ("beta_l" in over and over["beta_l"] == over["beta_s"]) or over.get("tau", 0) > 1:
         assert st.actions.get(B.GP_ACT_GROW, 0) == 0
+
+
+def test_sequence_lengths_around_chunk_and_page_edges():
+    # a request is cut into chunks of 32 pages (512 tokens), boundary requests into chunks of 8 pages; every
+    # length around those edges and around a page edge, a few steps each (the append crosses the edge), attention
+    # and boundary decisions against the oracle
+    lengths = list(range(505, 520)) + list(range(1018, 1030)) + [127, 128, 129, 255, 256, 257, 2047, 2048, 2049]
+    for n_prompt in lengths:
+        st = _single_request_case(W.Shape(1, 8, 2, 64), n_prompt, 3, seed=n_prompt, tau=-0.02)
+        assert st.steps == 3 and st.attn_max_abs <= LS.ATTN_MAX_ABS
+
+
+def test_host_entry_point_with_pageable_buffers():
+    # gp_decode_step_host writes pinned outputs over the bus as it runs; pageable buffers take the staged copies
+    import torch
+    cfg = B.make_config(1, 8, 2, 64, n_pages=32, max_pages_per_req=4, max_requests=8, host_staging=True)
+    results = []
+    for pinned in (True, False):
+        pool = B.Pool(cfg)
+        try:
+            rng = np.random.default_rng(0)
+            bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+            kt, vt = bits(1, 20, 2, 64), bits(1, 20, 2, 64)
+            for i in range(3):
+                assert pool.request_add(-1, 0, kt, vt, 20, 0) == (B.GP_OK, i)
+            fix = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+            outs = []
+            for t in range(14):                                   # crosses the boundary at n = 32
+                q, k, v = bits(1, 3, 8, 64), bits(1, 3, 2, 64), bits(1, 3, 2, 64)
+                out = fix(torch.zeros((1, 3, 8, 64), dtype=torch.float32))
+                act = fix(torch.zeros(3, dtype=torch.int32))
+                ids = fix(torch.arange(3, dtype=torch.int32))
+                tq, tk, tv = (fix(torch.from_numpy(x.view(np.int16))) for x in (q, k, v))
+                pool.decode_step_host(ids, tq, tk, tv, out, act)
+                outs.append((out.clone().numpy(), act.clone().numpy()))
+            results.append(outs)
+            assert B.gp_debug_pool(pool.handle)[2][7] == 0
+        finally:
+            pool.close()
+    for (o1, a1), (o2, a2) in zip(*results):
+        assert np.array_equal(o1, o2) and np.array_equal(a1, a2)
+    assert any((a != B.GP_ACT_NONE).any() for _, a in results[0])
