@@ -494,9 +494,13 @@ class _ScaledStream:
         return self._mul(q, self.q_scale), self._mul(k, self.k_scale), v
 
 
-@pytest.mark.parametrize("config,q_scale,k_scale,steps", [(1, 16.0, 8.0, 256), (1, 16.0, 1.0, 120), (1, 64.0, 32.0, 120),
-                                                          (1, 1.0 / 64, 1.0 / 64, 120), (2, 8.0, 4.0, 40)])
-def test_saturated_and_flat_softmax(config, q_scale, k_scale, steps):
+_ALWAYS_SHRINK = dict(policy=B.GP_POLICY_SHRINK, shrink_below=0.5, tau=1.0, min_capacity=48)
+
+
+@pytest.mark.parametrize("config,q_scale,k_scale,steps,over", [
+    (1, 16.0, 8.0, 256, {}), (1, 16.0, 1.0, 120, {}), (1, 64.0, 32.0, 120, {}), (1, 1.0 / 64, 1.0 / 64, 120, {}),
+    (2, 8.0, 4.0, 40, {}), (1, 16.0, 8.0, 120, _ALWAYS_SHRINK), (5, 16.0, 4.0, 60, _ALWAYS_SHRINK)])
+def test_saturated_and_flat_softmax(config, q_scale, k_scale, steps, over):
     # Logits in the tens, hundreds or thousands: the summary probabilities of a candidate set span far more than
     # the 2^64 range the one-pass selection handles (many underflow to denormals or exactly zero, a mass of equal
     # scores under a few large ones), so working sets and eviction lists come from the general radix descent;
@@ -505,9 +509,11 @@ def test_saturated_and_flat_softmax(config, q_scale, k_scale, steps):
     wl = W.parity_instance(config)
     plain = wl.stream
     object.__setattr__(wl, "stream", lambda spec: _ScaledStream(plain(spec), q_scale, k_scale))
-    st = LS.run_lockstep(wl, max_steps=steps)
+    st = LS.run_lockstep(wl, max_steps=steps, **over)
     _report(f"config {config}, q x{q_scale}, k x{k_scale}", st)
     assert st.decisions["sel"] > 0
+    if over:
+        assert st.actions.get(B.GP_ACT_SHRINK, 0) > 0
 
 
 @pytest.mark.parametrize("name,shape,n_prompt,over", [
