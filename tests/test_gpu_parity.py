@@ -250,10 +250,19 @@ def test_equal_scores_take_the_general_selection_paths(shrink):
 
 def test_candidate_set_larger_than_the_staging_buffers():
     # more than 6144 candidate tokens: the scores of a unit no longer fit the selection kernel's shared memory
-    # (they go through global scratch) and its softmax factors are recomputed per token instead of tabulated
+    # and go through global scratch
     st = _single_request_case(W.Shape(1, 4, 2, 64), 6300, 80)
     _report("6300-token prompt", st)
     assert st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) >= 1
+    # more (page, column) pairs than the table of softmax factors holds (6528): with 8 heads per group, 13200
+    # tokens are 825 candidate pages x 8 columns for a working-set job and x 16 for an eviction job, and the
+    # factors are recomputed per token
+    st = _single_request_case(W.Shape(1, 16, 2, 64), 13200, 80)
+    _report("13200-token prompt, G = 8", st)
+    assert st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) >= 1
+    st = _single_request_case(W.Shape(1, 16, 2, 64), 13200, 40, policy=B.GP_POLICY_SHRINK, shrink_below=0.5, tau=1.0)
+    _report("13200-token prompt, G = 8, shrink", st)
+    assert st.actions.get(B.GP_ACT_SHRINK, 0) >= 1
 
 
 def test_shrink_at_the_default_floor_and_beyond_the_staging_buffers():
