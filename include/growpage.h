@@ -82,7 +82,8 @@ typedef struct gp_config {
   int32_t head_dim;          /* d_h: 64 or 128                                                     */
   int32_t page_size;         /* b: tokens per page, 16                                             */
   int32_t max_requests;      /* M: summary slots = highest request id + 1 (App. D.1, default 512)  */
-  int32_t max_pages_per_req; /* per-request page cap and page-table stride, >= 1                   */
+  int32_t max_pages_per_req; /* per-request page cap and page-table stride, >= 1; at most 62 000
+                                (the selection kernel keeps one bit per candidate token on chip)  */
   int32_t recent_window;     /* |R_t| protected tokens; must equal page_size                       */
   int32_t k_loc;             /* block-local retention quota of Eq. 10 (default page_size / 4)      */
   int32_t host_staging;      /* 1: reserve staging so that gp_decode_step_host can be used         */

@@ -1228,9 +1228,12 @@ static auto compact_kernel_of(const GpDev& p) -> void (*)(const GpDev, const int
   return shr ? gp_compact_kernel<64, true> : gp_compact_kernel<64, false>;
 }
 
-size_t gp_bsel_smem(const GpDev& p) {
-  return SelGeom::BUF_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)p.cap * GP_PAGE / 32 + 2) * 4 + 512;
+// shared memory of the selection kernel for a per-request page cap (its bitmap of block-local picks has one bit
+// per candidate token)
+size_t gp_bsel_smem_for_cap(long long cap) {
+  return SelGeom::BUF_BYTES + SelGeom::H_BYTES + SelGeom::MISC_BYTES + ((size_t)cap * GP_PAGE / 32 + 2) * 4 + 512;
 }
+size_t gp_bsel_smem(const GpDev& p) { return gp_bsel_smem_for_cap(p.cap); }
 
 // one-time setup for a pool: opts the selection kernel into its shared memory and sizes both grids to
 // exactly one resident wave, so that no CTA waits for another to leave before it can start

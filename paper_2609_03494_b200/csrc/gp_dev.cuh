@@ -263,6 +263,8 @@ void gp_attention_setup(const GpDev& p);
 // merge of the split requests' partial outputs for the units [lh0, lh0 + lh_n) (per-layer entry point)
 void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl);
 void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact);
+size_t gp_bsel_smem_for_cap(long long cap);
+#define GP_MAX_DYN_SMEM (227 * 1024)   // opt-in shared memory per CTA on sm_100
 // boundary chain: probabilities + working sets + selection + decision, then compaction.
 // `ev`, when not null, is recorded between the two kernels.  `pdl`: launch with programmatic stream serialization.
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,

@@ -77,6 +77,7 @@ bool valid_config(const gp_config* c) {
   if (c->page_size != GP_PAGE || c->recent_window != c->page_size) return false;
   if (c->max_requests < 1 || c->max_requests > GP_MAX_REQ) return false;
   if (c->max_pages_per_req < 1 || c->max_pages_per_req > (1 << 20)) return false;
+  if (gp_bsel_smem_for_cap(c->max_pages_per_req) > GP_MAX_DYN_SMEM) return false;   // about 62 000 pages
   if (c->n_pages < 1 || c->n_pages > 0x7fffffffLL / GP_PAGE) return false;
   if (c->k_loc < 0 || c->k_loc > GP_PAGE) return false;
   if (c->max_batch_tokens < 0) return false;
