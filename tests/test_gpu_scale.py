@@ -204,3 +204,86 @@ def test_invariants_under_continuous_batching(name, tau, shrink_below):
             assert seen["fallback"] > 0 and seen["stalled"] > 0
     finally:
         gpu.close()
+
+
+def test_pool_larger_than_four_giga_elements():
+    """36 layers x 4300 pages of the 8B shape: 11 GB of K/V, element offsets beyond 2^32 (the full multi-layer
+    configuration is ten times this).  Eight requests with 8192-token prompts fill 4096 pages; the prompts are
+    drawn on the device.  Checked: the pool holds, bit for bit, what was ingested, at the highest offsets too;
+    attention outputs equal the float64 softmax-weighted mean of what the pool holds; the boundary step (8192
+    candidates per unit, 288 units per request) leaves a valid state."""
+    import torch
+
+    L, Hq, Hkv, d, b = 36, 32, 8, 128, 16
+    n_req, n_prompt = 8, 8192
+    P0 = n_prompt // b + 1
+    cfg = B.make_config(L, Hq, Hkv, d, n_pages=4300, max_pages_per_req=P0 + 2, max_requests=n_req, tau=-1.0)
+    gpu = B.Pool(cfg, 0)
+    dev = "cuda:0"
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(17)
+    try:
+        keep = {}
+        for i in range(n_req):
+            k = torch.randn((L, n_prompt, Hkv, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+            v = torch.randn((L, n_prompt, Hkv, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+            assert gpu.request_add(-1, 0, k, v, n_prompt, 0) == (B.GP_OK, i)
+            # what the checks below need of this prompt: the last layer, both end heads
+            keep[i] = {(l, h): (k[l, :, h].view(torch.int16).cpu().numpy().view(np.uint16),
+                                v[l, :, h].view(torch.int16).cpu().numpy().view(np.uint16))
+                       for (l, h) in ((0, 0), (L - 1, Hkv - 1))}
+            del k, v
+        P, n, pos, table = B.gp_debug_request(gpu.handle, n_req - 1, cfg.max_pages_per_req)
+        assert (P, n, pos) == (P0, n_prompt, n_prompt) and max(table) >= 4000
+        for i in (0, n_req - 1):
+            for (l, h), (k_src, v_src) in keep[i].items():
+                kk, vv = B.gp_debug_kv(gpu.handle, i, l, h, n_prompt, d)
+                assert np.array_equal(kk, k_src) and np.array_equal(vv, v_src), f"request {i} ({l},{h}): pool differs from the prompt"
+        ids = torch.arange(n_req, dtype=torch.int32, device=dev)
+        G = Hq // Hkv
+        out = torch.zeros((L, n_req, Hq, d), dtype=torch.float32, device=dev)
+        act = torch.zeros(n_req, dtype=torch.int32, device=dev)
+        for t in range(b + 2):
+            q = torch.randn((L, n_req, Hq, d), generator=gen, device=dev).to(torch.bfloat16)
+            k = torch.randn((L, n_req, Hkv, d), generator=gen, device=dev).to(torch.bfloat16)
+            v = torch.randn((L, n_req, Hkv, d), generator=gen, device=dev).to(torch.bfloat16)
+            gpu.decode_step(ids, q, k, v, out, act)
+            a = act.cpu().numpy()
+            at_boundary = t == b - 1
+            assert ((a == B.GP_ACT_GROW).all() if at_boundary else (a == B.GP_ACT_NONE).all()), (t, a)
+            if t in (0, b - 1, b + 1):
+                for i, l, h in ((0, 0, 0), (n_req - 1, L - 1, Hkv - 1), (3, 17, 4)):
+                    n1 = n_prompt + t + 1
+                    kk, vv = B.gp_debug_kv(gpu.handle, i, l, h, n1, d)
+                    kk, vv = H.decode_bits(kk), H.decode_bits(vv)
+                    qq = q[l, i, h * G:(h + 1) * G].to(torch.float64).cpu().numpy()
+                    z = qq @ kk.T / np.sqrt(d)
+                    p = np.exp(z - z.max(axis=1, keepdims=True))
+                    want = (p / p.sum(axis=1, keepdims=True)) @ vv
+                    got = out[l, i, h * G:(h + 1) * G].cpu().numpy().astype(np.float64)
+                    assert np.abs(got - want).max() <= ATTN_MAX_ABS, f"step {t} request {i} ({l},{h})"
+        _pool_accounting(gpu, cfg, list(range(n_req)))
+        for i in range(n_req):
+            P, n, pos, _ = B.gp_debug_request(gpu.handle, i, cfg.max_pages_per_req)
+            assert (P, n, pos) == (P0 + 1, n_prompt + b + 2, n_prompt + b + 2)
+        # a second boundary under pressure: the pool has 4300 - 8 * 514 = 188 pages left, the cap is P0 + 2
+        for t in range(b + 2, 3 * b + 2):
+            q = torch.randn((L, n_req, Hq, d), generator=gen, device=dev).to(torch.bfloat16)
+            k = torch.randn((L, n_req, Hkv, d), generator=gen, device=dev).to(torch.bfloat16)
+            v = torch.randn((L, n_req, Hkv, d), generator=gen, device=dev).to(torch.bfloat16)
+            gpu.decode_step(ids, q, k, v, out, act)
+            a = act.cpu().numpy()
+            if t == 2 * b - 1:
+                assert (a == B.GP_ACT_GROW).all(), a                     # second boundary: up to the cap
+            elif t == 3 * b - 1:
+                assert (a == B.GP_ACT_COMPRESS_FALLBACK).all(), a        # third boundary, at the cap: compresses
+            else:
+                assert (a == B.GP_ACT_NONE).all(), (t, a)
+        _pool_accounting(gpu, cfg, list(range(n_req)))
+        for i in (0, n_req - 1):
+            P, n, pos, _ = B.gp_debug_request(gpu.handle, i, cfg.max_pages_per_req)
+            assert (P, n) == (P0 + 2, (P0 + 1) * b + 2)                  # two steps after the compression
+            tok = B.gp_debug_retained(gpu.handle, i, L - 1, Hkv - 1, n).astype(np.int64)
+            assert (np.diff(tok) > 0).all() and np.array_equal(tok[-b:], np.arange(pos - b, pos))
+    finally:
+        gpu.close()
