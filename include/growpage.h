@@ -46,10 +46,9 @@ extern "C" {
 #define GP_ACT_STALLED          (-1)  /* full and neither a page nor copy-on-write targets could
                                          be had: page state untouched, the caller should release
                                          (preempt) the request; it is skipped while it stays full */
-#define GP_ACT_SCRATCH          (-2)  /* the batch exceeds max_batch_tokens: either the request was
-                                         stepped without its boundary (its last page is now full and
-                                         the next step reports it stalled), or it was not stepped at
-                                         all (its state is unchanged)                              */
+#define GP_ACT_SCRATCH          (-2)  /* the batch exceeds max_batch_tokens and this request's work did
+                                         not fit the step's scratch: it was not stepped, its state is
+                                         unchanged, and it can be stepped again in a later batch     */
 #define GP_ACT_INVALID          (-3)  /* id out of range, not live, or repeated in the batch      */
 
 typedef struct gp_pool gp_pool; /* opaque */

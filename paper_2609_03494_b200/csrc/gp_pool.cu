@@ -350,11 +350,10 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   int rc_off, n_rc; long long tok_off, tok_tot;
   plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
   // A batch whose summed lengths exceed max_batch_tokens (the caller's bound; with shared prompt pages the sum
-  // can exceed what the pool holds) does not fit the scratch: a boundary request whose logits do not fit is
-  // stepped without its boundary, and a request whose work items do not fit is not stepped at all.  The
+  // can exceed what the pool holds) does not fit the scratch: a request whose boundary logits or whose work
+  // items do not fit is not stepped (its state stays as it is, it can be stepped again in a later batch).  The
   // offsets are then taken again over what is left, so that the item list has no holes.
-  if (isb && tok_off + nc > p.max_batch_tokens) { isb = 0; nc = 0; act = GP_ACT_SCRATCH; }
-  const bool dropped = chunks > 0 && rc_off + chunks > p.max_rc;
+  const bool dropped = chunks > 0 && ((isb && tok_off + nc > p.max_batch_tokens) || rc_off + chunks > p.max_rc);
   if (dropped) { chunks = 0; isb = 0; nc = 0; act = GP_ACT_SCRATCH; }
   if (__syncthreads_or(dropped)) plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
   int bnd_idx, n_bnd, n_active; long long d0, d1;
