@@ -486,7 +486,9 @@ class OraclePool:
         b = c.page_size
         overrides = overrides or {}
         order = sorted(rec.boundary)
-        index_of = {rid: i for i, rid in enumerate(rec.req_ids)}
+        index_of: Dict[int, int] = {}
+        for i, rid in enumerate(rec.req_ids):           # a repeated id is stepped at its first batch slot only
+            index_of.setdefault(rid, i)
         # pass 1: grants, ascending request id
         compress: List[int] = []
         for rid in order:

@@ -461,6 +461,11 @@ def test_invalid_ids_and_duplicates_are_reported_per_request():
     rec = pool.decode_step([a, 3, a], *_rand_step(c, 3))
     assert [int(x) for x in rec.actions] == [O.ACT_NONE, O.ACT_INVALID, O.ACT_INVALID]
     assert pool.request_state(a)[1] == 3
+    # the same at a capacity boundary (page size 4, one page: the fourth token fills it): the action belongs to the
+    # first batch slot that names the request, the repeat stays invalid
+    rec = pool.decode_step([a, a], *_rand_step(c, 2))
+    assert int(rec.actions[0]) in (O.ACT_GROW, O.ACT_COMPRESS_FALLBACK, O.ACT_STALLED) and int(rec.actions[1]) == O.ACT_INVALID
+    assert pool.request_state(a)[2] == 4
     assert pool.release(2) == O.ERR_INVALID
     for i in range(3):
         assert pool.request_add(-1, 0, kt, kt.copy(), 2, 0)[0] == O.OK
