@@ -126,7 +126,8 @@ int gp_pool_destroy(gp_pool* pool);
  * The request starts with max(initial_pages, floor(n_prompt / b) + 1) pages.
  * On success *out_req receives the request id (the lowest free slot).  The summaries of the slot
  * are not cleared: the first decode step overwrites them.  Synchronises `stream`.
- * Errors: GP_ERR_INVALID, GP_ERR_NO_SLOT, GP_ERR_NO_PAGES (nothing is changed in these cases). */
+ * Errors, checked in this order: GP_ERR_INVALID (arguments; donor dead or with fewer shareable pages),
+ * GP_ERR_NO_SLOT, GP_ERR_NO_PAGES (nothing is changed in these cases). */
 int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
                    const void* k_tail, const void* v_tail, int32_t n_tail,
                    int32_t initial_pages, void* stream, int32_t* out_req);

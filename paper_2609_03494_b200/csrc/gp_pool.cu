@@ -439,8 +439,10 @@ __global__ void gp_admit_kernel(GpDev p, int r, int share_from, int n_shared, in
   const int lane = threadIdx.x;
   const int need = P_target - n_shared;
   const int top = *p.free_top;
+  // refusals in a fixed order: what is wrong with the arguments, then the slot, then the pages
   int st = GP_OK;
   if (n_shared > 0 && (!p.live[share_from] || p.n_pristine[share_from] < n_shared)) st = GP_ERR_INVALID;
+  else if (r < 0) st = GP_ERR_NO_SLOT;
   else if (need > top || P_target > p.cap) st = GP_ERR_NO_PAGES;
   __syncwarp();
   if (st == GP_OK) {
@@ -703,11 +705,14 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   int slot = -1;
   for (int i = 0; i < c.max_requests; ++i)
     if (!pool->live[i]) { slot = i; break; }
-  if (slot < 0) return GP_ERR_NO_SLOT;
+  if (slot < 0 && n_shared_pages == 0) return GP_ERR_NO_SLOT;
   const long long n_prompt = (long long)n_shared_pages * GP_PAGE + n_tail;
   long long P = n_prompt / GP_PAGE + 1;
   if (initial_pages > P) P = initial_pages;
-  if (P > c.max_pages_per_req) return GP_ERR_NO_PAGES;
+  // with shared pages the donor's count of shareable pages lives on the device: the kernel below gives the
+  // refusals in the documented order (invalid arguments, no slot, no pages)
+  if (P > c.max_pages_per_req && n_shared_pages == 0) return GP_ERR_NO_PAGES;
+  if (P > c.max_pages_per_req) P = (long long)c.max_pages_per_req + 1;      // still refused, and fits an int
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   gp_admit_kernel<<<1, 32, 0, s>>>(pool->dev, slot, share_from, n_shared_pages, n_tail, (int)P, pool->d_status);

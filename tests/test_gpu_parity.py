@@ -581,3 +581,88 @@ def test_largest_page_cap_still_launches_the_selection_kernel():
     st = LS.run_lockstep(wl, tau=-0.02)
     _report("cap 62000", st)
     assert st.decisions["act"] >= 2
+
+
+@pytest.mark.parametrize("seed,pol", [(2024, {}), (7, dict(policy=B.GP_POLICY_SHRINK, shrink_below=0.0, min_capacity=48)),
+                                      (11, dict(policy=B.GP_POLICY_RANDOM, policy_seed=5, p_compress=0.5))])
+def test_random_admissions_sharing_steps_and_releases(seed, pol):
+    # a seeded random walk over the public calls: admissions with and without shared prompt pages (from donors at
+    # any stage, with tails of any length, valid and invalid), decode steps on random subsets in random order,
+    # releases; after every call the two sides must agree on statuses, ids, actions, page counts, token counts,
+    # positions, free pages and the multiset of reference counts, and on the attention outputs
+    import torch
+    L, Hq, Hkv, d, b = 1, 4, 2, 64, 16
+    kw = dict(n_pages=72, max_pages_per_req=9, max_requests=8, k_loc=2, tau=0.0)
+    gpu = B.Pool(B.make_config(L, Hq, Hkv, d, **kw, **pol))
+    ora = O.OraclePool(O.OracleConfig(L, Hq, Hkv, d, **kw, **pol))
+    rng = np.random.default_rng(seed)
+    bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    o_map = {O.OK: B.GP_OK, O.ERR_INVALID: B.GP_ERR_INVALID, O.ERR_NO_SLOT: B.GP_ERR_NO_SLOT, O.ERR_NO_PAGES: B.GP_ERR_NO_PAGES}
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to("cuda:0")
+    live = []
+    counts = {"add": 0, "add_shared": 0, "add_refused": 0, "step": 0, "release": 0}
+    actions_seen = {}
+
+    def check_state():
+        n_free, ref, counters = B.gp_debug_pool(gpu.handle, kw["n_pages"])
+        assert counters[7] == 0 and n_free == ora.n_free()
+        assert sorted(ref[ref > 0].tolist()) == sorted(ora.refcount[ora.refcount > 0].tolist())
+        for rid in live:
+            assert B.gp_debug_request(gpu.handle, rid, 9)[:3] == ora.request_state(rid)[:3], rid
+
+    try:
+        for it in range(420):
+            u = rng.random()
+            if u < 0.2 or not live:
+                share = int(rng.choice(live)) if live and rng.random() < 0.6 else int(rng.integers(-1, 8))
+                n_sh = int(rng.integers(0, 5)) if share >= 0 else 0
+                n_tail = int(rng.integers(0, 45))
+                init = int(rng.integers(0, 7))
+                kt, vt = (bits(L, n_tail, Hkv, d), bits(L, n_tail, Hkv, d)) if n_tail else (None, None)
+                g_st, g_rid = gpu.request_add(share, n_sh, kt, vt, n_tail, init)
+                o_st, o_rid = ora.request_add(share, n_sh, None if kt is None else H.decode_bits(kt),
+                                              None if vt is None else H.decode_bits(vt), n_tail, init)
+                assert g_st == o_map[o_st], (it, "add", share, n_sh, n_tail, init, g_st, o_st)
+                if g_st == B.GP_OK:
+                    assert g_rid == o_rid
+                    live.append(g_rid)
+                    counts["add_shared" if n_sh else "add"] += 1
+                else:
+                    counts["add_refused"] += 1
+            elif u < 0.94:
+                k_sub = int(rng.integers(1, len(live) + 1))
+                rids = [int(x) for x in rng.permutation(live)[:k_sub]]
+                if rng.random() < 0.1 and len(rids) < 8:              # a batch holds at most max_requests ids
+                    rids.append(int(rng.integers(0, 8)))              # a repeated, dead or live extra id
+                Bn = len(rids)
+                q, k, v = bits(L, Bn, Hq, d), bits(L, Bn, Hkv, d), bits(L, Bn, Hkv, d)
+                out = torch.zeros((L, Bn, Hq, d), dtype=torch.float32, device="cuda:0")
+                act = torch.zeros(Bn, dtype=torch.int32, device="cuda:0")
+                gpu.decode_step(torch.tensor(rids, dtype=torch.int32, device="cuda:0"), dev(q), dev(k), dev(v), out, act)
+                rec = ora.decode_step(rids, H.decode_bits(q), H.decode_bits(k), H.decode_bits(v))
+                a = act.cpu().numpy()
+                assert np.array_equal(a, rec.actions), (it, rids, a, rec.actions)
+                stepped = [i for i in range(Bn) if a[i] >= 0]
+                if stepped:
+                    err = np.abs(out.cpu().numpy().astype(np.float64)[:, stepped] - rec.out[:, stepped]).max()
+                    assert err <= LS.ATTN_MAX_ABS, (it, err)
+                for x in a:
+                    actions_seen[int(x)] = actions_seen.get(int(x), 0) + 1
+                counts["step"] += 1
+            else:
+                rid = int(rng.choice(live))
+                gpu.release(rid)
+                assert ora.release(rid) == O.OK
+                live.remove(rid)
+                counts["release"] += 1
+            check_state()
+        print("\\nrandom walk:", counts, "actions", actions_seen)
+        assert counts["add_shared"] >= 5 and counts["add_refused"] >= 3 and counts["release"] >= 5
+        assert actions_seen.get(B.GP_ACT_COMPRESS, 0) + actions_seen.get(B.GP_ACT_COMPRESS_FALLBACK, 0) + actions_seen.get(B.GP_ACT_SHRINK, 0)
+        assert actions_seen.get(B.GP_ACT_INVALID, 0)
+        if pol.get("policy") == B.GP_POLICY_SHRINK:
+            assert actions_seen.get(B.GP_ACT_SHRINK, 0)
+        else:
+            assert actions_seen.get(B.GP_ACT_GROW, 0)
+    finally:
+        gpu.close()
