@@ -666,3 +666,26 @@ def test_random_admissions_sharing_steps_and_releases(seed, pol):
             assert actions_seen.get(B.GP_ACT_GROW, 0)
     finally:
         gpu.close()
+
+
+def test_random_shapes_and_settings():
+    # a dozen seeded draws of geometry (layers, heads, group size, head dimension), prompt lengths, quota, coverage,
+    # smoothing, threshold, RoPE and policy, each a short lockstep run of three requests
+    rng = np.random.default_rng(99)
+    for trial in range(12):
+        G = int(rng.choice([1, 2, 4, 8]))
+        Hkv = int(rng.choice([1, 2, 3, 4]))
+        d = int(rng.choice([64, 128]))
+        L = int(rng.integers(1, 4))
+        shape = W.Shape(L, Hkv * G, Hkv, d)
+        reqs = [W.RequestSpec(i, int(rng.integers(1, 330)), 44, float(rng.uniform(0.01, 0.2))) for i in range(3)]
+        cap = max(r.prompt_len for r in reqs) // 16 + 3
+        wl = W.Workload(f"draw{trial}", 1000 + trial, shape, reqs, n_resident=3, initial_pages=int(rng.integers(0, 4)),
+                        max_pages_per_req=cap, n_pages=3 * cap - int(rng.integers(0, 4)))
+        over = dict(k_loc=int(rng.integers(0, 9)), top_p=float(rng.choice([0.8, 0.95, 0.99, 0.999])),
+                    beta_s=float(rng.choice([0.0, 0.5, 0.9])), beta_l=float(rng.choice([0.99, 0.999])),
+                    tau=float(rng.choice([-0.05, -0.01, 0.0])), rope_theta=float(rng.choice([0.0, 1e4])))
+        if rng.random() < 0.4:
+            over.update(policy=B.GP_POLICY_SHRINK, shrink_below=float(rng.choice([-0.03, 0.5])), min_capacity=48)
+        st = LS.run_lockstep(wl, **over)
+        _report(f"draw {trial}: {shape} prompts {[r.prompt_len for r in reqs]} {over}", st)
