@@ -689,3 +689,13 @@ def test_random_shapes_and_settings():
             over.update(policy=B.GP_POLICY_SHRINK, shrink_below=float(rng.choice([-0.03, 0.5])), min_capacity=48)
         st = LS.run_lockstep(wl, **over)
         _report(f"draw {trial}: {shape} prompts {[r.prompt_len for r in reqs]} {over}", st)
+
+
+def test_a_32k_token_request_at_the_32b_head_shape():
+    # the longest sequence of the multi-layer configurations (32 768 tokens, 64 query heads over 8 KV heads): 64
+    # work items per (layer, head), candidate sets five times the selection kernel's staging buffers, 2047
+    # candidate pages; grows to its cap, then a fallback compression over 32k candidates
+    st = _single_request_case(W.Shape(1, 64, 8, 128), 32760, 60)
+    _report("32760-token request, 32B head shape", st)
+    assert st.actions.get(B.GP_ACT_GROW, 0) == 3 and st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) == 1
+    assert st.decisions["sel"] == 8
