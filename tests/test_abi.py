@@ -34,6 +34,7 @@ def test_config_defaults_and_pool_bytes_need_no_gpu():
     cfg = B.gp_config_default()
     assert (cfg.beta_s, cfg.beta_l, cfg.top_p, cfg.tau) == (0.9, 0.999, 0.99, 0.0)
     assert cfg.page_size == 16 and cfg.recent_window == 16 and cfg.k_loc == 4 and cfg.max_requests == 512
+    assert (cfg.policy, cfg.p_compress, cfg.shrink_below, cfg.min_capacity) == (B.GP_POLICY_DEMAND, 0.7, -0.005, 1024)
     assert B.gp_pool_bytes(cfg) == 0                       # geometry not filled in: invalid
     cfg = B.make_config(1, 32, 8, 128, n_pages=1024, max_pages_per_req=64, max_requests=64)
     nbytes = B.gp_pool_bytes(cfg)

@@ -33,6 +33,8 @@ def test_defaults_match_the_paper():
     assert c.max_requests == g["M"]
     # quota is the paper's fraction of a block: 64 of 256 tokens
     assert c.k_loc / c.page_size == g["k_loc"] / g["b"]
+    # the ablation's policies
+    assert c.p_compress == g["p_compress"] and c.shrink_below == g["shrink_below"] and c.min_capacity == g["min_capacity"]
 
 
 # ----------------------------------------------------------------------------- attention
