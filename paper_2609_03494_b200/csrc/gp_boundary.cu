@@ -854,17 +854,20 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const int LH = p.L * p.Hkv;
   const int G = p.G, G2 = 2 * p.G;
   constexpr int NT = SHR ? 4 : 3;                           // jobs per unit: K^S, K^L, eviction list(s)
-  gp_pdl_wait();
-  gp_pdl_launch_dependents();
-  // the first item's descriptor is fetched before the number of items is known (same round trip); slots of
-  // bnd_info past the count hold stale but readable data that is then not used
+  // What the plan kernel wrote (counts, boundary records) is read before the wait for the attention kernel: the
+  // plan kernel had completed before any CTA of the attention kernel let this grid be scheduled, and the
+  // attention kernel does not touch these words; the loads go to the L2 (an L1 line could date from the step
+  // before).  The first item's record is fetched before the number of items is known (same round trip); slots
+  // of bnd_info past the count hold stale but readable data that is then not used.
   int4 inf_first = make_int4(0, 0, 0, 0), inf2_first = inf_first;
   {
     const int b0 = (int)(blockIdx.x / (NT * LH));
-    if (b0 < p.M) { inf_first = p.bnd_info[2 * b0]; inf2_first = p.bnd_info[2 * b0 + 1]; }
+    if (b0 < p.M) { inf_first = __ldcg(p.bnd_info + 2 * b0); inf2_first = __ldcg(p.bnd_info + 2 * b0 + 1); }
   }
-  const int n_bnd = p.hdr[HDR_N_BND];
-  const int n_mc = out ? p.hdr[HDR_N_MC] : 0, n_rc = p.hdr[HDR_N_RC];   // out == null: already merged layer by layer
+  const int n_bnd = __ldcg(p.hdr + HDR_N_BND);
+  const int n_mc = out ? __ldcg(p.hdr + HDR_N_MC) : 0, n_rc = __ldcg(p.hdr + HDR_N_RC);   // out == null: already merged layer by layer
+  gp_pdl_wait();
+  gp_pdl_launch_dependents();
   const long long items = (long long)n_bnd * LH * NT;
   if (tid == 0) GP_T_STAMP(59);
 

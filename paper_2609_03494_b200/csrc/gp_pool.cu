@@ -219,8 +219,10 @@ __device__ void prepare_row(const GpDev& p, const int* __restrict__ req_ids, int
 #pragma unroll
   for (int e = 0; e < PER; ++e) qf[e] = __bfloat162float(qrow[lane + 32 * e]);
   if (r < 0 || r >= p.M || __any_sync(0xffffffffu, dup)) return;
-  const int live = p.live[r], n_old = p.n[r], Pr = p.P[r], started = p.started[r], par = p.sum_par[r];
-  const long long pos = p.pos[r];
+  // (loads from the L2: in the whole-step launch these CTAs do not wait for the kernel before them, see below)
+  const int live = __ldcg(p.live + r), n_old = __ldcg(p.n + r), Pr = __ldcg(p.P + r), started = __ldcg(p.started + r),
+            par = __ldcg(p.sum_par + r);
+  const long long pos = __ldcg(p.pos + r);
   double ov0[PER], ov1[PER];
   {
     const double* o0 = p.summ + gp_summ_off(p, l, r, 0, x, head);
@@ -285,10 +287,18 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
   __shared__ int s_chunks[GP_MAX_REQ], s_pos[GP_MAX_REQ];
   __shared__ int s_bin[GP_COST_BINS], s_binbase[GP_COST_BINS], s_nmc;
-  __shared__ int s_peek[GP_MAX_REQ];       // the free list from its top down, for the decisions of this step
   const int i = threadIdx.x;
   const bool in = i < n_req;
-  gp_pdl_wait();
+  // What runs before the wait for the kernel before this one.  In a whole-step launch that kernel is the
+  // compaction of the step before (or something the caller put in between, which then has completed): this
+  // grid became schedulable only after that step's decisions had completed, and compaction touches neither the
+  // requests' counters, nor the summaries, nor anything the plan writes except the step stamp.  So the summary
+  // CTAs do not wait at all, and CTA 0 plans the whole step first and waits only before it looks at the free
+  // list (which compaction's last CTA may still change) and stamps the step.  CTA 0 does wait, so the grid as
+  // a whole still ends after everything before it.  The layer-by-layer launches (plan_on == 0) have no CTA 0
+  // work and keep the wait in every CTA, so that completion stays transitive.  The next kernel may be scheduled
+  // as soon as every CTA of this grid has started; it waits for this grid's end at its own top.
+  if (!plan_on) gp_pdl_wait();
   gp_pdl_launch_dependents();
   if (blockIdx.x > 0) {                       // summary CTAs: one warp per (unit, view, head)
     const int rows = 2 * p.G, upc = 32 / rows;             // units per CTA and pass
@@ -304,7 +314,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     return;
   }
   if (!plan_on) return;
-  const int free_top0 = *p.free_top;
   const long long t_plan0 = GP_T_NOW();
   (void)t_plan0;
   s_first[i] = 0x7fffffff;
@@ -321,13 +330,13 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   long long nc = 0, pos = 0;
   int isb = 0;
   int cp = p.chunk_pages;                 // pages per work item of this request
+  int live = 0;
+  if (in && r >= 0 && r < p.M) {          // independent loads, issued together (from the L2: before the wait)
+    live = __ldcg(p.live + r); n_old = __ldcg(p.n + r); Pr = __ldcg(p.P + r); pos = __ldcg(p.pos + r);
+    started = __ldcg(p.started + r); par = __ldcg(p.sum_par + r);
+  }
   if (in) {
     const bool inrange = r >= 0 && r < p.M;
-    int live = 0;
-    if (i < free_top0) s_peek[i] = p.free_stack[free_top0 - 1 - i];
-    if (inrange) {                    // independent loads, issued together
-      live = p.live[r]; n_old = p.n[r]; Pr = p.P[r]; pos = p.pos[r]; started = p.started[r]; par = p.sum_par[r];
-    }
     const bool valid = inrange && live && s_first[r] == i;
     if (!valid) {
       act = GP_ACT_INVALID;
@@ -393,7 +402,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       p.bnd_info[2 * bnd_idx] = make_int4(i, r, Pr, (int)pos);     // pos: position of this step's token
       p.bnd_info[2 * bnd_idx + 1] = make_int4((int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32), 0, 0);
       reinterpret_cast<int4*>(p.bnd_acc)[bnd_idx] = make_int4(0, 0, 0, 0);
-      if (bnd_idx < free_top0) p.free_peek[1 + bnd_idx] = s_peek[bnd_idx];
     }
     // descriptors of this request's chunks: four 16-byte stores each
     const int flags = isb | (started ? 2 : 0);
@@ -425,12 +433,19 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (threadIdx.x == 0) {
     p.hdr[HDR_N_MC] = s_nmc;
-    p.free_peek[0] = free_top0;
     GP_T_ADD(26, 1); GP_T_ADD(27, t_plan1 - t_plan0); GP_T_ADD(28, t_plan2 - t_plan1); GP_T_ADD(29, GP_T_NOW() - t_plan2);
     p.hdr[HDR_N_RC] = n_rc;
     p.hdr[HDR_N_BND] = n_bnd;
     p.hdr[HDR_WORK_ATTN] = 0;
     p.hdr[HDR_N_ACTIVE] = n_active;
+  }
+  // ---- from here on the kernel before this one has completed --------------------------------------------
+  gp_pdl_wait();
+  const int free_top0 = *p.free_top;
+  // the top of the free list, one page per boundary request: what this step's grants can take
+  if (in && isb && bnd_idx < free_top0) p.free_peek[1 + bnd_idx] = p.free_stack[free_top0 - 1 - bnd_idx];
+  if (threadIdx.x == 0) {
+    p.free_peek[0] = free_top0;
     p.hdr[HDR_STEP] += 1;
   }
 }
