@@ -198,39 +198,26 @@ __device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long
 // reaches its capacity boundary, the calibrated (Eq. 12) and rotated summaries q~ in fp64 for the attention
 // kernel's logits.  One warp per (view, head) row; a CTA takes as many units at a time as its warps cover.
 template <int D>
-__device__ void prepare_row(const GpDev& p, const int* __restrict__ req_ids, int n_req, const __nv_bfloat16* __restrict__ q,
-                            int bi, int lh, int row) {
+__device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __restrict__ q, int bi, int lh, int row, int r,
+                            int n_old, int Pr, int started, int par, long long pos) {
   constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int G = p.G;
   const int l = lh / p.Hkv, h = lh % p.Hkv;
   const int x = row / G, g = row % G;
   const int head = h * G + g;
-  // two round trips in all: the request id (with the ids before it, for the duplicate check and the query
-  // row, which do not depend on it), then the request's state and the old summary from both of its buffers
-  const int r = req_ids[bi];
-  bool dup = false;                                          // only the first batch slot naming a request counts
-  for (int j0 = 0; j0 < bi; j0 += 32) {
-    const int j = j0 + lane;
-    dup |= j < bi && req_ids[j] == r;
-  }
+  // one round trip: the query row and the old summary from the request's current buffer (the request's state
+  // was staged in shared memory by the CTA)
   const __nv_bfloat16* qrow = q + (((size_t)l * n_req + bi) * p.Hq + head) * D;
   float qf[PER];
 #pragma unroll
   for (int e = 0; e < PER; ++e) qf[e] = __bfloat162float(qrow[lane + 32 * e]);
-  if (r < 0 || r >= p.M || __any_sync(0xffffffffu, dup)) return;
-  // (loads from the L2: in the whole-step launch these CTAs do not wait for the kernel before them, see below)
-  const int live = __ldcg(p.live + r), n_old = __ldcg(p.n + r), Pr = __ldcg(p.P + r), started = __ldcg(p.started + r),
-            par = __ldcg(p.sum_par + r);
-  const long long pos = __ldcg(p.pos + r);
-  double ov0[PER], ov1[PER];
+  double ovv[PER];
   {
-    const double* o0 = p.summ + gp_summ_off(p, l, r, 0, x, head);
-    const double* o1 = p.summ + gp_summ_off(p, l, r, 1, x, head);
+    const double* o0 = p.summ + gp_summ_off(p, l, r, par, x, head);
 #pragma unroll
-    for (int e = 0; e < PER; ++e) { ov0[e] = __ldcg(o0 + lane + 32 * e); ov1[e] = __ldcg(o1 + lane + 32 * e); }
+    for (int e = 0; e < PER; ++e) ovv[e] = __ldcg(o0 + lane + 32 * e);
   }
-  if (!live) return;
   const bool need_qt = (n_old + 1 == Pr * GP_PAGE) && Pr > 1;
   {
     const double beta = x ? p.beta_l : p.beta_s;
@@ -240,7 +227,7 @@ __device__ void prepare_row(const GpDev& p, const int* __restrict__ req_ids, int
 #pragma unroll
     for (int e = 0; e < PER; ++e) {
       const double qv = (double)qf[e];
-      const double ov = par ? ov1[e] : ov0[e];
+      const double ov = ovv[e];
       sq += qv * qv;
       nv[e] = started ? beta * ov + (1.0 - beta) * qv : qv;              // Eq. 6
       newp[lane + 32 * e] = nv[e];
@@ -286,6 +273,8 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __shared__ long long sw[33];
   __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
   __shared__ int s_chunks[GP_MAX_REQ], s_pos[GP_MAX_REQ];
+  __shared__ int s_req[GP_MAX_REQ], s_state[GP_MAX_REQ];     // summary CTAs: request of a batch slot, flags
+  __shared__ long long s_pos64[GP_MAX_REQ];
   __shared__ int s_bin[GP_COST_BINS], s_binbase[GP_COST_BINS], s_nmc;
   const int i = threadIdx.x;
   const bool in = i < n_req;
@@ -301,14 +290,40 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   if (!plan_on) gp_pdl_wait();
   gp_pdl_launch_dependents();
   if (blockIdx.x > 0) {                       // summary CTAs: one warp per (unit, view, head)
+    // The state of the batch's requests is staged once per CTA, from the L2 (these CTAs may run before the wait,
+    // and an L1 line could date from the step before): request of a slot (-1: not stepped by these CTAs:
+    // out of range, dead, or named by an earlier slot), tokens, pages, flags, position.
+    if (i < GP_MAX_REQ) s_first[i] = 0x7fffffff;
+    __syncthreads();
+    int r = -1;
+    if (in) {
+      r = req_ids[i];
+      if (r >= 0 && r < p.M) atomicMin(&s_first[r], i); else r = -1;
+    }
+    __syncthreads();
+    if (in) {
+      int ok = 0;
+      if (r >= 0 && s_first[r] == i && __ldcg(p.live + r)) {
+        ok = 1;
+        s_chunks[i] = __ldcg(p.n + r);
+        s_pos[i] = __ldcg(p.P + r);
+        s_state[i] = (__ldcg(p.started + r) ? 1 : 0) | (__ldcg(p.sum_par + r) ? 2 : 0);
+        s_pos64[i] = __ldcg(p.pos + r);
+      }
+      s_req[i] = ok ? r : -1;
+    }
+    __syncthreads();
     const int rows = 2 * p.G, upc = 32 / rows;             // units per CTA and pass
     const int warp = threadIdx.x >> 5;
     const long long units = (long long)n_req * lh_n;
     if (warp < upc * rows) {
       for (long long u = ((long long)blockIdx.x - 1) * upc + warp / rows; u < units; u += ((long long)gridDim.x - 1) * upc) {
         const int bi = (int)(u / lh_n), lh = lh0 + (int)(u % lh_n);
-        if (p.d == 128) prepare_row<128>(p, req_ids, n_req, q, bi, lh, warp % rows);
-        else prepare_row<64>(p, req_ids, n_req, q, bi, lh, warp % rows);
+        const int rr = s_req[bi];
+        if (rr < 0) continue;
+        const int st = s_state[bi];
+        if (p.d == 128) prepare_row<128>(p, n_req, q, bi, lh, warp % rows, rr, s_chunks[bi], s_pos[bi], st & 1, (st >> 1) & 1, s_pos64[bi]);
+        else prepare_row<64>(p, n_req, q, bi, lh, warp % rows, rr, s_chunks[bi], s_pos[bi], st & 1, (st >> 1) & 1, s_pos64[bi]);
       }
     }
     return;
