@@ -699,3 +699,50 @@ def test_a_32k_token_request_at_the_32b_head_shape():
     _report("32760-token request, 32B head shape", st)
     assert st.actions.get(B.GP_ACT_GROW, 0) == 3 and st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) == 1
     assert st.decisions["sel"] == 8
+
+
+def test_overlapped_launches_equal_plain_launches():
+    # In the normal mode the kernels of a step are chained with programmatic dependent launch and the plan of a
+    # step runs beside the compaction of the step before; in profiling mode every kernel is launched the plain
+    # way, after the one before it has ended.  Same inputs, both modes: outputs, actions, page tables, retained
+    # sets and summaries must be equal bit for bit.
+    import torch
+    wl = W.layer8b(seed=5, n_requests=24, n_steps=200, prompt_range=(100, 700))
+    s = wl.shape
+    n, T = len(wl.requests), 200
+    q = np.empty((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=np.uint16)
+    k = np.empty((T, s.n_layers, n, s.n_kv_heads, s.head_dim), dtype=np.uint16)
+    v = np.empty_like(k)
+    prompts = []
+    for i in range(n):
+        st = wl.stream(wl.requests[i])
+        prompts.append(st.prompt_kv())
+        q[:, :, i], k[:, :, i], v[:, :, i] = st.steps(0, T)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).to("cuda:0")
+    qd, kd, vd = dev(q), dev(k), dev(v)
+    ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+    results = []
+    for plain in (False, True):
+        pool = B.Pool(B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
+                                    max_pages_per_req=wl.max_pages_per_req, max_requests=n, tau=-0.003))
+        try:
+            for i in range(n):
+                assert pool.request_add(-1, 0, prompts[i][0], prompts[i][1], wl.requests[i].prompt_len, 0)[0] == B.GP_OK
+            B.gp_set_profiling(pool.handle, plain)
+            outs = torch.zeros((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda:0")
+            acts = torch.zeros((T, n), dtype=torch.int32, device="cuda:0")
+            for t in range(T):
+                pool.decode_step(ids, qd[t], kd[t], vd[t], outs[t], acts[t])
+            torch.cuda.synchronize()
+            state = [B.gp_debug_request(pool.handle, i, wl.max_pages_per_req) for i in range(n)]
+            kept = [B.gp_debug_retained(pool.handle, i, 0, 3, state[i][1]) for i in range(n)]
+            summ = [B.gp_debug_summaries(pool.handle, i, s.n_layers, s.n_q_heads, s.head_dim) for i in range(0, n, 5)]
+            assert B.gp_debug_pool(pool.handle)[2][7] == 0
+            results.append((outs.cpu().numpy(), acts.cpu().numpy(), state, kept, summ))
+        finally:
+            pool.close()
+    a, b_ = results
+    assert np.array_equal(a[1], b_[1]) and a[2] == b_[2]
+    assert all(np.array_equal(x, y) for x, y in zip(a[3], b_[3])) and all(np.array_equal(x, y) for x, y in zip(a[4], b_[4]))
+    assert np.array_equal(a[0], b_[0])
+    assert (a[1] == B.GP_ACT_GROW).any() and (a[1] == B.GP_ACT_COMPRESS).any()
