@@ -143,7 +143,8 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
  * Asynchronous on `stream`; nothing is read back to the host, so (with profiling off) a sequence of
  * steps can be captured into a CUDA graph and replayed.  The step's kernels are chained with
  * programmatic dependent launch.  Steps of one pool must be issued on one stream (or otherwise
- * serialised): they share scratch inside the blob. */
+ * serialised): they share scratch inside the blob.  See gp_set_early_plan for an option that lets
+ * the step's first kernel start its work beside the last kernel of the step before. */
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
                    const void* q, const void* k, const void* v,
                    void* out, int32_t* dev_actions, void* stream);
@@ -217,6 +218,19 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
 /* With profiling on, every kernel of gp_decode_step is bracketed by CUDA events on the step's
  * stream (this serialises nothing but adds event records).  Off by default. */
 int gp_set_profiling(gp_pool* pool, int32_t enable);
+
+/* Early planning (off by default).  The first kernel of gp_decode_step is launched as a programmatic
+ * dependent of whatever kernel precedes it on the stream.  With the option off it waits for that
+ * kernel to end before it reads anything: always safe.  With it on, it reads dev_req_ids and q, plans
+ * the step and updates the query summaries before that wait, beside the compaction kernel of the
+ * step before, and waits only before it looks at the free list.  That is correct only if
+ * dev_req_ids and q are complete in memory by the time the preceding kernel on the stream lets
+ * its dependents be scheduled: true when they were produced by copies or by kernels that do not
+ * signal programmatic launch completion (or when nothing was enqueued since the step before);
+ * not true when the query projection enqueued just before the step signals completion ahead of its
+ * stores.  gp_decode_step_host always plans early (its inputs arrive by copies).  The
+ * layer-by-layer calls are not affected. */
+int gp_set_early_plan(gp_pool* pool, int32_t enable);
 
 /* Synchronises, then returns the accumulated device time in milliseconds and the launch count of
  * each kernel since profiling was switched on (host arrays of GP_N_KERNELS), and resets them. */

@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
     L.gp_attn_layer.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
     L.gp_step_end.argtypes = [vp, vp, i32, vp, vp]
     L.gp_set_profiling.argtypes = [vp, i32]
+    L.gp_set_early_plan.argtypes = [vp, i32]
     L.gp_get_kernel_times.argtypes = [vp, vp, vp]
     L.gp_launch_count.argtypes = [vp]; L.gp_launch_count.restype = i64
     L.gp_attention_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
@@ -201,6 +202,10 @@ def gp_debug_pool(pool: int, n_pages: int = 0):
     _check(lib().gp_debug_pool(C.c_void_p(pool), C.byref(n_free), ref.ctypes.data_as(C.c_void_p) if n_pages else None,
                                counters.ctypes.data_as(C.c_void_p)), "gp_debug_pool")
     return int(n_free.value), ref[:n_pages], counters
+
+
+def gp_set_early_plan(pool: int, enable: bool) -> None:
+    _check(lib().gp_set_early_plan(C.c_void_p(pool), 1 if enable else 0), "gp_set_early_plan")
 
 
 def gp_set_profiling(pool: int, enable: bool) -> None:

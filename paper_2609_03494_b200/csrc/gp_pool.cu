@@ -29,6 +29,7 @@ struct gp_pool {
   uint8_t* dbg;                   // gather target of the debug getters
   // measurement
   int profiling;
+  int early_plan;                 // gp_set_early_plan: the plan kernel reads the caller's inputs before its wait
   cudaEvent_t ev[GP_N_KERNELS + 1];
   float ms[GP_N_KERNELS];
   int64_t launches[GP_N_KERNELS];
@@ -267,8 +268,9 @@ __device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __re
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
                const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n) {
-  // plan_on: CTA 0 plans (off for the per-layer calls after the step's first); the summary CTAs cover the
-  // (layer, KV head) units [lh0, lh0 + lh_n) (none when lh_n is 0: the query rows come layer by layer)
+  // plan_on: 0: no planning (the per-layer calls after the step's first); 1: CTA 0 plans; 2: CTA 0 plans and
+  // the caller's inputs may be read before the wait for the preceding kernel (see below).  The summary CTAs
+  // cover the (layer, KV head) units [lh0, lh0 + lh_n) (none when lh_n is 0: the query rows come layer by layer)
   __shared__ int sv[33];
   __shared__ long long sw[33];
   __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
@@ -287,7 +289,10 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   // a whole still ends after everything before it.  The layer-by-layer launches (plan_on == 0) have no CTA 0
   // work and keep the wait in every CTA, so that completion stays transitive.  The next kernel may be scheduled
   // as soon as every CTA of this grid has started; it waits for this grid's end at its own top.
-  if (!plan_on) gp_pdl_wait();
+  // All of this reads the caller's request ids and queries before the wait, which is only right if they were
+  // complete before the preceding kernel could signal: the caller says so (plan_on == 2); otherwise every CTA
+  // waits first (the later wait of CTA 0 is then a no-op).
+  if (plan_on != 2) gp_pdl_wait();
   gp_pdl_launch_dependents();
   if (blockIdx.x > 0) {                       // summary CTAs: one warp per (unit, view, head)
     // The state of the batch's requests is staged once per CTA, from the L2 (these CTAs may run before the wait,
@@ -624,6 +629,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   pool->bytes = bytes;
   pool->live.assign(cfg->max_requests, 0);
   pool->profiling = 0;
+  pool->early_plan = 0;
   pool->step_open = 0; pool->step_n_req = 0; pool->step_layers_done = 0;
   pool->launch_count = 0;
   memset(pool->ms, 0, sizeof(pool->ms));
@@ -791,7 +797,7 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   const bool prof = pool->profiling != 0;
   if (prof) cudaEventRecord(pool->ev[0], s);
   const bool pdl = !prof;                      // events between the kernels need them serialised the plain way
-  launch_plan(pool, dev_req_ids, n_req, dev_actions, q, 1, 0, LH, s, pdl);
+  launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl);
   if (prof) cudaEventRecord(pool->ev[1], s);
   gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH);
   if (prof) cudaEventRecord(pool->ev[2], s);
@@ -889,9 +895,12 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
   const bool direct = cudaHostGetDevicePointer(&d_out, out, 0) == cudaSuccess &&
                       cudaHostGetDevicePointer(&d_act, actions, 0) == cudaSuccess;
   if (!direct) (void)cudaGetLastError();           // pageable memory: not an error, the staged path takes over
+  const int early = pool->early_plan;
+  pool->early_plan = 1;                            // the inputs arrive by the copies above: complete before any kernel
   const int st = gp_decode_step(pool, pool->st_ids, n_req, pool->st_q, pool->st_k, pool->st_v,
                                 direct ? d_out : static_cast<void*>(pool->st_out),
                                 direct ? static_cast<int32_t*>(d_act) : pool->st_act, stream);
+  pool->early_plan = early;
   if (st != GP_OK) return st;
   if (!direct) {
     GP_CUDA(cudaMemcpyAsync(out, pool->st_out, qb * 2, cudaMemcpyDeviceToHost, s));
@@ -1032,6 +1041,12 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
     for (int i = 0; i < 12; ++i) counters[i] = c[i];
     counters[7] = err;
   }
+  return GP_OK;
+}
+
+int gp_set_early_plan(gp_pool* pool, int32_t enable) {
+  if (!pool) return GP_ERR_INVALID;
+  pool->early_plan = enable ? 1 : 0;
   return GP_OK;
 }
 

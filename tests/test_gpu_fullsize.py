@@ -38,6 +38,7 @@ def test_bench_configuration_sampled_requests():
     cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
                         max_pages_per_req=wl.max_pages_per_req, max_requests=nreq, k_loc=wl.k_loc, host_staging=True)
     gpu = B.Pool(cfg, 0)
+    B.gp_set_early_plan(gpu.handle, True)          # as in the benchmark: the inputs are resident tensors
     ocfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=len(SAMPLE) * wl.max_pages_per_req,
                           max_pages_per_req=wl.max_pages_per_req, max_requests=len(SAMPLE), k_loc=wl.k_loc)
     ora = O.OraclePool(ocfg)

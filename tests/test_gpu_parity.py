@@ -702,10 +702,10 @@ def test_a_32k_token_request_at_the_32b_head_shape():
 
 
 def test_overlapped_launches_equal_plain_launches():
-    # In the normal mode the kernels of a step are chained with programmatic dependent launch and the plan of a
-    # step runs beside the compaction of the step before; in profiling mode every kernel is launched the plain
-    # way, after the one before it has ended.  Same inputs, both modes: outputs, actions, page tables, retained
-    # sets and summaries must be equal bit for bit.
+    # In the normal mode the kernels of a step are chained with programmatic dependent launch; with early
+    # planning on, the plan of a step also runs beside the compaction of the step before; in profiling mode every
+    # kernel is launched the plain way, after the one before it has ended.  Same inputs, all three: outputs,
+    # actions, page tables, retained sets and summaries must be equal bit for bit.
     import torch
     wl = W.layer8b(seed=5, n_requests=24, n_steps=200, prompt_range=(100, 700))
     s = wl.shape
@@ -722,13 +722,14 @@ def test_overlapped_launches_equal_plain_launches():
     qd, kd, vd = dev(q), dev(k), dev(v)
     ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
     results = []
-    for plain in (False, True):
+    for plain, early in ((False, False), (True, False), (False, True)):
         pool = B.Pool(B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
                                     max_pages_per_req=wl.max_pages_per_req, max_requests=n, tau=-0.003))
         try:
             for i in range(n):
                 assert pool.request_add(-1, 0, prompts[i][0], prompts[i][1], wl.requests[i].prompt_len, 0)[0] == B.GP_OK
             B.gp_set_profiling(pool.handle, plain)
+            B.gp_set_early_plan(pool.handle, early)
             outs = torch.zeros((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda:0")
             acts = torch.zeros((T, n), dtype=torch.int32, device="cuda:0")
             for t in range(T):
@@ -741,8 +742,9 @@ def test_overlapped_launches_equal_plain_launches():
             results.append((outs.cpu().numpy(), acts.cpu().numpy(), state, kept, summ))
         finally:
             pool.close()
-    a, b_ = results
-    assert np.array_equal(a[1], b_[1]) and a[2] == b_[2]
-    assert all(np.array_equal(x, y) for x, y in zip(a[3], b_[3])) and all(np.array_equal(x, y) for x, y in zip(a[4], b_[4]))
-    assert np.array_equal(a[0], b_[0])
+    a = results[0]
+    for b_ in results[1:]:
+        assert np.array_equal(a[1], b_[1]) and a[2] == b_[2]
+        assert all(np.array_equal(x, y) for x, y in zip(a[3], b_[3])) and all(np.array_equal(x, y) for x, y in zip(a[4], b_[4]))
+        assert np.array_equal(a[0], b_[0])
     assert (a[1] == B.GP_ACT_GROW).any() and (a[1] == B.GP_ACT_COMPRESS).any()
