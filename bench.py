@@ -162,6 +162,7 @@ class Job:
         self.act_dev = torch.zeros(self.nreq, dtype=torch.int32, device=dev)
         self.out_host = torch.zeros((s.n_layers, self.nreq, s.n_q_heads, s.head_dim), dtype=torch.float32).pin_memory()
         self.act_host = torch.zeros(self.nreq, dtype=torch.int32).pin_memory()
+        self._host_ptrs = None
         self.live = False
         self.by_layer = False           # True: steps go through gp_step_begin / gp_attn_layer / gp_step_end
         self.reset()
@@ -186,8 +187,15 @@ class Job:
         self.t += 1
 
     def step_host(self):
-        self.pool.decode_step_host(self.ids_host, self.q_host[self.t], self.k_host[self.t], self.v_host[self.t],
-                                   self.out_host, self.act_host)
+        # gp_decode_step_host through the binding, with the host addresses of this step's inputs worked out here
+        # (the tensors are contiguous [T][...]): the call a C caller makes, without a tensor view per argument
+        if self._host_ptrs is None:
+            self._host_ptrs = (self.pool.handle, self.ids_host.data_ptr(), self.q_host.data_ptr(), self.k_host.data_ptr(),
+                               self.v_host.data_ptr(), self.out_host.data_ptr(), self.act_host.data_ptr(),
+                               self.q_host[0].numel() * 2, self.k_host[0].numel() * 2, self.pool.stream())
+        h, ids, qp, kp, vp, op, ap, qs, ks, strm = self._host_ptrs
+        t = self.t
+        self.B.gp_decode_step_host(h, ids, self.nreq, qp + t * qs, kp + t * ks, vp + t * ks, op, ap, strm)
         self.t += 1
 
     def roll(self, t_to):
