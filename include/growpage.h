@@ -167,10 +167,12 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
 int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions,
                 void* stream);
 
-/* As gp_decode_step with HOST pointers: copies the inputs to staging inside the blob, runs the
- * step, delivers `out` and `actions` and synchronises `stream`.  When `out` and `actions` are
- * page-locked, mapped host memory (cudaHostAlloc / cudaHostRegister: "pinned"), the kernels write
- * them directly while they run; otherwise the results are staged on the device and copied back.
+/* As gp_decode_step with HOST pointers: brings the inputs to staging inside the blob, runs the
+ * step, delivers `out` and `actions` and synchronises `stream`.  When the four input buffers are
+ * page-locked, mapped host memory (cudaHostAlloc / cudaHostRegister: "pinned"), 16-byte aligned, and
+ * n_req is a multiple of 4, one kernel fetches them over the bus; otherwise four copies do.  When
+ * `out` and `actions` are pinned, the kernels write them directly while they run; otherwise the
+ * results are staged on the device and copied back.
  * Needs host_staging = 1 at creation, else GP_ERR_STATE. */
 int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req,
                         const void* q, const void* k, const void* v,

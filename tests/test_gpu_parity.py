@@ -542,7 +542,8 @@ def test_sequence_lengths_around_chunk_and_page_edges():
 
 
 def test_host_entry_point_with_pageable_buffers():
-    # gp_decode_step_host writes pinned outputs over the bus as it runs; pageable buffers take the staged copies
+    # gp_decode_step_host fetches pinned inputs with one kernel over the bus (the ids fill whole 16-byte pieces
+    # here: four requests) and writes pinned outputs over the bus as it runs; pageable buffers take copies
     import torch
     cfg = B.make_config(1, 8, 2, 64, n_pages=32, max_pages_per_req=4, max_requests=8, host_staging=True)
     results = []
@@ -552,15 +553,15 @@ def test_host_entry_point_with_pageable_buffers():
             rng = np.random.default_rng(0)
             bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
             kt, vt = bits(1, 20, 2, 64), bits(1, 20, 2, 64)
-            for i in range(3):
+            for i in range(4):
                 assert pool.request_add(-1, 0, kt, vt, 20, 0) == (B.GP_OK, i)
             fix = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
             outs = []
             for t in range(14):                                   # crosses the boundary at n = 32
-                q, k, v = bits(1, 3, 8, 64), bits(1, 3, 2, 64), bits(1, 3, 2, 64)
-                out = fix(torch.zeros((1, 3, 8, 64), dtype=torch.float32))
-                act = fix(torch.zeros(3, dtype=torch.int32))
-                ids = fix(torch.arange(3, dtype=torch.int32))
+                q, k, v = bits(1, 4, 8, 64), bits(1, 4, 2, 64), bits(1, 4, 2, 64)
+                out = fix(torch.zeros((1, 4, 8, 64), dtype=torch.float32))
+                act = fix(torch.zeros(4, dtype=torch.int32))
+                ids = fix(torch.arange(4, dtype=torch.int32))
                 tq, tk, tv = (fix(torch.from_numpy(x.view(np.int16))) for x in (q, k, v))
                 pool.decode_step_host(ids, tq, tk, tv, out, act)
                 outs.append((out.clone().numpy(), act.clone().numpy()))
