@@ -169,8 +169,8 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
 
 /* As gp_decode_step with HOST pointers: brings the inputs to staging inside the blob, runs the
  * step, delivers `out` and `actions` and synchronises `stream`.  When the four input buffers are
- * page-locked, mapped host memory (cudaHostAlloc / cudaHostRegister: "pinned"), 16-byte aligned, and
- * n_req is a multiple of 4, one kernel fetches them over the bus; otherwise four copies do.  When
+ * page-locked, mapped host memory (cudaHostAlloc / cudaHostRegister: "pinned") and q, k, v are
+ * 16-byte aligned, one kernel fetches them over the bus; otherwise four copies do.  When
  * `out` and `actions` are pinned, the kernels write them directly while they run; otherwise the
  * results are staged on the device and copied back.
  * Needs host_staging = 1 at creation, else GP_ERR_STATE. */

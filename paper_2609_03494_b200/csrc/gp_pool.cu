@@ -872,18 +872,20 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
   return GP_OK;
 }
 
-// The step's inputs, read from page-locked mapped host memory over the bus by one kernel: four ranges of 16-byte
-// pieces, every piece its own load, all in flight together (four separate copies cost their set-up four times).
-__global__ void gp_fetch_inputs_kernel(uint4* __restrict__ d0, const uint4* __restrict__ s0, long long n0,
+// The step's inputs, read from page-locked mapped host memory over the bus by one kernel: the request ids word
+// by word, queries, keys and values in 16-byte pieces, every piece its own load, all in flight together (four
+// separate copies cost their set-up four times).
+__global__ void gp_fetch_inputs_kernel(int* __restrict__ d_ids, const int* __restrict__ s_ids, int n_ids,
                                        uint4* __restrict__ d1, const uint4* __restrict__ s1, long long n1,
                                        uint4* __restrict__ d2, const uint4* __restrict__ s2, long long n2,
                                        uint4* __restrict__ d3, const uint4* __restrict__ s3, long long n3) {
-  const long long total = n0 + n1 + n2 + n3;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-    if (i < n0) d0[i] = s0[i];
-    else if (i < n0 + n1) d1[i - n0] = s1[i - n0];
-    else if (i < n0 + n1 + n2) d2[i - n0 - n1] = s2[i - n0 - n1];
-    else d3[i - n0 - n1 - n2] = s3[i - n0 - n1 - n2];
+  const long long total = n1 + n2 + n3;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (tid < n_ids) d_ids[tid] = s_ids[tid];
+  for (long long i = tid; i < total; i += (long long)gridDim.x * blockDim.x) {
+    if (i < n1) d1[i] = s1[i];
+    else if (i < n1 + n2) d2[i - n1] = s2[i - n1];
+    else d3[i - n1 - n2] = s3[i - n1 - n2];
   }
 }
 
@@ -901,18 +903,18 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
   // Inputs: from mapped page-locked buffers one kernel fetches all four over the bus; otherwise four copies.
   {
     void *mi = nullptr, *mq = nullptr, *mk = nullptr, *mv = nullptr;
-    const size_t ib = ((size_t)n_req * 4 + 15) / 16 * 16;       // the staging area is padded; a few bytes past the ids
-    const bool mapped = ((uintptr_t)host_req_ids % 16 == 0) && ((uintptr_t)q % 16 == 0) && ((uintptr_t)k % 16 == 0) &&
-                        ((uintptr_t)v % 16 == 0) && ((size_t)n_req * 4 % 16 == 0) &&
+    const bool mapped = ((uintptr_t)host_req_ids % 4 == 0) && ((uintptr_t)q % 16 == 0) && ((uintptr_t)k % 16 == 0) &&
+                        ((uintptr_t)v % 16 == 0) &&
                         cudaHostGetDevicePointer(&mi, const_cast<int32_t*>(host_req_ids), 0) == cudaSuccess &&
                         cudaHostGetDevicePointer(&mq, const_cast<void*>(q), 0) == cudaSuccess &&
                         cudaHostGetDevicePointer(&mk, const_cast<void*>(k), 0) == cudaSuccess &&
                         cudaHostGetDevicePointer(&mv, const_cast<void*>(v), 0) == cudaSuccess;
     if (mapped) {
-      const long long pieces = (long long)(ib + qb + 2 * kb) / 16;
+      const long long pieces = (long long)(qb + 2 * kb) / 16;         // a row is 128 or 256 bytes: whole pieces
       int grid = (int)((pieces + 255) / 256);
       if (grid > pool->num_sms * 8) grid = pool->num_sms * 8;
-      gp_fetch_inputs_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<uint4*>(pool->st_ids), static_cast<const uint4*>(mi), (long long)ib / 16,
+      if (grid * 256 < n_req) grid = (n_req + 255) / 256;
+      gp_fetch_inputs_kernel<<<grid, 256, 0, s>>>(pool->st_ids, static_cast<const int*>(mi), n_req,
                                                  static_cast<uint4*>(pool->st_q), static_cast<const uint4*>(mq), (long long)qb / 16,
                                                  static_cast<uint4*>(pool->st_k), static_cast<const uint4*>(mk), (long long)kb / 16,
                                                  static_cast<uint4*>(pool->st_v), static_cast<const uint4*>(mv), (long long)kb / 16);
