@@ -48,7 +48,7 @@ struct Geo {
   static constexpr int TILE_BYTES = 2 * GP_PAGE * ROW_BYTES;
   static constexpr int KSTEPS = D / 16;
   static constexpr int DTILES = D / 8;
-  static constexpr int SLOT_DESC = 256;                                // 64 ints: descriptor, then the page ids
+  static constexpr int SLOT_DESC = 384;                                // 96 ints: descriptor (32), then up to 64 page ids
   static constexpr int SLOT_PAGES = 32;                                // first page id (int index)
   static constexpr int SLOT_BYTES = (SLOT_DESC + 8 * ROW_BYTES + 2 * ROW_BYTES + 127) / 128 * 128;
 };
@@ -159,7 +159,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     };
     long long itA = item_of_tick(0), itB = total, itC = total;
     int hB = 0, hC = 0;                        // descriptor header, word `lane` (lanes 0..15)
-    int pC = -1;                               // page id of tile `lane` of the item
+    int pC = -1, pC2 = -1;                     // page ids of tiles `lane` and `lane + 32` of the item
     int slC = 0;                               // slot of the item in stage C
     uint32_t n_pub = 0;
     bool sentinel_out = false;
@@ -196,12 +196,13 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       // ---- issue the loads of the young stages --------------------------------------------------
       int hNew = 0;
       if (itA < total && lane < GP_DESC_INTS) hNew = p.rcx[(size_t)(itA / lh_n) * GP_DESC_INTS + lane];
-      int pNew = -1;
+      int pNew = -1, pNew2 = -1;
       int slNew = 0;
       // ---- page ids of stage C have arrived: into the slot, which is then complete ----------------------
       if (itC < total) {
         int* sd = reinterpret_cast<int*>(smem + L.off_slots + slC * GEO::SLOT_BYTES);
         sd[GEO::SLOT_PAGES + lane] = pC;
+        sd[GEO::SLOT_PAGES + 32 + lane] = pC2;
         __syncwarp();
         if (lane == 0) mbar_arrive(&slot_full[slC]);
       }
@@ -230,6 +231,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           const int chunk = __shfl_sync(0xffffffffu, hB, 4);
           const int nchunks = __shfl_sync(0xffffffffu, hB, 5);
           if (lane < npg) pNew = p.page_table[(size_t)r * p.cap + pg0 + lane];
+          if (lane + 32 < npg) pNew2 = p.page_table[(size_t)r * p.cap + pg0 + 32 + lane];
           if (lane < 14) sd[lane] = hB;
           if (lane == 14) sd[14] = lh;
           __syncwarp();
@@ -258,7 +260,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       }
       if (sentinel_out && itC >= total) break;
       // ---- rotate -----------------------------------------------------------------------------------------
-      itC = itB; hC = hB; pC = pNew; slC = slNew;
+      itC = itB; hC = hB; pC = pNew; pC2 = pNew2; slC = slNew;
       itB = itA; hB = hNew;
       itA = item_of_tick((long long)tick + 1);
     }

@@ -23,7 +23,7 @@
 #define GP_MAX_REQ 1024        // upper limit of max_requests (shared-memory arrays are sized by it)
 #define GP_SCORE_TILE 128      // candidate tokens per boundary-scoring tile
 #define GP_MOVE_TOK 64         // source slots per compaction chunk
-#define GP_COST_BINS 160       // cost classes of attention work items (pages, x4 at a boundary)
+#define GP_COST_BINS 288       // cost classes of attention work items (pages, x4 at a boundary)
 #define GP_DESC_INTS 16        // ints per attention work descriptor
 
 // pages per work item of a request that is at its capacity boundary

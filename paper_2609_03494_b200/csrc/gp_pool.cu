@@ -62,9 +62,9 @@ inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 int chunk_pages_setting() {
   const char* e = getenv("GP_CHUNK_PAGES");
-  int v = e ? atoi(e) : 32;
+  int v = e ? atoi(e) : 64;
   if (v < 1) v = 1;
-  if (v > 32) v = 32;
+  if (v > 64) v = 64;
   return v;
 }
 
