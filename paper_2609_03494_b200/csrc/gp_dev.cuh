@@ -26,9 +26,6 @@
 #define GP_COST_BINS 288       // cost classes of attention work items (pages, x4 at a boundary)
 #define GP_DESC_INTS 16        // ints per attention work descriptor
 
-// pages per work item of a request that is at its capacity boundary
-__host__ __device__ inline int gp_boundary_chunk(int chunk_pages) { return chunk_pages / 4 > 4 ? chunk_pages / 4 : 4; }
-
 // plan header slots (int32)
 enum {
   HDR_N_RC = 0,      // (request, chunk) work items of this step
@@ -59,6 +56,7 @@ struct GpDev {
   int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;
   long long n_pages, max_batch_tokens;
   double beta_s, beta_l, top_p, tau, rope_theta;
+  int bchunk_pages;                      // pages per work item of a request at its capacity boundary
   int policy;                            // GP_POLICY_* (0 demand, 1 inverse, 2 random, 3 shrink)
   unsigned long long policy_seed;
   double p_compress;

@@ -60,6 +60,17 @@ struct Layout {
 
 inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// pages per attention work item: 64 (two page ids per producer lane), and half of that for requests at their
+// capacity boundary; both can be overridden from the environment for experiments
+int chunk_pages_setting();
+int bchunk_pages_setting() {
+  const char* e = getenv("GP_BCHUNK_PAGES");
+  int v = e ? atoi(e) : chunk_pages_setting() / 2;
+  if (v < 4) v = 4;
+  if (v > 64) v = 64;
+  return v;
+}
+
 int chunk_pages_setting() {
   const char* e = getenv("GP_CHUNK_PAGES");
   int v = e ? atoi(e) : 64;
@@ -98,7 +109,8 @@ Layout make_layout(const gp_config& c) {
   const size_t np = (size_t)c.n_pages;
   L.max_batch_tokens = c.max_batch_tokens > 0 ? c.max_batch_tokens : (long long)(np * b);
   const int ch = chunk_pages_setting();
-  L.max_rc = (int)((size_t)L.max_batch_tokens / (b * gp_boundary_chunk(ch)) + 2 * M + 1);
+  const int bch = bchunk_pages_setting() < ch ? bchunk_pages_setting() : ch;
+  L.max_rc = (int)((size_t)L.max_batch_tokens / (b * bch) + 2 * M + 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
   L.kv = take(LH * np * 2 * b * d * 2);
@@ -365,10 +377,10 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     } else {
       pages = n_old / GP_PAGE + 1;
       if (n_old + 1 == Pr * GP_PAGE) {
-        // a page of a boundary request also pays for the fp64 summary logits: four times smaller items
-        // keep the cost of an item about the same
+        // a page of a boundary request also pays for the fp64 summary logits: its items are half as large
+        // (measured best: 16, 24, 40 and 48 pages against 64 for the others were all slower)
         isb = 1; nc = (long long)(Pr - 1) * GP_PAGE;
-        cp = gp_boundary_chunk(p.chunk_pages);
+        cp = p.bchunk_pages;
       }
       chunks = (pages + cp - 1) / cp;
       cp = (pages + chunks - 1) / chunks;            // equal sizes: chunks of cp pages, the last one shorter
@@ -644,6 +656,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.L = cfg->n_layers; d.Hq = cfg->n_q_heads; d.Hkv = cfg->n_kv_heads; d.G = cfg->n_q_heads / cfg->n_kv_heads;
   d.d = cfg->head_dim; d.M = cfg->max_requests; d.cap = cfg->max_pages_per_req; d.k_loc = cfg->k_loc;
   d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc;
+  d.bchunk_pages = bchunk_pages_setting();
   d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
   d.z_stride = (L.max_batch_tokens + GP_PAGE - 1) / GP_PAGE * GP_PAGE;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
