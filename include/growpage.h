@@ -159,7 +159,9 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
  *                   work has run, `out` is complete.  Every layer exactly once, in any order;
  *   gp_step_end     working sets, decisions, allocation, compaction; writes `dev_actions`.
  * Same ids, n_req and stream discipline as gp_decode_step; between gp_step_begin and gp_step_end no other
- * step of the pool may be issued (GP_ERR_STATE).  The results equal gp_decode_step's bit for bit. */
+ * step of the pool may be issued (GP_ERR_STATE).  Actions, page state, retained sets and summaries
+ * equal gp_decode_step's bit for bit; the attention outputs agree to fp32 rounding (long requests
+ * are cut into work items of different sizes, so partial results are merged in another order). */
 int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions,
                   void* stream);
 int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req,

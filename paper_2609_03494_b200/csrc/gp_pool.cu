@@ -61,7 +61,11 @@ struct Layout {
 inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // pages per attention work item: 64 (two page ids per producer lane), and half of that for requests at their
-// capacity boundary; both can be overridden from the environment for experiments
+// capacity boundary; both can be overridden from the environment for experiments.  When an attention launch has
+// fewer (request, layer, head) units than CTAs (small batches; a layer-by-layer launch, which covers one layer's
+// heads only), smaller items (32 and 8 pages) keep more CTAs busy (measured: the 36-layer shape with 16
+// requests, layer by layer, takes 1030 us per step that way, 1252 with the large items).
+constexpr int GP_FINE_CHUNK = 32, GP_FINE_BCHUNK = 8;
 int chunk_pages_setting();
 int bchunk_pages_setting() {
   const char* e = getenv("GP_BCHUNK_PAGES");
@@ -109,7 +113,8 @@ Layout make_layout(const gp_config& c) {
   const size_t np = (size_t)c.n_pages;
   L.max_batch_tokens = c.max_batch_tokens > 0 ? c.max_batch_tokens : (long long)(np * b);
   const int ch = chunk_pages_setting();
-  const int bch = bchunk_pages_setting() < ch ? bchunk_pages_setting() : ch;
+  int bch = bchunk_pages_setting() < ch ? bchunk_pages_setting() : ch;
+  if (bch > GP_FINE_BCHUNK) bch = GP_FINE_BCHUNK;            // small launches cut finer
   L.max_rc = (int)((size_t)L.max_batch_tokens / (b * bch) + 2 * M + 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
@@ -279,7 +284,8 @@ __device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __re
 // step's append (trailing check: n + 1 == P b) and hands each a slice of the logit scratch.
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
-               const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n) {
+               const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n, int cp_norm, int cp_bnd) {
+  // cp_norm, cp_bnd: pages per work item, for requests in general and for those at their capacity boundary
   // plan_on: 0: no planning (the per-layer calls after the step's first); 1: CTA 0 plans; 2: CTA 0 plans and
   // the caller's inputs may be read before the wait for the preceding kernel (see below).  The summary CTAs
   // cover the (layer, KV head) units [lh0, lh0 + lh_n) (none when lh_n is 0: the query rows come layer by layer)
@@ -361,7 +367,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   int chunks = 0, pages = 0, n_old = 0, act = GP_ACT_NONE, Pr = 0, started = 0, par = 0;
   long long nc = 0, pos = 0;
   int isb = 0;
-  int cp = p.chunk_pages;                 // pages per work item of this request
+  int cp = cp_norm;                       // pages per work item of this request
   int live = 0;
   if (in && r >= 0 && r < p.M) {          // independent loads, issued together (from the L2: before the wait)
     live = __ldcg(p.live + r); n_old = __ldcg(p.n + r); Pr = __ldcg(p.P + r); pos = __ldcg(p.pos + r);
@@ -380,7 +386,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
         // a page of a boundary request also pays for the fp64 summary logits: its items are half as large
         // (measured best: 16, 24, 40 and 48 pages against 64 for the others were all slower)
         isb = 1; nc = (long long)(Pr - 1) * GP_PAGE;
-        cp = p.bchunk_pages;
+        cp = cp_bnd;
       }
       chunks = (pages + cp - 1) / cp;
       cp = (pages + chunks - 1) / chunks;            // equal sizes: chunks of cp pages, the last one shorter
@@ -787,14 +793,19 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
 
 // CTA 0 plans (when plan_on); the others update the query summaries of the units [lh0, lh0 + lh_n)
 static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_t* actions, const void* q, int plan_on,
-                        int lh0, int lh_n, cudaStream_t s, bool pdl) {
+                        int lh0, int lh_n, cudaStream_t s, bool pdl, bool by_layer = false) {
   const GpDev& d = pool->dev;
   const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
   const long long want = ((long long)n_req * lh_n + upc - 1) / upc;
   const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
   const int prep = (int)(want < room ? want : room);
+  // work-item size: large when one attention launch has at least a (request, layer, head) unit per CTA, fine
+  // otherwise (a layer-by-layer launch covers one layer's heads only)
+  const long long launch_units = (long long)n_req * (by_layer ? d.Hkv : d.L * d.Hkv);
+  const bool fine = launch_units < pool->attn_grid;
   gp_launch(gp_plan_kernel, 1 + prep, GP_PLAN_THREADS, 0, s, pdl, d, ids, n_req, actions,
-            static_cast<const __nv_bfloat16*>(q), plan_on, lh0, lh_n);
+            static_cast<const __nv_bfloat16*>(q), plan_on, lh0, lh_n, fine ? GP_FINE_CHUNK : d.chunk_pages,
+            fine ? GP_FINE_BCHUNK : d.bchunk_pages);
 }
 
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
@@ -839,7 +850,7 @@ int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int3
   if (n_req == 0) return GP_OK;
   if (!dev_req_ids || !dev_actions) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
-  launch_plan(pool, dev_req_ids, n_req, dev_actions, nullptr, 1, 0, 0, static_cast<cudaStream_t>(stream), true);
+  launch_plan(pool, dev_req_ids, n_req, dev_actions, nullptr, 1, 0, 0, static_cast<cudaStream_t>(stream), true, true);
   pool->launch_count += 1;
   pool->step_open = 1;
   pool->step_n_req = n_req;

@@ -356,7 +356,8 @@ def test_shrink_policy_of_eq13(config, over, mixed):
 
 def test_layer_by_layer_entry_points_equal_the_whole_step():
     # gp_step_begin / gp_attn_layer (layers in a shuffled order) / gp_step_end against gp_decode_step on the same
-    # inputs: outputs, actions, page state, retained sets and summaries bit for bit; and the state checks
+    # inputs: actions, page state, retained sets and summaries bit for bit, outputs to fp32 rounding; and the
+    # state checks
     import torch
     shape = W.Shape(5, 8, 2, 64)
     reqs = [W.RequestSpec(i, 150 + 37 * i, 60, 0.05) for i in range(6)]
@@ -414,7 +415,9 @@ def test_layer_by_layer_entry_points_equal_the_whole_step():
     assert np.array_equal(whole[1], layered[1]) and whole[2] == layered[2]
     assert all(np.array_equal(a, b_) for a, b_ in zip(whole[3], layered[3]))
     assert all(np.array_equal(a, b_) for a, b_ in zip(whole[4], layered[4]))
-    assert np.array_equal(whole[0], layered[0])
+    # the two entry points cut long requests into work items of different sizes, so the attention outputs agree
+    # to the rounding of the order in which partial results are merged, not to the bit
+    assert np.abs(whole[0] - layered[0]).max() <= 2e-6
     assert (whole[1] == B.GP_ACT_GROW).any() and (whole[1] == B.GP_ACT_COMPRESS).any()
 
 
