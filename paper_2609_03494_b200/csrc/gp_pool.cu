@@ -62,9 +62,9 @@ inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // pages per attention work item: 64 (two page ids per producer lane), and half of that for requests at their
 // capacity boundary; both can be overridden from the environment for experiments.  When an attention launch has
-// fewer (request, layer, head) units than CTAs (small batches; a layer-by-layer launch, which covers one layer's
-// heads only), smaller items (32 and 8 pages) keep more CTAs busy (measured: the 36-layer shape with 16
-// requests, layer by layer, takes 1030 us per step that way, 1252 with the large items).
+// less than one such item of work per CTA (small batches, short sequences; a layer-by-layer launch, which covers
+// one layer's heads only), smaller items (32 and 8 pages) keep more CTAs busy (measured: the 36-layer shape with
+// 16 requests, layer by layer, takes 1030 us per step that way, 1252 with the large items).
 constexpr int GP_FINE_CHUNK = 32, GP_FINE_BCHUNK = 8;
 int chunk_pages_setting();
 int bchunk_pages_setting() {
@@ -284,8 +284,11 @@ __device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __re
 // step's append (trailing check: n + 1 == P b) and hands each a slice of the logit scratch.
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
-               const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n, int cp_norm, int cp_bnd) {
-  // cp_norm, cp_bnd: pages per work item, for requests in general and for those at their capacity boundary
+               const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n, int cp_norm, int cp_bnd,
+               int launch_units, int launch_grid) {
+  // cp_norm, cp_bnd: pages per work item, for requests in general and for those at their capacity boundary, when
+  // the attention launch has work for large items; launch_units: (layer, head) units per request in one
+  // attention launch; launch_grid: its CTAs
   // plan_on: 0: no planning (the per-layer calls after the step's first); 1: CTA 0 plans; 2: CTA 0 plans and
   // the caller's inputs may be read before the wait for the preceding kernel (see below).  The summary CTAs
   // cover the (layer, KV head) units [lh0, lh0 + lh_n) (none when lh_n is 0: the query rows come layer by layer)
@@ -382,15 +385,24 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       act = GP_ACT_STALLED;
     } else {
       pages = n_old / GP_PAGE + 1;
-      if (n_old + 1 == Pr * GP_PAGE) {
-        // a page of a boundary request also pays for the fp64 summary logits: its items are half as large
-        // (measured best: 16, 24, 40 and 48 pages against 64 for the others were all slower)
-        isb = 1; nc = (long long)(Pr - 1) * GP_PAGE;
-        cp = cp_bnd;
-      }
-      chunks = (pages + cp - 1) / cp;
-      cp = (pages + chunks - 1) / chunks;            // equal sizes: chunks of cp pages, the last one shorter
+      if (n_old + 1 == Pr * GP_PAGE) { isb = 1; nc = (long long)(Pr - 1) * GP_PAGE; }
     }
+  }
+  {
+    // Large items when an attention launch has at least one of them per CTA (pages of the batch x units per
+    // request / CTAs >= an item), fine ones otherwise: small batches, short sequences, layer-by-layer launches.
+    // Measured on one layer of the 8B shape: 8 to 48 requests of 30 to 50 pages are 2 to 8 us per step faster
+    // with fine items, 64 requests of 44 pages and more 3 us faster with large ones.
+    int e0, tot_pages; long long d0, d1;
+    plan_scan(pages, 0, e0, d0, tot_pages, d1, sv, sw);
+    if ((long long)tot_pages * launch_units < (long long)cp_norm * launch_grid) { cp_norm = GP_FINE_CHUNK; cp_bnd = GP_FINE_BCHUNK; }
+  }
+  if (pages > 0) {
+    // a page of a boundary request also pays for the fp64 summary logits: its items are half as large
+    // (measured best: 16, 24, 40 and 48 pages against 64 for the others were all slower)
+    cp = isb ? cp_bnd : cp_norm;
+    chunks = (pages + cp - 1) / cp;
+    cp = (pages + chunks - 1) / chunks;              // equal sizes: chunks of cp pages, the last one shorter
   }
   const long long t_plan1 = GP_T_NOW();
   (void)t_plan1;
@@ -799,13 +811,9 @@ static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_
   const long long want = ((long long)n_req * lh_n + upc - 1) / upc;
   const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
   const int prep = (int)(want < room ? want : room);
-  // work-item size: large when one attention launch has at least a (request, layer, head) unit per CTA, fine
-  // otherwise (a layer-by-layer launch covers one layer's heads only)
-  const long long launch_units = (long long)n_req * (by_layer ? d.Hkv : d.L * d.Hkv);
-  const bool fine = launch_units < pool->attn_grid;
   gp_launch(gp_plan_kernel, 1 + prep, GP_PLAN_THREADS, 0, s, pdl, d, ids, n_req, actions,
-            static_cast<const __nv_bfloat16*>(q), plan_on, lh0, lh_n, fine ? GP_FINE_CHUNK : d.chunk_pages,
-            fine ? GP_FINE_BCHUNK : d.bchunk_pages);
+            static_cast<const __nv_bfloat16*>(q), plan_on, lh0, lh_n, d.chunk_pages, d.bchunk_pages,
+            by_layer ? d.Hkv : d.L * d.Hkv, pool->attn_grid);
 }
 
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
