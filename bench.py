@@ -312,7 +312,7 @@ def run_ours(args):
     roofline = {
         "bound": "hbm", "kernel": "gp_attn_kernel<128> (append + paged GQA attention + boundary logits)",
         "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
-        "peak_kind": f"of {peak_kind}",
+        "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": round(achieved / NOMINAL_HBM_GBS, 4),
         "traffic": None if ratio is None else round(ratio * attn_bytes / K),
         "algorithmic_bytes_per_launch": round(attn_bytes / K),
         "launch_us": round(attn_ms * 1e3 / K, 2),
