@@ -111,15 +111,17 @@ int gp_config_default(gp_config* cfg);
 size_t gp_pool_bytes(const gp_config* cfg);
 
 /* Creates a pool inside `dev_blob` (device pointer, 256-byte aligned, at least gp_pool_bytes(cfg)
- * bytes, on CUDA device `device`).  The blob is cleared; every page starts on the free list
- * (Sec. 4.2 "global free-page pool").  Synchronous.  The blob must outlive the pool. */
+ * bytes, on CUDA device `device`).  The blob is cleared; every page starts on the free list (the
+ * pool-wide stock of free pages that growth draws on, Sec. 4.2).  Synchronous.  The blob must outlive
+ * the pool.  The only memory the library obtains itself is 64 bytes of page-locked host memory per pool
+ * for the kernels' error word (see gp_pool_status). */
 int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int device, gp_pool** out);
 
 /* Frees the host-side handle.  Synchronises the device first.  The blob is left to its owner. */
 int gp_pool_destroy(gp_pool* pool);
 
-/* Admits a request (App. D.1 "query slots are bound to requests when they enter the running
- * queue"; App. D.2 prefix sharing).  Its first `n_shared_pages` pages are shared by reference
+/* Admits a request: binds a summary slot to it at admission (App. D.1) and gives it its pages, the
+ * leading ones possibly shared (App. D.2 prefix sharing).  Its first `n_shared_pages` pages are shared by reference
  * count with live request `share_from` (-1 for none), which must still hold them as untouched
  * full prompt pages.  The rest of the prompt, `n_tail` tokens, is copied from k_tail / v_tail:
  * device pointers, bf16 [L][n_tail][H_kv][d], keys already in cache form (post-RoPE).
@@ -127,6 +129,7 @@ int gp_pool_destroy(gp_pool* pool);
  * On success *out_req receives the request id (the lowest free slot).  The summaries of the slot
  * are not cleared: the first decode step overwrites them.  Synchronises `stream`.
  * Errors, checked in this order: GP_ERR_INVALID (arguments; donor dead or with fewer shareable pages),
+ * GP_ERR_STATE (between gp_step_begin and gp_step_end: the open step holds a snapshot of the free list),
  * GP_ERR_NO_SLOT, GP_ERR_NO_PAGES (nothing is changed in these cases). */
 int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
                    const void* k_tail, const void* v_tail, int32_t n_tail,
@@ -140,6 +143,8 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
  *                the new one included; rows of requests whose action is GP_ACT_INVALID, or that
  *                were already full on entry, are not written
  *   dev_actions  device int32 [n_req]: GP_ACT_* per request
+ * q, k, v and out must be 16-byte aligned (the kernels move rows in 16-byte pieces), dev_req_ids and
+ * dev_actions 4-byte aligned: GP_ERR_INVALID otherwise, nothing is launched.
  * Asynchronous on `stream`; nothing is read back to the host, so (with profiling off) a sequence of
  * steps can be captured into a CUDA graph and replayed.  The step's kernels are chained with
  * programmatic dependent launch.  Steps of one pool must be issued on one stream (or otherwise
@@ -158,8 +163,11 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
  *                   out [n_req][H_q][d] fp32 are this layer's tensors (device pointers); when the call's
  *                   work has run, `out` is complete.  Every layer exactly once, in any order;
  *   gp_step_end     working sets, decisions, allocation, compaction; writes `dev_actions`.
- * Same ids, n_req and stream discipline as gp_decode_step; between gp_step_begin and gp_step_end no other
- * step of the pool may be issued (GP_ERR_STATE).  Actions, page state, retained sets and summaries
+ * Same ids, n_req, alignment and stream discipline as gp_decode_step; between gp_step_begin and gp_step_end
+ * no other step of the pool may be issued, and no request admitted or released (GP_ERR_STATE: the open step
+ * holds a snapshot of the free list).  A layer given twice is refused (GP_ERR_STATE), and so is gp_step_end
+ * while layers are missing; gp_step_abort leaves an open step without committing it: no request has advanced,
+ * rows the finished layers appended lie beyond the occupied slots and are overwritten by the next step.  Actions, page state, retained sets and summaries
  * equal gp_decode_step's bit for bit; the attention outputs agree to fp32 rounding (long requests
  * are cut into work items of different sizes, so partial results are merged in another order). */
 int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions,
@@ -168,6 +176,7 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
                   const void* q, const void* k, const void* v, void* out, void* stream);
 int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions,
                 void* stream);
+int gp_step_abort(gp_pool* pool);
 
 /* As gp_decode_step with HOST pointers: brings the inputs to staging inside the blob, runs the
  * step, delivers `out` and `actions` and synchronises `stream`.  When the four input buffers are
@@ -175,14 +184,26 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
  * 16-byte aligned, one kernel fetches them over the bus; otherwise four copies do.  When
  * `out` and `actions` are pinned, the kernels write them directly while they run; otherwise the
  * results are staged on the device and copied back.
- * Needs host_staging = 1 at creation, else GP_ERR_STATE. */
+ * Needs host_staging = 1 at creation, else GP_ERR_STATE.  After its synchronisation the call looks at the
+ * kernels' error word and returns GP_ERR_CUDA when a kernel reported an internal error (gp_pool_status). */
 int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req,
                         const void* q, const void* k, const void* v,
                         void* out, int32_t* actions, void* stream);
 
 /* Ends a request: every page of its table loses one reference and returns to the free list at
- * zero; the summary slot is recycled without clearing (App. D.1).  Asynchronous on `stream`. */
+ * zero; the summary slot is recycled without clearing (App. D.1).  Asynchronous on `stream`.
+ * GP_ERR_STATE between gp_step_begin and gp_step_end. */
 int gp_release(gp_pool* pool, int32_t req, void* stream);
+
+/* Internal errors reported by the kernels (a bounded wait that ran out, a failed bounds check, free-list
+ * accounting gone wrong): GP_OK, or GP_ERR_CUDA with the bits in *error_bits (may be NULL).  The kernels set
+ * the bits in a word of page-locked host memory, so this call neither synchronises nor copies; it reflects
+ * the work that has completed.  gp_decode_step is asynchronous and cannot report them itself:
+ * call this after synchronising its stream.  The bits are sticky for the life of the pool:
+ *   1 a bounded wait inside the attention kernel gave up   2 free-list accounting out of range
+ *   4 an index failed a bounds check (the access was skipped)   8 a bounded wait inside the compaction kernel gave up
+ * (bits 7 and up say which wait of the attention kernel it was). */
+int gp_pool_status(gp_pool* pool, int32_t* error_bits);
 
 /* Text for a status code. */
 const char* gp_strerror(int status);
@@ -258,7 +279,8 @@ int64_t gp_launch_count(gp_pool* pool);
  *
  *   q     device bf16 [n_req][n_q_heads][d]
  *   k, v  device bf16 [n_req][n_kv_heads][max_len][d], rows in plain order (no page layout, no swizzle)
- *   lens  device int32 [n_req]: tokens of each request, 1..max_len (values above max_len are clipped)
+ *   lens  device int32 [n_req]: tokens of each request, 1..max_len (values above max_len are clipped;
+ *         a request with lens <= 0 attends to nothing and gets an output row of zeros)
  *   out   device fp32 [n_req][n_q_heads][d]: softmax(q.K/sqrt(d)).V per query head, KV head g / G
  *
  * Limits: d is 64 or 128, G = n_q_heads / n_kv_heads <= 8, n_req * n_q_heads <= GP_NOALLOC_MAX_ROWS;

@@ -163,7 +163,7 @@ def attention_decode(q_hat: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndar
 def summary_attention(q_tilde: np.ndarray, Kc: np.ndarray) -> np.ndarray:
     """Attention of one temporal view over the candidate set of one KV head: each of the
     G query heads of the group takes its own softmax over C, the group mean is the head's
-    distribution (Sec. 3.2, App. D.1 "native GQA head mapping").  q_tilde [G][d], Kc [|C|][d]."""
+    distribution (Sec. 3.2; query heads keep their own KV head, App. D.1).  q_tilde [G][d], Kc [|C|][d]."""
     d = q_tilde.shape[-1]
     z = q_tilde @ Kc.T / math.sqrt(d)                    # [G][|C|]
     w = np.exp(z - z.max(axis=1, keepdims=True))

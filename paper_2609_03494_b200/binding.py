@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
     L.gp_step_begin.argtypes = [vp, vp, i32, vp, vp]
     L.gp_attn_layer.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
     L.gp_step_end.argtypes = [vp, vp, i32, vp, vp]
+    L.gp_step_abort.argtypes = [vp]
+    L.gp_pool_status.argtypes = [vp, C.POINTER(i32)]
     L.gp_set_profiling.argtypes = [vp, i32]
     L.gp_set_early_plan.argtypes = [vp, i32]
     L.gp_get_kernel_times.argtypes = [vp, vp, vp]
@@ -147,6 +149,17 @@ def gp_attn_layer(pool: int, layer: int, dev_req_ids_ptr: int, n_req: int, q_ptr
 def gp_step_end(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: int, stream: int) -> None:
     _check(lib().gp_step_end(C.c_void_p(pool), C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(dev_actions_ptr),
                              C.c_void_p(stream)), "gp_step_end")
+
+
+def gp_step_abort(pool: int) -> None:
+    _check(lib().gp_step_abort(C.c_void_p(pool)), "gp_step_abort")
+
+
+def gp_pool_status(pool: int) -> Tuple[int, int]:
+    """Returns (status, error bits) of the kernels' error word; the status is returned, not raised."""
+    bits = C.c_int32(0)
+    st = lib().gp_pool_status(C.c_void_p(pool), C.byref(bits))
+    return int(st), int(bits.value)
 
 
 def gp_release(pool: int, req: int, stream: int) -> None:

@@ -118,9 +118,6 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   const int comb_w = L.comb_warp / 4;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef GP_TRACE
-  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 32] = (long long)gt; }
-#endif
   if (tid == 0) {
     for (int i = 0; i < NI_MAX; ++i) { mbar_init(&slot_full[i], 2); mbar_init(&slot_empty[i], NCW + 1); }
     mbar_init(qt_full, 1);
@@ -211,10 +208,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       if (tick >= 1 && !sentinel_out) {
         const int sl = n_pub % NI;
         slNew = sl;
-        const long long t_p0 = GP_T_NOW();
-        (void)t_p0;
         if (!wait_polling(&slot_empty[sl], ((n_pub / NI) & 1u) ^ 1u)) break;
-        if (lane == 0) GP_T_ADD(11, GP_T_NOW() - t_p0);
         uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
         int* sd = reinterpret_cast<int*>(slot);
         if (itB >= total) {
@@ -277,10 +271,6 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     const int row = lane >> 2;
     const int qc = (lane & 3) * 2;
     uint32_t qt_uses = 0, my_tiles = 0;
-    const bool tr = (cw == 0 && lane == 0);
-    const long long t_loop0 = GP_T_NOW();
-    (void)tr; (void)t_loop0;
-    if (tr) GP_T_STAMP(64);
     // Each consumer warp fetches its own tiles (tile j of an item belongs to warp j mod 4) into its private
     // ring of NSW stages: as soon as it is done with a stage it issues the copy of its next tile but NSW - 1,
     // which may belong to a later item (the fetch position runs ahead of the compute position, across item
@@ -327,16 +317,12 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     };
     for (uint32_t it = 0;; ++it) {
       const int sl = it % NI;
-      const long long t_a = GP_T_NOW();
-      (void)t_a;
       if (!top_up(it)) break;
       if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc, 4)) break;
       const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
       if (npg < 0) break;
-      if (tr) { GP_T_ADD(0, 1); GP_T_ADD(2, GP_T_NOW() - t_a); if (it == 0) GP_T_STAMP(65); if (it == 1) GP_T_STAMP(69); if (it == 2) GP_T_STAMP(70); }
-      const long long t_a2 = GP_T_NOW(); (void)t_a2;
       const int bi = sd[0], pg0 = sd[2], chunk = sd[4], nchunks = sd[5], n_old = sd[6];
       const int flags = sd[8], Pr = sd[9], lh = sd[14];
       const int l = lh / p.Hkv, h = lh % p.Hkv;
@@ -382,10 +368,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         }
       }
       if (need_qt) {
-        const long long t_q = GP_T_NOW();
-        (void)t_q;
         if (!wait_bar(qt_full, qt_uses & 1u, s_misc, 5)) break;
-        if (tr) { GP_T_ADD(15, GP_T_NOW() - t_q); GP_T_ADD(7, 1); }
       }
 
       const bool last_chunk = (chunk == nchunks - 1);
@@ -395,12 +378,8 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       float m_run = -INFINITY, l_run = 0.f;
       bool ok = true;
 
-      if (tr) GP_T_ADD(77, GP_T_NOW() - t_a2);
-      long long t_prev = GP_T_NOW(); (void)t_prev;
       for (int pgl = (cw + it) % NCW; pgl < npg; pgl += NCW) {
         const uint32_t st = cw * NSW + (my_tiles % NSW);
-        const long long t_b = GP_T_NOW();
-        (void)t_b;
         {
           // one copy group per tile, in fetch order: all but the groups younger than this tile's must be done
           const uint32_t younger = my_fetch - my_tiles - 1;
@@ -408,9 +387,6 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           __syncwarp();
         }
         ++my_tiles;
-        const long long t_c = GP_T_NOW();
-        (void)t_c;
-        if (tr) { GP_T_ADD(1, 1); GP_T_ADD(3, t_c - t_b); if (my_tiles == 1) GP_T_STAMP(66); if (pgl < NCW) { GP_T_ADD(71, t_c - t_b); GP_T_ADD(72, 1); } }
         uint8_t* tile = smem + st * GEO::TILE_BYTES;
         const int tok0 = (pg0 + pgl) * GP_PAGE;
         const bool has_new = last_chunk && (pgl == npg - 1);
@@ -499,9 +475,6 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
             mma_bf16(o[jd + 1], pa[0], pa[1], pa[2], pa[3], v2, v3);
           }
         }
-        const long long t_d = GP_T_NOW();
-        (void)t_d;
-        if (tr) GP_T_ADD(4, t_d - t_c);
         // Boundary unit: fp64 logits of the calibrated summaries against the 16 keys of a candidate page,
         // Z[token][n] = sum_d K[token][d] q~[n][d], n = view * G + head.  One m8n8k4 DMMA covers 8 tokens,
         // 8 columns and 4 values of d; inside a 16-byte chunk of a key row lane t of a quad takes the
@@ -578,15 +551,11 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
               }
             }
           }
-          if (tr) { GP_T_ADD(8, GP_T_NOW() - t_d); GP_T_ADD(9, 1); }
         }
         __syncwarp();
         if (!top_up(it)) { ok = false; break; }            // the stage is free: fetch the next tile into it
       }
-      if (tr) GP_T_ADD(78, GP_T_NOW() - t_prev);
       if (!ok) break;
-      const long long t_e = GP_T_NOW();
-      (void)t_e;
 
       // ---- hand the partial result to the merger warp ---------------------------------------------
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
@@ -609,13 +578,8 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         if (lane == 0) mbar_arrive(qt_empty);
       }
       if (lane == 0) mbar_arrive(&slot_empty[sl]);
-      if (tr) { GP_T_ADD(5, GP_T_NOW() - t_e); if (it == 0) GP_T_STAMP(67); }
     }
     cp_async_wait<0>();                  // after an abort copies may still be in flight: let them land
-    if (tr) GP_T_ADD(6, GP_T_NOW() - t_loop0);
-#ifdef GP_TRACE
-    if (tr) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 35] = (long long)gt; }
-#endif
   } else if (warp == 2) {
     // ================================= merger =============================================
     for (uint32_t it = 0;; ++it) {
@@ -660,14 +624,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       if (lane == 0) mbar_arrive(&slot_empty[sl]);
     }
   }
-#ifdef GP_TRACE
-  if (lane == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 40 + warp] = (long long)gt; }
-#endif
   __syncthreads();
-#ifdef GP_TRACE
-  if (tid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 33] = (long long)gt; }
-  if (tid == 128) { unsigned long long gt; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + 34] = (long long)gt; }
-#endif
 }
 
 }  // namespace

@@ -109,13 +109,9 @@ __device__ __noinline__ int top_p_count(const GpDev& p, const double* a, int n, 
     const int w = kWidths[lvl];
     shift -= w;
     const int nb = 1 << w;
-    const long long t_l0 = GP_T_NOW();
-    (void)t_l0;
     for (int i = tid; i < nb + (nb >> 3); i += BT) { hcnt[i] = 0; hlo[i] = 0; hhi[i] = 0; }
     if (tid == 0) s_res[0] = -1;
     __syncthreads();
-    const long long t_l1 = GP_T_NOW();
-    (void)t_l1;
     for (int i = tid; i < n; i += BT) {
       const double v = a[i];
       const unsigned long long key = (unsigned long long)__double_as_longlong(v);
@@ -126,8 +122,6 @@ __device__ __noinline__ int top_p_count(const GpDev& p, const double* a, int n, 
       }
     }
     __syncthreads();
-    const long long t_l2 = GP_T_NOW();
-    (void)t_l2;
     const int per = nb / BT > 0 ? nb / BT : 1;
     const int lo = tid * per, hi = lo + per;     // this thread's bins [lo, hi)
     unsigned c = 0; unsigned long long s = 0;
@@ -220,7 +214,6 @@ __device__ __forceinline__ void warp_sort(double& v, int& tag) {
 __device__ int top_p_fast(const GpDev& p, const double* a, int n, unsigned long long p_fix, const FastHist& H,
                           unsigned* wc, unsigned long long* wsum, long long* s_res, double* list, int* s_cnt) {
   const int tid = threadIdx.x;
-  const long long f2 = GP_T_NOW(); (void)f2;
   for (int i = tid; i < n; i += SEL_T) {
     const double v = a[i];
     const int bin = (int)(((unsigned long long)__double_as_longlong(v) >> FSHIFT) & (FBINS - 1));
@@ -231,7 +224,6 @@ __device__ int top_p_fast(const GpDev& p, const double* a, int n, unsigned long 
     add64_split(&H.clo[bin >> 4], &H.chi[bin >> 4], f);
   }
   __syncthreads();
-  const long long f3 = GP_T_NOW(); (void)f3;
   {                                               // summary level: thread t owns bin t; higher bins = larger scores
     const unsigned c = tid < CBINS ? H.ccnt[tid] : 0u;
     const unsigned long long m = tid < CBINS ? ((unsigned long long)H.chi[tid] << 32) + H.clo[tid] : 0ull;
@@ -258,7 +250,6 @@ __device__ int top_p_fast(const GpDev& p, const double* a, int n, unsigned long 
     }
   }
   __syncthreads();
-  if (tid == 0) { GP_T_ADD(54, 1); GP_T_ADD(57, f3 - f2); GP_T_ADD(58, GP_T_NOW() - f3); }
   const int bstar = (int)s_res[4];
   const unsigned cnt_above = (unsigned)s_res[5];
   const unsigned long long sum_above = (unsigned long long)s_res[6];
@@ -405,8 +396,6 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
       need_eq = (int)ne - (int)cnt_below;
     }
   }
-  const long long t_s4 = GP_T_NOW();
-  (void)t_s4;
   for (int i = tid; i < nC; i += SEL_T) {
     if (!((loc[i >> 5] >> (i & 31)) & 1u)) {
       const unsigned long long key = (unsigned long long)__double_as_longlong(a[i]);
@@ -423,7 +412,6 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
       }
     }
     if (cntv != (int)ne) atomicOr(p.err, GP_E_BOUNDS);
-    GP_T_ADD(21, GP_T_NOW() - t_s4);
   }
 }
 
@@ -671,11 +659,9 @@ __device__ __noinline__ bool job_softmax(const GpDev& p, const double* __restric
       if (task == 2) xv[1][u] = ld_early2(xb + view_stride + 2 * (size_t)k);
     }
   }
-  const long long j0 = GP_T_NOW(); (void)j0;
   double m = fmax(keep[0].x, keep[1].x);
   for (int t = t0 + KEEP * tstep; t < ntile; t += tstep) m = fmax(m, __ldcg(zs + ((size_t)t * G2 + mycol) * 2));
   column_reduce<true>(m, ncols, red, sM);
-  const long long j1 = GP_T_NOW(); (void)j1;
   const double mc = sM[myc];
   double acc = 0.0;
 #pragma unroll
@@ -696,7 +682,6 @@ __device__ __noinline__ bool job_softmax(const GpDev& p, const double* __restric
   column_reduce<false>(acc, ncols, red, sZ);
   if (tid < ncols) sZ[tid] = 1.0 / ((double)GG * sZ[tid]);     // group mean and normaliser in one factor
   __syncthreads();
-  const long long j2 = GP_T_NOW(); (void)j2;
   unsigned top_bits = 0;
   for (int k0 = tid; k0 - tid < nv; k0 += U * SEL_T) {   // uniform trip count: the shuffles below need whole warps
     if (k0 != tid) {
@@ -754,7 +739,6 @@ __device__ __noinline__ bool job_softmax(const GpDev& p, const double* __restric
       }
     }
   }
-  if (tid == 0) { GP_T_ADD(12, j1 - j0); GP_T_ADD(13, j2 - j1); GP_T_ADD(14, GP_T_NOW() - j2); GP_T_ADD(30, 1); }
   // bits 62..58 of every score, as a set: the fast selection path needs them all equal.  (The block-wide
   // barrier reductions combine predicates, not words, so the sets are OR-ed by hand: per warp, then over the
   // warps through shared memory; `red` is free here.)
@@ -869,7 +853,6 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   gp_pdl_wait();
   gp_pdl_launch_dependents();
   const long long items = (long long)n_bnd * LH * NT;
-  if (tid == 0) GP_T_STAMP(59);
 
   // CTAs without a job merge the split requests' attention partials while the others work; when fewer than a
   // quarter of the CTAs are idle, everybody merges after the jobs instead
@@ -879,7 +862,6 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   if (idle_merge && (long long)blockIdx.x >= n_busy)
     merge_partials(p, n_req, out, n_mc, n_rc, (int)blockIdx.x - (int)n_busy, n_idle, 0, LH);
 
-  if (tid == 0) GP_T_STAMP(60);
   for (long long item = blockIdx.x; item < items + n_bnd; item += gridDim.x) {
     if (item >= items) {
       // pages of C that other requests share: each needs a copy-on-write target if this request compresses
@@ -915,8 +897,6 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       continue;
     }
     if (SHR && job == 3 && Pr - 1 < p.min_pages_after_shrink) continue;      // this boundary cannot be a Shrink
-    const long long t_s0 = GP_T_NOW();
-    (void)t_s0;
     const size_t view_stride = (size_t)p.z_stride * G;
     const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;   // [2 views][nC][G] exp(logit - page max)
     double* a = nC <= SEL_CAP ? sbuf : p.scores + ((size_t)job * LH + lh) * p.max_batch_tokens + off;
@@ -933,8 +913,6 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       }
     }
     fast_hist_zero(H, task < 2);                   // the factors' table shared this memory
-    const long long t_s1 = GP_T_NOW();
-    (void)t_s1;
     if (task < 2) {
       __syncthreads();
       // ---- Eq. 7 -------------------------------------------------------------------------------------------
@@ -943,7 +921,6 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       if (tid == 0) {
         Kout[task] = K;
         atomicAdd(&p.bnd_acc[4 * bidx + task], K);            // Eq. 8 needs only the sums over layers and heads
-        GP_T_ADD(16, 1); GP_T_ADD(17, t_s1 - t_s0); GP_T_ADD(18, GP_T_NOW() - t_s1); GP_T_ADD(25, nC);
       }
       continue;
     }
@@ -965,8 +942,6 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       }
     }
     __syncthreads();
-    const long long t_s3 = GP_T_NOW();
-    (void)t_s3;
     // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
     if (!uniform || !evict_fast(a, nC, loc, H, wc, s_res, flist, flist_slot, &s_i[6], ev, (unsigned)ne))
       evict_general(p, a, nC, loc, hcnt, wc, s_res, s_i, ev, (unsigned)ne);
@@ -977,11 +952,9 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       for (int j = 0; j < ne; ++j) rank += (ev[j] < mine);
       evout[rank] = mine;
     }
-    if (tid == 0) { GP_T_ADD(31, 1); GP_T_ADD(19, t_s3 - t_s1); GP_T_ADD(20, GP_T_NOW() - t_s3); GP_T_ADD(22, t_s1 - t_s0); }
   }
 
   // ---- the last CTA takes the decisions ----------------------------------------------------------------------
-  if (tid == 0) GP_T_STAMP(61);
   __syncthreads();
   if (tid == 0) {
     __threadfence();
@@ -992,12 +965,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (s_i[2]) {
     __threadfence();
-    const long long t_d0 = GP_T_NOW();
-    (void)t_d0;
-    if (tid == 0) GP_T_STAMP(62);
     decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(sbuf));
-    if (tid == 0) GP_T_STAMP(63);
-    if (tid == 0) { GP_T_ADD(23, GP_T_NOW() - t_d0); GP_T_ADD(24, 1); }
   }
 
   if (!idle_merge) merge_partials(p, n_req, out, n_mc, n_rc, (int)gridDim.x - 1 - (int)blockIdx.x, (int)gridDim.x, 0, LH);
@@ -1032,7 +1000,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   gp_pdl_launch_dependents();
   // the first round trip fetches everything at once: the header, the list of compressing requests (its first
   // CT entries before their count is known; entries past the count are never looked at) and the first ticket
-  if (tid == 0) { GP_T_STAMP(36); s_i[0] = atomicAdd(&p.hdr[HDR_WORK_CMP], 1); s_i[3] = 0; }
+  if (tid == 0) { s_i[0] = atomicAdd(&p.hdr[HDR_WORK_CMP], 1); s_i[3] = 0; }
   if (tid <= p.M) s_info[tid] = p.cmp_info[tid];
   const int n_cmp = p.hdr[HDR_N_CMP];
   const int n_items = p.hdr[HDR_N_CITEM];
@@ -1040,19 +1008,14 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   const int stamp = p.hdr[HDR_STEP];
   for (int i = tid + CT; i <= n_cmp; i += CT) s_info[i] = p.cmp_info[i];
 
-  const long long t_c0 = GP_T_NOW();
-  (void)t_c0;
   for (bool first = true;; first = false) {
     __syncthreads();
-    const long long t_c1 = GP_T_NOW();
-    (void)t_c1;
     if (!first) {
       if (tid == 0) s_i[0] = atomicAdd(&p.hdr[HDR_WORK_CMP], 1);
       __syncthreads();
     }
     const int item = s_i[0];
     if (item >= n_items) break;
-    if (tid == 0) { GP_T_ADD(48, 1); GP_T_ADD(49, GP_T_NOW() - t_c1); }
     // item -> (compressing request, layer/head, chunk); chunks of a unit are consecutive and ascending
     int lo = 0, hi = n_cmp;
     while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (LH * s_info[mid].w <= item) lo = mid; else hi = mid; }
@@ -1127,8 +1090,6 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
         dst_code[k2] = (tl << 5) | ((cp ^ (i & 7)) << 1) | isv;   // slot of the chunk, logical 16-byte piece, K or V
       }
     }
-    const long long t_c2 = GP_T_NOW();
-    (void)t_c2;
     // Touch every loaded value so that the loads have completed before the flag below is published: the
     // next chunk's CTA may overwrite the tail of this chunk's sources as soon as it sees the flag.
     unsigned touched = (unsigned)tokv;
@@ -1148,9 +1109,6 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
       }
     }
     __syncthreads();
-    const long long t_c3 = GP_T_NOW();
-    (void)t_c3;
-    if (tid == 0) { GP_T_ADD(50, t_c2 - t_c1); GP_T_ADD(51, t_c3 - t_c2); }
 #pragma unroll
     for (int k2 = 0; k2 < PIECES; ++k2) {
       if (dst_code[k2] >= 0) {
@@ -1167,7 +1125,6 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
     }
   }
   __syncthreads();
-  if (tid == 0) { GP_T_ADD(52, GP_T_NOW() - t_c0); GP_T_ADD(53, 1); GP_T_STAMP(37); GP_T_STAMP(38); }
   if (tid == 0 && s_i[3] > 0)
     atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 8), (unsigned long long)s_i[3]);
 
@@ -1219,7 +1176,6 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
       __syncwarp();
     }
   }
-  if (tid == 0) GP_T_STAMP(38);
 }
 
 }  // namespace

@@ -2,7 +2,8 @@
 //
 // HBM layout (all regions carved from the caller's blob, 256-byte aligned):
 //   kv        bf16  [L][n_pages][H_kv][2 (K|V)][b][d]   one (layer, page, KV head) tile is a
-//                   contiguous 2*b*d*2 bytes, so a single bulk copy stages K and V of a page.
+//                   contiguous 2*b*d*2 bytes: a warp stages K and V of a page with 512-byte rows of
+//                   16-byte asynchronous copies.
 //                   Inside a row of d elements the 16-byte chunks are XOR-swizzled with the
 //                   slot index: logical chunk c of slot s lives at chunk c ^ (s & 7).  A tile
 //                   copied verbatim to shared memory is then bank-conflict free for ldmatrix.
@@ -17,11 +18,8 @@
 #include <stdint.h>
 
 #define GP_PAGE 16             // tokens per page (b)
-#define GP_ATTN_WARPS 4
-#define GP_ATTN_STAGES 3
 #define GP_SPIN_LIMIT (1u << 21)
 #define GP_MAX_REQ 1024        // upper limit of max_requests (shared-memory arrays are sized by it)
-#define GP_SCORE_TILE 128      // candidate tokens per boundary-scoring tile
 #define GP_MOVE_TOK 64         // source slots per compaction chunk
 #define GP_COST_BINS 288       // cost classes of attention work items (pages, x4 at a boundary)
 #define GP_DESC_INTS 16        // ints per attention work descriptor
@@ -31,7 +29,7 @@ enum {
   HDR_N_RC = 0,      // (request, chunk) work items of this step
   HDR_N_BND,         // requests at a capacity boundary
   HDR_N_CMP,         // requests that compress
-  HDR_WORK_ATTN,     // dynamic work counter of the attention kernel
+  HDR_SPARE0,        // unused
   HDR_DONE_CMP,      // CTAs of the compaction kernel that have finished
   HDR_STEP,          // step serial number
   HDR_N_ACTIVE,      // requests actually stepped
@@ -104,7 +102,6 @@ struct GpDev {
   double* scores;
   long long* counters;                   // [16]
   int* err;
-  long long* trace;                      // development builds only (-DGP_TRACE), else null
 };
 
 __device__ __forceinline__ size_t gp_tile_off(const GpDev& p, int l, long long page, int h) {
@@ -118,18 +115,6 @@ __device__ __forceinline__ size_t gp_tok_off(const GpDev& p, int l, long long pa
 __device__ __forceinline__ size_t gp_summ_off(const GpDev& p, int l, int r, int buf, int x, int head) {
   return ((((((size_t)l * p.M + r) * 2 + buf) * 2 + x) * p.Hq) + head) * (size_t)p.d;
 }
-
-// ---- optional cycle trace (compiled in only with -DGP_TRACE, for development builds) ----------------
-#ifdef GP_TRACE
-#define GP_TRACE_WORDS 96
-#define GP_T_ADD(slot, val) atomicAdd(reinterpret_cast<unsigned long long*>(&p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + (slot)]), (unsigned long long)(val))
-#define GP_T_NOW() clock64()
-#define GP_T_STAMP(slot) do { unsigned long long gt_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt_)); p.trace[(blockIdx.x % 1024) * GP_TRACE_WORDS + (slot)] = (long long)gt_; } while (0)
-#else
-#define GP_T_ADD(slot, val) do { } while (0)
-#define GP_T_NOW() 0ll
-#define GP_T_STAMP(slot) do { } while (0)
-#endif
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -126,7 +126,7 @@ __global__ void na_merge_kernel(const float* __restrict__ scratch, int d, float*
       a += wt * base[s * NA_STRIDE + c];
       ls += wt * base[s * NA_STRIDE + NA_MAX_D + 1];
     }
-    out[(size_t)row * d + c] = a / ls;
+    out[(size_t)row * d + c] = ls > 0.f ? a / ls : 0.f;       // a request without tokens: a row of zeros
   }
 }
 

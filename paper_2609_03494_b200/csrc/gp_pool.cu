@@ -22,6 +22,10 @@ struct gp_pool {
   std::vector<uint8_t> live;      // host mirror of the slot free list
   int num_sms, attn_grid, sel_grid, compact_grid;
   int step_open, step_n_req, step_layers_done;      // per-layer entry points: a step begun and not yet ended
+  std::vector<uint8_t> step_layer_seen;             // layers gp_attn_layer has run in the open step
+  // error bits set by the kernels (GP_E_*): one int of page-locked host memory that the device addresses directly,
+  // so that the host reads it without a copy once the work that could set it has completed
+  int* h_err;
   // staging for the host-pointer entry point (inside the blob)
   int* st_ids; void* st_q; void* st_k; void* st_v; float* st_out; int* st_act;
   // small device words
@@ -36,16 +40,6 @@ struct gp_pool {
   int64_t launch_count;
 };
 
-#ifdef GP_TRACE
-static long long* g_trace_dev = nullptr;
-extern "C" int gp_trace_read(long long* out, int reset) {
-  if (!g_trace_dev || cudaDeviceSynchronize() != cudaSuccess) return -1;
-  const size_t nb = sizeof(long long) * 1024 * GP_TRACE_WORDS;
-  if (cudaMemcpy(out, g_trace_dev, nb, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
-  if (reset) cudaMemset(g_trace_dev, 0, nb);
-  return 0;
-}
-#endif
 
 namespace {
 
@@ -60,28 +54,15 @@ struct Layout {
 
 inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
-// pages per attention work item: 64 (two page ids per producer lane), and half of that for requests at their
-// capacity boundary; both can be overridden from the environment for experiments.  When an attention launch has
-// less than one such item of work per CTA (small batches, short sequences; a layer-by-layer launch, which covers
-// one layer's heads only), smaller items (32 and 8 pages) keep more CTAs busy (measured: the 36-layer shape with
-// 16 requests, layer by layer, takes 1030 us per step that way, 1252 with the large items).
+// Pages per attention work item: 64 (two page ids per producer lane), and half of that for requests at their
+// capacity boundary, whose pages also pay for the fp64 logits.  When an attention launch has less than one such
+// item of work per CTA (small batches, short sequences; a layer-by-layer launch, which covers one layer's heads
+// only), smaller items (32 and 8 pages) keep more CTAs busy (measured: the 36-layer shape with 16 requests,
+// layer by layer, takes 1030 us per step that way, 1252 with the large items).
+constexpr int GP_CHUNK = 64, GP_BCHUNK = 32;
 constexpr int GP_FINE_CHUNK = 32, GP_FINE_BCHUNK = 8;
-int chunk_pages_setting();
-int bchunk_pages_setting() {
-  const char* e = getenv("GP_BCHUNK_PAGES");
-  int v = e ? atoi(e) : chunk_pages_setting() / 2;
-  if (v < 4) v = 4;
-  if (v > 64) v = 64;
-  return v;
-}
-
-int chunk_pages_setting() {
-  const char* e = getenv("GP_CHUNK_PAGES");
-  int v = e ? atoi(e) : 64;
-  if (v < 1) v = 1;
-  if (v > 64) v = 64;
-  return v;
-}
+int chunk_pages_setting() { return GP_CHUNK; }
+int bchunk_pages_setting() { return GP_BCHUNK; }
 
 bool valid_config(const gp_config* c) {
   if (!c) return false;
@@ -355,8 +336,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     return;
   }
   if (!plan_on) return;
-  const long long t_plan0 = GP_T_NOW();
-  (void)t_plan0;
   s_first[i] = 0x7fffffff;
   if (i < GP_COST_BINS) s_bin[i] = 0;
   if (i == 0) s_nmc = 0;
@@ -404,8 +383,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     chunks = (pages + cp - 1) / cp;
     cp = (pages + chunks - 1) / chunks;              // equal sizes: chunks of cp pages, the last one shorter
   }
-  const long long t_plan1 = GP_T_NOW();
-  (void)t_plan1;
   int rc_off, n_rc; long long tok_off, tok_tot;
   plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
   // A batch whose summed lengths exceed max_batch_tokens (the caller's bound; with shared prompt pages the sum
@@ -441,8 +418,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   }
   __syncthreads();
   const int sorted0 = s_binbase[key] + within;
-  const long long t_plan2 = GP_T_NOW();
-  (void)t_plan2;
   s_chunks[i] = chunks; s_pos[i] = (int)pos;
   if (in) {
     p.b_nold[i] = n_old;
@@ -483,10 +458,8 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (threadIdx.x == 0) {
     p.hdr[HDR_N_MC] = s_nmc;
-    GP_T_ADD(26, 1); GP_T_ADD(27, t_plan1 - t_plan0); GP_T_ADD(28, t_plan2 - t_plan1); GP_T_ADD(29, GP_T_NOW() - t_plan2);
     p.hdr[HDR_N_RC] = n_rc;
     p.hdr[HDR_N_BND] = n_bnd;
-    p.hdr[HDR_WORK_ATTN] = 0;
     p.hdr[HDR_N_ACTIVE] = n_active;
   }
   // ---- from here on the kernel before this one has completed --------------------------------------------
@@ -606,6 +579,18 @@ __global__ void gp_gather_kernel(GpDev p, int r, int l, int h, int n, int* tok_o
     if ((x) != cudaSuccess) return GP_ERR_CUDA; \
   } while (0)
 
+void pool_free(gp_pool* pool) {
+  if (pool->h_err) cudaFreeHost(pool->h_err);
+  delete pool;
+}
+
+// the kernels' error bits, once the work that could set them has completed
+int kernel_status(const gp_pool* pool) {
+  return *reinterpret_cast<volatile const int*>(pool->h_err) ? GP_ERR_CUDA : GP_OK;
+}
+
+bool misaligned(const void* ptr, uintptr_t a) { return (reinterpret_cast<uintptr_t>(ptr) & (a - 1)) != 0; }
+
 int check_req(gp_pool* pool, int32_t req) {
   if (!pool) return GP_ERR_INVALID;
   if (req < 0 || req >= pool->cfg.max_requests || !pool->live[req]) return GP_ERR_INVALID;
@@ -661,11 +646,13 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   pool->profiling = 0;
   pool->early_plan = 0;
   pool->step_open = 0; pool->step_n_req = 0; pool->step_layers_done = 0;
+  pool->step_layer_seen.assign(cfg->n_layers, 0);
+  pool->h_err = nullptr;
   pool->launch_count = 0;
   memset(pool->ms, 0, sizeof(pool->ms));
   memset(pool->launches, 0, sizeof(pool->launches));
   cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
   pool->num_sms = prop.multiProcessorCount;
   pool->attn_grid = pool->num_sms * gp_attention_ctas_per_sm(cfg->head_dim);
 
@@ -691,7 +678,18 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.free_stack = reinterpret_cast<int*>(base + L.free_stack);
   int* words = reinterpret_cast<int*>(base + L.words);
   d.free_top = words + 0;
-  d.err = words + 1;
+  {
+    void* herr = nullptr; void* derr = nullptr;
+    if (cudaHostAlloc(&herr, 64, cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer(&derr, herr, 0) != cudaSuccess) {
+      if (herr) cudaFreeHost(herr);
+      pool_free(pool);
+      return GP_ERR_CUDA;
+    }
+    memset(herr, 0, 64);
+    pool->h_err = static_cast<int*>(herr);
+    d.err = static_cast<int*>(derr);
+  }
   pool->d_status = words + 2;
   d.hdr = words + 64;
   d.page_table = reinterpret_cast<int*>(base + L.page_table);
@@ -722,14 +720,6 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.partials = reinterpret_cast<float*>(base + L.partials);
   d.scores = reinterpret_cast<double*>(base + L.scores);
   d.counters = reinterpret_cast<long long*>(base + L.counters);
-  d.trace = nullptr;
-#ifdef GP_TRACE
-  if (!g_trace_dev) {
-    cudaMalloc(&g_trace_dev, sizeof(long long) * 1024 * GP_TRACE_WORDS);
-    cudaMemset(g_trace_dev, 0, sizeof(long long) * 1024 * GP_TRACE_WORDS);
-  }
-  d.trace = g_trace_dev;
-#endif
   gp_attention_setup(d);
   gp_boundary_setup(d, pool->num_sms, &pool->sel_grid, &pool->compact_grid);
   pool->dbg = base + L.dbg;
@@ -742,13 +732,13 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
     pool->st_ids = nullptr; pool->st_q = pool->st_k = pool->st_v = nullptr; pool->st_out = nullptr; pool->st_act = nullptr;
   }
   // Stale pages are read (masked) by the attention kernel, so they must hold finite numbers.
-  if (cudaMemset(dev_blob, 0, L.total) != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+  if (cudaMemset(dev_blob, 0, L.total) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
   gp_init_kernel<<<1024, 256>>>(d);
   pool->launch_count++;
   for (int i = 0; i <= GP_N_KERNELS; ++i) {
-    if (cudaEventCreate(&pool->ev[i]) != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+    if (cudaEventCreate(&pool->ev[i]) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
   }
-  if (cudaDeviceSynchronize() != cudaSuccess) { delete pool; return GP_ERR_CUDA; }
+  if (cudaDeviceSynchronize() != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
   *out = pool;
   return GP_OK;
 }
@@ -758,7 +748,7 @@ int gp_pool_destroy(gp_pool* pool) {
   cudaSetDevice(pool->device);
   cudaDeviceSynchronize();
   for (int i = 0; i <= GP_N_KERNELS; ++i) cudaEventDestroy(pool->ev[i]);
-  delete pool;
+  pool_free(pool);
   return GP_OK;
 }
 
@@ -767,6 +757,7 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   if (!pool || !out_req || n_tail < 0 || n_shared_pages < 0 || initial_pages < 0) return GP_ERR_INVALID;
   if (n_tail > 0 && (!k_tail || !v_tail)) return GP_ERR_INVALID;
   *out_req = -1;
+  if (pool->step_open) return GP_ERR_STATE;      // the open step's plan holds a snapshot of the free list
   if (n_shared_pages > 0 && check_req(pool, share_from) != GP_OK) return GP_ERR_INVALID;
   const gp_config& c = pool->cfg;
   int slot = -1;
@@ -822,6 +813,9 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
   if (pool->step_open) return GP_ERR_STATE;
   if (n_req == 0) return GP_OK;
   if (!dev_req_ids || !q || !k || !v || !out || !dev_actions) return GP_ERR_INVALID;
+  // the kernels move query, key and value rows with 16-byte copies and write `out` in 8-byte pieces
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(out, 16) ||
+      misaligned(dev_req_ids, 4) || misaligned(dev_actions, 4)) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const GpDev& d = pool->dev;
@@ -856,13 +850,14 @@ int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int3
   if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
   if (pool->step_open) return GP_ERR_STATE;
   if (n_req == 0) return GP_OK;
-  if (!dev_req_ids || !dev_actions) return GP_ERR_INVALID;
+  if (!dev_req_ids || !dev_actions || misaligned(dev_req_ids, 4) || misaligned(dev_actions, 4)) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
   launch_plan(pool, dev_req_ids, n_req, dev_actions, nullptr, 1, 0, 0, static_cast<cudaStream_t>(stream), true, true);
   pool->launch_count += 1;
   pool->step_open = 1;
   pool->step_n_req = n_req;
   pool->step_layers_done = 0;
+  pool->step_layer_seen.assign(pool->cfg.n_layers, 0);
   GP_CUDA(cudaGetLastError());
   return GP_OK;
 }
@@ -871,6 +866,9 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
                   const void* v, void* out, void* stream) {
   if (!pool || !pool->step_open || n_req != pool->step_n_req) return pool && !pool->step_open ? GP_ERR_STATE : GP_ERR_INVALID;
   if (layer < 0 || layer >= pool->cfg.n_layers || !dev_req_ids || !q || !k || !v || !out) return GP_ERR_INVALID;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(out, 16) || misaligned(dev_req_ids, 4))
+    return GP_ERR_INVALID;
+  if (pool->step_layer_seen[layer]) return GP_ERR_STATE;          // every layer once
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const GpDev& d = pool->dev;
@@ -887,6 +885,7 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
   gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
   pool->launch_count += 3;
   pool->step_layers_done += 1;
+  pool->step_layer_seen[layer] = 1;
   GP_CUDA(cudaGetLastError());
   return GP_OK;
 }
@@ -894,13 +893,22 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
 int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions, void* stream) {
   if (!pool || !pool->step_open) return pool ? GP_ERR_STATE : GP_ERR_INVALID;
   if (n_req != pool->step_n_req || !dev_req_ids || !dev_actions) return GP_ERR_INVALID;
-  if (pool->step_layers_done != pool->cfg.n_layers) return GP_ERR_STATE;       // every layer exactly once
+  if (pool->step_layers_done != pool->cfg.n_layers) return GP_ERR_STATE;       // layers missing: run them, or gp_step_abort
   GP_CUDA(cudaSetDevice(pool->device));
   gp_launch_boundary(pool->dev, dev_req_ids, n_req, dev_actions, nullptr, pool->sel_grid, pool->compact_grid,
                      static_cast<cudaStream_t>(stream), nullptr, true);
   pool->launch_count += 2;
   pool->step_open = 0;
   GP_CUDA(cudaGetLastError());
+  return GP_OK;
+}
+
+int gp_step_abort(gp_pool* pool) {
+  if (!pool) return GP_ERR_INVALID;
+  if (!pool->step_open) return GP_ERR_STATE;
+  // Nothing of an open step is committed before gp_step_end: the requests' counters are untouched, rows appended
+  // by the layers that ran lie beyond the occupied slots, and the summaries went to the buffer not in use.
+  pool->step_open = 0;
   return GP_OK;
 }
 
@@ -924,7 +932,7 @@ __global__ void gp_fetch_inputs_kernel(int* __restrict__ d_ids, const int* __res
 int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
                         const void* v, void* out, int32_t* actions, void* stream) {
   if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
-  if (!pool->st_ids) return GP_ERR_STATE;
+  if (!pool->st_ids || pool->step_open) return GP_ERR_STATE;
   if (n_req == 0) return GP_OK;
   if (!host_req_ids || !q || !k || !v || !out || !actions) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
@@ -979,12 +987,20 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
     GP_CUDA(cudaMemcpyAsync(actions, pool->st_act, (size_t)n_req * 4, cudaMemcpyDeviceToHost, s));
   }
   GP_CUDA(cudaStreamSynchronize(s));
-  return GP_OK;
+  return kernel_status(pool);
+}
+
+int gp_pool_status(gp_pool* pool, int32_t* error_bits) {
+  if (!pool) return GP_ERR_INVALID;
+  const int e = *reinterpret_cast<volatile const int*>(pool->h_err);
+  if (error_bits) *error_bits = e;
+  return e ? GP_ERR_CUDA : GP_OK;
 }
 
 int gp_release(gp_pool* pool, int32_t req, void* stream) {
   const int st = check_req(pool, req);
   if (st != GP_OK) return st;
+  if (pool->step_open) return GP_ERR_STATE;      // the open step's plan holds a snapshot of the free list
   GP_CUDA(cudaSetDevice(pool->device));
   gp_release_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(pool->dev, req);
   pool->launch_count++;
@@ -1102,9 +1118,9 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
   if (!pool) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
   GP_CUDA(cudaDeviceSynchronize());
-  int top = 0, err = 0;
+  int top = 0;
   GP_CUDA(cudaMemcpy(&top, pool->dev.free_top, 4, cudaMemcpyDeviceToHost));
-  GP_CUDA(cudaMemcpy(&err, pool->dev.err, 4, cudaMemcpyDeviceToHost));
+  const int err = *reinterpret_cast<volatile const int*>(pool->h_err);
   if (n_free) *n_free = top;
   if (refcounts) GP_CUDA(cudaMemcpy(refcounts, pool->dev.refcount, (size_t)pool->cfg.n_pages * 4, cudaMemcpyDeviceToHost));
   if (counters) {

@@ -1,0 +1,136 @@
+"""Refusals of the C ABI that protect the pool and the GPU: misaligned tensors are turned away before any
+launch, the pool cannot be changed between gp_step_begin and gp_step_end, an open step can be abandoned,
+and the kernels' error word reaches the caller."""
+import numpy as np
+import pytest
+
+from paper_2609_03494_b200 import binding as B
+from paper_2609_03494_b200 import workload as W
+
+pytestmark = pytest.mark.gpu
+
+L, HQ, HKV, D = 2, 8, 2, 64
+
+
+def _pool(**kw):
+    cfg = B.make_config(L, HQ, HKV, D, n_pages=40, max_pages_per_req=6, max_requests=8, **kw)
+    return B.Pool(cfg)
+
+
+def _bits(rng, *shape):
+    return W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+
+
+def _dev(torch, a):
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+
+
+def _invariants(pool, live):
+    n_free, ref, counters = B.gp_debug_pool(pool.handle, 40)
+    assert counters[7] == 0
+    assert int((ref > 0).sum()) + n_free == 40
+    held = 0
+    for r in live:
+        P, n, pos, table = B.gp_debug_request(pool.handle, r, 6)
+        assert len(set(table)) == P and n <= P * 16
+        held += P
+    assert int(ref.sum()) == held
+    return n_free
+
+
+def test_misaligned_tensors_are_refused_before_any_launch():
+    import torch
+    rng = np.random.default_rng(3)
+    pool = _pool()
+    try:
+        assert pool.request_add(-1, 0, _bits(rng, L, 20, HKV, D), _bits(rng, L, 20, HKV, D), 20, 0) == (B.GP_OK, 0)
+        ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+        act = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = torch.zeros((L, 1, HQ, D), dtype=torch.float32, device="cuda")
+        big = torch.zeros(L * HQ * D + 64, dtype=torch.int16, device="cuda")
+        q = big.data_ptr()
+        launches = B.gp_launch_count(pool.handle)
+        s = pool.stream()
+        for bad in (dict(q=q + 2), dict(k=q + 8), dict(v=q + 4), dict(out=out.data_ptr() + 4),
+                    dict(ids=ids.data_ptr() + 2), dict(act=act.data_ptr() + 1)):
+            a = dict(ids=ids.data_ptr(), q=q, k=q, v=q, out=out.data_ptr(), act=act.data_ptr())
+            a.update(bad)
+            with pytest.raises(B.GpError) as e:
+                B.gp_decode_step(pool.handle, a["ids"], 1, a["q"], a["k"], a["v"], a["out"], a["act"], s)
+            assert e.value.status == B.GP_ERR_INVALID, bad
+        B.gp_step_begin(pool.handle, ids.data_ptr(), 1, act.data_ptr(), s)
+        with pytest.raises(B.GpError) as e:
+            B.gp_attn_layer(pool.handle, 0, ids.data_ptr(), 1, q + 2, q, q, out.data_ptr(), s)
+        assert e.value.status == B.GP_ERR_INVALID
+        B.gp_step_abort(pool.handle)
+        assert B.gp_launch_count(pool.handle) == launches + 1           # only the plan of gp_step_begin ran
+        torch.cuda.synchronize()
+        assert B.gp_pool_status(pool.handle) == (B.GP_OK, 0)
+    finally:
+        pool.close()
+
+
+def test_pool_is_closed_to_admissions_and_releases_inside_an_open_step_and_a_step_can_be_abandoned():
+    import torch
+    rng = np.random.default_rng(5)
+    prompts = [(_bits(rng, L, n, HKV, D), _bits(rng, L, n, HKV, D), n) for n in (31, 20, 47)]
+    q, k, v = _bits(rng, L, 3, HQ, D), _bits(rng, L, 3, HKV, D), _bits(rng, L, 3, HKV, D)
+
+    def fresh():
+        p = _pool(host_staging=True, tau=-1.0)
+        for kt, vt, n in prompts:
+            assert p.request_add(-1, 0, kt, vt, n, 0)[0] == B.GP_OK
+        return p
+
+    ids = torch.arange(3, dtype=torch.int32, device="cuda")
+    qd, kd, vd = _dev(torch, q), _dev(torch, k), _dev(torch, v)
+    results = []
+    for disturb in (False, True):
+        pool = fresh()
+        try:
+            out = torch.zeros((L, 3, HQ, D), dtype=torch.float32, device="cuda")
+            act = torch.zeros(3, dtype=torch.int32, device="cuda")
+            s = pool.stream()
+            if disturb:
+                free0 = _invariants(pool, [0, 1, 2])
+                B.gp_step_begin(pool.handle, ids.data_ptr(), 3, act.data_ptr(), s)
+                B.gp_attn_layer(pool.handle, 1, ids.data_ptr(), 3, qd[1].data_ptr(), kd[1].data_ptr(), vd[1].data_ptr(),
+                                out[1].data_ptr(), s)
+                # nothing that touches the free list or the slots may pass while the step is open
+                with pytest.raises(B.GpError) as e:
+                    pool.release(1)
+                assert e.value.status == B.GP_ERR_STATE
+                assert pool.request_add(-1, 0, prompts[0][0], prompts[0][1], 31, 0)[0] == B.GP_ERR_STATE
+                with pytest.raises(B.GpError) as e:
+                    pool.decode_step(ids, qd, kd, vd, out, act)
+                assert e.value.status == B.GP_ERR_STATE
+                ph = lambda t: t.cpu().pin_memory()
+                with pytest.raises(B.GpError) as e:
+                    pool.decode_step_host(ph(ids), ph(qd), ph(kd), ph(vd), ph(out), ph(act))
+                assert e.value.status == B.GP_ERR_STATE
+                with pytest.raises(B.GpError) as e:              # the same layer twice
+                    B.gp_attn_layer(pool.handle, 1, ids.data_ptr(), 3, qd[1].data_ptr(), kd[1].data_ptr(),
+                                    vd[1].data_ptr(), out[1].data_ptr(), s)
+                assert e.value.status == B.GP_ERR_STATE
+                with pytest.raises(B.GpError) as e:              # a layer is missing
+                    B.gp_step_end(pool.handle, ids.data_ptr(), 3, act.data_ptr(), s)
+                assert e.value.status == B.GP_ERR_STATE
+                B.gp_step_abort(pool.handle)
+                with pytest.raises(B.GpError) as e:
+                    B.gp_step_abort(pool.handle)
+                assert e.value.status == B.GP_ERR_STATE
+                assert _invariants(pool, [0, 1, 2]) == free0
+                assert [B.gp_debug_request(pool.handle, r, 6)[1] for r in range(3)] == [31, 20, 47]
+                out.zero_()
+            # the abandoned step left nothing behind: the same step now gives what an undisturbed pool gives
+            pool.decode_step(ids, qd, kd, vd, out, act)
+            torch.cuda.synchronize()
+            summ = [B.gp_debug_summaries(pool.handle, r, L, HQ, D) for r in range(3)]
+            results.append((out.cpu().numpy(), act.cpu().numpy(), summ, _invariants(pool, [0, 1, 2])))
+            assert B.gp_pool_status(pool.handle) == (B.GP_OK, 0)
+        finally:
+            pool.close()
+    (o1, a1, s1, f1), (o2, a2, s2, f2) = results
+    assert np.array_equal(o1, o2) and np.array_equal(a1, a2) and f1 == f2
+    assert all(np.array_equal(x, y) for x, y in zip(s1, s2))
+    assert a1.tolist() == [B.GP_ACT_GROW, B.GP_ACT_NONE, B.GP_ACT_GROW]      # 32 and 48 tokens fill two and three pages

@@ -11,6 +11,9 @@ from tests import lockstep as LS
 pytestmark = pytest.mark.gpu
 
 
+NO_NEAR_TIES = {"ws": 0, "sel": 0, "act": 0}
+
+
 def _report(name, st):
     print(f"\n[{name}] steps {st.steps} tokens {st.tokens} attn max {st.attn_max_abs:.2e} mean {st.attn_mean_abs:.2e} "
           f"summary rel {st.summary_max_rel:.1e} decisions {st.decisions} near-ties {st.near_ties} actions {st.actions}")
@@ -21,6 +24,7 @@ def test_config1_tiny_every_step():
     _report("tiny", st)
     assert st.steps == 256 and st.tokens == 1024
     assert st.actions.get(B.GP_ACT_COMPRESS, 0) > 0
+    assert st.near_ties == NO_NEAR_TIES
 
 
 @pytest.mark.parametrize("config", [2, 3, 4, 5])
@@ -28,6 +32,7 @@ def test_configs_2_to_5_reduced(config):
     st = LS.run_lockstep(W.parity_instance(config))
     _report(f"config{config}", st)
     assert st.decisions["sel"] > 0
+    assert st.near_ties == NO_NEAR_TIES       # the standard configurations need no excuse: every decision is the oracle's
     if config == 5:
         assert st.counters[4] > 0            # copy-on-write happened
 

@@ -605,3 +605,108 @@ def test_shrink_with_shared_prompt_pages_copies_before_it_writes():
     np.testing.assert_array_equal(pool.requests[b_].K[:, :, :24], K_before)
     pool.release(a); pool.release(b_)
     assert pool.n_free() == c.n_pages
+
+
+# ----------------------------------------------------------------------------- near-tie margins and moved rows
+def test_working_set_margin_is_the_distance_of_the_running_sum_from_p_at_the_crossing():
+    # dyadic weights: every cumulative sum is exact, so the margins below are hand arithmetic
+    a = np.array([0.125, 0.5, 0.125, 0.25])                 # descending: 0.5, 0.25, 0.125, 0.125 -> sums 0.5, 0.75, 0.875, 1
+    k, m = O.p_coverage_demand_with_margin(a, 0.7)           # crossing at k = 2: above by 0.05, the sum before is 0.2 short
+    assert k == 2 and abs(m - (0.75 - 0.7) / 0.7) < 1e-15
+    k, m = O.p_coverage_demand_with_margin(a, 0.52)          # same k, but now the sum before (0.5) is the closer one
+    assert k == 2 and abs(m - (0.52 - 0.5) / 0.52) < 1e-15
+    k, m = O.p_coverage_demand_with_margin(a, 0.4)           # k = 1: the sum before is the empty sum
+    assert k == 1 and abs(m - (0.5 - 0.4) / 0.4) < 1e-15
+    k, m = O.p_coverage_demand_with_margin(a, 0.875)         # hits p exactly: a tie in the sense of the protocol
+    assert k == 3 and m == 0.0
+    k, m = O.p_coverage_demand_with_margin(a, 0.875 * (1 + 1e-7))
+    assert k == 4 and 0.9e-7 < m < 1.1e-7                    # just missed: a near-tie (< 1e-6)
+    assert O.p_coverage_demand(a, 0.7) == 2
+
+
+def test_selection_margin_is_the_smallest_relative_gap_at_any_local_or_global_cut():
+    # two blocks of four, one local pick each, two global picks
+    s = np.array([8.0, 4.0, 2.0, 1.0, 16.0, 3.0, 0.5, 0.25])
+    keep, margin = O.select_retained(s, 2, 4, 4, 1)
+    np.testing.assert_array_equal(keep, [0, 1, 4, 5])        # locals 0 and 4; of the rest {4, 2, 1, 3, .5, .25} the best two
+    # local cuts: (8 - 4) / 8 and (16 - 3) / 16; global cut between 3 (kept) and 2 (dropped)
+    assert abs(margin - (3.0 - 2.0) / 3.0) < 1e-15
+    # now the tightest cut is a local one: block 0's best two are 8 and 7.75 with a quota of one
+    s = np.array([8.0, 7.75, 2.0, 1.0, 16.0, 3.0, 0.5, 0.25])
+    keep, margin = O.select_retained(s, 2, 4, 4, 1)
+    np.testing.assert_array_equal(keep, [0, 1, 4, 5])
+    assert abs(margin - 0.25 / 8.0) < 1e-15
+    # no cut at all (everything kept): the margin is infinite; _top on its own
+    keep, gap = O._top(np.arange(4), np.array([1.0, 4.0, 2.0, 3.0]), 4)
+    assert gap == math.inf and sorted(keep.tolist()) == [0, 1, 2, 3]
+    keep, gap = O._top(np.arange(4), np.array([1.0, 4.0, 2.0, 3.0]), 2)
+    assert keep.tolist() == [1, 3] and abs(gap - (3.0 - 2.0) / 3.0) < 1e-15
+
+
+def _boundary_with_forced_working_sets(monkeypatch, k_s, k_l, margins, **cfg_over):
+    """Runs one request into its first boundary with Eq. 7's results replaced by the given ones, so that the
+    bookkeeping around them (Eq. 8, the decision, the near-tie flag) can be checked by hand."""
+    c = _cfg(n_layers=1, n_kv_heads=2, n_q_heads=4, **cfg_over)
+    pool = O.OraclePool(c)
+    n0 = 3 * c.page_size - 1                                  # three pages, one slot free
+    kt = RNG.standard_normal((1, n0, 2, c.head_dim))
+    assert pool.request_add(-1, 0, kt, kt.copy(), n0, 0) == (O.OK, 0)
+    seq = iter([(k_s[0], margins[0]), (k_l[0], margins[1]), (k_s[1], margins[2]), (k_l[1], margins[3])])
+    monkeypatch.setattr(O, "p_coverage_demand_with_margin", lambda a, p: next(seq))
+    rec = pool.step_compute([0], *_rand_step(c, 1))
+    return rec.boundary[0], c
+
+
+def test_action_near_tie_flag_says_whether_a_near_tied_working_set_could_flip_the_decision(monkeypatch):
+    # |C| = 8, two KV heads: Delta = (sum K^S - sum K^L) / (2 * 8)
+    info, c = _boundary_with_forced_working_sets(monkeypatch, (3, 4), (3, 4), (1e-9, 0.1, 0.1, 0.1))
+    assert info.delta == 0.0 and not info.want_grow           # Delta = 0 compresses
+    assert info.action_near_tie                               # one size off by one makes Delta = +1/16 > tau: it could grow
+    info, c = _boundary_with_forced_working_sets(monkeypatch, (6, 5), (3, 3), (1e-9, 0.1, 0.1, 0.1))
+    assert info.delta == 5 / 16 and info.want_grow
+    assert not info.action_near_tie                           # 4/16 and 6/16 are on the same side of tau
+    info, c = _boundary_with_forced_working_sets(monkeypatch, (3, 4), (3, 4), (1e-5, 0.1, 0.1, 0.1))
+    assert not info.action_near_tie                           # a margin of 1e-5 is not a near-tie
+    info, c = _boundary_with_forced_working_sets(monkeypatch, (4, 4), (3, 3), (1e-9, 1e-9, 0.1, 0.1), tau=0.0)
+    assert info.want_grow and info.action_near_tie            # two near-ties: 2/16 could become 0/16
+
+
+def _compress_with_keep(keep_slots, shared_pages):
+    """One request of three 16-token pages at its boundary, compressed with a prescribed keep set; when
+    shared_pages > 0 its leading prompt pages are shared with a donor.  Returns the boundary record."""
+    c = O.OracleConfig(1, 2, 1, 8, n_pages=16, max_pages_per_req=4, k_loc=0, max_requests=4)
+    pool = O.OraclePool(c)
+    kt = RNG.standard_normal((1, 47, 1, 8))
+    assert pool.request_add(-1, 0, kt, kt.copy(), 47, 0) == (O.OK, 0)
+    rid = 0
+    if shared_pages:
+        tail = 47 - 16 * shared_pages
+        kt2 = RNG.standard_normal((1, tail, 1, 8))
+        assert pool.request_add(0, shared_pages, kt2, kt2.copy(), tail, 0) == (O.OK, 1)
+        rid = 1
+    q, k, v = RNG.standard_normal((1, 1, 2, 8)), RNG.standard_normal((1, 1, 1, 8)), RNG.standard_normal((1, 1, 1, 8))
+    rec = pool.decode_step([rid], q, k, v, overrides={rid: {"keep": {(0, 0): np.asarray(keep_slots)}}})
+    info = rec.boundary[rid]
+    assert info.action == O.ACT_COMPRESS and pool.requests[rid].n == 32
+    assert pool.counters["moved_rows"] == info.moved_tokens
+    return info
+
+
+def test_moved_rows_counts_the_slots_that_change_place_and_whole_copied_pages():
+    # |C| = 32, 16 go.  Keep slots 0..7 and 16..23: 0..7 stay where they are, 16..23 move to 8..15, the 16 protected
+    # slots 32..47 move to 16..31
+    keep = list(range(0, 8)) + list(range(16, 24))
+    assert _compress_with_keep(keep, 0).moved_tokens == 8 + 16
+    # keep the whole first page: only the protected page moves (slots 32..47 -> 16..31)
+    assert _compress_with_keep(list(range(16)), 0).moved_tokens == 16
+    # keep the whole second page: it moves down one page, and so does the protected page
+    assert _compress_with_keep(list(range(16, 32)), 0).moved_tokens == 32
+    # the first page is shared with a donor: it is copied to a fresh page, so its kept slots count although
+    # their slot numbers do not change
+    info = _compress_with_keep(keep, 1)
+    assert info.cow_pages == 1 and info.moved_tokens == 8 + 8 + 16
+    info = _compress_with_keep(list(range(16)), 1)
+    assert info.cow_pages == 1 and info.moved_tokens == 16 + 16
+    # both candidate pages shared: every kept slot is written to a fresh page
+    info = _compress_with_keep(list(range(4, 20)), 2)
+    assert info.cow_pages == 2 and info.moved_tokens == 16 + 16

@@ -1,13 +1,15 @@
-"""The allocation-free attention entry point against the pool's own decode step.
+"""The allocation-free attention entry point against the pool's own decode step and against the float64 oracle.
 
 Some callers cannot give the library scratch memory or let it allocate (all device memory is committed to
 the KV pool, or the host forbids allocator calls from plug-ins); `gp_attention_noalloc` serves them from a
 fixed array inside the library.  This test feeds it the same keys and values the pool holds after a decode
 step and expects the same attention output, on two consecutive calls (the array keeps the first call's
-contents, which must not leak into the second).  It is collected last on purpose."""
+contents, which must not leak into the second), and compares it with the oracle's dense attention on
+requests of ragged lengths, one of them empty.  It is collected last on purpose."""
 import numpy as np
 import pytest
 
+from oracle import growpage_oracle as O
 from paper_2609_03494_b200 import binding as B
 from paper_2609_03494_b200 import workload as W
 
@@ -58,6 +60,32 @@ def test_noalloc_attention_matches_the_pool_on_two_calls(hq, hkv, d, prompts):
             assert float(err.max()) <= ATTN_MAX_ABS and float(err.mean()) <= ATTN_MEAN_ABS, (step, float(err.max()))
     finally:
         pool.close()
+
+
+@pytest.mark.parametrize("hq,hkv,d,lens", [(8, 2, 64, (37, 0, 300, 1)), (32, 8, 128, (513, 16, 0, 95)), (16, 2, 128, (129,))])
+def test_noalloc_attention_matches_the_oracle_and_an_empty_request_gives_zeros(hq, hkv, d, lens):
+    import torch
+    rng = np.random.default_rng(19)
+    n_req, max_len = len(lens), max(lens) + 5
+    bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    q, K, V = bits(n_req, hq, d), bits(n_req, hkv, max_len, d), bits(n_req, hkv, max_len, d)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+    qd, Kd, Vd = dev(q), dev(K), dev(V)
+    lens_d = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    f = W.bf16_bits_to_f64
+    for call in range(2):                                    # the second call finds the first one's partials in the array
+        out = torch.full((n_req, hq, d), float("nan"), dtype=torch.float32, device="cuda")
+        B.gp_attention_noalloc(qd.data_ptr(), Kd.data_ptr(), Vd.data_ptr(), lens_d.data_ptr(), n_req, hq, hkv, d,
+                               max_len, out.data_ptr(), 0)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy().astype(np.float64)
+        for r, n in enumerate(lens):
+            if n == 0:
+                assert np.array_equal(got[r], np.zeros((hq, d))), "an empty request must give a row of zeros"
+                continue
+            want = O.attention_decode(f(q[r]), f(K[r, :, :n]), f(V[r, :, :n]))
+            err = np.abs(got[r] - want)
+            assert err.max() <= ATTN_MAX_ABS and err.mean() <= ATTN_MEAN_ABS, (call, r, err.max())
 
 
 def test_noalloc_rejects_what_does_not_fit():
