@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the GrowPage decode path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload layer|stack]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--boundary async|sync]
+                    [--workload layer|stack] [--policy P] [--entry step|layers]
 
 Workload: the one-layer Qwen3-8B-shaped configuration (32 query / 8 KV heads, head_dim 128, bf16,
 page 16; 64 concurrent requests, prompts uniform in [128, 1024], 4096 decode steps each, per-request
@@ -11,7 +12,14 @@ boundary logits, working sets + selection + decision + allocator, compaction.
 
 The K timed steps are steps [S0, S0 + K) of the 4096-step job with S0 = (4096 - K) // 2, reached by
 running the S0 preceding steps untimed; K = 4096 (the default) times the whole job.  Warm-up steps
-run on the same pool, which is then re-initialised.  Prints ONE JSON line (rank 0).
+run on the same pool, which is then re-initialised.  The headline is the asynchronous boundary mode
+(the boundary chain of a step runs beside the next step and the requests it concerns sit that step
+out; tokens are counted, not request-steps); the synchronous mode is timed in the same run, with
+and without early planning, and reported beside it.  Prints ONE JSON line (rank 0).
+
+`--gpus N` with N > 1 starts N ranks itself (one per GPU, torch.distributed.run on 127.0.0.1) unless
+it already runs inside such a launch; every rank owns a pool and its own requests, nothing is
+exchanged on the data path (weak scaling).
 """
 from __future__ import annotations
 
@@ -19,6 +27,7 @@ import argparse
 import concurrent.futures as cf
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
@@ -37,6 +46,10 @@ METRIC = "decode tokens/s (attn+KV budgeting) @Qwen3-8B shape; % of HBM roofline
 JOB_STEPS = 4096
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per algorithmic byte of the attention kernel, from one ncu capture of a launch of this workload
+# (dram__bytes_read.sum + dram__bytes_write.sum over the launch's algorithmic bytes); not measured by this run
+TRAFFIC_RATIO = 1.03
+TRAFFIC_SOURCE = "profiles/attention_qwen3_8b_layer.md (ncu capture of one launch), scaled by this run's algorithmic bytes"
 
 
 def measured_peak():
@@ -46,18 +59,6 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
-
-
-def traffic_ratio():
-    """DRAM bytes per algorithmic byte of the attention kernel, from the committed ncu summary."""
-    path = os.path.join(ROOT, "profiles", "attention_qwen3_8b_layer.md")
-    try:
-        for line in open(path):
-            if line.startswith("dram_bytes_per_algorithmic_byte"):
-                return float(line.split("=")[1].split()[0])
-    except Exception:
-        pass
-    return None
 
 
 # --------------------------------------------------------------------------------------------------
@@ -138,24 +139,34 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------------------
-class Job:
-    def __init__(self, wl, torch, device, q_all, k_all, v_all, prompts, host_staging=True, policy=0):
-        from paper_2609_03494_b200 import binding as B
-        self.B, self.torch, self.wl, self.device = B, torch, wl, device
-        s = wl.shape
-        self.nreq = len(wl.requests)
-        cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
-                            max_pages_per_req=wl.max_pages_per_req, max_requests=max(4, self.nreq), k_loc=wl.k_loc,
-                            host_staging=host_staging, policy=policy)
-        self.pool = B.Pool(cfg, device)
-        # every step's inputs are resident tensors written long before the step is enqueued, and nothing else is
-        # enqueued between steps: the precondition of early planning holds
-        B.gp_set_early_plan(self.pool.handle, True)
+class Inputs:
+    """The job's inputs, once on the host (pinned) and once on the device; shared by the pools of a run."""
+
+    def __init__(self, wl, torch, device, t_end):
+        self.q_host, self.k_host, self.v_host, prompts = generate_inputs(wl, t_end, torch, pin=True)
         dev = f"cuda:{device}"
-        self.q_host, self.k_host, self.v_host = q_all, k_all, v_all
-        self.q_dev, self.k_dev, self.v_dev = q_all.to(dev), k_all.to(dev), v_all.to(dev)
+        self.q_dev, self.k_dev, self.v_dev = self.q_host.to(dev), self.k_host.to(dev), self.v_host.to(dev)
         self.prompts_dev = [(torch.from_numpy(k.view(np.int16)).to(dev), torch.from_numpy(v.view(np.int16)).to(dev))
                             for k, v in prompts]
+
+
+class Job:
+    """One pool and the requests of the workload in it.  Step t of the job feeds every request the synthetic
+    inputs of step t; a request that sits a step out (asynchronous boundary mode) skips that step's inputs,
+    which are independent draws per step."""
+
+    def __init__(self, wl, torch, device, inp: Inputs, host_staging=True, policy=0, async_boundary=False, async_slots=0):
+        from paper_2609_03494_b200 import binding as B
+        self.B, self.torch, self.wl, self.device, self.inp = B, torch, wl, device, inp
+        s = wl.shape
+        self.nreq = len(wl.requests)
+        self.M = max(4, self.nreq)
+        cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
+                            max_pages_per_req=wl.max_pages_per_req, max_requests=self.M, k_loc=wl.k_loc,
+                            host_staging=host_staging, policy=policy, async_boundary=async_boundary, async_slots=async_slots)
+        self.pool = B.Pool(cfg, device)
+        self.is_async = async_boundary
+        dev = f"cuda:{device}"
         self.ids_dev = torch.arange(self.nreq, dtype=torch.int32, device=dev)
         self.ids_host = torch.arange(self.nreq, dtype=torch.int32).pin_memory()
         self.out_dev = torch.zeros((s.n_layers, self.nreq, s.n_q_heads, s.head_dim), dtype=torch.float32, device=dev)
@@ -173,26 +184,26 @@ class Job:
             for r in range(self.nreq):
                 self.pool.release(r)
         for i, spec in enumerate(self.wl.requests):
-            kd, vd = self.prompts_dev[i]
+            kd, vd = self.inp.prompts_dev[i]
             st, rid = self.pool.request_add(-1, 0, kd, vd, spec.prompt_len, self.wl.initial_pages)
             assert st == B.GP_OK and rid == i, (st, rid)
         self.live = True
-        self.P = np.array([max(self.wl.initial_pages, sp.prompt_len // 16 + 1) for sp in self.wl.requests])
-        self.n = np.array([sp.prompt_len for sp in self.wl.requests])
         self.t = 0
 
     def step(self):
         f = self.pool.decode_step_layers if self.by_layer else self.pool.decode_step
-        f(self.ids_dev, self.q_dev[self.t], self.k_dev[self.t], self.v_dev[self.t], self.out_dev, self.act_dev)
+        i = self.inp
+        f(self.ids_dev, i.q_dev[self.t], i.k_dev[self.t], i.v_dev[self.t], self.out_dev, self.act_dev)
         self.t += 1
 
     def step_host(self):
         # gp_decode_step_host through the binding, with the host addresses of this step's inputs worked out here
         # (the tensors are contiguous [T][...]): the call a C caller makes, without a tensor view per argument
+        i = self.inp
         if self._host_ptrs is None:
-            self._host_ptrs = (self.pool.handle, self.ids_host.data_ptr(), self.q_host.data_ptr(), self.k_host.data_ptr(),
-                               self.v_host.data_ptr(), self.out_host.data_ptr(), self.act_host.data_ptr(),
-                               self.q_host[0].numel() * 2, self.k_host[0].numel() * 2, self.pool.stream())
+            self._host_ptrs = (self.pool.handle, self.ids_host.data_ptr(), i.q_host.data_ptr(), i.k_host.data_ptr(),
+                               i.v_host.data_ptr(), self.out_host.data_ptr(), self.act_host.data_ptr(),
+                               i.q_host[0].numel() * 2, i.k_host[0].numel() * 2, self.pool.stream())
         h, ids, qp, kp, vp, op, ap, qs, ks, strm = self._host_ptrs
         t = self.t
         self.B.gp_decode_step_host(h, ids, self.nreq, qp + t * qs, kp + t * ks, vp + t * ks, op, ap, strm)
@@ -202,68 +213,44 @@ class Job:
         while self.t < t_to:
             self.step()
 
-    # host mirror of (P, n) driven by the actions the step returned: algorithmic bytes come from here
-    def mirror(self, actions):
-        B = self.B
-        s = self.wl.shape
-        Wb = s.token_bytes
-        fixed = 2 * s.n_q_heads * s.head_dim + 4 * s.n_q_heads * s.head_dim        # query rows in, output rows out
-        n_new = self.n + 1
-        attn = float(s.n_layers * (n_new.sum() * Wb + self.nreq * (Wb + fixed)) + 4 * self.P.sum())
-        at_b = n_new == self.P * 16
-        score = float(s.n_layers * ((self.P[at_b] - 1) * 16).sum() * (Wb // 2))
-        self.n = n_new
-        grow = actions == B.GP_ACT_GROW
-        comp = (actions == B.GP_ACT_COMPRESS) | (actions == B.GP_ACT_COMPRESS_FALLBACK)
-        shrink = actions == B.GP_ACT_SHRINK
-        self.P = self.P + grow
-        self.n = np.where(comp, (self.P - 1) * 16, self.n)
-        self.n = np.where(shrink, (self.P - 2) * 16, self.n)
-        self.P = self.P - shrink
-        return attn, score
+    def state(self):
+        P, n = self.B.gp_debug_state(self.pool.handle, self.M)
+        return P[:self.nreq].astype(np.int64), n[:self.nreq].astype(np.int64)
 
-    def moved_rows(self):
-        return int(self.B.gp_debug_pool(self.pool.handle)[2][8])
-
-    def check_healthy(self):
+    def counters(self):
         c = self.B.gp_debug_pool(self.pool.handle)[2]
         assert c[7] == 0, f"kernel error bits {c[7]}"
         return c
 
+    def step_bytes(self, P, n_old, actions):
+        """Algorithmic bytes of the step just run, from the requests' pages and tokens before it and its actions:
+        attention (keys and values of every retained token, the appended row, query in, output out, page ids) and
+        boundary scoring (the keys of the candidate set)."""
+        B = self.B
+        s = self.wl.shape
+        Wb = s.token_bytes
+        fixed = 2 * s.n_q_heads * s.head_dim + 4 * s.n_q_heads * s.head_dim
+        stepped = np.isin(actions, (B.GP_ACT_NONE, B.GP_ACT_PENDING, B.GP_ACT_GROW, B.GP_ACT_COMPRESS,
+                                    B.GP_ACT_COMPRESS_FALLBACK, B.GP_ACT_SHRINK)) | ((actions == B.GP_ACT_STALLED) & (n_old < P * 16))
+        n_new = n_old + 1
+        attn = float(s.n_layers * ((n_new[stepped] * Wb).sum() + stepped.sum() * (Wb + fixed)) + 4 * P[stepped].sum())
+        at_b = stepped & (n_new == P * 16)
+        score = float(s.n_layers * ((P[at_b] - 1) * 16).sum() * (Wb // 2))
+        return attn, score, int(stepped.sum()), int(n_new[stepped].sum())
 
-def run_ours(args):
-    import torch
-    rank, local_rank, world = shard.init("nccl")
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
-    device = local_rank
-    torch.cuda.set_device(device)
-    K, Wm = args.steps, args.warmup
-    stack = args.workload == "stack"
-    job_steps = 96 if stack else JOB_STEPS
-    K = max(1, min(K, job_steps))
-    S0 = (job_steps - K) // 2
-    wl = W.stack8b_resident(seed=shard.shard_seed(2, rank)) if stack else W.layer8b(seed=shard.shard_seed(1, rank))
-    s = wl.shape
-    t_gen = time.time()
-    q_all, k_all, v_all, prompts = generate_inputs(wl, S0 + K, torch, pin=True)
-    t_gen = time.time() - t_gen
-    policy = {"demand": 0, "inverse": 1, "random": 2, "shrink": 3}[args.policy]
-    job = Job(wl, torch, device, q_all, k_all, v_all, prompts, policy=policy)
-    job.by_layer = args.entry == "layers"
+
+def timed_window(job, torch, device, S0, K, rank, sample_clocks=False):
+    """K steps from step S0 on, device time by CUDA events on the launching stream; returns (ms on this rank,
+    tokens decoded on this rank, kernels launched, clock record or None)."""
     B = job.B
     stream = torch.cuda.current_stream(device)
-
-    # ---- warm-up ------------------------------------------------------------------------------------
-    for _ in range(max(Wm, 3)):
-        job.step()
-    torch.cuda.synchronize(device)
     job.reset()
-
-    # ---- timed, inputs resident in HBM -----------------------------------------------------------------
     job.roll(S0)
+    torch.cuda.synchronize(device)
+    tok0 = int(job.counters()[6])
     launches0 = B.gp_launch_count(job.pool.handle)
-    sampler = ClockSampler(device)
-    if rank == 0:
+    sampler = ClockSampler(device) if (sample_clocks and rank == 0) else None
+    if sampler:
         sampler.start()
         time.sleep(0.3)
     shard.barrier(device)
@@ -272,86 +259,147 @@ def run_ours(args):
     e0.record(stream)
     for _ in range(K):
         job.step()
+    B.gp_async_join(job.pool.handle, job.pool.stream())      # the last step's boundary work belongs to the timed region
     e1.record(stream)
     torch.cuda.synchronize(device)
     shard.barrier(device)
-    ms_local = e0.elapsed_time(e1)
-    clocks = sampler.stop() if rank == 0 else None
-    gpu_launches = B.gp_launch_count(job.pool.handle) - launches0
-    counters = job.check_healthy()
-    tokens_local = K * job.nreq
-    value, ms = shard.job_throughput(tokens_local, ms_local, device)
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    launches = B.gp_launch_count(job.pool.handle) - launches0
+    tokens = int(job.counters()[6]) - tok0
+    return ms, tokens, launches, clocks
 
-    # ---- per-kernel timing pass (CUDA events around every kernel, on the launching stream) -------------------
-    job.reset()
-    job.roll(S0)
+
+def run_ours(args):
+    import torch
+    rank, local_rank, world = shard.init("nccl")
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    device = local_rank
+    torch.cuda.set_device(device)
+    K, Wm = args.steps, max(args.warmup, 3)
+    stack = args.workload == "stack"
+    job_steps = 96 if stack else JOB_STEPS
+    K = max(1, min(K, job_steps))
+    S0 = (job_steps - K) // 2
+    wl = W.stack8b_resident(seed=shard.shard_seed(2, rank)) if stack else W.layer8b(seed=shard.shard_seed(1, rank))
+    s = wl.shape
+    t_gen = time.time()
+    inp = Inputs(wl, torch, device, S0 + K)
+    t_gen = time.time() - t_gen
+    policy = {"demand": 0, "inverse": 1, "random": 2, "shrink": 3}[args.policy]
+    by_layer = args.entry == "layers"
+    head_async = args.boundary == "async" and not by_layer      # the layer-by-layer calls exist in the synchronous mode only
+    jobs = {"sync": Job(wl, torch, device, inp, policy=policy)}
+    if head_async or args.boundary == "both":
+        jobs["async"] = Job(wl, torch, device, inp, policy=policy, async_boundary=True, async_slots=args.async_slots)
+    head = jobs["async"] if head_async else jobs["sync"]
+    head.by_layer = by_layer
+    B = head.B
+
+    # ---- warm-up ------------------------------------------------------------------------------------
+    for job in jobs.values():
+        for _ in range(Wm):
+            job.step()
     torch.cuda.synchronize(device)
-    moved0 = job.moved_rows()
-    by_layer, job.by_layer = job.by_layer, False        # per-kernel times come from the whole-step entry (same kernels)
-    B.gp_set_profiling(job.pool.handle, True)
+
+    # ---- timed, inputs resident in HBM: the headline mode, then the others for comparison ----------------------
+    ms_local, tokens_local, gpu_launches, clocks = timed_window(head, torch, device, S0, K, rank, sample_clocks=True)
+    value, ms = shard.job_throughput(tokens_local, ms_local, device)
+    modes = {}
+    if not by_layer:
+        sj = jobs["sync"]
+        for name, early in (("sync", False), ("sync_early_plan", True)):
+            B.gp_set_early_plan(sj.pool.handle, early)
+            m, tk, _, _ = timed_window(sj, torch, device, S0, K, rank)
+            v, m = shard.job_throughput(tk, m, device)
+            modes[name] = {"ms_per_step": round(m / K, 5), "tokens_per_s": round(v, 1)}
+        B.gp_set_early_plan(sj.pool.handle, False)
+        if "async" in jobs:
+            if head_async:
+                modes["async"] = {"ms_per_step": round(ms / K, 5), "tokens_per_s": round(value, 1)}
+            else:
+                m, tk, _, _ = timed_window(jobs["async"], torch, device, S0, K, rank)
+                v, m = shard.job_throughput(tk, m, device)
+                modes["async"] = {"ms_per_step": round(m / K, 5), "tokens_per_s": round(v, 1)}
+
+    # ---- per-kernel timing pass (CUDA events around every kernel, on the launching streams) and the byte count -------
+    head.by_layer = False               # per-kernel times come from the whole-step entry (same kernels)
+    head.reset()
+    head.roll(S0)
+    torch.cuda.synchronize(device)
+    moved0 = int(head.counters()[8])
+    B.gp_set_profiling(head.pool.handle, True)
     attn_bytes = score_bytes = 0.0
-    n_sum = 0
+    n_tok = n_kv = 0
     for _ in range(K):
-        job.step()
-        acts = job.act_dev.cpu().numpy()
-        a, sc = job.mirror(acts)
+        P, n_old = head.state()
+        head.step()
+        acts = head.act_dev.cpu().numpy()
+        a, sc, st_n, kv_n = head.step_bytes(P, n_old, acts)
         attn_bytes += a
         score_bytes += sc
-        n_sum += int(job.n.sum())
-    kms, kn = B.gp_get_kernel_times(job.pool.handle)
-    B.gp_set_profiling(job.pool.handle, False)
-    job.by_layer = by_layer
-    moved = job.moved_rows() - moved0
+        n_tok += st_n
+        n_kv += kv_n
+    kms, kn = B.gp_get_kernel_times(head.pool.handle)
+    B.gp_set_profiling(head.pool.handle, False)
+    head.by_layer = by_layer
+    moved = int(head.counters()[8]) - moved0
     compact_bytes = 2.0 * moved * (2 * s.head_dim * 2 + 4)
-    summ_bytes = float(K) * job.nreq * s.n_layers * 2 * s.n_q_heads * s.head_dim * 8 * 2      # both views, read + write, fp64
+    summ_bytes = float(n_tok) * s.n_layers * 2 * s.n_q_heads * s.head_dim * 8 * 2      # both views, read + write, fp64
     step_bytes = attn_bytes + score_bytes + compact_bytes + summ_bytes
     peak, peak_kind = measured_peak()
     attn_ms = float(kms[1])
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
-    ratio = traffic_ratio()
+    step_gbs = step_bytes / (ms_local * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": "gp_attn_kernel<128> (append + paged GQA attention + boundary logits)",
         "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
         "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": round(achieved / NOMINAL_HBM_GBS, 4),
-        "traffic": None if ratio is None else round(ratio * attn_bytes / K),
+        "traffic": round(TRAFFIC_RATIO * attn_bytes / K), "traffic_source": TRAFFIC_SOURCE,
         "algorithmic_bytes_per_launch": round(attn_bytes / K),
         "launch_us": round(attn_ms * 1e3 / K, 2),
+        "whole_step_frac_of_nominal_8tbs": round(step_gbs / NOMINAL_HBM_GBS, 4),
         "kernel_share_of_step": {name: round(float(kms[i]) / float(kms.sum()), 4) for i, name in enumerate(B.KERNEL_NAMES)},
         "kernel_us_per_step": {name: round(float(kms[i]) * 1e3 / K, 2) for i, name in enumerate(B.KERNEL_NAMES)},
     }
-    step_gbs = step_bytes / (ms_local * 1e-3) / 1e9
     step_roofline = {
+        "what": "bytes of K/V, page ids, queries, outputs, summaries, scored keys and moved rows of the timed steps over the "
+                "timed window's device time; the north star's figure (target 0.70 of 8 TB/s)",
         "algorithmic_bytes_per_step": round(step_bytes / K),
         "attention": round(attn_bytes / K), "scoring": round(score_bytes / K), "compaction": round(compact_bytes / K),
         "summaries": round(summ_bytes / K),
         "achieved_gbs": round(step_gbs, 1), "frac_of_8tbs": round(step_gbs / NOMINAL_HBM_GBS, 4),
-        "frac_of_measured": round(step_gbs / peak, 4), "mean_tokens_per_request": round(n_sum / K / job.nreq, 1),
+        "frac_of_measured": round(step_gbs / peak, 4), "mean_tokens_per_request": round(n_kv / max(n_tok, 1), 1),
+        "tokens_per_step": round(n_tok / K, 2),
     }
 
     # ---- end to end: host buffers, copies inside the timed region -----------------------------------------------
-    job.reset()
-    job.roll(S0)
+    head.reset()
+    head.roll(S0)
     torch.cuda.synchronize(device)
+    tok0 = int(head.counters()[6])
     shard.barrier(device)
     t0 = time.perf_counter()
     for _ in range(K):
-        job.step_host()
+        head.step_host()
+    B.gp_async_join(head.pool.handle, head.pool.stream())
     torch.cuda.synchronize(device)
     e2e_ms_local = (time.perf_counter() - t0) * 1e3
     shard.barrier(device)
-    e2e_value, _ = shard.job_throughput(tokens_local, e2e_ms_local, device)
-    h2d = int(s.n_layers * job.nreq * (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim * 2 + 4 * job.nreq)
-    d2h = int(s.n_layers * job.nreq * s.n_q_heads * s.head_dim * 4 + 4 * job.nreq)
-    job.check_healthy()
+    e2e_tokens = int(head.counters()[6]) - tok0
+    e2e_value, _ = shard.job_throughput(e2e_tokens, e2e_ms_local, device)
+    h2d = int(s.n_layers * head.nreq * (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim * 2 + 4 * head.nreq)
+    d2h = int(s.n_layers * head.nreq * s.n_q_heads * s.head_dim * 4 + 4 * head.nreq)
+    counters = head.counters()
 
-    # ---- CPU baseline: the oracle as it stands, on a bounded sample -------------------------------------------------
+    # ---- CPU baseline: the oracle as it stands, on a bounded sample, one process per host core ---------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = time_oracle(wl, n_requests=8, n_steps=256, warmup=0) if not stack else time_oracle(wl, n_requests=2, n_steps=32, warmup=0)
+        cpu = time_oracle_all_cores(wl, n_steps=2048 if not stack else 32, stack=stack)
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": max(Wm, 3),
+            "metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": ("qwen3-8b-stack-resident: L=36, 32q/8kv heads, d=128, page 16, 16 requests x 96 decode "
@@ -359,10 +407,14 @@ def run_ours(args):
                                     "workload)") if stack else
                                    ("qwen3-8b-layer: L=1, 32q/8kv heads, d=128, page 16, 64 requests x 4096 decode steps, "
                                     "prompts U[128,1024], heavy-hitter fraction logU[0.5%,20%], seed 1"),
-                       "entry": "gp_decode_step" if not job.by_layer else "gp_step_begin + gp_attn_layer per layer + gp_step_end",
-                       "policy": args.policy, "early_plan": True, "requests_per_gpu": job.nreq, "timed_steps": [S0, S0 + K], "job_steps": job_steps,
+                       "entry": "gp_decode_step" if not by_layer else "gp_step_begin + gp_attn_layer per layer + gp_step_end",
+                       "boundary": ("async: the boundary chain of a step runs beside the next step, the requests it concerns sit "
+                                    "that step out; value counts decoded tokens") if head_async else "sync",
+                       "early_plan": False, "policy": args.policy, "requests_per_gpu": head.nreq,
+                       "timed_steps": [S0, S0 + K], "job_steps": job_steps,
                        "l2": "per-step working set (all resident K/V) is larger than L2; no flush needed",
                        "input_generation_s": round(t_gen, 1)},
+            "modes": modes,
             "roofline": roofline, "step_roofline": step_roofline,
             "cpu_baseline": cpu,
             "e2e": {"value": round(e2e_value, 1), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
@@ -373,18 +425,24 @@ def run_ours(args):
                        "stalled": int(counters[3]), "shrink": int(counters[10])},
         }
         print(json.dumps(line))
-    job.pool.close()
+    for job in jobs.values():
+        job.pool.close()
     shard.finish()
 
 
 # --------------------------------------------------------------------------------------------------
 # the oracle as CPU baseline / reference arm
 # --------------------------------------------------------------------------------------------------
-def time_oracle(wl, n_requests: int, n_steps: int, warmup: int, budget_s: float = 25.0):
+def _oracle_run(wl_args, req_lo, req_hi, n_steps, warmup, budget_s):
+    """Runs requests [req_lo, req_hi) of the workload through a pool of the oracle for `n_steps` decode steps;
+    returns (wall seconds of the decode steps, request-steps done, steps done)."""
     from oracle import growpage_oracle as O
     from paper_2609_03494_b200 import harness as H
+    stack, seed = wl_args
+    wl = W.stack8b_resident(seed=seed) if stack else W.layer8b(seed=seed)
     s = wl.shape
-    sub = W.Workload(wl.name, wl.seed, s, wl.requests[:n_requests], n_resident=n_requests,
+    n_requests = req_hi - req_lo
+    sub = W.Workload(wl.name, wl.seed, s, wl.requests[req_lo:req_hi], n_resident=n_requests,
                      initial_pages=wl.initial_pages, max_pages_per_req=wl.max_pages_per_req,
                      n_pages=n_requests * wl.max_pages_per_req, k_loc=wl.k_loc)
     cfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=sub.n_pages,
@@ -410,30 +468,60 @@ def time_oracle(wl, n_requests: int, n_steps: int, warmup: int, budget_s: float 
 
     for _ in range(warmup):
         one()
-    cpu0, wall, done = time.process_time(), 0.0, 0
+    wall, done = 0.0, 0
     for _ in range(n_steps):
         wall += one()
         done += 1
         if wall > budget_s:
             break
+    return wall, done * n_requests, done
+
+
+def time_oracle(wl_args, n_requests: int, n_steps: int, warmup: int, budget_s: float = 25.0):
+    """The oracle in this process (numpy; as many threads as its BLAS takes)."""
+    cpu0 = time.process_time()
+    wall, units, done = _oracle_run(wl_args, 0, n_requests, n_steps, warmup, budget_s)
     cpu_used = time.process_time() - cpu0
     cores = max(1, int(round(cpu_used / max(wall, 1e-9))))
-    return {"value": round(done * n_requests / wall, 2), "unit": "tokens/s", "cores": cores, "kind": "oracle",
+    return {"value": round(units / wall, 2), "unit": "tokens/s", "cores": cores, "kind": "oracle",
             "sample": f"first {n_requests} requests of the workload, decode steps {warmup}..{warmup + done} of the job "
                       f"(float64 numpy, {os.cpu_count()} host cores present, timed region excludes input decoding)",
             "steps": done, "wall_s": round(wall, 4)}
+
+
+def time_oracle_all_cores(wl, n_steps: int, stack: bool):
+    """One process per host core, each with its own oracle pool and its share of the requests (requests are
+    independent while neither the pool nor the cap binds, as here); throughput = all request-steps over the
+    slowest process's decode time."""
+    n_proc = max(1, min(os.cpu_count() or 1, len(wl.requests)))
+    per = len(wl.requests) // n_proc
+    parts = [(i * per, (i + 1) * per) for i in range(n_proc)]
+    os.environ.setdefault("OMP_NUM_THREADS", "1")
+    t0 = time.perf_counter()
+    with cf.ProcessPoolExecutor(max_workers=n_proc) as ex:
+        futs = [ex.submit(_oracle_run, (stack, wl.seed), lo, hi, n_steps, 0, 20.0) for lo, hi in parts]
+        res = [f.result() for f in futs]
+    wall_all = time.perf_counter() - t0
+    slowest = max(r[0] for r in res)
+    units = sum(r[1] for r in res)
+    steps = min(r[2] for r in res)
+    return {"value": round(units / slowest, 2), "unit": "tokens/s", "cores": n_proc, "kind": "oracle",
+            "sample": f"{n_proc} processes x {per} requests of the workload ({n_proc * per} of {len(wl.requests)}), decode steps "
+                      f"0..{steps} of the job, not the timed window (float64 numpy, one thread per process; the figure "
+                      f"divides by the slowest process's decode time; input decoding excluded)",
+            "steps": steps, "wall_s": round(slowest, 4), "wall_with_setup_s": round(wall_all, 2)}
 
 
 def run_reference(args):
     rank, _, world = shard.env_world()
     if rank != 0:
         return
-    wl = W.layer8b(seed=1)
     K, Wm = max(1, args.steps), max(0, args.warmup)
     n_req = 4
-    res = time_oracle(wl, n_requests=n_req, n_steps=K, warmup=Wm, budget_s=150.0)
+    res = time_oracle((False, 1), n_requests=n_req, n_steps=K, warmup=Wm, budget_s=150.0)
     line = {
-        "impl": "reference", "metric": METRIC, "value": res["value"], "unit": "tokens/s", "n_gpus": world,
+        "impl": "reference", "metric": METRIC, "value": res["value"], "unit": "tokens/s",
+        "n_gpus": world if world > 1 else max(1, args.gpus),
         "steps": res["steps"], "warmup": Wm, "ms_per_step": round(1e3 * res["wall_s"] / res["steps"], 4),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "qwen3-8b-layer (bounded sample: each step decodes the first 4 of the 64 requests once, "
@@ -446,6 +534,18 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def spawn_ranks(n: int) -> int:
+    """`--gpus N` outside a torchrun launch: start N ranks of this command, one per GPU, on this node."""
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    return subprocess.call(cmd, env=env)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -453,6 +553,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--boundary", default="async", choices=["async", "sync", "both"],
+                    help="async (headline): boundary work beside the next step; sync: inside the step; both: headline sync, "
+                         "async timed beside it")
+    ap.add_argument("--async-slots", type=int, default=0, help="thread blocks the attention kernel leaves to the boundary kernels")
     ap.add_argument("--entry", default="step", choices=["step", "layers"],
                     help="step: gp_decode_step; layers: the same step through gp_step_begin / gp_attn_layer / gp_step_end")
     ap.add_argument("--workload", default="layer", choices=["layer", "stack"],
@@ -462,6 +566,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "RANK" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
     else:
         run_ours(args)
 

@@ -43,6 +43,12 @@ extern "C" {
 #define GP_ACT_COMPRESS_FALLBACK  3   /* wanted to grow, cap or free list said no, compressed     */
 #define GP_ACT_SHRINK             4   /* GP_POLICY_SHRINK: two pages worth of slots freed in place,
                                          the last page returned to the pool (Eq. 13)              */
+#define GP_ACT_PENDING            5   /* asynchronous boundary work only: the request reached its capacity boundary
+                                         with this step; its demand estimate, decision and compaction run beside the
+                                         next step (gp_boundary_outcome tells the decision afterwards)             */
+#define GP_ACT_HELD               6   /* asynchronous boundary work only: the request reached its boundary at the step
+                                         before and sits this step out (not stepped, nothing of it read or written by
+                                         the step; `out` row not written); it decodes again from the next step on   */
 #define GP_ACT_STALLED          (-1)  /* full and neither a page nor copy-on-write targets could
                                          be had: page state untouched, the caller should release
                                          (preempt) the request; it is skipped while it stays full */
@@ -88,6 +94,11 @@ typedef struct gp_config {
   int32_t host_staging;      /* 1: reserve staging so that gp_decode_step_host can be used         */
   int32_t policy;            /* GP_POLICY_*: how Delta_t becomes an action (default: demand)       */
   int32_t policy_seed;       /* GP_POLICY_RANDOM: seed of its counter-based draws                  */
+  int32_t async_boundary;    /* 1: asynchronous boundary work (App. "Asynchronous Decoding and Compression"),
+                                see gp_decode_step; default 0                                       */
+  int32_t async_slots;       /* asynchronous boundary work: thread blocks of the attention kernel's grid
+                                given up so that the boundary kernels find room on the SMs beside it;
+                                0 = a default (48)                                                    */
   int64_t n_pages;           /* physical pages; one page id covers all layers and KV heads         */
   int64_t min_capacity;      /* GP_POLICY_SHRINK: tokens of capacity a Shrink must leave, default 1024 */
   int64_t max_batch_tokens;  /* bound on the summed sequence lengths of one decode batch, used to
@@ -95,6 +106,15 @@ typedef struct gp_config {
                                 no prompt pages are shared (a shared page counts once in the pool
                                 and once per request in a batch).  A batch above the bound is not
                                 an error: requests that do not fit report GP_ACT_SCRATCH          */
+  int64_t max_boundary_tokens; /* bound on the summed candidate tokens of the requests that reach their
+                                boundary in one step; sizes the boundary scratch (summary logits,
+                                per-page softmax partials, large-set scores), 50 to 60 bytes per token,
+                                layer and KV head.  0 = max_batch_tokens: every request of a batch may be
+                                at its boundary (equal prompts reach it together).  On average one
+                                request in sixteen is, so a large pool can set an eighth of that, at
+                                least one request at the page cap.  More boundary tokens in a step are
+                                not an error: the requests that do not fit report GP_ACT_SCRATCH, are
+                                not stepped, and reach their boundary in a later step               */
   double  beta_s, beta_l;    /* Eq. 6, defaults 0.9 and 0.999                                      */
   double  top_p;             /* Eq. 7, default 0.99                                                */
   double  tau;               /* decision threshold, default 0                                      */
@@ -149,10 +169,35 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
  * steps can be captured into a CUDA graph and replayed.  The step's kernels are chained with
  * programmatic dependent launch.  Steps of one pool must be issued on one stream (or otherwise
  * serialised): they share scratch inside the blob.  See gp_set_early_plan for an option that lets
- * the step's first kernel start its work beside the last kernel of the step before. */
+ * the step's first kernel start its work beside the last kernel of the step before.
+ *
+ * Asynchronous boundary work (gp_config.async_boundary = 1; App. "Asynchronous Decoding and Compression":
+ * requests that compress leave the decode batch, the others keep decoding, the compressed ones rejoin a later
+ * batch).  Here the whole boundary chain of a step (demand estimate, decision, page grant or eviction and
+ * compaction) leaves the step's critical path: it runs on a stream the pool owns, beside the next step, on
+ * SM room the attention kernel leaves free (async_slots).  A request that reaches its boundary at step t
+ * reports GP_ACT_PENDING at step t, is skipped at step t + 1 (GP_ACT_HELD if the batch names it: the caller
+ * keeps that token's inputs for step t + 2), and decodes again from step t + 2 on, by which time its pages
+ * are in their new state; a request whose boundary ended without pages reports GP_ACT_STALLED then.  "Step"
+ * counts the pool's decode steps, whatever their batches.  Every token still sees exactly the state the
+ * synchronous mode gives it; only the step at which it is decoded moves.  `dev_actions` carries what is
+ * known when the step's own work ends (NONE, PENDING, HELD, STALLED, SCRATCH, INVALID); the decisions are
+ * read with gp_boundary_outcome.  gp_request_add, gp_release and the introspection calls wait for
+ * outstanding boundary work themselves; a caller that touches the pool's pages in any other way, or ends
+ * a stream capture, calls gp_async_join first.  The layer-by-layer calls and CUDA-graph capture are not
+ * available in this mode (GP_ERR_STATE from gp_step_begin). */
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
                    const void* q, const void* k, const void* v,
                    void* out, int32_t* dev_actions, void* stream);
+
+/* Asynchronous boundary work: makes `stream` wait for the boundary work of the steps issued so far. */
+int gp_async_join(gp_pool* pool, void* stream);
+
+/* The decision taken at the request's most recent capacity boundary (GP_ACT_GROW, GP_ACT_COMPRESS,
+ * GP_ACT_COMPRESS_FALLBACK, GP_ACT_SHRINK, GP_ACT_STALLED; GP_ACT_NONE if it has not reached one) and the
+ * number of that decode step, counted from 0 over the pool's decode steps (host outputs, either may be NULL).
+ * Synchronises the device.  In the synchronous mode it repeats what dev_actions said. */
+int gp_boundary_outcome(gp_pool* pool, int32_t req, int32_t* action, int64_t* step);
 
 /* The same step, layer by layer, for a model's forward pass, where layer l + 1's query exists only after
  * layer l's attention output (the paper's setting: attention and the summary update run inside every
@@ -213,6 +258,10 @@ const char* gp_strerror(int status);
 /* Pages P, occupied slots n, absolute position pos and the page table (host int32, room for
  * max_pages_per_req entries; may be NULL) of a live request. */
 int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t* pos, int32_t* page_table);
+
+/* Pages and occupied slots of every request slot at once: host int32 [max_requests] each (either may be
+ * NULL); slots that are not live read 0. */
+int gp_debug_state(gp_pool* pool, int32_t* P, int32_t* n);
 
 /* Original token index of every occupied slot of one (layer, KV head) stream, in slot order:
  * host int32 [n].  This is the retained-index set of Sec. 3.3. */

@@ -31,6 +31,13 @@ design notes; the ones with no independent check are marked "parity unpinned":
   * simultaneous boundaries: grants, then copy-on-write targets, each in ascending
     request id; references to replaced pages are dropped after all compactions
   * every shared page below the last one is replaced at a compression
+  * asynchronous decoding and compression (App. "Asynchronous Decoding and Compression"): the appendix lets
+    requests that compress leave the batch while the others decode, and rejoin a later batch; requests that grow
+    resume once the page is installed.  Reading taken when `async_boundary` is set: the whole boundary chain of a
+    request (demand estimate, decision, grant or compaction) runs beside the pool's next decode step, so every
+    request that reaches its boundary at step t, whatever the decision turns out to be, sits step t + 1 out
+    (ACT_HELD) and decodes again from step t + 2; the step reports ACT_PENDING for it and the decision is read
+    afterwards.  Each token meets exactly the state it meets in the synchronous order
   * Shrink (Eq. 13, App. "capacity-control policies"): evicts 2b tokens of C by the same Eq. 10 rule with the
     target |C| - 2b, hands the request's last page back once compaction is over, and is replaced by
     Compress & Hold when the capacity left, (P - 1) b tokens, would be under the minimum capacity
@@ -55,6 +62,8 @@ ACT_GROW = 1
 ACT_COMPRESS = 2
 ACT_COMPRESS_FALLBACK = 3
 ACT_SHRINK = 4
+ACT_PENDING = 5        # asynchronous boundary work: boundary reached, decision under way
+ACT_HELD = 6           # asynchronous boundary work: sitting out the step after its boundary
 ACT_STALLED = -1
 ACT_INVALID = -3
 
@@ -267,10 +276,11 @@ class OracleConfig:
     p_compress: float = 0.7
     shrink_below: float = -0.005     # Eq. 13: Shrink when Delta_t is under this
     min_capacity: int = 1024         # tokens; a Shrink that would leave less is a Compress & Hold
+    async_boundary: bool = False     # boundary work of step t beside step t + 1; the request sits that step out
 
 
 class _Request:
-    __slots__ = ("P", "n", "pos", "started", "n_pristine", "table", "K", "V", "tok", "S", "Lg")
+    __slots__ = ("P", "n", "pos", "started", "n_pristine", "table", "K", "V", "tok", "S", "Lg", "bstep", "last_act")
 
 
 @dataclasses.dataclass
@@ -312,6 +322,7 @@ class OraclePool:
         self.refcount = np.zeros(cfg.n_pages, dtype=np.int64)
         self.free: List[int] = list(range(cfg.n_pages - 1, -1, -1))   # pop() hands out page 0 first
         self.requests: Dict[int, _Request] = {}
+        self.serial = 0                                   # decode steps so far
         self.counters = {"grow": 0, "compress": 0, "fallback": 0, "shrink": 0, "stalled": 0, "cow_pages": 0,
                          "moved_rows": 0, "scored_tokens": 0}
 
@@ -371,6 +382,7 @@ class OraclePool:
         while len(r.table) < P:
             r.table.append(self._take_page())
         r.P, r.n, r.pos, r.started = P, n_prompt, n_prompt, False
+        r.bstep, r.last_act = None, ACT_NONE
         r.n_pristine = n_prompt // b                     # only full prompt pages can be shared
         r.S = np.zeros((c.n_layers, c.n_q_heads, c.head_dim))
         r.Lg = np.zeros((c.n_layers, c.n_q_heads, c.head_dim))
@@ -408,6 +420,9 @@ class OraclePool:
                 actions[i] = ACT_INVALID
                 continue
             seen.add(rid)
+            if c.async_boundary and r.bstep == self.serial - 1:
+                actions[i] = ACT_HELD                # its boundary work runs beside this step: not stepped
+                continue
             if r.n >= r.P * b:                       # stalled earlier and never resolved
                 actions[i] = ACT_STALLED
                 continue
@@ -428,6 +443,10 @@ class OraclePool:
             # 4. capacity boundary: the allocation is exhausted (Sec. 3.3)
             if r.n == r.P * b:
                 boundary[int(rid)] = self._demand(int(rid), r, q[:, i], t)
+                r.bstep = self.serial
+                if c.async_boundary:
+                    actions[i] = ACT_PENDING
+        self.serial += 1
         return StepRecord([int(x) for x in req_ids], out, actions, boundary)
 
     def _demand(self, rid: int, r: _Request, q: np.ndarray, t: int) -> BoundaryInfo:
@@ -536,7 +555,9 @@ class OraclePool:
         for page in released:
             self._drop_ref(page)
         for rid in order:
-            rec.actions[index_of[rid]] = rec.boundary[rid].action
+            self.requests[rid].last_act = rec.boundary[rid].action
+            if not c.async_boundary:                    # the asynchronous step has reported ACT_PENDING already
+                rec.actions[index_of[rid]] = rec.boundary[rid].action
 
     def _compress(self, r: _Request, info: BoundaryInfo, keep_override: dict, cow: set, n_evict: int) -> None:
         """Eq. 9, Eq. 10 and the compaction, independently for every (layer, KV head).  `n_evict` tokens of C
@@ -587,3 +608,8 @@ class OraclePool:
 
     def n_free(self) -> int:
         return len(self.free)
+
+    def boundary_outcome(self, rid: int) -> Tuple[int, int]:
+        """(decision, step number) of the request's most recent boundary; (ACT_NONE, -1) before the first."""
+        r = self.requests[rid]
+        return (ACT_NONE, -1) if r.bstep is None else (r.last_act, r.bstep)

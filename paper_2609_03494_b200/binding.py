@@ -17,6 +17,7 @@ GP_OK, GP_ERR_INVALID, GP_ERR_NO_SLOT, GP_ERR_NO_PAGES, GP_ERR_CUDA, GP_ERR_STAT
 GP_ERR_TOO_LARGE = -6
 GP_NOALLOC_MAX_ROWS = 2048
 GP_ACT_NONE, GP_ACT_GROW, GP_ACT_COMPRESS, GP_ACT_COMPRESS_FALLBACK, GP_ACT_SHRINK = 0, 1, 2, 3, 4
+GP_ACT_PENDING, GP_ACT_HELD = 5, 6
 GP_ACT_STALLED, GP_ACT_SCRATCH, GP_ACT_INVALID = -1, -2, -3
 GP_POLICY_DEMAND, GP_POLICY_INVERSE, GP_POLICY_RANDOM, GP_POLICY_SHRINK = 0, 1, 2, 3
 GP_N_KERNELS = 4
@@ -28,8 +29,9 @@ class gp_config(C.Structure):
         ("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
         ("page_size", C.c_int32), ("max_requests", C.c_int32), ("max_pages_per_req", C.c_int32),
         ("recent_window", C.c_int32), ("k_loc", C.c_int32), ("host_staging", C.c_int32),
-        ("policy", C.c_int32), ("policy_seed", C.c_int32),
+        ("policy", C.c_int32), ("policy_seed", C.c_int32), ("async_boundary", C.c_int32), ("async_slots", C.c_int32),
         ("n_pages", C.c_int64), ("min_capacity", C.c_int64), ("max_batch_tokens", C.c_int64),
+        ("max_boundary_tokens", C.c_int64),
         ("beta_s", C.c_double), ("beta_l", C.c_double), ("top_p", C.c_double), ("tau", C.c_double),
         ("rope_theta", C.c_double), ("p_compress", C.c_double), ("shrink_below", C.c_double),
     ]
@@ -58,6 +60,7 @@ def lib() -> C.CDLL:
     L.gp_release.argtypes = [vp, i32, vp]
     L.gp_strerror.argtypes = [C.c_int]; L.gp_strerror.restype = C.c_char_p
     L.gp_debug_request.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i64), vp]
+    L.gp_debug_state.argtypes = [vp, vp, vp]
     L.gp_debug_retained.argtypes = [vp, i32, i32, i32, vp]
     L.gp_debug_kv.argtypes = [vp, i32, i32, i32, vp, vp]
     L.gp_debug_summaries.argtypes = [vp, i32, vp]
@@ -68,6 +71,8 @@ def lib() -> C.CDLL:
     L.gp_step_end.argtypes = [vp, vp, i32, vp, vp]
     L.gp_step_abort.argtypes = [vp]
     L.gp_pool_status.argtypes = [vp, C.POINTER(i32)]
+    L.gp_async_join.argtypes = [vp, vp]
+    L.gp_boundary_outcome.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i64)]
     L.gp_set_profiling.argtypes = [vp, i32]
     L.gp_set_early_plan.argtypes = [vp, i32]
     L.gp_get_kernel_times.argtypes = [vp, vp, vp]
@@ -162,6 +167,17 @@ def gp_pool_status(pool: int) -> Tuple[int, int]:
     return int(st), int(bits.value)
 
 
+def gp_async_join(pool: int, stream: int) -> None:
+    _check(lib().gp_async_join(C.c_void_p(pool), C.c_void_p(stream)), "gp_async_join")
+
+
+def gp_boundary_outcome(pool: int, req: int) -> Tuple[int, int]:
+    """(action, step) of the request's most recent capacity boundary."""
+    act, step = C.c_int32(0), C.c_int64(-1)
+    _check(lib().gp_boundary_outcome(C.c_void_p(pool), req, C.byref(act), C.byref(step)), "gp_boundary_outcome")
+    return int(act.value), int(step.value)
+
+
 def gp_release(pool: int, req: int, stream: int) -> None:
     _check(lib().gp_release(C.c_void_p(pool), req, C.c_void_p(stream)), "gp_release")
 
@@ -176,6 +192,14 @@ def gp_debug_request(pool: int, req: int, cap: int):
     _check(lib().gp_debug_request(C.c_void_p(pool), req, C.byref(P), C.byref(n), C.byref(pos),
                                   table.ctypes.data_as(C.c_void_p)), "gp_debug_request")
     return int(P.value), int(n.value), int(pos.value), table[:P.value].tolist()
+
+
+def gp_debug_state(pool: int, max_requests: int) -> Tuple[np.ndarray, np.ndarray]:
+    P = np.zeros(max_requests, dtype=np.int32)
+    n = np.zeros(max_requests, dtype=np.int32)
+    _check(lib().gp_debug_state(C.c_void_p(pool), P.ctypes.data_as(C.c_void_p), n.ctypes.data_as(C.c_void_p)),
+           "gp_debug_state")
+    return P, n
 
 
 def gp_debug_retained(pool: int, req: int, layer: int, kv_head: int, n: int) -> np.ndarray:
@@ -323,7 +347,8 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
                 max_requests: int = 512, k_loc: int = 4, host_staging: bool = False, max_batch_tokens: int = 0,
                 beta_s: float = 0.9, beta_l: float = 0.999, top_p: float = 0.99, tau: float = 0.0,
                 rope_theta: float = 0.0, policy: int = 0, policy_seed: int = 0, p_compress: float = 0.7,
-                shrink_below: float = -0.005, min_capacity: int = 1024) -> gp_config:
+                shrink_below: float = -0.005, min_capacity: int = 1024, async_boundary: bool = False,
+                async_slots: int = 0, max_boundary_tokens: int = 0) -> gp_config:
     cfg = gp_config_default()
     cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
     cfg.n_pages, cfg.max_pages_per_req, cfg.max_requests = n_pages, max_pages_per_req, max_requests
@@ -331,4 +356,5 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
     cfg.beta_s, cfg.beta_l, cfg.top_p, cfg.tau, cfg.rope_theta = beta_s, beta_l, top_p, tau, rope_theta
     cfg.policy, cfg.policy_seed, cfg.p_compress = policy, policy_seed, p_compress
     cfg.shrink_below, cfg.min_capacity = shrink_below, min_capacity
+    cfg.async_boundary, cfg.async_slots, cfg.max_boundary_tokens = 1 if async_boundary else 0, async_slots, max_boundary_tokens
     return cfg

@@ -32,7 +32,7 @@ constexpr int NBINS = 2048;
 constexpr int NBINS_PAD = NBINS + NBINS / 8;     // bins are stored at b + (b >> 3): a thread's 8 consecutive bins and
 #define HIDX(b) ((b) + ((b) >> 3))              // its neighbours' then fall into different banks
 constexpr double TWO62 = 4611686018427387904.0;
-constexpr int SEL_T = 512;           // threads of the selection kernel
+constexpr int SEL_T = 256;           // threads of the selection kernel
 constexpr int SEL_NW = SEL_T / 32;
 constexpr int SEL_CAP = 6144;        // candidate tokens whose scores are staged in shared memory
 constexpr int CT = 256;              // threads of the compaction kernel
@@ -418,7 +418,12 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
 // ------------------------------------------------------------------------------------------------------
 // decision + allocator, run by the last CTA of the selection kernel
 // ------------------------------------------------------------------------------------------------------
-__device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr) {
+__device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr,
+                                    int serial) {
+  // In the asynchronous boundary mode this runs beside the next decode step: it touches only the requests at
+  // this step's boundary (which sit that step out), reads the free list itself (the boundary chains run one
+  // after the other and nothing else takes or returns pages meanwhile) and reports through last_act only
+  // (`actions` is null: the caller's array belongs to a step that has ended).
   int* s_want = s_arr;
   int* s_ksh = s_arr + GP_MAX_REQ;
   int* s_P = s_arr + 2 * GP_MAX_REQ;
@@ -436,18 +441,19 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
 #pragma unroll
   for (int k = 0; k < RPT; ++k) {
     const int i = tid + k * SEL_T;
-    fl[k] = i < n_req ? p.b_flags[i] : 0;
-    rq[k] = i < n_req ? req_ids[i] : 0;
-    no[k] = i < n_req ? p.b_nold[i] : 0;
+    const bool on = !p.async && i < n_req;
+    fl[k] = on ? p.b_flags[i] : 0;
+    rq[k] = on ? req_ids[i] : 0;
+    no[k] = on ? p.b_nold[i] : 0;
   }
   const int n_active = p.hdr[HDR_N_ACTIVE];
   int top0 = 0;
   if (n_bnd > 0) {
-    top0 = __ldcg(p.free_peek);
+    top0 = p.async ? __ldcg(p.free_top) : __ldcg(p.free_peek);
     for (int e = tid; e < n_bnd; e += blockDim.x) {
       const int4 inf = p.bnd_info[2 * e];
       const int4 acc = __ldcg(reinterpret_cast<const int4*>(p.bnd_acc) + e);
-      s_free[e] = __ldcg(p.free_peek + 1 + e);
+      s_free[e] = p.async ? (e < top0 ? __ldcg(p.free_stack + top0 - 1 - e) : 0) : __ldcg(p.free_peek + 1 + e);
       const int r = inf.y, Pr = inf.z;
       const int nC = (Pr - 1) * GP_PAGE;
       // Eq. 8 with a common |C|: Delta = (sum K^S - sum K^L) / (N |C|), one division of exact integers
@@ -485,8 +491,10 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     }
   }
   if (tid == 0) {
-    atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 5), 1ull);
-    atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 6), (unsigned long long)n_active);
+    if (!p.async) {
+      atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 5), 1ull);
+      atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 6), (unsigned long long)n_active);
+    }
     p.hdr[HDR_WORK_CMP] = 0;
     if (n_bnd == 0) { p.hdr[HDR_N_CMP] = 0; p.hdr[HDR_N_CITEM] = 0; p.hdr[HDR_N_COW] = 0; }
   }
@@ -498,6 +506,10 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     s_order[rank] = e;
   }
   __syncthreads();
+  auto report = [&](int bi, int r, int act) {
+    if (actions) actions[bi] = act;
+    p.last_act[r] = act;
+  };
   if (tid == 0) {                                        // sequential allocator: shared memory only
     int top = top0;
     int n_cmp = 0, chunks = 0;
@@ -512,11 +524,11 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
         p.refcount[page] = 1;
         p.page_table[(size_t)r * p.cap + Pr] = page;
         p.P[r] = Pr + 1;
-        actions[bi] = GP_ACT_GROW;
+        report(bi, r, GP_ACT_GROW);
         s_want[e] |= 2;
         ++grow;
       } else if (Pr == 1) {
-        actions[bi] = GP_ACT_STALLED;
+        report(bi, r, GP_ACT_STALLED);
         s_want[e] |= 4;
         ++stall;
       }
@@ -526,7 +538,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       if (s_want[e] & 6) continue;
       const int r = s_req[e], bi = s_bi[e];
       if (s_ksh[e] > top) {
-        actions[bi] = GP_ACT_STALLED;
+        report(bi, r, GP_ACT_STALLED);
         ++stall;
         continue;
       }
@@ -537,9 +549,9 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       p.cmp_info[n_cmp] = make_int4(r, s_P[e], e | (shrink ? CMP_SHRINK : 0), chunks);
       chunks += (s_P[e] * GP_PAGE + MOVE_TOK - 1) / MOVE_TOK;
       ++n_cmp;
-      if (s_want[e] & 1) { actions[bi] = GP_ACT_COMPRESS_FALLBACK; ++fall; }
-      else if (shrink) { actions[bi] = GP_ACT_SHRINK; ++shr; }
-      else { actions[bi] = GP_ACT_COMPRESS; ++comp; }
+      if (s_want[e] & 1) { report(bi, r, GP_ACT_COMPRESS_FALLBACK); ++fall; }
+      else if (shrink) { report(bi, r, GP_ACT_SHRINK); ++shr; }
+      else { report(bi, r, GP_ACT_COMPRESS); ++comp; }
       // a compression frees one page worth of slots; a Shrink frees two and gives the last page back (the
       // compaction kernel returns it once nothing reads it any more)
       p.n[r] = (s_P[e] - (shrink ? 2 : 1)) * GP_PAGE;
@@ -806,32 +818,110 @@ struct SelGeom {
   static constexpr size_t MISC_BYTES = SEL_NW * 8 + SEL_NW * 4 + 8 * 8 + 32 * 4 + 16 * 4 + (SEL_NW * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
 };
 
+// shared memory of the selection kernel
+struct SelSmem {
+  double* sbuf;                      // [SEL_CAP] a^S, a^L or s
+  unsigned* hcnt;                    // histogram planes; the softmax factors F share them before the bins are used
+  unsigned long long* hsum;
+  unsigned long long* wsum;          // [SEL_NW]
+  unsigned* wc;                      // [SEL_NW]
+  long long* s_res;                  // [8]
+  int* ev;                           // [32]
+  int* s_i;                          // [16]
+  double* red;                       // [SEL_NW][16]
+  double* sM;                        // [16]
+  double* sZ;                        // [16]
+  double* flist;                     // [32] members of the crossing bin
+  int* flist_slot;                   // [32]
+  unsigned* loc;                     // [cap*b/32 + 1] block-local picks, one bit per candidate
+  FastHist H;
+};
+constexpr int SEL_F_CAP = (int)(SelGeom::H_BYTES / sizeof(double));
+
+// One selection job of a boundary unit: per-head softmax over the candidate set and the group mean from the
+// attention kernel's per-page partials (`z`, `zs`), then either the working-set size of one view (task 0: K^S,
+// 1: K^L; Eq. 7) or the `ne` slots a compression would evict (task 2; Eq. 9, Eq. 10).  The outputs go to Kout / acc
+// (the request's running sum for Eq. 8) and evout.
+__device__ __forceinline__ void sel_job(const GpDev& p, const SelSmem& S, const double* z, size_t view_stride, const double* zs,
+                                     double* a, int nC, int task, int ne, int* Kout, int* acc, int* evout) {
+  const int tid = threadIdx.x;
+  if (task == 2) for (int i = tid; i < (nC + 31) / 32; i += SEL_T) S.loc[i] = 0;
+  if (tid == 0) { S.s_res[0] = -1; S.s_i[0] = 0; S.s_i[5] = 0; S.s_i[6] = 0; S.s_i[7] = 0; }
+  bool uniform;
+  double* F = reinterpret_cast<double*>(S.hcnt);
+  switch (p.G) {
+    case 1: uniform = job_softmax<1>(p, z, view_stride, zs, a, nC, task, S.red, S.sM, S.sZ, F, SEL_F_CAP); break;
+    case 2: uniform = job_softmax<2>(p, z, view_stride, zs, a, nC, task, S.red, S.sM, S.sZ, F, SEL_F_CAP); break;
+    case 4: uniform = job_softmax<4>(p, z, view_stride, zs, a, nC, task, S.red, S.sM, S.sZ, F, SEL_F_CAP); break;
+    default: uniform = job_softmax<8>(p, z, view_stride, zs, a, nC, task, S.red, S.sM, S.sZ, F, SEL_F_CAP); break;
+  }
+  fast_hist_zero(S.H, task < 2);                   // the factors' table shared this memory
+  if (task < 2) {
+    __syncthreads();
+    // ---- Eq. 7 -------------------------------------------------------------------------------------------
+    int K = uniform ? top_p_fast(p, a, nC, p.p_fix, S.H, S.wc, S.wsum, S.s_res, S.flist, &S.s_i[5]) : -1;
+    if (K < 0) { __syncthreads(); K = top_p_count<SEL_T>(p, a, nC, p.p_fix, S.hcnt, S.hsum, S.wc, S.wsum, S.s_res); }
+    if (tid == 0) {
+      Kout[task] = K;
+      atomicAdd(acc + task, K);                    // Eq. 8 needs only the sums over layers and heads
+    }
+    return;
+  }
+  // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
+  const int nblk = nC / GP_PAGE;
+  const int K_t = nC - ne;
+  const int kq = min(p.k_loc, K_t / nblk);
+  if (kq > 0) {
+    for (int i = tid; i < nC; i += SEL_T) {
+      const double s = a[i];
+      const int b0 = i & ~15;
+      int rank = 0;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const double sj = a[b0 + j];
+        rank += (sj > s) || (sj == s && (b0 + j) < i);
+      }
+      if (rank < kq) atomicOr(&S.loc[i >> 5], 1u << (i & 31));
+    }
+  }
+  __syncthreads();
+  // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
+  if (!uniform || !evict_fast(a, nC, S.loc, S.H, S.wc, S.s_res, S.flist, S.flist_slot, &S.s_i[6], S.ev, (unsigned)ne))
+    evict_general(p, a, nC, S.loc, S.hcnt, S.wc, S.s_res, S.s_i, S.ev, (unsigned)ne);
+  __syncthreads();
+  if (tid < ne) {                                   // the evicted slots in ascending order, by rank
+    const int mine = S.ev[tid];
+    int rank = 0;
+    for (int j = 0; j < ne; ++j) rank += (S.ev[j] < mine);
+    evout[rank] = mine;
+  }
+}
+
 template <bool SHR>      // SHR: the pool runs the Shrink policy (a fourth job per unit)
-__global__ void __launch_bounds__(SEL_T, 1)
+__global__ void __launch_bounds__(SEL_T, 2)
 gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
-               float* __restrict__ out) {
+               float* __restrict__ out, int serial) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
-  double* sbuf = reinterpret_cast<double*>(smem);                              // [SEL_CAP] a^S, a^L or s
-  unsigned* hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::BUF_BYTES);
-  unsigned long long* hsum = reinterpret_cast<unsigned long long*>(hcnt + FB_PAD);   // two u32 planes (low, high)
-  unsigned long long* wsum = hsum + FB_PAD;                                    // [SEL_NW]
-  unsigned* wc = reinterpret_cast<unsigned*>(wsum + SEL_NW);                   // [SEL_NW]
-  long long* s_res = reinterpret_cast<long long*>(wc + SEL_NW);                // [8]
-  int* ev = reinterpret_cast<int*>(s_res + 8);                                 // [32]
-  int* s_i = ev + 32;                                                          // [16]
-  double* red = reinterpret_cast<double*>(s_i + 16);                           // [SEL_NW][16]
-  double* sM = red + SEL_NW * 16;                                                   // [16]
-  double* sZ = sM + 16;                                                        // [16]
-  double* flist = sZ + 16;                                                     // [32] members of the crossing bin
-  int* flist_slot = reinterpret_cast<int*>(flist + 32);                        // [32]
-  unsigned* coarse = reinterpret_cast<unsigned*>(flist_slot + 32);             // [3][CBINS] summary bins
-  unsigned* loc = coarse + 3 * CBINS;                                          // [cap*b/32 + 1]
-  double* F = reinterpret_cast<double*>(hcnt);                                 // softmax factors, before the bins are used
-  constexpr int F_CAP = (int)(SelGeom::H_BYTES / sizeof(double));
-  FastHist H;
-  H.cnt = hcnt; H.lo = reinterpret_cast<unsigned*>(hsum); H.hi = H.lo + FB_PAD;
-  H.ccnt = coarse; H.clo = coarse + CBINS; H.chi = coarse + 2 * CBINS;
+  SelSmem S;
+  S.sbuf = reinterpret_cast<double*>(smem);
+  S.hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::BUF_BYTES);
+  S.hsum = reinterpret_cast<unsigned long long*>(S.hcnt + FB_PAD);           // two u32 planes (low, high)
+  S.wsum = S.hsum + FB_PAD;
+  S.wc = reinterpret_cast<unsigned*>(S.wsum + SEL_NW);
+  S.s_res = reinterpret_cast<long long*>(S.wc + SEL_NW);
+  S.ev = reinterpret_cast<int*>(S.s_res + 8);
+  S.s_i = S.ev + 32;
+  S.red = reinterpret_cast<double*>(S.s_i + 16);
+  S.sM = S.red + SEL_NW * 16;
+  S.sZ = S.sM + 16;
+  S.flist = S.sZ + 16;
+  S.flist_slot = reinterpret_cast<int*>(S.flist + 32);
+  unsigned* coarse = reinterpret_cast<unsigned*>(S.flist_slot + 32);           // [3][CBINS] summary bins
+  S.loc = coarse + 3 * CBINS;
+  S.H.cnt = S.hcnt; S.H.lo = reinterpret_cast<unsigned*>(S.hsum); S.H.hi = S.H.lo + FB_PAD;
+  S.H.ccnt = coarse; S.H.clo = coarse + CBINS; S.H.chi = coarse + 2 * CBINS;
+  int* s_i = S.s_i;
   // the decision scratch aliases the score staging area: it is used after the last item only
 
   const int tid = threadIdx.x;
@@ -850,9 +940,9 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   }
   const int n_bnd = __ldcg(p.hdr + HDR_N_BND);
   const int n_mc = out ? __ldcg(p.hdr + HDR_N_MC) : 0, n_rc = __ldcg(p.hdr + HDR_N_RC);   // out == null: already merged layer by layer
+  const long long items = (long long)n_bnd * LH * NT;
   gp_pdl_wait();
   gp_pdl_launch_dependents();
-  const long long items = (long long)n_bnd * LH * NT;
 
   // CTAs without a job merge the split requests' attention partials while the others work; when fewer than a
   // quarter of the CTAs are idle, everybody merges after the jobs instead
@@ -899,59 +989,9 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     if (SHR && job == 3 && Pr - 1 < p.min_pages_after_shrink) continue;      // this boundary cannot be a Shrink
     const size_t view_stride = (size_t)p.z_stride * G;
     const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;   // [2 views][nC][G] exp(logit - page max)
-    double* a = nC <= SEL_CAP ? sbuf : p.scores + ((size_t)job * LH + lh) * p.max_batch_tokens + off;
-    if (task == 2) for (int i = tid; i < (nC + 31) / 32; i += SEL_T) loc[i] = 0;
-    if (tid == 0) { s_res[0] = -1; s_i[0] = 0; s_i[5] = 0; s_i[6] = 0; s_i[7] = 0; }
-    bool uniform;
-    {
-      const double* zs = p.zstat + ((size_t)lh * (p.max_batch_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
-      switch (G) {
-        case 1: uniform = job_softmax<1>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
-        case 2: uniform = job_softmax<2>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
-        case 4: uniform = job_softmax<4>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
-        default: uniform = job_softmax<8>(p, z, view_stride, zs, a, nC, task, red, sM, sZ, F, F_CAP); break;
-      }
-    }
-    fast_hist_zero(H, task < 2);                   // the factors' table shared this memory
-    if (task < 2) {
-      __syncthreads();
-      // ---- Eq. 7 -------------------------------------------------------------------------------------------
-      int K = uniform ? top_p_fast(p, a, nC, p.p_fix, H, wc, wsum, s_res, flist, &s_i[5]) : -1;
-      if (K < 0) { __syncthreads(); K = top_p_count<SEL_T>(p, a, nC, p.p_fix, hcnt, hsum, wc, wsum, s_res); }
-      if (tid == 0) {
-        Kout[task] = K;
-        atomicAdd(&p.bnd_acc[4 * bidx + task], K);            // Eq. 8 needs only the sums over layers and heads
-      }
-      continue;
-    }
-    // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
-    const int nblk = Pr - 1;
-    const int K_t = nC - ne;
-    const int kq = min(p.k_loc, K_t / nblk);
-    if (kq > 0) {
-      for (int i = tid; i < nC; i += SEL_T) {
-        const double s = a[i];
-        const int b0 = i & ~15;
-        int rank = 0;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const double sj = a[b0 + j];
-          rank += (sj > s) || (sj == s && (b0 + j) < i);
-        }
-        if (rank < kq) atomicOr(&loc[i >> 5], 1u << (i & 31));
-      }
-    }
-    __syncthreads();
-    // ---- global cut: the b lowest of the rest are evicted (score asc, slot desc) --------------------------------
-    if (!uniform || !evict_fast(a, nC, loc, H, wc, s_res, flist, flist_slot, &s_i[6], ev, (unsigned)ne))
-      evict_general(p, a, nC, loc, hcnt, wc, s_res, s_i, ev, (unsigned)ne);
-    __syncthreads();
-    if (tid < ne) {                                          // the evicted slots in ascending order, by rank
-      const int mine = ev[tid];
-      int rank = 0;
-      for (int j = 0; j < ne; ++j) rank += (ev[j] < mine);
-      evout[rank] = mine;
-    }
+    const double* zs = p.zstat + ((size_t)lh * (p.max_boundary_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
+    double* a = nC <= SEL_CAP ? S.sbuf : p.scores + ((size_t)job * LH + lh) * p.max_boundary_tokens + off;
+    sel_job(p, S, z, view_stride, zs, a, nC, task, ne, Kout, p.bnd_acc + 4 * bidx, evout);
   }
 
   // ---- the last CTA takes the decisions ----------------------------------------------------------------------
@@ -965,7 +1005,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (s_i[2]) {
     __threadfence();
-    decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(sbuf));
+    decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(S.sbuf), serial);
   }
 
   if (!idle_merge) merge_partials(p, n_req, out, n_mc, n_rc, (int)gridDim.x - 1 - (int)blockIdx.x, (int)gridDim.x, 0, LH);
@@ -985,7 +1025,7 @@ gp_merge_kernel(const __grid_constant__ GpDev p, int n_req, float* __restrict__ 
 // ------------------------------------------------------------------------------------------------------
 template <int D, bool SHR>
 __global__ void __launch_bounds__(CT)
-gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req) {
+gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int serial) {
   constexpr int CH = D / 8;
   constexpr int ROW_BYTES = D * 2;
   constexpr int PIECES = MOVE_TOK * 2 * CH / CT;        // 16-byte pieces per thread per chunk
@@ -1005,7 +1045,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   const int n_cmp = p.hdr[HDR_N_CMP];
   const int n_items = p.hdr[HDR_N_CITEM];
   const int n_cow = p.hdr[HDR_N_COW];
-  const int stamp = p.hdr[HDR_STEP];
+  const int stamp = serial + 1;       // unique per decode step of the pool: the chunk flags are never cleared
   for (int i = tid + CT; i <= n_cmp; i += CT) s_info[i] = p.cmp_info[i];
 
   for (bool first = true;; first = false) {
@@ -1181,7 +1221,7 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 }  // namespace
 
 // the compaction kernel of a pool: head dimension, and whether the Shrink policy is on
-static auto compact_kernel_of(const GpDev& p) -> void (*)(const GpDev, const int*, int) {
+static auto compact_kernel_of(const GpDev& p) -> void (*)(const GpDev, const int*, int, int) {
   const bool shr = p.policy == GP_POLICY_SHRINK;
   if (p.d == 128) return shr ? gp_compact_kernel<128, true> : gp_compact_kernel<128, false>;
   return shr ? gp_compact_kernel<64, true> : gp_compact_kernel<64, false>;
@@ -1214,11 +1254,13 @@ void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, i
 }
 
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
-                        int grid_compact, cudaStream_t s, cudaEvent_t ev, bool pdl) {
+                        int grid_compact, cudaStream_t s, cudaEvent_t ev, bool pdl, int serial) {
   const size_t sel_sm = gp_bsel_smem(p);
   const bool shr = p.policy == GP_POLICY_SHRINK;
-  gp_launch(shr ? gp_bsel_kernel<true> : gp_bsel_kernel<false>, grid_sel, SEL_T, sel_sm, s, pdl, p, req_ids, n_req,
-            actions, out);
+  // asynchronous mode: the kernel before this one on its stream belongs to another step (an event wait lies in
+  // between): plain launch; the compaction kernel follows as a programmatic dependent as usual
+  gp_launch(shr ? gp_bsel_kernel<true> : gp_bsel_kernel<false>, grid_sel, SEL_T, sel_sm, s, pdl && !p.async, p, req_ids,
+            n_req, actions, out, serial);
   if (ev) cudaEventRecord(ev, s);
-  gp_launch(compact_kernel_of(p), grid_compact, CT, 0, s, pdl, p, req_ids, n_req);
+  gp_launch(compact_kernel_of(p), grid_compact, CT, 0, s, pdl, p, req_ids, n_req, serial);
 }

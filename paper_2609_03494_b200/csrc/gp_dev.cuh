@@ -10,7 +10,7 @@
 //   tok       int32 [L][n_pages][H_kv][b]               original token index of every slot
 //   summaries fp64  [L][M][2][2][H_q][d]                Eq. 11 layout (short then long), double-buffered
 //   page_table / shadow int32 [M][cap]                  shadow holds copy-on-write targets
-//   scores    fp64  [2][L*H_kv][max_batch_tokens]       a^S, a^L of the requests at a boundary
+//   scores    fp64  [jobs][L*H_kv][max_boundary_tokens] scores of candidate sets too large for shared memory
 //   partials  fp32  split-KV partial outputs
 #pragma once
 #include <cuda_bf16.h>
@@ -53,6 +53,8 @@ struct GpDev {
   // geometry
   int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;
   long long n_pages, max_batch_tokens;
+  long long max_boundary_tokens;         // bound on the summed candidate tokens of one step's boundary requests
+  int async;                             // 1: the boundary chain of a step runs beside the next step (see gp_decode_step)
   double beta_s, beta_l, top_p, tau, rope_theta;
   int bchunk_pages;                      // pages per work item of a request at its capacity boundary
   int policy;                            // GP_POLICY_* (0 demand, 1 inverse, 2 random, 3 shrink)
@@ -71,6 +73,8 @@ struct GpDev {
   int* shadow;
   // per request
   int* P; int* n; int* started; int* live; int* n_pristine; long long* pos;
+  int* bstep;                            // [M] number of the decode step at which the request last reached its boundary
+  int* last_act;                         // [M] decision taken at that boundary (GP_ACT_*)
   double* summ;
   int* Kx;                               // [M][L][H_kv][2]
   double* delta;                         // [M]
@@ -90,9 +94,9 @@ struct GpDev {
   int* free_peek;                        // [M+1] free_top at plan time, then the top entries of the free list, top first
   int4* cmp_info;                        // [M+1] compressing requests: {request, P, index in bnd_info, first compaction chunk}
   double* zbuf;                          // [L*H_kv][2][z_stride][G] boundary units, per view (short, long): exp(summary logit - its page's max)
-  long long z_stride;                    // max_batch_tokens rounded up to a multiple of the page size
+  long long z_stride;                    // max_boundary_tokens rounded up to a multiple of the page size
   double* qtil;                          // [M][L*H_kv][2][G][d] calibrated, rotated summaries q~ of boundary requests, by batch slot
-  double* zstat;                         // [L*H_kv][max_batch_tokens / b][2][G][2] per-page softmax partials (max, sum)
+  double* zstat;                         // [L*H_kv][max_boundary_tokens / b][2][G][2] per-page softmax partials (max, sum)
   int* sum_par;                          // [M] which of the two summary buffers is current
   int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
   int* evict2;                           // [M][L*H_kv][2b] slots a Shrink evicts, ascending (Shrink policy only)
@@ -215,7 +219,7 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 
 // ---- host-visible launchers (one per translation unit) -------------------------------------------
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n);
+                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n, int serial);
 size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
 // ---- programmatic dependent launch -------------------------------------------------------------------
@@ -251,4 +255,4 @@ size_t gp_bsel_smem_for_cap(long long cap);
 // boundary chain: probabilities + working sets + selection + decision, then compaction.
 // `ev`, when not null, is recorded between the two kernels.  `pdl`: launch with programmatic stream serialization.
 void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel,
-                        int grid_compact, cudaStream_t s, cudaEvent_t ev, bool pdl);
+                        int grid_compact, cudaStream_t s, cudaEvent_t ev, bool pdl, int serial);

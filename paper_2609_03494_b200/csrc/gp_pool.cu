@@ -12,11 +12,20 @@
 #include "gp_dev.cuh"
 
 #define GP_PLAN_THREADS 1024
+#define GP_NEVER (-(1 << 30))      // bstep of a request that has not reached a boundary
 
 struct gp_pool {
   gp_config cfg;
   int device;
   GpDev dev;
+  // asynchronous boundary mode: steps alternate between two sets of the scratch that a step's boundary chain
+  // still reads while the next step runs (dev, dev_alt); the chain runs on `side`
+  GpDev dev_alt;
+  cudaStream_t side;
+  cudaEvent_t e_attn[2], e_chain[2];
+  int chain_pending[2];
+  int attn_grid_async, sel_grid_async, compact_grid_async;
+  long long serial;                                 // decode steps issued so far
   void* blob;
   size_t bytes;
   std::vector<uint8_t> live;      // host mirror of the slot free list
@@ -34,7 +43,9 @@ struct gp_pool {
   // measurement
   int profiling;
   int early_plan;                 // gp_set_early_plan: the plan kernel reads the caller's inputs before its wait
+  int first_plain;                // the step's first kernel follows a kernel of another kind: plain launch
   cudaEvent_t ev[GP_N_KERNELS + 1];
+  cudaEvent_t ev_side[3];                           // asynchronous mode: around the two kernels on `side`
   float ms[GP_N_KERNELS];
   int64_t launches[GP_N_KERNELS];
   int64_t launch_count;
@@ -46,10 +57,11 @@ namespace {
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
       b_flags, mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
+      bnd_info2, bnd_acc2, zbuf2, zstat2,
       evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
   int max_rc;
-  long long max_batch_tokens;
+  long long max_batch_tokens, max_boundary_tokens;
 };
 
 inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -77,7 +89,8 @@ bool valid_config(const gp_config* c) {
   if (gp_bsel_smem_for_cap(c->max_pages_per_req) > GP_MAX_DYN_SMEM) return false;   // about 62 000 pages
   if (c->n_pages < 1 || c->n_pages > 0x7fffffffLL / GP_PAGE) return false;
   if (c->k_loc < 0 || c->k_loc > GP_PAGE) return false;
-  if (c->max_batch_tokens < 0) return false;
+  if (c->max_batch_tokens < 0 || c->max_boundary_tokens < 0) return false;
+  if (c->async_boundary < 0 || c->async_boundary > 1 || c->async_slots < 0 || c->async_slots > 4096) return false;
   if (!(c->beta_s >= 0.0 && c->beta_s < 1.0 && c->beta_l >= 0.0 && c->beta_l < 1.0)) return false;
   if (!(c->top_p > 0.0 && c->top_p < 1.0)) return false;
   if (!(c->rope_theta >= 0.0)) return false;
@@ -93,6 +106,11 @@ Layout make_layout(const gp_config& c) {
   const size_t LH = (size_t)c.n_layers * c.n_kv_heads, G = c.n_q_heads / c.n_kv_heads;
   const size_t np = (size_t)c.n_pages;
   L.max_batch_tokens = c.max_batch_tokens > 0 ? c.max_batch_tokens : (long long)(np * b);
+  // candidate tokens of one step's boundary requests: by default every request of a batch may be at its boundary
+  // (equal prompts reach it together); a caller that knows better sizes the boundary scratch smaller
+  L.max_boundary_tokens = c.max_boundary_tokens > 0 ? c.max_boundary_tokens : L.max_batch_tokens;
+  if (L.max_boundary_tokens < (long long)(cap * b) && L.max_batch_tokens >= (long long)(cap * b)) L.max_boundary_tokens = (long long)(cap * b);
+  const size_t Tb = (size_t)L.max_boundary_tokens;
   const int ch = chunk_pages_setting();
   int bch = bchunk_pages_setting() < ch ? bchunk_pages_setting() : ch;
   if (bch > GP_FINE_BCHUNK) bch = GP_FINE_BCHUNK;            // small launches cut finer
@@ -106,7 +124,7 @@ Layout make_layout(const gp_config& c) {
   L.words = take(256 * 4);                       // free_top, err, plan header, status
   L.page_table = take(M * cap * 4);
   L.shadow = take(M * cap * 4);
-  L.reqi = take(5 * M * 4);                      // P, n, started, live, n_pristine
+  L.reqi = take(7 * M * 4);                      // P, n, started, live, n_pristine, bstep, last_act
   L.sum_par = take(M * 4);
   L.pos = take(M * 8);
   L.summ = take((size_t)c.n_layers * M * 2 * 2 * c.n_q_heads * d * 8);
@@ -120,15 +138,23 @@ Layout make_layout(const gp_config& c) {
   L.bnd_acc = take(M * 16);
   L.free_peek = take((M + 1) * 4);
   L.cmp_info = take((M + 1) * 16);
-  L.zbuf = take(LH * (size_t)(L.max_batch_tokens + b) * 2 * G * 8);
+  L.zbuf = take(LH * (Tb + b) * 2 * G * 8);
   L.qtil = take(M * LH * 2 * (size_t)G * d * 8);
-  L.zstat = take(LH * ((size_t)L.max_batch_tokens / b + 1) * 2 * G * 2 * 8);
+  L.zstat = take(LH * (Tb / b + 1) * 2 * G * 2 * 8);
   L.evict = take(M * LH * b * 4);
   L.evict2 = take(c.policy == GP_POLICY_SHRINK ? M * LH * 2 * b * 4 : 16);
-  L.cflags = take(LH * ((size_t)L.max_batch_tokens / GP_MOVE_TOK + 2 * M + 1) * 4);
+  L.cflags = take(LH * ((Tb + M * b) / GP_MOVE_TOK + 2 * M + 1) * 4);
   L.rope_cs = take(M * (d / 2) * 2 * 8);
   L.partials = take((size_t)L.max_rc * LH * G * (d + 2) * 4);
-  L.scores = take((c.policy == GP_POLICY_SHRINK ? 4 : 3) * LH * (size_t)L.max_batch_tokens * 8);
+  L.scores = take((c.policy == GP_POLICY_SHRINK ? 4 : 3) * LH * Tb * 8);
+  if (c.async_boundary) {                        // the second set of what a boundary chain reads beside the next step
+    L.bnd_info2 = take(M * 32);
+    L.bnd_acc2 = take(M * 16);
+    L.zbuf2 = take(LH * (Tb + b) * 2 * G * 8);
+    L.zstat2 = take(LH * (Tb / b + 1) * 2 * G * 2 * 8);
+  } else {
+    L.bnd_info2 = L.bnd_acc2 = L.zbuf2 = L.zstat2 = 0;
+  }
   L.counters = take(16 * 8);
   L.dbg = take(cap * b * (4 + 2 * d * 2));
   if (c.host_staging) {
@@ -154,6 +180,7 @@ __global__ void gp_init_kernel(GpDev p) {
   // page 0 is handed out first
   for (long long i = i0; i < p.n_pages; i += stride) p.free_stack[i] = (int)(p.n_pages - 1 - i);
   for (long long i = i0; i < (long long)p.M * p.cap; i += stride) p.shadow[i] = -1;
+  for (long long i = i0; i < p.M; i += stride) p.bstep[i] = GP_NEVER;
   if (i0 == 0) *p.free_top = (int)p.n_pages;
 }
 
@@ -266,7 +293,10 @@ __device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __re
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
                const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n, int cp_norm, int cp_bnd,
-               int launch_units, int launch_grid) {
+               int launch_units, int launch_grid, int serial) {
+  // serial: number of this decode step (asynchronous boundary mode: a request that reached its boundary at
+  // step serial - 1 sits this step out; its counters and pages belong to that step's boundary chain, which may
+  // still be running)
   // cp_norm, cp_bnd: pages per work item, for requests in general and for those at their capacity boundary, when
   // the attention launch has work for large items; launch_units: (layer, head) units per request in one
   // attention launch; launch_grid: its CTAs
@@ -310,7 +340,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     __syncthreads();
     if (in) {
       int ok = 0;
-      if (r >= 0 && s_first[r] == i && __ldcg(p.live + r)) {
+      if (r >= 0 && s_first[r] == i && __ldcg(p.live + r) && !(p.async && __ldcg(p.bstep + r) == serial - 1)) {
         ok = 1;
         s_chunks[i] = __ldcg(p.n + r);
         s_pos[i] = __ldcg(p.P + r);
@@ -350,16 +380,19 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   long long nc = 0, pos = 0;
   int isb = 0;
   int cp = cp_norm;                       // pages per work item of this request
-  int live = 0;
+  int live = 0, held = 0;
   if (in && r >= 0 && r < p.M) {          // independent loads, issued together (from the L2: before the wait)
     live = __ldcg(p.live + r); n_old = __ldcg(p.n + r); Pr = __ldcg(p.P + r); pos = __ldcg(p.pos + r);
     started = __ldcg(p.started + r); par = __ldcg(p.sum_par + r);
+    if (p.async) held = __ldcg(p.bstep + r) == serial - 1;
   }
   if (in) {
     const bool inrange = r >= 0 && r < p.M;
     const bool valid = inrange && live && s_first[r] == i;
     if (!valid) {
       act = GP_ACT_INVALID;
+    } else if (held) {
+      act = GP_ACT_HELD;                  // its boundary chain may still be running: nothing of it is looked at
     } else if (n_old >= Pr * GP_PAGE) {
       act = GP_ACT_STALLED;
     } else {
@@ -389,7 +422,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   // can exceed what the pool holds) does not fit the scratch: a request whose boundary logits or whose work
   // items do not fit is not stepped (its state stays as it is, it can be stepped again in a later batch).  The
   // offsets are then taken again over what is left, so that the item list has no holes.
-  const bool dropped = chunks > 0 && ((isb && tok_off + nc > p.max_batch_tokens) || rc_off + chunks > p.max_rc);
+  const bool dropped = chunks > 0 && ((isb && tok_off + nc > p.max_boundary_tokens) || rc_off + chunks > p.max_rc);
   if (dropped) { chunks = 0; isb = 0; nc = 0; act = GP_ACT_SCRATCH; }
   if (__syncthreads_or(dropped)) plan_scan(chunks, nc, rc_off, tok_off, n_rc, tok_tot, sv, sw);
   int bnd_idx, n_bnd, n_active; long long d0, d1;
@@ -422,6 +455,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   if (in) {
     p.b_nold[i] = n_old;
     p.b_flags[i] = chunks > 0;
+    if (isb) { p.bstep[r] = serial; if (p.async) act = GP_ACT_PENDING; }
     actions[i] = act;
     if (isb) {
       p.bnd_info[2 * bnd_idx] = make_int4(i, r, Pr, (int)pos);     // pos: position of this step's token
@@ -464,13 +498,15 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   }
   // ---- from here on the kernel before this one has completed --------------------------------------------
   gp_pdl_wait();
-  const int free_top0 = *p.free_top;
-  // the top of the free list, one page per boundary request: what this step's grants can take
-  if (in && isb && bnd_idx < free_top0) p.free_peek[1 + bnd_idx] = p.free_stack[free_top0 - 1 - bnd_idx];
-  if (threadIdx.x == 0) {
-    p.free_peek[0] = free_top0;
-    p.hdr[HDR_STEP] += 1;
+  if (!p.async) {
+    // the top of the free list, one page per boundary request: what this step's grants can take.  (In the
+    // asynchronous mode the free list belongs to the boundary chains, which run one after the other: the
+    // decision step reads it itself.)
+    const int free_top0 = *p.free_top;
+    if (in && isb && bnd_idx < free_top0) p.free_peek[1 + bnd_idx] = p.free_stack[free_top0 - 1 - bnd_idx];
+    if (threadIdx.x == 0) p.free_peek[0] = free_top0;
   }
+  if (threadIdx.x == 0) p.hdr[HDR_STEP] += 1;
 }
 
 __global__ void gp_admit_kernel(GpDev p, int r, int share_from, int n_shared, int n_tail, int P_target, int* status) {
@@ -500,6 +536,7 @@ __global__ void gp_admit_kernel(GpDev p, int r, int share_from, int n_shared, in
       const int n0 = n_shared * GP_PAGE + n_tail;
       *p.free_top = top - need;
       p.P[r] = P_target; p.n[r] = n0; p.pos[r] = n0; p.started[r] = 0; p.live[r] = 1;
+      p.bstep[r] = GP_NEVER; p.last_act[r] = GP_ACT_NONE;
       p.n_pristine[r] = n0 / GP_PAGE;
     }
   }
@@ -581,7 +618,21 @@ __global__ void gp_gather_kernel(GpDev p, int r, int l, int h, int n, int* tok_o
 
 void pool_free(gp_pool* pool) {
   if (pool->h_err) cudaFreeHost(pool->h_err);
+  for (int i = 0; i < 2; ++i) {
+    if (pool->e_attn[i]) cudaEventDestroy(pool->e_attn[i]);
+    if (pool->e_chain[i]) cudaEventDestroy(pool->e_chain[i]);
+  }
+  for (int i = 0; i < 3; ++i)
+    if (pool->ev_side[i]) cudaEventDestroy(pool->ev_side[i]);
+  if (pool->side) cudaStreamDestroy(pool->side);
   delete pool;
+}
+
+// asynchronous boundary mode: `s` waits for the boundary chains issued so far
+int join_side(gp_pool* pool, cudaStream_t s) {
+  for (int i = 0; i < 2; ++i)
+    if (pool->chain_pending[i] && cudaStreamWaitEvent(s, pool->e_chain[i], 0) != cudaSuccess) return GP_ERR_CUDA;
+  return GP_OK;
 }
 
 // the kernels' error bits, once the work that could set them has completed
@@ -645,10 +696,12 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   pool->live.assign(cfg->max_requests, 0);
   pool->profiling = 0;
   pool->early_plan = 0;
+  pool->first_plain = 0;
   pool->step_open = 0; pool->step_n_req = 0; pool->step_layers_done = 0;
   pool->step_layer_seen.assign(cfg->n_layers, 0);
   pool->h_err = nullptr;
   pool->launch_count = 0;
+  pool->serial = 0;
   memset(pool->ms, 0, sizeof(pool->ms));
   memset(pool->launches, 0, sizeof(pool->launches));
   cudaDeviceProp prop;
@@ -663,7 +716,9 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc;
   d.bchunk_pages = bchunk_pages_setting();
   d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
-  d.z_stride = (L.max_batch_tokens + GP_PAGE - 1) / GP_PAGE * GP_PAGE;
+  d.max_boundary_tokens = L.max_boundary_tokens;
+  d.async = cfg->async_boundary;
+  d.z_stride = (L.max_boundary_tokens + GP_PAGE - 1) / GP_PAGE * GP_PAGE;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
   d.policy = cfg->policy; d.policy_seed = (unsigned long long)(unsigned)cfg->policy_seed; d.p_compress = cfg->p_compress;
   d.shrink_below = cfg->shrink_below;
@@ -697,6 +752,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   int* reqi = reinterpret_cast<int*>(base + L.reqi);
   const int M = cfg->max_requests;
   d.P = reqi; d.n = reqi + M; d.started = reqi + 2 * M; d.live = reqi + 3 * M; d.n_pristine = reqi + 4 * M;
+  d.bstep = reqi + 5 * M; d.last_act = reqi + 6 * M;
   d.pos = reinterpret_cast<long long*>(base + L.pos);
   d.summ = reinterpret_cast<double*>(base + L.summ);
   d.Kx = reinterpret_cast<int*>(base + L.Kx);
@@ -722,6 +778,32 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.counters = reinterpret_cast<long long*>(base + L.counters);
   gp_attention_setup(d);
   gp_boundary_setup(d, pool->num_sms, &pool->sel_grid, &pool->compact_grid);
+  pool->dev_alt = d;
+  pool->side = nullptr;
+  pool->chain_pending[0] = pool->chain_pending[1] = 0;
+  if (cfg->async_boundary) {
+    GpDev& a = pool->dev_alt;
+    a.hdr = words + 128;
+    a.bnd_info = reinterpret_cast<int4*>(base + L.bnd_info2);
+    a.bnd_acc = reinterpret_cast<int*>(base + L.bnd_acc2);
+    a.zbuf = reinterpret_cast<double*>(base + L.zbuf2);
+    a.zstat = reinterpret_cast<double*>(base + L.zstat2);
+    // the boundary kernels run beside the attention kernel on the room it leaves: `slots` of its thread blocks
+    int slots = cfg->async_slots > 0 ? cfg->async_slots : 48;
+    if (slots > pool->attn_grid / 2) slots = pool->attn_grid / 2;
+    pool->attn_grid_async = pool->attn_grid - slots;
+    pool->sel_grid_async = slots < pool->sel_grid ? slots : pool->sel_grid;
+    pool->compact_grid_async = 2 * slots < pool->compact_grid ? 2 * slots : pool->compact_grid;
+    int lo = 0, hi = 0;
+    cudaDeviceGetStreamPriorityRange(&lo, &hi);                 // hi = the numerically lowest = most urgent
+    if (cudaStreamCreateWithPriority(&pool->side, cudaStreamNonBlocking, hi) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
+    for (int i = 0; i < 2; ++i) {
+      if (cudaEventCreateWithFlags(&pool->e_attn[i], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&pool->e_chain[i], cudaEventDisableTiming) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
+    }
+    for (int i = 0; i < 3; ++i)
+      if (cudaEventCreate(&pool->ev_side[i]) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
+  }
   pool->dbg = base + L.dbg;
   if (cfg->host_staging) {
     pool->st_ids = reinterpret_cast<int*>(base + L.st_ids);
@@ -773,6 +855,7 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   if (P > c.max_pages_per_req) P = (long long)c.max_pages_per_req + 1;      // still refused, and fits an int
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (join_side(pool, s) != GP_OK) return GP_ERR_CUDA;        // the free list belongs to the boundary chains in flight
   gp_admit_kernel<<<1, 32, 0, s>>>(pool->dev, slot, share_from, n_shared_pages, n_tail, (int)P, pool->d_status);
   pool->launch_count++;
   int st = GP_ERR_CUDA;
@@ -796,15 +879,16 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
 
 // CTA 0 plans (when plan_on); the others update the query summaries of the units [lh0, lh0 + lh_n)
 static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_t* actions, const void* q, int plan_on,
-                        int lh0, int lh_n, cudaStream_t s, bool pdl, bool by_layer = false) {
-  const GpDev& d = pool->dev;
+                        int lh0, int lh_n, cudaStream_t s, bool pdl, bool by_layer = false, const GpDev* dev = nullptr,
+                        int attn_grid = 0) {
+  const GpDev& d = dev ? *dev : pool->dev;
   const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
   const long long want = ((long long)n_req * lh_n + upc - 1) / upc;
   const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
   const int prep = (int)(want < room ? want : room);
   gp_launch(gp_plan_kernel, 1 + prep, GP_PLAN_THREADS, 0, s, pdl, d, ids, n_req, actions,
             static_cast<const __nv_bfloat16*>(q), plan_on, lh0, lh_n, d.chunk_pages, d.bchunk_pages,
-            by_layer ? d.Hkv : d.L * d.Hkv, pool->attn_grid);
+            by_layer ? d.Hkv : d.L * d.Hkv, attn_grid ? attn_grid : pool->attn_grid, (int)(pool->serial & 0x3fffffff));
 }
 
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
@@ -818,29 +902,96 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
       misaligned(dev_req_ids, 4) || misaligned(dev_actions, 4)) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const GpDev& d = pool->dev;
-  const int LH = d.L * d.Hkv;
   const bool prof = pool->profiling != 0;
-  if (prof) cudaEventRecord(pool->ev[0], s);
   const bool pdl = !prof;                      // events between the kernels need them serialised the plain way
-  launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl);
-  if (prof) cudaEventRecord(pool->ev[1], s);
-  gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH);
-  if (prof) cudaEventRecord(pool->ev[2], s);
-  gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s,
-                     prof ? pool->ev[3] : nullptr, pdl);
-  if (prof) cudaEventRecord(pool->ev[4], s);
-  pool->launch_count += GP_N_KERNELS;
+  const int serial = (int)(pool->serial & 0x3fffffff);
+  if (!pool->cfg.async_boundary) {
+    const GpDev& d = pool->dev;
+    const int LH = d.L * d.Hkv;
+    if (prof) cudaEventRecord(pool->ev[0], s);
+    // first_plain: the kernel before the plan on the stream is not one of this library's (the host entry point's
+    // fetch of the inputs): no programmatic dependence on it
+    launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl && !pool->first_plain);
+    if (prof) cudaEventRecord(pool->ev[1], s);
+    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH, serial);
+    if (prof) cudaEventRecord(pool->ev[2], s);
+    gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s,
+                       prof ? pool->ev[3] : nullptr, pdl, serial);
+    if (prof) cudaEventRecord(pool->ev[4], s);
+    pool->launch_count += GP_N_KERNELS;
+  } else {
+    // Asynchronous boundary work.  On the caller's stream: plan, attention, merge of the split requests' partial
+    // outputs (the step's `out` is complete when the stream gets there).  On the pool's stream, after the
+    // attention kernel: working sets + decisions, compaction.  Step t uses scratch set t mod 2 and first waits
+    // for the chain of step t - 2, which read that set; the same wait, one step later, puts the chain of step
+    // t - 1 before the plan of step t + 1, the first to look at the requests that chain changes (they sit
+    // step t out).
+    const int par = (int)(pool->serial & 1);
+    const GpDev& d = par ? pool->dev_alt : pool->dev;
+    const int LH = d.L * d.Hkv;
+    if (pool->chain_pending[par]) GP_CUDA(cudaStreamWaitEvent(s, pool->e_chain[par], 0));
+    // the chain of the step before this one changes the pages and counters of requests this step skips, and
+    // the free list, which this step's own chain reads after it (same stream): nothing to wait for here
+    if (prof) cudaEventRecord(pool->ev[0], s);
+    launch_plan(pool, dev_req_ids, n_req, dev_actions, q, 1, 0, LH, s, pdl && !pool->first_plain, false, &d, pool->attn_grid_async);
+    if (prof) cudaEventRecord(pool->ev[1], s);
+    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid_async, s, pdl, 0, LH, serial);
+    if (prof) cudaEventRecord(pool->ev[2], s);
+    gp_launch_merge(d, n_req, static_cast<float*>(out), 0, LH, pool->num_sms, s, pdl);
+    GP_CUDA(cudaEventRecord(pool->e_attn[par], s));
+    GP_CUDA(cudaStreamWaitEvent(pool->side, pool->e_attn[par], 0));
+    if (prof) cudaEventRecord(pool->ev_side[0], pool->side);
+    gp_launch_boundary(d, dev_req_ids, n_req, nullptr, nullptr, pool->sel_grid_async, pool->compact_grid_async, pool->side,
+                       prof ? pool->ev_side[1] : nullptr, true, serial);
+    if (prof) cudaEventRecord(pool->ev_side[2], pool->side);
+    GP_CUDA(cudaEventRecord(pool->e_chain[par], pool->side));
+    pool->chain_pending[par] = 1;
+    pool->launch_count += GP_N_KERNELS + 1;
+  }
+  pool->serial += 1;
   GP_CUDA(cudaGetLastError());
   if (prof) {
-    GP_CUDA(cudaEventSynchronize(pool->ev[GP_N_KERNELS]));
-    for (int i = 0; i < GP_N_KERNELS; ++i) {
-      float t = 0.f;
-      GP_CUDA(cudaEventElapsedTime(&t, pool->ev[i], pool->ev[i + 1]));
-      pool->ms[i] += t;
-      pool->launches[i] += 1;
+    if (!pool->cfg.async_boundary) {
+      GP_CUDA(cudaEventSynchronize(pool->ev[GP_N_KERNELS]));
+      for (int i = 0; i < GP_N_KERNELS; ++i) {
+        float t = 0.f;
+        GP_CUDA(cudaEventElapsedTime(&t, pool->ev[i], pool->ev[i + 1]));
+        pool->ms[i] += t;
+        pool->launches[i] += 1;
+      }
+    } else {
+      GP_CUDA(cudaEventSynchronize(pool->ev[2]));
+      GP_CUDA(cudaEventSynchronize(pool->ev_side[2]));
+      for (int i = 0; i < GP_N_KERNELS; ++i) {
+        float t = 0.f;
+        if (i < 2) GP_CUDA(cudaEventElapsedTime(&t, pool->ev[i], pool->ev[i + 1]));
+        else GP_CUDA(cudaEventElapsedTime(&t, pool->ev_side[i - 2], pool->ev_side[i - 1]));
+        pool->ms[i] += t;
+        pool->launches[i] += 1;
+      }
     }
   }
+  return GP_OK;
+}
+
+int gp_async_join(gp_pool* pool, void* stream) {
+  if (!pool) return GP_ERR_INVALID;
+  if (!pool->cfg.async_boundary) return GP_OK;
+  GP_CUDA(cudaSetDevice(pool->device));
+  return join_side(pool, static_cast<cudaStream_t>(stream));
+}
+
+int gp_boundary_outcome(gp_pool* pool, int32_t req, int32_t* action, int64_t* step) {
+  const int st = check_req(pool, req);
+  if (st != GP_OK) return st;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  int a = 0, b = 0;
+  GP_CUDA(cudaMemcpy(&a, pool->dev.last_act + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&b, pool->dev.bstep + req, 4, cudaMemcpyDeviceToHost));
+  if (b == GP_NEVER) a = GP_ACT_NONE;
+  if (action) *action = a;
+  if (step) *step = b == GP_NEVER ? -1 : (int64_t)((pool->serial & ~0x3fffffffLL) | (long long)b);
   return GP_OK;
 }
 
@@ -848,7 +999,7 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
 // attention output ---------------------------------------------------------------------------------------
 int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions, void* stream) {
   if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
-  if (pool->step_open) return GP_ERR_STATE;
+  if (pool->step_open || pool->cfg.async_boundary) return GP_ERR_STATE;
   if (n_req == 0) return GP_OK;
   if (!dev_req_ids || !dev_actions || misaligned(dev_req_ids, 4) || misaligned(dev_actions, 4)) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
@@ -881,7 +1032,7 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
   float* ob = reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(out) - qs * 4);
   const int lh0 = layer * d.Hkv, lh_n = d.Hkv;
   launch_plan(pool, dev_req_ids, n_req, nullptr, qb, 0, lh0, lh_n, s, true);
-  gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n);
+  gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n, 0);
   gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
   pool->launch_count += 3;
   pool->step_layers_done += 1;
@@ -896,7 +1047,8 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
   if (pool->step_layers_done != pool->cfg.n_layers) return GP_ERR_STATE;       // layers missing: run them, or gp_step_abort
   GP_CUDA(cudaSetDevice(pool->device));
   gp_launch_boundary(pool->dev, dev_req_ids, n_req, dev_actions, nullptr, pool->sel_grid, pool->compact_grid,
-                     static_cast<cudaStream_t>(stream), nullptr, true);
+                     static_cast<cudaStream_t>(stream), nullptr, true, (int)(pool->serial & 0x3fffffff));
+  pool->serial += 1;
   pool->launch_count += 2;
   pool->step_open = 0;
   GP_CUDA(cudaGetLastError());
@@ -975,12 +1127,17 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
   const bool direct = cudaHostGetDevicePointer(&d_out, out, 0) == cudaSuccess &&
                       cudaHostGetDevicePointer(&d_act, actions, 0) == cudaSuccess;
   if (!direct) (void)cudaGetLastError();           // pageable memory: not an error, the staged path takes over
+  // The inputs arrive by the fetch kernel or the copies above, which end before the plan kernel starts: that
+  // kernel is launched the plain way here (not as a programmatic dependent of the fetch kernel, whose stores it
+  // reads), so planning ahead of its wait, which is then no wait at all, is safe whatever the option says.
   const int early = pool->early_plan;
-  pool->early_plan = 1;                            // the inputs arrive by the copies above: complete before any kernel
+  pool->early_plan = 1;
+  pool->first_plain = 1;
   const int st = gp_decode_step(pool, pool->st_ids, n_req, pool->st_q, pool->st_k, pool->st_v,
                                 direct ? d_out : static_cast<void*>(pool->st_out),
                                 direct ? static_cast<int32_t*>(d_act) : pool->st_act, stream);
   pool->early_plan = early;
+  pool->first_plain = 0;
   if (st != GP_OK) return st;
   if (!direct) {
     GP_CUDA(cudaMemcpyAsync(out, pool->st_out, qb * 2, cudaMemcpyDeviceToHost, s));
@@ -1002,6 +1159,7 @@ int gp_release(gp_pool* pool, int32_t req, void* stream) {
   if (st != GP_OK) return st;
   if (pool->step_open) return GP_ERR_STATE;      // the open step's plan holds a snapshot of the free list
   GP_CUDA(cudaSetDevice(pool->device));
+  if (join_side(pool, static_cast<cudaStream_t>(stream)) != GP_OK) return GP_ERR_CUDA;
   gp_release_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(pool->dev, req);
   pool->launch_count++;
   pool->live[req] = 0;
@@ -1038,6 +1196,16 @@ int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t
   if (page_table && Pv > 0)
     GP_CUDA(cudaMemcpy(page_table, pool->dev.page_table + (size_t)req * pool->cfg.max_pages_per_req, (size_t)Pv * 4,
                        cudaMemcpyDeviceToHost));
+  return GP_OK;
+}
+
+int gp_debug_state(gp_pool* pool, int32_t* P, int32_t* n) {
+  if (!pool) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  GP_CUDA(cudaDeviceSynchronize());
+  const size_t nb = (size_t)pool->cfg.max_requests * 4;
+  if (P) GP_CUDA(cudaMemcpy(P, pool->dev.P, nb, cudaMemcpyDeviceToHost));
+  if (n) GP_CUDA(cudaMemcpy(n, pool->dev.n, nb, cudaMemcpyDeviceToHost));
   return GP_OK;
 }
 

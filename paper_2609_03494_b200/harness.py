@@ -37,6 +37,9 @@ class _Resident:
     cache: Optional[Tuple[np.ndarray, np.ndarray, np.ndarray]] = None
 
 
+HELD = 6                 # action code of a request that sat a step out (asynchronous boundary work)
+
+
 class Scheduler:
     def __init__(self, wl: W.Workload):
         self.wl = wl
@@ -102,6 +105,8 @@ class Scheduler:
         out = []
         for idx, act in zip(specs, actions):
             res = self.resident[idx]
+            if int(act) == HELD:             # asynchronous boundary work: sat the step out, its token comes next step
+                continue
             res.step += 1
             self.tokens += 1
             if int(act) < 0:

@@ -51,14 +51,15 @@ def make_pools(wl: W.Workload, device: int = 0, **over):
     kw = dict(n_pages=wl.n_pages, max_pages_per_req=wl.max_pages_per_req,
               max_requests=max(4, wl.n_resident), k_loc=wl.k_loc)
     tun = {k: over[k] for k in ("beta_s", "beta_l", "top_p", "tau", "rope_theta", "policy", "policy_seed", "p_compress",
-                                    "shrink_below", "min_capacity")
+                                    "shrink_below", "min_capacity", "async_boundary")
            if k in over}
     for k in ("n_pages", "max_pages_per_req", "k_loc", "max_requests"):
         if k in over:
             kw[k] = over[k]
     ocfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, **kw, **tun)
     gcfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, **kw, **tun,
-                         max_batch_tokens=over.get("max_batch_tokens", 0))
+                         max_batch_tokens=over.get("max_batch_tokens", 0), async_slots=over.get("async_slots", 0),
+                         max_boundary_tokens=over.get("max_boundary_tokens", 0))
     return B.Pool(gcfg, device), O.OraclePool(ocfg)
 
 
@@ -110,7 +111,19 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
             g_act = act_t.cpu().numpy()
 
             # ---- attention outputs --------------------------------------------------------------------------
-            stepped = [i for i in range(Bn) if rec.actions[i] == 0]
+            stepped = [i for i in range(Bn) if rec.actions[i] in (O.ACT_NONE, O.ACT_PENDING)]
+            # what the GPU decided at this step's boundaries: in the step's actions, or, with asynchronous boundary
+            # work, asked for afterwards (the call waits for the boundary chain)
+            is_async = bool(over.get("async_boundary", False))
+            g_dec = {}
+            for rid in rec.boundary:
+                i = rids.index(rid)
+                if is_async:
+                    assert int(g_act[i]) == B.GP_ACT_PENDING, f"step {st.steps} req {rid}: action {g_act[i]}, expected pending"
+                    g_dec[rid], at = B.gp_boundary_outcome(gpu.handle, rid)
+                    assert at == ora.serial - 1, f"step {st.steps} req {rid}: boundary step gpu {at} oracle {ora.serial - 1}"
+                else:
+                    g_dec[rid] = int(g_act[i])
             if stepped:
                 err = np.abs(g_out[:, stepped] - rec.out[:, stepped])
                 st.attn_max_abs = max(st.attn_max_abs, float(err.max()))
@@ -135,24 +148,23 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
                     if np.array_equal(ks, info.K_s) and np.array_equal(kl, info.K_l):
                         assert delta == info.delta, f"Delta gpu {delta} oracle {info.delta}"
                 st.decisions["act"] += 1
-                g_want = int(g_act[i]) in (B.GP_ACT_GROW, B.GP_ACT_COMPRESS_FALLBACK) or \
-                    (int(g_act[i]) == B.GP_ACT_STALLED and info.n_c == 0)
-                if info.n_c > 0 and int(g_act[i]) != B.GP_ACT_STALLED and g_want != info.want_grow:
+                g_want = g_dec[rid] in (B.GP_ACT_GROW, B.GP_ACT_COMPRESS_FALLBACK) or \
+                    (g_dec[rid] == B.GP_ACT_STALLED and info.n_c == 0)
+                if info.n_c > 0 and g_dec[rid] != B.GP_ACT_STALLED and g_want != info.want_grow:
                     assert info.action_near_tie, f"step {st.steps} req {rid}: grow decision differs outside a near-tie"
                     st.near_ties["act"] += 1
                     overrides.setdefault(rid, {})["want_grow"] = g_want
-                g_shrink = int(g_act[i]) == B.GP_ACT_SHRINK
-                if int(g_act[i]) in (B.GP_ACT_COMPRESS, B.GP_ACT_SHRINK) and g_shrink != info.want_shrink:
+                g_shrink = g_dec[rid] == B.GP_ACT_SHRINK
+                if g_dec[rid] in (B.GP_ACT_COMPRESS, B.GP_ACT_SHRINK) and g_shrink != info.want_shrink:
                     assert info.action_near_tie, f"step {st.steps} req {rid}: shrink decision differs outside a near-tie"
                     st.near_ties["act"] += 1
                     overrides.setdefault(rid, {})["want_shrink"] = g_shrink
             # ---- retained sets of the requests the GPU compressed -----------------------------------------------
             for rid, info in rec.boundary.items():
-                i = rids.index(rid)
-                if int(g_act[i]) not in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK, B.GP_ACT_SHRINK):
+                if g_dec[rid] not in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK, B.GP_ACT_SHRINK):
                     continue
                 r = ora.requests[rid]
-                K_t = info.n_c - (2 * b if int(g_act[i]) == B.GP_ACT_SHRINK else b)    # Eq. 13: a Shrink evicts two pages
+                K_t = info.n_c - (2 * b if g_dec[rid] == B.GP_ACT_SHRINK else b)    # Eq. 13: a Shrink evicts two pages
                 for l in range(s.n_layers):
                     for h in range(s.n_kv_heads):
                         st.decisions["sel"] += 1
@@ -176,6 +188,10 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
                 a_g, a_o = int(g_act[i]), int(rec.actions[i])
                 assert a_g == a_o, f"step {st.steps} req {rid}: action gpu {a_g} oracle {a_o}"
                 st.actions[a_g] = st.actions.get(a_g, 0) + 1
+            for rid, info in rec.boundary.items():          # the decisions themselves (asynchronous mode: not in the actions)
+                assert g_dec[rid] == info.action, f"step {st.steps} req {rid}: decision gpu {g_dec[rid]} oracle {info.action}"
+                if is_async:
+                    st.actions[g_dec[rid]] = st.actions.get(g_dec[rid], 0) + 1
             if check_pool_every and (st.steps % check_pool_every == 0 or rec.boundary):
                 for rid in rids:
                     if rid not in ora.requests:

@@ -710,3 +710,70 @@ def test_moved_rows_counts_the_slots_that_change_place_and_whole_copied_pages():
     # both candidate pages shared: every kept slot is written to a fresh page
     info = _compress_with_keep(list(range(4, 20)), 2)
     assert info.cow_pages == 2 and info.moved_tokens == 16 + 16
+
+
+# ----------------------------------------------------------------------------- asynchronous boundary work
+def _run_oracle_job(async_boundary, n_req=3, n_tokens=40, seed=5):
+    """Feeds every request its own fixed token stream; a request that is held keeps its token for the next step.
+    Returns per request the list of (token index, output, retained ids after the step) and the step log."""
+    c = _cfg(n_layers=1, n_pages=40, max_pages_per_req=8, async_boundary=async_boundary, tau=-0.03)
+    rng = np.random.default_rng(seed)
+    pool = O.OraclePool(c)
+    streams = []
+    for r in range(n_req):
+        n0 = 5 + 3 * r
+        kt = rng.standard_normal((1, n0, c.n_kv_heads, c.head_dim))
+        assert pool.request_add(-1, 0, kt, kt + 1.0, n0, 0) == (O.OK, r)
+        streams.append([(rng.standard_normal((1, c.n_q_heads, c.head_dim)), rng.standard_normal((1, c.n_kv_heads, c.head_dim)),
+                         rng.standard_normal((1, c.n_kv_heads, c.head_dim))) for _ in range(n_tokens)])
+    done = [0] * n_req
+    per_token = [[] for _ in range(n_req)]
+    log = []
+    while min(done) < n_tokens:
+        rids = [r for r in range(n_req) if done[r] < n_tokens]
+        q = np.stack([streams[r][done[r]][0] for r in rids], axis=1)
+        k = np.stack([streams[r][done[r]][1] for r in rids], axis=1)
+        v = np.stack([streams[r][done[r]][2] for r in rids], axis=1)
+        before = {r: pool.request_state(r)[:3] for r in rids}
+        rec = pool.decode_step(rids, q, k, v)
+        for i, r in enumerate(rids):
+            a = int(rec.actions[i])
+            log.append((pool.serial - 1, r, a))
+            if a == O.ACT_HELD:
+                assert pool.request_state(r)[2] == before[r][2]            # the position does not move while sitting out
+                continue
+            assert a >= 0
+            per_token[r].append((done[r], rec.out[:, i].copy(), pool.requests[r].pos))
+            done[r] += 1
+        _check_invariants(pool)
+    final = {r: (pool.request_state(r)[:3], [pool.retained(r, 0, h).tolist() for h in range(c.n_kv_heads)],
+                 pool.summaries(r)) for r in range(n_req)}
+    return per_token, log, final, pool
+
+
+def test_sitting_out_changes_when_a_token_is_decoded_not_what_it_sees():
+    sync_tok, sync_log, sync_final, sp = _run_oracle_job(False)
+    asyn_tok, asyn_log, asyn_final, ap = _run_oracle_job(True)
+    # the pool never runs short here, so a request's own history decides everything: token for token the same
+    # outputs, and the same pages, retained tokens and summaries at the end; no token lost or decoded twice
+    for r in range(3):
+        assert [t for t, _, _ in asyn_tok[r]] == list(range(40))
+        for (t1, o1, p1), (t2, o2, p2) in zip(sync_tok[r], asyn_tok[r]):
+            assert t1 == t2 and p1 == p2 and np.array_equal(o1, o2)
+        assert sync_final[r][0] == asyn_final[r][0] and sync_final[r][1] == asyn_final[r][1]
+        assert np.array_equal(sync_final[r][2], asyn_final[r][2])
+    for name in ("grow", "compress", "fallback", "moved_rows", "scored_tokens"):
+        assert sp.counters[name] == ap.counters[name]
+    assert sp.counters["grow"] > 0 and sp.counters["compress"] > 0
+    # every boundary is reported as pending, is followed by exactly one step out, and costs exactly that step
+    pend = [(s, r) for s, r, a in asyn_log if a == O.ACT_PENDING]
+    held = [(s, r) for s, r, a in asyn_log if a == O.ACT_HELD]
+    assert len(pend) > 0 and sorted((s + 1, r) for s, r in pend if (s + 1, r) in held) == sorted(held)
+    assert all(a not in (O.ACT_PENDING, O.ACT_HELD) for _, _, a in sync_log)
+    n_b = {r: sum(1 for _, rr in pend if rr == r) for r in range(3)}
+    last_async = {r: max(s for s, rr, a in asyn_log if rr == r and a != O.ACT_HELD) for r in range(3)}
+    assert all(last_async[r] == 39 + n_b[r] - (1 if (last_async[r], r) in pend else 0) for r in range(3))
+    # the decision is remembered with the step it belongs to
+    for r in range(3):
+        act, at = ap.boundary_outcome(r)
+        assert at == max(s for s, rr in pend if rr == r) and act in (O.ACT_GROW, O.ACT_COMPRESS, O.ACT_COMPRESS_FALLBACK)
