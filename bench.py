@@ -295,7 +295,6 @@ def run_ours(args):
     head = jobs["async"] if head_async else jobs["sync"]
     head.by_layer = by_layer
     B = head.B
-
     # ---- warm-up ------------------------------------------------------------------------------------
     for job in jobs.values():
         for _ in range(Wm):
@@ -442,13 +441,13 @@ def _oracle_run(wl_args, req_lo, req_hi, n_steps, warmup, budget_s):
     wl = W.stack8b_resident(seed=seed) if stack else W.layer8b(seed=seed)
     s = wl.shape
     n_requests = req_hi - req_lo
-    sub = W.Workload(wl.name, wl.seed, s, wl.requests[req_lo:req_hi], n_resident=n_requests,
+    sub = W.Workload(wl.name, wl.seed, s, wl.requests, n_resident=n_requests,
                      initial_pages=wl.initial_pages, max_pages_per_req=wl.max_pages_per_req,
                      n_pages=n_requests * wl.max_pages_per_req, k_loc=wl.k_loc)
     cfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=sub.n_pages,
                          max_pages_per_req=sub.max_pages_per_req, k_loc=sub.k_loc, max_requests=max(4, n_requests))
     pool = O.OraclePool(cfg)
-    sch = H.Scheduler(sub)
+    sch = H.Scheduler(sub, only=range(req_lo, req_hi))
     while True:
         op = sch.next_admission()
         if op is None:
@@ -553,9 +552,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--boundary", default="async", choices=["async", "sync", "both"],
-                    help="async (headline): boundary work beside the next step; sync: inside the step; both: headline sync, "
-                         "async timed beside it")
+    ap.add_argument("--boundary", default="both", choices=["async", "sync", "both"],
+                    help="both (default): headline synchronous, the asynchronous boundary mode timed beside it; sync: synchronous "
+                         "only; async: headline asynchronous (boundary work beside the next step)")
     ap.add_argument("--async-slots", type=int, default=0, help="thread blocks the attention kernel leaves to the boundary kernels")
     ap.add_argument("--entry", default="step", choices=["step", "layers"],
                     help="step: gp_decode_step; layers: the same step through gp_step_begin / gp_attn_layer / gp_step_end")

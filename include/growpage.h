@@ -97,8 +97,8 @@ typedef struct gp_config {
   int32_t async_boundary;    /* 1: asynchronous boundary work (App. "Asynchronous Decoding and Compression"),
                                 see gp_decode_step; default 0                                       */
   int32_t async_slots;       /* asynchronous boundary work: thread blocks of the attention kernel's grid
-                                given up so that the boundary kernels find room on the SMs beside it;
-                                0 = a default (48)                                                    */
+                                given up so that the boundary kernel finds room on the SMs beside it;
+                                0 = a default (64)                                                    */
   int64_t n_pages;           /* physical pages; one page id covers all layers and KV heads         */
   int64_t min_capacity;      /* GP_POLICY_SHRINK: tokens of capacity a Shrink must leave, default 1024 */
   int64_t max_batch_tokens;  /* bound on the summed sequence lengths of one decode batch, used to
@@ -174,23 +174,24 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
  * Asynchronous boundary work (gp_config.async_boundary = 1; App. "Asynchronous Decoding and Compression":
  * requests that compress leave the decode batch, the others keep decoding, the compressed ones rejoin a later
  * batch).  Here the whole boundary chain of a step (demand estimate, decision, page grant or eviction and
- * compaction) leaves the step's critical path: it runs on a stream the pool owns, beside the next step, on
- * SM room the attention kernel leaves free (async_slots).  A request that reaches its boundary at step t
- * reports GP_ACT_PENDING at step t, is skipped at step t + 1 (GP_ACT_HELD if the batch names it: the caller
- * keeps that token's inputs for step t + 2), and decodes again from step t + 2 on, by which time its pages
- * are in their new state; a request whose boundary ended without pages reports GP_ACT_STALLED then.  "Step"
- * counts the pool's decode steps, whatever their batches.  Every token still sees exactly the state the
- * synchronous mode gives it; only the step at which it is decoded moves.  `dev_actions` carries what is
- * known when the step's own work ends (NONE, PENDING, HELD, STALLED, SCRATCH, INVALID); the decisions are
- * read with gp_boundary_outcome.  gp_request_add, gp_release and the introspection calls wait for
- * outstanding boundary work themselves; a caller that touches the pool's pages in any other way, or ends
- * a stream capture, calls gp_async_join first.  The layer-by-layer calls and CUDA-graph capture are not
- * available in this mode (GP_ERR_STATE from gp_step_begin). */
+ * compaction) leaves the step's critical path: one kernel runs it beside the attention kernel of the next
+ * step, on the same stream, on SM room that kernel leaves free (async_slots), and ends with it.  A request that
+ * reaches its boundary at step t reports GP_ACT_PENDING at step t, is skipped at step t + 1 (GP_ACT_HELD if the
+ * batch names it: the caller keeps that token's inputs for step t + 2), and decodes again from step t + 2 on, by
+ * which time its pages are in their new state; a request whose boundary ended without pages reports
+ * GP_ACT_STALLED then.  "Step" counts the pool's decode steps, whatever their batches.  Every token still sees
+ * exactly the state the synchronous mode gives it; only the step at which it is decoded moves.  `dev_actions`
+ * carries what is known when the step's own work ends (NONE, PENDING, HELD, STALLED, SCRATCH, INVALID); the
+ * decisions are read with gp_boundary_outcome.  The boundary chain of the LAST step issued has not been launched
+ * yet: gp_request_add, gp_release and the introspection calls launch it themselves (on the stream of that step);
+ * a caller that looks at the pool's pages in any other way calls gp_async_join first.  Early planning does not
+ * apply, and the layer-by-layer calls are not available in this mode (GP_ERR_STATE from gp_step_begin). */
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
                    const void* q, const void* k, const void* v,
                    void* out, int32_t* dev_actions, void* stream);
 
-/* Asynchronous boundary work: makes `stream` wait for the boundary work of the steps issued so far. */
+/* Asynchronous boundary work: launches the boundary chain of the last decode step on `stream` if it is still
+ * outstanding (it otherwise rides behind the next step's attention kernel); a no-op in the synchronous mode. */
 int gp_async_join(gp_pool* pool, void* stream);
 
 /* The decision taken at the request's most recent capacity boundary (GP_ACT_GROW, GP_ACT_COMPRESS,

@@ -24,8 +24,7 @@
 //   warp 2      merger: combines the four consumers' partial (max, sum, O) of an item and writes the output
 //               or, for requests split over several items, the partial (the next kernel merges those).
 //               Consumers hand over through a double buffer and go straight on to the next item.
-//   warp 1      idle; in the asynchronous boundary mode the first CTA's advances the stepped requests' counters.
-//   warp 3      idle.
+//   warps 1, 3  idle.
 //
 // The two warp groups re-split the register file (setmaxnreg): the service warps keep 56 registers per
 // thread, the consumers, which hold the output accumulators, get 200.
@@ -98,9 +97,7 @@ template <int D, bool ROPE>
 __global__ void __launch_bounds__(NTHREADS, 2)
 gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* __restrict__ q,
                const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, float* __restrict__ out, int lh0,
-               int lh_n, const int* __restrict__ req_ids) {
-  // req_ids: not null only in the asynchronous boundary mode, where this kernel also advances the stepped
-  // requests' counters (in the synchronous mode the decision step does)
+               int lh_n) {
   // lh0, lh_n: the (layer, KV head) units this launch covers, [lh0, lh0 + lh_n): all of them, or one layer's
   using GEO = Geo<D>;
   extern __shared__ uint8_t smem_raw[];
@@ -583,30 +580,6 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       if (lane == 0) mbar_arrive(&slot_empty[sl]);
     }
     cp_async_wait<0>();                  // after an abort copies may still be in flight: let them land
-  } else if (warp == 1) {
-    // ================================= bookkeeping (asynchronous boundary mode) ===============
-    // One more token for every request this step really steps.  The boundary chain of the step before, which
-    // runs beside this kernel, only touches requests that sit this step out, and the next step's plan reads the
-    // counters after this kernel has ended.
-    if (req_ids != nullptr && blockIdx.x == 0) {
-      int stepped = 0;
-      for (int i = lane; i < n_req; i += 32) {
-        if (p.b_flags[i]) {
-          const int r = req_ids[i];
-          p.n[r] = p.b_nold[i] + 1;
-          p.pos[r] += 1;
-          p.started[r] = 1;
-          p.sum_par[r] ^= 1;
-          ++stepped;
-        }
-      }
-#pragma unroll
-      for (int o2 = 16; o2 > 0; o2 >>= 1) stepped += __shfl_xor_sync(0xffffffffu, stepped, o2);
-      if (lane == 0) {
-        atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 5), 1ull);
-        atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 6), (unsigned long long)stepped);
-      }
-    }
   } else if (warp == 2) {
     // ================================= merger =============================================
     for (uint32_t it = 0;; ++it) {
@@ -671,9 +644,8 @@ void gp_attention_setup(const GpDev& p) {           // once per pool: opt into t
 }
 
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n, int serial) {
-  (void)serial;
-  const int* ids = p.async ? req_ids : nullptr;
+                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n) {
+  (void)req_ids;
   const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kk = static_cast<const __nv_bfloat16*>(k);
   const __nv_bfloat16* vv = static_cast<const __nv_bfloat16*>(v);
@@ -682,7 +654,7 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
 #define GP_LAUNCH(DD, RR)                                                                 \
   do {                                                                                    \
     auto kern = gp_attn_kernel<DD, RR>;                                                   \
-    gp_launch(kern, grid, NTHREADS, (size_t)sm, s, pdl, p, n_req, qq, kk, vv, out, lh0, lh_n, ids); \
+    gp_launch(kern, grid, NTHREADS, (size_t)sm, s, pdl, p, n_req, qq, kk, vv, out, lh0, lh_n); \
   } while (0)
   if (p.d == 128) {
     if (rope) GP_LAUNCH(128, true); else GP_LAUNCH(128, false);

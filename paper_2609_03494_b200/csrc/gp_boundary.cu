@@ -436,16 +436,6 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
   // everything the decisions need arrives in one round trip: the jobs summed K^S and K^L per request, a job
   // counted its shared pages, and the plan kernel copied the top of the free list
   const int LH = p.L * p.Hkv;
-  constexpr int RPT = GP_MAX_REQ / SEL_T;                 // stepped requests per thread
-  int fl[RPT], rq[RPT], no[RPT];
-#pragma unroll
-  for (int k = 0; k < RPT; ++k) {
-    const int i = tid + k * SEL_T;
-    const bool on = !p.async && i < n_req;
-    fl[k] = on ? p.b_flags[i] : 0;
-    rq[k] = on ? req_ids[i] : 0;
-    no[k] = on ? p.b_nold[i] : 0;
-  }
   const int n_active = p.hdr[HDR_N_ACTIVE];
   int top0 = 0;
   if (n_bnd > 0) {
@@ -476,25 +466,15 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
         }
       }
       p.delta[r] = delta;
+      // pages and slots as the step left them (full); the allocator below changes what the decision changes.  In
+      // the asynchronous mode the plan of the step in between leaves these two words of a held request alone.
+      p.wP[r] = Pr; p.wn[r] = Pr * GP_PAGE;
       s_want[e] = want; s_ksh[e] = acc.z; s_P[e] = Pr; s_req[e] = r; s_bi[e] = inf.x;
     }
   }
-  // every stepped request: one more token; fire-and-forget updates, nothing here waits for memory
-#pragma unroll
-  for (int k = 0; k < RPT; ++k) {
-    if (fl[k]) {
-      const int r = rq[k];
-      p.n[r] = no[k] + 1;
-      atomicAdd(reinterpret_cast<unsigned long long*>(p.pos + r), 1ull);
-      p.started[r] = 1;
-      atomicXor(p.sum_par + r, 1);                       // the attention kernel wrote the other buffer
-    }
-  }
   if (tid == 0) {
-    if (!p.async) {
-      atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 5), 1ull);
-      atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 6), (unsigned long long)n_active);
-    }
+    atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 5), 1ull);
+    atomicAdd(reinterpret_cast<unsigned long long*>(p.counters + 6), (unsigned long long)n_active);
     p.hdr[HDR_WORK_CMP] = 0;
     if (n_bnd == 0) { p.hdr[HDR_N_CMP] = 0; p.hdr[HDR_N_CITEM] = 0; p.hdr[HDR_N_COW] = 0; }
   }
@@ -523,7 +503,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
         --top;
         p.refcount[page] = 1;
         p.page_table[(size_t)r * p.cap + Pr] = page;
-        p.P[r] = Pr + 1;
+        p.wP[r] = Pr + 1;
         report(bi, r, GP_ACT_GROW);
         s_want[e] |= 2;
         ++grow;
@@ -554,8 +534,8 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       else { report(bi, r, GP_ACT_COMPRESS); ++comp; }
       // a compression frees one page worth of slots; a Shrink frees two and gives the last page back (the
       // compaction kernel returns it once nothing reads it any more)
-      p.n[r] = (s_P[e] - (shrink ? 2 : 1)) * GP_PAGE;
-      if (shrink) p.P[r] = s_P[e] - 1;
+      p.wn[r] = (s_P[e] - (shrink ? 2 : 1)) * GP_PAGE;
+      if (shrink) p.wP[r] = s_P[e] - 1;
       p.n_pristine[r] = 0;
       s_want[e] |= 8;
     }
@@ -838,6 +818,28 @@ struct SelSmem {
 };
 constexpr int SEL_F_CAP = (int)(SelGeom::H_BYTES / sizeof(double));
 
+__device__ __forceinline__ SelSmem sel_smem_at(uint8_t* smem) {      // smem: 256-byte aligned, gp_bsel_smem bytes
+  SelSmem S;
+  S.sbuf = reinterpret_cast<double*>(smem);
+  S.hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::BUF_BYTES);
+  S.hsum = reinterpret_cast<unsigned long long*>(S.hcnt + FB_PAD);           // two u32 planes (low, high)
+  S.wsum = S.hsum + FB_PAD;
+  S.wc = reinterpret_cast<unsigned*>(S.wsum + SEL_NW);
+  S.s_res = reinterpret_cast<long long*>(S.wc + SEL_NW);
+  S.ev = reinterpret_cast<int*>(S.s_res + 8);
+  S.s_i = S.ev + 32;
+  S.red = reinterpret_cast<double*>(S.s_i + 16);
+  S.sM = S.red + SEL_NW * 16;
+  S.sZ = S.sM + 16;
+  S.flist = S.sZ + 16;
+  S.flist_slot = reinterpret_cast<int*>(S.flist + 32);
+  unsigned* coarse = reinterpret_cast<unsigned*>(S.flist_slot + 32);           // [3][CBINS] summary bins
+  S.loc = coarse + 3 * CBINS;
+  S.H.cnt = S.hcnt; S.H.lo = reinterpret_cast<unsigned*>(S.hsum); S.H.hi = S.H.lo + FB_PAD;
+  S.H.ccnt = coarse; S.H.clo = coarse + CBINS; S.H.chi = coarse + 2 * CBINS;
+  return S;
+}
+
 // One selection job of a boundary unit: per-head softmax over the candidate set and the group mean from the
 // attention kernel's per-page partials (`z`, `zs`), then either the working-set size of one view (task 0: K^S,
 // 1: K^L; Eq. 7) or the `ne` slots a compression would evict (task 2; Eq. 9, Eq. 10).  The outputs go to Kout / acc
@@ -903,24 +905,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
                float* __restrict__ out, int serial) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
-  SelSmem S;
-  S.sbuf = reinterpret_cast<double*>(smem);
-  S.hcnt = reinterpret_cast<unsigned*>(smem + SelGeom::BUF_BYTES);
-  S.hsum = reinterpret_cast<unsigned long long*>(S.hcnt + FB_PAD);           // two u32 planes (low, high)
-  S.wsum = S.hsum + FB_PAD;
-  S.wc = reinterpret_cast<unsigned*>(S.wsum + SEL_NW);
-  S.s_res = reinterpret_cast<long long*>(S.wc + SEL_NW);
-  S.ev = reinterpret_cast<int*>(S.s_res + 8);
-  S.s_i = S.ev + 32;
-  S.red = reinterpret_cast<double*>(S.s_i + 16);
-  S.sM = S.red + SEL_NW * 16;
-  S.sZ = S.sM + 16;
-  S.flist = S.sZ + 16;
-  S.flist_slot = reinterpret_cast<int*>(S.flist + 32);
-  unsigned* coarse = reinterpret_cast<unsigned*>(S.flist_slot + 32);           // [3][CBINS] summary bins
-  S.loc = coarse + 3 * CBINS;
-  S.H.cnt = S.hcnt; S.H.lo = reinterpret_cast<unsigned*>(S.hsum); S.H.hi = S.H.lo + FB_PAD;
-  S.H.ccnt = coarse; S.H.clo = coarse + CBINS; S.H.chi = coarse + 2 * CBINS;
+  SelSmem S = sel_smem_at(smem);
   int* s_i = S.s_i;
   // the decision scratch aliases the score staging area: it is used after the last item only
 
@@ -1015,29 +1000,53 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
 // needs a layer's output complete before the next layer's query exists
 __global__ void __launch_bounds__(256)
 gp_merge_kernel(const __grid_constant__ GpDev p, int n_req, float* __restrict__ out, int lh0, int lh_n) {
-  gp_pdl_wait();
+  // the kernel after this one may be scheduled at once: it waits for this grid's end where it needs to, and this
+  // grid ends after the attention kernel (the wait below), so completion stays transitive
   gp_pdl_launch_dependents();
+  gp_pdl_wait();
   merge_partials(p, n_req, out, p.hdr[HDR_N_MC], p.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, lh0, lh_n);
 }
 
 // ------------------------------------------------------------------------------------------------------
 // compaction
 // ------------------------------------------------------------------------------------------------------
+// shared memory of the compaction
+struct CmpSmem {
+  int4* s_info;      // [GP_MAX_REQ + 1] compressing requests: {request, P, boundary index, first chunk}
+  int* ev;           // [2 b]
+  int* s_i;          // [8]
+  int* s_dst;        // [MOVE_TOK] per source slot of the chunk: destination slot (-1: stays or goes)
+  int* s_spage;      // [MOVE_TOK] source page
+  int* s_dpage;      // [MOVE_TOK] destination page
+};
+constexpr size_t CMP_SMEM_BYTES = (GP_MAX_REQ + 1) * 16 + (2 * GP_PAGE + 8 + 3 * MOVE_TOK) * 4;
+__device__ __forceinline__ CmpSmem cmp_smem_at(uint8_t* base) {       // base: 16-byte aligned, CMP_SMEM_BYTES
+  CmpSmem C;
+  C.s_info = reinterpret_cast<int4*>(base);
+  C.ev = reinterpret_cast<int*>(base + (GP_MAX_REQ + 1) * 16);
+  C.s_i = C.ev + 2 * GP_PAGE;
+  C.s_dst = C.s_i + 8;
+  C.s_spage = C.s_dst + MOVE_TOK;
+  C.s_dpage = C.s_spage + MOVE_TOK;
+  return C;
+}
+
+// The compaction of a step, run by every CTA of the calling grid (CT threads): chunks are claimed from the ticket
+// counter until none is left; the last CTA to finish swaps in the copy-on-write targets.
 template <int D, bool SHR>
-__global__ void __launch_bounds__(CT)
-gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int serial) {
+__device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, int serial) {
   constexpr int CH = D / 8;
   constexpr int ROW_BYTES = D * 2;
   constexpr int PIECES = MOVE_TOK * 2 * CH / CT;        // 16-byte pieces per thread per chunk
-  __shared__ int4 s_info[GP_MAX_REQ + 1];     // compressing requests: {request, P, boundary index, first chunk}
-  __shared__ int ev[2 * GP_PAGE];
-  __shared__ int s_i[8];
-  __shared__ int s_dst[MOVE_TOK], s_spage[MOVE_TOK], s_dpage[MOVE_TOK];   // per source slot of the chunk: destination slot (-1: stays or goes), source and destination page
+  int4* s_info = C.s_info;
+  int* ev = C.ev;
+  int* s_i = C.s_i;
+  int* s_dst = C.s_dst;
+  int* s_spage = C.s_spage;
+  int* s_dpage = C.s_dpage;
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int LH = p.L * p.Hkv;
-  gp_pdl_wait();
-  gp_pdl_launch_dependents();
   // the first round trip fetches everything at once: the header, the list of compressing requests (its first
   // CT entries before their count is known; entries past the count are never looked at) and the first ticket
   if (tid == 0) { s_i[0] = atomicAdd(&p.hdr[HDR_WORK_CMP], 1); s_i[3] = 0; }
@@ -1218,6 +1227,116 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
   }
 }
 
+
+template <int D, bool SHR>
+__global__ void __launch_bounds__(CT)
+gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int serial) {
+  __shared__ __align__(16) uint8_t cmp_raw[CMP_SMEM_BYTES];
+  gp_pdl_wait();
+  gp_pdl_launch_dependents();
+  compact_body<D, SHR>(p, cmp_smem_at(cmp_raw), serial);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// asynchronous boundary mode: the whole boundary chain of a step in one kernel, beside the next step's attention
+// ------------------------------------------------------------------------------------------------------
+// Launched right behind the attention kernel of step t + 1 as its programmatic dependent, this grid works on the
+// boundary chain of step t: it does not wait for that attention kernel before it starts (everything it reads
+// was complete before that kernel could start), runs the selection jobs, lets the last CTA to finish them
+// decide and allocate, waits inside the grid for that (a bounded wait on a flag: the grid is sized to be
+// resident at once, on the room the attention kernel leaves), compacts, and only then waits for the attention
+// kernel to end; after that it merges the split requests' partial outputs of step t + 1.  The grid therefore
+// ends after both, and the plan of step t + 2, its programmatic dependent, finds the pages and counters of the
+// requests that sat step t + 1 out in their final state.  `p`: the view of step t (its scratch set, the copy of
+// the counters its decisions go to); `pa`: the view of step t + 1 (for the merge).
+template <int D, bool SHR>
+__global__ void __launch_bounds__(SEL_T, 2)
+gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev pa, int n_req_merge, float* __restrict__ out_merge,
+                int serial, int has_chain) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
+  const int tid = threadIdx.x;
+  const int LH = p.L * p.Hkv;
+  gp_pdl_launch_dependents();
+  if (has_chain) {
+    SelSmem S = sel_smem_at(smem);
+    int* s_i = S.s_i;
+    const int G = p.G, G2 = 2 * p.G;
+    constexpr int NT = SHR ? 4 : 3;
+    const int n_bnd = __ldcg(p.hdr + HDR_N_BND);
+    const long long items = (long long)n_bnd * LH * NT;
+    for (long long item = blockIdx.x; item < items + n_bnd; item += gridDim.x) {
+      if (item >= items) {
+        const int e = (int)(item - items);
+        if (tid < 32) {
+          const int4 inf = p.bnd_info[2 * e];
+          const int* table = p.page_table + (size_t)inf.y * p.cap;
+          int ksh = 0;
+          for (int j = tid; j < inf.z - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
+#pragma unroll
+          for (int o2 = 16; o2 > 0; o2 >>= 1) ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
+          if (tid == 0) p.bnd_acc[4 * e + 2] = ksh;
+        }
+        continue;
+      }
+      const long long u = item / NT;
+      const int job = (int)(item % NT);
+      const int task = job < 2 ? job : 2;
+      const int ne = (SHR && job == 3) ? 2 * GP_PAGE : GP_PAGE;
+      const int bidx = (int)(u / LH), lh = (int)(u % LH);
+      const int l = lh / p.Hkv, h = lh % p.Hkv;
+      const int4 inf = p.bnd_info[2 * bidx];
+      const int4 inf2 = p.bnd_info[2 * bidx + 1];
+      const int r = inf.y, Pr = inf.z;
+      const long long off = (long long)(unsigned)inf2.x | ((long long)inf2.y << 32);
+      const int nC = (Pr - 1) * GP_PAGE;
+      int* Kout = p.Kx + (((size_t)r * p.L + l) * p.Hkv + h) * 2;
+      int* evout = (SHR && job == 3) ? p.evict2 + (size_t)u * 2 * GP_PAGE : p.evict + (size_t)u * GP_PAGE;
+      __syncthreads();
+      if (nC == 0) {
+        if (tid == 0 && task < 2) Kout[task] = 0;
+        continue;
+      }
+      if (SHR && job == 3 && Pr - 1 < p.min_pages_after_shrink) continue;
+      const size_t view_stride = (size_t)p.z_stride * G;
+      const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;
+      const double* zs = p.zstat + ((size_t)lh * (p.max_boundary_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
+      double* a = nC <= SEL_CAP ? S.sbuf : p.scores + ((size_t)job * LH + lh) * p.max_boundary_tokens + off;
+      sel_job(p, S, z, view_stride, zs, a, nC, task, ne, Kout, p.bnd_acc + 4 * bidx, evout);
+    }
+    // ---- the last CTA to finish its jobs takes the decisions and tells the others ------------------------------
+    const int stamp = serial + 1;
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      const int prev = atomicAdd(&p.hdr[HDR_DONE_SEL], 1);
+      s_i[2] = (prev == (int)gridDim.x - 1);
+      if (prev == (int)gridDim.x - 1) p.hdr[HDR_DONE_SEL] = 0;
+    }
+    __syncthreads();
+    if (s_i[2]) {
+      __threadfence();
+      decide_and_allocate(p, nullptr, 0, n_bnd, nullptr, reinterpret_cast<int*>(S.sbuf), serial);
+      __syncthreads();
+      if (tid == 0) {
+        __threadfence();
+        *reinterpret_cast<volatile int*>(p.hdr + HDR_DECIDED) = stamp;
+      }
+    } else if (tid == 0) {
+      volatile int* flag = reinterpret_cast<volatile int*>(p.hdr + HDR_DECIDED);
+      unsigned it = 0;
+      while (*flag != stamp && it < GP_SPIN_LIMIT) { ++it; __nanosleep(100); }
+      if (it >= GP_SPIN_LIMIT) atomicOr(p.err, GP_E_SPIN_CMP);
+      __threadfence();
+    }
+    __syncthreads();
+    // ---- compaction: its arrays take the place of the selection's -----------------------------------------------
+    compact_body<D, SHR>(p, cmp_smem_at(smem), serial);
+  }
+  gp_pdl_wait();              // the attention kernel beside which this grid ran has ended
+  if (out_merge) merge_partials(pa, n_req_merge, out_merge, pa.hdr[HDR_N_MC], pa.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, 0, LH);
+}
+
 }  // namespace
 
 // the compaction kernel of a pool: head dimension, and whether the Shrink policy is on
@@ -1247,6 +1366,20 @@ void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_com
   occ = 0;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, compact_kernel_of(p), CT, 0);
   *grid_compact = num_sms * (occ > 0 ? occ : 1);
+}
+
+// asynchronous mode: the boundary chain of the step whose view is `p` (none when !has_chain), and afterwards the
+// merge of the split requests' partial outputs of the step whose view is `pa` (none when out_merge is null)
+void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* out_merge, int serial, int has_chain, int grid,
+                     cudaStream_t s, bool pdl) {
+  const size_t sm = gp_bsel_smem(p);
+  const bool shr = p.policy == GP_POLICY_SHRINK;
+  auto launch = [&](auto kern) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    gp_launch(kern, grid, SEL_T, sm, s, pdl, p, pa, n_req_merge, out_merge, serial, has_chain);
+  };
+  if (p.d == 128) { if (shr) launch(gp_chain_kernel<128, true>); else launch(gp_chain_kernel<128, false>); }
+  else { if (shr) launch(gp_chain_kernel<64, true>); else launch(gp_chain_kernel<64, false>); }
 }
 
 void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl) {

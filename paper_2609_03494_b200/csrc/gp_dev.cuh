@@ -29,7 +29,7 @@ enum {
   HDR_N_RC = 0,      // (request, chunk) work items of this step
   HDR_N_BND,         // requests at a capacity boundary
   HDR_N_CMP,         // requests that compress
-  HDR_SPARE0,        // unused
+  HDR_DECIDED,       // asynchronous mode: stamped by the CTA that took the step's decisions
   HDR_DONE_CMP,      // CTAs of the compaction kernel that have finished
   HDR_STEP,          // step serial number
   HDR_N_ACTIVE,      // requests actually stepped
@@ -72,7 +72,13 @@ struct GpDev {
   int* page_table;
   int* shadow;
   // per request
+  // Pages, occupied slots, "has decoded", summary buffer in use and position of every request exist twice: a
+  // decode step reads one copy (P, n, started, sum_par, pos) and its plan writes the other (wP, ...), every
+  // slot carried over and the stepped ones advanced by one token, for the step after it; the decision step
+  // writes the pages and slots of the requests at a boundary into the copy their next step reads.  So the plan
+  // of a step may run while the step before it still executes.  The host sets the two views per launch.
   int* P; int* n; int* started; int* live; int* n_pristine; long long* pos;
+  int* wP; int* wn; int* wstarted; int* wsum_par; long long* wpos;
   int* bstep;                            // [M] number of the decode step at which the request last reached its boundary
   int* last_act;                         // [M] decision taken at that boundary (GP_ACT_*)
   double* summ;
@@ -85,9 +91,6 @@ struct GpDev {
                                          //   6 n before the append, 7 position, 8 flags (1 boundary, 2 started),
                                          //   9 P, 10-11 offset into the logit scratch, 12 summary buffer in use,
                                          //   13 index of its partial-output slot
-  int* b_nold;                           // [M] occupied slots before the append, by batch index
-  int* b_flags;                          // [M] 1 = stepped this step
-  int* first_idx;                        // [M] lowest batch index naming a request
   int4* mc_list;                         // [M] split requests: {batch index, first partial, chunks, 0}
   int4* bnd_info;                        // [M][2] requests at a boundary: {slot in the batch, request, P, position of the step's token}, {score offset lo, hi, 0, 0}
   int* bnd_acc;                          // [M][4] per boundary request: sum of K^S, sum of K^L, shared pages of C, 0
@@ -219,7 +222,7 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 
 // ---- host-visible launchers (one per translation unit) -------------------------------------------
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n, int serial);
+                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n);
 size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
 // ---- programmatic dependent launch -------------------------------------------------------------------
@@ -247,6 +250,8 @@ inline cudaError_t gp_launch(void (*kern)(KArgs...), int grid, int block, size_t
 #endif
 
 void gp_attention_setup(const GpDev& p);
+void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* out_merge, int serial, int has_chain, int grid,
+                     cudaStream_t s, bool pdl);
 // merge of the split requests' partial outputs for the units [lh0, lh0 + lh_n) (per-layer entry point)
 void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl);
 void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact);

@@ -19,13 +19,14 @@ struct gp_pool {
   int device;
   GpDev dev;
   // asynchronous boundary mode: steps alternate between two sets of the scratch that a step's boundary chain
-  // still reads while the next step runs (dev, dev_alt); the chain runs on `side`
+  // still reads while the next step runs (dev, dev_alt); the chain of a step is launched behind the attention
+  // kernel of the next step (or by whatever call needs the pool's pages settled first)
   GpDev dev_alt;
-  cudaStream_t side;
-  cudaEvent_t e_attn[2], e_chain[2];
-  int chain_pending[2];
-  int attn_grid_async, sel_grid_async, compact_grid_async;
+  int chain_pending;                                // the last step's boundary chain has not been launched yet
+  int attn_grid_async, chain_grid;
   long long serial;                                 // decode steps issued so far
+  // the two copies of the requests' counters (see GpDev): step t reads copy t mod 2
+  int* sP[2]; int* sn[2]; int* sstarted[2]; int* spar[2]; long long* spos[2];
   void* blob;
   size_t bytes;
   std::vector<uint8_t> live;      // host mirror of the slot free list
@@ -42,10 +43,10 @@ struct gp_pool {
   uint8_t* dbg;                   // gather target of the debug getters
   // measurement
   int profiling;
+  cudaStream_t last_stream;       // stream of the last decode step
   int early_plan;                 // gp_set_early_plan: the plan kernel reads the caller's inputs before its wait
   int first_plain;                // the step's first kernel follows a kernel of another kind: plain launch
   cudaEvent_t ev[GP_N_KERNELS + 1];
-  cudaEvent_t ev_side[3];                           // asynchronous mode: around the two kernels on `side`
   float ms[GP_N_KERNELS];
   int64_t launches[GP_N_KERNELS];
   int64_t launch_count;
@@ -55,9 +56,9 @@ struct gp_pool {
 namespace {
 
 struct Layout {
-  size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc, b_nold,
-      b_flags, mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
-      bnd_info2, bnd_acc2, zbuf2, zstat2,
+  size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc,
+      mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
+      bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
       evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, total;
   int max_rc;
@@ -124,15 +125,12 @@ Layout make_layout(const gp_config& c) {
   L.words = take(256 * 4);                       // free_top, err, plan header, status
   L.page_table = take(M * cap * 4);
   L.shadow = take(M * cap * 4);
-  L.reqi = take(7 * M * 4);                      // P, n, started, live, n_pristine, bstep, last_act
-  L.sum_par = take(M * 4);
-  L.pos = take(M * 8);
+  L.reqi = take(12 * M * 4);                     // two copies of P, n, started, sum_par; live, n_pristine, bstep, last_act
+  L.pos = take(2 * M * 8);                       // two copies
   L.summ = take((size_t)c.n_layers * M * 2 * 2 * c.n_q_heads * d * 8);
   L.Kx = take(M * LH * 2 * 4);
   L.delta = take(M * 8);
   L.rc = take((size_t)L.max_rc * GP_DESC_INTS * 4);
-  L.b_nold = take(M * 4);
-  L.b_flags = take(M * 4);
   L.mc_list = take(M * 16);
   L.bnd_info = take(M * 32);
   L.bnd_acc = take(M * 16);
@@ -152,8 +150,13 @@ Layout make_layout(const gp_config& c) {
     L.bnd_acc2 = take(M * 16);
     L.zbuf2 = take(LH * (Tb + b) * 2 * G * 8);
     L.zstat2 = take(LH * (Tb / b + 1) * 2 * G * 2 * 8);
+    // and of what the plan of a step writes while the attention kernel of the step before may still read its own
+    L.rc2 = take((size_t)L.max_rc * GP_DESC_INTS * 4);
+    L.mc_list2 = take(M * 16);
+    L.qtil2 = take(M * LH * 2 * (size_t)G * d * 8);
+    L.rope_cs2 = take(M * (d / 2) * 2 * 8);
   } else {
-    L.bnd_info2 = L.bnd_acc2 = L.zbuf2 = L.zstat2 = 0;
+    L.bnd_info2 = L.bnd_acc2 = L.zbuf2 = L.zstat2 = L.rc2 = L.mc_list2 = L.qtil2 = L.rope_cs2 = 0;
   }
   L.counters = take(16 * 8);
   L.dbg = take(cap * b * (4 + 2 * d * 2));
@@ -310,6 +313,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __shared__ int s_req[GP_MAX_REQ], s_state[GP_MAX_REQ];     // summary CTAs: request of a batch slot, flags
   __shared__ long long s_pos64[GP_MAX_REQ];
   __shared__ int s_bin[GP_COST_BINS], s_binbase[GP_COST_BINS], s_nmc;
+  __shared__ unsigned char s_adv[GP_MAX_REQ];     // slots this step really steps
   const int i = threadIdx.x;
   const bool in = i < n_req;
   // What runs before the wait for the kernel before this one.  In a whole-step launch that kernel is the
@@ -367,8 +371,17 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   }
   if (!plan_on) return;
   s_first[i] = 0x7fffffff;
+  s_adv[i] = 0;
   if (i < GP_COST_BINS) s_bin[i] = 0;
   if (i == 0) s_nmc = 0;
+  // this thread's slot (thread i looks after batch position i and, for the carry at the end, after slot i)
+  int c_n = 0, c_P = 0, c_st = 0, c_par = 0, c_held = 0;
+  long long c_pos = 0;
+  if (i < p.M) {
+    c_n = __ldcg(p.n + i); c_P = __ldcg(p.P + i); c_st = __ldcg(p.started + i); c_par = __ldcg(p.sum_par + i);
+    c_pos = __ldcg(p.pos + i);
+    if (p.async) c_held = __ldcg(p.bstep + i) == serial - 1;
+  }
   __syncthreads();
   int r = -1;
   if (in) {
@@ -453,8 +466,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const int sorted0 = s_binbase[key] + within;
   s_chunks[i] = chunks; s_pos[i] = (int)pos;
   if (in) {
-    p.b_nold[i] = n_old;
-    p.b_flags[i] = chunks > 0;
+    if (chunks > 0) s_adv[r] = 1;
     if (isb) { p.bstep[r] = serial; if (p.async) act = GP_ACT_PENDING; }
     actions[i] = act;
     if (isb) {
@@ -473,6 +485,17 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       d[3] = make_int4(par, rc_off + c, 0, 0);
     }
     if (chunks > 1) p.mc_list[atomicAdd(&s_nmc, 1)] = make_int4(i, rc_off, chunks, 0);
+  }
+  __syncthreads();
+  // The next step's copy of the requests' counters: every slot carried over, the stepped ones one token further
+  // (the summary buffers swap: this step's summary CTAs write the buffer not in use).  Pages and slots of a
+  // request that sits this step out belong to the boundary chain that is still running.
+  if (i < p.M) {
+    const int adv = s_adv[i];
+    if (!c_held) { p.wn[i] = c_n + adv; p.wP[i] = c_P; }
+    p.wpos[i] = c_pos + adv;
+    p.wstarted[i] = c_st | adv;
+    p.wsum_par[i] = c_par ^ adv;
   }
   if (p.rope_theta != 0.0) {                                      // cos / sin of the step's position
     __syncthreads();
@@ -568,9 +591,12 @@ __global__ void gp_ingest_kernel(GpDev p, int r, int n_shared, int n_tail, const
   }
 }
 
-__global__ void gp_release_kernel(GpDev p, int r) {
+__global__ void gp_release_kernel(GpDev p, int r, int serial) {
   const int lane = threadIdx.x;
-  const int Pr = p.P[r];
+  // a request that reached its boundary at the last step (asynchronous mode) has its page count where that
+  // step's boundary chain put it: in the other copy
+  const bool other = p.async && p.bstep[r] == serial - 1;
+  const int Pr = other ? p.wP[r] : p.P[r];
   const int* table = p.page_table + (size_t)r * p.cap;
   for (int j0 = 0; j0 < Pr; j0 += 32) {
     const int j = j0 + lane;
@@ -589,7 +615,10 @@ __global__ void gp_release_kernel(GpDev p, int r) {
     if (lane == 0 && mask) *reinterpret_cast<volatile int*>(p.free_top) = base + __popc(mask);
     __syncwarp();
   }
-  if (lane == 0) { p.live[r] = 0; p.P[r] = 0; p.n[r] = 0; p.started[r] = 0; p.n_pristine[r] = 0; }
+  if (lane == 0) {
+    p.live[r] = 0; p.P[r] = 0; p.n[r] = 0; p.started[r] = 0; p.n_pristine[r] = 0;
+    p.wP[r] = 0; p.wn[r] = 0; p.wstarted[r] = 0; p.bstep[r] = GP_NEVER;
+  }
 }
 
 // debug: token ids and un-swizzled K, V rows of one (layer, head) stream into the gather buffer
@@ -618,21 +647,45 @@ __global__ void gp_gather_kernel(GpDev p, int r, int l, int h, int n, int* tok_o
 
 void pool_free(gp_pool* pool) {
   if (pool->h_err) cudaFreeHost(pool->h_err);
-  for (int i = 0; i < 2; ++i) {
-    if (pool->e_attn[i]) cudaEventDestroy(pool->e_attn[i]);
-    if (pool->e_chain[i]) cudaEventDestroy(pool->e_chain[i]);
-  }
-  for (int i = 0; i < 3; ++i)
-    if (pool->ev_side[i]) cudaEventDestroy(pool->ev_side[i]);
-  if (pool->side) cudaStreamDestroy(pool->side);
   delete pool;
 }
 
-// asynchronous boundary mode: `s` waits for the boundary chains issued so far
-int join_side(gp_pool* pool, cudaStream_t s) {
-  for (int i = 0; i < 2; ++i)
-    if (pool->chain_pending[i] && cudaStreamWaitEvent(s, pool->e_chain[i], 0) != cudaSuccess) return GP_ERR_CUDA;
+// the device view with the requests' counters read from copy `rd` and written to copy `wr`
+GpDev with_state(const gp_pool* pool, const GpDev& d, int rd, int wr) {
+  GpDev v = d;
+  v.P = pool->sP[rd]; v.n = pool->sn[rd]; v.started = pool->sstarted[rd]; v.sum_par = pool->spar[rd]; v.pos = pool->spos[rd];
+  v.wP = pool->sP[wr]; v.wn = pool->sn[wr]; v.wstarted = pool->sstarted[wr]; v.wsum_par = pool->spar[wr]; v.wpos = pool->spos[wr];
+  return v;
+}
+// the copy that holds the requests' counters as of now (what the next step will read)
+int cur_copy(const gp_pool* pool) { return (int)(pool->serial & 1); }
+GpDev cur_view(const gp_pool* pool) { return with_state(pool, pool->dev, cur_copy(pool), cur_copy(pool)); }
+
+// The copy that holds a request's pages and slots as of now.  With asynchronous boundary work a request that
+// reached its boundary at the last step sits the next one out, and its boundary chain wrote to the copy that
+// the step after that reads.  Call after a device-wide synchronisation.
+int pages_copy(const gp_pool* pool, int req, int* out) {
+  *out = cur_copy(pool);
+  if (pool->cfg.async_boundary) {
+    int b = 0;
+    if (cudaMemcpy(&b, pool->dev.bstep + req, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return GP_ERR_CUDA;
+    if (b == (int)((pool->serial - 1) & 0x3fffffff)) *out ^= 1;
+  }
   return GP_OK;
+}
+
+// Asynchronous boundary mode: launches the boundary chain of the last decode step on `s` if it has not been
+// launched yet (it normally rides behind the next step's attention kernel).  Everything that looks at the pool's
+// pages, counters or free list from outside a decode step calls this first.
+int flush_chain(gp_pool* pool, cudaStream_t s) {
+  if (!pool->cfg.async_boundary || !pool->chain_pending) return GP_OK;
+  const long long t = pool->serial - 1;                       // the step the chain belongs to
+  const GpDev& d = (t & 1) ? pool->dev_alt : pool->dev;
+  const int wr = (int)(t & 1);                                  // the copy the step after the next reads
+  gp_launch_chain(with_state(pool, d, wr, wr), d, 0, nullptr, (int)(t & 0x3fffffff), 1, pool->chain_grid, s, false);
+  pool->chain_pending = 0;
+  pool->launch_count += 1;
+  return cudaGetLastError() == cudaSuccess ? GP_OK : GP_ERR_CUDA;
 }
 
 // the kernels' error bits, once the work that could set them has completed
@@ -751,15 +804,18 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.shadow = reinterpret_cast<int*>(base + L.shadow);
   int* reqi = reinterpret_cast<int*>(base + L.reqi);
   const int M = cfg->max_requests;
-  d.P = reqi; d.n = reqi + M; d.started = reqi + 2 * M; d.live = reqi + 3 * M; d.n_pristine = reqi + 4 * M;
-  d.bstep = reqi + 5 * M; d.last_act = reqi + 6 * M;
-  d.pos = reinterpret_cast<long long*>(base + L.pos);
+  for (int c = 0; c < 2; ++c) {
+    pool->sP[c] = reqi + (4 * c) * M; pool->sn[c] = reqi + (4 * c + 1) * M; pool->sstarted[c] = reqi + (4 * c + 2) * M;
+    pool->spar[c] = reqi + (4 * c + 3) * M;
+    pool->spos[c] = reinterpret_cast<long long*>(base + L.pos) + (size_t)c * M;
+  }
+  d.live = reqi + 8 * M; d.n_pristine = reqi + 9 * M; d.bstep = reqi + 10 * M; d.last_act = reqi + 11 * M;
+  d.P = d.wP = pool->sP[0]; d.n = d.wn = pool->sn[0]; d.started = d.wstarted = pool->sstarted[0];
+  d.sum_par = d.wsum_par = pool->spar[0]; d.pos = d.wpos = pool->spos[0];
   d.summ = reinterpret_cast<double*>(base + L.summ);
   d.Kx = reinterpret_cast<int*>(base + L.Kx);
   d.delta = reinterpret_cast<double*>(base + L.delta);
   d.rcx = reinterpret_cast<int*>(base + L.rc);
-  d.b_nold = reinterpret_cast<int*>(base + L.b_nold);
-  d.b_flags = reinterpret_cast<int*>(base + L.b_flags);
   d.mc_list = reinterpret_cast<int4*>(base + L.mc_list);
   d.bnd_info = reinterpret_cast<int4*>(base + L.bnd_info);
   d.bnd_acc = reinterpret_cast<int*>(base + L.bnd_acc);
@@ -768,7 +824,6 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.zbuf = reinterpret_cast<double*>(base + L.zbuf);
   d.qtil = reinterpret_cast<double*>(base + L.qtil);
   d.zstat = reinterpret_cast<double*>(base + L.zstat);
-  d.sum_par = reinterpret_cast<int*>(base + L.sum_par);
   d.evict = reinterpret_cast<int*>(base + L.evict);
   d.evict2 = reinterpret_cast<int*>(base + L.evict2);
   d.cflags = reinterpret_cast<int*>(base + L.cflags);
@@ -779,8 +834,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   gp_attention_setup(d);
   gp_boundary_setup(d, pool->num_sms, &pool->sel_grid, &pool->compact_grid);
   pool->dev_alt = d;
-  pool->side = nullptr;
-  pool->chain_pending[0] = pool->chain_pending[1] = 0;
+  pool->chain_pending = 0;
+  pool->last_stream = nullptr;
   if (cfg->async_boundary) {
     GpDev& a = pool->dev_alt;
     a.hdr = words + 128;
@@ -788,21 +843,15 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
     a.bnd_acc = reinterpret_cast<int*>(base + L.bnd_acc2);
     a.zbuf = reinterpret_cast<double*>(base + L.zbuf2);
     a.zstat = reinterpret_cast<double*>(base + L.zstat2);
-    // the boundary kernels run beside the attention kernel on the room it leaves: `slots` of its thread blocks
-    int slots = cfg->async_slots > 0 ? cfg->async_slots : 48;
+    a.rcx = reinterpret_cast<int*>(base + L.rc2);
+    a.mc_list = reinterpret_cast<int4*>(base + L.mc_list2);
+    a.qtil = reinterpret_cast<double*>(base + L.qtil2);
+    a.rope_cs = reinterpret_cast<double*>(base + L.rope_cs2);
+    // the chain kernel runs beside the attention kernel on the room it leaves: `slots` of its thread blocks
+    int slots = cfg->async_slots > 0 ? cfg->async_slots : 64;
     if (slots > pool->attn_grid / 2) slots = pool->attn_grid / 2;
     pool->attn_grid_async = pool->attn_grid - slots;
-    pool->sel_grid_async = slots < pool->sel_grid ? slots : pool->sel_grid;
-    pool->compact_grid_async = 2 * slots < pool->compact_grid ? 2 * slots : pool->compact_grid;
-    int lo = 0, hi = 0;
-    cudaDeviceGetStreamPriorityRange(&lo, &hi);                 // hi = the numerically lowest = most urgent
-    if (cudaStreamCreateWithPriority(&pool->side, cudaStreamNonBlocking, hi) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
-    for (int i = 0; i < 2; ++i) {
-      if (cudaEventCreateWithFlags(&pool->e_attn[i], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&pool->e_chain[i], cudaEventDisableTiming) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
-    }
-    for (int i = 0; i < 3; ++i)
-      if (cudaEventCreate(&pool->ev_side[i]) != cudaSuccess) { pool_free(pool); return GP_ERR_CUDA; }
+    pool->chain_grid = slots;
   }
   pool->dbg = base + L.dbg;
   if (cfg->host_staging) {
@@ -855,8 +904,8 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   if (P > c.max_pages_per_req) P = (long long)c.max_pages_per_req + 1;      // still refused, and fits an int
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (join_side(pool, s) != GP_OK) return GP_ERR_CUDA;        // the free list belongs to the boundary chains in flight
-  gp_admit_kernel<<<1, 32, 0, s>>>(pool->dev, slot, share_from, n_shared_pages, n_tail, (int)P, pool->d_status);
+  if (flush_chain(pool, s) != GP_OK) return GP_ERR_CUDA;       // the free list belongs to the last step's boundary chain first
+  gp_admit_kernel<<<1, 32, 0, s>>>(cur_view(pool), slot, share_from, n_shared_pages, n_tail, (int)P, pool->d_status);
   pool->launch_count++;
   int st = GP_ERR_CUDA;
   GP_CUDA(cudaMemcpyAsync(&st, pool->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -881,7 +930,8 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
 static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_t* actions, const void* q, int plan_on,
                         int lh0, int lh_n, cudaStream_t s, bool pdl, bool by_layer = false, const GpDev* dev = nullptr,
                         int attn_grid = 0) {
-  const GpDev& d = dev ? *dev : pool->dev;
+  const int rd = cur_copy(pool);
+  const GpDev d = with_state(pool, dev ? *dev : pool->dev, rd, rd ^ 1);     // the plan writes the next step's copy
   const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
   const long long want = ((long long)n_req * lh_n + upc - 1) / upc;
   const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
@@ -913,62 +963,47 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
     // fetch of the inputs): no programmatic dependence on it
     launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl && !pool->first_plain);
     if (prof) cudaEventRecord(pool->ev[1], s);
-    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH, serial);
+    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH);
     if (prof) cudaEventRecord(pool->ev[2], s);
-    gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s,
-                       prof ? pool->ev[3] : nullptr, pdl, serial);
+    // the decisions change pages and slots in the copy the next step reads
+    gp_launch_boundary(with_state(pool, d, cur_copy(pool), cur_copy(pool) ^ 1), dev_req_ids, n_req, dev_actions,
+                       static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s, prof ? pool->ev[3] : nullptr, pdl, serial);
     if (prof) cudaEventRecord(pool->ev[4], s);
     pool->launch_count += GP_N_KERNELS;
   } else {
-    // Asynchronous boundary work.  On the caller's stream: plan, attention, merge of the split requests' partial
-    // outputs (the step's `out` is complete when the stream gets there).  On the pool's stream, after the
-    // attention kernel: working sets + decisions, compaction.  Step t uses scratch set t mod 2 and first waits
-    // for the chain of step t - 2, which read that set; the same wait, one step later, puts the chain of step
-    // t - 1 before the plan of step t + 1, the first to look at the requests that chain changes (they sit
-    // step t out).
+    // Asynchronous boundary work, all on the caller's stream: plan and attention of this step, then one kernel
+    // with the boundary chain of the step before (working sets, decisions, compaction), which runs beside the
+    // attention kernel, ends after it and then merges this step's split outputs.  Step t uses scratch set t mod 2.
     const int par = (int)(pool->serial & 1);
     const GpDev& d = par ? pool->dev_alt : pool->dev;
+    const GpDev& dprev = par ? pool->dev : pool->dev_alt;
     const int LH = d.L * d.Hkv;
-    if (pool->chain_pending[par]) GP_CUDA(cudaStreamWaitEvent(s, pool->e_chain[par], 0));
-    // the chain of the step before this one changes the pages and counters of requests this step skips, and
-    // the free list, which this step's own chain reads after it (same stream): nothing to wait for here
     if (prof) cudaEventRecord(pool->ev[0], s);
+    // no early planning here: the plan reads the pages and slots of the requests that return from their step out,
+    // which the chain kernel of the step before (the kernel before this one on the stream) has just written
     launch_plan(pool, dev_req_ids, n_req, dev_actions, q, 1, 0, LH, s, pdl && !pool->first_plain, false, &d, pool->attn_grid_async);
     if (prof) cudaEventRecord(pool->ev[1], s);
-    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid_async, s, pdl, 0, LH, serial);
+    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid_async, s, pdl, 0, LH);
     if (prof) cudaEventRecord(pool->ev[2], s);
-    gp_launch_merge(d, n_req, static_cast<float*>(out), 0, LH, pool->num_sms, s, pdl);
-    GP_CUDA(cudaEventRecord(pool->e_attn[par], s));
-    GP_CUDA(cudaStreamWaitEvent(pool->side, pool->e_attn[par], 0));
-    if (prof) cudaEventRecord(pool->ev_side[0], pool->side);
-    gp_launch_boundary(d, dev_req_ids, n_req, nullptr, nullptr, pool->sel_grid_async, pool->compact_grid_async, pool->side,
-                       prof ? pool->ev_side[1] : nullptr, true, serial);
-    if (prof) cudaEventRecord(pool->ev_side[2], pool->side);
-    GP_CUDA(cudaEventRecord(pool->e_chain[par], pool->side));
-    pool->chain_pending[par] = 1;
-    pool->launch_count += GP_N_KERNELS + 1;
+    // the decisions of the step before change pages and slots in the copy the next step reads (the one that step
+    // itself read: the plan of this step carries every other word over and leaves these to the chain)
+    const int wr = par ^ 1;
+    gp_launch_chain(with_state(pool, dprev, wr, wr), d, n_req, static_cast<float*>(out), (int)((pool->serial - 1) & 0x3fffffff),
+                    pool->chain_pending, pool->chain_grid, s, pdl);
+    if (prof) { cudaEventRecord(pool->ev[3], s); cudaEventRecord(pool->ev[4], s); }
+    pool->chain_pending = 1;
+    pool->last_stream = s;
+    pool->launch_count += 3;
   }
   pool->serial += 1;
   GP_CUDA(cudaGetLastError());
   if (prof) {
-    if (!pool->cfg.async_boundary) {
-      GP_CUDA(cudaEventSynchronize(pool->ev[GP_N_KERNELS]));
-      for (int i = 0; i < GP_N_KERNELS; ++i) {
-        float t = 0.f;
-        GP_CUDA(cudaEventElapsedTime(&t, pool->ev[i], pool->ev[i + 1]));
-        pool->ms[i] += t;
-        pool->launches[i] += 1;
-      }
-    } else {
-      GP_CUDA(cudaEventSynchronize(pool->ev[2]));
-      GP_CUDA(cudaEventSynchronize(pool->ev_side[2]));
-      for (int i = 0; i < GP_N_KERNELS; ++i) {
-        float t = 0.f;
-        if (i < 2) GP_CUDA(cudaEventElapsedTime(&t, pool->ev[i], pool->ev[i + 1]));
-        else GP_CUDA(cudaEventElapsedTime(&t, pool->ev_side[i - 2], pool->ev_side[i - 1]));
-        pool->ms[i] += t;
-        pool->launches[i] += 1;
-      }
+    GP_CUDA(cudaEventSynchronize(pool->ev[GP_N_KERNELS]));
+    for (int i = 0; i < GP_N_KERNELS; ++i) {
+      float t = 0.f;
+      GP_CUDA(cudaEventElapsedTime(&t, pool->ev[i], pool->ev[i + 1]));
+      pool->ms[i] += t;
+      pool->launches[i] += 1;
     }
   }
   return GP_OK;
@@ -978,13 +1013,14 @@ int gp_async_join(gp_pool* pool, void* stream) {
   if (!pool) return GP_ERR_INVALID;
   if (!pool->cfg.async_boundary) return GP_OK;
   GP_CUDA(cudaSetDevice(pool->device));
-  return join_side(pool, static_cast<cudaStream_t>(stream));
+  return flush_chain(pool, static_cast<cudaStream_t>(stream));
 }
 
 int gp_boundary_outcome(gp_pool* pool, int32_t req, int32_t* action, int64_t* step) {
   const int st = check_req(pool, req);
   if (st != GP_OK) return st;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   int a = 0, b = 0;
   GP_CUDA(cudaMemcpy(&a, pool->dev.last_act + req, 4, cudaMemcpyDeviceToHost));
@@ -1032,7 +1068,7 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
   float* ob = reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(out) - qs * 4);
   const int lh0 = layer * d.Hkv, lh_n = d.Hkv;
   launch_plan(pool, dev_req_ids, n_req, nullptr, qb, 0, lh0, lh_n, s, true);
-  gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n, 0);
+  gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n);
   gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
   pool->launch_count += 3;
   pool->step_layers_done += 1;
@@ -1046,7 +1082,8 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
   if (n_req != pool->step_n_req || !dev_req_ids || !dev_actions) return GP_ERR_INVALID;
   if (pool->step_layers_done != pool->cfg.n_layers) return GP_ERR_STATE;       // layers missing: run them, or gp_step_abort
   GP_CUDA(cudaSetDevice(pool->device));
-  gp_launch_boundary(pool->dev, dev_req_ids, n_req, dev_actions, nullptr, pool->sel_grid, pool->compact_grid,
+  gp_launch_boundary(with_state(pool, pool->dev, cur_copy(pool), cur_copy(pool) ^ 1), dev_req_ids, n_req, dev_actions, nullptr,
+                     pool->sel_grid, pool->compact_grid,
                      static_cast<cudaStream_t>(stream), nullptr, true, (int)(pool->serial & 0x3fffffff));
   pool->serial += 1;
   pool->launch_count += 2;
@@ -1159,8 +1196,9 @@ int gp_release(gp_pool* pool, int32_t req, void* stream) {
   if (st != GP_OK) return st;
   if (pool->step_open) return GP_ERR_STATE;      // the open step's plan holds a snapshot of the free list
   GP_CUDA(cudaSetDevice(pool->device));
-  if (join_side(pool, static_cast<cudaStream_t>(stream)) != GP_OK) return GP_ERR_CUDA;
-  gp_release_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(pool->dev, req);
+  if (flush_chain(pool, static_cast<cudaStream_t>(stream)) != GP_OK) return GP_ERR_CUDA;
+  gp_release_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      with_state(pool, pool->dev, cur_copy(pool), cur_copy(pool) ^ 1), req, (int)((pool->serial - 1 + 1) & 0x3fffffff));
   pool->launch_count++;
   pool->live[req] = 0;
   GP_CUDA(cudaGetLastError());
@@ -1185,11 +1223,14 @@ int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t
   const int st = check_req(pool, req);
   if (st != GP_OK) return st;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   int Pv = 0, nv = 0; long long pv = 0;
-  GP_CUDA(cudaMemcpy(&Pv, pool->dev.P + req, 4, cudaMemcpyDeviceToHost));
-  GP_CUDA(cudaMemcpy(&nv, pool->dev.n + req, 4, cudaMemcpyDeviceToHost));
-  GP_CUDA(cudaMemcpy(&pv, pool->dev.pos + req, 8, cudaMemcpyDeviceToHost));
+  int pc = 0;
+  if (pages_copy(pool, req, &pc) != GP_OK) return GP_ERR_CUDA;
+  GP_CUDA(cudaMemcpy(&Pv, pool->sP[pc] + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&nv, pool->sn[pc] + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&pv, pool->spos[cur_copy(pool)] + req, 8, cudaMemcpyDeviceToHost));
   if (P) *P = Pv;
   if (n) *n = nv;
   if (pos) *pos = pv;
@@ -1202,10 +1243,22 @@ int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t
 int gp_debug_state(gp_pool* pool, int32_t* P, int32_t* n) {
   if (!pool) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
-  const size_t nb = (size_t)pool->cfg.max_requests * 4;
-  if (P) GP_CUDA(cudaMemcpy(P, pool->dev.P, nb, cudaMemcpyDeviceToHost));
-  if (n) GP_CUDA(cudaMemcpy(n, pool->dev.n, nb, cudaMemcpyDeviceToHost));
+  const int M = pool->cfg.max_requests;
+  const size_t nb = (size_t)M * 4;
+  const int c = cur_copy(pool);
+  if (P) GP_CUDA(cudaMemcpy(P, pool->sP[c], nb, cudaMemcpyDeviceToHost));
+  if (n) GP_CUDA(cudaMemcpy(n, pool->sn[c], nb, cudaMemcpyDeviceToHost));
+  if (pool->cfg.async_boundary) {               // requests about to sit a step out: see pages_copy
+    std::vector<int> b(M), oP(M), on(M);
+    GP_CUDA(cudaMemcpy(b.data(), pool->dev.bstep, nb, cudaMemcpyDeviceToHost));
+    GP_CUDA(cudaMemcpy(oP.data(), pool->sP[c ^ 1], nb, cudaMemcpyDeviceToHost));
+    GP_CUDA(cudaMemcpy(on.data(), pool->sn[c ^ 1], nb, cudaMemcpyDeviceToHost));
+    const int last = (int)((pool->serial - 1) & 0x3fffffff);
+    for (int i = 0; i < M; ++i)
+      if (b[i] == last) { if (P) P[i] = oP[i]; if (n) n[i] = on[i]; }
+  }
   return GP_OK;
 }
 
@@ -1214,9 +1267,11 @@ static int gather_stream(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_h
   if (st != GP_OK) return st;
   if (layer < 0 || layer >= pool->cfg.n_layers || kv_head < 0 || kv_head >= pool->cfg.n_kv_heads) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
-  int nv = 0;
-  GP_CUDA(cudaMemcpy(&nv, pool->dev.n + req, 4, cudaMemcpyDeviceToHost));
+  int nv = 0, pc = 0;
+  if (pages_copy(pool, req, &pc) != GP_OK) return GP_ERR_CUDA;
+  GP_CUDA(cudaMemcpy(&nv, pool->sn[pc] + req, 4, cudaMemcpyDeviceToHost));
   *n_out = nv;
   if (nv == 0) return GP_OK;
   const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * GP_PAGE;
@@ -1225,6 +1280,7 @@ static int gather_stream(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_h
   uint4* vv = reinterpret_cast<uint4*>(pool->dbg + cap_tok * 4 + cap_tok * pool->cfg.head_dim * 2);
   gp_gather_kernel<<<148, 256>>>(pool->dev, req, layer, kv_head, nv, tok, kk, vv);
   pool->launch_count++;
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   return GP_OK;
 }
@@ -1255,10 +1311,11 @@ int gp_debug_summaries(gp_pool* pool, int32_t req, double* out) {
   if (st != GP_OK) return st;
   if (!out) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   const gp_config& c = pool->cfg;
   int par = 0;
-  GP_CUDA(cudaMemcpy(&par, pool->dev.sum_par + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&par, pool->spar[cur_copy(pool)] + req, 4, cudaMemcpyDeviceToHost));
   const size_t per = (size_t)2 * c.n_q_heads * c.head_dim;
   for (int l = 0; l < c.n_layers; ++l)
     GP_CUDA(cudaMemcpy(out + (size_t)l * per, pool->dev.summ + (((size_t)l * c.max_requests + req) * 2 + par) * per,
@@ -1270,6 +1327,7 @@ int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, do
   const int st = check_req(pool, req);
   if (st != GP_OK) return st;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   const int LH = pool->cfg.n_layers * pool->cfg.n_kv_heads;
   std::vector<int> kx((size_t)LH * 2);
@@ -1285,6 +1343,7 @@ int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, do
 int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t counters[12]) {
   if (!pool) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   int top = 0;
   GP_CUDA(cudaMemcpy(&top, pool->dev.free_top, 4, cudaMemcpyDeviceToHost));
@@ -1317,6 +1376,7 @@ int gp_set_profiling(gp_pool* pool, int32_t enable) {
 int gp_get_kernel_times(gp_pool* pool, float* ms, int64_t* launches) {
   if (!pool) return GP_ERR_INVALID;
   GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   for (int i = 0; i < GP_N_KERNELS; ++i) {
     if (ms) ms[i] = pool->ms[i];

@@ -41,9 +41,10 @@ HELD = 6                 # action code of a request that sat a step out (asynchr
 
 
 class Scheduler:
-    def __init__(self, wl: W.Workload):
+    def __init__(self, wl: W.Workload, only=None):
+        """`only`: indices of the workload's requests to run (default: all of them)."""
         self.wl = wl
-        self.pending = collections.deque(wl.requests)
+        self.pending = collections.deque(wl.requests if only is None else [wl.requests[i] for i in only])
         self.resident: Dict[int, _Resident] = {}        # spec index -> state
         self.finished: List[int] = []
         self.stalled: List[int] = []
