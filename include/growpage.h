@@ -314,6 +314,18 @@ int gp_get_kernel_times(gp_pool* pool, float* ms, int64_t* launches);
 /* Kernels launched by this pool since creation (all calls). */
 int64_t gp_launch_count(gp_pool* pool);
 
+/* ---- test support --------------------------------------------------------------------------------------------- */
+
+/* Every wait of one thread block for another inside the kernels is bounded: after a number of iterations it gives
+ * up, sets an error bit (gp_pool_status) and the kernel runs to its end, with wrong results for the work concerned
+ * but without hanging and with the pool's page accounting intact.  This call lets a test see that happen without
+ * any fault: `what` names hand-overs that are then simply not made (1 the attention kernel's first thread block
+ * never completes its second work item for its consumer warps; 2 the first chunk of every compaction unit never
+ * says that its sources are read; 4 asynchronous mode: the deciding thread block never tells the others; 0 none),
+ * `spin_limit` the iterations after which waits give up (0 = the default, 2^21).  Applies to the steps issued
+ * after it.  The error bits stay set; results of such a pool are not meaningful afterwards. */
+int gp_test_withhold(gp_pool* pool, int32_t what, int32_t spin_limit);
+
 /* ---- attention without any allocation ------------------------------------------------------------ */
 
 #define GP_NOALLOC_SPLITS   8      /* parts a request's tokens are split into                           */

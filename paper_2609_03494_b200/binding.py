@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
     L.gp_pool_status.argtypes = [vp, C.POINTER(i32)]
     L.gp_async_join.argtypes = [vp, vp]
     L.gp_boundary_outcome.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i64)]
+    L.gp_test_withhold.argtypes = [vp, i32, i32]
     L.gp_set_profiling.argtypes = [vp, i32]
     L.gp_set_early_plan.argtypes = [vp, i32]
     L.gp_get_kernel_times.argtypes = [vp, vp, vp]
@@ -239,6 +240,10 @@ def gp_debug_pool(pool: int, n_pages: int = 0):
     _check(lib().gp_debug_pool(C.c_void_p(pool), C.byref(n_free), ref.ctypes.data_as(C.c_void_p) if n_pages else None,
                                counters.ctypes.data_as(C.c_void_p)), "gp_debug_pool")
     return int(n_free.value), ref[:n_pages], counters
+
+
+def gp_test_withhold(pool: int, what: int, spin_limit: int) -> None:
+    _check(lib().gp_test_withhold(C.c_void_p(pool), what, spin_limit), "gp_test_withhold")
 
 
 def gp_set_early_plan(pool: int, enable: bool) -> None:

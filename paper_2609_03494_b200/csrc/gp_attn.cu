@@ -78,8 +78,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // bounded, abort-aware wait
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int where = 0) {
-  for (uint32_t it = 0; it < GP_SPIN_LIMIT; ++it) {
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int where, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 63u && *abort_flag) return false;
   }
@@ -118,6 +118,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
   const int comb_w = L.comb_warp / 4;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t lim = p.spin_limit;
   if (tid == 0) {
     for (int i = 0; i < NI_MAX; ++i) { mbar_init(&slot_full[i], 2); mbar_init(&slot_empty[i], NCW + 1); }
     mbar_init(qt_full, 1);
@@ -158,7 +159,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     int hB = 0, hC = 0;                        // descriptor header, word `lane` (lanes 0..15)
     int pC = -1, pC2 = -1;                     // page ids of tiles `lane` and `lane + 32` of the item
     int slC = 0;                               // slot of the item in stage C
-    uint32_t n_pub = 0;
+    uint32_t n_pub = 0, n_comp = 0;          // items published (stage B), items completed (stage C)
     bool sentinel_out = false;
     // The q~ buffer is single: the copy for a boundary item is issued once the consumers are done with the
     // previous boundary item.  The producer never blocks on that (it would hold back the slots of other
@@ -180,7 +181,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       }
     };
     auto wait_polling = [&](uint64_t* bar, uint32_t parity) -> bool {     // bounded, abort-aware, keeps q~ moving
-      for (uint32_t w = 0; w < GP_SPIN_LIMIT; ++w) {
+      for (uint32_t w = 0; w < lim; ++w) {
         if (mbar_try_wait(bar, parity)) return true;
         poll_qt();
         if ((w & 63u) == 63u && s_misc[0]) return false;
@@ -201,7 +202,10 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         sd[GEO::SLOT_PAGES + lane] = pC;
         sd[GEO::SLOT_PAGES + 32 + lane] = pC2;
         __syncwarp();
-        if (lane == 0) mbar_arrive(&slot_full[slC]);
+        // (test support: the first CTA's second item can be withheld, so that the consumers' bounded wait runs out)
+        const bool withheld = (p.withhold & GP_WITHHOLD_ITEM) && blockIdx.x == 0 && n_comp == 1;
+        ++n_comp;
+        if (lane == 0 && !withheld) mbar_arrive(&slot_full[slC]);
       }
       poll_qt();
       // ---- header of stage B has arrived: load its page ids and fill its slot -----------------------
@@ -263,7 +267,6 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       if (!wait_polling(qt_empty, (qt_head & 1u) ^ 1u)) break;
       poll_qt();
     }
-    if (s_misc[0] && lane == 0) atomicOr(p.err, GP_E_SPIN | (1 << (7 + s_misc[1])));
   } else if (warp >= 4) {
     // ================================= consumers ==========================================
     const int cw = warp - 4;
@@ -289,7 +292,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           // nothing the current item needs may wait for a later item to be published
           if (f_it > it_now) {
             if (!mbar_test_wait(&slot_full[f_it % NI], (f_it / NI) & 1u)) break;
-          } else if (!wait_bar(&slot_full[f_it % NI], (f_it / NI) & 1u, s_misc, 3)) {
+          } else if (!wait_bar(&slot_full[f_it % NI], (f_it / NI) & 1u, s_misc, 3, lim)) {
             return false;
           }
           f_npg = fsd[3];
@@ -318,7 +321,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     for (uint32_t it = 0;; ++it) {
       const int sl = it % NI;
       if (!top_up(it)) break;
-      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc, 4)) break;
+      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc, 4, lim)) break;
       const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
@@ -368,7 +371,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
         }
       }
       if (need_qt) {
-        if (!wait_bar(qt_full, qt_uses & 1u, s_misc, 5)) break;
+        if (!wait_bar(qt_full, qt_uses & 1u, s_misc, 5, lim)) break;
       }
 
       const bool last_chunk = (chunk == nchunks - 1);
@@ -561,7 +564,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
       const int cb = it % NCOMB;
-      if (!wait_bar(&comb_empty[cb], ((it / NCOMB) & 1u) ^ 1u, s_misc, 6)) break;
+      if (!wait_bar(&comb_empty[cb], ((it / NCOMB) & 1u) ^ 1u, s_misc, 6, lim)) break;
       float* my_comb = comb + (cb * NCW + cw) * comb_w;
       if (row < G) {
         if ((lane & 3) == 0) { my_comb[row] = m_run; my_comb[8 + row] = l_run; }
@@ -584,7 +587,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     // ================================= merger =============================================
     for (uint32_t it = 0;; ++it) {
       const int sl = it % NI;
-      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc, 7)) break;
+      if (!wait_bar(&slot_full[sl], (it / NI) & 1u, s_misc, 7, lim)) break;
       const uint8_t* slot = smem + L.off_slots + sl * GEO::SLOT_BYTES;
       const int* sd = reinterpret_cast<const int*>(slot);
       const int npg = sd[3];
@@ -592,7 +595,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       const int bi = sd[0], nchunks = sd[5], rc_i = sd[13], lh = sd[14];
       const int l = lh / p.Hkv, h = lh % p.Hkv;
       const int cb = it % NCOMB;
-      if (!wait_bar(&comb_full[cb], (it / NCOMB) & 1u, s_misc, 8)) break;
+      if (!wait_bar(&comb_full[cb], (it / NCOMB) & 1u, s_misc, 8, lim)) break;
       const float* cbuf = comb + (size_t)cb * NCW * comb_w;
       const size_t out_row0 = (((size_t)l * n_req + bi) * p.Hq + h * G) * D;
       const int PSTRIDE = G * (D + 2);
@@ -625,6 +628,8 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
     }
   }
   __syncthreads();
+  // a wait of this CTA gave up (whichever warp it was, and however late): say so, with the code of the wait
+  if (tid == 0 && s_misc[0]) atomicOr(p.err, GP_E_SPIN | (1 << (7 + s_misc[1])));
 }
 
 }  // namespace

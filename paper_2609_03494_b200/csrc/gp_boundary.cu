@@ -1149,12 +1149,13 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
     if (tid == 0) {
       // No fence on either side: the flag only says that loads have returned (they have: their values were
       // consumed above), and the stores below are issued after the flag has been seen.
-      *reinterpret_cast<volatile int*>(p.cflags + item) = stamp;      // "my sources are read"
+      if (!((p.withhold & GP_WITHHOLD_CHUNK) && j == 0))               // (test support: see GP_WITHHOLD_CHUNK)
+        *reinterpret_cast<volatile int*>(p.cflags + item) = stamp;      // "my sources are read"
       if (j > 0) {                                          // the previous chunk's tail is my first destination
         volatile int* prev = reinterpret_cast<volatile int*>(p.cflags + item - 1);
         unsigned it = 0;
-        while (*prev != stamp && it < GP_SPIN_LIMIT) ++it;
-        if (it >= GP_SPIN_LIMIT) atomicOr(p.err, GP_E_SPIN_CMP);
+        while (*prev != stamp && it < p.spin_limit) ++it;
+        if (it >= p.spin_limit) atomicOr(p.err, GP_E_SPIN_CMP);
       }
     }
     __syncthreads();
@@ -1318,15 +1319,15 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
       __threadfence();
       decide_and_allocate(p, nullptr, 0, n_bnd, nullptr, reinterpret_cast<int*>(S.sbuf), serial);
       __syncthreads();
-      if (tid == 0) {
+      if (tid == 0 && !(p.withhold & GP_WITHHOLD_DECIDED)) {      // (test support: see GP_WITHHOLD_DECIDED)
         __threadfence();
         *reinterpret_cast<volatile int*>(p.hdr + HDR_DECIDED) = stamp;
       }
     } else if (tid == 0) {
       volatile int* flag = reinterpret_cast<volatile int*>(p.hdr + HDR_DECIDED);
       unsigned it = 0;
-      while (*flag != stamp && it < GP_SPIN_LIMIT) { ++it; __nanosleep(100); }
-      if (it >= GP_SPIN_LIMIT) atomicOr(p.err, GP_E_SPIN_CMP);
+      while (*flag != stamp && it < p.spin_limit) { ++it; __nanosleep(100); }
+      if (it >= p.spin_limit) atomicOr(p.err, GP_E_SPIN_CMP);
       __threadfence();
     }
     __syncthreads();

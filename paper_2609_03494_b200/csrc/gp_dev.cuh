@@ -41,6 +41,13 @@ enum {
   HDR_COUNT = 16
 };
 
+// hand-overs a test can withhold (gp_test_withhold): the bounded wait for it then runs out
+enum {
+  GP_WITHHOLD_ITEM = 1,     // attention kernel, first CTA: its second work item is never published to the consumers
+  GP_WITHHOLD_CHUNK = 2,    // compaction: the first chunk of a unit never says that its sources are read
+  GP_WITHHOLD_DECIDED = 4,  // asynchronous chain kernel: the deciding CTA never tells the others
+};
+
 // error bits
 enum {
   GP_E_SPIN = 1,        // a bounded wait gave up
@@ -54,6 +61,8 @@ struct GpDev {
   int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;
   long long n_pages, max_batch_tokens;
   long long max_boundary_tokens;         // bound on the summed candidate tokens of one step's boundary requests
+  unsigned spin_limit;                   // iterations after which a bounded wait gives up (GP_SPIN_LIMIT; tests shorten it)
+  int withhold;                          // test support, GP_WITHHOLD_*: a hand-over inside a kernel that is made not to happen
   int async;                             // 1: the boundary chain of a step runs beside the next step (see gp_decode_step)
   double beta_s, beta_l, top_p, tau, rope_theta;
   int bchunk_pages;                      // pages per work item of a request at its capacity boundary

@@ -308,7 +308,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   // cover the (layer, KV head) units [lh0, lh0 + lh_n) (none when lh_n is 0: the query rows come layer by layer)
   __shared__ int sv[33];
   __shared__ long long sw[33];
-  __shared__ int s_first[GP_MAX_REQ];      // lowest batch index naming a request
+  __shared__ __align__(16) int s_first[GP_MAX_REQ];      // lowest batch index naming a request
   __shared__ int s_chunks[GP_MAX_REQ], s_pos[GP_MAX_REQ];
   __shared__ int s_req[GP_MAX_REQ], s_state[GP_MAX_REQ];     // summary CTAs: request of a batch slot, flags
   __shared__ long long s_pos64[GP_MAX_REQ];
@@ -444,8 +444,23 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   // Work items are listed by descending cost (pages, times four for boundary requests, which also pay for the
   // fp64 logits): the attention kernel deals them out in that order, largest first.  Counting sort.
   const int key = chunks > 0 ? min(GP_COST_BINS - 1, cp * (isb ? 4 : 1)) : 0;
+  // Items of equal cost keep the batch's order (a rank counted over the earlier batch slots, not the order in
+  // which atomics land), so that the same batch is dealt to the thread blocks the same way every time and the
+  // attention outputs repeat bit for bit.
+  s_first[i] = chunks > 0 ? (key << 16) | chunks : 0;        // s_first has served its purpose: cost class and items
+  if (chunks > 0) atomicAdd(&s_bin[key], chunks);
+  __syncthreads();
   int within = 0;
-  if (chunks > 0) within = atomicAdd(&s_bin[key], chunks);
+  if (chunks > 0) {
+    const int4* e4 = reinterpret_cast<const int4*>(s_first);
+    int j = 0;
+    for (; j + 4 <= i; j += 4) {
+      const int4 e = e4[j >> 2];
+      within += ((e.x >> 16) == key ? (e.x & 0xffff) : 0) + ((e.y >> 16) == key ? (e.y & 0xffff) : 0) +
+                ((e.z >> 16) == key ? (e.z & 0xffff) : 0) + ((e.w >> 16) == key ? (e.w & 0xffff) : 0);
+    }
+    for (; j < i; ++j) { const int e = s_first[j]; within += (e >> 16) == key ? (e & 0xffff) : 0; }
+  }
   __syncthreads();
   if (threadIdx.x < 32) {                             // descending exclusive scan over the cost bins
     int carry = 0;
@@ -771,6 +786,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
   d.max_boundary_tokens = L.max_boundary_tokens;
   d.async = cfg->async_boundary;
+  d.spin_limit = GP_SPIN_LIMIT;
+  d.withhold = 0;
   d.z_stride = (L.max_boundary_tokens + GP_PAGE - 1) / GP_PAGE * GP_PAGE;
   d.beta_s = cfg->beta_s; d.beta_l = cfg->beta_l; d.top_p = cfg->top_p; d.tau = cfg->tau; d.rope_theta = cfg->rope_theta;
   d.policy = cfg->policy; d.policy_seed = (unsigned long long)(unsigned)cfg->policy_seed; d.p_compress = cfg->p_compress;
@@ -1355,6 +1372,16 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
     GP_CUDA(cudaMemcpy(c, pool->dev.counters, 96, cudaMemcpyDeviceToHost));
     for (int i = 0; i < 12; ++i) counters[i] = c[i];
     counters[7] = err;
+  }
+  return GP_OK;
+}
+
+int gp_test_withhold(gp_pool* pool, int32_t what, int32_t spin_limit) {
+  if (!pool || what < 0 || what > 7 || spin_limit < 0) return GP_ERR_INVALID;
+  GpDev* views[2] = {&pool->dev, &pool->dev_alt};
+  for (GpDev* v : views) {
+    v->withhold = what;
+    v->spin_limit = spin_limit > 0 ? (unsigned)spin_limit : GP_SPIN_LIMIT;
   }
   return GP_OK;
 }

@@ -303,16 +303,19 @@ def parity_instance(config: int) -> Workload:
     if config == 2:
         return layer8b(n_requests=8, n_steps=320, prompt_range=(128, 512))
     if config == 3:
-        wl = stack8b(n_layers=4, n_resident=6, n_total=10, out_range=(48, 160), prompt_range=(40, 120))
-        # same pressure as the full config: the pool holds far less than the residents ask for
-        wl.n_pages = 6 * 9
+        # 12 layers, 8 residents of 14 requests, outputs up to 320 tokens; same pressure as the full config: the
+        # pool holds far less than the residents ask for, so grants are refused, requests stall and are replaced
+        wl = stack8b(n_layers=12, n_resident=8, n_total=14, out_range=(64, 320), prompt_range=(64, 256))
+        wl.n_pages = 8 * 14
         return wl
     if config == 4:
-        wl = stack32b(n_layers=2, n_requests=4, out_range=(128, 320), prompt_range=(64, 160))
-        wl.n_pages = 4 * 40
+        # 4 layers of the 64-query-head shape, 6 requests that run hundreds of steps past their direction shift
+        wl = stack32b(n_layers=4, n_requests=6, out_range=(256, 640), prompt_range=(64, 192))
+        wl.n_pages = 6 * 56
         return wl
     if config == 5:
-        return prefix_stress(n_groups=2, group_size=3, prompt_len=128, n_steps=96, initial_pages=8,
+        # 4 groups of 4 on a shared 256-token prompt, 512 steps
+        return prefix_stress(n_groups=4, group_size=4, prompt_len=256, n_steps=512, initial_pages=8,
                              extra_pages=2)
     raise ValueError(config)
 

@@ -134,3 +134,98 @@ def test_pool_is_closed_to_admissions_and_releases_inside_an_open_step_and_a_ste
     assert np.array_equal(o1, o2) and np.array_equal(a1, a2) and f1 == f2
     assert all(np.array_equal(x, y) for x, y in zip(s1, s2))
     assert a1.tolist() == [B.GP_ACT_GROW, B.GP_ACT_NONE, B.GP_ACT_GROW]      # 32 and 48 tokens fill two and three pages
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# bounded waits that run out: the kernel gives up, says so, and ends; nothing hangs, nothing faults
+# ----------------------------------------------------------------------------------------------------------------
+def _accounting_intact(pool, n_pages, live, cap):
+    n_free, ref, _ = B.gp_debug_pool(pool.handle, n_pages)
+    held = 0
+    for r in live:
+        P, n, pos, table = B.gp_debug_request(pool.handle, r, cap)
+        assert len(set(table)) == P and 0 < n <= P * 16
+        held += P
+    assert int((ref > 0).sum()) + n_free == n_pages and int(ref.sum()) == held
+
+
+def _one_step(pool, torch, rng, n_req, hq, hkv, d, host=False):
+    q, k, v = _bits(rng, 1, n_req, hq, d), _bits(rng, 1, n_req, hkv, d), _bits(rng, 1, n_req, hkv, d)
+    out = torch.zeros((1, n_req, hq, d), dtype=torch.float32, device="cuda")
+    act = torch.zeros(n_req, dtype=torch.int32, device="cuda")
+    ids = torch.arange(n_req, dtype=torch.int32, device="cuda")
+    if host:
+        ph = lambda t: t.cpu().pin_memory()
+        args = [ph(ids), ph(_dev(torch, q)), ph(_dev(torch, k)), ph(_dev(torch, v)), ph(out), ph(act)]
+        pool.decode_step_host(*args)
+        return args[4].numpy().copy(), args[5].numpy().copy()
+    pool.decode_step(ids, _dev(torch, q), _dev(torch, k), _dev(torch, v), out, act)
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), act.cpu().numpy()
+
+
+def test_attention_wait_that_runs_out_is_reported_and_the_kernel_drains():
+    import torch
+    # 80 requests x 8 heads = 640 work items on 296 thread blocks: the first block has a second item, which the test
+    # withholds from its consumer warps; their wait gives up after 3000 tries
+    n_req, hq, hkv, d, cap = 80, 8, 8, 64, 4
+    cfg = B.make_config(1, hq, hkv, d, n_pages=n_req * cap, max_pages_per_req=cap, max_requests=n_req, host_staging=True)
+    results = []
+    for withhold in (0, 1):
+        rng = np.random.default_rng(11)
+        pool = B.Pool(cfg)
+        try:
+            for _ in range(n_req):
+                assert pool.request_add(-1, 0, _bits(rng, 1, 20, hkv, d), _bits(rng, 1, 20, hkv, d), 20, 0)[0] == B.GP_OK
+            B.gp_test_withhold(pool.handle, withhold, 3000)
+            if withhold:
+                with pytest.raises(B.GpError) as e:              # the host entry point looks at the error word itself
+                    _one_step(pool, torch, rng, n_req, hq, hkv, d, host=True)
+                assert e.value.status == B.GP_ERR_CUDA
+                st, bits = B.gp_pool_status(pool.handle)
+                assert st == B.GP_ERR_CUDA and (bits & 1) and (bits >> 7), bits      # a wait gave up, and which one
+                _accounting_intact(pool, n_req * cap, range(n_req), cap)
+                assert B.gp_debug_pool(pool.handle)[2][7] == bits
+            else:
+                results.append(_one_step(pool, torch, rng, n_req, hq, hkv, d, host=True))
+                assert B.gp_pool_status(pool.handle) == (B.GP_OK, 0)
+        finally:
+            pool.close()
+    # the device is as usable as before: an ordinary pool gives the ordinary result
+    rng = np.random.default_rng(11)
+    pool = B.Pool(cfg)
+    try:
+        for _ in range(n_req):
+            pool.request_add(-1, 0, _bits(rng, 1, 20, hkv, d), _bits(rng, 1, 20, hkv, d), 20, 0)
+        out, act = _one_step(pool, torch, rng, n_req, hq, hkv, d, host=True)
+        diff = np.abs(out - results[0][0])
+        assert np.array_equal(act, results[0][1]) and diff.max() == 0.0, (float(diff.max()), np.argwhere(diff > 0)[:4].tolist(), int((diff > 0).sum()))
+    finally:
+        pool.close()
+
+
+@pytest.mark.parametrize("async_boundary,what,bit", [(False, 2, 8), (True, 2, 8), (True, 4, 8)])
+def test_compaction_and_decision_waits_that_run_out_are_reported(async_boundary, what, bit):
+    import torch
+    # one request of eight pages that fills its last slot with the first step and compresses: two chunks per unit
+    n_req, hq, hkv, d, cap = 3, 8, 2, 64, 9
+    cfg = B.make_config(1, hq, hkv, d, n_pages=n_req * cap, max_pages_per_req=cap, max_requests=4, async_boundary=async_boundary)
+    rng = np.random.default_rng(13)
+    pool = B.Pool(cfg)
+    try:
+        for _ in range(n_req):
+            assert pool.request_add(-1, 0, _bits(rng, 1, 127, hkv, d), _bits(rng, 1, 127, hkv, d), 127, 0)[0] == B.GP_OK
+        B.gp_test_withhold(pool.handle, what, 2000)
+        out, act = _one_step(pool, torch, rng, n_req, hq, hkv, d)
+        assert act.tolist() == [B.GP_ACT_PENDING if async_boundary else B.GP_ACT_COMPRESS] * n_req
+        B.gp_async_join(pool.handle, pool.stream())
+        torch.cuda.synchronize()
+        st, bits = B.gp_pool_status(pool.handle)
+        assert st == B.GP_ERR_CUDA and (bits & bit), bits
+        _accounting_intact(pool, n_req * cap, range(n_req), cap)
+        assert [B.gp_debug_request(pool.handle, r, cap)[:2] for r in range(n_req)] == [(8, 112)] * n_req
+        B.gp_test_withhold(pool.handle, 0, 0)
+        out, act = _one_step(pool, torch, rng, n_req, hq, hkv, d)        # the pool still steps
+        assert np.isfinite(out).all() and act.tolist() == [B.GP_ACT_HELD if async_boundary else B.GP_ACT_NONE] * n_req
+    finally:
+        pool.close()
