@@ -533,6 +533,33 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_size(args):
+    """The configurations whose full size only the GPU can hold (36 or 64 layers on a 120 GB pool; 256 requests on
+    shared 2048-token prompts): `steps` decode steps with continuous batching on device-drawn inputs, device time
+    by CUDA events around the decode steps, and the any-size invariants checked on the state read back."""
+    import torch
+    from paper_2609_03494_b200 import synth
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    sc = {"config3": synth.config3, "config4": synth.config4, "config5": synth.config5}[args.workload]()
+    K = args.steps if args.steps != JOB_STEPS else (256 if args.workload != "config5" else 2048)
+    res = synth.run_at_size(sc, n_steps=K, chunk=8, async_boundary=args.boundary == "async", check_every=8,
+                            seed={"config3": 2, "config4": 3, "config5": 4}[args.workload])
+    peak, peak_kind = measured_peak()
+    line = {"metric": METRIC, "value": res["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1, "steps": K, "warmup": 0,
+            "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic (drawn on the device)",
+            "config": {"workload": f"{res['config']} at its stated size (not the headline workload): {res['layers']} layers, "
+                                   f"{sc.n_resident} residents, pool {res['pool_kv_gb']} GB of K/V in a blob of {res['blob_gb']} GB",
+                       "boundary": "async" if res["async_boundary"] else "sync"},
+            "step_roofline": {"what": "keys and values of the residents' retained tokens over the decode steps' device time (attention "
+                                      "traffic only; boundary scoring and compaction not counted)",
+                              "achieved_gbs": res["attention_bytes_over_step_time_gbs"],
+                              "frac_of_8tbs": round(res["attention_bytes_over_step_time_gbs"] / NOMINAL_HBM_GBS, 4),
+                              "frac_of_measured": round(res["attention_bytes_over_step_time_gbs"] / peak, 4), "peak_kind": peak_kind},
+            "size_run": res}
+    print(json.dumps(line))
+
+
 def spawn_ranks(n: int) -> int:
     """`--gpus N` outside a torchrun launch: start N ranks of this command, one per GPU, on this node."""
     with socket.socket() as sk:
@@ -558,13 +585,17 @@ def main():
     ap.add_argument("--async-slots", type=int, default=0, help="thread blocks the attention kernel leaves to the boundary kernels")
     ap.add_argument("--entry", default="step", choices=["step", "layers"],
                     help="step: gp_decode_step; layers: the same step through gp_step_begin / gp_attn_layer / gp_step_end")
-    ap.add_argument("--workload", default="layer", choices=["layer", "stack"],
-                    help="layer: the headline one-layer Qwen3-8B-shaped workload; stack: the 36-layer shape, 16 resident requests")
+    ap.add_argument("--workload", default="layer", choices=["layer", "stack", "config3", "config4", "config5"],
+                    help="layer: the headline one-layer Qwen3-8B-shaped workload; stack: the 36-layer shape, 16 resident requests; "
+                         "config3 / config4 / config5: the multi-layer and prefix-sharing configurations at their stated sizes, "
+                         "inputs drawn on the device (throughput and invariants, no per-kernel pass)")
     ap.add_argument("--policy", default="demand", choices=["demand", "inverse", "random", "shrink"],
                     help="capacity-control policy (the paper's default, or one of its ablation's controls)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload.startswith("config"):
+        run_size(args)
     elif args.gpus > 1 and "RANK" not in os.environ:
         sys.exit(spawn_ranks(args.gpus))
     else:

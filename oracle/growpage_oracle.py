@@ -203,19 +203,20 @@ def _top(cands: np.ndarray, s: np.ndarray, k: int) -> Tuple[np.ndarray, float]:
 
 
 def select_retained(s: np.ndarray, n_blocks: int, b: int, K_t: int, k_loc: int) -> Tuple[np.ndarray, float]:
-    """Eq. 10 for one (layer, KV head).  Candidates are slots 0 .. n_blocks*b - 1, block j is
-    slots [j*b, (j+1)*b).  Every block keeps its k' = min(k_loc, floor(K_t / n_blocks)) best
-    slots; the global best of the remaining candidates fill up to K_t.  Returns the retained
-    slots in ascending order and the smallest relative score gap met at any cut."""
-    n_c = n_blocks * b
-    assert s.shape[0] == n_c
+    """Eq. 10 for one (layer, KV head).  Candidates are slots 0 .. len(s) - 1, block j is the
+    candidates among slots [j*b, (j+1)*b): n_blocks blocks, the last of which is short when the
+    protected window is smaller than a block.  Every block keeps its k' = min(k_loc, floor(K_t /
+    n_blocks)) best slots; the global best of the remaining candidates fill up to K_t.  Returns the
+    retained slots in ascending order and the smallest relative score gap met at any cut."""
+    n_c = s.shape[0]
+    assert (n_blocks - 1) * b < n_c <= n_blocks * b
     if K_t <= 0:
         return np.zeros(0, dtype=np.int64), math.inf
     k_prime = min(k_loc, K_t // n_blocks)
     margin = math.inf
     local = []
     for j in range(n_blocks):
-        blk = np.arange(j * b, (j + 1) * b, dtype=np.int64)
+        blk = np.arange(j * b, min((j + 1) * b, n_c), dtype=np.int64)
         keep, gap = _top(blk, s, k_prime)
         local.append(keep)
         margin = min(margin, gap)
@@ -268,7 +269,7 @@ class OracleConfig:
     beta_l: float = 0.999
     top_p: float = 0.99
     tau: float = 0.0
-    recent_window: int = 16          # equals the page size in this build
+    recent_window: int = 16          # |R_t|: protected newest tokens; at most the page size and a divisor of it
     k_loc: int = 4                   # a quarter of a page, the paper's 64 of 256
     rope_theta: float = 0.0
     policy: int = 0                  # 0 demand (Eq. 8), 1 inverse, 2 random, 3 shrink (Eq. 13): the ablation's controls
@@ -288,8 +289,11 @@ class BoundaryInfo:
     req: int
     P: int
     n_c: int
-    a_s: Optional[np.ndarray] = None       # [L][H_kv][|C|]
+    n_e: int = 0                            # candidates of Eq. 10: history minus the protected window (= n_c when R = b)
+    a_s: Optional[np.ndarray] = None       # [L][H_kv][|C|]: the views over the demand support (Eq. 7)
     a_l: Optional[np.ndarray] = None
+    e_s: Optional[np.ndarray] = None       # [L][H_kv][n_e]: the views over the eviction support (Eq. 9, Eq. 10)
+    e_l: Optional[np.ndarray] = None
     K_s: Optional[np.ndarray] = None       # [L][H_kv] int
     K_l: Optional[np.ndarray] = None
     ws_margin: Optional[np.ndarray] = None  # [L][H_kv][2]
@@ -316,7 +320,7 @@ class StepRecord:
 class OraclePool:
     def __init__(self, cfg: OracleConfig):
         assert cfg.n_q_heads % cfg.n_kv_heads == 0
-        assert cfg.recent_window == cfg.page_size
+        assert 0 < cfg.recent_window <= cfg.page_size and cfg.page_size % cfg.recent_window == 0
         self.cfg = cfg
         self.G = cfg.n_q_heads // cfg.n_kv_heads
         self.refcount = np.zeros(cfg.n_pages, dtype=np.int64)
@@ -454,8 +458,9 @@ class OraclePool:
         c = self.cfg
         b = c.page_size
         G = self.G
-        n_c = (r.P - 1) * b                          # history minus the most recent block
-        info = BoundaryInfo(req=rid, P=r.P, n_c=n_c)
+        n_c = (r.P - 1) * b                          # Eq. 7's support: history minus the most recent block
+        n_e = r.P * b - c.recent_window              # Eq. 10's candidates: history minus the protected window
+        info = BoundaryInfo(req=rid, P=r.P, n_c=n_c, n_e=n_e)
         if n_c == 0:
             info.want_grow = True
             return info
@@ -465,6 +470,9 @@ class OraclePool:
         info.K_s = np.empty((L, H), dtype=np.int64)
         info.K_l = np.empty((L, H), dtype=np.int64)
         info.ws_margin = np.empty((L, H, 2))
+        two = n_e != n_c                             # R < b: the two supports differ, each has its own softmax
+        info.e_s = np.empty((L, H, n_e)) if two else info.a_s
+        info.e_l = np.empty((L, H, n_e)) if two else info.a_l
         for l in range(L):
             qs = rope(rms_calibrate(r.S[l], q[l]), t, c.rope_theta)       # Eq. 12, then RoPE at
             ql = rope(rms_calibrate(r.Lg[l], q[l]), t, c.rope_theta)      # the current position
@@ -472,6 +480,9 @@ class OraclePool:
                 Kc = r.K[l, h, :n_c]
                 info.a_s[l, h] = summary_attention(qs[h * G:(h + 1) * G], Kc)
                 info.a_l[l, h] = summary_attention(ql[h * G:(h + 1) * G], Kc)
+                if two:
+                    info.e_s[l, h] = summary_attention(qs[h * G:(h + 1) * G], r.K[l, h, :n_e])
+                    info.e_l[l, h] = summary_attention(ql[h * G:(h + 1) * G], r.K[l, h, :n_e])
                 info.K_s[l, h], info.ws_margin[l, h, 0] = p_coverage_demand_with_margin(info.a_s[l, h], c.top_p)
                 info.K_l[l, h], info.ws_margin[l, h, 1] = p_coverage_demand_with_margin(info.a_l[l, h], c.top_p)
         # Eq. 8 with a candidate set common to all heads: the mean of K/|C| is sum(K)/(N |C|),
@@ -485,7 +496,7 @@ class OraclePool:
             info.want_grow = not (random_draw(c.policy_seed, rid, r.pos - 1) < c.p_compress)
             return info              # no working-set near-tie can change a coin
         # Eq. 13: a Shrink needs two blocks of candidates and must leave the minimum capacity
-        can_shrink = c.policy == 3 and r.P >= 3 and (r.P - 1) * b >= c.min_capacity
+        can_shrink = c.policy == 3 and r.P >= 3 and (r.P - 1) * b >= c.min_capacity and n_e > 2 * b
         if c.policy == 3:
             info.want_shrink = can_shrink and shrink_policy(info.delta, c.tau, c.shrink_below) == ACT_SHRINK
         # could a +-1 change of near-tied working-set sizes change the decision?
@@ -565,8 +576,10 @@ class OraclePool:
         at a Shrink."""
         c = self.cfg
         b = c.page_size
-        n_c = info.n_c
-        K_t = n_c - n_evict
+        R = c.recent_window
+        n_c = info.n_e                       # the candidates: everything but the protected window
+        K_t = n_c - n_evict                  # (P - 1) b - |R| at a compression: one block of slots is freed
+        n_blocks = -(-n_c // b)
         moved = 0
         for l in range(c.n_layers):
             for h in range(c.n_kv_heads):
@@ -574,21 +587,21 @@ class OraclePool:
                     keep = np.sort(np.asarray(keep_override[(l, h)], dtype=np.int64))
                     margin = 0.0
                 else:
-                    s = token_scores(info.a_s[l, h], info.a_l[l, h])
-                    keep, margin = select_retained(s, r.P - 1, b, K_t, c.k_loc)
+                    s = token_scores(info.e_s[l, h], info.e_l[l, h])
+                    keep, margin = select_retained(s, n_blocks, b, K_t, c.k_loc)
                 assert keep.size == K_t
                 info.keep[(l, h)] = keep
                 info.keep_tok[(l, h)] = r.tok[l, h, keep].copy()
                 info.sel_margin[(l, h)] = margin
                 # retained history in slot order, then the protected page
-                src = np.concatenate([keep, np.arange(n_c, n_c + b, dtype=np.int64)])
+                src = np.concatenate([keep, np.arange(n_c, n_c + R, dtype=np.int64)])
                 dst = np.arange(src.size)
                 moved += int(((src != dst) | np.isin(src // b, list(cow))).sum())
                 r.K[l, h, :src.size] = r.K[l, h, src]
                 r.V[l, h, :src.size] = r.V[l, h, src]
                 r.tok[l, h, :src.size] = r.tok[l, h, src]
                 r.tok[l, h, src.size:r.P * b] = -1
-        r.n = K_t + b
+        r.n = K_t + R
         info.moved_tokens = moved
         self.counters["moved_rows"] += moved
 

@@ -287,3 +287,21 @@ def test_pool_larger_than_four_giga_elements():
             assert (np.diff(tok) > 0).all() and np.array_equal(tok[-b:], np.arange(pos - b, pos))
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("async_boundary", [False, True])
+def test_36_layers_64_residents_with_device_side_inputs_and_continuous_batching(async_boundary):
+    """The full 36-layer stack with 64 resident requests (a quarter of the configuration's residents on a pool
+    scaled to the same pressure), inputs drawn on the device, requests finishing, stalling and being replaced:
+    the scheduler loop and checks that the full-size runs of the benchmark use (`synth.run_at_size`)."""
+    from paper_2609_03494_b200 import synth
+    sc = synth.config3(n_layers=36, n_resident=64)
+    sc.n_pages = 64 * 44                       # under what 64 residents of up to 1024 + 300 tokens ask for
+    sc.cap_pages = 90
+    res = synth.run_at_size(sc, n_steps=160, chunk=8, async_boundary=async_boundary, tau=-0.05, life_fraction=0.02,
+                            check_every=4, boundary_tokens_div=2)
+    print("\n", res)
+    assert res["layers"] == 36 and res["steps"] == 160 and res["tokens"] > 160 * 40
+    assert res["checked"]["attention"] >= 20 and res["checked"]["retained"] >= 30
+    assert res["scheduler"]["finished"] > 0 and res["scheduler"]["admitted"] > 64        # continuous batching happened
+    assert res["events"]["grow"] > 0 and res["events"]["compress"] + res["events"]["fallback"] > 0
