@@ -80,6 +80,9 @@ typedef struct gp_pool gp_pool; /* opaque */
 #define GP_POLICY_RANDOM   2
 #define GP_POLICY_SHRINK   3
 
+#define GP_METRIC_TOP_P    0
+#define GP_METRIC_ENTROPY  1
+
 typedef struct gp_config {
   int32_t n_layers;          /* L                                                                  */
   int32_t n_q_heads;         /* H_q, a multiple of n_kv_heads; group size G = H_q/H_kv <= 8        */
@@ -96,6 +99,10 @@ typedef struct gp_config {
   int32_t policy_seed;       /* GP_POLICY_RANDOM: seed of its counter-based draws                  */
   int32_t async_boundary;    /* 1: asynchronous boundary work (App. "Asynchronous Decoding and Compression"),
                                 see gp_decode_step; default 0                                       */
+  int32_t demand_metric;     /* GP_METRIC_TOP_P (default): working-set size of Eq. 7; GP_METRIC_ENTROPY: the
+                                ablation's other metric, the view's attention entropy H over ln |C| in the
+                                place of K / |C| (Delta_t is then a floating-point mean)               */
+  int32_t reserved;         /* keep 0                                                              */
   int32_t async_slots;       /* asynchronous boundary work: thread blocks of the attention kernel's grid
                                 given up so that the boundary kernel finds room on the SMs beside it;
                                 0 = a default (64)                                                    */
@@ -278,6 +285,10 @@ int gp_debug_summaries(gp_pool* pool, int32_t req, double* out);
 /* Working-set sizes of the request's most recent boundary: host int32 [L][H_kv] each, and
  * Delta_t (Eq. 7, Eq. 8). */
 int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, double* delta);
+
+/* Entropy metric only: the entropies of the two views at the request's most recent boundary, host double
+ * [L][H_kv] each (either may be NULL). */
+int gp_debug_entropy(gp_pool* pool, int32_t req, double* H_S, double* H_L);
 
 /* Free pages, per-page reference counts (host int32 [n_pages], may be NULL) and event counters:
  * [0] grow [1] compress [2] fallback-compress [3] stalled [4] copy-on-write pages

@@ -96,6 +96,18 @@ def p_coverage_demand_with_margin(a: np.ndarray, p: float) -> Tuple[int, float]:
     return k, float(margin)
 
 
+def entropy_ratio(a: np.ndarray) -> Tuple[float, float]:
+    """The ablation's other working-set metric ("Dual-Timescale Signal Ablation"): Shannon entropy of the view's
+    attention distribution, H = -sum a_i ln a_i (terms with a_i = 0 contribute nothing), and its ratio to the
+    entropy ln |C| of the uniform distribution, which plays the part of r^x of Eq. 7.  The paper names the metric
+    without a formula; the normalisation by ln |C| is this build's reading (it makes the ratio 1 for a flat view
+    and 0 for a one-hot one, like K/|C|).  Returns (H, ratio)."""
+    a = np.asarray(a, dtype=np.float64)
+    nz = a[a > 0.0]
+    H = float(-(nz * np.log(nz)).sum())
+    return H, (H / math.log(a.shape[0]) if a.shape[0] > 1 else 0.0)
+
+
 def subset_output(a: np.ndarray, v: np.ndarray, S) -> Tuple[np.ndarray, float]:
     """Eq. 3: output over the retained subset S with renormalised weights, and m(S)."""
     a = np.asarray(a, dtype=np.float64)
@@ -278,6 +290,7 @@ class OracleConfig:
     shrink_below: float = -0.005     # Eq. 13: Shrink when Delta_t is under this
     min_capacity: int = 1024         # tokens; a Shrink that would leave less is a Compress & Hold
     async_boundary: bool = False     # boundary work of step t beside step t + 1; the request sits that step out
+    demand_metric: int = 0           # 0: Top-p working set (Eq. 7); 1: attention entropy (the ablation's other metric)
 
 
 class _Request:
@@ -297,6 +310,8 @@ class BoundaryInfo:
     K_s: Optional[np.ndarray] = None       # [L][H_kv] int
     K_l: Optional[np.ndarray] = None
     ws_margin: Optional[np.ndarray] = None  # [L][H_kv][2]
+    H_s: Optional[np.ndarray] = None       # [L][H_kv] entropies of the two views (entropy metric only)
+    H_l: Optional[np.ndarray] = None
     delta: float = 0.0
     want_grow: bool = False
     want_shrink: bool = False               # policy 3 only, and only where a Shrink is admissible
@@ -470,6 +485,9 @@ class OraclePool:
         info.K_s = np.empty((L, H), dtype=np.int64)
         info.K_l = np.empty((L, H), dtype=np.int64)
         info.ws_margin = np.empty((L, H, 2))
+        use_entropy = c.demand_metric == 1
+        if use_entropy:
+            info.H_s, info.H_l = np.empty((L, H)), np.empty((L, H))
         two = n_e != n_c                             # R < b: the two supports differ, each has its own softmax
         info.e_s = np.empty((L, H, n_e)) if two else info.a_s
         info.e_l = np.empty((L, H, n_e)) if two else info.a_l
@@ -483,12 +501,26 @@ class OraclePool:
                 if two:
                     info.e_s[l, h] = summary_attention(qs[h * G:(h + 1) * G], r.K[l, h, :n_e])
                     info.e_l[l, h] = summary_attention(ql[h * G:(h + 1) * G], r.K[l, h, :n_e])
+                if use_entropy:
+                    info.H_s[l, h], info.H_l[l, h] = entropy_ratio(info.a_s[l, h])[0], entropy_ratio(info.a_l[l, h])[0]
+                    info.K_s[l, h] = info.K_l[l, h] = 0
+                    info.ws_margin[l, h] = math.inf
+                    continue
                 info.K_s[l, h], info.ws_margin[l, h, 0] = p_coverage_demand_with_margin(info.a_s[l, h], c.top_p)
                 info.K_l[l, h], info.ws_margin[l, h, 1] = p_coverage_demand_with_margin(info.a_l[l, h], c.top_p)
         # Eq. 8 with a candidate set common to all heads: the mean of K/|C| is sum(K)/(N |C|),
         # so Delta is one division of exact integers and its sign is exact.
         num = int(info.K_s.sum()) - int(info.K_l.sum())
         info.delta = num / float(L * H * n_c)
+        if use_entropy:
+            # the same mean aggregation with H / ln |C| in the place of K / |C|; the differences are summed unit by
+            # unit in (layer, head) order
+            acc = 0.0
+            for l in range(L):
+                for h in range(H):
+                    acc += info.H_s[l, h] - info.H_l[l, h]
+            info.delta = acc / (float(L * H) * math.log(n_c)) if n_c > 1 else 0.0
+            info.action_near_tie = abs(info.delta - c.tau) < 1e-12
         info.want_grow = info.delta > c.tau
         if c.policy == 1:            # inverse: grows when Delta <= tau, compresses when Delta > tau
             info.want_grow = not info.want_grow

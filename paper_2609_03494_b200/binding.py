@@ -20,6 +20,7 @@ GP_ACT_NONE, GP_ACT_GROW, GP_ACT_COMPRESS, GP_ACT_COMPRESS_FALLBACK, GP_ACT_SHRI
 GP_ACT_PENDING, GP_ACT_HELD = 5, 6
 GP_ACT_STALLED, GP_ACT_SCRATCH, GP_ACT_INVALID = -1, -2, -3
 GP_POLICY_DEMAND, GP_POLICY_INVERSE, GP_POLICY_RANDOM, GP_POLICY_SHRINK = 0, 1, 2, 3
+GP_METRIC_TOP_P, GP_METRIC_ENTROPY = 0, 1
 GP_N_KERNELS = 4
 KERNEL_NAMES = ("plan", "attention", "select_decide", "compact")
 
@@ -29,7 +30,8 @@ class gp_config(C.Structure):
         ("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
         ("page_size", C.c_int32), ("max_requests", C.c_int32), ("max_pages_per_req", C.c_int32),
         ("recent_window", C.c_int32), ("k_loc", C.c_int32), ("host_staging", C.c_int32),
-        ("policy", C.c_int32), ("policy_seed", C.c_int32), ("async_boundary", C.c_int32), ("async_slots", C.c_int32),
+        ("policy", C.c_int32), ("policy_seed", C.c_int32), ("async_boundary", C.c_int32), ("demand_metric", C.c_int32),
+        ("reserved", C.c_int32), ("async_slots", C.c_int32),
         ("n_pages", C.c_int64), ("min_capacity", C.c_int64), ("max_batch_tokens", C.c_int64),
         ("max_boundary_tokens", C.c_int64),
         ("beta_s", C.c_double), ("beta_l", C.c_double), ("top_p", C.c_double), ("tau", C.c_double),
@@ -66,6 +68,7 @@ def lib() -> C.CDLL:
     L.gp_debug_summaries.argtypes = [vp, i32, vp]
     L.gp_debug_boundary.argtypes = [vp, i32, vp, vp, C.POINTER(C.c_double)]
     L.gp_debug_pool.argtypes = [vp, C.POINTER(i64), vp, vp]
+    L.gp_debug_entropy.argtypes = [vp, i32, vp, vp]
     L.gp_step_begin.argtypes = [vp, vp, i32, vp, vp]
     L.gp_attn_layer.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
     L.gp_step_end.argtypes = [vp, vp, i32, vp, vp]
@@ -233,6 +236,14 @@ def gp_debug_boundary(pool: int, req: int, L: int, Hkv: int):
     return ks, kl, float(delta.value)
 
 
+def gp_debug_entropy(pool: int, req: int, L: int, Hkv: int):
+    hs = np.zeros((L, Hkv), dtype=np.float64)
+    hl = np.zeros((L, Hkv), dtype=np.float64)
+    _check(lib().gp_debug_entropy(C.c_void_p(pool), req, hs.ctypes.data_as(C.c_void_p), hl.ctypes.data_as(C.c_void_p)),
+           "gp_debug_entropy")
+    return hs, hl
+
+
 def gp_debug_pool(pool: int, n_pages: int = 0):
     n_free = C.c_int64()
     counters = np.zeros(12, dtype=np.int64)
@@ -353,7 +364,7 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
                 beta_s: float = 0.9, beta_l: float = 0.999, top_p: float = 0.99, tau: float = 0.0,
                 rope_theta: float = 0.0, policy: int = 0, policy_seed: int = 0, p_compress: float = 0.7,
                 shrink_below: float = -0.005, min_capacity: int = 1024, async_boundary: bool = False,
-                async_slots: int = 0, max_boundary_tokens: int = 0) -> gp_config:
+                async_slots: int = 0, max_boundary_tokens: int = 0, demand_metric: int = 0) -> gp_config:
     cfg = gp_config_default()
     cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
     cfg.n_pages, cfg.max_pages_per_req, cfg.max_requests = n_pages, max_pages_per_req, max_requests
@@ -362,4 +373,5 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
     cfg.policy, cfg.policy_seed, cfg.p_compress = policy, policy_seed, p_compress
     cfg.shrink_below, cfg.min_capacity = shrink_below, min_capacity
     cfg.async_boundary, cfg.async_slots, cfg.max_boundary_tokens = 1 if async_boundary else 0, async_slots, max_boundary_tokens
+    cfg.demand_metric = demand_metric
     return cfg

@@ -451,6 +451,13 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       int want = 1;
       if (nC > 0) {
         delta = (double)((long long)acc.x - (long long)acc.y) / ((double)LH * (double)nC);
+        if (p.metric == GP_METRIC_ENTROPY) {
+          // the same mean with H / ln |C| in the place of K / |C|, summed unit by unit in (layer, head) order
+          const double* hx = p.Hx + (size_t)r * LH * 2;
+          double accd = 0.0;
+          for (int u2 = 0; u2 < LH; ++u2) accd += __ldcg(hx + 2 * u2) - __ldcg(hx + 2 * u2 + 1);
+          delta = nC > 1 ? accd / ((double)LH * log((double)nC)) : 0.0;
+        }
         want = delta > p.tau;
         if (p.policy == 1) {                                  // the reversed reading of the demand signal
           want = !want;
@@ -845,7 +852,7 @@ __device__ __forceinline__ SelSmem sel_smem_at(uint8_t* smem) {      // smem: 25
 // 1: K^L; Eq. 7) or the `ne` slots a compression would evict (task 2; Eq. 9, Eq. 10).  The outputs go to Kout / acc
 // (the request's running sum for Eq. 8) and evout.
 __device__ __forceinline__ void sel_job(const GpDev& p, const SelSmem& S, const double* z, size_t view_stride, const double* zs,
-                                     double* a, int nC, int task, int ne, int* Kout, int* acc, int* evout) {
+                                     double* a, int nC, int task, int ne, int* Kout, int* acc, int* evout, double* Hout) {
   const int tid = threadIdx.x;
   if (task == 2) for (int i = tid; i < (nC + 31) / 32; i += SEL_T) S.loc[i] = 0;
   if (tid == 0) { S.s_res[0] = -1; S.s_i[0] = 0; S.s_i[5] = 0; S.s_i[6] = 0; S.s_i[7] = 0; }
@@ -856,6 +863,25 @@ __device__ __forceinline__ void sel_job(const GpDev& p, const SelSmem& S, const 
     case 2: uniform = job_softmax<2>(p, z, view_stride, zs, a, nC, task, S.red, S.sM, S.sZ, F, SEL_F_CAP); break;
     case 4: uniform = job_softmax<4>(p, z, view_stride, zs, a, nC, task, S.red, S.sM, S.sZ, F, SEL_F_CAP); break;
     default: uniform = job_softmax<8>(p, z, view_stride, zs, a, nC, task, S.red, S.sM, S.sZ, F, SEL_F_CAP); break;
+  }
+  if (task < 2 && p.metric == GP_METRIC_ENTROPY) {
+    // the ablation's other metric: H = -sum a ln a of the view, summed in a fixed order (per thread over its
+    // strided candidates, then a fixed tree), so that the same input gives the same bits on every run
+    __syncthreads();
+    double hsum = 0.0;
+    for (int i = tid; i < nC; i += SEL_T) { const double v = a[i]; if (v > 0.0) hsum -= v * log(v); }
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) hsum += __shfl_xor_sync(0xffffffffu, hsum, o2);
+    if ((tid & 31) == 0) S.red[tid >> 5] = hsum;
+    __syncthreads();
+    if (tid == 0) {
+      double tot = 0.0;
+      for (int w = 0; w < SEL_NW; ++w) tot += S.red[w];
+      Kout[task] = 0;
+      Hout[task] = tot;
+    }
+    __syncthreads();
+    return;
   }
   fast_hist_zero(S.H, task < 2);                   // the factors' table shared this memory
   if (task < 2) {
@@ -976,7 +1002,8 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;   // [2 views][nC][G] exp(logit - page max)
     const double* zs = p.zstat + ((size_t)lh * (p.max_boundary_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
     double* a = nC <= SEL_CAP ? S.sbuf : p.scores + ((size_t)job * LH + lh) * p.max_boundary_tokens + off;
-    sel_job(p, S, z, view_stride, zs, a, nC, task, ne, Kout, p.bnd_acc + 4 * bidx, evout);
+    sel_job(p, S, z, view_stride, zs, a, nC, task, ne, Kout, p.bnd_acc + 4 * bidx, evout,
+              p.Hx + (((size_t)r * p.L + l) * p.Hkv + h) * 2);
   }
 
   // ---- the last CTA takes the decisions ----------------------------------------------------------------------
@@ -1303,7 +1330,8 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
       const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;
       const double* zs = p.zstat + ((size_t)lh * (p.max_boundary_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
       double* a = nC <= SEL_CAP ? S.sbuf : p.scores + ((size_t)job * LH + lh) * p.max_boundary_tokens + off;
-      sel_job(p, S, z, view_stride, zs, a, nC, task, ne, Kout, p.bnd_acc + 4 * bidx, evout);
+      sel_job(p, S, z, view_stride, zs, a, nC, task, ne, Kout, p.bnd_acc + 4 * bidx, evout,
+              p.Hx + (((size_t)r * p.L + l) * p.Hkv + h) * 2);
     }
     // ---- the last CTA to finish its jobs takes the decisions and tells the others ------------------------------
     const int stamp = serial + 1;

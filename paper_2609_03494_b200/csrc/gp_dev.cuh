@@ -66,6 +66,8 @@ struct GpDev {
   int async;                             // 1: the boundary chain of a step runs beside the next step (see gp_decode_step)
   double beta_s, beta_l, top_p, tau, rope_theta;
   int bchunk_pages;                      // pages per work item of a request at its capacity boundary
+  int metric;                            // GP_METRIC_*: working-set size (Eq. 7) or attention entropy
+  double* Hx;                            // [M][L][H_kv][2] entropies of the two views at a request's last boundary (entropy metric)
   int policy;                            // GP_POLICY_* (0 demand, 1 inverse, 2 random, 3 shrink)
   unsigned long long policy_seed;
   double p_compress;

@@ -56,7 +56,7 @@ struct gp_pool {
 namespace {
 
 struct Layout {
-  size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, delta, rc,
+  size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, Hx, delta, rc,
       mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
       bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
       evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
@@ -91,6 +91,7 @@ bool valid_config(const gp_config* c) {
   if (c->n_pages < 1 || c->n_pages > 0x7fffffffLL / GP_PAGE) return false;
   if (c->k_loc < 0 || c->k_loc > GP_PAGE) return false;
   if (c->max_batch_tokens < 0 || c->max_boundary_tokens < 0) return false;
+  if (c->demand_metric < GP_METRIC_TOP_P || c->demand_metric > GP_METRIC_ENTROPY || c->reserved != 0) return false;
   if (c->async_boundary < 0 || c->async_boundary > 1 || c->async_slots < 0 || c->async_slots > 4096) return false;
   if (!(c->beta_s >= 0.0 && c->beta_s < 1.0 && c->beta_l >= 0.0 && c->beta_l < 1.0)) return false;
   if (!(c->top_p > 0.0 && c->top_p < 1.0)) return false;
@@ -129,6 +130,7 @@ Layout make_layout(const gp_config& c) {
   L.pos = take(2 * M * 8);                       // two copies
   L.summ = take((size_t)c.n_layers * M * 2 * 2 * c.n_q_heads * d * 8);
   L.Kx = take(M * LH * 2 * 4);
+  L.Hx = take(c.demand_metric == GP_METRIC_ENTROPY ? M * LH * 2 * 8 : 16);
   L.delta = take(M * 8);
   L.rc = take((size_t)L.max_rc * GP_DESC_INTS * 4);
   L.mc_list = take(M * 16);
@@ -831,6 +833,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.sum_par = d.wsum_par = pool->spar[0]; d.pos = d.wpos = pool->spos[0];
   d.summ = reinterpret_cast<double*>(base + L.summ);
   d.Kx = reinterpret_cast<int*>(base + L.Kx);
+  d.Hx = reinterpret_cast<double*>(base + L.Hx);
+  d.metric = cfg->demand_metric;
   d.delta = reinterpret_cast<double*>(base + L.delta);
   d.rcx = reinterpret_cast<int*>(base + L.rc);
   d.mc_list = reinterpret_cast<int4*>(base + L.mc_list);
@@ -1354,6 +1358,23 @@ int gp_debug_boundary(gp_pool* pool, int32_t req, int32_t* K_S, int32_t* K_L, do
     if (K_L) K_L[i] = kx[2 * i + 1];
   }
   if (delta) GP_CUDA(cudaMemcpy(delta, pool->dev.delta + req, 8, cudaMemcpyDeviceToHost));
+  return GP_OK;
+}
+
+int gp_debug_entropy(gp_pool* pool, int32_t req, double* H_S, double* H_L) {
+  const int st = check_req(pool, req);
+  if (st != GP_OK) return st;
+  if (pool->cfg.demand_metric != GP_METRIC_ENTROPY) return GP_ERR_STATE;
+  GP_CUDA(cudaSetDevice(pool->device));
+  if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
+  GP_CUDA(cudaDeviceSynchronize());
+  const int LH = pool->cfg.n_layers * pool->cfg.n_kv_heads;
+  std::vector<double> hx((size_t)LH * 2);
+  GP_CUDA(cudaMemcpy(hx.data(), pool->dev.Hx + (size_t)req * LH * 2, (size_t)LH * 16, cudaMemcpyDeviceToHost));
+  for (int i = 0; i < LH; ++i) {
+    if (H_S) H_S[i] = hx[2 * i];
+    if (H_L) H_L[i] = hx[2 * i + 1];
+  }
   return GP_OK;
 }
 

@@ -51,7 +51,7 @@ def make_pools(wl: W.Workload, device: int = 0, **over):
     kw = dict(n_pages=wl.n_pages, max_pages_per_req=wl.max_pages_per_req,
               max_requests=max(4, wl.n_resident), k_loc=wl.k_loc)
     tun = {k: over[k] for k in ("beta_s", "beta_l", "top_p", "tau", "rope_theta", "policy", "policy_seed", "p_compress",
-                                    "shrink_below", "min_capacity", "async_boundary")
+                                    "shrink_below", "min_capacity", "async_boundary", "demand_metric")
            if k in over}
     for k in ("n_pages", "max_pages_per_req", "k_loc", "max_requests"):
         if k in over:
@@ -145,7 +145,12 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
                                 f"step {st.steps} req {rid} K^{name}[{l},{h}] gpu {gk[l, h]} oracle {ok[l, h]} "
                                 f"margin {info.ws_margin[l, h, col]}")
                             st.near_ties["ws"] += 1
-                    if np.array_equal(ks, info.K_s) and np.array_equal(kl, info.K_l):
+                    if over.get("demand_metric", 0) == 1:
+                        # entropy metric: floating-point sums of logarithms on both sides, compared to rounding
+                        hs, hl = B.gp_debug_entropy(gpu.handle, rid, s.n_layers, s.n_kv_heads)
+                        assert np.allclose(hs, info.H_s, rtol=1e-11, atol=1e-13) and np.allclose(hl, info.H_l, rtol=1e-11, atol=1e-13)
+                        assert abs(delta - info.delta) <= 1e-12, f"Delta gpu {delta} oracle {info.delta}"
+                    elif np.array_equal(ks, info.K_s) and np.array_equal(kl, info.K_l):
                         assert delta == info.delta, f"Delta gpu {delta} oracle {info.delta}"
                 st.decisions["act"] += 1
                 g_want = g_dec[rid] in (B.GP_ACT_GROW, B.GP_ACT_COMPRESS_FALLBACK) or \

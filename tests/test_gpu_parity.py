@@ -757,3 +757,83 @@ def test_overlapped_launches_equal_plain_launches():
         assert all(np.array_equal(x, y) for x, y in zip(a[3], b_[3])) and all(np.array_equal(x, y) for x, y in zip(a[4], b_[4]))
         assert np.array_equal(a[0], b_[0])
     assert (a[1] == B.GP_ACT_GROW).any() and (a[1] == B.GP_ACT_COMPRESS).any()
+
+
+@pytest.mark.parametrize("config,over", [(1, {}), (1, dict(tau=-0.2)), (2, dict(tau=-0.02)), (5, dict(async_boundary=True))])
+def test_entropy_as_the_working_set_metric(config, over):
+    # the ablation's other demand metric: Delta_t from the views' entropies; selection and compaction unchanged
+    st = LS.run_lockstep(W.parity_instance(config), demand_metric=B.GP_METRIC_ENTROPY, max_steps=200, **over)
+    _report(f"entropy config{config} {over}", st)
+    assert st.decisions["act"] > 0 and st.near_ties["act"] == 0
+    if over.get("tau", 0.0) <= -0.2:
+        assert st.actions.get(B.GP_ACT_GROW, 0) > 0
+
+
+def test_preempted_request_is_readmitted_with_its_history_and_fresh_summaries():
+    """The scheduler's preemption (App. D.1: a preempted request gives its slot and pages back and, when it is
+    scheduled again, binds a slot anew and starts its summaries over): a request is released in mid-generation and
+    admitted again with everything it has seen so far as its prompt.  Both sides do the same; the slot's stale
+    summaries must not leak into the second life (the first step overwrites them), and the pages come back."""
+    import torch
+    L, Hq, Hkv, d, b = 2, 8, 2, 64, 16
+    kw = dict(n_pages=40, max_pages_per_req=12, max_requests=4, k_loc=4, tau=-0.05)
+    gpu = B.Pool(B.make_config(L, Hq, Hkv, d, **kw))
+    ora = O.OraclePool(O.OracleConfig(L, Hq, Hkv, d, **kw))
+    rng = np.random.default_rng(23)
+    bits = lambda *shape: W.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to("cuda:0")
+    f = W.bf16_bits_to_f64
+    try:
+        hist_k, hist_v = bits(L, 40, Hkv, d), bits(L, 40, Hkv, d)          # the prompt, then every decoded token
+        other_k, other_v = bits(L, 25, Hkv, d), bits(L, 25, Hkv, d)
+        for (k0, v0, n0) in ((hist_k, hist_v, 40), (other_k, other_v, 25)):
+            g = gpu.request_add(-1, 0, k0, v0, n0, 0)
+            o = ora.request_add(-1, 0, f(k0), f(v0), n0, 0)
+            assert g == (B.GP_OK, o[1])
+
+        def steps(n, rids):
+            nonlocal hist_k, hist_v
+            for _ in range(n):
+                q, k, v = bits(L, len(rids), Hq, d), bits(L, len(rids), Hkv, d), bits(L, len(rids), Hkv, d)
+                out = torch.zeros((L, len(rids), Hq, d), dtype=torch.float32, device="cuda:0")
+                act = torch.zeros(len(rids), dtype=torch.int32, device="cuda:0")
+                gpu.decode_step(torch.tensor(rids, dtype=torch.int32, device="cuda:0"), dev(q), dev(k), dev(v), out, act)
+                rec = ora.decode_step(rids, f(q), f(k), f(v))
+                assert act.cpu().tolist() == rec.actions.tolist()
+                assert np.abs(out.cpu().numpy() - rec.out).max() <= LS.ATTN_MAX_ABS
+                if 0 in rids:
+                    i = rids.index(0)
+                    hist_k = np.concatenate([hist_k, k[:, i:i + 1]], axis=1)
+                    hist_v = np.concatenate([hist_v, v[:, i:i + 1]], axis=1)
+
+        def same_state(rid):
+            assert B.gp_debug_request(gpu.handle, rid, 12)[:3] == ora.request_state(rid)[:3]
+            g, o = B.gp_debug_summaries(gpu.handle, rid, L, Hq, d), ora.summaries(rid)
+            assert (np.linalg.norm(g - o, axis=-1) / np.linalg.norm(o, axis=-1)).max() <= LS.SUMMARY_REL
+            for l in range(L):
+                for h in range(Hkv):
+                    n = ora.request_state(rid)[1]
+                    assert np.array_equal(B.gp_debug_retained(gpu.handle, rid, l, h, n), ora.retained(rid, l, h))
+
+        steps(37, [0, 1])                                   # past two boundaries of request 0 (48 and 64 or 48 again)
+        same_state(0); same_state(1)
+        stale = B.gp_debug_summaries(gpu.handle, 0, L, Hq, d)
+        free_before = B.gp_debug_pool(gpu.handle)[0]
+        held = B.gp_debug_request(gpu.handle, 0, 12)[0]
+        gpu.release(0); assert ora.release(0) == O.OK                              # preempted
+        assert B.gp_debug_pool(gpu.handle)[0] == free_before + held == ora.n_free()
+        steps(5, [1])                                       # the other request goes on alone
+        n_hist = hist_k.shape[1]
+        g = gpu.request_add(-1, 0, hist_k, hist_v, n_hist, 0)                      # scheduled again: same slot, new life
+        o = ora.request_add(-1, 0, f(hist_k), f(hist_v), n_hist, 0)
+        assert g == (B.GP_OK, 0) and o == (O.OK, 0)
+        assert B.gp_debug_request(gpu.handle, 0, 12)[:3] == (n_hist // b + 1, n_hist, n_hist)
+        steps(1, [0, 1])
+        fresh = B.gp_debug_summaries(gpu.handle, 0, L, Hq, d)
+        assert np.array_equal(fresh[:, 0], fresh[:, 1]) and not np.allclose(fresh, stale)   # S = L = the first query again
+        steps(40, [0, 1])
+        same_state(0); same_state(1)
+        n_free, ref, counters = B.gp_debug_pool(gpu.handle, 40)
+        assert counters[7] == 0 and n_free == ora.n_free()
+    finally:
+        gpu.close()

@@ -777,3 +777,132 @@ def test_sitting_out_changes_when_a_token_is_decoded_not_what_it_sees():
     for r in range(3):
         act, at = ap.boundary_outcome(r)
         assert at == max(s for s, rr in pend if rr == r) and act in (O.ACT_GROW, O.ACT_COMPRESS, O.ACT_COMPRESS_FALLBACK)
+
+
+# ----------------------------------------------------------------------------- protected window smaller than a block
+def _best_subset_ragged(s, b, K_t, k_prime):
+    """Exhaustive optimum of Eq. 10 over len(s) candidates in blocks of b, the last one short: the K_t slots of
+    largest total score among the choices that keep at least min(k', block size) slots of every block."""
+    n = len(s)
+    n_blocks = -(-n // b)
+    size = np.bincount(np.arange(n) // b, minlength=n_blocks)
+    best, best_val = None, -1.0
+    for comb in itertools.combinations(range(n), K_t):
+        cnt = np.bincount(np.asarray(comb) // b, minlength=n_blocks)
+        if np.all(cnt >= np.minimum(k_prime, size)):
+            val = s[list(comb)].sum()
+            if val > best_val:
+                best, best_val = comb, val
+    return np.asarray(best)
+
+
+@pytest.mark.parametrize("P,b,R,k_loc", [(3, 4, 2, 1), (2, 6, 2, 2), (3, 4, 1, 1), (4, 3, 1, 0)])
+def test_selection_with_a_short_last_block_is_the_constrained_optimum(P, b, R, k_loc):
+    # the paper's geometry in small: blocks of b slots, a protected window of R < b newest tokens; the candidates
+    # are all P b - R others, the target (P - 1) b - R of them, so exactly one block worth of slots goes
+    n_e, K_t = P * b - R, (P - 1) * b - R
+    for _ in range(5):
+        s = RNG.random(n_e) ** 3
+        keep, _ = O.select_retained(s, P, b, K_t, k_loc)
+        assert keep.size == K_t == n_e - b and np.all(np.diff(keep) > 0)
+        np.testing.assert_array_equal(keep, _best_subset_ragged(s, b, K_t, min(k_loc, K_t // P)))
+
+
+def test_two_supports_demand_leaves_out_the_newest_block_eviction_only_the_protected_window():
+    b, R = 8, 2
+    c = O.OracleConfig(2, 4, 2, 8, n_pages=12, max_pages_per_req=4, page_size=b, recent_window=R, k_loc=2, max_requests=2)
+    pool = O.OraclePool(c)
+    n0 = 3 * b - 1
+    kt = RNG.standard_normal((2, n0, 2, 8))
+    assert pool.request_add(-1, 0, kt, kt * 0.5, n0, 0) == (O.OK, 0)
+    r = pool.requests[0]
+    q, k, v = _rand_step(c, 1)
+    rec = pool.step_compute([0], q, k, v)
+    info = rec.boundary[0]
+    assert (info.n_c, info.n_e) == (2 * b, 3 * b - R)             # |C_t| of Eq. 7 and the candidates of Eq. 10
+    assert info.a_s.shape[-1] == 2 * b and info.e_s.shape[-1] == 3 * b - R
+    for a in (info.a_s, info.a_l, info.e_s, info.e_l):               # each support has its own normalisation
+        np.testing.assert_allclose(a.sum(axis=-1), 1.0, rtol=1e-12)
+    # the demand views do not see the newest block: changing its keys changes neither K^S nor K^L nor Delta ...
+    ks, kl, delta = info.K_s.copy(), info.K_l.copy(), info.delta
+    saved = r.K[:, :, 2 * b:3 * b - R].copy()
+    r.K[:, :, 2 * b:3 * b - R] *= 3.0
+    info2 = pool._demand(0, r, q[:, 0], r.pos - 1)
+    assert np.array_equal(info2.K_s, ks) and np.array_equal(info2.K_l, kl) and info2.delta == delta
+    assert not np.allclose(info2.e_s, info.e_s)                   # ... but the eviction scores do
+    r.K[:, :, 2 * b:3 * b - R] = saved
+    tok_before = r.tok[:, :, :3 * b].copy()
+    pool.step_apply(rec)
+    assert info.action == O.ACT_COMPRESS                          # first boundary: both summaries equal, Delta = 0
+    assert r.n == 2 * b and r.P == 3                              # exactly one block of slots is free again
+    for l in range(2):
+        for h in range(2):
+            kept = r.tok[l, h, :r.n]
+            assert np.all(np.diff(kept) > 0) and kept.size == 2 * b
+            assert np.array_equal(kept[-R:], tok_before[l, h, 3 * b - R:3 * b])      # the R newest tokens survive
+            assert np.isin(kept[:-R], tok_before[l, h, :3 * b - R]).all()
+            # tokens of the newest block outside the window are ordinary candidates: some may go, some stay
+            assert info.keep[(l, h)].size == 2 * b - R
+            # every block, the short last one included, keeps its quota
+            cnt = np.bincount(info.keep[(l, h)] // b, minlength=3)
+            assert (cnt >= min(c.k_loc, (2 * b - R) // 3)).all()
+    _check_invariants(pool)
+
+
+def test_paper_geometry_runs_and_keeps_its_invariants():
+    # b = 256, |R| = 16, k_loc = 64 (Sec. 5.1, App. B.2) on a small head shape: boundaries every 256 tokens
+    c = O.OracleConfig(1, 2, 1, 8, n_pages=8, max_pages_per_req=3, page_size=256, recent_window=16, k_loc=64, max_requests=2,
+                       tau=-1.0)
+    pool = O.OraclePool(c)
+    n0 = 300
+    kt = RNG.standard_normal((1, n0, 1, 8))
+    assert pool.request_add(-1, 0, kt, kt.copy(), n0, 0) == (O.OK, 0)
+    r = pool.requests[0]
+    assert r.P == 2
+    acts = []
+    for t in range(600):
+        rec = pool.decode_step([0], *_rand_step(c, 1))
+        if rec.actions[0] != O.ACT_NONE:
+            acts.append((t, int(rec.actions[0]), r.P, r.n))
+            info = rec.boundary[0]
+            if rec.actions[0] == O.ACT_COMPRESS_FALLBACK:
+                assert info.n_c == 2 * 256 and info.n_e == 3 * 256 - 16 and info.keep[(0, 0)].size == 2 * 256 - 16
+                assert r.n == 2 * 256 and np.array_equal(r.tok[0, 0, r.n - 16:r.n], np.arange(r.pos - 16, r.pos))
+    # 300 + 212 tokens fill two blocks: grant; 256 more fill three: at the cap, compress; then every 256 tokens
+    assert [a[:2] for a in acts] == [(211, O.ACT_GROW), (467, O.ACT_COMPRESS_FALLBACK)], acts
+    _check_invariants(pool)
+
+
+# ----------------------------------------------------------------------------- entropy as the working-set metric
+def test_entropy_metric_closed_forms_and_its_use_in_the_decision():
+    n = 64
+    H, r = O.entropy_ratio(np.full(n, 1.0 / n))
+    assert abs(H - math.log(n)) < 1e-12 and abs(r - 1.0) < 1e-12            # flat view: the whole set
+    one_hot = np.zeros(n); one_hot[17] = 1.0
+    assert O.entropy_ratio(one_hot) == (0.0, 0.0)                           # one token: nothing to spread over
+    a = np.array([0.5, 0.25, 0.25])
+    assert abs(O.entropy_ratio(a)[0] - 1.5 * math.log(2.0)) < 1e-15          # 0.5 ln 2 + 2 * 0.25 ln 4
+    two = np.zeros(n); two[:2] = 0.5
+    assert abs(O.entropy_ratio(two)[1] - math.log(2) / math.log(n)) < 1e-15
+    # like K / |C|, the ratio grows when mass spreads: the sign convention of Delta_t carries over
+    g = np.exp(-0.3 * np.arange(n)); g /= g.sum()
+    w = np.exp(-0.05 * np.arange(n)); w /= w.sum()
+    assert O.entropy_ratio(w)[1] > O.entropy_ratio(g)[1] and O.p_coverage_demand(w, 0.99) > O.p_coverage_demand(g, 0.99)
+    # in the state machine: Delta_t from entropies, same decision rule, same compression afterwards
+    c = _cfg(n_layers=2, demand_metric=1, tau=0.0)
+    pool = O.OraclePool(c)
+    n0 = 3 * c.page_size - 1
+    kt = RNG.standard_normal((2, n0, 2, c.head_dim))
+    assert pool.request_add(-1, 0, kt, kt.copy(), n0, 0) == (O.OK, 0)
+    rec = pool.decode_step([0], *_rand_step(c, 1))
+    info = rec.boundary[0]
+    assert info.delta == 0.0 and info.action == O.ACT_COMPRESS              # first step: both summaries are the query
+    for t in range(3 * c.page_size):
+        rec = pool.decode_step([0], *_rand_step(c, 1))
+        if 0 in rec.boundary:
+            info = rec.boundary[0]
+            want = sum(O.entropy_ratio(info.a_s[l, h])[1] - O.entropy_ratio(info.a_l[l, h])[1]
+                       for l in range(2) for h in range(2)) / 4.0             # Eq. 8 with the entropy ratios
+            assert abs(info.delta - want) < 1e-12 and info.want_grow == (info.delta > 0.0)
+            assert not info.K_s.any()
+    _check_invariants(pool)
