@@ -231,6 +231,18 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
                 void* stream);
 int gp_step_abort(gp_pool* pool);
 
+/* gp_attn_layer with the model's query / key normalisation fused in (Sec. 3.2: the summaries follow the query
+ * after its normalisation and before its rotation).  q_raw [n_req][H_q][d] and k_raw [n_req][H_kv][d] are the
+ * projections' bf16 outputs; per head, x <- x / sqrt(mean(x^2) + eps) * weight (q_weight, k_weight: device fp32
+ * [d], one learned weight per element of the head dimension).  The normalised query, rounded to bf16, is the
+ * query of the layer (attention rotates it when RoPE is on, the summaries take it as it is); the normalised key
+ * is rotated to its position when RoPE is on and rounded to bf16 in that cache form.  Arithmetic in fp64, rounded
+ * double -> float -> bf16.  Otherwise as gp_attn_layer (v in cache form, same alignment rules; the weights 4-byte
+ * aligned). */
+int gp_attn_layer_qknorm(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req,
+                         const void* q_raw, const void* k_raw, const void* v, const float* q_weight,
+                         const float* k_weight, double eps, void* out, void* stream);
+
 /* As gp_decode_step with HOST pointers: brings the inputs to staging inside the blob, runs the
  * step, delivers `out` and `actions` and synchronises `stream`.  When the four input buffers are
  * page-locked, mapped host memory (cudaHostAlloc / cudaHostRegister: "pinned") and q, k, v are

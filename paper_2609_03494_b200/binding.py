@@ -72,6 +72,7 @@ def lib() -> C.CDLL:
     L.gp_step_begin.argtypes = [vp, vp, i32, vp, vp]
     L.gp_attn_layer.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp]
     L.gp_step_end.argtypes = [vp, vp, i32, vp, vp]
+    L.gp_attn_layer_qknorm.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp, C.c_double, vp, vp]
     L.gp_step_abort.argtypes = [vp]
     L.gp_pool_status.argtypes = [vp, C.POINTER(i32)]
     L.gp_async_join.argtypes = [vp, vp]
@@ -153,6 +154,14 @@ def gp_attn_layer(pool: int, layer: int, dev_req_ids_ptr: int, n_req: int, q_ptr
     _check(lib().gp_attn_layer(C.c_void_p(pool), layer, C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(q_ptr),
                                C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr), C.c_void_p(stream)),
            "gp_attn_layer")
+
+
+def gp_attn_layer_qknorm(pool: int, layer: int, dev_req_ids_ptr: int, n_req: int, q_raw_ptr: int, k_raw_ptr: int, v_ptr: int,
+                         q_weight_ptr: int, k_weight_ptr: int, eps: float, out_ptr: int, stream: int) -> None:
+    _check(lib().gp_attn_layer_qknorm(C.c_void_p(pool), layer, C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(q_raw_ptr),
+                                      C.c_void_p(k_raw_ptr), C.c_void_p(v_ptr), C.c_void_p(q_weight_ptr),
+                                      C.c_void_p(k_weight_ptr), eps, C.c_void_p(out_ptr), C.c_void_p(stream)),
+           "gp_attn_layer_qknorm")
 
 
 def gp_step_end(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: int, stream: int) -> None:

@@ -38,6 +38,7 @@ struct gp_pool {
   int* h_err;
   // staging for the host-pointer entry point (inside the blob)
   int* st_ids; void* st_q; void* st_k; void* st_v; float* st_out; int* st_act;
+  __nv_bfloat16* qn; __nv_bfloat16* kn;             // one layer's normalised queries and keys (gp_attn_layer_qknorm)
   // small device words
   int* d_status;
   uint8_t* dbg;                   // gather target of the debug getters
@@ -60,7 +61,7 @@ struct Layout {
       mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
       bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
       evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
-      st_ids, st_q, st_k, st_v, st_out, st_act, total;
+      st_ids, st_q, st_k, st_v, st_out, st_act, qn, kn, total;
   int max_rc;
   long long max_batch_tokens, max_boundary_tokens;
 };
@@ -172,6 +173,8 @@ Layout make_layout(const gp_config& c) {
   } else {
     L.st_ids = L.st_q = L.st_k = L.st_v = L.st_out = L.st_act = 0;
   }
+  L.qn = take(M * c.n_q_heads * d * 2);              // one layer's normalised queries and keys (fused QK-norm)
+  L.kn = take(M * c.n_kv_heads * d * 2);
   L.total = o;
   return L;
 }
@@ -222,6 +225,20 @@ __device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long
   __syncthreads();
 }
 
+// Fused QK-norm of the layer-by-layer entry (null weights: queries and keys arrive normalised).  Queries and keys
+// of the call are raw; the summary CTAs, which read every query row anyway, normalise them per head (RMS over the
+// head dimension, a learned weight per element), rotate the key to its cache form and leave both, rounded to
+// bf16, where the attention kernel then finds them.
+struct GpNorm {
+  const float* wq; const float* wk;
+  double eps;
+  const __nv_bfloat16* k_raw;
+  __nv_bfloat16* qn; __nv_bfloat16* kn;
+};
+
+// double -> float -> bf16, each round-to-nearest-even (the order a host library takes)
+__device__ __forceinline__ __nv_bfloat16 to_bf16(double x) { return __float2bfloat16_rn((float)x); }
+
 // Summary update of one (batch slot, layer, KV head) unit, run by the CTAs of the plan kernel other than the
 // first, concurrently with the planning: Eq. 6 on the un-rotated query of every head of the group (read from
 // one of the request's two buffers, written to the other; the decision step flips the buffers of the requests
@@ -230,7 +247,7 @@ __device__ __forceinline__ void plan_scan(int v, long long w, int& ev, long long
 // kernel's logits.  One warp per (view, head) row; a CTA takes as many units at a time as its warps cover.
 template <int D>
 __device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __restrict__ q, int bi, int lh, int row, int r,
-                            int n_old, int Pr, int started, int par, long long pos) {
+                            int n_old, int Pr, int started, int par, long long pos, const GpNorm& nm) {
   constexpr int PER = D / 32;
   const int lane = threadIdx.x & 31;
   const int G = p.G;
@@ -243,6 +260,50 @@ __device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __re
   float qf[PER];
 #pragma unroll
   for (int e = 0; e < PER; ++e) qf[e] = __bfloat162float(qrow[lane + 32 * e]);
+  if (nm.wq) {
+    // the raw query row becomes the normalised one (Sec. 3.2: the summaries follow the query after its
+    // normalisation and before its rotation); the short view's warp leaves it for the attention kernel
+    double ssq = 0.0;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) ssq += (double)qf[e] * (double)qf[e];
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o2);
+    const double scale = 1.0 / sqrt(ssq / (double)D + nm.eps);
+    __nv_bfloat16* qout = nm.qn + (((size_t)l * n_req + bi) * p.Hq + head) * D;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+      const __nv_bfloat16 v = to_bf16((double)qf[e] * scale * (double)nm.wq[lane + 32 * e]);
+      qf[e] = __bfloat162float(v);
+      if (x == 0) qout[lane + 32 * e] = v;
+    }
+    if (row == 0) {                        // the unit's key row: normalise, rotate to the token's position, leave
+      const __nv_bfloat16* krow = nm.k_raw + (((size_t)l * n_req + bi) * p.Hkv + h) * D;
+      double kv[PER];
+      double ks = 0.0;
+#pragma unroll
+      for (int e = 0; e < PER; ++e) { kv[e] = (double)__bfloat162float(krow[lane + 32 * e]); ks += kv[e] * kv[e]; }
+#pragma unroll
+      for (int o2 = 16; o2 > 0; o2 >>= 1) ks += __shfl_xor_sync(0xffffffffu, ks, o2);
+      const double kscale = 1.0 / sqrt(ks / (double)D + nm.eps);
+#pragma unroll
+      for (int e = 0; e < PER; ++e) kv[e] = kv[e] * kscale * (double)nm.wk[lane + 32 * e];
+      __nv_bfloat16* kout = nm.kn + (((size_t)l * n_req + bi) * p.Hkv + h) * D;
+      if (p.rope_theta != 0.0) {
+#pragma unroll
+        for (int e = 0; e < PER / 2; ++e) {
+          const int j = lane + 32 * e;
+          const double inv = pow(p.rope_theta, -2.0 * (double)j / (double)D);
+          double si, co;
+          sincos((double)pos * inv, &si, &co);
+          kout[j] = to_bf16(kv[e] * co - kv[e + PER / 2] * si);
+          kout[j + D / 2] = to_bf16(kv[e + PER / 2] * co + kv[e] * si);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < PER; ++e) kout[lane + 32 * e] = to_bf16(kv[e]);
+      }
+    }
+  }
   double ovv[PER];
   {
     const double* o0 = p.summ + gp_summ_off(p, l, r, par, x, head);
@@ -298,7 +359,7 @@ __device__ void prepare_row(const GpDev& p, int n_req, const __nv_bfloat16* __re
 __global__ void __launch_bounds__(GP_PLAN_THREADS)
 gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
                const __nv_bfloat16* __restrict__ q, int plan_on, int lh0, int lh_n, int cp_norm, int cp_bnd,
-               int launch_units, int launch_grid, int serial) {
+               int launch_units, int launch_grid, int serial, const GpNorm nm) {
   // serial: number of this decode step (asynchronous boundary mode: a request that reached its boundary at
   // step serial - 1 sits this step out; its counters and pages belong to that step's boundary chain, which may
   // still be running)
@@ -365,8 +426,8 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
         const int rr = s_req[bi];
         if (rr < 0) continue;
         const int st = s_state[bi];
-        if (p.d == 128) prepare_row<128>(p, n_req, q, bi, lh, warp % rows, rr, s_chunks[bi], s_pos[bi], st & 1, (st >> 1) & 1, s_pos64[bi]);
-        else prepare_row<64>(p, n_req, q, bi, lh, warp % rows, rr, s_chunks[bi], s_pos[bi], st & 1, (st >> 1) & 1, s_pos64[bi]);
+        if (p.d == 128) prepare_row<128>(p, n_req, q, bi, lh, warp % rows, rr, s_chunks[bi], s_pos[bi], st & 1, (st >> 1) & 1, s_pos64[bi], nm);
+        else prepare_row<64>(p, n_req, q, bi, lh, warp % rows, rr, s_chunks[bi], s_pos[bi], st & 1, (st >> 1) & 1, s_pos64[bi], nm);
       }
     }
     return;
@@ -875,6 +936,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
     pool->chain_grid = slots;
   }
   pool->dbg = base + L.dbg;
+  pool->qn = reinterpret_cast<__nv_bfloat16*>(base + L.qn);
+  pool->kn = reinterpret_cast<__nv_bfloat16*>(base + L.kn);
   if (cfg->host_staging) {
     pool->st_ids = reinterpret_cast<int*>(base + L.st_ids);
     pool->st_q = base + L.st_q; pool->st_k = base + L.st_k; pool->st_v = base + L.st_v;
@@ -950,7 +1013,7 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
 // CTA 0 plans (when plan_on); the others update the query summaries of the units [lh0, lh0 + lh_n)
 static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_t* actions, const void* q, int plan_on,
                         int lh0, int lh_n, cudaStream_t s, bool pdl, bool by_layer = false, const GpDev* dev = nullptr,
-                        int attn_grid = 0) {
+                        int attn_grid = 0, const GpNorm* norm = nullptr) {
   const int rd = cur_copy(pool);
   const GpDev d = with_state(pool, dev ? *dev : pool->dev, rd, rd ^ 1);     // the plan writes the next step's copy
   const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
@@ -959,7 +1022,8 @@ static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_
   const int prep = (int)(want < room ? want : room);
   gp_launch(gp_plan_kernel, 1 + prep, GP_PLAN_THREADS, 0, s, pdl, d, ids, n_req, actions,
             static_cast<const __nv_bfloat16*>(q), plan_on, lh0, lh_n, d.chunk_pages, d.bchunk_pages,
-            by_layer ? d.Hkv : d.L * d.Hkv, attn_grid ? attn_grid : pool->attn_grid, (int)(pool->serial & 0x3fffffff));
+            by_layer ? d.Hkv : d.L * d.Hkv, attn_grid ? attn_grid : pool->attn_grid, (int)(pool->serial & 0x3fffffff),
+            norm ? *norm : GpNorm{nullptr, nullptr, 0.0, nullptr, nullptr, nullptr});
 }
 
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
@@ -1090,6 +1154,40 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
   const int lh0 = layer * d.Hkv, lh_n = d.Hkv;
   launch_plan(pool, dev_req_ids, n_req, nullptr, qb, 0, lh0, lh_n, s, true);
   gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n);
+  gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
+  pool->launch_count += 3;
+  pool->step_layers_done += 1;
+  pool->step_layer_seen[layer] = 1;
+  GP_CUDA(cudaGetLastError());
+  return GP_OK;
+}
+
+int gp_attn_layer_qknorm(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req, const void* q_raw,
+                         const void* k_raw, const void* v, const float* q_weight, const float* k_weight, double eps, void* out,
+                         void* stream) {
+  if (!pool || !pool->step_open || n_req != pool->step_n_req) return pool && !pool->step_open ? GP_ERR_STATE : GP_ERR_INVALID;
+  if (layer < 0 || layer >= pool->cfg.n_layers || !dev_req_ids || !q_raw || !k_raw || !v || !out || !q_weight || !k_weight)
+    return GP_ERR_INVALID;
+  if (misaligned(q_raw, 16) || misaligned(k_raw, 16) || misaligned(v, 16) || misaligned(out, 16) || misaligned(dev_req_ids, 4) ||
+      misaligned(q_weight, 4) || misaligned(k_weight, 4) || !(eps >= 0.0))
+    return GP_ERR_INVALID;
+  if (pool->step_layer_seen[layer]) return GP_ERR_STATE;          // every layer once
+  GP_CUDA(cudaSetDevice(pool->device));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const GpDev& d = pool->dev;
+  const size_t qs = (size_t)layer * n_req * d.Hq * d.d, ks = (size_t)layer * n_req * d.Hkv * d.d;
+  auto shifted = [](const void* ptr, size_t bytes) { return reinterpret_cast<uintptr_t>(ptr) - bytes; };
+  const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(shifted(q_raw, qs * 2));
+  const __nv_bfloat16* vb = reinterpret_cast<const __nv_bfloat16*>(shifted(v, ks * 2));
+  float* ob = reinterpret_cast<float*>(shifted(out, qs * 4));
+  GpNorm nm;
+  nm.wq = q_weight; nm.wk = k_weight; nm.eps = eps;
+  nm.k_raw = reinterpret_cast<const __nv_bfloat16*>(shifted(k_raw, ks * 2));
+  nm.qn = reinterpret_cast<__nv_bfloat16*>(shifted(pool->qn, qs * 2));
+  nm.kn = reinterpret_cast<__nv_bfloat16*>(shifted(pool->kn, ks * 2));
+  const int lh0 = layer * d.Hkv, lh_n = d.Hkv;
+  launch_plan(pool, dev_req_ids, n_req, nullptr, qb, 0, lh0, lh_n, s, true, false, nullptr, 0, &nm);
+  gp_launch_attention(d, dev_req_ids, n_req, nm.qn, nm.kn, vb, ob, pool->attn_grid, s, true, lh0, lh_n);
   gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
   pool->launch_count += 3;
   pool->step_layers_done += 1;

@@ -837,3 +837,73 @@ def test_preempted_request_is_readmitted_with_its_history_and_fresh_summaries():
         assert counters[7] == 0 and n_free == ora.n_free()
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("rope_theta,hq,hkv,d", [(0.0, 8, 2, 64), (1e4, 8, 2, 128), (1e6, 16, 2, 64)])
+def test_layer_entry_with_fused_query_key_normalisation(rope_theta, hq, hkv, d):
+    """gp_attn_layer_qknorm takes the projections' raw outputs; the oracle is fed what a plain implementation of
+    the model's normalisation gives: per head x / sqrt(mean(x^2) + eps) * weight in float64, the key then rotated
+    to its position, both rounded to bf16.  Everything downstream (attention, summaries taken after the
+    normalisation and before the rotation, boundaries, retained sets) must agree as in the other lockstep tests."""
+    import torch
+    L, b, eps = 3, 16, 1e-6
+    kw = dict(n_pages=48, max_pages_per_req=5, max_requests=4, k_loc=4, tau=-0.03, rope_theta=rope_theta)   # the cap forces compressions
+    gpu = B.Pool(B.make_config(L, hq, hkv, d, **kw))
+    ora = O.OraclePool(O.OracleConfig(L, hq, hkv, d, **kw))
+    rng = np.random.default_rng(31)
+    bits = lambda *shape: W.f32_to_bf16_bits((2.5 * rng.standard_normal(shape)).astype(np.float32))
+    f = W.bf16_bits_to_f64
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to("cuda:0")
+    wq = (1.0 + 0.3 * rng.standard_normal((L, d))).astype(np.float32)
+    wk = (1.0 + 0.3 * rng.standard_normal((L, d))).astype(np.float32)
+    wq_d, wk_d = torch.from_numpy(wq).cuda(), torch.from_numpy(wk).cuda()
+    round_bf16 = lambda x: W.f32_to_bf16_bits(x.astype(np.float32))              # double -> float -> bf16
+
+    def normalise(x_bits, w):                                                      # [.., heads, d] per head
+        x = f(x_bits)
+        return x / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps) * w.astype(np.float64)
+
+    try:
+        prompts = (21, 40, 13)
+        for n0 in prompts:
+            kp, vp = bits(L, n0, hkv, d), bits(L, n0, hkv, d)
+            assert gpu.request_add(-1, 0, kp, vp, n0, 0)[0] == B.GP_OK
+            assert ora.request_add(-1, 0, f(kp), f(vp), n0, 0)[0] == O.OK
+        n_req = len(prompts)
+        ids = torch.arange(n_req, dtype=torch.int32, device="cuda:0")
+        seen = {}
+        for t in range(60):
+            q_raw, k_raw, v = bits(L, n_req, hq, d), bits(L, n_req, hkv, d), bits(L, n_req, hkv, d)
+            pos = [ora.request_state(r)[2] for r in range(n_req)]
+            q_n = np.stack([round_bf16(normalise(q_raw[l], wq[l])) for l in range(L)])
+            k_n = np.stack([np.stack([round_bf16(O.rope(normalise(k_raw[l, r], wk[l]), pos[r], rope_theta)) for r in range(n_req)])
+                            for l in range(L)])
+            rec = ora.decode_step(list(range(n_req)), f(q_n), f(k_n), f(v))
+            out = torch.zeros((L, n_req, hq, d), dtype=torch.float32, device="cuda:0")
+            act = torch.zeros(n_req, dtype=torch.int32, device="cuda:0")
+            qd, kd, vd = dev(q_raw), dev(k_raw), dev(v)
+            s_ = gpu.stream()
+            B.gp_step_begin(gpu.handle, ids.data_ptr(), n_req, act.data_ptr(), s_)
+            for l in rng.permutation(L):
+                l = int(l)
+                B.gp_attn_layer_qknorm(gpu.handle, l, ids.data_ptr(), n_req, qd[l].data_ptr(), kd[l].data_ptr(), vd[l].data_ptr(),
+                                       wq_d[l].data_ptr(), wk_d[l].data_ptr(), eps, out[l].data_ptr(), s_)
+            B.gp_step_end(gpu.handle, ids.data_ptr(), n_req, act.data_ptr(), s_)
+            assert act.cpu().tolist() == rec.actions.tolist(), t
+            assert np.abs(out.cpu().numpy() - rec.out).max() <= LS.ATTN_MAX_ABS, t
+            for a in rec.actions.tolist():
+                seen[a] = seen.get(a, 0) + 1
+        assert seen.get(B.GP_ACT_GROW, 0) > 0 and seen.get(B.GP_ACT_COMPRESS, 0) + seen.get(B.GP_ACT_COMPRESS_FALLBACK, 0) > 0, seen
+        for r in range(n_req):
+            assert B.gp_debug_request(gpu.handle, r, 5)[:3] == ora.request_state(r)[:3]
+            g, o = B.gp_debug_summaries(gpu.handle, r, L, hq, d), ora.summaries(r)
+            assert (np.linalg.norm(g - o, axis=-1) / np.linalg.norm(o, axis=-1)).max() <= LS.SUMMARY_REL
+            n = ora.request_state(r)[1]
+            for l in range(L):
+                for h in range(hkv):
+                    assert np.array_equal(B.gp_debug_retained(gpu.handle, r, l, h, n), ora.retained(r, l, h))
+                    kk, _ = B.gp_debug_kv(gpu.handle, r, l, h, n, d)
+                    assert np.array_equal(f(kk), ora.requests[r].K[l, h, :n]), "the cached keys are not the normalised, rotated ones"
+        assert B.gp_debug_pool(gpu.handle)[2][7] == 0
+    finally:
+        gpu.close()
