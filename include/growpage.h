@@ -88,12 +88,22 @@ typedef struct gp_config {
   int32_t n_q_heads;         /* H_q, a multiple of n_kv_heads; group size G = H_q/H_kv <= 8        */
   int32_t n_kv_heads;        /* H_kv                                                               */
   int32_t head_dim;          /* d_h: 64 or 128                                                     */
-  int32_t page_size;         /* b: tokens per page, 16                                             */
+  int32_t page_size;         /* b: tokens per page, a power of two from 16 to 256 (the paper's default: 256).
+                                The page is the unit in which capacity grows, local-quota blocks are formed
+                                and slots are freed; n_pages, max_pages_per_req, initial_pages and every
+                                page count the calls report are in these pages.  Inside, a page is a group
+                                of page_size / 16 tiles of 16 tokens that are taken, shared and returned
+                                together                                                            */
   int32_t max_requests;      /* M: summary slots = highest request id + 1 (App. D.1, default 512)  */
-  int32_t max_pages_per_req; /* per-request page cap and page-table stride, >= 1; at most 62 000
-                                (the selection kernel keeps one bit per candidate token on chip)  */
-  int32_t recent_window;     /* |R_t| protected tokens; must equal page_size                       */
-  int32_t k_loc;             /* block-local retention quota of Eq. 10 (default page_size / 4)      */
+  int32_t max_pages_per_req; /* per-request page cap and page-table stride, >= 1; at most about 61 000
+                                * 16 / page_size (the selection kernel keeps one bit per candidate token on
+                                chip)                                                             */
+  int32_t recent_window;     /* |R_t| protected newest tokens: 16 (the paper's default; equals the page at
+                                page_size 16).  With a larger page the working sets of Eq. 7 are taken over
+                                the history minus the newest page, the candidates of Eq. 10 are the history
+                                minus these 16 tokens, each with its own softmax (App. D.1, Sec. 3.3)   */
+  int32_t k_loc;             /* block-local retention quota of Eq. 10, at most page_size (default 4 = a
+                                quarter of the default page of 16; the paper's 64 at its page of 256)  */
   int32_t host_staging;      /* 1: reserve staging so that gp_decode_step_host can be used         */
   int32_t policy;            /* GP_POLICY_*: how Delta_t becomes an action (default: demand)       */
   int32_t policy_seed;       /* GP_POLICY_RANDOM: seed of its counter-based draws                  */

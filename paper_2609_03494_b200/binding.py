@@ -373,7 +373,7 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
                 beta_s: float = 0.9, beta_l: float = 0.999, top_p: float = 0.99, tau: float = 0.0,
                 rope_theta: float = 0.0, policy: int = 0, policy_seed: int = 0, p_compress: float = 0.7,
                 shrink_below: float = -0.005, min_capacity: int = 1024, async_boundary: bool = False,
-                async_slots: int = 0, max_boundary_tokens: int = 0, demand_metric: int = 0) -> gp_config:
+                async_slots: int = 0, max_boundary_tokens: int = 0, demand_metric: int = 0, page_size: int = 16) -> gp_config:
     cfg = gp_config_default()
     cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
     cfg.n_pages, cfg.max_pages_per_req, cfg.max_requests = n_pages, max_pages_per_req, max_requests
@@ -383,4 +383,5 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
     cfg.shrink_below, cfg.min_capacity = shrink_below, min_capacity
     cfg.async_boundary, cfg.async_slots, cfg.max_boundary_tokens = 1 if async_boundary else 0, async_slots, max_boundary_tokens
     cfg.demand_metric = demand_metric
+    cfg.page_size = page_size
     return cfg

@@ -445,7 +445,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       const int4 acc = __ldcg(reinterpret_cast<const int4*>(p.bnd_acc) + e);
       s_free[e] = p.async ? (e < top0 ? __ldcg(p.free_stack + top0 - 1 - e) : 0) : __ldcg(p.free_peek + 1 + e);
       const int r = inf.y, Pr = inf.z;
-      const int nC = (Pr - 1) * GP_PAGE;
+      const int nC = (Pr - p.sub) * GP_PAGE;                // |C_t| of Eq. 7: history minus the newest page of the method
       // Eq. 8 with a common |C|: Delta = (sum K^S - sum K^L) / (N |C|), one division of exact integers
       double delta = 0.0;
       int want = 1;
@@ -469,7 +469,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
           zz ^= zz >> 31;
           want = !((double)(zz >> 11) * (1.0 / 9007199254740992.0) < p.p_compress);
         } else if (p.policy == GP_POLICY_SHRINK) {            // Eq. 13: the third action, where it is admissible
-          if (!want && delta < p.shrink_below && Pr - 1 >= p.min_pages_after_shrink) want = 16;
+          if (!want && delta < p.shrink_below && Pr - p.sub >= p.min_pages_after_shrink) want = 16;
         }
       }
       p.delta[r] = delta;
@@ -501,20 +501,24 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     int top = top0;
     int n_cmp = 0, chunks = 0;
     unsigned long long grow = 0, comp = 0, fall = 0, stall = 0, cow = 0, scored = 0, shr = 0;
+    const int sub = p.sub;
     for (int k = 0; k < n_bnd; ++k) {                    // pass 1: grants, ascending request id
       const int e = s_order[k];
       const int r = s_req[e], Pr = s_P[e], bi = s_bi[e];
-      scored += (unsigned long long)(Pr - 1) * GP_PAGE;
-      if ((s_want[e] & 1) && Pr < p.cap && top > 0) {
-        const int page = s_free[top0 - top];
-        --top;
-        p.refcount[page] = 1;
-        p.page_table[(size_t)r * p.cap + Pr] = page;
-        p.wP[r] = Pr + 1;
+      scored += (unsigned long long)(Pr - sub) * GP_PAGE;
+      if ((s_want[e] & 1) && Pr + sub <= p.cap && top >= sub) {
+        // one page of the method: `sub` tiles from the top of the free list
+        for (int t = 0; t < sub; ++t) {
+          const int page = (sub == 1 && !p.async) ? s_free[top0 - top] : p.free_stack[top - 1];
+          --top;
+          p.refcount[page] = 1;
+          p.page_table[(size_t)r * p.cap + Pr + t] = page;
+        }
+        p.wP[r] = Pr + sub;
         report(bi, r, GP_ACT_GROW);
         s_want[e] |= 2;
         ++grow;
-      } else if (Pr == 1) {
+      } else if (Pr == sub) {
         report(bi, r, GP_ACT_STALLED);
         s_want[e] |= 4;
         ++stall;
@@ -541,8 +545,8 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       else { report(bi, r, GP_ACT_COMPRESS); ++comp; }
       // a compression frees one page worth of slots; a Shrink frees two and gives the last page back (the
       // compaction kernel returns it once nothing reads it any more)
-      p.wn[r] = (s_P[e] - (shrink ? 2 : 1)) * GP_PAGE;
-      if (shrink) p.wP[r] = s_P[e] - 1;
+      p.wn[r] = (s_P[e] - (shrink ? 2 : 1) * sub) * GP_PAGE;
+      if (shrink) p.wP[r] = s_P[e] - sub;
       p.n_pristine[r] = 0;
       s_want[e] |= 8;
     }
@@ -568,9 +572,9 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     const int* table = p.page_table + (size_t)r * p.cap;
     int* shadow = p.shadow + (size_t)r * p.cap;
     int running = 0;
-    for (int j0 = 0; j0 < Pr - 1; j0 += 32) {
+    for (int j0 = 0; j0 < Pr - p.sub; j0 += 32) {
       const int j = j0 + lane;
-      const bool sh = j < Pr - 1 && p.refcount[table[j]] > 1;
+      const bool sh = j < Pr - p.sub && p.refcount[table[j]] > 1;
       const unsigned mask = __ballot_sync(0xffffffffu, sh);
       if (sh) {
         const int newp = p.free_stack[base - 1 - (running + __popc(mask & ((1u << lane) - 1u)))];
@@ -802,7 +806,7 @@ __device__ __noinline__ void merge_partials(const GpDev& p, int n_req, float* __
 struct SelGeom {
   static constexpr size_t BUF_BYTES = SEL_CAP * sizeof(double);
   static constexpr size_t H_BYTES = (size_t)FB_PAD * 12;
-  static constexpr size_t MISC_BYTES = SEL_NW * 8 + SEL_NW * 4 + 8 * 8 + 32 * 4 + 16 * 4 + (SEL_NW * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
+  static constexpr size_t MISC_BYTES = SEL_NW * 8 + SEL_NW * 4 + 8 * 8 + 2 * GP_MAX_BLK * 4 + 16 * 4 + (SEL_NW * 16 + 32) * 8 + 32 * 8 + 32 * 4 + 3 * CBINS * 4;
 };
 
 // shared memory of the selection kernel
@@ -813,7 +817,7 @@ struct SelSmem {
   unsigned long long* wsum;          // [SEL_NW]
   unsigned* wc;                      // [SEL_NW]
   long long* s_res;                  // [8]
-  int* ev;                           // [32]
+  int* ev;                           // [2 * GP_MAX_BLK] evicted slots of the job
   int* s_i;                          // [16]
   double* red;                       // [SEL_NW][16]
   double* sM;                        // [16]
@@ -834,7 +838,7 @@ __device__ __forceinline__ SelSmem sel_smem_at(uint8_t* smem) {      // smem: 25
   S.wc = reinterpret_cast<unsigned*>(S.wsum + SEL_NW);
   S.s_res = reinterpret_cast<long long*>(S.wc + SEL_NW);
   S.ev = reinterpret_cast<int*>(S.s_res + 8);
-  S.s_i = S.ev + 32;
+  S.s_i = S.ev + 2 * GP_MAX_BLK;
   S.red = reinterpret_cast<double*>(S.s_i + 16);
   S.sM = S.red + SEL_NW * 16;
   S.sZ = S.sM + 16;
@@ -895,19 +899,29 @@ __device__ __forceinline__ void sel_job(const GpDev& p, const SelSmem& S, const 
     }
     return;
   }
-  // ---- Eq. 10, block-local quota: the k' best slots of every page of C (score desc, slot asc) -------------
-  const int nblk = nC / GP_PAGE;
+  // ---- Eq. 10, block-local quota: the k' best slots of every block of C (score desc, slot asc); a block is a
+  // page of the method, the last one short when the protected window is smaller than the page -----------------
+  const int blk = p.blk;
+  const int nblk = (nC + blk - 1) / blk;
   const int K_t = nC - ne;
   const int kq = min(p.k_loc, K_t / nblk);
   if (kq > 0) {
     for (int i = tid; i < nC; i += SEL_T) {
       const double s = a[i];
-      const int b0 = i & ~15;
       int rank = 0;
+      if (blk == GP_PAGE) {
+        const int b0 = i & ~15;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const double sj = a[b0 + j];
-        rank += (sj > s) || (sj == s && (b0 + j) < i);
+        for (int j = 0; j < 16; ++j) {
+          const double sj = a[b0 + j];
+          rank += (sj > s) || (sj == s && (b0 + j) < i);
+        }
+      } else {
+        const int b0 = (i / blk) * blk, b1 = min(b0 + blk, nC);
+        for (int j = b0; j < b1; ++j) {
+          const double sj = a[j];
+          rank += (sj > s) || (sj == s && j < i);
+        }
       }
       if (rank < kq) atomicOr(&S.loc[i >> 5], 1u << (i & 31));
     }
@@ -917,8 +931,8 @@ __device__ __forceinline__ void sel_job(const GpDev& p, const SelSmem& S, const 
   if (!uniform || !evict_fast(a, nC, S.loc, S.H, S.wc, S.s_res, S.flist, S.flist_slot, &S.s_i[6], S.ev, (unsigned)ne))
     evict_general(p, a, nC, S.loc, S.hcnt, S.wc, S.s_res, S.s_i, S.ev, (unsigned)ne);
   __syncthreads();
-  if (tid < ne) {                                   // the evicted slots in ascending order, by rank
-    const int mine = S.ev[tid];
+  for (int t = tid; t < ne; t += SEL_T) {                    // the evicted slots in ascending order, by rank
+    const int mine = S.ev[t];
     int rank = 0;
     for (int j = 0; j < ne; ++j) rank += (S.ev[j] < mine);
     evout[rank] = mine;
@@ -971,7 +985,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
         const int4 inf = p.bnd_info[2 * e];
         const int* table = p.page_table + (size_t)inf.y * p.cap;
         int ksh = 0;
-        for (int j = tid; j < inf.z - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
+        for (int j = tid; j < inf.z - p.sub; j += 32) ksh += (p.refcount[table[j]] > 1);
 #pragma unroll
         for (int o2 = 16; o2 > 0; o2 >>= 1) ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
         if (tid == 0) p.bnd_acc[4 * e + 2] = ksh;
@@ -981,7 +995,7 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     const long long u = item / NT;
     const int job = (int)(item % NT);               // 0: K^S, 1: K^L, 2: eviction list, 3: a Shrink's eviction list
     const int task = job < 2 ? job : 2;
-    const int ne = (SHR && job == 3) ? 2 * GP_PAGE : GP_PAGE;
+    const int ne = (SHR && job == 3) ? 2 * p.blk : p.blk;        // slots a compression (a Shrink) frees
     const int bidx = (int)(u / LH), lh = (int)(u % LH);
     const int l = lh / p.Hkv, h = lh % p.Hkv;
     const bool is_first = item == (long long)blockIdx.x;
@@ -989,15 +1003,18 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     const int4 inf2 = is_first ? inf2_first : p.bnd_info[2 * bidx + 1];    // {offset into the logit scratch}
     const int r = inf.y, Pr = inf.z;
     const long long off = (long long)(unsigned)inf2.x | ((long long)inf2.y << 32);
-    const int nC = (Pr - 1) * GP_PAGE;
+    // two supports (they coincide when the page is 16 tokens): the working sets of Eq. 7 leave out the newest page
+    // of the method, the eviction candidates of Eq. 10 only the protected window, the newest 16-token tile
+    const int nC_d = (Pr - p.sub) * GP_PAGE, nC_e = (Pr - 1) * GP_PAGE;
+    const int nC = task < 2 ? nC_d : nC_e;
     int* Kout = p.Kx + (((size_t)r * p.L + l) * p.Hkv + h) * 2;
-    int* evout = (SHR && job == 3) ? p.evict2 + (size_t)u * 2 * GP_PAGE : p.evict + (size_t)u * GP_PAGE;
+    int* evout = (SHR && job == 3) ? p.evict2 + (size_t)u * 2 * p.blk : p.evict + (size_t)u * p.blk;
     __syncthreads();
-    if (nC == 0) {
+    if (nC_d == 0) {                         // one page of the method: nothing to estimate from, nothing to evict
       if (tid == 0 && task < 2) Kout[task] = 0;
       continue;
     }
-    if (SHR && job == 3 && Pr - 1 < p.min_pages_after_shrink) continue;      // this boundary cannot be a Shrink
+    if (SHR && job == 3 && Pr - p.sub < p.min_pages_after_shrink) continue;      // this boundary cannot be a Shrink
     const size_t view_stride = (size_t)p.z_stride * G;
     const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;   // [2 views][nC][G] exp(logit - page max)
     const double* zs = p.zstat + ((size_t)lh * (p.max_boundary_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
@@ -1040,18 +1057,18 @@ gp_merge_kernel(const __grid_constant__ GpDev p, int n_req, float* __restrict__ 
 // shared memory of the compaction
 struct CmpSmem {
   int4* s_info;      // [GP_MAX_REQ + 1] compressing requests: {request, P, boundary index, first chunk}
-  int* ev;           // [2 b]
+  int* ev;           // [2 * GP_MAX_BLK] slots the unit's compression (or Shrink) evicts
   int* s_i;          // [8]
   int* s_dst;        // [MOVE_TOK] per source slot of the chunk: destination slot (-1: stays or goes)
   int* s_spage;      // [MOVE_TOK] source page
   int* s_dpage;      // [MOVE_TOK] destination page
 };
-constexpr size_t CMP_SMEM_BYTES = (GP_MAX_REQ + 1) * 16 + (2 * GP_PAGE + 8 + 3 * MOVE_TOK) * 4;
+constexpr size_t CMP_SMEM_BYTES = (GP_MAX_REQ + 1) * 16 + (2 * GP_MAX_BLK + 8 + 3 * MOVE_TOK) * 4;
 __device__ __forceinline__ CmpSmem cmp_smem_at(uint8_t* base) {       // base: 16-byte aligned, CMP_SMEM_BYTES
   CmpSmem C;
   C.s_info = reinterpret_cast<int4*>(base);
   C.ev = reinterpret_cast<int*>(base + (GP_MAX_REQ + 1) * 16);
-  C.s_i = C.ev + 2 * GP_PAGE;
+  C.s_i = C.ev + 2 * GP_MAX_BLK;
   C.s_dst = C.s_i + 8;
   C.s_spage = C.s_dst + MOVE_TOK;
   C.s_dpage = C.s_spage + MOVE_TOK;
@@ -1106,40 +1123,40 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
     const int* shadow = p.shadow + (size_t)r * p.cap;
     const int n_src = Pr * GP_PAGE;
     const int c0 = j * MOVE_TOK;
-    // second round trip: the eviction list, and for every source slot of the chunk its page and the pages
-    // before it that it can move to (a slot moves down by at most one page, two at a Shrink) with their
-    // copy-on-write targets
+    // second round trip: the eviction list and, for every source slot of the chunk, its page and its
+    // copy-on-write target
     const bool shrink = SHR && (inf.z & CMP_SHRINK) != 0;
     const int e_bnd = inf.z & (CMP_SHRINK - 1);
-    const int ne = shrink ? 2 * GP_PAGE : GP_PAGE;
-    int t0 = 0, s0 = -1, tm = 0, sm = -1, tm2 = 0, sm2 = -1;
+    const int ne = shrink ? 2 * p.blk : p.blk;             // slots freed: one page of the method, two at a Shrink
+    int t0 = 0, s0 = -1;
     const int my_i = c0 + tid;                             // the slot this thread plans (first MOVE_TOK threads)
     if (tid < MOVE_TOK && my_i < n_src) {
       const int pg = my_i / GP_PAGE;
       t0 = table[pg]; s0 = shadow[pg];
-      if (pg > 0) { tm = table[pg - 1]; sm = shadow[pg - 1]; }
-      if (shrink && pg > 1) { tm2 = table[pg - 2]; sm2 = shadow[pg - 2]; }
     }
-    if (tid < ne) ev[tid] = shrink ? p.evict2[((size_t)e_bnd * LH + lh) * 2 * GP_PAGE + tid]
-                                   : p.evict[((size_t)e_bnd * LH + lh) * GP_PAGE + tid];
+    for (int t = tid; t < ne; t += CT)
+      ev[t] = shrink ? p.evict2[((size_t)e_bnd * LH + lh) * 2 * p.blk + t] : p.evict[((size_t)e_bnd * LH + lh) * p.blk + t];
     __syncthreads();
     int tokv = 0, tok_dst = -1, tok_page = 0;
     if (tid < MOVE_TOK) {
       int ds = -1, dpage = 0;
       if (my_i < n_src) {
         int sh = 0; bool evicted = false;
+        if (ne == GP_PAGE) {
 #pragma unroll
-        for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < my_i); evicted |= (ev[e2] == my_i); }
-        if (shrink) {
-#pragma unroll
-          for (int e2 = GP_PAGE; e2 < 2 * GP_PAGE; ++e2) { sh += (ev[e2] < my_i); evicted |= (ev[e2] == my_i); }
+          for (int e2 = 0; e2 < GP_PAGE; ++e2) { sh += (ev[e2] < my_i); evicted |= (ev[e2] == my_i); }
+        } else {
+          for (int e2 = 0; e2 < ne; ++e2) { sh += (ev[e2] < my_i); evicted |= (ev[e2] == my_i); }
         }
         const int pg = my_i / GP_PAGE;
         const bool cow = (pg < Pr - 1) && (s0 >= 0);
         if (!evicted && (sh > 0 || cow)) {
           ds = my_i - sh;
-          const int back = pg - ds / GP_PAGE;              // 0, 1, or (Shrink only) 2 pages down
-          dpage = back == 0 ? (s0 >= 0 ? s0 : t0) : back == 1 ? (sm >= 0 ? sm : tm) : (sm2 >= 0 ? sm2 : tm2);
+          // the destination tile: as many tiles down as evicted slots lie before this one (third round trip,
+          // from the L2, only for slots that move across a tile boundary)
+          const int dpg = ds / GP_PAGE;
+          if (dpg == pg) dpage = s0 >= 0 ? s0 : t0;
+          else { const int sd = shadow[dpg]; dpage = sd >= 0 ? sd : table[dpg]; }
           tokv = p.tok[gp_tok_off(p, l, t0, h) + (my_i % GP_PAGE)];
           tok_dst = ds; tok_page = dpage;
         }
@@ -1178,8 +1195,12 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
       // consumed above), and the stores below are issued after the flag has been seen.
       if (!((p.withhold & GP_WITHHOLD_CHUNK) && j == 0))               // (test support: see GP_WITHHOLD_CHUNK)
         *reinterpret_cast<volatile int*>(p.cflags + item) = stamp;      // "my sources are read"
-      if (j > 0) {                                          // the previous chunk's tail is my first destination
-        volatile int* prev = reinterpret_cast<volatile int*>(p.cflags + item - 1);
+      // my destinations reach back as far as a slot can move down, `ne` slots: into the sources of the chunks
+      // before this one, all of which must have been read (tickets are handed out in order, so those chunks are
+      // running or done)
+      const int reach = (ne + MOVE_TOK - 1) / MOVE_TOK;
+      for (int back = 1; back <= reach && back <= j; ++back) {
+        volatile int* prev = reinterpret_cast<volatile int*>(p.cflags + item - back);
         unsigned it = 0;
         while (*prev != stamp && it < p.spin_limit) ++it;
         if (it >= p.spin_limit) atomicOr(p.err, GP_E_SPIN_CMP);
@@ -1242,12 +1263,14 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
         if (lane == 0 && mask) *reinterpret_cast<volatile int*>(p.free_top) = base + __popc(mask);
         __syncwarp();
       }
-      if (SHR && (s_info[ci].z & CMP_SHRINK) && lane == 0) {      // the page the request no longer owns
-        const int last = table[Pr - 1];
-        if (atomicSub(&p.refcount[last], 1) == 1) {
-          const int top = *reinterpret_cast<volatile int*>(p.free_top);
-          p.free_stack[top] = last;
-          *reinterpret_cast<volatile int*>(p.free_top) = top + 1;
+      if (SHR && (s_info[ci].z & CMP_SHRINK) && lane == 0) {      // the page of the method the request no longer owns
+        for (int t = p.sub; t >= 1; --t) {
+          const int last = table[Pr - t];
+          if (atomicSub(&p.refcount[last], 1) == 1) {
+            const int top = *reinterpret_cast<volatile int*>(p.free_top);
+            p.free_stack[top] = last;
+            *reinterpret_cast<volatile int*>(p.free_top) = top + 1;
+          }
         }
       }
       __syncwarp();
@@ -1300,7 +1323,7 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
           const int4 inf = p.bnd_info[2 * e];
           const int* table = p.page_table + (size_t)inf.y * p.cap;
           int ksh = 0;
-          for (int j = tid; j < inf.z - 1; j += 32) ksh += (p.refcount[table[j]] > 1);
+          for (int j = tid; j < inf.z - p.sub; j += 32) ksh += (p.refcount[table[j]] > 1);
 #pragma unroll
           for (int o2 = 16; o2 > 0; o2 >>= 1) ksh += __shfl_xor_sync(0xffffffffu, ksh, o2);
           if (tid == 0) p.bnd_acc[4 * e + 2] = ksh;
@@ -1310,22 +1333,25 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
       const long long u = item / NT;
       const int job = (int)(item % NT);
       const int task = job < 2 ? job : 2;
-      const int ne = (SHR && job == 3) ? 2 * GP_PAGE : GP_PAGE;
+      const int ne = (SHR && job == 3) ? 2 * p.blk : p.blk;        // slots a compression (a Shrink) frees
       const int bidx = (int)(u / LH), lh = (int)(u % LH);
       const int l = lh / p.Hkv, h = lh % p.Hkv;
       const int4 inf = p.bnd_info[2 * bidx];
       const int4 inf2 = p.bnd_info[2 * bidx + 1];
       const int r = inf.y, Pr = inf.z;
       const long long off = (long long)(unsigned)inf2.x | ((long long)inf2.y << 32);
-      const int nC = (Pr - 1) * GP_PAGE;
+      // two supports (they coincide when the page is 16 tokens): the working sets of Eq. 7 leave out the newest page
+    // of the method, the eviction candidates of Eq. 10 only the protected window, the newest 16-token tile
+    const int nC_d = (Pr - p.sub) * GP_PAGE, nC_e = (Pr - 1) * GP_PAGE;
+    const int nC = task < 2 ? nC_d : nC_e;
       int* Kout = p.Kx + (((size_t)r * p.L + l) * p.Hkv + h) * 2;
-      int* evout = (SHR && job == 3) ? p.evict2 + (size_t)u * 2 * GP_PAGE : p.evict + (size_t)u * GP_PAGE;
+      int* evout = (SHR && job == 3) ? p.evict2 + (size_t)u * 2 * p.blk : p.evict + (size_t)u * p.blk;
       __syncthreads();
-      if (nC == 0) {
+      if (nC_d == 0) {                         // one page of the method: nothing to estimate from, nothing to evict
         if (tid == 0 && task < 2) Kout[task] = 0;
         continue;
       }
-      if (SHR && job == 3 && Pr - 1 < p.min_pages_after_shrink) continue;
+      if (SHR && job == 3 && Pr - p.sub < p.min_pages_after_shrink) continue;
       const size_t view_stride = (size_t)p.z_stride * G;
       const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;
       const double* zs = p.zstat + ((size_t)lh * (p.max_boundary_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;

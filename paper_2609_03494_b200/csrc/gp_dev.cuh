@@ -17,7 +17,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#define GP_PAGE 16             // tokens per page (b)
+#define GP_PAGE 16             // tokens per physical page: the unit of the K/V tiles, the page tables and the free list.
+                               // The method's page (gp_config.page_size, b = 16 ... 256 tokens: the unit in which capacity
+                               // grows, blocks are formed and slots are freed) is `sub` of these, always taken together.
+#define GP_MAX_BLK 256         // largest page_size
 #define GP_SPIN_LIMIT (1u << 21)
 #define GP_MAX_REQ 1024        // upper limit of max_requests (shared-memory arrays are sized by it)
 #define GP_MOVE_TOK 64         // source slots per compaction chunk
@@ -58,7 +61,8 @@ enum {
 
 struct GpDev {
   // geometry
-  int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;
+  int L, Hq, Hkv, G, d, M, cap, k_loc, chunk_pages, max_rc;     // cap, n_pages: in physical pages
+  int sub, blk;                          // physical pages per page of the method (page_size / 16), and its tokens (page_size)
   long long n_pages, max_batch_tokens;
   long long max_boundary_tokens;         // bound on the summed candidate tokens of one step's boundary requests
   unsigned spin_limit;                   // iterations after which a bounded wait gives up (GP_SPIN_LIMIT; tests shorten it)
@@ -72,7 +76,8 @@ struct GpDev {
   unsigned long long policy_seed;
   double p_compress;
   double shrink_below;                   // Eq. 13: Shrink under this
-  int min_pages_after_shrink;            // a Shrink must leave at least this many pages (the minimum capacity)
+  int min_pages_after_shrink;            // a Shrink must leave at least this many physical pages (the minimum capacity,
+                                         // and two pages of the method)
   unsigned long long p_fix;              // top_p in 2^62 fixed point
   // pool
   __nv_bfloat16* kv;
@@ -112,8 +117,8 @@ struct GpDev {
   double* qtil;                          // [M][L*H_kv][2][G][d] calibrated, rotated summaries q~ of boundary requests, by batch slot
   double* zstat;                         // [L*H_kv][max_boundary_tokens / b][2][G][2] per-page softmax partials (max, sum)
   int* sum_par;                          // [M] which of the two summary buffers is current
-  int* evict;                            // [M][L*H_kv][b] slots a compression evicts, ascending
-  int* evict2;                           // [M][L*H_kv][2b] slots a Shrink evicts, ascending (Shrink policy only)
+  int* evict;                            // [M][L*H_kv][page_size] slots a compression evicts, ascending
+  int* evict2;                           // [M][L*H_kv][2 page_size] slots a Shrink evicts, ascending (Shrink policy only)
   int* cflags;                           // compaction chunk flags, stamped with the step number
   double* rope_cs;                       // [M][d/2][2] cos, sin at the step's position
   float* partials;

@@ -85,12 +85,15 @@ bool valid_config(const gp_config* c) {
   const int G = c->n_q_heads / c->n_kv_heads;
   if (G > 8 || (G & (G - 1))) return false;
   if (c->head_dim != 64 && c->head_dim != 128) return false;
-  if (c->page_size != GP_PAGE || c->recent_window != c->page_size) return false;
+  // page_size: 16, 32, ..., 256 tokens; the protected window is one 16-token tile (so it equals the page at 16)
+  if (c->page_size < GP_PAGE || c->page_size > GP_MAX_BLK || (c->page_size & (c->page_size - 1))) return false;
+  if (c->recent_window != GP_PAGE) return false;
+  const long long sub = c->page_size / GP_PAGE;
   if (c->max_requests < 1 || c->max_requests > GP_MAX_REQ) return false;
-  if (c->max_pages_per_req < 1 || c->max_pages_per_req > (1 << 20)) return false;
-  if (gp_bsel_smem_for_cap(c->max_pages_per_req) > GP_MAX_DYN_SMEM) return false;   // about 62 000 pages
-  if (c->n_pages < 1 || c->n_pages > 0x7fffffffLL / GP_PAGE) return false;
-  if (c->k_loc < 0 || c->k_loc > GP_PAGE) return false;
+  if (c->max_pages_per_req < 1 || c->max_pages_per_req * sub > (1 << 20)) return false;
+  if (gp_bsel_smem_for_cap(c->max_pages_per_req * sub) > GP_MAX_DYN_SMEM) return false;   // about 61 000 tiles of 16 tokens
+  if (c->n_pages < 1 || c->n_pages * sub > 0x7fffffffLL / GP_PAGE) return false;
+  if (c->k_loc < 0 || c->k_loc > c->page_size) return false;
   if (c->max_batch_tokens < 0 || c->max_boundary_tokens < 0) return false;
   if (c->demand_metric < GP_METRIC_TOP_P || c->demand_metric > GP_METRIC_ENTROPY || c->reserved != 0) return false;
   if (c->async_boundary < 0 || c->async_boundary > 1 || c->async_slots < 0 || c->async_slots > 4096) return false;
@@ -105,9 +108,11 @@ bool valid_config(const gp_config* c) {
 
 Layout make_layout(const gp_config& c) {
   Layout L;
-  const size_t M = c.max_requests, cap = c.max_pages_per_req, b = GP_PAGE, d = c.head_dim;
+  // everything below is in physical (16-token) pages: a page of the method is `sub` of them
+  const size_t sub = (size_t)c.page_size / GP_PAGE, blk = (size_t)c.page_size;
+  const size_t M = c.max_requests, cap = (size_t)c.max_pages_per_req * sub, b = GP_PAGE, d = c.head_dim;
   const size_t LH = (size_t)c.n_layers * c.n_kv_heads, G = c.n_q_heads / c.n_kv_heads;
-  const size_t np = (size_t)c.n_pages;
+  const size_t np = (size_t)c.n_pages * sub;
   L.max_batch_tokens = c.max_batch_tokens > 0 ? c.max_batch_tokens : (long long)(np * b);
   // candidate tokens of one step's boundary requests: by default every request of a batch may be at its boundary
   // (equal prompts reach it together); a caller that knows better sizes the boundary scratch smaller
@@ -142,8 +147,8 @@ Layout make_layout(const gp_config& c) {
   L.zbuf = take(LH * (Tb + b) * 2 * G * 8);
   L.qtil = take(M * LH * 2 * (size_t)G * d * 8);
   L.zstat = take(LH * (Tb / b + 1) * 2 * G * 2 * 8);
-  L.evict = take(M * LH * b * 4);
-  L.evict2 = take(c.policy == GP_POLICY_SHRINK ? M * LH * 2 * b * 4 : 16);
+  L.evict = take(M * LH * blk * 4);
+  L.evict2 = take(c.policy == GP_POLICY_SHRINK ? M * LH * 2 * blk * 4 : 16);
   L.cflags = take(LH * ((Tb + M * b) / GP_MOVE_TOK + 2 * M + 1) * 4);
   L.rope_cs = take(M * (d / 2) * 2 * 8);
   L.partials = take((size_t)L.max_rc * LH * G * (d + 2) * 4);
@@ -638,7 +643,7 @@ __global__ void gp_admit_kernel(GpDev p, int r, int share_from, int n_shared, in
       *p.free_top = top - need;
       p.P[r] = P_target; p.n[r] = n0; p.pos[r] = n0; p.started[r] = 0; p.live[r] = 1;
       p.bstep[r] = GP_NEVER; p.last_act[r] = GP_ACT_NONE;
-      p.n_pristine[r] = n0 / GP_PAGE;
+      p.n_pristine[r] = (n0 / p.blk) * p.sub;                 // only full pages of the method can be shared
     }
   }
   if (lane == 0) *status = st;
@@ -792,7 +797,7 @@ int gp_config_default(gp_config* cfg) {
   cfg->page_size = GP_PAGE;
   cfg->max_requests = 512;
   cfg->recent_window = GP_PAGE;
-  cfg->k_loc = GP_PAGE / 4;
+  cfg->k_loc = GP_PAGE / 4;          // a quarter of the page; the paper's 64 at its page size of 256
   cfg->beta_s = 0.9;
   cfg->beta_l = 0.999;
   cfg->top_p = 0.99;
@@ -843,10 +848,11 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   uint8_t* base = static_cast<uint8_t*>(dev_blob);
   GpDev& d = pool->dev;
   d.L = cfg->n_layers; d.Hq = cfg->n_q_heads; d.Hkv = cfg->n_kv_heads; d.G = cfg->n_q_heads / cfg->n_kv_heads;
-  d.d = cfg->head_dim; d.M = cfg->max_requests; d.cap = cfg->max_pages_per_req; d.k_loc = cfg->k_loc;
+  d.sub = cfg->page_size / GP_PAGE; d.blk = cfg->page_size;
+  d.d = cfg->head_dim; d.M = cfg->max_requests; d.cap = cfg->max_pages_per_req * d.sub; d.k_loc = cfg->k_loc;
   d.chunk_pages = chunk_pages_setting(); d.max_rc = L.max_rc;
   d.bchunk_pages = bchunk_pages_setting();
-  d.n_pages = cfg->n_pages; d.max_batch_tokens = L.max_batch_tokens;
+  d.n_pages = cfg->n_pages * d.sub; d.max_batch_tokens = L.max_batch_tokens;
   d.max_boundary_tokens = L.max_boundary_tokens;
   d.async = cfg->async_boundary;
   d.spin_limit = GP_SPIN_LIMIT;
@@ -856,8 +862,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.policy = cfg->policy; d.policy_seed = (unsigned long long)(unsigned)cfg->policy_seed; d.p_compress = cfg->p_compress;
   d.shrink_below = cfg->shrink_below;
   {
-    const long long mp = (cfg->min_capacity + GP_PAGE - 1) / GP_PAGE;      // (P - 1) b >= min_capacity
-    d.min_pages_after_shrink = (int)(mp > (1 << 21) ? (1 << 21) : (mp < 2 ? 2 : mp));
+    const long long mp = (cfg->min_capacity + GP_PAGE - 1) / GP_PAGE;      // (P - 1) b >= min_capacity, and P >= 3
+    d.min_pages_after_shrink = (int)(mp > (1 << 21) ? (1 << 21) : (mp < 2 * d.sub ? 2 * d.sub : mp));
   }
   d.p_fix = (unsigned long long)llrint(cfg->top_p * 4611686018427387904.0);
   d.kv = reinterpret_cast<__nv_bfloat16*>(base + L.kv);
@@ -979,8 +985,9 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   for (int i = 0; i < c.max_requests; ++i)
     if (!pool->live[i]) { slot = i; break; }
   if (slot < 0 && n_shared_pages == 0) return GP_ERR_NO_SLOT;
-  const long long n_prompt = (long long)n_shared_pages * GP_PAGE + n_tail;
-  long long P = n_prompt / GP_PAGE + 1;
+  const int sub = c.page_size / GP_PAGE;
+  const long long n_prompt = (long long)n_shared_pages * c.page_size + n_tail;
+  long long P = n_prompt / c.page_size + 1;
   if (initial_pages > P) P = initial_pages;
   // with shared pages the donor's count of shareable pages lives on the device: the kernel below gives the
   // refusals in the documented order (invalid arguments, no slot, no pages)
@@ -989,7 +996,8 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   GP_CUDA(cudaSetDevice(pool->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (flush_chain(pool, s) != GP_OK) return GP_ERR_CUDA;       // the free list belongs to the last step's boundary chain first
-  gp_admit_kernel<<<1, 32, 0, s>>>(cur_view(pool), slot, share_from, n_shared_pages, n_tail, (int)P, pool->d_status);
+  // the kernels count in physical pages
+  gp_admit_kernel<<<1, 32, 0, s>>>(cur_view(pool), slot, share_from, n_shared_pages * sub, n_tail, (int)(P * sub), pool->d_status);
   pool->launch_count++;
   int st = GP_ERR_CUDA;
   GP_CUDA(cudaMemcpyAsync(&st, pool->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -999,7 +1007,7 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
     const long long total = (long long)c.n_layers * n_tail * c.n_kv_heads * 2 * (c.head_dim / 8);
     int grid = (int)((total + 255) / 256);
     if (grid > 148 * 16) grid = 148 * 16;
-    gp_ingest_kernel<<<grid, 256, 0, s>>>(pool->dev, slot, n_shared_pages, n_tail,
+    gp_ingest_kernel<<<grid, 256, 0, s>>>(pool->dev, slot, n_shared_pages * sub, n_tail,
                                          static_cast<const __nv_bfloat16*>(k_tail),
                                          static_cast<const __nv_bfloat16*>(v_tail));
     pool->launch_count++;
@@ -1350,12 +1358,17 @@ int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t
   GP_CUDA(cudaMemcpy(&Pv, pool->sP[pc] + req, 4, cudaMemcpyDeviceToHost));
   GP_CUDA(cudaMemcpy(&nv, pool->sn[pc] + req, 4, cudaMemcpyDeviceToHost));
   GP_CUDA(cudaMemcpy(&pv, pool->spos[cur_copy(pool)] + req, 8, cudaMemcpyDeviceToHost));
-  if (P) *P = Pv;
+  if (P) *P = Pv / (pool->cfg.page_size / GP_PAGE);
   if (n) *n = nv;
   if (pos) *pos = pv;
   if (page_table && Pv > 0)
-    GP_CUDA(cudaMemcpy(page_table, pool->dev.page_table + (size_t)req * pool->cfg.max_pages_per_req, (size_t)Pv * 4,
-                       cudaMemcpyDeviceToHost));
+  {
+    // pages of the method: the group of tiles that starts at table entry j * sub (see gp_debug_pool)
+    const int sub = pool->cfg.page_size / GP_PAGE;
+    std::vector<int> tiles((size_t)Pv);
+    GP_CUDA(cudaMemcpy(tiles.data(), pool->dev.page_table + (size_t)req * pool->dev.cap, (size_t)Pv * 4, cudaMemcpyDeviceToHost));
+    for (int j = 0; j < Pv / sub; ++j) page_table[j] = tiles[(size_t)j * sub] / sub;
+  }
   return GP_OK;
 }
 
@@ -1378,6 +1391,7 @@ int gp_debug_state(gp_pool* pool, int32_t* P, int32_t* n) {
     for (int i = 0; i < M; ++i)
       if (b[i] == last) { if (P) P[i] = oP[i]; if (n) n[i] = on[i]; }
   }
+  if (P) for (int i = 0; i < M; ++i) P[i] /= pool->cfg.page_size / GP_PAGE;
   return GP_OK;
 }
 
@@ -1393,7 +1407,7 @@ static int gather_stream(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_h
   GP_CUDA(cudaMemcpy(&nv, pool->sn[pc] + req, 4, cudaMemcpyDeviceToHost));
   *n_out = nv;
   if (nv == 0) return GP_OK;
-  const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * GP_PAGE;
+  const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * pool->cfg.page_size;
   int* tok = reinterpret_cast<int*>(pool->dbg);
   uint4* kk = reinterpret_cast<uint4*>(pool->dbg + cap_tok * 4);
   uint4* vv = reinterpret_cast<uint4*>(pool->dbg + cap_tok * 4 + cap_tok * pool->cfg.head_dim * 2);
@@ -1417,7 +1431,7 @@ int gp_debug_kv(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_head, void
   int n = 0;
   const int st = gather_stream(pool, req, layer, kv_head, &n);
   if (st != GP_OK) return st;
-  const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * GP_PAGE;
+  const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * pool->cfg.page_size;
   const size_t rowb = (size_t)pool->cfg.head_dim * 2;
   if (n > 0 && k_rows) GP_CUDA(cudaMemcpy(k_rows, pool->dbg + cap_tok * 4, n * rowb, cudaMemcpyDeviceToHost));
   if (n > 0 && v_rows)
@@ -1484,12 +1498,21 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
   int top = 0;
   GP_CUDA(cudaMemcpy(&top, pool->dev.free_top, 4, cudaMemcpyDeviceToHost));
   const int err = *reinterpret_cast<volatile const int*>(pool->h_err);
-  if (n_free) *n_free = top;
-  if (refcounts) GP_CUDA(cudaMemcpy(refcounts, pool->dev.refcount, (size_t)pool->cfg.n_pages * 4, cudaMemcpyDeviceToHost));
+  if (n_free) *n_free = top / (pool->cfg.page_size / GP_PAGE);
+  if (refcounts) {
+    // One count per page of the method.  Its 16-token tiles are taken from the free list, shared and returned
+    // together and in whole aligned groups (the list starts in tile order and every pop and push is a multiple of
+    // the group), so page i is tiles [i * sub, (i + 1) * sub) and its count is that of its first tile.
+    const int sub = pool->cfg.page_size / GP_PAGE;
+    std::vector<int> ref((size_t)pool->dev.n_pages);
+    GP_CUDA(cudaMemcpy(ref.data(), pool->dev.refcount, ref.size() * 4, cudaMemcpyDeviceToHost));
+    for (long long i = 0; i < pool->cfg.n_pages; ++i) refcounts[i] = ref[(size_t)i * sub];
+  }
   if (counters) {
     long long c[12];
     GP_CUDA(cudaMemcpy(c, pool->dev.counters, 96, cudaMemcpyDeviceToHost));
     for (int i = 0; i < 12; ++i) counters[i] = c[i];
+    counters[4] /= pool->cfg.page_size / GP_PAGE;          // copy-on-write: counted per 16-token tile, reported per page
     counters[7] = err;
   }
   return GP_OK;

@@ -56,8 +56,8 @@ def make_pools(wl: W.Workload, device: int = 0, **over):
     for k in ("n_pages", "max_pages_per_req", "k_loc", "max_requests"):
         if k in over:
             kw[k] = over[k]
-    ocfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, **kw, **tun)
-    gcfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, **kw, **tun,
+    ocfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, page_size=s.page_size, recent_window=16, **kw, **tun)
+    gcfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, page_size=s.page_size, **kw, **tun,
                          max_batch_tokens=over.get("max_batch_tokens", 0), async_slots=over.get("async_slots", 0),
                          max_boundary_tokens=over.get("max_boundary_tokens", 0))
     return B.Pool(gcfg, device), O.OraclePool(ocfg)
@@ -169,22 +169,25 @@ def run_lockstep(wl: W.Workload, max_steps: Optional[int] = None, summary_every:
                 if g_dec[rid] not in (B.GP_ACT_COMPRESS, B.GP_ACT_COMPRESS_FALLBACK, B.GP_ACT_SHRINK):
                     continue
                 r = ora.requests[rid]
-                K_t = info.n_c - (2 * b if g_dec[rid] == B.GP_ACT_SHRINK else b)    # Eq. 13: a Shrink evicts two pages
+                R = ora.cfg.recent_window
+                # the candidates of Eq. 10 are everything but the protected window; a page worth of them goes (Eq. 13:
+                # a Shrink evicts two pages)
+                K_t = info.n_e - (2 * b if g_dec[rid] == B.GP_ACT_SHRINK else b)
                 for l in range(s.n_layers):
                     for h in range(s.n_kv_heads):
                         st.decisions["sel"] += 1
-                        keep, margin = O.select_retained(O.token_scores(info.a_s[l, h], info.a_l[l, h]),
-                                                         r.P - 1, b, K_t, ora.cfg.k_loc)
+                        keep, margin = O.select_retained(O.token_scores(info.e_s[l, h], info.e_l[l, h]),
+                                                         -(-info.n_e // b), b, K_t, ora.cfg.k_loc)
                         want_tok = r.tok[l, h, keep]
-                        got = B.gp_debug_retained(gpu.handle, rid, l, h, K_t + b)
+                        got = B.gp_debug_retained(gpu.handle, rid, l, h, K_t + R)
                         got_hist, got_prot = got[:K_t], got[K_t:]
-                        assert np.array_equal(got_prot, r.tok[l, h, info.n_c:info.n_c + b]), "protected page lost"
+                        assert np.array_equal(got_prot, r.tok[l, h, info.n_e:info.n_e + R]), "protected window lost"
                         if not np.array_equal(got_hist, want_tok):
                             assert margin < NEAR_TIE, (f"step {st.steps} req {rid} ({l},{h}): retained set differs, "
                                                        f"margin {margin}")
-                            assert np.all(np.diff(got_hist) > 0) and np.isin(got_hist, r.tok[l, h, :info.n_c]).all()
+                            assert np.all(np.diff(got_hist) > 0) and np.isin(got_hist, r.tok[l, h, :info.n_e]).all()
                             st.near_ties["sel"] += 1
-                            slots = np.searchsorted(r.tok[l, h, :info.n_c], got_hist)
+                            slots = np.searchsorted(r.tok[l, h, :info.n_e], got_hist)
                             overrides.setdefault(rid, {}).setdefault("keep", {})[(l, h)] = slots
             ora.step_apply(rec, overrides)
 

@@ -44,8 +44,8 @@ def test_config_defaults_and_pool_bytes_need_no_gpu():
     assert B.gp_pool_bytes(bad) == 0
     bad = B.make_config(1, 30, 8, 128, n_pages=1024, max_pages_per_req=64)
     assert B.gp_pool_bytes(bad) == 0
-    assert B.gp_pool_bytes(B.make_config(1, 32, 8, 128, n_pages=70000, max_pages_per_req=62000)) > 0
-    assert B.gp_pool_bytes(B.make_config(1, 32, 8, 128, n_pages=70000, max_pages_per_req=63000)) == 0   # selection kernel's shared memory
+    assert B.gp_pool_bytes(B.make_config(1, 32, 8, 128, n_pages=70000, max_pages_per_req=61000)) > 0
+    assert B.gp_pool_bytes(B.make_config(1, 32, 8, 128, n_pages=70000, max_pages_per_req=62000)) == 0   # selection kernel's shared memory
     assert B.lib().gp_strerror(B.GP_ERR_NO_PAGES).decode().startswith("not enough")
 
 

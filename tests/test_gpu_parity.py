@@ -586,9 +586,9 @@ def test_largest_page_cap_still_launches_the_selection_kernel():
     # the selection kernel's shared memory grows with the per-request page cap (one bit per candidate token);
     # at the largest cap the configuration check admits, the kernel must still launch and decide as the oracle
     wl = W.Workload("cap", 41, W.Shape(1, 4, 1, 64), [W.RequestSpec(0, 200, 40, 0.05)], n_resident=1, initial_pages=0,
-                    max_pages_per_req=62000, n_pages=64)
+                    max_pages_per_req=61000, n_pages=64)
     st = LS.run_lockstep(wl, tau=-0.02)
-    _report("cap 62000", st)
+    _report("cap 61000", st)
     assert st.decisions["act"] >= 2
 
 
