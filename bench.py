@@ -48,7 +48,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per algorithmic byte of the attention kernel, from one ncu capture of a launch of this workload
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch's algorithmic bytes); not measured by this run
-TRAFFIC_RATIO = 1.03
+TRAFFIC_RATIO = 1.02
 TRAFFIC_SOURCE = "profiles/attention_qwen3_8b_layer.md (ncu capture of one launch), scaled by this run's algorithmic bytes"
 
 
