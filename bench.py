@@ -244,15 +244,17 @@ def timed_window(job, torch, device, S0, K, rank, sample_clocks=False):
     tokens decoded on this rank, kernels launched, clock record or None)."""
     B = job.B
     stream = torch.cuda.current_stream(device)
+    # the clock sampler starts before the untimed roll to the window, so that the GPU is under load, not waking up
+    # from an idle pause, when the timed steps begin
+    sampler = ClockSampler(device) if (sample_clocks and rank == 0) else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
     job.reset()
     job.roll(S0)
     torch.cuda.synchronize(device)
     tok0 = int(job.counters()[6])
     launches0 = B.gp_launch_count(job.pool.handle)
-    sampler = ClockSampler(device) if (sample_clocks and rank == 0) else None
-    if sampler:
-        sampler.start()
-        time.sleep(0.3)
     shard.barrier(device)
     torch.cuda.synchronize(device)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
