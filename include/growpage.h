@@ -182,8 +182,9 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
  *   dev_actions  device int32 [n_req]: GP_ACT_* per request
  * q, k, v and out must be 16-byte aligned (the kernels move rows in 16-byte pieces), dev_req_ids and
  * dev_actions 4-byte aligned: GP_ERR_INVALID otherwise, nothing is launched.
- * Asynchronous on `stream`; nothing is read back to the host, so (with profiling off) a sequence of
- * steps can be captured into a CUDA graph and replayed.  The step's kernels are chained with
+ * Asynchronous on `stream`; nothing is read back to the host and the step's number lives on the device,
+ * so (with profiling off, synchronous mode) a step over fixed buffers, or a sequence of steps, can be captured
+ * into a CUDA graph and replayed any number of times.  The step's kernels are chained with
  * programmatic dependent launch.  Steps of one pool must be issued on one stream (or otherwise
  * serialised): they share scratch inside the blob.  See gp_set_early_plan for an option that lets
  * the step's first kernel start its work beside the last kernel of the step before.
@@ -202,7 +203,8 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages,
  * decisions are read with gp_boundary_outcome.  The boundary chain of the LAST step issued has not been launched
  * yet: gp_request_add, gp_release and the introspection calls launch it themselves (on the stream of that step);
  * a caller that looks at the pool's pages in any other way calls gp_async_join first.  Early planning does not
- * apply, and the layer-by-layer calls are not available in this mode (GP_ERR_STATE from gp_step_begin). */
+ * apply, the layer-by-layer calls are not available in this mode (GP_ERR_STATE from gp_step_begin), and its steps
+ * are numbered on the host: do not replay them from a CUDA graph. */
 int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
                    const void* q, const void* k, const void* v,
                    void* out, int32_t* dev_actions, void* stream);

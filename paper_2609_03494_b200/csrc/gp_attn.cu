@@ -97,8 +97,10 @@ template <int D, bool ROPE>
 __global__ void __launch_bounds__(NTHREADS, 2)
 gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* __restrict__ q,
                const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, float* __restrict__ out, int lh0,
-               int lh_n) {
+               int lh_n, int adv_lh) {
   // lh0, lh_n: the (layer, KV head) units this launch covers, [lh0, lh0 + lh_n): all of them, or one layer's
+  // adv_lh: the unit whose append also moves the request's counters on by one token (-1: none; the layer-by-layer
+  // step does that at its end)
   using GEO = Geo<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
@@ -408,6 +410,12 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
             fence_proxy_async();
           }
           if (lane == 0) p.tok[gp_tok_off(p, l, page, h) + s] = sd[7];
+          if (lane == 1 && lh == adv_lh) {
+            // the request is one token further; the summary CTAs of this step have written the buffer not in use
+            // (the plan kernel had completed before this kernel passed its wait)
+            const int r = sd[1];
+            p.n[r] = n_new; p.pos[r] = (long long)sd[7] + 1; p.started[r] = 1; p.sum_par[r] = sd[12] ^ 1;
+          }
           __syncwarp();
         }
         const uint32_t kt = smem_u32(tile);
@@ -649,7 +657,7 @@ void gp_attention_setup(const GpDev& p) {           // once per pool: opt into t
 }
 
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n) {
+                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n, int adv_lh) {
   (void)req_ids;
   const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kk = static_cast<const __nv_bfloat16*>(k);
@@ -659,7 +667,7 @@ void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const vo
 #define GP_LAUNCH(DD, RR)                                                                 \
   do {                                                                                    \
     auto kern = gp_attn_kernel<DD, RR>;                                                   \
-    gp_launch(kern, grid, NTHREADS, (size_t)sm, s, pdl, p, n_req, qq, kk, vv, out, lh0, lh_n); \
+    gp_launch(kern, grid, NTHREADS, (size_t)sm, s, pdl, p, n_req, qq, kk, vv, out, lh0, lh_n, adv_lh); \
   } while (0)
   if (p.d == 128) {
     if (rope) GP_LAUNCH(128, true); else GP_LAUNCH(128, false);

@@ -475,7 +475,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       p.delta[r] = delta;
       // pages and slots as the step left them (full); the allocator below changes what the decision changes.  In
       // the asynchronous mode the plan of the step in between leaves these two words of a held request alone.
-      p.wP[r] = Pr; p.wn[r] = Pr * GP_PAGE;
+      p.P[r] = Pr; p.n[r] = Pr * GP_PAGE;
       s_want[e] = want; s_ksh[e] = acc.z; s_P[e] = Pr; s_req[e] = r; s_bi[e] = inf.x;
     }
   }
@@ -514,7 +514,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
           p.refcount[page] = 1;
           p.page_table[(size_t)r * p.cap + Pr + t] = page;
         }
-        p.wP[r] = Pr + sub;
+        p.P[r] = Pr + sub;
         report(bi, r, GP_ACT_GROW);
         s_want[e] |= 2;
         ++grow;
@@ -545,8 +545,8 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       else { report(bi, r, GP_ACT_COMPRESS); ++comp; }
       // a compression frees one page worth of slots; a Shrink frees two and gives the last page back (the
       // compaction kernel returns it once nothing reads it any more)
-      p.wn[r] = (s_P[e] - (shrink ? 2 : 1) * sub) * GP_PAGE;
-      if (shrink) p.wP[r] = s_P[e] - sub;
+      p.n[r] = (s_P[e] - (shrink ? 2 : 1) * sub) * GP_PAGE;
+      if (shrink) p.P[r] = s_P[e] - sub;
       p.n_pristine[r] = 0;
       s_want[e] |= 8;
     }
@@ -1034,6 +1034,19 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (s_i[2]) {
     __threadfence();
+    if (!out) {
+      // Layer-by-layer step: the requests' counters move on here, at the end of the step (a whole-step launch
+      // does it where the attention kernel appends the token): one token further, the summary buffers swapped.
+      // The first work item of a request names it once.
+      for (int idx = tid; idx < n_rc; idx += SEL_T) {
+        const int4 d0 = *reinterpret_cast<const int4*>(p.rcx + (size_t)idx * GP_DESC_INTS);
+        if (p.rcx[(size_t)idx * GP_DESC_INTS + 4] == 0) {
+          const int r = d0.y;
+          p.n[r] += 1; p.pos[r] += 1; p.started[r] = 1; p.sum_par[r] ^= 1;
+        }
+      }
+      __syncthreads();
+    }
     decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(S.sbuf), serial);
   }
 
@@ -1098,7 +1111,10 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
   const int n_cmp = p.hdr[HDR_N_CMP];
   const int n_items = p.hdr[HDR_N_CITEM];
   const int n_cow = p.hdr[HDR_N_COW];
-  const int stamp = serial + 1;       // unique per decode step of the pool: the chunk flags are never cleared
+  // unique per decode step of the pool (the chunk flags are never cleared): the host's step count in the
+  // asynchronous mode, where the two scratch sets count on their own; otherwise the counter the plan kernel keeps
+  // on the device, so that a step replayed from a CUDA graph gets a stamp of its own
+  const int stamp = p.async ? serial + 1 : p.hdr[HDR_STEP];
   for (int i = tid + CT; i <= n_cmp; i += CT) s_info[i] = p.cmp_info[i];
 
   for (bool first = true;; first = false) {

@@ -88,13 +88,12 @@ struct GpDev {
   int* page_table;
   int* shadow;
   // per request
-  // Pages, occupied slots, "has decoded", summary buffer in use and position of every request exist twice: a
-  // decode step reads one copy (P, n, started, sum_par, pos) and its plan writes the other (wP, ...), every
-  // slot carried over and the stepped ones advanced by one token, for the step after it; the decision step
-  // writes the pages and slots of the requests at a boundary into the copy their next step reads.  So the plan
-  // of a step may run while the step before it still executes.  The host sets the two views per launch.
+  // Pages, occupied slots, "has decoded", summary buffer in use and position of every request.  A decode step's
+  // plan only reads them; the attention kernel advances a stepped request by one token where it appends the
+  // token (after the plan has completed), the decision step then sets pages and slots of the requests at a
+  // boundary.  In the asynchronous mode a request that sits a step out is touched by that step's kernels not at
+  // all, so the boundary chain that runs beside them owns its words.
   int* P; int* n; int* started; int* live; int* n_pristine; long long* pos;
-  int* wP; int* wn; int* wstarted; int* wsum_par; long long* wpos;
   int* bstep;                            // [M] number of the decode step at which the request last reached its boundary
   int* last_act;                         // [M] decision taken at that boundary (GP_ACT_*)
   double* summ;
@@ -238,7 +237,7 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 
 // ---- host-visible launchers (one per translation unit) -------------------------------------------
 void gp_launch_attention(const GpDev& p, const int* req_ids, int n_req, const void* q, const void* k, const void* v,
-                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n);
+                         float* out, int grid, cudaStream_t s, bool pdl, int lh0, int lh_n, int adv_lh);
 size_t gp_attention_smem(int d, int G);
 int gp_attention_ctas_per_sm(int d);
 // ---- programmatic dependent launch -------------------------------------------------------------------

@@ -25,8 +25,6 @@ struct gp_pool {
   int chain_pending;                                // the last step's boundary chain has not been launched yet
   int attn_grid_async, chain_grid;
   long long serial;                                 // decode steps issued so far
-  // the two copies of the requests' counters (see GpDev): step t reads copy t mod 2
-  int* sP[2]; int* sn[2]; int* sstarted[2]; int* spar[2]; long long* spos[2];
   void* blob;
   size_t bytes;
   std::vector<uint8_t> live;      // host mirror of the slot free list
@@ -132,8 +130,8 @@ Layout make_layout(const gp_config& c) {
   L.words = take(256 * 4);                       // free_top, err, plan header, status
   L.page_table = take(M * cap * 4);
   L.shadow = take(M * cap * 4);
-  L.reqi = take(12 * M * 4);                     // two copies of P, n, started, sum_par; live, n_pristine, bstep, last_act
-  L.pos = take(2 * M * 8);                       // two copies
+  L.reqi = take(8 * M * 4);                      // P, n, started, sum_par, live, n_pristine, bstep, last_act
+  L.pos = take(M * 8);
   L.summ = take((size_t)c.n_layers * M * 2 * 2 * c.n_q_heads * d * 8);
   L.Kx = take(M * LH * 2 * 4);
   L.Hx = take(c.demand_metric == GP_METRIC_ENTROPY ? M * LH * 2 * 8 : 16);
@@ -381,7 +379,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __shared__ int s_req[GP_MAX_REQ], s_state[GP_MAX_REQ];     // summary CTAs: request of a batch slot, flags
   __shared__ long long s_pos64[GP_MAX_REQ];
   __shared__ int s_bin[GP_COST_BINS], s_binbase[GP_COST_BINS], s_nmc;
-  __shared__ unsigned char s_adv[GP_MAX_REQ];     // slots this step really steps
   const int i = threadIdx.x;
   const bool in = i < n_req;
   // What runs before the wait for the kernel before this one.  In a whole-step launch that kernel is the
@@ -439,17 +436,12 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   }
   if (!plan_on) return;
   s_first[i] = 0x7fffffff;
-  s_adv[i] = 0;
   if (i < GP_COST_BINS) s_bin[i] = 0;
   if (i == 0) s_nmc = 0;
-  // this thread's slot (thread i looks after batch position i and, for the carry at the end, after slot i)
-  int c_n = 0, c_P = 0, c_st = 0, c_par = 0, c_held = 0;
-  long long c_pos = 0;
-  if (i < p.M) {
-    c_n = __ldcg(p.n + i); c_P = __ldcg(p.P + i); c_st = __ldcg(p.started + i); c_par = __ldcg(p.sum_par + i);
-    c_pos = __ldcg(p.pos + i);
-    if (p.async) c_held = __ldcg(p.bstep + i) == serial - 1;
-  }
+  // The number this step goes by: the host's count of decode steps in the asynchronous mode (the two scratch sets
+  // count on their own); otherwise the pool's own counter on the device, so that a step replayed from a CUDA graph
+  // still gets a number of its own.
+  const int step_no = p.async ? serial : __ldcg(p.hdr + HDR_STEP);
   __syncthreads();
   int r = -1;
   if (in) {
@@ -549,8 +541,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   const int sorted0 = s_binbase[key] + within;
   s_chunks[i] = chunks; s_pos[i] = (int)pos;
   if (in) {
-    if (chunks > 0) s_adv[r] = 1;
-    if (isb) { p.bstep[r] = serial; if (p.async) act = GP_ACT_PENDING; }
+    if (isb) { p.bstep[r] = step_no; if (p.async) act = GP_ACT_PENDING; }
     actions[i] = act;
     if (isb) {
       p.bnd_info[2 * bnd_idx] = make_int4(i, r, Pr, (int)pos);     // pos: position of this step's token
@@ -570,16 +561,6 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     if (chunks > 1) p.mc_list[atomicAdd(&s_nmc, 1)] = make_int4(i, rc_off, chunks, 0);
   }
   __syncthreads();
-  // The next step's copy of the requests' counters: every slot carried over, the stepped ones one token further
-  // (the summary buffers swap: this step's summary CTAs write the buffer not in use).  Pages and slots of a
-  // request that sits this step out belong to the boundary chain that is still running.
-  if (i < p.M) {
-    const int adv = s_adv[i];
-    if (!c_held) { p.wn[i] = c_n + adv; p.wP[i] = c_P; }
-    p.wpos[i] = c_pos + adv;
-    p.wstarted[i] = c_st | adv;
-    p.wsum_par[i] = c_par ^ adv;
-  }
   if (p.rope_theta != 0.0) {                                      // cos / sin of the step's position
     __syncthreads();
     const int half = p.d / 2;
@@ -674,12 +655,9 @@ __global__ void gp_ingest_kernel(GpDev p, int r, int n_shared, int n_tail, const
   }
 }
 
-__global__ void gp_release_kernel(GpDev p, int r, int serial) {
+__global__ void gp_release_kernel(GpDev p, int r) {
   const int lane = threadIdx.x;
-  // a request that reached its boundary at the last step (asynchronous mode) has its page count where that
-  // step's boundary chain put it: in the other copy
-  const bool other = p.async && p.bstep[r] == serial - 1;
-  const int Pr = other ? p.wP[r] : p.P[r];
+  const int Pr = p.P[r];
   const int* table = p.page_table + (size_t)r * p.cap;
   for (int j0 = 0; j0 < Pr; j0 += 32) {
     const int j = j0 + lane;
@@ -699,8 +677,7 @@ __global__ void gp_release_kernel(GpDev p, int r, int serial) {
     __syncwarp();
   }
   if (lane == 0) {
-    p.live[r] = 0; p.P[r] = 0; p.n[r] = 0; p.started[r] = 0; p.n_pristine[r] = 0;
-    p.wP[r] = 0; p.wn[r] = 0; p.wstarted[r] = 0; p.bstep[r] = GP_NEVER;
+    p.live[r] = 0; p.P[r] = 0; p.n[r] = 0; p.started[r] = 0; p.n_pristine[r] = 0; p.bstep[r] = GP_NEVER;
   }
 }
 
@@ -733,30 +710,6 @@ void pool_free(gp_pool* pool) {
   delete pool;
 }
 
-// the device view with the requests' counters read from copy `rd` and written to copy `wr`
-GpDev with_state(const gp_pool* pool, const GpDev& d, int rd, int wr) {
-  GpDev v = d;
-  v.P = pool->sP[rd]; v.n = pool->sn[rd]; v.started = pool->sstarted[rd]; v.sum_par = pool->spar[rd]; v.pos = pool->spos[rd];
-  v.wP = pool->sP[wr]; v.wn = pool->sn[wr]; v.wstarted = pool->sstarted[wr]; v.wsum_par = pool->spar[wr]; v.wpos = pool->spos[wr];
-  return v;
-}
-// the copy that holds the requests' counters as of now (what the next step will read)
-int cur_copy(const gp_pool* pool) { return (int)(pool->serial & 1); }
-GpDev cur_view(const gp_pool* pool) { return with_state(pool, pool->dev, cur_copy(pool), cur_copy(pool)); }
-
-// The copy that holds a request's pages and slots as of now.  With asynchronous boundary work a request that
-// reached its boundary at the last step sits the next one out, and its boundary chain wrote to the copy that
-// the step after that reads.  Call after a device-wide synchronisation.
-int pages_copy(const gp_pool* pool, int req, int* out) {
-  *out = cur_copy(pool);
-  if (pool->cfg.async_boundary) {
-    int b = 0;
-    if (cudaMemcpy(&b, pool->dev.bstep + req, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return GP_ERR_CUDA;
-    if (b == (int)((pool->serial - 1) & 0x3fffffff)) *out ^= 1;
-  }
-  return GP_OK;
-}
-
 // Asynchronous boundary mode: launches the boundary chain of the last decode step on `s` if it has not been
 // launched yet (it normally rides behind the next step's attention kernel).  Everything that looks at the pool's
 // pages, counters or free list from outside a decode step calls this first.
@@ -764,8 +717,7 @@ int flush_chain(gp_pool* pool, cudaStream_t s) {
   if (!pool->cfg.async_boundary || !pool->chain_pending) return GP_OK;
   const long long t = pool->serial - 1;                       // the step the chain belongs to
   const GpDev& d = (t & 1) ? pool->dev_alt : pool->dev;
-  const int wr = (int)(t & 1);                                  // the copy the step after the next reads
-  gp_launch_chain(with_state(pool, d, wr, wr), d, 0, nullptr, (int)(t & 0x3fffffff), 1, pool->chain_grid, s, false);
+  gp_launch_chain(d, d, 0, nullptr, (int)(t & 0x3fffffff), 1, pool->chain_grid, s, false);
   pool->chain_pending = 0;
   pool->launch_count += 1;
   return cudaGetLastError() == cudaSuccess ? GP_OK : GP_ERR_CUDA;
@@ -890,14 +842,9 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.shadow = reinterpret_cast<int*>(base + L.shadow);
   int* reqi = reinterpret_cast<int*>(base + L.reqi);
   const int M = cfg->max_requests;
-  for (int c = 0; c < 2; ++c) {
-    pool->sP[c] = reqi + (4 * c) * M; pool->sn[c] = reqi + (4 * c + 1) * M; pool->sstarted[c] = reqi + (4 * c + 2) * M;
-    pool->spar[c] = reqi + (4 * c + 3) * M;
-    pool->spos[c] = reinterpret_cast<long long*>(base + L.pos) + (size_t)c * M;
-  }
-  d.live = reqi + 8 * M; d.n_pristine = reqi + 9 * M; d.bstep = reqi + 10 * M; d.last_act = reqi + 11 * M;
-  d.P = d.wP = pool->sP[0]; d.n = d.wn = pool->sn[0]; d.started = d.wstarted = pool->sstarted[0];
-  d.sum_par = d.wsum_par = pool->spar[0]; d.pos = d.wpos = pool->spos[0];
+  d.P = reqi; d.n = reqi + M; d.started = reqi + 2 * M; d.sum_par = reqi + 3 * M;
+  d.live = reqi + 4 * M; d.n_pristine = reqi + 5 * M; d.bstep = reqi + 6 * M; d.last_act = reqi + 7 * M;
+  d.pos = reinterpret_cast<long long*>(base + L.pos);
   d.summ = reinterpret_cast<double*>(base + L.summ);
   d.Kx = reinterpret_cast<int*>(base + L.Kx);
   d.Hx = reinterpret_cast<double*>(base + L.Hx);
@@ -997,7 +944,7 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (flush_chain(pool, s) != GP_OK) return GP_ERR_CUDA;       // the free list belongs to the last step's boundary chain first
   // the kernels count in physical pages
-  gp_admit_kernel<<<1, 32, 0, s>>>(cur_view(pool), slot, share_from, n_shared_pages * sub, n_tail, (int)(P * sub), pool->d_status);
+  gp_admit_kernel<<<1, 32, 0, s>>>(pool->dev, slot, share_from, n_shared_pages * sub, n_tail, (int)(P * sub), pool->d_status);
   pool->launch_count++;
   int st = GP_ERR_CUDA;
   GP_CUDA(cudaMemcpyAsync(&st, pool->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -1022,8 +969,7 @@ int gp_request_add(gp_pool* pool, int32_t share_from, int32_t n_shared_pages, co
 static void launch_plan(gp_pool* pool, const int32_t* ids, int32_t n_req, int32_t* actions, const void* q, int plan_on,
                         int lh0, int lh_n, cudaStream_t s, bool pdl, bool by_layer = false, const GpDev* dev = nullptr,
                         int attn_grid = 0, const GpNorm* norm = nullptr) {
-  const int rd = cur_copy(pool);
-  const GpDev d = with_state(pool, dev ? *dev : pool->dev, rd, rd ^ 1);     // the plan writes the next step's copy
+  const GpDev& d = dev ? *dev : pool->dev;
   const int upc = 32 / (2 * d.G);                            // units a CTA takes per pass (one warp per row)
   const long long want = ((long long)n_req * lh_n + upc - 1) / upc;
   const long long room = 2LL * pool->num_sms - 1;            // two 1024-thread CTAs per SM, one wave
@@ -1056,10 +1002,9 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
     // fetch of the inputs): no programmatic dependence on it
     launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl && !pool->first_plain);
     if (prof) cudaEventRecord(pool->ev[1], s);
-    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH);
+    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH, 0);
     if (prof) cudaEventRecord(pool->ev[2], s);
-    // the decisions change pages and slots in the copy the next step reads
-    gp_launch_boundary(with_state(pool, d, cur_copy(pool), cur_copy(pool) ^ 1), dev_req_ids, n_req, dev_actions,
+    gp_launch_boundary(d, dev_req_ids, n_req, dev_actions,
                        static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s, prof ? pool->ev[3] : nullptr, pdl, serial);
     if (prof) cudaEventRecord(pool->ev[4], s);
     pool->launch_count += GP_N_KERNELS;
@@ -1076,12 +1021,11 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
     // which the chain kernel of the step before (the kernel before this one on the stream) has just written
     launch_plan(pool, dev_req_ids, n_req, dev_actions, q, 1, 0, LH, s, pdl && !pool->first_plain, false, &d, pool->attn_grid_async);
     if (prof) cudaEventRecord(pool->ev[1], s);
-    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid_async, s, pdl, 0, LH);
+    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid_async, s, pdl, 0, LH, 0);
     if (prof) cudaEventRecord(pool->ev[2], s);
-    // the decisions of the step before change pages and slots in the copy the next step reads (the one that step
-    // itself read: the plan of this step carries every other word over and leaves these to the chain)
-    const int wr = par ^ 1;
-    gp_launch_chain(with_state(pool, dprev, wr, wr), d, n_req, static_cast<float*>(out), (int)((pool->serial - 1) & 0x3fffffff),
+    // the decisions of the step before set pages and slots of requests that sit this step out: nothing else of
+    // this step looks at those words
+    gp_launch_chain(dprev, d, n_req, static_cast<float*>(out), (int)((pool->serial - 1) & 0x3fffffff),
                     pool->chain_pending, pool->chain_grid, s, pdl);
     if (prof) { cudaEventRecord(pool->ev[3], s); cudaEventRecord(pool->ev[4], s); }
     pool->chain_pending = 1;
@@ -1161,7 +1105,7 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
   float* ob = reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(out) - qs * 4);
   const int lh0 = layer * d.Hkv, lh_n = d.Hkv;
   launch_plan(pool, dev_req_ids, n_req, nullptr, qb, 0, lh0, lh_n, s, true);
-  gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n);
+  gp_launch_attention(d, dev_req_ids, n_req, qb, kb, vb, ob, pool->attn_grid, s, true, lh0, lh_n, -1);
   gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
   pool->launch_count += 3;
   pool->step_layers_done += 1;
@@ -1195,7 +1139,7 @@ int gp_attn_layer_qknorm(gp_pool* pool, int32_t layer, const int32_t* dev_req_id
   nm.kn = reinterpret_cast<__nv_bfloat16*>(shifted(pool->kn, ks * 2));
   const int lh0 = layer * d.Hkv, lh_n = d.Hkv;
   launch_plan(pool, dev_req_ids, n_req, nullptr, qb, 0, lh0, lh_n, s, true, false, nullptr, 0, &nm);
-  gp_launch_attention(d, dev_req_ids, n_req, nm.qn, nm.kn, vb, ob, pool->attn_grid, s, true, lh0, lh_n);
+  gp_launch_attention(d, dev_req_ids, n_req, nm.qn, nm.kn, vb, ob, pool->attn_grid, s, true, lh0, lh_n, -1);
   gp_launch_merge(d, n_req, ob, lh0, lh_n, pool->num_sms, s, true);
   pool->launch_count += 3;
   pool->step_layers_done += 1;
@@ -1209,7 +1153,7 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
   if (n_req != pool->step_n_req || !dev_req_ids || !dev_actions) return GP_ERR_INVALID;
   if (pool->step_layers_done != pool->cfg.n_layers) return GP_ERR_STATE;       // layers missing: run them, or gp_step_abort
   GP_CUDA(cudaSetDevice(pool->device));
-  gp_launch_boundary(with_state(pool, pool->dev, cur_copy(pool), cur_copy(pool) ^ 1), dev_req_ids, n_req, dev_actions, nullptr,
+  gp_launch_boundary(pool->dev, dev_req_ids, n_req, dev_actions, nullptr,
                      pool->sel_grid, pool->compact_grid,
                      static_cast<cudaStream_t>(stream), nullptr, true, (int)(pool->serial & 0x3fffffff));
   pool->serial += 1;
@@ -1324,8 +1268,7 @@ int gp_release(gp_pool* pool, int32_t req, void* stream) {
   if (pool->step_open) return GP_ERR_STATE;      // the open step's plan holds a snapshot of the free list
   GP_CUDA(cudaSetDevice(pool->device));
   if (flush_chain(pool, static_cast<cudaStream_t>(stream)) != GP_OK) return GP_ERR_CUDA;
-  gp_release_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
-      with_state(pool, pool->dev, cur_copy(pool), cur_copy(pool) ^ 1), req, (int)((pool->serial - 1 + 1) & 0x3fffffff));
+  gp_release_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(pool->dev, req);
   pool->launch_count++;
   pool->live[req] = 0;
   GP_CUDA(cudaGetLastError());
@@ -1353,11 +1296,9 @@ int gp_debug_request(gp_pool* pool, int32_t req, int32_t* P, int32_t* n, int64_t
   if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
   int Pv = 0, nv = 0; long long pv = 0;
-  int pc = 0;
-  if (pages_copy(pool, req, &pc) != GP_OK) return GP_ERR_CUDA;
-  GP_CUDA(cudaMemcpy(&Pv, pool->sP[pc] + req, 4, cudaMemcpyDeviceToHost));
-  GP_CUDA(cudaMemcpy(&nv, pool->sn[pc] + req, 4, cudaMemcpyDeviceToHost));
-  GP_CUDA(cudaMemcpy(&pv, pool->spos[cur_copy(pool)] + req, 8, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&Pv, pool->dev.P + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&nv, pool->dev.n + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&pv, pool->dev.pos + req, 8, cudaMemcpyDeviceToHost));
   if (P) *P = Pv / (pool->cfg.page_size / GP_PAGE);
   if (n) *n = nv;
   if (pos) *pos = pv;
@@ -1379,18 +1320,8 @@ int gp_debug_state(gp_pool* pool, int32_t* P, int32_t* n) {
   GP_CUDA(cudaDeviceSynchronize());
   const int M = pool->cfg.max_requests;
   const size_t nb = (size_t)M * 4;
-  const int c = cur_copy(pool);
-  if (P) GP_CUDA(cudaMemcpy(P, pool->sP[c], nb, cudaMemcpyDeviceToHost));
-  if (n) GP_CUDA(cudaMemcpy(n, pool->sn[c], nb, cudaMemcpyDeviceToHost));
-  if (pool->cfg.async_boundary) {               // requests about to sit a step out: see pages_copy
-    std::vector<int> b(M), oP(M), on(M);
-    GP_CUDA(cudaMemcpy(b.data(), pool->dev.bstep, nb, cudaMemcpyDeviceToHost));
-    GP_CUDA(cudaMemcpy(oP.data(), pool->sP[c ^ 1], nb, cudaMemcpyDeviceToHost));
-    GP_CUDA(cudaMemcpy(on.data(), pool->sn[c ^ 1], nb, cudaMemcpyDeviceToHost));
-    const int last = (int)((pool->serial - 1) & 0x3fffffff);
-    for (int i = 0; i < M; ++i)
-      if (b[i] == last) { if (P) P[i] = oP[i]; if (n) n[i] = on[i]; }
-  }
+  if (P) GP_CUDA(cudaMemcpy(P, pool->dev.P, nb, cudaMemcpyDeviceToHost));
+  if (n) GP_CUDA(cudaMemcpy(n, pool->dev.n, nb, cudaMemcpyDeviceToHost));
   if (P) for (int i = 0; i < M; ++i) P[i] /= pool->cfg.page_size / GP_PAGE;
   return GP_OK;
 }
@@ -1402,9 +1333,8 @@ static int gather_stream(gp_pool* pool, int32_t req, int32_t layer, int32_t kv_h
   GP_CUDA(cudaSetDevice(pool->device));
   if (flush_chain(pool, pool->last_stream) != GP_OK) return GP_ERR_CUDA;
   GP_CUDA(cudaDeviceSynchronize());
-  int nv = 0, pc = 0;
-  if (pages_copy(pool, req, &pc) != GP_OK) return GP_ERR_CUDA;
-  GP_CUDA(cudaMemcpy(&nv, pool->sn[pc] + req, 4, cudaMemcpyDeviceToHost));
+  int nv = 0;
+  GP_CUDA(cudaMemcpy(&nv, pool->dev.n + req, 4, cudaMemcpyDeviceToHost));
   *n_out = nv;
   if (nv == 0) return GP_OK;
   const size_t cap_tok = (size_t)pool->cfg.max_pages_per_req * pool->cfg.page_size;
@@ -1448,7 +1378,7 @@ int gp_debug_summaries(gp_pool* pool, int32_t req, double* out) {
   GP_CUDA(cudaDeviceSynchronize());
   const gp_config& c = pool->cfg;
   int par = 0;
-  GP_CUDA(cudaMemcpy(&par, pool->spar[cur_copy(pool)] + req, 4, cudaMemcpyDeviceToHost));
+  GP_CUDA(cudaMemcpy(&par, pool->dev.sum_par + req, 4, cudaMemcpyDeviceToHost));
   const size_t per = (size_t)2 * c.n_q_heads * c.head_dim;
   for (int l = 0; l < c.n_layers; ++l)
     GP_CUDA(cudaMemcpy(out + (size_t)l * per, pool->dev.summ + (((size_t)l * c.max_requests + req) * 2 + par) * per,

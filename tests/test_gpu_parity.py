@@ -274,9 +274,9 @@ def test_shrink_at_the_default_floor_and_beyond_the_staging_buffers():
 
 
 def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches():
-    # gp_decode_step only enqueues kernels (chained with programmatic dependent launch): a sequence of steps can
-    # be captured into a CUDA graph once and replayed; the replay must leave exactly the state and outputs of
-    # the same steps launched directly
+    # gp_decode_step only enqueues kernels (chained with programmatic dependent launch) and keeps the step's number
+    # on the device: a sequence of steps, or one step over fixed buffers replayed once per token as a serving loop
+    # does, can come from a CUDA graph; either must leave exactly the state and outputs of direct launches
     import torch
     wl = W.parity_instance(2)
     s = wl.shape
@@ -294,7 +294,7 @@ def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches():
     qd, kd, vd = dev(q), dev(k), dev(v)
     ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
     results = []
-    for use_graph in (False, True):
+    for mode in ("direct", "sequence", "one_step"):
         pool = B.Pool(B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, tau=-0.05, **cfg))
         try:
             for i in range(n):
@@ -302,12 +302,26 @@ def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches():
             outs = torch.zeros((T, s.n_layers, n, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda:0")
             acts = torch.zeros((T, n), dtype=torch.int32, device="cuda:0")
             torch.cuda.synchronize()
-            if use_graph:
+            if mode == "sequence":             # all T steps in one graph, replayed once
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
                     for t in range(T):
                         pool.decode_step(ids, qd[t], kd[t], vd[t], outs[t], acts[t])
                 g.replay()
+            elif mode == "one_step":           # a serving loop: ONE captured step over fixed buffers, replayed per token
+                qs, ks, vs = torch.empty_like(qd[0]), torch.empty_like(kd[0]), torch.empty_like(vd[0])
+                o1, a1 = torch.zeros_like(outs[0]), torch.zeros_like(acts[0])
+                g = torch.cuda.CUDAGraph()
+                st = torch.cuda.Stream()
+                with torch.cuda.stream(st):
+                    for t in range(T):
+                        qs.copy_(qd[t]); ks.copy_(kd[t]); vs.copy_(vd[t])
+                        if t == 0:
+                            with torch.cuda.graph(g, stream=st):
+                                pool.decode_step(ids, qs, ks, vs, o1, a1)
+                        g.replay()
+                        outs[t].copy_(o1); acts[t].copy_(a1)
+                st.synchronize()
             else:
                 for t in range(T):
                     pool.decode_step(ids, qd[t], kd[t], vd[t], outs[t], acts[t])
@@ -318,11 +332,12 @@ def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches():
             results.append((outs.cpu().numpy(), acts.cpu().numpy(), state, kept))
         finally:
             pool.close()
-    direct, replay = results
-    assert np.array_equal(direct[1], replay[1]) and direct[2] == replay[2]
-    assert all(np.array_equal(a, b_) for a, b_ in zip(direct[3], replay[3]))
-    assert np.array_equal(direct[0], replay[0])
-    assert (direct[1] != B.GP_ACT_NONE).any()
+    for replay in results[1:]:
+        direct = results[0]
+        assert np.array_equal(direct[1], replay[1]) and direct[2] == replay[2]
+        assert all(np.array_equal(a, b_) for a, b_ in zip(direct[3], replay[3]))
+        assert np.array_equal(direct[0], replay[0])
+    assert (results[0][1] != B.GP_ACT_NONE).any()
 
 
 @pytest.mark.parametrize("over", [dict(policy=B.GP_POLICY_INVERSE), dict(policy=B.GP_POLICY_INVERSE, tau=-0.05),
