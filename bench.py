@@ -155,7 +155,8 @@ class Job:
     inputs of step t; a request that sits a step out (asynchronous boundary mode) skips that step's inputs,
     which are independent draws per step."""
 
-    def __init__(self, wl, torch, device, inp: Inputs, host_staging=True, policy=0, async_boundary=False, async_slots=0):
+    def __init__(self, wl, torch, device, inp: Inputs, host_staging=True, policy=0, async_boundary=False, async_slots=0,
+                 overlap_slots=0):
         from paper_2609_03494_b200 import binding as B
         self.B, self.torch, self.wl, self.device, self.inp = B, torch, wl, device, inp
         s = wl.shape
@@ -163,7 +164,8 @@ class Job:
         self.M = max(4, self.nreq)
         cfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, n_pages=wl.n_pages,
                             max_pages_per_req=wl.max_pages_per_req, max_requests=self.M, k_loc=wl.k_loc,
-                            host_staging=host_staging, policy=policy, async_boundary=async_boundary, async_slots=async_slots)
+                            host_staging=host_staging, policy=policy, async_boundary=async_boundary, async_slots=async_slots,
+                            overlap_slots=overlap_slots)
         self.pool = B.Pool(cfg, device)
         self.is_async = async_boundary
         dev = f"cuda:{device}"
@@ -315,6 +317,16 @@ def run_ours(args):
             v, m = shard.job_throughput(tk, m, device)
             modes[name] = {"ms_per_step": round(m / K, 5), "tokens_per_s": round(v, 1)}
         B.gp_set_early_plan(sj.pool.handle, False)
+        for ov in [-1] + [int(x) for x in args.overlap_slots.split(",") if x]:
+            oj = Job(wl, torch, device, inp, policy=policy, overlap_slots=ov)
+            for _ in range(Wm):
+                oj.step()
+            for name, early in (("sync_four_kernels", False),) if ov == -1 else ((f"overlap{ov}", False), (f"overlap{ov}_early_plan", True)):
+                B.gp_set_early_plan(oj.pool.handle, early)
+                m, tk, _, _ = timed_window(oj, torch, device, S0, K, rank)
+                v, m = shard.job_throughput(tk, m, device)
+                modes[name] = {"ms_per_step": round(m / K, 5), "tokens_per_s": round(v, 1)}
+            oj.pool.close()
         if "async" in jobs:
             if head_async:
                 modes["async"] = {"ms_per_step": round(ms / K, 5), "tokens_per_s": round(value, 1)}
@@ -585,6 +597,7 @@ def main():
                     help="both (default): headline synchronous, the asynchronous boundary mode timed beside it; sync: synchronous "
                          "only; async: headline asynchronous (boundary work beside the next step)")
     ap.add_argument("--async-slots", type=int, default=0, help="thread blocks the attention kernel leaves to the boundary kernels")
+    ap.add_argument("--overlap-slots", default="", help="comma-separated overlap_slots values to time as extra modes (synchronous mode, boundary work beside the attention kernel)")
     ap.add_argument("--entry", default="step", choices=["step", "layers"],
                     help="step: gp_decode_step; layers: the same step through gp_step_begin / gp_attn_layer / gp_step_end")
     ap.add_argument("--workload", default="layer", choices=["layer", "stack", "config3", "config4", "config5"],

@@ -112,7 +112,14 @@ typedef struct gp_config {
   int32_t demand_metric;     /* GP_METRIC_TOP_P (default): working-set size of Eq. 7; GP_METRIC_ENTROPY: the
                                 ablation's other metric, the view's attention entropy H over ln |C| in the
                                 place of K / |C| (Delta_t is then a floating-point mean)               */
-  int32_t reserved;         /* keep 0                                                              */
+  int32_t overlap_slots;     /* synchronous mode, how the boundary work of a step (selection jobs, decisions,
+                                compaction) is launched.  0 (default): one kernel behind the attention kernel,
+                                whose thread blocks take their places as that kernel's leave and whose jobs
+                                start as soon as the boundary requests' summary logits are reported complete
+                                (three launches per step).  N > 0: the same kernel, beside the attention
+                                kernel on N thread-block slots that kernel's grid gives up.  -1: a selection
+                                and a compaction kernel, one after the other (four launches per step; what
+                                gp_step_end runs).  Same results in every case                        */
   int32_t async_slots;       /* asynchronous boundary work: thread blocks of the attention kernel's grid
                                 given up so that the boundary kernel finds room on the SMs beside it;
                                 0 = a default (64)                                                    */
@@ -323,7 +330,9 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
 
 /* ---- measurement ----------------------------------------------------------------------------- */
 
-#define GP_N_KERNELS 4   /* plan, attention (+ boundary logits), selection + decision, compaction */
+#define GP_N_KERNELS 4   /* plan, attention (+ boundary logits), selection + decision, compaction; with the boundary
+                            work in one kernel (overlap_slots >= 0, the default) the third entry is that kernel and
+                            the fourth stays zero */
 
 /* With profiling on, every kernel of gp_decode_step is bracketed by CUDA events on the step's
  * stream (this serialises nothing but adds event records).  Off by default. */
@@ -356,7 +365,8 @@ int64_t gp_launch_count(gp_pool* pool);
  * but without hanging and with the pool's page accounting intact.  This call lets a test see that happen without
  * any fault: `what` names hand-overs that are then simply not made (1 the attention kernel's first thread block
  * never completes its second work item for its consumer warps; 2 the first chunk of every compaction unit never
- * says that its sources are read; 4 asynchronous mode: the deciding thread block never tells the others; 0 none),
+ * says that its sources are read; 4 the deciding thread block of the boundary kernel never tells the others; 8 the
+ * attention kernel never reports a boundary unit's summary logits complete; 0 none),
  * `spin_limit` the iterations after which waits give up (0 = the default, 2^21).  Applies to the steps issued
  * after it.  The error bits stay set; results of such a pool are not meaningful afterwards. */
 int gp_test_withhold(gp_pool* pool, int32_t what, int32_t spin_limit);

@@ -22,7 +22,7 @@ GP_ACT_STALLED, GP_ACT_SCRATCH, GP_ACT_INVALID = -1, -2, -3
 GP_POLICY_DEMAND, GP_POLICY_INVERSE, GP_POLICY_RANDOM, GP_POLICY_SHRINK = 0, 1, 2, 3
 GP_METRIC_TOP_P, GP_METRIC_ENTROPY = 0, 1
 GP_N_KERNELS = 4
-KERNEL_NAMES = ("plan", "attention", "select_decide", "compact")
+KERNEL_NAMES = ("plan", "attention", "boundary_or_select_decide", "compact_four_kernel_path")
 
 
 class gp_config(C.Structure):
@@ -31,7 +31,7 @@ class gp_config(C.Structure):
         ("page_size", C.c_int32), ("max_requests", C.c_int32), ("max_pages_per_req", C.c_int32),
         ("recent_window", C.c_int32), ("k_loc", C.c_int32), ("host_staging", C.c_int32),
         ("policy", C.c_int32), ("policy_seed", C.c_int32), ("async_boundary", C.c_int32), ("demand_metric", C.c_int32),
-        ("reserved", C.c_int32), ("async_slots", C.c_int32),
+        ("overlap_slots", C.c_int32), ("async_slots", C.c_int32),
         ("n_pages", C.c_int64), ("min_capacity", C.c_int64), ("max_batch_tokens", C.c_int64),
         ("max_boundary_tokens", C.c_int64),
         ("beta_s", C.c_double), ("beta_l", C.c_double), ("top_p", C.c_double), ("tau", C.c_double),
@@ -373,7 +373,8 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
                 beta_s: float = 0.9, beta_l: float = 0.999, top_p: float = 0.99, tau: float = 0.0,
                 rope_theta: float = 0.0, policy: int = 0, policy_seed: int = 0, p_compress: float = 0.7,
                 shrink_below: float = -0.005, min_capacity: int = 1024, async_boundary: bool = False,
-                async_slots: int = 0, max_boundary_tokens: int = 0, demand_metric: int = 0, page_size: int = 16) -> gp_config:
+                async_slots: int = 0, max_boundary_tokens: int = 0, demand_metric: int = 0, page_size: int = 16,
+                overlap_slots: int = 0) -> gp_config:
     cfg = gp_config_default()
     cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
     cfg.n_pages, cfg.max_pages_per_req, cfg.max_requests = n_pages, max_pages_per_req, max_requests
@@ -382,6 +383,7 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
     cfg.policy, cfg.policy_seed, cfg.p_compress = policy, policy_seed, p_compress
     cfg.shrink_below, cfg.min_capacity = shrink_below, min_capacity
     cfg.async_boundary, cfg.async_slots, cfg.max_boundary_tokens = 1 if async_boundary else 0, async_slots, max_boundary_tokens
+    cfg.overlap_slots = overlap_slots
     cfg.demand_metric = demand_metric
     cfg.page_size = page_size
     return cfg

@@ -234,6 +234,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
           if (lane + 32 < npg) pNew2 = p.page_table[(size_t)r * p.cap + pg0 + 32 + lane];
           if (lane < 14) sd[lane] = hB;
           if (lane == 14) sd[14] = lh;
+          if (lane == 15) sd[15] = hB;            // index among the step's boundary requests
           __syncwarp();
           if (lane == 0) {
             const bool has_new = (chunk == nchunks - 1);
@@ -568,6 +569,13 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
       }
       if (!ok) break;
 
+      // ---- a request at its boundary: this warp's share of the unit's summary logits (and the appended row, and the
+      // request's counters) is written; the boundary work that may run beside this kernel counts the reports
+      if (flags & 1) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0 && !(p.withhold & GP_WITHHOLD_READY)) atomicAdd(p.unit_ready + (size_t)sd[15] * LH + lh, 1);
+      }
       // ---- hand the partial result to the merger warp ---------------------------------------------
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
       l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);

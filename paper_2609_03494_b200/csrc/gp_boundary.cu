@@ -1319,12 +1319,18 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 template <int D, bool SHR>
 __global__ void __launch_bounds__(SEL_T, 2)
 gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev pa, int n_req_merge, float* __restrict__ out_merge,
-                int serial, int has_chain) {
+                int serial, int has_chain, const int* __restrict__ req_ids, int* __restrict__ actions) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
   const int tid = threadIdx.x;
   const int LH = p.L * p.Hkv;
-  gp_pdl_launch_dependents();
+  // Synchronous mode (same_step): the chain belongs to the step whose attention kernel runs beside this grid.
+  // A selection job then waits until the consumer warps of that kernel have reported the unit's summary logits
+  // complete (the requests at their boundary come first in its deal), the decisions are reported through
+  // `actions` as usual, and the next kernel on the stream may only be scheduled once the attention kernel has
+  // ended (its early part reads counters that kernel advances).
+  const bool same_step = !p.async;
+  if (!same_step) gp_pdl_launch_dependents();
   if (has_chain) {
     SelSmem S = sel_smem_at(smem);
     int* s_i = S.s_i;
@@ -1368,6 +1374,18 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
         continue;
       }
       if (SHR && job == 3 && Pr - p.sub < p.min_pages_after_shrink) continue;
+      if (same_step) {
+        // every work item of the request reports once per consumer warp for this unit (bounded wait; the
+        // attention kernel's thread blocks were all resident before this grid could be scheduled)
+        if (tid == 0) {
+          const volatile int* rdy = p.unit_ready + (size_t)bidx * LH + lh;
+          unsigned it = 0;
+          while (*rdy < inf2.z && it < p.spin_limit) { ++it; __nanosleep(200); }
+          if (it >= p.spin_limit) atomicOr(p.err, GP_E_SPIN_SEL);
+          __threadfence();
+        }
+        __syncthreads();
+      }
       const size_t view_stride = (size_t)p.z_stride * G;
       const double* z = p.zbuf + (size_t)lh * 2 * view_stride + (size_t)off * G;
       const double* zs = p.zstat + ((size_t)lh * (p.max_boundary_tokens / GP_PAGE) + off / GP_PAGE) * G2 * 2;
@@ -1376,7 +1394,7 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
               p.Hx + (((size_t)r * p.L + l) * p.Hkv + h) * 2);
     }
     // ---- the last CTA to finish its jobs takes the decisions and tells the others ------------------------------
-    const int stamp = serial + 1;
+    const int stamp = same_step ? p.hdr[HDR_STEP] : serial + 1;
     __syncthreads();
     if (tid == 0) {
       __threadfence();
@@ -1387,7 +1405,7 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
     __syncthreads();
     if (s_i[2]) {
       __threadfence();
-      decide_and_allocate(p, nullptr, 0, n_bnd, nullptr, reinterpret_cast<int*>(S.sbuf), serial);
+      decide_and_allocate(p, req_ids, n_req_merge, n_bnd, same_step ? actions : nullptr, reinterpret_cast<int*>(S.sbuf), serial);
       __syncthreads();
       if (tid == 0 && !(p.withhold & GP_WITHHOLD_DECIDED)) {      // (test support: see GP_WITHHOLD_DECIDED)
         __threadfence();
@@ -1405,6 +1423,7 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
     compact_body<D, SHR>(p, cmp_smem_at(smem), serial);
   }
   gp_pdl_wait();              // the attention kernel beside which this grid ran has ended
+  if (same_step) gp_pdl_launch_dependents();
   if (out_merge) merge_partials(pa, n_req_merge, out_merge, pa.hdr[HDR_N_MC], pa.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, 0, LH);
 }
 
@@ -1442,12 +1461,12 @@ void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_com
 // asynchronous mode: the boundary chain of the step whose view is `p` (none when !has_chain), and afterwards the
 // merge of the split requests' partial outputs of the step whose view is `pa` (none when out_merge is null)
 void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* out_merge, int serial, int has_chain, int grid,
-                     cudaStream_t s, bool pdl) {
+                     cudaStream_t s, bool pdl, const int* req_ids, int* actions) {
   const size_t sm = gp_bsel_smem(p);
   const bool shr = p.policy == GP_POLICY_SHRINK;
   auto launch = [&](auto kern) {
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    gp_launch(kern, grid, SEL_T, sm, s, pdl, p, pa, n_req_merge, out_merge, serial, has_chain);
+    gp_launch(kern, grid, SEL_T, sm, s, pdl, p, pa, n_req_merge, out_merge, serial, has_chain, req_ids, actions);
   };
   if (p.d == 128) { if (shr) launch(gp_chain_kernel<128, true>); else launch(gp_chain_kernel<128, false>); }
   else { if (shr) launch(gp_chain_kernel<64, true>); else launch(gp_chain_kernel<64, false>); }

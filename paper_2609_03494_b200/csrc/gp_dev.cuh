@@ -26,6 +26,7 @@
 #define GP_MOVE_TOK 64         // source slots per compaction chunk
 #define GP_COST_BINS 288       // cost classes of attention work items (pages, x4 at a boundary)
 #define GP_DESC_INTS 16        // ints per attention work descriptor
+#define GP_ATTN_CONSUMERS 4    // consumer warps of an attention thread block: each reports once per item it worked on
 
 // plan header slots (int32)
 enum {
@@ -48,7 +49,8 @@ enum {
 enum {
   GP_WITHHOLD_ITEM = 1,     // attention kernel, first CTA: its second work item is never published to the consumers
   GP_WITHHOLD_CHUNK = 2,    // compaction: the first chunk of a unit never says that its sources are read
-  GP_WITHHOLD_DECIDED = 4,  // asynchronous chain kernel: the deciding CTA never tells the others
+  GP_WITHHOLD_DECIDED = 4,  // boundary kernel: the deciding CTA never tells the others
+  GP_WITHHOLD_READY = 8,    // attention kernel: the consumer warps never report a boundary unit's logits complete
 };
 
 // error bits
@@ -57,6 +59,7 @@ enum {
   GP_E_FREELIST = 2,    // free-list accounting went negative or overflowed
   GP_E_BOUNDS = 4,      // an index failed a bounds check and the access was skipped
   GP_E_SPIN_CMP = 8,    // the compaction kernel's bounded wait on the previous chunk gave up
+  GP_E_SPIN_SEL = 16,   // a selection job's bounded wait for its unit's summary logits gave up
 };
 
 struct GpDev {
@@ -108,6 +111,7 @@ struct GpDev {
                                          //   13 index of its partial-output slot
   int4* mc_list;                         // [M] split requests: {batch index, first partial, chunks, 0}
   int4* bnd_info;                        // [M][2] requests at a boundary: {slot in the batch, request, P, position of the step's token}, {score offset lo, hi, 0, 0}
+  int* unit_ready;                       // [M][L H_kv] per boundary unit: consumer warps of the attention kernel done with it
   int* bnd_acc;                          // [M][4] per boundary request: sum of K^S, sum of K^L, shared pages of C, 0
   int* free_peek;                        // [M+1] free_top at plan time, then the top entries of the free list, top first
   int4* cmp_info;                        // [M+1] compressing requests: {request, P, index in bnd_info, first compaction chunk}
@@ -266,7 +270,7 @@ inline cudaError_t gp_launch(void (*kern)(KArgs...), int grid, int block, size_t
 
 void gp_attention_setup(const GpDev& p);
 void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* out_merge, int serial, int has_chain, int grid,
-                     cudaStream_t s, bool pdl);
+                     cudaStream_t s, bool pdl, const int* req_ids = nullptr, int* actions = nullptr);
 // merge of the split requests' partial outputs for the units [lh0, lh0 + lh_n) (per-layer entry point)
 void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl);
 void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact);

@@ -24,6 +24,7 @@ struct gp_pool {
   GpDev dev_alt;
   int chain_pending;                                // the last step's boundary chain has not been launched yet
   int attn_grid_async, chain_grid;
+  int attn_grid_ov, chain_grid_ov;                  // synchronous mode with the boundary work beside the attention kernel
   long long serial;                                 // decode steps issued so far
   void* blob;
   size_t bytes;
@@ -57,7 +58,7 @@ namespace {
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, Hx, delta, rc,
       mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
-      bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
+      unit_ready, bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
       evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, qn, kn, total;
   int max_rc;
@@ -93,8 +94,9 @@ bool valid_config(const gp_config* c) {
   if (c->n_pages < 1 || c->n_pages * sub > 0x7fffffffLL / GP_PAGE) return false;
   if (c->k_loc < 0 || c->k_loc > c->page_size) return false;
   if (c->max_batch_tokens < 0 || c->max_boundary_tokens < 0) return false;
-  if (c->demand_metric < GP_METRIC_TOP_P || c->demand_metric > GP_METRIC_ENTROPY || c->reserved != 0) return false;
+  if (c->demand_metric < GP_METRIC_TOP_P || c->demand_metric > GP_METRIC_ENTROPY) return false;
   if (c->async_boundary < 0 || c->async_boundary > 1 || c->async_slots < 0 || c->async_slots > 4096) return false;
+  if (c->overlap_slots < -1 || c->overlap_slots > 4096) return false;
   if (!(c->beta_s >= 0.0 && c->beta_s < 1.0 && c->beta_l >= 0.0 && c->beta_l < 1.0)) return false;
   if (!(c->top_p > 0.0 && c->top_p < 1.0)) return false;
   if (!(c->rope_theta >= 0.0)) return false;
@@ -140,6 +142,7 @@ Layout make_layout(const gp_config& c) {
   L.mc_list = take(M * 16);
   L.bnd_info = take(M * 32);
   L.bnd_acc = take(M * 16);
+  L.unit_ready = take((size_t)M * LH * 4);
   L.free_peek = take((M + 1) * 4);
   L.cmp_info = take((M + 1) * 16);
   L.zbuf = take(LH * (Tb + b) * 2 * G * 8);
@@ -545,7 +548,8 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
     actions[i] = act;
     if (isb) {
       p.bnd_info[2 * bnd_idx] = make_int4(i, r, Pr, (int)pos);     // pos: position of this step's token
-      p.bnd_info[2 * bnd_idx + 1] = make_int4((int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32), 0, 0);
+      // .z: reports the attention kernel makes per (layer, head) unit of this request (one per consumer warp and item)
+      p.bnd_info[2 * bnd_idx + 1] = make_int4((int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32), GP_ATTN_CONSUMERS * chunks, 0);
       reinterpret_cast<int4*>(p.bnd_acc)[bnd_idx] = make_int4(0, 0, 0, 0);
     }
     // descriptors of this request's chunks: four 16-byte stores each
@@ -556,7 +560,7 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       d[0] = make_int4(i, r, pg0, min(cp, pages - pg0));
       d[1] = make_int4(c, chunks, n_old, (int)pos);
       d[2] = make_int4(flags, Pr, (int)(unsigned)(tok_off & 0xffffffffLL), (int)(tok_off >> 32));
-      d[3] = make_int4(par, rc_off + c, 0, 0);
+      d[3] = make_int4(par, rc_off + c, 0, isb ? bnd_idx : 0);
     }
     if (chunks > 1) p.mc_list[atomicAdd(&s_nmc, 1)] = make_int4(i, rc_off, chunks, 0);
   }
@@ -576,6 +580,8 @@ gp_plan_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       }
     }
   }
+  // the attention kernel counts, per unit of a boundary request, the work items its consumer warps have finished
+  for (int idx = threadIdx.x; idx < n_bnd * p.L * p.Hkv; idx += GP_PLAN_THREADS) p.unit_ready[idx] = 0;
   __syncthreads();
   if (threadIdx.x == 0) {
     p.hdr[HDR_N_MC] = s_nmc;
@@ -854,6 +860,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.mc_list = reinterpret_cast<int4*>(base + L.mc_list);
   d.bnd_info = reinterpret_cast<int4*>(base + L.bnd_info);
   d.bnd_acc = reinterpret_cast<int*>(base + L.bnd_acc);
+  d.unit_ready = reinterpret_cast<int*>(base + L.unit_ready);
   d.free_peek = reinterpret_cast<int*>(base + L.free_peek);
   d.cmp_info = reinterpret_cast<int4*>(base + L.cmp_info);
   d.zbuf = reinterpret_cast<double*>(base + L.zbuf);
@@ -887,6 +894,16 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
     if (slots > pool->attn_grid / 2) slots = pool->attn_grid / 2;
     pool->attn_grid_async = pool->attn_grid - slots;
     pool->chain_grid = slots;
+  }
+  pool->attn_grid_ov = pool->attn_grid;
+  pool->chain_grid_ov = 0;
+  if (!cfg->async_boundary && cfg->overlap_slots == 0) {
+    pool->chain_grid_ov = pool->sel_grid;          // the whole grid, behind the attention kernel's
+  } else if (!cfg->async_boundary && cfg->overlap_slots > 0) {
+    int slots = cfg->overlap_slots;
+    if (slots > pool->attn_grid / 2) slots = pool->attn_grid / 2;
+    pool->attn_grid_ov = pool->attn_grid - slots;
+    pool->chain_grid_ov = slots;
   }
   pool->dbg = base + L.dbg;
   pool->qn = reinterpret_cast<__nv_bfloat16*>(base + L.qn);
@@ -1000,14 +1017,31 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
     if (prof) cudaEventRecord(pool->ev[0], s);
     // first_plain: the kernel before the plan on the stream is not one of this library's (the host entry point's
     // fetch of the inputs): no programmatic dependence on it
-    launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl && !pool->first_plain);
-    if (prof) cudaEventRecord(pool->ev[1], s);
-    gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH, 0);
-    if (prof) cudaEventRecord(pool->ev[2], s);
-    gp_launch_boundary(d, dev_req_ids, n_req, dev_actions,
-                       static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s, prof ? pool->ev[3] : nullptr, pdl, serial);
-    if (prof) cudaEventRecord(pool->ev[4], s);
-    pool->launch_count += GP_N_KERNELS;
+    if (pool->chain_grid_ov > 0) {
+      // Three kernels.  The boundary work of the step (selection jobs, decisions, compaction, then the merge of the
+      // split outputs) is one kernel behind the attention kernel.  Its thread blocks take their places as that
+      // kernel's leave (or, with overlap_slots > 0, run beside it on slots its grid leaves free), and a selection job
+      // starts as soon as the attention kernel has reported its unit's summary logits complete.
+      launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl && !pool->first_plain, false,
+                  nullptr, pool->attn_grid_ov);
+      if (prof) cudaEventRecord(pool->ev[1], s);
+      gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid_ov, s, pdl, 0, LH, 0);
+      if (prof) cudaEventRecord(pool->ev[2], s);
+      gp_launch_chain(d, d, n_req, static_cast<float*>(out), serial, 1, pool->chain_grid_ov, s, pdl, dev_req_ids, dev_actions);
+      if (prof) { cudaEventRecord(pool->ev[3], s); cudaEventRecord(pool->ev[4], s); }    // the last interval stays empty
+      pool->launch_count += 3;
+    } else {
+      // Four kernels, one after the other (overlap_slots = -1): the selection and compaction kernels of the
+      // layer-by-layer step
+      launch_plan(pool, dev_req_ids, n_req, dev_actions, q, pool->early_plan ? 2 : 1, 0, LH, s, pdl && !pool->first_plain);
+      if (prof) cudaEventRecord(pool->ev[1], s);
+      gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, pdl, 0, LH, 0);
+      if (prof) cudaEventRecord(pool->ev[2], s);
+      gp_launch_boundary(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, pool->compact_grid, s,
+                         prof ? pool->ev[3] : nullptr, pdl, serial);
+      if (prof) cudaEventRecord(pool->ev[4], s);
+      pool->launch_count += GP_N_KERNELS;
+    }
   } else {
     // Asynchronous boundary work, all on the caller's stream: plan and attention of this step, then one kernel
     // with the boundary chain of the step before (working sets, decisions, compaction), which runs beside the
@@ -1449,7 +1483,7 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
 }
 
 int gp_test_withhold(gp_pool* pool, int32_t what, int32_t spin_limit) {
-  if (!pool || what < 0 || what > 7 || spin_limit < 0) return GP_ERR_INVALID;
+  if (!pool || what < 0 || what > 15 || spin_limit < 0) return GP_ERR_INVALID;
   GpDev* views[2] = {&pool->dev, &pool->dev_alt};
   for (GpDev* v : views) {
     v->withhold = what;

@@ -59,6 +59,7 @@ def make_pools(wl: W.Workload, device: int = 0, **over):
     ocfg = O.OracleConfig(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, page_size=s.page_size, recent_window=16, **kw, **tun)
     gcfg = B.make_config(s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, page_size=s.page_size, **kw, **tun,
                          max_batch_tokens=over.get("max_batch_tokens", 0), async_slots=over.get("async_slots", 0),
+                         overlap_slots=over.get("overlap_slots", 0),
                          max_boundary_tokens=over.get("max_boundary_tokens", 0))
     return B.Pool(gcfg, device), O.OraclePool(ocfg)
 

@@ -204,7 +204,7 @@ def test_attention_wait_that_runs_out_is_reported_and_the_kernel_drains():
         pool.close()
 
 
-@pytest.mark.parametrize("async_boundary,what,bit", [(False, 2, 8), (True, 2, 8), (True, 4, 8)])
+@pytest.mark.parametrize("async_boundary,what,bit", [(False, 2, 8), (True, 2, 8), (True, 4, 8), (False, 4, 8), (False, 8, 16)])
 def test_compaction_and_decision_waits_that_run_out_are_reported(async_boundary, what, bit):
     import torch
     # one request of eight pages that fills its last slot with the first step and compresses: two chunks per unit
