@@ -175,6 +175,9 @@ class Job:
         self.act_dev = torch.zeros(self.nreq, dtype=torch.int32, device=dev)
         self.out_host = torch.zeros((s.n_layers, self.nreq, s.n_q_heads, s.head_dim), dtype=torch.float32).pin_memory()
         self.act_host = torch.zeros(self.nreq, dtype=torch.int32).pin_memory()
+        # a second pair of result buffers for the pipelined host loop (step t + 1 is issued while t's results are read)
+        self.out_host2 = torch.zeros_like(self.out_host).pin_memory()
+        self.act_host2 = torch.zeros_like(self.act_host).pin_memory()
         self._host_ptrs = None
         self.live = False
         self.by_layer = False           # True: steps go through gp_step_begin / gp_attn_layer / gp_step_end
@@ -209,6 +212,16 @@ class Job:
         h, ids, qp, kp, vp, op, ap, qs, ks, strm = self._host_ptrs
         t = self.t
         self.B.gp_decode_step_host(h, ids, self.nreq, qp + t * qs, kp + t * ks, vp + t * ks, op, ap, strm)
+        self.t += 1
+
+    def step_host_async(self, which):
+        # the same through gp_decode_step_host_async, results into buffer pair `which`
+        assert self._host_ptrs is not None          # worked out by step_host's first call
+        h, ids, qp, kp, vp, op, ap, qs, ks, strm = self._host_ptrs
+        if which:
+            op, ap = self.out_host2.data_ptr(), self.act_host2.data_ptr()
+        t = self.t
+        self.B.gp_decode_step_host_async(h, ids, self.nreq, qp + t * qs, kp + t * ks, vp + t * ks, op, ap, strm)
         self.t += 1
 
     def roll(self, t_to):
@@ -397,8 +410,38 @@ def run_ours(args):
         head.step_host()
     B.gp_async_join(head.pool.handle, head.pool.stream())
     torch.cuda.synchronize(device)
+    e2e_block_ms = (time.perf_counter() - t0) * 1e3
+    shard.barrier(device)
+    e2e_block_tokens = int(head.counters()[6]) - tok0
+    e2e_block_value, _ = shard.job_throughput(e2e_block_tokens, e2e_block_ms, device)
+    # The same with the host one step behind the GPU, as a serving loop with asynchronous scheduling runs it: step t
+    # is issued (gp_decode_step_host_async: inputs fetched from pinned host memory, results written to pinned host
+    # memory by the kernels), then the host waits for step t - 1 and reads its actions.  Every step's inputs cross
+    # the bus inside the timed region, every step's results are read by the host inside it.
+    head.reset()
+    head.roll(max(S0 - 2, 0))
+    while head.t < S0:                      # untimed: the path's own first calls (its stream and events are made then)
+        head.step_host_async(head.t & 1)
+    torch.cuda.synchronize(device)
+    tok0 = int(head.counters()[6])
+    evs = [torch.cuda.Event(), torch.cuda.Event()]
+    act_np = [head.act_host.numpy(), head.act_host2.numpy()]      # views of the pinned result buffers
+    acts_seen = 0
+    shard.barrier(device)
+    t0 = time.perf_counter()
+    for j in range(K):
+        head.step_host_async(j & 1)
+        evs[j & 1].record()
+        if j > 0:
+            evs[(j - 1) & 1].synchronize()
+            acts_seen += int(np.count_nonzero(act_np[(j - 1) & 1]))
+    evs[(K - 1) & 1].synchronize()
+    acts_seen += int(np.count_nonzero(act_np[(K - 1) & 1]))
+    B.gp_async_join(head.pool.handle, head.pool.stream())
+    torch.cuda.synchronize(device)
     e2e_ms_local = (time.perf_counter() - t0) * 1e3
     shard.barrier(device)
+    assert B.gp_pool_status(head.pool.handle)[0] == B.GP_OK
     e2e_tokens = int(head.counters()[6]) - tok0
     e2e_value, _ = shard.job_throughput(e2e_tokens, e2e_ms_local, device)
     h2d = int(s.n_layers * head.nreq * (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim * 2 + 4 * head.nreq)
@@ -431,7 +474,11 @@ def run_ours(args):
             "roofline": roofline, "step_roofline": step_roofline,
             "cpu_baseline": cpu,
             "e2e": {"value": round(e2e_value, 1), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms_local / K, 5)},
+                    "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms_local / K, 5),
+                    "how": "gp_decode_step_host_async, the host reads step t - 1's results while step t runs",
+                    "blocking": {"value": round(e2e_block_value, 1), "ms_per_step": round(e2e_block_ms / K, 5),
+                                 "how": "gp_decode_step_host, one synchronisation per step"},
+                    "boundary_actions_read": acts_seen},
             "gpu_launches": int(gpu_launches),
             "clocks": clocks,
             "events": {"grow": int(counters[0]), "compress": int(counters[1]), "fallback": int(counters[2]),

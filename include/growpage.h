@@ -274,6 +274,16 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
                         const void* q, const void* k, const void* v,
                         void* out, int32_t* actions, void* stream);
 
+/* The same step without the synchronisation at the end: everything is enqueued on `stream` and the call returns.
+ * The caller's input buffers must stay as they are until the step's first kernel has run, `out` and `actions`
+ * hold the results once the work enqueued by this call has completed (an event recorded on `stream` after the
+ * call, or a synchronisation), and kernel-reported errors are read with gp_pool_status then.  A serving loop
+ * can so issue step t + 1 while it still reads the results of step t from a second pair of output buffers: the
+ * GPU never waits for the host's wake-up and launches between steps. */
+int gp_decode_step_host_async(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req,
+                              const void* q, const void* k, const void* v,
+                              void* out, int32_t* actions, void* stream);
+
 /* Ends a request: every page of its table loses one reference and returns to the free list at
  * zero; the summary slot is recycled without clearing (App. D.1).  Asynchronous on `stream`.
  * GP_ERR_STATE between gp_step_begin and gp_step_end. */

@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
     L.gp_request_add.argtypes = [vp, i32, i32, vp, vp, i32, i32, vp, C.POINTER(i32)]
     L.gp_decode_step.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.gp_decode_step_host.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
+    L.gp_decode_step_host_async.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.gp_release.argtypes = [vp, i32, vp]
     L.gp_strerror.argtypes = [C.c_int]; L.gp_strerror.restype = C.c_char_p
     L.gp_debug_request.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i64), vp]
@@ -142,6 +143,13 @@ def gp_decode_step_host(pool: int, host_req_ids_ptr: int, n_req: int, q_ptr: int
     _check(lib().gp_decode_step_host(C.c_void_p(pool), C.c_void_p(host_req_ids_ptr), n_req, C.c_void_p(q_ptr),
                                      C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr),
                                      C.c_void_p(actions_ptr), C.c_void_p(stream)), "gp_decode_step_host")
+
+
+def gp_decode_step_host_async(pool: int, host_req_ids_ptr: int, n_req: int, q_ptr: int, k_ptr: int, v_ptr: int,
+                              out_ptr: int, actions_ptr: int, stream: int) -> None:
+    _check(lib().gp_decode_step_host_async(C.c_void_p(pool), C.c_void_p(host_req_ids_ptr), n_req, C.c_void_p(q_ptr),
+                                           C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr),
+                                           C.c_void_p(actions_ptr), C.c_void_p(stream)), "gp_decode_step_host_async")
 
 
 def gp_step_begin(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: int, stream: int) -> None:
@@ -351,6 +359,12 @@ class Pool:
         """All arguments are host tensors (pinned recommended)."""
         gp_decode_step_host(self.handle, req_ids.data_ptr(), int(req_ids.numel()), q.data_ptr(), k.data_ptr(),
                             v.data_ptr(), out.data_ptr(), actions.data_ptr(), self.stream())
+
+    def decode_step_host_async(self, req_ids, q, k, v, out, actions) -> None:
+        """As decode_step_host, without the synchronisation at the end: results are there once the stream has run
+        the work (the caller records an event or synchronises)."""
+        gp_decode_step_host_async(self.handle, req_ids.data_ptr(), int(req_ids.numel()), q.data_ptr(), k.data_ptr(),
+                                  v.data_ptr(), out.data_ptr(), actions.data_ptr(), self.stream())
 
     def release(self, req: int) -> None:
         gp_release(self.handle, req, self.stream())

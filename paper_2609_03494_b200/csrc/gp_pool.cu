@@ -37,6 +37,12 @@ struct gp_pool {
   int* h_err;
   // staging for the host-pointer entry point (inside the blob)
   int* st_ids; void* st_q; void* st_k; void* st_v; float* st_out; int* st_act;
+  // The host entry points fetch a step's inputs on a stream of their own into one of two staging sets, so that the
+  // fetch of step t + 1 runs beside the kernels of step t when the caller issues steps ahead.
+  int* st2_ids; void* st2_q; void* st2_k; void* st2_v;
+  cudaStream_t fetch_stream;
+  cudaEvent_t ev_fetch[2], ev_used[2];              // set fetched; set no longer read by the step that used it
+  long long host_steps;                             // steps issued through the host entry points
   __nv_bfloat16* qn; __nv_bfloat16* kn;             // one layer's normalised queries and keys (gp_attn_layer_qknorm)
   // small device words
   int* d_status;
@@ -60,7 +66,7 @@ struct Layout {
       mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
       unit_ready, bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
       evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
-      st_ids, st_q, st_k, st_v, st_out, st_act, qn, kn, total;
+      st_ids, st_q, st_k, st_v, st_out, st_act, st2_ids, st2_q, st2_k, st2_v, qn, kn, total;
   int max_rc;
   long long max_batch_tokens, max_boundary_tokens;
 };
@@ -174,10 +180,14 @@ Layout make_layout(const gp_config& c) {
     L.st_q = take((size_t)c.n_layers * M * c.n_q_heads * d * 2);
     L.st_k = take((size_t)c.n_layers * M * c.n_kv_heads * d * 2);
     L.st_v = take((size_t)c.n_layers * M * c.n_kv_heads * d * 2);
+    L.st2_ids = take(M * 4);
+    L.st2_q = take((size_t)c.n_layers * M * c.n_q_heads * d * 2);
+    L.st2_k = take((size_t)c.n_layers * M * c.n_kv_heads * d * 2);
+    L.st2_v = take((size_t)c.n_layers * M * c.n_kv_heads * d * 2);
     L.st_out = take((size_t)c.n_layers * M * c.n_q_heads * d * 4);
     L.st_act = take(M * 4);
   } else {
-    L.st_ids = L.st_q = L.st_k = L.st_v = L.st_out = L.st_act = 0;
+    L.st_ids = L.st_q = L.st_k = L.st_v = L.st_out = L.st_act = L.st2_ids = L.st2_q = L.st2_k = L.st2_v = 0;
   }
   L.qn = take(M * c.n_q_heads * d * 2);              // one layer's normalised queries and keys (fused QK-norm)
   L.kn = take(M * c.n_kv_heads * d * 2);
@@ -713,6 +723,10 @@ __global__ void gp_gather_kernel(GpDev p, int r, int l, int h, int n, int* tok_o
 
 void pool_free(gp_pool* pool) {
   if (pool->h_err) cudaFreeHost(pool->h_err);
+  if (pool->fetch_stream) {
+    cudaStreamDestroy(pool->fetch_stream);
+    for (int i = 0; i < 2; ++i) { cudaEventDestroy(pool->ev_fetch[i]); cudaEventDestroy(pool->ev_used[i]); }
+  }
   delete pool;
 }
 
@@ -911,6 +925,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   if (cfg->host_staging) {
     pool->st_ids = reinterpret_cast<int*>(base + L.st_ids);
     pool->st_q = base + L.st_q; pool->st_k = base + L.st_k; pool->st_v = base + L.st_v;
+    pool->st2_ids = reinterpret_cast<int*>(base + L.st2_ids);
+    pool->st2_q = base + L.st2_q; pool->st2_k = base + L.st2_k; pool->st2_v = base + L.st2_v;
     pool->st_out = reinterpret_cast<float*>(base + L.st_out);
     pool->st_act = reinterpret_cast<int*>(base + L.st_act);
   } else {
@@ -1223,8 +1239,8 @@ __global__ void gp_fetch_inputs_kernel(int* __restrict__ d_ids, const int* __res
   }
 }
 
-int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
-                        const void* v, void* out, int32_t* actions, void* stream) {
+static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
+                     const void* v, void* out, int32_t* actions, void* stream, bool wait) {
   if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
   if (!pool->st_ids || pool->step_open) return GP_ERR_STATE;
   if (n_req == 0) return GP_OK;
@@ -1234,7 +1250,16 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
   const gp_config& c = pool->cfg;
   const size_t qb = (size_t)c.n_layers * n_req * c.n_q_heads * c.head_dim * 2;
   const size_t kb = (size_t)c.n_layers * n_req * c.n_kv_heads * c.head_dim * 2;
-  // Inputs: from mapped page-locked buffers one kernel fetches all four over the bus; otherwise four copies.
+  // Inputs: from mapped page-locked buffers one kernel fetches all four over the bus into one of two staging sets.
+  // When the caller issues steps ahead (gp_decode_step_host_async) the fetch runs on a stream of its own, beside
+  // the kernels of the step before it: it waits until the step that last used the set has read it, and the step
+  // waits for its fetch.  The call that waits for its step fetches on the caller's stream (nothing to overlap
+  // with).  Pageable memory: four copies on the caller's stream.
+  const int set = (int)(pool->host_steps & 1);
+  int* st_ids = set ? pool->st2_ids : pool->st_ids;
+  void* st_q = set ? pool->st2_q : pool->st_q;
+  void* st_k = set ? pool->st2_k : pool->st_k;
+  void* st_v = set ? pool->st2_v : pool->st_v;
   {
     void *mi = nullptr, *mq = nullptr, *mk = nullptr, *mv = nullptr;
     const bool mapped = ((uintptr_t)host_req_ids % 4 == 0) && ((uintptr_t)q % 16 == 0) && ((uintptr_t)k % 16 == 0) &&
@@ -1243,24 +1268,47 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
                         cudaHostGetDevicePointer(&mq, const_cast<void*>(q), 0) == cudaSuccess &&
                         cudaHostGetDevicePointer(&mk, const_cast<void*>(k), 0) == cudaSuccess &&
                         cudaHostGetDevicePointer(&mv, const_cast<void*>(v), 0) == cudaSuccess;
-    if (mapped) {
+    if (mapped && wait) {
       const long long pieces = (long long)(qb + 2 * kb) / 16;         // a row is 128 or 256 bytes: whole pieces
       int grid = (int)((pieces + 255) / 256);
       if (grid > pool->num_sms * 8) grid = pool->num_sms * 8;
       if (grid * 256 < n_req) grid = (n_req + 255) / 256;
-      gp_fetch_inputs_kernel<<<grid, 256, 0, s>>>(pool->st_ids, static_cast<const int*>(mi), n_req,
-                                                 static_cast<uint4*>(pool->st_q), static_cast<const uint4*>(mq), (long long)qb / 16,
-                                                 static_cast<uint4*>(pool->st_k), static_cast<const uint4*>(mk), (long long)kb / 16,
-                                                 static_cast<uint4*>(pool->st_v), static_cast<const uint4*>(mv), (long long)kb / 16);
+      gp_fetch_inputs_kernel<<<grid, 256, 0, s>>>(st_ids, static_cast<const int*>(mi), n_req,
+                                                 static_cast<uint4*>(st_q), static_cast<const uint4*>(mq), (long long)qb / 16,
+                                                 static_cast<uint4*>(st_k), static_cast<const uint4*>(mk), (long long)kb / 16,
+                                                 static_cast<uint4*>(st_v), static_cast<const uint4*>(mv), (long long)kb / 16);
       pool->launch_count++;
+    } else if (mapped) {
+      if (!pool->fetch_stream) {
+        GP_CUDA(cudaStreamCreateWithFlags(&pool->fetch_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+          GP_CUDA(cudaEventCreateWithFlags(&pool->ev_fetch[i], cudaEventDisableTiming));
+          GP_CUDA(cudaEventCreateWithFlags(&pool->ev_used[i], cudaEventDisableTiming));
+          GP_CUDA(cudaEventRecord(pool->ev_used[i], s));
+        }
+      }
+      cudaStream_t fs = pool->fetch_stream;
+      GP_CUDA(cudaStreamWaitEvent(fs, pool->ev_used[set], 0));
+      const long long pieces = (long long)(qb + 2 * kb) / 16;         // a row is 128 or 256 bytes: whole pieces
+      int grid = (int)((pieces + 255) / 256);
+      if (grid > pool->num_sms * 8) grid = pool->num_sms * 8;
+      if (grid * 256 < n_req) grid = (n_req + 255) / 256;
+      gp_fetch_inputs_kernel<<<grid, 256, 0, fs>>>(st_ids, static_cast<const int*>(mi), n_req,
+                                                  static_cast<uint4*>(st_q), static_cast<const uint4*>(mq), (long long)qb / 16,
+                                                  static_cast<uint4*>(st_k), static_cast<const uint4*>(mk), (long long)kb / 16,
+                                                  static_cast<uint4*>(st_v), static_cast<const uint4*>(mv), (long long)kb / 16);
+      pool->launch_count++;
+      GP_CUDA(cudaEventRecord(pool->ev_fetch[set], fs));
+      GP_CUDA(cudaStreamWaitEvent(s, pool->ev_fetch[set], 0));
     } else {
       (void)cudaGetLastError();                    // pageable memory: not an error
-      GP_CUDA(cudaMemcpyAsync(pool->st_ids, host_req_ids, (size_t)n_req * 4, cudaMemcpyHostToDevice, s));
-      GP_CUDA(cudaMemcpyAsync(pool->st_q, q, qb, cudaMemcpyHostToDevice, s));
-      GP_CUDA(cudaMemcpyAsync(pool->st_k, k, kb, cudaMemcpyHostToDevice, s));
-      GP_CUDA(cudaMemcpyAsync(pool->st_v, v, kb, cudaMemcpyHostToDevice, s));
+      GP_CUDA(cudaMemcpyAsync(st_ids, host_req_ids, (size_t)n_req * 4, cudaMemcpyHostToDevice, s));
+      GP_CUDA(cudaMemcpyAsync(st_q, q, qb, cudaMemcpyHostToDevice, s));
+      GP_CUDA(cudaMemcpyAsync(st_k, k, kb, cudaMemcpyHostToDevice, s));
+      GP_CUDA(cudaMemcpyAsync(st_v, v, kb, cudaMemcpyHostToDevice, s));
     }
   }
+  pool->host_steps += 1;
   // Outputs: when the caller's buffers are page-locked and mapped (the usual pinned allocation), the kernels
   // write them over the bus while they run and nothing is left to copy when the step ends.  (The same was tried
   // for the inputs and was slower: rows read over the bus by the kernels stall the pipelines that wait for them.)
@@ -1275,18 +1323,30 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
   const int early = pool->early_plan;
   pool->early_plan = 1;
   pool->first_plain = 1;
-  const int st = gp_decode_step(pool, pool->st_ids, n_req, pool->st_q, pool->st_k, pool->st_v,
+  const int st = gp_decode_step(pool, st_ids, n_req, st_q, st_k, st_v,
                                 direct ? d_out : static_cast<void*>(pool->st_out),
                                 direct ? static_cast<int32_t*>(d_act) : pool->st_act, stream);
   pool->early_plan = early;
   pool->first_plain = 0;
   if (st != GP_OK) return st;
+  if (pool->fetch_stream) GP_CUDA(cudaEventRecord(pool->ev_used[set], s));       // the set may be fetched into again
   if (!direct) {
     GP_CUDA(cudaMemcpyAsync(out, pool->st_out, qb * 2, cudaMemcpyDeviceToHost, s));
     GP_CUDA(cudaMemcpyAsync(actions, pool->st_act, (size_t)n_req * 4, cudaMemcpyDeviceToHost, s));
   }
+  if (!wait) return GP_OK;
   GP_CUDA(cudaStreamSynchronize(s));
   return kernel_status(pool);
+}
+
+int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
+                        const void* v, void* out, int32_t* actions, void* stream) {
+  return host_step(pool, host_req_ids, n_req, q, k, v, out, actions, stream, true);
+}
+
+int gp_decode_step_host_async(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
+                              const void* v, void* out, int32_t* actions, void* stream) {
+  return host_step(pool, host_req_ids, n_req, q, k, v, out, actions, stream, false);
 }
 
 int gp_pool_status(gp_pool* pool, int32_t* error_bits) {

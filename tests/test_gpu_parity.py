@@ -564,13 +564,15 @@ def test_sequence_lengths_around_chunk_and_page_edges():
         assert st.steps == 3 and st.attn_max_abs <= LS.ATTN_MAX_ABS
 
 
-def test_host_entry_point_with_pageable_buffers():
+def test_host_entry_point_with_pageable_buffers_and_without_the_final_wait():
     # gp_decode_step_host fetches pinned inputs with one kernel over the bus (the ids fill whole 16-byte pieces
-    # here: four requests) and writes pinned outputs over the bus as it runs; pageable buffers take copies
+    # here: four requests) and writes pinned outputs over the bus as it runs; pageable buffers take copies.
+    # gp_decode_step_host_async is the same without the synchronisation at the end: the loop below issues step t,
+    # then waits for step t - 1 and reads its results from the other of two pairs of result buffers.
     import torch
     cfg = B.make_config(1, 8, 2, 64, n_pages=32, max_pages_per_req=4, max_requests=8, host_staging=True)
     results = []
-    for pinned in (True, False):
+    for mode in ("pinned", "pageable", "pinned, one step behind"):
         pool = B.Pool(cfg)
         try:
             rng = np.random.default_rng(0)
@@ -578,22 +580,37 @@ def test_host_entry_point_with_pageable_buffers():
             kt, vt = bits(1, 20, 2, 64), bits(1, 20, 2, 64)
             for i in range(4):
                 assert pool.request_add(-1, 0, kt, vt, 20, 0) == (B.GP_OK, i)
-            fix = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
-            outs = []
+            fix = (lambda t: t) if mode == "pageable" else (lambda t: t.pin_memory())
+            outs, pending, keep = [], None, []
             for t in range(14):                                   # crosses the boundary at n = 32
                 q, k, v = bits(1, 4, 8, 64), bits(1, 4, 2, 64), bits(1, 4, 2, 64)
                 out = fix(torch.zeros((1, 4, 8, 64), dtype=torch.float32))
                 act = fix(torch.zeros(4, dtype=torch.int32))
                 ids = fix(torch.arange(4, dtype=torch.int32))
                 tq, tk, tv = (fix(torch.from_numpy(x.view(np.int16))) for x in (q, k, v))
-                pool.decode_step_host(ids, tq, tk, tv, out, act)
-                outs.append((out.clone().numpy(), act.clone().numpy()))
+                if mode.endswith("behind"):
+                    keep.append((ids, tq, tk, tv))                # the inputs stay as they are until their step has run
+                    pool.decode_step_host_async(ids, tq, tk, tv, out, act)
+                    ev = torch.cuda.Event()
+                    ev.record()
+                    if pending is not None:
+                        pending[0].synchronize()
+                        outs.append((pending[1].clone().numpy(), pending[2].clone().numpy()))
+                    pending = (ev, out, act)
+                else:
+                    pool.decode_step_host(ids, tq, tk, tv, out, act)
+                    outs.append((out.clone().numpy(), act.clone().numpy()))
+            if pending is not None:
+                pending[0].synchronize()
+                outs.append((pending[1].clone().numpy(), pending[2].clone().numpy()))
+                assert B.gp_pool_status(pool.handle) == (B.GP_OK, 0)
             results.append(outs)
             assert B.gp_debug_pool(pool.handle)[2][7] == 0
         finally:
             pool.close()
-    for (o1, a1), (o2, a2) in zip(*results):
-        assert np.array_equal(o1, o2) and np.array_equal(a1, a2)
+    for other in results[1:]:
+        for (o1, a1), (o2, a2) in zip(results[0], other):
+            assert np.array_equal(o1, o2) and np.array_equal(a1, a2)
     assert any((a != B.GP_ACT_NONE).any() for _, a in results[0])
 
 
