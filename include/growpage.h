@@ -123,6 +123,10 @@ typedef struct gp_config {
   int32_t async_slots;       /* asynchronous boundary work: thread blocks of the attention kernel's grid
                                 given up so that the boundary kernel finds room on the SMs beside it;
                                 0 = a default (64)                                                    */
+  int32_t kv_shard_count;    /* pools that together hold the model's KV heads (Eq. 11's heads per GPU): this pool
+                                has n_kv_heads of n_kv_heads * kv_shard_count, and Delta_t is a mean over all of
+                                them (gp_decode_step_local / gp_decode_step_finish); default 1               */
+  int32_t reserved;          /* keep 0                                                              */
   int64_t n_pages;           /* physical pages; one page id covers all layers and KV heads         */
   int64_t min_capacity;      /* GP_POLICY_SHRINK: tokens of capacity a Shrink must leave, default 1024 */
   int64_t max_batch_tokens;  /* bound on the summed sequence lengths of one decode batch, used to
@@ -261,6 +265,28 @@ int gp_step_abort(gp_pool* pool);
 int gp_attn_layer_qknorm(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req,
                          const void* q_raw, const void* k_raw, const void* v, const float* q_weight,
                          const float* k_weight, double eps, void* out, void* stream);
+
+/* The step of a pool that holds a part of the model's KV heads (Eq. 11: "query heads per GPU"; every GPU of a
+ * tensor-parallel group has its own pool over the same requests, page ids and batches, with n_kv_heads of the
+ * model's n_kv_heads * kv_shard_count heads).  Scoring, working sets, selection and compaction are per (layer, KV
+ * head); the one coupling is the mean of Eq. 8, i.e. two integers per boundary request:
+ *   gp_decode_step_local   plan, attention, selection jobs (arguments as gp_decode_step, this pool's heads only);
+ *                          leaves, per boundary request in batch order, the sums of K^S and of K^L over this
+ *                          pool's units in the device array gp_shard_sums returns (int32 [max_requests][2],
+ *                          zero past the step's boundary requests);
+ *   (the caller adds the arrays of all pools up, element by element, in place: one all-reduce of
+ *    2 * max_requests int32 on `stream`, e.g. ncclAllReduce with ncclSum; nothing to do for a single pool)
+ *   gp_decode_step_finish  decisions from the completed sums (every pool takes the same ones, on its replica of the
+ *                          page tables and the free list), allocation, compaction; writes `dev_actions`.
+ * Between the two calls the pool accepts nothing else (GP_ERR_STATE).  Synchronous mode and the Top-p metric only
+ * (the entropy variant would sum doubles, in an order that differs from a single pool's).  With one pool the pair
+ * gives exactly what gp_decode_step gives. */
+int gp_decode_step_local(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req,
+                         const void* q, const void* k, const void* v,
+                         void* out, int32_t* dev_actions, void* stream);
+int gp_shard_sums(gp_pool* pool, int32_t** dev_sums, int64_t* n_ints);
+int gp_decode_step_finish(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions,
+                          void* stream);
 
 /* As gp_decode_step with HOST pointers: brings the inputs to staging inside the blob, runs the
  * step, delivers `out` and `actions` and synchronises `stream`.  When the four input buffers are

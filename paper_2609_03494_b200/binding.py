@@ -32,6 +32,7 @@ class gp_config(C.Structure):
         ("recent_window", C.c_int32), ("k_loc", C.c_int32), ("host_staging", C.c_int32),
         ("policy", C.c_int32), ("policy_seed", C.c_int32), ("async_boundary", C.c_int32), ("demand_metric", C.c_int32),
         ("overlap_slots", C.c_int32), ("async_slots", C.c_int32),
+        ("kv_shard_count", C.c_int32), ("reserved", C.c_int32),
         ("n_pages", C.c_int64), ("min_capacity", C.c_int64), ("max_batch_tokens", C.c_int64),
         ("max_boundary_tokens", C.c_int64),
         ("beta_s", C.c_double), ("beta_l", C.c_double), ("top_p", C.c_double), ("tau", C.c_double),
@@ -60,6 +61,9 @@ def lib() -> C.CDLL:
     L.gp_decode_step.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.gp_decode_step_host.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.gp_decode_step_host_async.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
+    L.gp_decode_step_local.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
+    L.gp_shard_sums.argtypes = [vp, C.POINTER(C.c_void_p), C.POINTER(C.c_int64)]
+    L.gp_decode_step_finish.argtypes = [vp, vp, i32, vp, vp]
     L.gp_release.argtypes = [vp, i32, vp]
     L.gp_strerror.argtypes = [C.c_int]; L.gp_strerror.restype = C.c_char_p
     L.gp_debug_request.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i64), vp]
@@ -179,6 +183,26 @@ def gp_step_end(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: in
 
 def gp_step_abort(pool: int) -> None:
     _check(lib().gp_step_abort(C.c_void_p(pool)), "gp_step_abort")
+
+
+def gp_decode_step_local(pool: int, dev_req_ids_ptr: int, n_req: int, q_ptr: int, k_ptr: int, v_ptr: int,
+                         out_ptr: int, dev_actions_ptr: int, stream: int) -> None:
+    _check(lib().gp_decode_step_local(C.c_void_p(pool), C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(q_ptr),
+                                      C.c_void_p(k_ptr), C.c_void_p(v_ptr), C.c_void_p(out_ptr),
+                                      C.c_void_p(dev_actions_ptr), C.c_void_p(stream)), "gp_decode_step_local")
+
+
+def gp_shard_sums(pool: int) -> Tuple[int, int]:
+    """Device address and length (int32 elements) of the array to be summed over the KV-head shards."""
+    ptr = C.c_void_p(0)
+    n = C.c_int64(0)
+    _check(lib().gp_shard_sums(C.c_void_p(pool), C.byref(ptr), C.byref(n)), "gp_shard_sums")
+    return int(ptr.value), int(n.value)
+
+
+def gp_decode_step_finish(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: int, stream: int) -> None:
+    _check(lib().gp_decode_step_finish(C.c_void_p(pool), C.c_void_p(dev_req_ids_ptr), n_req, C.c_void_p(dev_actions_ptr),
+                                       C.c_void_p(stream)), "gp_decode_step_finish")
 
 
 def gp_pool_status(pool: int) -> Tuple[int, int]:
@@ -388,7 +412,7 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
                 rope_theta: float = 0.0, policy: int = 0, policy_seed: int = 0, p_compress: float = 0.7,
                 shrink_below: float = -0.005, min_capacity: int = 1024, async_boundary: bool = False,
                 async_slots: int = 0, max_boundary_tokens: int = 0, demand_metric: int = 0, page_size: int = 16,
-                overlap_slots: int = 0) -> gp_config:
+                overlap_slots: int = 0, kv_shard_count: int = 1) -> gp_config:
     cfg = gp_config_default()
     cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, n_q_heads, n_kv_heads, head_dim
     cfg.n_pages, cfg.max_pages_per_req, cfg.max_requests = n_pages, max_pages_per_req, max_requests
@@ -398,6 +422,7 @@ def make_config(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n
     cfg.shrink_below, cfg.min_capacity = shrink_below, min_capacity
     cfg.async_boundary, cfg.async_slots, cfg.max_boundary_tokens = 1 if async_boundary else 0, async_slots, max_boundary_tokens
     cfg.overlap_slots = overlap_slots
+    cfg.kv_shard_count = kv_shard_count
     cfg.demand_metric = demand_metric
     cfg.page_size = page_size
     return cfg

@@ -419,7 +419,9 @@ __device__ __noinline__ void evict_general(const GpDev& p, const double* a, int 
 // decision + allocator, run by the last CTA of the selection kernel
 // ------------------------------------------------------------------------------------------------------
 __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_req, int n_bnd, int* actions, int* s_arr,
-                                    int serial) {
+                                    int serial, bool from_sums = false) {
+  // from_sums: the sums of K^S and K^L come from shard_sums (summed over the pools that hold the model's other KV
+  // heads) instead of this pool's own accumulators
   // In the asynchronous boundary mode this runs beside the next decode step: it touches only the requests at
   // this step's boundary (which sit that step out), reads the free list itself (the boundary chains run one
   // after the other and nothing else takes or returns pages meanwhile) and reports through last_act only
@@ -442,7 +444,8 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
     top0 = p.async ? __ldcg(p.free_top) : __ldcg(p.free_peek);
     for (int e = tid; e < n_bnd; e += blockDim.x) {
       const int4 inf = p.bnd_info[2 * e];
-      const int4 acc = __ldcg(reinterpret_cast<const int4*>(p.bnd_acc) + e);
+      int4 acc = __ldcg(reinterpret_cast<const int4*>(p.bnd_acc) + e);
+      if (from_sums) { acc.x = __ldcg(p.shard_sums + 2 * e); acc.y = __ldcg(p.shard_sums + 2 * e + 1); }
       s_free[e] = p.async ? (e < top0 ? __ldcg(p.free_stack + top0 - 1 - e) : 0) : __ldcg(p.free_peek + 1 + e);
       const int r = inf.y, Pr = inf.z;
       const int nC = (Pr - p.sub) * GP_PAGE;                // |C_t| of Eq. 7: history minus the newest page of the method
@@ -450,7 +453,7 @@ __device__ void decide_and_allocate(const GpDev& p, const int* req_ids, int n_re
       double delta = 0.0;
       int want = 1;
       if (nC > 0) {
-        delta = (double)((long long)acc.x - (long long)acc.y) / ((double)LH * (double)nC);
+        delta = (double)((long long)acc.x - (long long)acc.y) / ((double)p.units_total * (double)nC);
         if (p.metric == GP_METRIC_ENTROPY) {
           // the same mean with H / ln |C| in the place of K / |C|, summed unit by unit in (layer, head) order
           const double* hx = p.Hx + (size_t)r * LH * 2;
@@ -942,7 +945,10 @@ __device__ __forceinline__ void sel_job(const GpDev& p, const SelSmem& S, const 
 template <bool SHR>      // SHR: the pool runs the Shrink policy (a fourth job per unit)
 __global__ void __launch_bounds__(SEL_T, 2)
 gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
-               float* __restrict__ out, int serial) {
+               float* __restrict__ out, int serial, int decide) {
+  // decide == 0: the step of a pool that holds a part of the model's KV heads: the last thread block only hands
+  // out the sums of K^S and K^L per boundary request; the decisions follow in a kernel of their own once the
+  // sums of all parts are added up
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
   SelSmem S = sel_smem_at(smem);
@@ -1047,7 +1053,14 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
       }
       __syncthreads();
     }
-    decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(S.sbuf), serial);
+    if (decide) {
+      decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(S.sbuf), serial);
+    } else {
+      for (int e = tid; e < p.M; e += SEL_T) {
+        p.shard_sums[2 * e] = e < n_bnd ? __ldcg(p.bnd_acc + 4 * e) : 0;
+        p.shard_sums[2 * e + 1] = e < n_bnd ? __ldcg(p.bnd_acc + 4 * e + 1) : 0;
+      }
+    }
   }
 
   if (!idle_merge) merge_partials(p, n_req, out, n_mc, n_rc, (int)gridDim.x - 1 - (int)blockIdx.x, (int)gridDim.x, 0, LH);
@@ -1427,6 +1440,14 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
   if (out_merge) merge_partials(pa, n_req_merge, out_merge, pa.hdr[HDR_N_MC], pa.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, 0, LH);
 }
 
+// the decisions of a step whose sums of K^S and K^L were completed outside (KV heads spread over several pools)
+__global__ void __launch_bounds__(SEL_T)
+gp_decide_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
+                 int serial) {
+  __shared__ int s_arr[8 * GP_MAX_REQ];
+  decide_and_allocate(p, req_ids, n_req, __ldcg(p.hdr + HDR_N_BND), actions, s_arr, serial, true);
+}
+
 }  // namespace
 
 // the compaction kernel of a pool: head dimension, and whether the Shrink policy is on
@@ -1472,6 +1493,21 @@ void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* ou
   else { if (shr) launch(gp_chain_kernel<64, true>); else launch(gp_chain_kernel<64, false>); }
 }
 
+void gp_launch_select_only(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel, cudaStream_t s,
+                           bool pdl, int serial) {
+  const size_t sel_sm = gp_bsel_smem(p);
+  const bool shr = p.policy == GP_POLICY_SHRINK;
+  gp_launch(shr ? gp_bsel_kernel<true> : gp_bsel_kernel<false>, grid_sel, SEL_T, sel_sm, s, pdl, p, req_ids, n_req, actions, out,
+            serial, 0);
+}
+
+// plain launches: what comes before them on the stream (the caller's reduction of the sums) is not this library's
+void gp_launch_decide_compact(const GpDev& p, const int* req_ids, int n_req, int* actions, int grid_compact, cudaStream_t s,
+                              int serial) {
+  gp_launch(gp_decide_kernel, 1, SEL_T, 0, s, false, p, req_ids, n_req, actions, serial);
+  gp_launch(compact_kernel_of(p), grid_compact, CT, 0, s, true, p, req_ids, n_req, serial);
+}
+
 void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl) {
   gp_launch(gp_merge_kernel, grid, 256, 0, s, pdl, p, n_req, out, lh0, lh_n);
 }
@@ -1483,7 +1519,7 @@ void gp_launch_boundary(const GpDev& p, const int* req_ids, int n_req, int* acti
   // asynchronous mode: the kernel before this one on its stream belongs to another step (an event wait lies in
   // between): plain launch; the compaction kernel follows as a programmatic dependent as usual
   gp_launch(shr ? gp_bsel_kernel<true> : gp_bsel_kernel<false>, grid_sel, SEL_T, sel_sm, s, pdl && !p.async, p, req_ids,
-            n_req, actions, out, serial);
+            n_req, actions, out, serial, 1);
   if (ev) cudaEventRecord(ev, s);
   gp_launch(compact_kernel_of(p), grid_compact, CT, 0, s, pdl, p, req_ids, n_req, serial);
 }

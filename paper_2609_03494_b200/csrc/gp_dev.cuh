@@ -111,6 +111,9 @@ struct GpDev {
                                          //   13 index of its partial-output slot
   int4* mc_list;                         // [M] split requests: {batch index, first partial, chunks, 0}
   int4* bnd_info;                        // [M][2] requests at a boundary: {slot in the batch, request, P, position of the step's token}, {score offset lo, hi, 0, 0}
+  int* shard_sums;                       // [M][2] per boundary request: sum of K^S, sum of K^L over this pool's units (to be
+                                         // summed over the pools that hold the other KV heads), then over all units
+  int units_total;                       // (layer, KV head) units of the model: L H_kv times the number of KV-head shards
   int* unit_ready;                       // [M][L H_kv] per boundary unit: consumer warps of the attention kernel done with it
   int* bnd_acc;                          // [M][4] per boundary request: sum of K^S, sum of K^L, shared pages of C, 0
   int* free_peek;                        // [M+1] free_top at plan time, then the top entries of the free list, top first
@@ -272,6 +275,10 @@ void gp_attention_setup(const GpDev& p);
 void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* out_merge, int serial, int has_chain, int grid,
                      cudaStream_t s, bool pdl, const int* req_ids = nullptr, int* actions = nullptr);
 // merge of the split requests' partial outputs for the units [lh0, lh0 + lh_n) (per-layer entry point)
+void gp_launch_select_only(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel, cudaStream_t s,
+                           bool pdl, int serial);
+void gp_launch_decide_compact(const GpDev& p, const int* req_ids, int n_req, int* actions, int grid_compact, cudaStream_t s,
+                              int serial);
 void gp_launch_merge(const GpDev& p, int n_req, float* out, int lh0, int lh_n, int grid, cudaStream_t s, bool pdl);
 void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_compact);
 size_t gp_bsel_smem_for_cap(long long cap);

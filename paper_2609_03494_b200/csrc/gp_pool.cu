@@ -64,7 +64,7 @@ namespace {
 struct Layout {
   size_t kv, tok, refcount, free_stack, words, page_table, shadow, reqi, pos, summ, Kx, Hx, delta, rc,
       mc_list, bnd_info, bnd_acc, free_peek, cmp_info, zbuf, qtil, zstat, sum_par,
-      unit_ready, bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
+      unit_ready, shard_sums, bnd_info2, bnd_acc2, zbuf2, zstat2, rc2, mc_list2, qtil2, rope_cs2,
       evict, evict2, cflags, rope_cs, partials, scores, counters, dbg,
       st_ids, st_q, st_k, st_v, st_out, st_act, st2_ids, st2_q, st2_k, st2_v, qn, kn, total;
   int max_rc;
@@ -103,6 +103,9 @@ bool valid_config(const gp_config* c) {
   if (c->demand_metric < GP_METRIC_TOP_P || c->demand_metric > GP_METRIC_ENTROPY) return false;
   if (c->async_boundary < 0 || c->async_boundary > 1 || c->async_slots < 0 || c->async_slots > 4096) return false;
   if (c->overlap_slots < -1 || c->overlap_slots > 4096) return false;
+  if (c->kv_shard_count < 1 || c->kv_shard_count > 64 || c->reserved != 0) return false;
+  // spread over several pools, the mean of Eq. 8 is completed by adding up integers; the entropy variant sums doubles
+  if (c->kv_shard_count > 1 && (c->demand_metric != GP_METRIC_TOP_P || c->async_boundary)) return false;
   if (!(c->beta_s >= 0.0 && c->beta_s < 1.0 && c->beta_l >= 0.0 && c->beta_l < 1.0)) return false;
   if (!(c->top_p > 0.0 && c->top_p < 1.0)) return false;
   if (!(c->rope_theta >= 0.0)) return false;
@@ -149,6 +152,7 @@ Layout make_layout(const gp_config& c) {
   L.bnd_info = take(M * 32);
   L.bnd_acc = take(M * 16);
   L.unit_ready = take((size_t)M * LH * 4);
+  L.shard_sums = take((size_t)M * 2 * 4);
   L.free_peek = take((M + 1) * 4);
   L.cmp_info = take((M + 1) * 16);
   L.zbuf = take(LH * (Tb + b) * 2 * G * 8);
@@ -769,6 +773,7 @@ int gp_config_default(gp_config* cfg) {
   cfg->page_size = GP_PAGE;
   cfg->max_requests = 512;
   cfg->recent_window = GP_PAGE;
+  cfg->kv_shard_count = 1;
   cfg->k_loc = GP_PAGE / 4;          // a quarter of the page; the paper's 64 at its page size of 256
   cfg->beta_s = 0.9;
   cfg->beta_l = 0.999;
@@ -875,6 +880,8 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   d.bnd_info = reinterpret_cast<int4*>(base + L.bnd_info);
   d.bnd_acc = reinterpret_cast<int*>(base + L.bnd_acc);
   d.unit_ready = reinterpret_cast<int*>(base + L.unit_ready);
+  d.shard_sums = reinterpret_cast<int*>(base + L.shard_sums);
+  d.units_total = cfg->n_layers * cfg->n_kv_heads * cfg->kv_shard_count;
   d.free_peek = reinterpret_cast<int*>(base + L.free_peek);
   d.cmp_info = reinterpret_cast<int4*>(base + L.cmp_info);
   d.zbuf = reinterpret_cast<double*>(base + L.zbuf);
@@ -1138,7 +1145,7 @@ int gp_step_begin(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int3
 
 int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
                   const void* v, void* out, void* stream) {
-  if (!pool || !pool->step_open || n_req != pool->step_n_req) return pool && !pool->step_open ? GP_ERR_STATE : GP_ERR_INVALID;
+  if (!pool || pool->step_open != 1 || n_req != pool->step_n_req) return pool && pool->step_open != 1 ? GP_ERR_STATE : GP_ERR_INVALID;
   if (layer < 0 || layer >= pool->cfg.n_layers || !dev_req_ids || !q || !k || !v || !out) return GP_ERR_INVALID;
   if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(out, 16) || misaligned(dev_req_ids, 4))
     return GP_ERR_INVALID;
@@ -1167,7 +1174,7 @@ int gp_attn_layer(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int3
 int gp_attn_layer_qknorm(gp_pool* pool, int32_t layer, const int32_t* dev_req_ids, int32_t n_req, const void* q_raw,
                          const void* k_raw, const void* v, const float* q_weight, const float* k_weight, double eps, void* out,
                          void* stream) {
-  if (!pool || !pool->step_open || n_req != pool->step_n_req) return pool && !pool->step_open ? GP_ERR_STATE : GP_ERR_INVALID;
+  if (!pool || pool->step_open != 1 || n_req != pool->step_n_req) return pool && pool->step_open != 1 ? GP_ERR_STATE : GP_ERR_INVALID;
   if (layer < 0 || layer >= pool->cfg.n_layers || !dev_req_ids || !q_raw || !k_raw || !v || !out || !q_weight || !k_weight)
     return GP_ERR_INVALID;
   if (misaligned(q_raw, 16) || misaligned(k_raw, 16) || misaligned(v, 16) || misaligned(out, 16) || misaligned(dev_req_ids, 4) ||
@@ -1199,7 +1206,7 @@ int gp_attn_layer_qknorm(gp_pool* pool, int32_t layer, const int32_t* dev_req_id
 }
 
 int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions, void* stream) {
-  if (!pool || !pool->step_open) return pool ? GP_ERR_STATE : GP_ERR_INVALID;
+  if (!pool || pool->step_open != 1) return pool ? GP_ERR_STATE : GP_ERR_INVALID;
   if (n_req != pool->step_n_req || !dev_req_ids || !dev_actions) return GP_ERR_INVALID;
   if (pool->step_layers_done != pool->cfg.n_layers) return GP_ERR_STATE;       // layers missing: run them, or gp_step_abort
   GP_CUDA(cudaSetDevice(pool->device));
@@ -1215,10 +1222,55 @@ int gp_step_end(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_
 
 int gp_step_abort(gp_pool* pool) {
   if (!pool) return GP_ERR_INVALID;
-  if (!pool->step_open) return GP_ERR_STATE;
+  if (pool->step_open != 1) return GP_ERR_STATE;        // (a step begun with gp_decode_step_local has to be finished)
   // Nothing of an open step is committed before gp_step_end: the requests' counters are untouched, rows appended
   // by the layers that ran lie beyond the occupied slots, and the summaries went to the buffer not in use.
   pool->step_open = 0;
+  return GP_OK;
+}
+
+// ---- the step of a pool that holds a part of the model's KV heads --------------------------------------------
+int gp_decode_step_local(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, const void* q, const void* k,
+                         const void* v, void* out, int32_t* dev_actions, void* stream) {
+  if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
+  if (pool->step_open || pool->cfg.async_boundary) return GP_ERR_STATE;
+  if (n_req == 0) return GP_OK;
+  if (!dev_req_ids || !q || !k || !v || !out || !dev_actions) return GP_ERR_INVALID;
+  if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(out, 16) ||
+      misaligned(dev_req_ids, 4) || misaligned(dev_actions, 4)) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const GpDev& d = pool->dev;
+  const int LH = d.L * d.Hkv;
+  const int serial = (int)(pool->serial & 0x3fffffff);
+  launch_plan(pool, dev_req_ids, n_req, dev_actions, q, 1, 0, LH, s, true);
+  gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid, s, true, 0, LH, 0);
+  gp_launch_select_only(d, dev_req_ids, n_req, dev_actions, static_cast<float*>(out), pool->sel_grid, s, true, serial);
+  pool->launch_count += 3;
+  pool->step_open = 2;                           // between the two halves the pool takes nothing else
+  pool->step_n_req = n_req;
+  GP_CUDA(cudaGetLastError());
+  return GP_OK;
+}
+
+int gp_shard_sums(gp_pool* pool, int32_t** dev_sums, int64_t* n_ints) {
+  if (!pool || !dev_sums || !n_ints) return GP_ERR_INVALID;
+  *dev_sums = pool->dev.shard_sums;
+  *n_ints = 2LL * pool->cfg.max_requests;
+  return GP_OK;
+}
+
+int gp_decode_step_finish(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, int32_t* dev_actions, void* stream) {
+  if (!pool) return GP_ERR_INVALID;
+  if (pool->step_open != 2) return GP_ERR_STATE;
+  if (n_req != pool->step_n_req || !dev_req_ids || !dev_actions) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  gp_launch_decide_compact(pool->dev, dev_req_ids, n_req, dev_actions, pool->compact_grid, static_cast<cudaStream_t>(stream),
+                           (int)(pool->serial & 0x3fffffff));
+  pool->serial += 1;
+  pool->launch_count += 2;
+  pool->step_open = 0;
+  GP_CUDA(cudaGetLastError());
   return GP_OK;
 }
 

@@ -1,7 +1,13 @@
 """Multi-GPU plumbing.  The decode path shards by request: every GPU owns a pool and a disjoint set
 of requests, and no step of the path exchanges data between them.  What is left for
 `torch.distributed` is the rendezvous, the barrier around the timed region and the max-over-ranks
-of the device time.  Works with NCCL (one process per GPU) and with gloo (CPU tests)."""
+of the device time.  Works with NCCL (one process per GPU) and with gloo (CPU tests).
+
+The path also shards by KV head (Eq. 11: the query-state tensor is laid out by "query heads per GPU"): every rank
+of a tensor-parallel group holds a pool over the same requests with its slice of the heads; scoring, working
+sets, selection and compaction are per (layer, KV head), and the one exchange is the mean of Eq. 8: two integers
+per boundary request (sum of K^S, sum of K^L), added up over the ranks between gp_decode_step_local and
+gp_decode_step_finish."""
 from __future__ import annotations
 
 import os
@@ -81,3 +87,40 @@ def job_throughput(units_this_rank: float, ms_this_rank: float, device=None) -> 
     ms = max_over_ranks(ms_this_rank, device)
     units = sum_over_ranks(units_this_rank, device)
     return units / (ms * 1e-3), ms
+
+
+def kv_head_slice(n_q_heads: int, n_kv_heads: int, rank: int, world: int) -> Tuple[slice, slice]:
+    """The query heads and KV heads rank `rank` of `world` holds: whole GQA groups, contiguous, equally many each."""
+    if n_kv_heads % world or n_q_heads % n_kv_heads:
+        raise ValueError("the KV heads must divide evenly over the ranks, the query heads over the KV heads")
+    per = n_kv_heads // world
+    g = n_q_heads // n_kv_heads
+    return slice(rank * per * g, (rank + 1) * per * g), slice(rank * per, (rank + 1) * per)
+
+
+def complete_boundary_sums(sums, group=None) -> None:
+    """Adds the per-request sums of K^S and K^L up over the ranks, in place (`sums`: an int32 tensor, on the device
+    for NCCL, on the host for gloo).  One all-reduce; a no-op for a single process."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(sums, op=dist.ReduceOp.SUM, group=group)
+
+
+def shard_sums_tensor(pool):
+    """The pool's array of sums (gp_shard_sums) as a tensor that shares its memory: a view into the pool's blob."""
+    import torch
+    from . import binding as B
+    ptr, n = B.gp_shard_sums(pool.handle)
+    off = ptr - pool.blob.data_ptr()
+    return pool.blob[off:off + 4 * n].view(torch.int32)
+
+
+def sharded_decode_step(pool, req_ids, q, k, v, out, actions, group=None) -> None:
+    """One decode step of a pool that holds this rank's KV heads: the local half, the all-reduce of the sums, the
+    decisions and compaction.  q, k, v, out are this rank's head slices; every rank passes the same req_ids."""
+    from . import binding as B
+    n = int(req_ids.numel())
+    B.gp_decode_step_local(pool.handle, req_ids.data_ptr(), n, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                           actions.data_ptr(), pool.stream())
+    complete_boundary_sums(shard_sums_tensor(pool), group)
+    B.gp_decode_step_finish(pool.handle, req_ids.data_ptr(), n, actions.data_ptr(), pool.stream())

@@ -51,7 +51,7 @@ def test_config_defaults_and_pool_bytes_need_no_gpu():
 
 def test_struct_layout_matches_the_header():
     # 16 int32, 4 int64, 7 double, no padding surprises; and the same field order as the header's struct
-    assert ctypes.sizeof(B.gp_config) == 16 * 4 + 4 * 8 + 7 * 8
+    assert ctypes.sizeof(B.gp_config) == 18 * 4 + 4 * 8 + 7 * 8
     header = open(os.path.join(ROOT, "include", "growpage.h")).read()
     body = header[header.index("typedef struct gp_config {"):header.index("} gp_config;")]
     names = re.findall(r"^\s*(?:int32_t|int64_t|double)\s+([a-z_, ]+);", body, flags=re.M)
