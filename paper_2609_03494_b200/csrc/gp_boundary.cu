@@ -1471,6 +1471,11 @@ void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_com
   const bool shr = p.policy == GP_POLICY_SHRINK;
   auto sel = shr ? gp_bsel_kernel<true> : gp_bsel_kernel<false>;
   cudaFuncSetAttribute(sel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm);
+  {                                                  // the kernel with the whole boundary chain: same shared memory
+    auto opt_in = [&](auto kern) { cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sel_sm); };
+    if (p.d == 128) { if (shr) opt_in(gp_chain_kernel<128, true>); else opt_in(gp_chain_kernel<128, false>); }
+    else { if (shr) opt_in(gp_chain_kernel<64, true>); else opt_in(gp_chain_kernel<64, false>); }
+  }
   int occ = 0;
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, sel, SEL_T, sel_sm);
   *grid_sel = num_sms * (occ > 0 ? occ : 1);
@@ -1486,7 +1491,6 @@ void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* ou
   const size_t sm = gp_bsel_smem(p);
   const bool shr = p.policy == GP_POLICY_SHRINK;
   auto launch = [&](auto kern) {
-    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     gp_launch(kern, grid, SEL_T, sm, s, pdl, p, pa, n_req_merge, out_merge, serial, has_chain, req_ids, actions);
   };
   if (p.d == 128) { if (shr) launch(gp_chain_kernel<128, true>); else launch(gp_chain_kernel<128, false>); }
