@@ -471,6 +471,8 @@ def run_ours(args):
                        "l2": "per-step working set (all resident K/V) is larger than L2; no flush needed",
                        "input_generation_s": round(t_gen, 1)},
             "modes": modes,
+            "north_star": {"whole_step_frac_of_8tbs": step_roofline["frac_of_8tbs"], "target": 0.70,
+                           "met": bool(step_roofline["frac_of_8tbs"] >= 0.70)},
             "roofline": roofline, "step_roofline": step_roofline,
             "cpu_baseline": cpu,
             "e2e": {"value": round(e2e_value, 1), "unit": "tokens/s", "h2d_bytes_per_step": h2d,

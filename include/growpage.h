@@ -113,13 +113,16 @@ typedef struct gp_config {
                                 ablation's other metric, the view's attention entropy H over ln |C| in the
                                 place of K / |C| (Delta_t is then a floating-point mean)               */
   int32_t overlap_slots;     /* synchronous mode, how the boundary work of a step (selection jobs, decisions,
-                                compaction) is launched.  0 (default): one kernel behind the attention kernel,
-                                whose thread blocks take their places as that kernel's leave and whose jobs
-                                start as soon as the boundary requests' summary logits are reported complete
-                                (three launches per step).  N > 0: the same kernel, beside the attention
-                                kernel on N thread-block slots that kernel's grid gives up.  -1: a selection
-                                and a compaction kernel, one after the other (four launches per step; what
-                                gp_step_end runs).  Same results in every case                        */
+                                compaction) is launched.  -2: one kernel behind the attention kernel, whose
+                                thread blocks take their places as that kernel's leave and whose jobs start as
+                                soon as the boundary requests' summary logits are reported complete (three
+                                launches per step).  -1: a selection and a compaction kernel, one after the
+                                other (four launches per step; what gp_step_end runs).  0 (default): -2 when
+                                max_requests * n_layers * n_kv_heads <= 1024 (a step's boundary work is then a
+                                few hundred jobs at most and the saved kernel boundary counts), else -1 (the
+                                compaction of thousands of units wants its own, larger grid).  N > 0: as -2,
+                                beside the attention kernel on N thread-block slots that kernel's grid gives
+                                up.  Same results in every case                                        */
   int32_t async_slots;       /* asynchronous boundary work: thread blocks of the attention kernel's grid
                                 given up so that the boundary kernel finds room on the SMs beside it;
                                 0 = a default (64)                                                    */

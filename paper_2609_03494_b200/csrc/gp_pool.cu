@@ -102,7 +102,7 @@ bool valid_config(const gp_config* c) {
   if (c->max_batch_tokens < 0 || c->max_boundary_tokens < 0) return false;
   if (c->demand_metric < GP_METRIC_TOP_P || c->demand_metric > GP_METRIC_ENTROPY) return false;
   if (c->async_boundary < 0 || c->async_boundary > 1 || c->async_slots < 0 || c->async_slots > 4096) return false;
-  if (c->overlap_slots < -1 || c->overlap_slots > 4096) return false;
+  if (c->overlap_slots < -2 || c->overlap_slots > 4096) return false;
   if (c->kv_shard_count < 1 || c->kv_shard_count > 64 || c->reserved != 0) return false;
   // spread over several pools, the mean of Eq. 8 is completed by adding up integers; the entropy variant sums doubles
   if (c->kv_shard_count > 1 && (c->demand_metric != GP_METRIC_TOP_P || c->async_boundary)) return false;
@@ -918,7 +918,12 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
   }
   pool->attn_grid_ov = pool->attn_grid;
   pool->chain_grid_ov = 0;
-  if (!cfg->async_boundary && cfg->overlap_slots == 0) {
+  // One kernel behind the attention kernel pays while a step's boundary work is a few hundred jobs: it saves a kernel
+  // boundary and starts its jobs while the attention kernel drains (64 requests x 8 units: 68 us per step against
+  // 75).  With thousands of units the compaction moves hundreds of megabytes and wants the four-kernel path's larger
+  // compaction grid (36 layers x 256 residents: 4.8 ms against 5.2; 256 requests x 8 units: 0.49 against 0.52).
+  const bool fused_auto = (long long)cfg->max_requests * cfg->n_layers * cfg->n_kv_heads <= 1024;
+  if (!cfg->async_boundary && (cfg->overlap_slots == -2 || (cfg->overlap_slots == 0 && fused_auto))) {
     pool->chain_grid_ov = pool->sel_grid;          // the whole grid, behind the attention kernel's
   } else if (!cfg->async_boundary && cfg->overlap_slots > 0) {
     int slots = cfg->overlap_slots;

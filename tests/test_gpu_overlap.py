@@ -1,10 +1,10 @@
 """The ways a synchronous step can launch its boundary work (gp_config.overlap_slots).
 
-By default (0) the selection jobs, the decisions, the compaction and the merge of split outputs are one kernel
-behind the attention kernel, whose jobs start when that kernel has reported their unit's summary logits complete;
-every other test of the synchronous mode runs that way.  Here: the same kernel beside the attention kernel on
-thread-block slots that kernel's grid gives up (N > 0), and the selection and compaction kernels one after the other
-(-1, four launches).  Nothing about the results may change: the same lockstep comparison against the oracle
+With -2 the selection jobs, the decisions, the compaction and the merge of split outputs are one kernel behind the
+attention kernel, whose jobs start when that kernel has reported their unit's summary logits complete; with -1 a
+selection and a compaction kernel run one after the other (four launches); the default (0) picks between the two
+by the pool's size, so the other tests of the synchronous mode run one or the other.  Here both are forced, and
+the one kernel also runs beside the attention kernel on thread-block slots that kernel's grid gives up (N > 0).  Nothing about the results may change: the same lockstep comparison against the oracle
 (actions, working-set sizes, Delta, retained sets, page tables, free list, summaries, attention outputs), over the
 five configurations, the paper's page geometry, the Shrink policy, the entropy metric and RoPE, with slot counts
 from one thread block to half the grid."""
@@ -19,7 +19,7 @@ from tests import lockstep as LS
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("slots", [64, -1])
+@pytest.mark.parametrize("slots", [64, -1, -2])
 @pytest.mark.parametrize("config", [1, 2, 3, 4, 5])
 def test_lockstep_configurations_with_overlapped_boundary_work(config, slots):
     st = LS.run_lockstep(W.parity_instance(config), overlap_slots=slots)
