@@ -571,7 +571,7 @@ gp_attn_kernel(const __grid_constant__ GpDev p, int n_req, const __nv_bfloat16* 
 
       // ---- a request at its boundary: this warp's share of the unit's summary logits (and the appended row, and the
       // request's counters) is written; the boundary work that may run beside this kernel counts the reports
-      if (flags & 1) {
+      if ((flags & 1) && p.report_units) {
         __threadfence();
         __syncwarp();
         if (lane == 0 && !(p.withhold & GP_WITHHOLD_READY)) atomicAdd(p.unit_ready + (size_t)sd[15] * LH + lh, 1);

@@ -942,6 +942,29 @@ __device__ __forceinline__ void sel_job(const GpDev& p, const SelSmem& S, const 
   }
 }
 
+// Rarely taken tails of the selection kernel's last thread block, kept out of line so that they do not weigh on the
+// register allocation of the jobs.
+// Layer-by-layer step: the requests' counters move on at the end of the step (a whole-step launch does it where
+// the attention kernel appends the token): one token further, the summary buffers swapped.  The first work item of
+// a request names it once.
+__device__ __noinline__ void advance_counters(const GpDev& p, int n_rc) {
+  for (int idx = threadIdx.x; idx < n_rc; idx += blockDim.x) {
+    const int* d = p.rcx + (size_t)idx * GP_DESC_INTS;
+    if (d[4] == 0) {
+      const int r = d[1];
+      p.n[r] += 1; p.pos[r] += 1; p.started[r] = 1; p.sum_par[r] ^= 1;
+    }
+  }
+  __syncthreads();
+}
+// A pool that holds a part of the model's KV heads: its sums of K^S and K^L per boundary request, zero past them
+__device__ __noinline__ void publish_shard_sums(const GpDev& p, int n_bnd) {
+  for (int e = threadIdx.x; e < p.M; e += blockDim.x) {
+    p.shard_sums[2 * e] = e < n_bnd ? __ldcg(p.bnd_acc + 4 * e) : 0;
+    p.shard_sums[2 * e + 1] = e < n_bnd ? __ldcg(p.bnd_acc + 4 * e + 1) : 0;
+  }
+}
+
 template <bool SHR>      // SHR: the pool runs the Shrink policy (a fourth job per unit)
 __global__ void __launch_bounds__(SEL_T, 2)
 gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int* __restrict__ actions,
@@ -1040,27 +1063,9 @@ gp_bsel_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids,
   __syncthreads();
   if (s_i[2]) {
     __threadfence();
-    if (!out) {
-      // Layer-by-layer step: the requests' counters move on here, at the end of the step (a whole-step launch
-      // does it where the attention kernel appends the token): one token further, the summary buffers swapped.
-      // The first work item of a request names it once.
-      for (int idx = tid; idx < n_rc; idx += SEL_T) {
-        const int4 d0 = *reinterpret_cast<const int4*>(p.rcx + (size_t)idx * GP_DESC_INTS);
-        if (p.rcx[(size_t)idx * GP_DESC_INTS + 4] == 0) {
-          const int r = d0.y;
-          p.n[r] += 1; p.pos[r] += 1; p.started[r] = 1; p.sum_par[r] ^= 1;
-        }
-      }
-      __syncthreads();
-    }
-    if (decide) {
-      decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(S.sbuf), serial);
-    } else {
-      for (int e = tid; e < p.M; e += SEL_T) {
-        p.shard_sums[2 * e] = e < n_bnd ? __ldcg(p.bnd_acc + 4 * e) : 0;
-        p.shard_sums[2 * e + 1] = e < n_bnd ? __ldcg(p.bnd_acc + 4 * e + 1) : 0;
-      }
-    }
+    if (!out) advance_counters(p, n_rc);
+    if (decide) decide_and_allocate(p, req_ids, n_req, n_bnd, actions, reinterpret_cast<int*>(S.sbuf), serial);
+    else publish_shard_sums(p, n_bnd);
   }
 
   if (!idle_merge) merge_partials(p, n_req, out, n_mc, n_rc, (int)gridDim.x - 1 - (int)blockIdx.x, (int)gridDim.x, 0, LH);

@@ -113,6 +113,8 @@ struct GpDev {
   int4* bnd_info;                        // [M][2] requests at a boundary: {slot in the batch, request, P, position of the step's token}, {score offset lo, hi, 0, 0}
   int* shard_sums;                       // [M][2] per boundary request: sum of K^S, sum of K^L over this pool's units (to be
                                          // summed over the pools that hold the other KV heads), then over all units
+  int report_units;                      // the attention kernel reports boundary units complete (the boundary kernel that
+                                         // runs behind it starts its jobs on those reports)
   int units_total;                       // (layer, KV head) units of the model: L H_kv times the number of KV-head shards
   int* unit_ready;                       // [M][L H_kv] per boundary unit: consumer warps of the attention kernel done with it
   int* bnd_acc;                          // [M][4] per boundary request: sum of K^S, sum of K^L, shared pages of C, 0

@@ -931,6 +931,7 @@ int gp_pool_create(const gp_config* cfg, void* dev_blob, size_t bytes, int devic
     pool->attn_grid_ov = pool->attn_grid - slots;
     pool->chain_grid_ov = slots;
   }
+  pool->dev.report_units = pool->dev_alt.report_units = pool->chain_grid_ov > 0;
   pool->dbg = base + L.dbg;
   pool->qn = reinterpret_cast<__nv_bfloat16*>(base + L.qn);
   pool->kn = reinterpret_cast<__nv_bfloat16*>(base + L.kn);
