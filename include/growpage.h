@@ -405,7 +405,8 @@ int64_t gp_launch_count(gp_pool* pool);
  * any fault: `what` names hand-overs that are then simply not made (1 the attention kernel's first thread block
  * never completes its second work item for its consumer warps; 2 the first chunk of every compaction unit never
  * says that its sources are read; 4 the deciding thread block of the boundary kernel never tells the others; 8 the
- * attention kernel never reports a boundary unit's summary logits complete; 0 none),
+ * attention kernel never reports a boundary unit's summary logits complete; 0 none; and, not a withheld hand-over
+ * but a switch for tests: 16 the compaction claims a whole unit per ticket however few units there are),
  * `spin_limit` the iterations after which waits give up (0 = the default, 2^21).  Applies to the steps issued
  * after it.  The error bits stay set; results of such a pool are not meaningful afterwards. */
 int gp_test_withhold(gp_pool* pool, int32_t what, int32_t spin_limit);

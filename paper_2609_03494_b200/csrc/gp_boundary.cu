@@ -1106,8 +1106,14 @@ __device__ __forceinline__ CmpSmem cmp_smem_at(uint8_t* base) {       // base: 1
   return C;
 }
 
-// The compaction of a step, run by every CTA of the calling grid (CT threads): chunks are claimed from the ticket
-// counter until none is left; the last CTA to finish swaps in the copy-on-write targets.
+// The compaction of a step, run by every CTA of the calling grid (CT threads): work is claimed from the ticket
+// counter until none is left; the last CTA to finish swaps in the copy-on-write targets.  What a ticket stands for
+// depends on how much there is.  A few units (one layer, a handful of requests at their boundary): one 64-slot chunk
+// of a unit per ticket, so that all thread blocks have work; a chunk says when its sources are read, and waits for
+// that word from the chunks before it whose sources its destinations reach.  Units for every thread block twice
+// over: one unit per ticket, its chunks in ascending order by the same thread block (a chunk's destinations lie
+// below the next chunk's sources, and program order puts every chunk's reads before the next chunk's writes), which
+// saves the ticket, the eviction list and the waits per chunk and skips the chunks below the first evicted slot.
 template <int D, bool SHR>
 __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, int serial) {
   constexpr int CH = D / 8;
@@ -1135,6 +1141,8 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
   const int stamp = p.async ? serial + 1 : p.hdr[HDR_STEP];
   for (int i = tid + CT; i <= n_cmp; i += CT) s_info[i] = p.cmp_info[i];
 
+  const bool by_unit = (p.withhold & GP_TEST_COMPACT_BY_UNIT) || (long long)n_cmp * LH >= 2LL * (long long)gridDim.x;
+  const int n_work = by_unit ? n_cmp * LH : n_items;
   for (bool first = true;; first = false) {
     __syncthreads();
     if (!first) {
@@ -1142,34 +1150,57 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
       __syncthreads();
     }
     const int item = s_i[0];
-    if (item >= n_items) break;
-    // item -> (compressing request, layer/head, chunk); chunks of a unit are consecutive and ascending
-    int lo = 0, hi = n_cmp;
-    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (LH * s_info[mid].w <= item) lo = mid; else hi = mid; }
+    if (item >= n_work) break;
+    // ticket -> (compressing request, layer/head) and the chunks it covers; chunks of a unit are consecutive and
+    // ascending in the item numbering the flags go by
+    int lo, lh, j_begin, j_end;
+    if (by_unit) {
+      lo = item / LH; lh = item % LH;
+      j_begin = 0; j_end = s_info[lo + 1].w - s_info[lo].w;
+    } else {
+      lo = 0;
+      int hi = n_cmp;
+      while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (LH * s_info[mid].w <= item) lo = mid; else hi = mid; }
+      const int nchunk = s_info[lo + 1].w - s_info[lo].w;
+      const int rem = item - LH * s_info[lo].w;
+      lh = rem / nchunk; j_begin = rem % nchunk; j_end = j_begin + 1;
+    }
     const int4 inf = s_info[lo];
-    const int nchunk = s_info[lo + 1].w - inf.w;
-    const int rem = item - LH * inf.w;
-    const int lh = rem / nchunk, j = rem % nchunk;
     const int l = lh / p.Hkv, h = lh % p.Hkv;
     const int r = inf.x;
     const int Pr = inf.y;
     const int* table = p.page_table + (size_t)r * p.cap;
     const int* shadow = p.shadow + (size_t)r * p.cap;
     const int n_src = Pr * GP_PAGE;
-    const int c0 = j * MOVE_TOK;
     // second round trip: the eviction list and, for every source slot of the chunk, its page and its
     // copy-on-write target
     const bool shrink = SHR && (inf.z & CMP_SHRINK) != 0;
     const int e_bnd = inf.z & (CMP_SHRINK - 1);
     const int ne = shrink ? 2 * p.blk : p.blk;             // slots freed: one page of the method, two at a Shrink
+    for (int t = tid; t < ne; t += CT)
+      ev[t] = shrink ? p.evict2[((size_t)e_bnd * LH + lh) * 2 * p.blk + t] : p.evict[((size_t)e_bnd * LH + lh) * p.blk + t];
+    if (by_unit && n_cow == 0) {
+      // nothing is shared in this step: slots below the first evicted one stay where they are
+      __syncthreads();
+      if (tid < 32) {
+        int mn = 0x7fffffff;
+        for (int t = tid; t < ne; t += 32) mn = min(mn, ev[t]);
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o2));
+        if (tid == 0) s_i[5] = mn / MOVE_TOK;
+      }
+      __syncthreads();
+      j_begin = s_i[5];
+    }
+   for (int j = j_begin; j < j_end; ++j) {
+    if (j != j_begin) __syncthreads();                   // the chunk before has left the shared arrays
+    const int c0 = j * MOVE_TOK;
     int t0 = 0, s0 = -1;
     const int my_i = c0 + tid;                             // the slot this thread plans (first MOVE_TOK threads)
     if (tid < MOVE_TOK && my_i < n_src) {
       const int pg = my_i / GP_PAGE;
       t0 = table[pg]; s0 = shadow[pg];
     }
-    for (int t = tid; t < ne; t += CT)
-      ev[t] = shrink ? p.evict2[((size_t)e_bnd * LH + lh) * 2 * p.blk + t] : p.evict[((size_t)e_bnd * LH + lh) * p.blk + t];
     __syncthreads();
     int tokv = 0, tok_dst = -1, tok_page = 0;
     if (tid < MOVE_TOK) {
@@ -1224,7 +1255,7 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
     for (int k2 = 0; k2 < PIECES; ++k2) touched ^= val[k2].x ^ val[k2].y ^ val[k2].z ^ val[k2].w;
     if (touched == 0x9e3779b9u && c0 < 0) s_i[4] = 1;      // never true; keeps the dependency alive
     __syncthreads();
-    if (tid == 0) {
+    if (tid == 0 && !by_unit) {
       // No fence on either side: the flag only says that loads have returned (they have: their values were
       // consumed above), and the stores below are issued after the flag has been seen.
       if (!((p.withhold & GP_WITHHOLD_CHUNK) && j == 0))               // (test support: see GP_WITHHOLD_CHUNK)
@@ -1255,6 +1286,7 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
       atomicAdd(&s_i[3], 1);
       p.tok[gp_tok_off(p, l, tok_page, h) + (tok_dst % GP_PAGE)] = tokv;
     }
+   }
   }
   __syncthreads();
   if (tid == 0 && s_i[3] > 0)
@@ -1314,7 +1346,7 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
 
 
 template <int D, bool SHR>
-__global__ void __launch_bounds__(CT)
+__global__ void __launch_bounds__(CT, 4)
 gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_ids, int n_req, int serial) {
   __shared__ __align__(16) uint8_t cmp_raw[CMP_SMEM_BYTES];
   gp_pdl_wait();

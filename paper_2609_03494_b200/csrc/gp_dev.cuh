@@ -51,6 +51,7 @@ enum {
   GP_WITHHOLD_CHUNK = 2,    // compaction: the first chunk of a unit never says that its sources are read
   GP_WITHHOLD_DECIDED = 4,  // boundary kernel: the deciding CTA never tells the others
   GP_WITHHOLD_READY = 8,    // attention kernel: the consumer warps never report a boundary unit's logits complete
+  GP_TEST_COMPACT_BY_UNIT = 16,   // (not a withheld hand-over) the compaction claims whole units whatever their number
 };
 
 // error bits

@@ -1601,7 +1601,7 @@ int gp_debug_pool(gp_pool* pool, int64_t* n_free, int32_t* refcounts, int64_t co
 }
 
 int gp_test_withhold(gp_pool* pool, int32_t what, int32_t spin_limit) {
-  if (!pool || what < 0 || what > 15 || spin_limit < 0) return GP_ERR_INVALID;
+  if (!pool || what < 0 || what > 31 || spin_limit < 0) return GP_ERR_INVALID;
   GpDev* views[2] = {&pool->dev, &pool->dev_alt};
   for (GpDev* v : views) {
     v->withhold = what;

@@ -61,7 +61,10 @@ def make_pools(wl: W.Workload, device: int = 0, **over):
                          max_batch_tokens=over.get("max_batch_tokens", 0), async_slots=over.get("async_slots", 0),
                          overlap_slots=over.get("overlap_slots", 0),
                          max_boundary_tokens=over.get("max_boundary_tokens", 0))
-    return B.Pool(gcfg, device), O.OraclePool(ocfg)
+    pool = B.Pool(gcfg, device)
+    if over.get("compact_by_unit"):
+        B.gp_test_withhold(pool.handle, 16, 0)          # the compaction claims whole units whatever their number
+    return pool, O.OraclePool(ocfg)
 
 
 def _to_dev(torch, arr: np.ndarray, device: int):

@@ -46,3 +46,21 @@ def test_pages_of_256_tokens_with_overlapped_boundary_work():
     wl = W.Workload("b256", 77, s, reqs, n_resident=3, initial_pages=0, max_pages_per_req=4, n_pages=14, k_loc=64)
     st = LS.run_lockstep(wl, tau=-0.05, summary_every=64, check_pool_every=32, overlap_slots=32)
     assert st.actions.get(B.GP_ACT_GROW, 0) >= 3 and st.decisions["sel"] > 0
+
+
+@pytest.mark.parametrize("slots", [-1, -2])
+@pytest.mark.parametrize("config,over", [(1, dict(tau=-0.05)), (3, dict()), (5, dict()),
+                                         (5, dict(policy=B.GP_POLICY_SHRINK, min_capacity=64, tau=-0.03, shrink_below=-0.036))])
+def test_compaction_that_claims_whole_units(config, over, slots):
+    # with units for every thread block twice over the compaction claims a unit per ticket and moves its chunks in
+    # order, without the per-chunk flags; forced here on small pools, with copy-on-write pages and Shrinks among them
+    st = LS.run_lockstep(W.parity_instance(config), overlap_slots=slots, compact_by_unit=True, **over)
+    assert st.decisions["sel"] > 0 and st.counters[8] > 0
+
+
+def test_compaction_by_unit_with_pages_of_256_tokens():
+    s = W.Shape(1, 8, 2, 64, page_size=256)
+    reqs = [W.RequestSpec(i, p, 900, 0.05, share_group=-1) for i, p in enumerate((300, 40, 511))]
+    wl = W.Workload("b256", 77, s, reqs, n_resident=3, initial_pages=0, max_pages_per_req=4, n_pages=14, k_loc=64)
+    st = LS.run_lockstep(wl, tau=-0.05, summary_every=64, check_pool_every=32, compact_by_unit=True)
+    assert st.actions.get(B.GP_ACT_COMPRESS, 0) + st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) >= 3
