@@ -1,22 +1,31 @@
-// Capacity-boundary kernels (Sec. 3.2 - 3.3, App. D.1, App. D.2), launched every step after attention.
-// The attention kernel has already left, for every (request at a boundary, layer, KV head) unit and both
-// calibrated summaries, exp(logit - the page's maximum logit) of every candidate key, and per 16-token page
-// the maximum and the sum of those exponentials.
+// Capacity-boundary work (Sec. 3.2 - 3.3, App. D.1, App. D.2), every step, behind the attention kernel.
+// That kernel leaves, for every (request at a boundary, layer, KV head) unit and both calibrated summaries,
+// exp(logit - the page's maximum logit) of every candidate key, and per 16-token page the maximum and the sum of
+// those exponentials.  The work on them, in the order of its dependences:
 //
-//   gp_bsel_kernel    per unit, three independent jobs, one CTA each: per-head softmax over the candidate
+//   selection jobs    per unit, three independent jobs, one CTA each: per-head softmax over the candidate
 //                     set and group mean -> a^S or a^L and its working-set size K^S or K^L (Eq. 7); and,
 //                     speculatively, the b slots a compression would evict (Eq. 9, Eq. 10).  Under the
-//                     Shrink policy a fourth job lists the 2b slots a Shrink would evict (Eq. 13).  CTAs
-//                     without a job merge the partial attention outputs of requests that were split over
-//                     several work items.  The last CTA to finish aggregates Eq. 8, decides per request
-//                     (grow, compress, shrink) and runs the device allocator: grants first, then
-//                     copy-on-write targets, each in ascending request id.
-//   gp_compact_kernel per (compressing unit, chunk of 64 source slots): stable in-place compaction into
-//                     (P-1) b slots ((P-2) b at a Shrink), writing to copy-on-write targets where the
-//                     source page is shared.  Chunks are claimed in order from a ticket counter; a chunk
-//                     publishes "my sources are read" before the next chunk may overwrite their tail.  The
-//                     last CTA swaps in the target pages, drops the references to the replaced ones and
-//                     returns the last page of every request that shrank.
+//                     Shrink policy a fourth job lists the 2b slots a Shrink would evict (Eq. 13).
+//   decisions         by the CTA that finishes its jobs last: Eq. 8 per request, the action (grow, compress,
+//                     shrink), the device allocator: grants first, then copy-on-write targets, each in ascending
+//                     request id.
+//   compaction        per compressing unit: stable in-place compaction into (P-1) b slots ((P-2) b at a Shrink),
+//                     writing to copy-on-write targets where the source page is shared.  Work is claimed from a
+//                     ticket counter, a chunk of 64 source slots at a time (a chunk publishes "my sources are
+//                     read" before the next chunk may overwrite their tail) or, with many units, a unit at a
+//                     time.  The last CTA swaps in the target pages, drops the references to the replaced ones
+//                     and returns the last page of every request that shrank.
+//   merge             of the partial attention outputs of requests that were split over several work items.
+//
+// It comes in two shapes that run the same device functions:
+//   gp_chain_kernel                       all of it in one kernel (the deciding CTA tells the others through a flag):
+//                                         behind the attention kernel of its own step, with every job waiting for the
+//                                         attention kernel's report that its unit is complete (synchronous mode), or
+//                                         beside the attention kernel of the next step (asynchronous mode);
+//   gp_bsel_kernel, gp_compact_kernel     selection + decisions + merge, then compaction, as kernels of their own
+//   (and gp_decide_kernel)                (large pools, the layer-by-layer step; with the KV heads spread over several
+//                                         pools the decisions wait for the sums of all pools in a kernel of their own).
 //
 // Everything that decides an integer outcome is fp64.  Top-p counting and the eviction cut work on the
 // IEEE bit patterns of the (non-negative) scores: one pass into a two-level histogram (4096 fine bins under

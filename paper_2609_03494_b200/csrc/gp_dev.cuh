@@ -191,7 +191,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   }
   return false;
 }
-// 1-D bulk copy global -> shared of this CTA, completion counted on an mbarrier.  No multicast.
+// 1-D bulk copy global -> shared of this CTA (this CTA only), completion counted on an mbarrier.
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
