@@ -64,3 +64,10 @@ def test_compaction_by_unit_with_pages_of_256_tokens():
     wl = W.Workload("b256", 77, s, reqs, n_resident=3, initial_pages=0, max_pages_per_req=4, n_pages=14, k_loc=64)
     st = LS.run_lockstep(wl, tau=-0.05, summary_every=64, check_pool_every=32, compact_by_unit=True)
     assert st.actions.get(B.GP_ACT_COMPRESS, 0) + st.actions.get(B.GP_ACT_COMPRESS_FALLBACK, 0) >= 3
+
+
+def test_compaction_by_unit_in_the_asynchronous_mode():
+    st = LS.run_lockstep(W.parity_instance(1), async_boundary=True, compact_by_unit=True, tau=-0.05)
+    assert st.decisions["sel"] > 0 and st.counters[8] > 0
+    st = LS.run_lockstep(W.parity_instance(5), async_boundary=True, compact_by_unit=True)
+    assert st.decisions["sel"] > 0 and st.counters[4] > 0          # copy-on-write pages among them
