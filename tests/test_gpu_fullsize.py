@@ -2,7 +2,7 @@
 
 All 64 requests of the one-layer Qwen3-8B-shaped configuration run through the C-ABI on the GPU, back to back
 on one stream as in the benchmark (same pool parameters, host staging on).  The float64 oracle cannot follow
-64 requests at that size in seconds, so it follows a sample of them (four through the first 448 steps, two of
+64 requests at that size in seconds, so it follows a sample of them (sixteen through the first 512 steps, four of
 them on through step 2064, which covers the steps the benchmark times by default), each simulated alone: in this
 configuration the per-request page cap never binds and the pool holds every request at its cap, so a request's
 trajectory does not depend on the others.  Compared per step for the sampled requests: action and attention
@@ -24,9 +24,9 @@ from tests.lockstep import ATTN_MAX_ABS, ATTN_MEAN_ABS, NEAR_TIE, NEAR_TIE_FRACT
 
 pytestmark = pytest.mark.gpu
 
-SAMPLE = (5, 23, 41, 62)          # request indices the oracle follows through the first SHORT steps
-SHORT = 448                        # 28 capacity boundaries per request
-LONG_SAMPLE = (5, 41)              # ... and these two through all STEPS
+SAMPLE = tuple(range(1, 64, 4))    # request indices the oracle follows through the first SHORT steps (16 of the 64)
+SHORT = 512                        # 32 capacity boundaries per request
+LONG_SAMPLE = (5, 21, 41, 61)      # ... and these four through all STEPS
 STEPS = 2064                       # past the window the benchmark times by default (job steps 2038 to 2058)
 
 
