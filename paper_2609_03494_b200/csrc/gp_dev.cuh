@@ -33,7 +33,7 @@ enum {
   HDR_N_RC = 0,      // (request, chunk) work items of this step
   HDR_N_BND,         // requests at a capacity boundary
   HDR_N_CMP,         // requests that compress
-  HDR_DECIDED,       // asynchronous mode: stamped by the CTA that took the step's decisions
+  HDR_DECIDED,       // boundary work in one kernel: stamped by the CTA that took the step's decisions
   HDR_DONE_CMP,      // CTAs of the compaction kernel that have finished
   HDR_STEP,          // step serial number
   HDR_N_ACTIVE,      // requests actually stepped
