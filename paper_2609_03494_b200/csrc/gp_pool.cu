@@ -1347,15 +1347,14 @@ static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, 
       }
       cudaStream_t fs = pool->fetch_stream;
       GP_CUDA(cudaStreamWaitEvent(fs, pool->ev_used[set], 0));
-      const long long pieces = (long long)(qb + 2 * kb) / 16;         // a row is 128 or 256 bytes: whole pieces
-      int grid = (int)((pieces + 255) / 256);
-      if (grid > pool->num_sms * 8) grid = pool->num_sms * 8;
-      if (grid * 256 < n_req) grid = (n_req + 255) / 256;
-      gp_fetch_inputs_kernel<<<grid, 256, 0, fs>>>(st_ids, static_cast<const int*>(mi), n_req,
-                                                  static_cast<uint4*>(st_q), static_cast<const uint4*>(mq), (long long)qb / 16,
-                                                  static_cast<uint4*>(st_k), static_cast<const uint4*>(mk), (long long)kb / 16,
-                                                  static_cast<uint4*>(st_v), static_cast<const uint4*>(mv), (long long)kb / 16);
-      pool->launch_count++;
+      // Copies by the copy engine here, not the fetch kernel: they run beside the step before, whose attention
+      // kernel fills every SM's registers; a kernel that reads over the bus for 15 us held some of them and kept
+      // that step's attention thread blocks from starting (11 us per step).  The copies' set-up time, which is
+      // what the fetch kernel saves the call that waits, is hidden here.
+      GP_CUDA(cudaMemcpyAsync(st_ids, host_req_ids, (size_t)n_req * 4, cudaMemcpyHostToDevice, fs));
+      GP_CUDA(cudaMemcpyAsync(st_q, q, qb, cudaMemcpyHostToDevice, fs));
+      GP_CUDA(cudaMemcpyAsync(st_k, k, kb, cudaMemcpyHostToDevice, fs));
+      GP_CUDA(cudaMemcpyAsync(st_v, v, kb, cudaMemcpyHostToDevice, fs));
       GP_CUDA(cudaEventRecord(pool->ev_fetch[set], fs));
       GP_CUDA(cudaStreamWaitEvent(s, pool->ev_fetch[set], 0));
     } else {
