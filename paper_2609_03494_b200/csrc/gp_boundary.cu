@@ -1478,11 +1478,21 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
       __threadfence();
     }
     __syncthreads();
+    if (same_step) {
+      // The attention kernel of this step has ended by now (the decisions needed its last reports): the split
+      // requests' outputs are merged first, and then the next kernel on the stream may be scheduled.  With early
+      // planning that is the next step's plan, which so runs beside the compaction below: the decisions it reads
+      // are taken, the attention kernel has moved the requests on, and the compaction reads nothing the plan writes
+      // (the merge does: the lists of split requests, hence its place before).
+      gp_pdl_wait();
+      if (out_merge) merge_partials(pa, n_req_merge, out_merge, pa.hdr[HDR_N_MC], pa.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, 0, LH);
+      gp_pdl_launch_dependents();
+    }
     // ---- compaction: its arrays take the place of the selection's -----------------------------------------------
     compact_body<D, SHR>(p, cmp_smem_at(smem), serial);
   }
+  if (same_step) return;
   gp_pdl_wait();              // the attention kernel beside which this grid ran has ended
-  if (same_step) gp_pdl_launch_dependents();
   if (out_merge) merge_partials(pa, n_req_merge, out_merge, pa.hdr[HDR_N_MC], pa.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, 0, LH);
 }
 
