@@ -1378,7 +1378,11 @@ gp_compact_kernel(const __grid_constant__ GpDev p, const int* __restrict__ req_i
 template <int D, bool SHR>
 __global__ void __launch_bounds__(SEL_T, 2)
 gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev pa, int n_req_merge, float* __restrict__ out_merge,
-                int serial, int has_chain, const int* __restrict__ req_ids, int* __restrict__ actions) {
+                int serial, int has_chain, const int* __restrict__ req_ids, int* __restrict__ actions,
+                int* __restrict__ actions_copy) {
+  // actions_copy: where the step's actions are wanted as well once they are final (the host entry points: the
+  // caller's array in page-locked host memory; writing them there from the plan kernel made that kernel wait
+  // for the bus)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((256u - (smem_u32(smem_raw) & 255u)) & 255u);
   const int tid = threadIdx.x;
@@ -1485,6 +1489,8 @@ gp_chain_kernel(const __grid_constant__ GpDev p, const __grid_constant__ GpDev p
       // are taken, the attention kernel has moved the requests on, and the compaction reads nothing the plan writes
       // (the merge does: the lists of split requests, hence its place before).
       gp_pdl_wait();
+      if (actions_copy && blockIdx.x == gridDim.x - 1)
+        for (int i = tid; i < n_req_merge; i += SEL_T) actions_copy[i] = __ldcg(actions + i);
       if (out_merge) merge_partials(pa, n_req_merge, out_merge, pa.hdr[HDR_N_MC], pa.hdr[HDR_N_RC], (int)blockIdx.x, (int)gridDim.x, 0, LH);
       gp_pdl_launch_dependents();
     }
@@ -1543,11 +1549,11 @@ void gp_boundary_setup(const GpDev& p, int num_sms, int* grid_sel, int* grid_com
 // asynchronous mode: the boundary chain of the step whose view is `p` (none when !has_chain), and afterwards the
 // merge of the split requests' partial outputs of the step whose view is `pa` (none when out_merge is null)
 void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* out_merge, int serial, int has_chain, int grid,
-                     cudaStream_t s, bool pdl, const int* req_ids, int* actions) {
+                     cudaStream_t s, bool pdl, const int* req_ids, int* actions, int* actions_copy) {
   const size_t sm = gp_bsel_smem(p);
   const bool shr = p.policy == GP_POLICY_SHRINK;
   auto launch = [&](auto kern) {
-    gp_launch(kern, grid, SEL_T, sm, s, pdl, p, pa, n_req_merge, out_merge, serial, has_chain, req_ids, actions);
+    gp_launch(kern, grid, SEL_T, sm, s, pdl, p, pa, n_req_merge, out_merge, serial, has_chain, req_ids, actions, actions_copy);
   };
   if (p.d == 128) { if (shr) launch(gp_chain_kernel<128, true>); else launch(gp_chain_kernel<128, false>); }
   else { if (shr) launch(gp_chain_kernel<64, true>); else launch(gp_chain_kernel<64, false>); }

@@ -276,7 +276,7 @@ inline cudaError_t gp_launch(void (*kern)(KArgs...), int grid, int block, size_t
 
 void gp_attention_setup(const GpDev& p);
 void gp_launch_chain(const GpDev& p, const GpDev& pa, int n_req_merge, float* out_merge, int serial, int has_chain, int grid,
-                     cudaStream_t s, bool pdl, const int* req_ids = nullptr, int* actions = nullptr);
+                     cudaStream_t s, bool pdl, const int* req_ids = nullptr, int* actions = nullptr, int* actions_copy = nullptr);
 // merge of the split requests' partial outputs for the units [lh0, lh0 + lh_n) (per-layer entry point)
 void gp_launch_select_only(const GpDev& p, const int* req_ids, int n_req, int* actions, float* out, int grid_sel, cudaStream_t s,
                            bool pdl, int serial);

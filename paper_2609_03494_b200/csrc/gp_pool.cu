@@ -52,6 +52,7 @@ struct gp_pool {
   cudaStream_t last_stream;       // stream of the last decode step
   int early_plan;                 // gp_set_early_plan: the plan kernel reads the caller's inputs before its wait
   int first_plain;                // the step's first kernel follows a kernel of another kind: plain launch
+  int32_t* actions_copy;          // host entry points: the caller's (mapped) array the boundary kernel copies the actions to
   cudaEvent_t ev[GP_N_KERNELS + 1];
   float ms[GP_N_KERNELS];
   int64_t launches[GP_N_KERNELS];
@@ -1056,7 +1057,8 @@ int gp_decode_step(gp_pool* pool, const int32_t* dev_req_ids, int32_t n_req, con
       if (prof) cudaEventRecord(pool->ev[1], s);
       gp_launch_attention(d, dev_req_ids, n_req, q, k, v, static_cast<float*>(out), pool->attn_grid_ov, s, pdl, 0, LH, 0);
       if (prof) cudaEventRecord(pool->ev[2], s);
-      gp_launch_chain(d, d, n_req, static_cast<float*>(out), serial, 1, pool->chain_grid_ov, s, pdl, dev_req_ids, dev_actions);
+      gp_launch_chain(d, d, n_req, static_cast<float*>(out), serial, 1, pool->chain_grid_ov, s, pdl, dev_req_ids, dev_actions,
+                      pool->actions_copy);
       if (prof) { cudaEventRecord(pool->ev[3], s); cudaEventRecord(pool->ev[4], s); }    // the last interval stays empty
       pool->launch_count += 3;
     } else {
@@ -1380,9 +1382,15 @@ static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, 
   const int early = pool->early_plan;
   pool->early_plan = 1;
   pool->first_plain = 1;
+  // The actions: the plan kernel writes them all and the decisions overwrite some; written straight to host memory
+  // they made the plan kernel wait for the bus.  With the boundary work in one kernel they stay on the device and
+  // that kernel copies them to the caller's array once they are final (beside its compaction).
+  const bool act_late = direct && !pool->cfg.async_boundary && pool->chain_grid_ov > 0;
+  pool->actions_copy = act_late ? static_cast<int32_t*>(d_act) : nullptr;
   const int st = gp_decode_step(pool, st_ids, n_req, st_q, st_k, st_v,
                                 direct ? d_out : static_cast<void*>(pool->st_out),
-                                direct ? static_cast<int32_t*>(d_act) : pool->st_act, stream);
+                                direct && !act_late ? static_cast<int32_t*>(d_act) : pool->st_act, stream);
+  pool->actions_copy = nullptr;
   pool->early_plan = early;
   pool->first_plain = 0;
   if (st != GP_OK) return st;
