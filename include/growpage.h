@@ -303,15 +303,22 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
                         const void* q, const void* k, const void* v,
                         void* out, int32_t* actions, void* stream);
 
-/* The same step without the synchronisation at the end: everything is enqueued on `stream` and the call returns.
- * The caller's input buffers must stay as they are until the step's first kernel has run, `out` and `actions`
- * hold the results once the work enqueued by this call has completed (an event recorded on `stream` after the
- * call, or a synchronisation), and kernel-reported errors are read with gp_pool_status then.  A serving loop
- * can so issue step t + 1 while it still reads the results of step t from a second pair of output buffers: the
- * GPU never waits for the host's wake-up and launches between steps. */
+/* The same step without the synchronisation at the end: everything is enqueued and the call returns.  With
+ * page-locked buffers the copy engine moves the inputs in on a stream of the pool's own, beside the step before on
+ * `stream` (two staging sets), and the kernels write the results into the caller's buffers as they run: a serving
+ * loop issues step t + 1 while step t runs and reads the results of step t from a second pair of result buffers
+ * meanwhile; the GPU never waits for the host's wake-up and launches between steps.  The caller's input buffers
+ * must stay as they are, and `out` and `actions` are not to be read, until gp_decode_step_host_wait has returned for
+ * the call (calls are waited for in the order they were made; at most two can be outstanding: a third call first
+ * waits for the oldest itself) or `stream` has been synchronised. */
 int gp_decode_step_host_async(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req,
                               const void* q, const void* k, const void* v,
                               void* out, int32_t* actions, void* stream);
+
+/* Waits until the results of the oldest gp_decode_step_host_async call not yet waited for are in the caller's
+ * buffers (a device-wide synchronisation when there is none), then looks at the kernels' error word: GP_OK, or
+ * GP_ERR_CUDA when a kernel reported an internal error (gp_pool_status). */
+int gp_decode_step_host_wait(gp_pool* pool);
 
 /* Ends a request: every page of its table loses one reference and returns to the free list at
  * zero; the summary slot is recycled without clearing (App. D.1).  Asynchronous on `stream`.

@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
     L.gp_decode_step.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.gp_decode_step_host.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.gp_decode_step_host_async.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
+    L.gp_decode_step_host_wait.argtypes = [vp]
     L.gp_decode_step_local.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.gp_shard_sums.argtypes = [vp, C.POINTER(C.c_void_p), C.POINTER(C.c_int64)]
     L.gp_decode_step_finish.argtypes = [vp, vp, i32, vp, vp]
@@ -183,6 +184,10 @@ def gp_step_end(pool: int, dev_req_ids_ptr: int, n_req: int, dev_actions_ptr: in
 
 def gp_step_abort(pool: int) -> None:
     _check(lib().gp_step_abort(C.c_void_p(pool)), "gp_step_abort")
+
+
+def gp_decode_step_host_wait(pool: int) -> None:
+    _check(lib().gp_decode_step_host_wait(C.c_void_p(pool)), "gp_decode_step_host_wait")
 
 
 def gp_decode_step_local(pool: int, dev_req_ids_ptr: int, n_req: int, q_ptr: int, k_ptr: int, v_ptr: int,
@@ -385,10 +390,13 @@ class Pool:
                             v.data_ptr(), out.data_ptr(), actions.data_ptr(), self.stream())
 
     def decode_step_host_async(self, req_ids, q, k, v, out, actions) -> None:
-        """As decode_step_host, without the synchronisation at the end: results are there once the stream has run
-        the work (the caller records an event or synchronises)."""
+        """As decode_step_host, without the synchronisation at the end: results are there once host_wait has returned
+        for the call."""
         gp_decode_step_host_async(self.handle, req_ids.data_ptr(), int(req_ids.numel()), q.data_ptr(), k.data_ptr(),
                                   v.data_ptr(), out.data_ptr(), actions.data_ptr(), self.stream())
+
+    def host_wait(self) -> None:
+        gp_decode_step_host_wait(self.handle)
 
     def release(self, req: int) -> None:
         gp_release(self.handle, req, self.stream())

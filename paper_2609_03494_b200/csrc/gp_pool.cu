@@ -40,9 +40,12 @@ struct gp_pool {
   // The host entry points fetch a step's inputs on a stream of their own into one of two staging sets, so that the
   // fetch of step t + 1 runs beside the kernels of step t when the caller issues steps ahead.
   int* st2_ids; void* st2_q; void* st2_k; void* st2_v;
-  cudaStream_t fetch_stream;
-  cudaEvent_t ev_fetch[2], ev_used[2];              // set fetched; set no longer read by the step that used it
+  cudaStream_t fetch_stream;                        // inputs in, beside the steps on the caller's stream
+  cudaEvent_t ev_fetch[2], ev_used[2], ev_out[2];   // set fetched; its step has run; its results are in the caller's buffers
   long long host_steps;                             // steps issued through the host entry points
+  long long host_waited;                            // gp_decode_step_host_async calls whose results have been waited for
+  long long host_async_issued;                      // ... and issued
+  int host_async_set[2];                            // the staging sets of the (at most two) calls not yet waited for
   __nv_bfloat16* qn; __nv_bfloat16* kn;             // one layer's normalised queries and keys (gp_attn_layer_qknorm)
   // small device words
   int* d_status;
@@ -730,7 +733,7 @@ void pool_free(gp_pool* pool) {
   if (pool->h_err) cudaFreeHost(pool->h_err);
   if (pool->fetch_stream) {
     cudaStreamDestroy(pool->fetch_stream);
-    for (int i = 0; i < 2; ++i) { cudaEventDestroy(pool->ev_fetch[i]); cudaEventDestroy(pool->ev_used[i]); }
+    for (int i = 0; i < 2; ++i) { cudaEventDestroy(pool->ev_fetch[i]); cudaEventDestroy(pool->ev_used[i]); cudaEventDestroy(pool->ev_out[i]); }
   }
   delete pool;
 }
@@ -1299,6 +1302,7 @@ __global__ void gp_fetch_inputs_kernel(int* __restrict__ d_ids, const int* __res
   }
 }
 
+extern "C" int gp_decode_step_host_wait(gp_pool* pool);
 static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
                      const void* v, void* out, int32_t* actions, void* stream, bool wait) {
   if (!pool || n_req < 0 || n_req > pool->cfg.max_requests) return GP_ERR_INVALID;
@@ -1316,6 +1320,7 @@ static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, 
   // waits for its fetch.  The call that waits for its step fetches on the caller's stream (nothing to overlap
   // with).  Pageable memory: four copies on the caller's stream.
   const int set = (int)(pool->host_steps & 1);
+  bool staged_async = false;                 // inputs by the copy engine on the side stream (the call that does not wait)
   int* st_ids = set ? pool->st2_ids : pool->st_ids;
   void* st_q = set ? pool->st2_q : pool->st_q;
   void* st_k = set ? pool->st2_k : pool->st_k;
@@ -1344,7 +1349,9 @@ static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, 
         for (int i = 0; i < 2; ++i) {
           GP_CUDA(cudaEventCreateWithFlags(&pool->ev_fetch[i], cudaEventDisableTiming));
           GP_CUDA(cudaEventCreateWithFlags(&pool->ev_used[i], cudaEventDisableTiming));
+          GP_CUDA(cudaEventCreateWithFlags(&pool->ev_out[i], cudaEventDisableTiming));
           GP_CUDA(cudaEventRecord(pool->ev_used[i], s));
+          GP_CUDA(cudaEventRecord(pool->ev_out[i], s));
         }
       }
       cudaStream_t fs = pool->fetch_stream;
@@ -1359,6 +1366,7 @@ static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, 
       GP_CUDA(cudaMemcpyAsync(st_v, v, kb, cudaMemcpyHostToDevice, fs));
       GP_CUDA(cudaEventRecord(pool->ev_fetch[set], fs));
       GP_CUDA(cudaStreamWaitEvent(s, pool->ev_fetch[set], 0));
+      staged_async = true;
     } else {
       (void)cudaGetLastError();                    // pageable memory: not an error
       GP_CUDA(cudaMemcpyAsync(st_ids, host_req_ids, (size_t)n_req * 4, cudaMemcpyHostToDevice, s));
@@ -1376,6 +1384,16 @@ static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, 
   const bool direct = cudaHostGetDevicePointer(&d_out, out, 0) == cudaSuccess &&
                       cudaHostGetDevicePointer(&d_act, actions, 0) == cudaSuccess;
   if (!direct) (void)cudaGetLastError();           // pageable memory: not an error, the staged path takes over
+  // (Results through a staging set and the copy engine on a third stream, beside the next step, were tried for the
+  // call that does not wait: a megabyte takes the copy engine and the event that reports it 60 us, longer than the
+  // host may lag behind when it reads every step's results before it issues the step after the next: 92 us per
+  // step against 78 with the kernels writing the rows over the bus themselves.)
+  float* st_out = pool->st_out;
+  int* st_act = pool->st_act;
+  if (staged_async && pool->host_async_issued - pool->host_waited >= 2) {          // two calls outstanding: the older first
+    const int st0 = gp_decode_step_host_wait(pool);
+    if (st0 != GP_OK) return st0;
+  }
   // The inputs arrive by the fetch kernel or the copies above, which end before the plan kernel starts: that
   // kernel is launched the plain way here (not as a programmatic dependent of the fetch kernel, whose stores it
   // reads), so planning ahead of its wait, which is then no wait at all, is safe whatever the option says.
@@ -1388,16 +1406,21 @@ static int host_step(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, 
   const bool act_late = direct && !pool->cfg.async_boundary && pool->chain_grid_ov > 0;
   pool->actions_copy = act_late ? static_cast<int32_t*>(d_act) : nullptr;
   const int st = gp_decode_step(pool, st_ids, n_req, st_q, st_k, st_v,
-                                direct ? d_out : static_cast<void*>(pool->st_out),
-                                direct && !act_late ? static_cast<int32_t*>(d_act) : pool->st_act, stream);
+                                direct ? d_out : static_cast<void*>(st_out),
+                                direct && !act_late ? static_cast<int32_t*>(d_act) : st_act, stream);
   pool->actions_copy = nullptr;
   pool->early_plan = early;
   pool->first_plain = 0;
   if (st != GP_OK) return st;
   if (pool->fetch_stream) GP_CUDA(cudaEventRecord(pool->ev_used[set], s));       // the set may be fetched into again
   if (!direct) {
-    GP_CUDA(cudaMemcpyAsync(out, pool->st_out, qb * 2, cudaMemcpyDeviceToHost, s));
-    GP_CUDA(cudaMemcpyAsync(actions, pool->st_act, (size_t)n_req * 4, cudaMemcpyDeviceToHost, s));
+    GP_CUDA(cudaMemcpyAsync(out, st_out, qb * 2, cudaMemcpyDeviceToHost, s));
+    GP_CUDA(cudaMemcpyAsync(actions, st_act, (size_t)n_req * 4, cudaMemcpyDeviceToHost, s));
+  }
+  if (staged_async) {                          // what gp_decode_step_host_wait waits for: this call's work on `stream`
+    GP_CUDA(cudaEventRecord(pool->ev_out[set], s));
+    pool->host_async_set[pool->host_async_issued & 1] = set;
+    pool->host_async_issued += 1;
   }
   if (!wait) return GP_OK;
   GP_CUDA(cudaStreamSynchronize(s));
@@ -1412,6 +1435,18 @@ int gp_decode_step_host(gp_pool* pool, const int32_t* host_req_ids, int32_t n_re
 int gp_decode_step_host_async(gp_pool* pool, const int32_t* host_req_ids, int32_t n_req, const void* q, const void* k,
                               const void* v, void* out, int32_t* actions, void* stream) {
   return host_step(pool, host_req_ids, n_req, q, k, v, out, actions, stream, false);
+}
+
+int gp_decode_step_host_wait(gp_pool* pool) {
+  if (!pool) return GP_ERR_INVALID;
+  GP_CUDA(cudaSetDevice(pool->device));
+  if (pool->host_waited < pool->host_async_issued) {
+    GP_CUDA(cudaEventSynchronize(pool->ev_out[pool->host_async_set[pool->host_waited & 1]]));
+    pool->host_waited += 1;
+  } else {
+    GP_CUDA(cudaDeviceSynchronize());        // nothing of that kind outstanding: whatever else the pool has in flight
+  }
+  return kernel_status(pool);
 }
 
 int gp_pool_status(gp_pool* pool, int32_t* error_bits) {

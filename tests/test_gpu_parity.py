@@ -568,7 +568,8 @@ def test_host_entry_point_with_pageable_buffers_and_without_the_final_wait():
     # gp_decode_step_host fetches pinned inputs with one kernel over the bus (the ids fill whole 16-byte pieces
     # here: four requests) and writes pinned outputs over the bus as it runs; pageable buffers take copies.
     # gp_decode_step_host_async is the same without the synchronisation at the end: the loop below issues step t,
-    # then waits for step t - 1 and reads its results from the other of two pairs of result buffers.
+    # then waits for step t - 1 (gp_decode_step_host_wait) and reads its results from the other of two pairs of
+    # result buffers.
     import torch
     cfg = B.make_config(1, 8, 2, 64, n_pages=32, max_pages_per_req=4, max_requests=8, host_staging=True)
     results = []
@@ -591,17 +592,15 @@ def test_host_entry_point_with_pageable_buffers_and_without_the_final_wait():
                 if mode.endswith("behind"):
                     keep.append((ids, tq, tk, tv))                # the inputs stay as they are until their step has run
                     pool.decode_step_host_async(ids, tq, tk, tv, out, act)
-                    ev = torch.cuda.Event()
-                    ev.record()
                     if pending is not None:
-                        pending[0].synchronize()
+                        pool.host_wait()                          # the call before this one
                         outs.append((pending[1].clone().numpy(), pending[2].clone().numpy()))
-                    pending = (ev, out, act)
+                    pending = (None, out, act)
                 else:
                     pool.decode_step_host(ids, tq, tk, tv, out, act)
                     outs.append((out.clone().numpy(), act.clone().numpy()))
             if pending is not None:
-                pending[0].synchronize()
+                pool.host_wait()
                 outs.append((pending[1].clone().numpy(), pending[2].clone().numpy()))
                 assert B.gp_pool_status(pool.handle) == (B.GP_OK, 0)
             results.append(outs)
