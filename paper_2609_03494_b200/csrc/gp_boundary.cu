@@ -1239,23 +1239,21 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
     }
     __syncthreads();
 
+    // A thread's pieces of a chunk: piece k2 belongs to slot tl0 + k2 * TLS of the chunk, and is the same 16 bytes of
+    // its row every time (K or V, physical piece cp); a page's tile of this unit lies page_stride bytes after the
+    // one of the page before.
+    constexpr int PPS = 2 * CH, TLS = CT / PPS;
+    const int tl0 = tid / PPS, isv = (tid % PPS) / CH, cp = tid % CH;
+    uint8_t* const unit_base = reinterpret_cast<uint8_t*>(p.kv + gp_tile_off(p, l, 0, h)) + isv * GP_PAGE * ROW_BYTES;
+    const size_t page_stride = (size_t)p.Hkv * 2 * GP_PAGE * ROW_BYTES;
     uint4 val[PIECES];
-    int dst_code[PIECES];
 #pragma unroll
     for (int k2 = 0; k2 < PIECES; ++k2) {
-      const int piece = tid + k2 * CT;
-      const int tl = piece / (2 * CH), pc = piece % (2 * CH);
-      const int i = c0 + tl;
-      const int ds = s_dst[tl];
-      dst_code[k2] = -1;
+      const int tl = tl0 + k2 * TLS;
       val[k2] = make_uint4(0, 0, 0, 0);
-      if (ds >= 0) {
-        const int isv = pc / CH, cp = pc % CH;
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(p.kv + gp_tile_off(p, l, s_spage[tl], h)) +
-                             isv * GP_PAGE * ROW_BYTES + (i % GP_PAGE) * ROW_BYTES + (cp << 4);
-        val[k2] = *reinterpret_cast<const uint4*>(src);
-        dst_code[k2] = (tl << 5) | ((cp ^ (i & 7)) << 1) | isv;   // slot of the chunk, logical 16-byte piece, K or V
-      }
+      if (s_dst[tl] >= 0)
+        val[k2] = *reinterpret_cast<const uint4*>(unit_base + (size_t)s_spage[tl] * page_stride +
+                                                  ((c0 + tl) % GP_PAGE) * ROW_BYTES + (cp << 4));
     }
     // Touch every loaded value so that the loads have completed before the flag below is published: the
     // next chunk's CTA may overwrite the tail of this chunk's sources as soon as it sees the flag.
@@ -1283,12 +1281,12 @@ __device__ __forceinline__ void compact_body(const GpDev& p, const CmpSmem& C, i
     __syncthreads();
 #pragma unroll
     for (int k2 = 0; k2 < PIECES; ++k2) {
-      if (dst_code[k2] >= 0) {
-        const int tl = dst_code[k2] >> 5, c = (dst_code[k2] >> 1) & 15, isv = dst_code[k2] & 1;
-        const int ds = s_dst[tl];
-        uint8_t* dst = reinterpret_cast<uint8_t*>(p.kv + gp_tile_off(p, l, s_dpage[tl], h)) + isv * GP_PAGE * ROW_BYTES +
-                       (ds % GP_PAGE) * ROW_BYTES + ((c ^ (ds & 7)) << 4);
-        *reinterpret_cast<uint4*>(dst) = val[k2];
+      const int tl = tl0 + k2 * TLS;
+      const int ds = s_dst[tl];
+      if (ds >= 0) {
+        const int c = cp ^ ((c0 + tl) & 7);                 // the logical piece this thread holds (rows are swizzled by slot)
+        *reinterpret_cast<uint4*>(unit_base + (size_t)s_dpage[tl] * page_stride + (ds % GP_PAGE) * ROW_BYTES +
+                                  ((c ^ (ds & 7)) << 4)) = val[k2];
       }
     }
     if (tok_dst >= 0) {
